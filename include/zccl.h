@@ -1,0 +1,189 @@
+/*
+ * zccl.h -- C boundary of the B200 (sm_100a) implementation of ZCCL's data-parallel hot path:
+ * the fZ-light error-bounded lossy codec, the fused decompress-reduce-recompress hop of the ring
+ * reduce-scatter, and N-rank ring collectives emulated on N buffers in one GPU's memory.
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise
+ *   - Pointers marked [device] are device pointers owned by the caller; [host] are host pointers.  The library
+ *     owns only what zccl_ctx_create allocates and never allocates, frees or synchronises on the hot path.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only enqueue work;
+ *     they return before it has run.  Operations that share one context must be ordered on one stream (the
+ *     context's scan workspace is shared); use one context per concurrently used stream.
+ *   - Return value: ZCCL_OK, or a negative ZCCL_E_* for what the host can see at once (bad arguments, capacity
+ *     below the fixed part of a stream, CUDA launch failure).  What only the device can see (capacity overrun,
+ *     values out of range, malformed stream, degenerate range, scan time-out, precision warning) is recorded in
+ *     a device status word that zccl_status() reads and clears.  No kernel ever writes outside the capacities it
+ *     was given; after a device-side error the contents of the output are unspecified.
+ *   - fp32 data only.  Arithmetic is IEEE binary32, round to nearest even, no fused multiply-add, so that
+ *     streams and reconstructions are reproducible bit for bit.
+ *
+ * Stream layout (little endian; the paper, Section 3.3 and Section 3.5.2, fixes the ingredients: per-unit 4-byte
+ * outlier, per-block sign bits and one-byte code length, fixed-length bits, constant blocks stored as the code
+ * length alone, 4-byte per-chunk sizes gathered at the front of the buffer.  Their order and the header are this
+ * library's choice):
+ *   header 32 B : u32 magic "ZCL1"; u32 0x05000001; u64 n; f32 eb_abs; f32 s (step); u32 T = 4096; u32 nT
+ *   index 4*nT B: u32 per tile, inclusive prefix sum of tile blob sizes in 4-byte words
+ *   blobs       : per tile [i32 quantised first value][code-length byte per 32-element block, padded to 4 B]
+ *                 [per block with code length L > 0: u32 sign word, then L bit-plane words of |delta|]
+ */
+#ifndef ZCCL_H
+#define ZCCL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct zccl_ctx zccl_ctx;
+
+/* How `eb` is read.  The paper's tables quote value-range-relative bounds ("REL", Tables 1-4). */
+enum { ZCCL_EB_ABS = 0,    /* eb is the absolute bound eb_abs */
+       ZCCL_EB_REL = 1 };  /* eb_abs = eb * (max - min) of the input (of all ranks' inputs in zccl_sim_*) */
+
+enum { ZCCL_OK = 0,
+       ZCCL_E_ARG = -1,         /* NULL pointer, size beyond the context's limits, eb not positive and finite */
+       ZCCL_E_CUDA = -2,        /* a CUDA runtime call failed */
+       ZCCL_E_CAPACITY = -3,    /* an output buffer is too small */
+       ZCCL_E_RANGE = -4,       /* some |x / s| >= 2^30: codes do not fit 32-bit deltas */
+       ZCCL_E_BAD_STREAM = -5,  /* magic, version, sizes or index of a compressed stream are inconsistent */
+       ZCCL_E_TIMEOUT = -6,     /* a bounded device-side wait in the placement scan expired */
+       ZCCL_E_DEGENERATE = -7,  /* REL bound on an input whose range is zero (use ZCCL_EB_ABS) */
+       ZCCL_W_PRECISION = 1 };  /* some |code| > 2^15: fp32 rounding may exceed eb_abs by about |x| * 1.8e-7 */
+
+/* Flags of the reduce hop and of zccl_sim_allreduce. */
+enum { ZCCL_CONSISTENT_OWNER = 1u };  /* owner's copy of a reduced chunk = dequantised value, not the raw sum */
+
+enum { ZCCL_TILE = 4096, ZCCL_BLOCK = 32, ZCCL_HEADER_BYTES = 32, ZCCL_MAX_RANKS = 64 };
+
+/*
+ * Context: look-back scan workspace for streams of up to `max_elems` elements, the device status word, the
+ * resolved-bound block and, when max_ranks >= 2, an arena of compressed-chunk slots for zccl_sim_* sized for
+ * max_ranks ranks exchanging max_elems elements in total per rank buffer (about (max_ranks + 2) *
+ * zccl_compress_bound(max_elems) bytes).  Allocates on the current device; the only allocating call.
+ * Returns ZCCL_E_ARG for max_elems == 0 or max_ranks outside [0, ZCCL_MAX_RANKS], ZCCL_E_CUDA if allocation fails.
+ */
+int zccl_ctx_create(zccl_ctx** ctx /*[host] out*/, size_t max_elems, int max_ranks);
+
+/* Frees everything the context owns (synchronises the device first).  NULL is allowed. */
+void zccl_ctx_destroy(zccl_ctx* ctx);
+
+/* Worst-case stream size in bytes for n elements (every block at code length 31).  Pure host function. */
+size_t zccl_compress_bound(size_t n);
+
+/*
+ * Synchronises `stream`, returns the most severe condition recorded on the device since the last call
+ * (errors before the warning, ZCCL_OK if none) and clears the record.
+ */
+int zccl_status(zccl_ctx* ctx, void* stream);
+
+/* Static description of a status code. */
+const char* zccl_strerror(int code);
+
+/*
+ * fZ-light compression (Section 3.3; stream with the chunk-size index of Section 3.5.2).
+ * Per 4096-element tile: q_i = rint(x_i * r), r = 1/s, s = 2 * (eb_abs * (1 - 2^-6)); 1-D Lorenzo deltas with the
+ * tile's first code kept as a 4-byte outlier; per 32-element block the code length L = bit length of the largest
+ * |delta| and, if L > 0, sign bits and L bit planes; tiles placed by a device-wide prefix scan of their sizes.
+ *   x [device]          n floats (finite values); may be NULL only if n == 0
+ *   out [device]        receives the stream; 4-byte aligned; out_capacity bytes writable
+ *   out_bytes [device]  one size_t, receives the stream length in bytes (readable after the stream has run)
+ * Host-side errors: ZCCL_E_ARG (NULLs, n > max_elems, eb <= 0 or not finite, bad mode),
+ * ZCCL_E_CAPACITY (out_capacity < 32 + 4 * ceil(n / 4096)).  Device-side: CAPACITY (a tile would pass
+ * out_capacity; nothing is written beyond it), RANGE, DEGENERATE (REL with max == min), W_PRECISION.
+ */
+int zccl_compress(zccl_ctx* ctx, const float* x, size_t n, int eb_mode, float eb,
+                  void* out, size_t out_capacity, size_t* out_bytes, void* stream);
+
+/*
+ * fZ-light decompression (Section 3.3, Section 3.5.2): tile starts come from the index at the front; per block the
+ * magnitudes are rebuilt from the bit planes, signs applied, the Lorenzo recurrence undone by a running integer
+ * sum from the tile's outlier, and x'_i = float(q_i) * s.
+ *   in [device]   the stream; at most in_bytes_max bytes are read; 4-byte aligned
+ *   y [device]    receives n floats, n taken from the stream's header; y_capacity_elems must be >= n
+ * Host-side errors: ZCCL_E_ARG, ZCCL_E_CAPACITY (in_bytes_max < 32).  Device-side: BAD_STREAM (nothing outside
+ * in_bytes_max is read, inconsistent tiles are skipped), CAPACITY (n > y_capacity_elems: nothing is written).
+ */
+int zccl_decompress(zccl_ctx* ctx, const void* in, size_t in_bytes_max,
+                    float* y, size_t y_capacity_elems, void* stream);
+
+/*
+ * One reduce-scatter hop of the collective computation framework (Section 3.1.2; error chain of Eq. 2):
+ * out_c = compress( decompress(in_c) + local ), in one kernel, with no uncompressed intermediate in memory.
+ * y_i = fl32( fl32(float(q_i) * s) + local_i ), the decoded operand on the left; bound and step are in_c's.
+ *   in_c [device]      received compressed chunk (at most in_bytes_max bytes are read)
+ *   local [device]     this rank's uncompressed chunk, n floats (the paper's form), or NULL
+ *   local_c [device]   instead of `local`: a second compressed chunk of the same n and step (at most
+ *                      local_c_bytes_max bytes are read).  Exactly one of local / local_c is non-NULL.
+ *   n                  element count; must equal the count in in_c's header (else BAD_STREAM on the device)
+ *   out_c, out_capacity, out_bytes [device]  as in zccl_compress
+ *   raw_out [device]   NULL, or n floats receiving y (with ZCCL_CONSISTENT_OWNER in flags: float(q(y)) * s)
+ * Errors as for zccl_compress and zccl_decompress.
+ */
+int zccl_decompress_reduce_compress(zccl_ctx* ctx, const void* in_c, size_t in_bytes_max,
+                                    const float* local, const void* local_c, size_t local_c_bytes_max, size_t n,
+                                    void* out_c, size_t out_capacity, size_t* out_bytes,
+                                    float* raw_out, unsigned flags, void* stream);
+
+/*
+ * Ring Allreduce (sum) over nranks rank buffers in this GPU's memory (Section 3.5: ring reduce-scatter in the
+ * collective computation framework, then ring allgather in the data movement framework).
+ * Chunk c = elements [c*m, (c+1)*m) of every buffer, m = ceil(n_per_rank / nranks).  Rank r compresses chunk r;
+ * on hop k = 0..nranks-2 rank r takes rank r-1's stream of chunk (r-k-1) mod nranks, and runs the fused hop with
+ * its own uncompressed chunk; the last hop also leaves the reduced chunk (r+1) mod nranks uncompressed at its
+ * owner r.  Then nranks-1 forwarding hops copy compressed chunks between per-rank slots and every rank
+ * decompresses the nranks-1 chunks it does not own.  One bound for the whole collective; with ZCCL_EB_REL it is
+ * eb times the range over all ranks' inputs.
+ *   send [host]  nranks device pointers, each n_per_rank floats (read only)
+ *   recv [host]  nranks device pointers, each n_per_rank floats (must not overlap send)
+ * Needs a context created with max_ranks >= nranks and max_elems >= n_per_rank.
+ */
+int zccl_sim_allreduce(zccl_ctx* ctx, const float* const* send, float* const* recv, int nranks,
+                       size_t n_per_rank, int eb_mode, float eb, unsigned flags, void* stream);
+
+/*
+ * Ring Allgather in the data movement framework (Section 3.1.1, Section 3.5.1): each rank compresses its
+ * n_per_rank elements once, compressed bytes are forwarded nranks-1 times, each rank decompresses the nranks-1
+ * foreign contributions and copies its own uncompressed.
+ *   send [host]  nranks device pointers, each n_per_rank floats
+ *   recv [host]  nranks device pointers, each nranks * n_per_rank floats
+ * Needs a context with max_ranks >= nranks and max_elems >= nranks * n_per_rank.
+ */
+int zccl_sim_allgather(zccl_ctx* ctx, const float* const* send, float* const* recv, int nranks,
+                       size_t n_per_rank, int eb_mode, float eb, void* stream);
+
+/*
+ * Broadcast in the data movement framework (Section 3.1.1): the root compresses once; each of the nsinks
+ * receivers gets a copy of the compressed bytes and decompresses it once.
+ *   root [device] n floats;  recv [host] nsinks device pointers, each n floats
+ * Needs a context with max_ranks >= nsinks and max_elems >= n.
+ */
+int zccl_sim_bcast(zccl_ctx* ctx, const float* root, float* const* recv, int nsinks, size_t n,
+                   int eb_mode, float eb, void* stream);
+
+/*
+ * Compressed sizes of the last zccl_sim_* call, for reporting ratios (the paper's compressed_sizes array,
+ * Section 3.5.1).  Synchronises `stream`.  sizes [host] receives up to `capacity` entries and the call returns how
+ * many there are: allreduce nranks*nranks (entry k*nranks + r = bytes rank r produced at step k, k = 0 the
+ * initial compression), allgather nranks, bcast 1.  Negative on error.
+ */
+int zccl_sim_sizes(zccl_ctx* ctx, size_t* sizes, int capacity, void* stream);
+
+/*
+ * Host-buffer convenience forms: copy the input from host memory into a staging area of the context, run the
+ * device path, copy the result back, all enqueued on `stream` (pinned host memory makes the copies asynchronous).
+ * They exist so that end-to-end cost including PCIe transfers can be measured through this boundary.
+ *   zccl_compress_host:   x_host n floats -> out_host (out_capacity bytes), *out_bytes_host after the stream ran
+ *   zccl_decompress_host: in_host in_bytes bytes -> y_host (y_capacity_elems floats)
+ * Need max_elems >= n.  Errors as for the device forms.
+ */
+int zccl_compress_host(zccl_ctx* ctx, const float* x_host, size_t n, int eb_mode, float eb,
+                       void* out_host, size_t out_capacity, size_t* out_bytes_host, void* stream);
+int zccl_decompress_host(zccl_ctx* ctx, const void* in_host, size_t in_bytes,
+                         float* y_host, size_t y_capacity_elems, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZCCL_H */

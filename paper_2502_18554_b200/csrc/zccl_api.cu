@@ -1,0 +1,536 @@
+// C boundary: argument checks, context, job construction and launch order.  Every step of the path itself runs
+// in the kernels; nothing here touches data.
+#include "../../include/zccl.h"
+#include "zccl_internal.h"
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace zccl;
+
+struct zccl_ctx {
+    int device = 0;
+    int sm_count = 0;
+    size_t max_elems = 0;
+    int max_ranks = 0;
+    Workspace ws{};
+    void* small_block = nullptr;     // tile states + counters + params + sizes
+    uint8_t* arena = nullptr;        // compressed-chunk slots of the emulated ranks
+    size_t arena_bytes = 0;
+    size_t* sim_sizes = nullptr;     // device: sizes of the last zccl_sim_* call
+    int sim_sizes_count = 0;
+    int sim_sizes_cap = 0;
+    float* stage_x = nullptr;        // device staging of the host-buffer forms
+    uint8_t* stage_c = nullptr;
+    size_t stage_c_cap = 0;
+    size_t* stage_bytes = nullptr;   // device size_t
+};
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline size_t tiles_of(size_t n) { return (n + kTile - 1) / kTile; }
+
+size_t bound_of(size_t n)
+{
+    const size_t nT = tiles_of(n);
+    size_t total = kHeaderBytes + 4 * nT;
+    if (nT == 0) return total;
+    const size_t full = nT - 1;
+    total += full * (4 + kBlocksPerTile + (size_t)kBlocksPerTile * 128);
+    const size_t len = n - full * kTile;
+    const size_t nb = (len + kBlock - 1) / kBlock;
+    total += 4 + ((nb + 3) & ~(size_t)3) + nb * 128;
+    return total;
+}
+
+// eb -> (eb_abs, s, r) for an absolute bound, with the same IEEE operations the device uses for relative bounds.
+int resolve_abs_host(float eb, Params& p)
+{
+    volatile float ebq = eb * 0.984375f;
+    volatile float s = ebq * 2.0f;
+    if (!(s > 0.0f) || !std::isfinite((float)s)) return ZCCL_E_DEGENERATE;
+    volatile float r = 1.0f / s;
+    if (!std::isfinite((float)r)) return ZCCL_E_DEGENERATE;
+    p.eb_abs = eb; p.s = s; p.r = r; p.valid = 1;
+    return ZCCL_OK;
+}
+
+inline bool eb_ok(int mode, float eb)
+{
+    return (mode == ZCCL_EB_ABS || mode == ZCCL_EB_REL) && eb > 0.0f && std::isfinite(eb);
+}
+
+inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? ZCCL_OK : ZCCL_E_CUDA; }
+
+// Collects jobs and launches them in batches of at most kMaxJobs.
+struct Batcher {
+    JobBatch jb{};
+    void reset() { jb.count = 0; jb.total_tiles = 0; }
+    Batcher() { reset(); }
+    bool full() const { return jb.count == kMaxJobs; }
+    void add(const Job& j, size_t tiles)
+    {
+        Job& d = jb.job[jb.count++];
+        d = j;
+        d.tile_begin = jb.total_tiles;
+        jb.total_tiles += (uint32_t)(tiles ? tiles : 1);
+    }
+};
+
+struct RangeList {
+    std::vector<const float*> x;
+    std::vector<size_t> n;
+};
+
+// Resolves the bound: ABS on the host, REL by a device min/max pass over all listed buffers.
+int resolve_bound(zccl_ctx* c, const RangeList& rl, int mode, float eb, Params& hp, bool& on_device, cudaStream_t st)
+{
+    on_device = false;
+    if (mode == ZCCL_EB_ABS) return resolve_abs_host(eb, hp);
+    size_t total = 0;
+    for (size_t v : rl.n) total += v;
+    if (total == 0) return ZCCL_E_DEGENERATE;
+    RangeBatch rb{};
+    rb.count = 0;
+    for (size_t i = 0; i < rl.x.size(); ++i) {
+        if (rl.n[i] == 0) continue;
+        rb.x[rb.count] = rl.x[i];
+        rb.n[rb.count] = rl.n[i];
+        if (++rb.count == kMaxJobs) {
+            if (launch_range(rb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
+            rb.count = 0;
+        }
+    }
+    if (rb.count && launch_range(rb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
+    if (launch_resolve(mode, eb, c->ws, st) != cudaSuccess) return ZCCL_E_CUDA;
+    hp = Params{0.f, 1.f, 1.f, 1};
+    on_device = true;
+    return ZCCL_OK;
+}
+
+int flush_encode(zccl_ctx* c, Batcher& b, EncodeMode mode, bool dev_params, const Params& hp, cudaStream_t st)
+{
+    if (b.jb.count == 0) return ZCCL_OK;
+    if (b.jb.total_tiles > c->ws.max_tiles) return ZCCL_E_ARG;
+    cudaError_t e = launch_encode(b.jb, mode, c->ws, dev_params, hp, c->sm_count, st);
+    b.reset();
+    return cuda_rc(e);
+}
+int flush_decode(zccl_ctx* c, Batcher& b, cudaStream_t st)
+{
+    if (b.jb.count == 0) return ZCCL_OK;
+    cudaError_t e = launch_decode(b.jb, c->ws, c->sm_count, st);
+    b.reset();
+    return cuda_rc(e);
+}
+struct CopyBatcher {
+    CopyBatch cb{};
+    CopyBatcher() { cb.count = 0; }
+    void add(const void* src, void* dst, const size_t* bytes, size_t* bytes_out, size_t cap)
+    {
+        CopyJob& j = cb.job[cb.count++];
+        j.src = (const uint32_t*)src; j.dst = (uint32_t*)dst; j.bytes = bytes; j.bytes_out = bytes_out; j.cap = cap;
+    }
+    bool full() const { return cb.count == kMaxJobs; }
+};
+int flush_copy(zccl_ctx* c, CopyBatcher& b, cudaStream_t st)
+{
+    if (b.cb.count == 0) return ZCCL_OK;
+    cudaError_t e = launch_copy(b.cb, c->ws, c->sm_count, st);
+    b.cb.count = 0;
+    return cuda_rc(e);
+}
+
+inline void chunk_span(size_t n, int N, int c, size_t& off, size_t& len)
+{
+    const size_t m = (n + (size_t)N - 1) / (size_t)N;
+    size_t o = (size_t)c * m;
+    if (o > n) o = n;
+    off = o;
+    len = (n - o < m) ? n - o : m;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t zccl_compress_bound(size_t n) { return bound_of(n); }
+
+const char* zccl_strerror(int code)
+{
+    switch (code) {
+        case ZCCL_OK: return "ok";
+        case ZCCL_E_ARG: return "invalid argument";
+        case ZCCL_E_CUDA: return "CUDA runtime error";
+        case ZCCL_E_CAPACITY: return "output capacity too small";
+        case ZCCL_E_RANGE: return "value out of quantisable range";
+        case ZCCL_E_BAD_STREAM: return "malformed compressed stream";
+        case ZCCL_E_TIMEOUT: return "placement scan timed out";
+        case ZCCL_E_DEGENERATE: return "degenerate value range or step";
+        case ZCCL_W_PRECISION: return "warning: codes beyond 2^15, bound may be exceeded by fp32 rounding";
+        default: return "unknown status";
+    }
+}
+
+int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
+{
+    if (!out || max_elems == 0 || max_ranks < 0 || max_ranks > ZCCL_MAX_RANKS) return ZCCL_E_ARG;
+    zccl_ctx* c = new (std::nothrow) zccl_ctx();
+    if (!c) return ZCCL_E_ARG;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return ZCCL_E_CUDA; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) { delete c; return ZCCL_E_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    c->max_elems = max_elems;
+    c->max_ranks = max_ranks;
+
+    const size_t max_tiles = tiles_of(max_elems) + (size_t)(max_ranks > kMaxJobs ? max_ranks : kMaxJobs) + 64;
+    if (max_tiles > 0xFFFFFFFFull) { delete c; return ZCCL_E_ARG; }
+    c->sim_sizes_cap = 2 * (max_ranks > 1 ? max_ranks * max_ranks : 1) + 2;
+    const size_t off_state = 0;
+    const size_t off_small = align_up(off_state + 8 * max_tiles, 256);
+    const size_t off_sizes = off_small + 256;
+    const size_t small_bytes = off_sizes + sizeof(size_t) * (size_t)(c->sim_sizes_cap + 1);
+    bool ok = cudaMalloc(&c->small_block, small_bytes) == cudaSuccess;
+    if (ok) ok = cudaMemset(c->small_block, 0, small_bytes) == cudaSuccess;
+    if (ok) {
+        uint8_t* b = (uint8_t*)c->small_block;
+        c->ws.tile_state = (unsigned long long*)(b + off_state);
+        uint32_t* sm = (uint32_t*)(b + off_small);
+        c->ws.ticket = sm + 0;
+        c->ws.done = sm + 1;
+        c->ws.epoch = sm + 2;
+        c->ws.status = sm + 3;
+        c->ws.params = (Params*)(sm + 4);
+        c->ws.minmax = sm + 8;
+        c->ws.max_tiles = (uint32_t)max_tiles;
+        c->sim_sizes = (size_t*)(b + off_sizes);
+        c->stage_bytes = c->sim_sizes + c->sim_sizes_cap;
+        const uint32_t init[3] = {1u, 0xFFFFFFFFu, 0u};   // epoch, min key, max key
+        ok = cudaMemcpy(c->ws.epoch, &init[0], 4, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->ws.minmax, &init[1], 8, cudaMemcpyHostToDevice) == cudaSuccess;
+    }
+    if (ok && max_ranks >= 2) {
+        c->arena_bytes = (size_t)(max_ranks + 2) * align_up(bound_of(max_elems) + (size_t)max_ranks * 1024, 256);
+        ok = cudaMalloc((void**)&c->arena, c->arena_bytes) == cudaSuccess;
+    }
+    if (ok) {
+        c->stage_c_cap = align_up(bound_of(max_elems), 256);
+        ok = cudaMalloc((void**)&c->stage_x, sizeof(float) * max_elems) == cudaSuccess &&
+             cudaMalloc((void**)&c->stage_c, c->stage_c_cap) == cudaSuccess;
+    }
+    if (!ok) { zccl_ctx_destroy(c); return ZCCL_E_CUDA; }
+    *out = c;
+    return ZCCL_OK;
+}
+
+void zccl_ctx_destroy(zccl_ctx* c)
+{
+    if (!c) return;
+    cudaDeviceSynchronize();
+    if (c->small_block) cudaFree(c->small_block);
+    if (c->arena) cudaFree(c->arena);
+    if (c->stage_x) cudaFree(c->stage_x);
+    if (c->stage_c) cudaFree(c->stage_c);
+    delete c;
+}
+
+int zccl_status(zccl_ctx* c, void* stream)
+{
+    if (!c) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint32_t bits = 0;
+    if (cudaMemcpyAsync(&bits, c->ws.status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZCCL_E_CUDA;
+    if (cudaMemsetAsync(c->ws.status, 0, 4, st) != cudaSuccess) return ZCCL_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZCCL_E_CUDA;
+    if (bits & kStTimeout) return ZCCL_E_TIMEOUT;
+    if (bits & kStBadStream) return ZCCL_E_BAD_STREAM;
+    if (bits & kStDegenerate) return ZCCL_E_DEGENERATE;
+    if (bits & kStRange) return ZCCL_E_RANGE;
+    if (bits & kStCapacity) return ZCCL_E_CAPACITY;
+    if (bits & kStPrecision) return ZCCL_W_PRECISION;
+    return ZCCL_OK;
+}
+
+int zccl_compress(zccl_ctx* c, const float* x, size_t n, int eb_mode, float eb,
+                  void* out, size_t out_capacity, size_t* out_bytes, void* stream)
+{
+    if (!c || !out || !out_bytes || (!x && n) || !eb_ok(eb_mode, eb) || n > c->max_elems) return ZCCL_E_ARG;
+    if (((uintptr_t)out & 3u) || ((uintptr_t)x & 3u)) return ZCCL_E_ARG;
+    if (out_capacity < kHeaderBytes + 4 * tiles_of(n)) return ZCCL_E_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    Params hp{};
+    bool dev = false;
+    RangeList rl;
+    rl.x.push_back(x); rl.n.push_back(n);
+    int rc = resolve_bound(c, rl, eb_mode, eb, hp, dev, st);
+    if (rc != ZCCL_OK) return rc;
+    Batcher b;
+    Job j{};
+    j.x = x; j.out = (uint32_t*)out; j.out_bytes = out_bytes; j.n = n; j.out_cap = out_capacity;
+    b.add(j, tiles_of(n));
+    return flush_encode(c, b, kEncodeRaw, dev, hp, st);
+}
+
+int zccl_decompress(zccl_ctx* c, const void* in, size_t in_bytes_max, float* y, size_t y_capacity_elems, void* stream)
+{
+    if (!c || !in || (!y && y_capacity_elems)) return ZCCL_E_ARG;
+    if (((uintptr_t)in & 3u) || ((uintptr_t)y & 3u)) return ZCCL_E_ARG;
+    if (in_bytes_max < (size_t)kHeaderBytes) return ZCCL_E_CAPACITY;
+    if (tiles_of(y_capacity_elems) >= 0xFFFFFFFFull) return ZCCL_E_ARG;
+    Batcher b;
+    Job j{};
+    j.in_c = (const uint32_t*)in; j.in_cap = in_bytes_max; j.y = y; j.n = y_capacity_elems;
+    b.add(j, tiles_of(y_capacity_elems));
+    return flush_decode(c, b, (cudaStream_t)stream);
+}
+
+int zccl_decompress_reduce_compress(zccl_ctx* c, const void* in_c, size_t in_bytes_max,
+                                    const float* local, const void* local_c, size_t local_c_bytes_max, size_t n,
+                                    void* out_c, size_t out_capacity, size_t* out_bytes,
+                                    float* raw_out, unsigned flags, void* stream)
+{
+    if (!c || !in_c || !out_c || !out_bytes || n > c->max_elems) return ZCCL_E_ARG;
+    if ((local == nullptr) == (local_c == nullptr)) return ZCCL_E_ARG;
+    if (((uintptr_t)in_c & 3u) || ((uintptr_t)local & 3u) || ((uintptr_t)local_c & 3u) || ((uintptr_t)out_c & 3u) ||
+        ((uintptr_t)raw_out & 3u)) return ZCCL_E_ARG;
+    if (in_bytes_max < (size_t)kHeaderBytes || (local_c && local_c_bytes_max < (size_t)kHeaderBytes)) return ZCCL_E_CAPACITY;
+    if (out_capacity < kHeaderBytes + 4 * tiles_of(n)) return ZCCL_E_CAPACITY;
+    Batcher b;
+    Job j{};
+    j.x = local; j.in_c = (const uint32_t*)in_c; j.in_c2 = (const uint32_t*)local_c;
+    j.in_cap = in_bytes_max; j.in2_cap = local_c_bytes_max;
+    j.out = (uint32_t*)out_c; j.out_cap = out_capacity; j.out_bytes = out_bytes; j.y = raw_out; j.n = n; j.flags = flags;
+    b.add(j, tiles_of(n));
+    return flush_encode(c, b, kEncodeFused, false, Params{0.f, 1.f, 1.f, 1}, (cudaStream_t)stream);
+}
+
+int zccl_sim_allreduce(zccl_ctx* c, const float* const* send, float* const* recv, int N,
+                       size_t n, int eb_mode, float eb, unsigned flags, void* stream)
+{
+    if (!c || !send || !recv || N < 1 || N > c->max_ranks || !eb_ok(eb_mode, eb) || n > c->max_elems) return ZCCL_E_ARG;
+    for (int r = 0; r < N; ++r) if (!send[r] || !recv[r]) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t m = (n + (size_t)N - 1) / (size_t)N;
+    const size_t slot = align_up(bound_of(m), 256);
+    const size_t need = ((size_t)N * N + 2 * (size_t)N) * slot;
+    if (need > c->arena_bytes) return ZCCL_E_ARG;
+    uint8_t* cur0 = c->arena;
+    uint8_t* nxt0 = c->arena + (size_t)N * slot;
+    uint8_t* gs0 = c->arena + 2 * (size_t)N * slot;
+    auto gslot = [&](int r, int ch) { return gs0 + ((size_t)r * N + ch) * slot; };
+    size_t* hop_sz = c->sim_sizes;                       // [N][N]: step k, rank r
+    size_t* g_sz = c->sim_sizes + (size_t)N * N;         // [N][N]: rank r, chunk ch
+    c->sim_sizes_count = N * N;
+    if (cudaMemsetAsync(c->sim_sizes, 0, sizeof(size_t) * 2 * (size_t)N * N, st) != cudaSuccess) return ZCCL_E_CUDA;
+
+    Params hp{};
+    bool dev = false;
+    RangeList rl;
+    for (int r = 0; r < N; ++r) { rl.x.push_back(send[r]); rl.n.push_back(n); }
+    int rc = resolve_bound(c, rl, eb_mode, eb, hp, dev, st);
+    if (rc != ZCCL_OK) return rc;
+
+    // step 0: rank r compresses its chunk r
+    Batcher b;
+    for (int r = 0; r < N; ++r) {
+        size_t off, len; chunk_span(n, N, r, off, len);
+        Job j{};
+        j.x = send[r] + off; j.n = len; j.out = (uint32_t*)(cur0 + (size_t)r * slot); j.out_cap = slot;
+        j.out_bytes = hop_sz + r;
+        b.add(j, tiles_of(len));
+        if (b.full() && (rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+    }
+    if ((rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+    if (N == 1) return cuda_rc(cudaMemcpyAsync(recv[0], send[0], sizeof(float) * n, cudaMemcpyDeviceToDevice, st));
+
+    // reduce-scatter hops: fused decode + add own chunk + re-encode
+    uint8_t* cur = cur0;
+    uint8_t* nxt = nxt0;
+    for (int k = 0; k + 1 < N; ++k) {
+        const bool last = (k == N - 2);
+        for (int r = 0; r < N; ++r) {
+            const int from = (r - 1 + N) % N;
+            const int ch = ((r - k - 1) % N + N) % N;
+            size_t off, len; chunk_span(n, N, ch, off, len);
+            Job j{};
+            j.in_c = (const uint32_t*)(cur + (size_t)from * slot); j.in_cap = slot;
+            j.x = send[r] + off; j.n = len;
+            j.out = (uint32_t*)(nxt + (size_t)r * slot); j.out_cap = slot;
+            j.out_bytes = hop_sz + (size_t)(k + 1) * N + r;
+            j.y = last ? recv[r] + off : nullptr;
+            j.flags = flags;
+            b.add(j, tiles_of(len));
+            if (b.full() && (rc = flush_encode(c, b, kEncodeFused, false, hp, st)) != ZCCL_OK) return rc;
+        }
+        if ((rc = flush_encode(c, b, kEncodeFused, false, hp, st)) != ZCCL_OK) return rc;
+        uint8_t* t = cur; cur = nxt; nxt = t;
+    }
+
+    // allgather stage: N-1 forwarding hops of compressed chunks between per-rank slots
+    const size_t* own_sz = hop_sz + (size_t)(N - 1) * N;   // rank r owns chunk (r+1) mod N in cur[r]
+    CopyBatcher cb;
+    for (int h = 0; h + 1 < N; ++h) {
+        for (int r = 0; r < N; ++r) {
+            const int from = (r - 1 + N) % N;
+            const int ch = ((r - h) % N + N) % N;
+            const uint8_t* src = h == 0 ? cur + (size_t)from * slot : gslot(from, ch);
+            const size_t* sz = h == 0 ? own_sz + from : g_sz + (size_t)from * N + ch;
+            cb.add(src, gslot(r, ch), sz, g_sz + (size_t)r * N + ch, slot);
+            if (cb.full() && (rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+        }
+        if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+    }
+    // every rank decompresses the chunks it does not own
+    for (int r = 0; r < N; ++r) {
+        for (int ch = 0; ch < N; ++ch) {
+            if (ch == (r + 1) % N) continue;
+            size_t off, len; chunk_span(n, N, ch, off, len);
+            Job j{};
+            j.in_c = (const uint32_t*)gslot(r, ch); j.in_cap = slot; j.y = recv[r] + off; j.n = len;
+            b.add(j, tiles_of(len));
+            if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+        }
+    }
+    return flush_decode(c, b, st);
+}
+
+int zccl_sim_allgather(zccl_ctx* c, const float* const* send, float* const* recv, int N,
+                       size_t n, int eb_mode, float eb, void* stream)
+{
+    if (!c || !send || !recv || N < 1 || N > c->max_ranks || !eb_ok(eb_mode, eb) || n * (size_t)N > c->max_elems)
+        return ZCCL_E_ARG;
+    for (int r = 0; r < N; ++r) if (!send[r] || !recv[r]) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t slot = align_up(bound_of(n), 256);
+    if ((size_t)N * N * slot > c->arena_bytes) return ZCCL_E_ARG;
+    auto gslot = [&](int r, int src) { return c->arena + ((size_t)r * N + src) * slot; };
+    size_t* own_sz = c->sim_sizes;                     // [N]
+    size_t* g_sz = c->sim_sizes + N;                   // [N][N]
+    c->sim_sizes_count = N;
+    if (cudaMemsetAsync(c->sim_sizes, 0, sizeof(size_t) * ((size_t)N * N + N), st) != cudaSuccess) return ZCCL_E_CUDA;
+
+    Params hp{};
+    bool dev = false;
+    RangeList rl;
+    for (int r = 0; r < N; ++r) { rl.x.push_back(send[r]); rl.n.push_back(n); }
+    int rc = resolve_bound(c, rl, eb_mode, eb, hp, dev, st);
+    if (rc != ZCCL_OK) return rc;
+
+    Batcher b;
+    for (int r = 0; r < N; ++r) {   // compress once
+        Job j{};
+        j.x = send[r]; j.n = n; j.out = (uint32_t*)gslot(r, r); j.out_cap = slot; j.out_bytes = own_sz + r;
+        b.add(j, tiles_of(n));
+        if (b.full() && (rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+    }
+    if ((rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+
+    CopyBatcher cb;
+    for (int h = 0; h + 1 < N; ++h) {   // forward compressed bytes around the ring
+        for (int r = 0; r < N; ++r) {
+            const int from = (r - 1 + N) % N;
+            const int src = ((r - 1 - h) % N + N) % N;
+            const size_t* sz = h == 0 ? own_sz + from : g_sz + (size_t)from * N + src;
+            cb.add(gslot(from, src), gslot(r, src), sz, g_sz + (size_t)r * N + src, slot);
+            if (cb.full() && (rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+        }
+        if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+    }
+    for (int r = 0; r < N; ++r) {
+        for (int src = 0; src < N; ++src) {
+            if (src == r) {   // own contribution stays uncompressed
+                if (cudaMemcpyAsync(recv[r] + (size_t)src * n, send[r], sizeof(float) * n, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                    return ZCCL_E_CUDA;
+                continue;
+            }
+            Job j{};
+            j.in_c = (const uint32_t*)gslot(r, src); j.in_cap = slot; j.y = recv[r] + (size_t)src * n; j.n = n;
+            b.add(j, tiles_of(n));
+            if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+        }
+    }
+    return flush_decode(c, b, st);
+}
+
+int zccl_sim_bcast(zccl_ctx* c, const float* root, float* const* recv, int nsinks, size_t n,
+                   int eb_mode, float eb, void* stream)
+{
+    if (!c || (!root && n) || !recv || nsinks < 0 || nsinks > c->max_ranks || !eb_ok(eb_mode, eb) || n > c->max_elems)
+        return ZCCL_E_ARG;
+    for (int r = 0; r < nsinks; ++r) if (!recv[r]) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t slot = align_up(bound_of(n), 256);
+    if ((size_t)(nsinks + 1) * slot > c->arena_bytes) return ZCCL_E_ARG;
+    auto rslot = [&](int rank) { return c->arena + (size_t)rank * slot; };   // rank 0 = root, sinks are 1..nsinks
+    size_t* sz = c->sim_sizes;   // [nsinks + 1]
+    c->sim_sizes_count = 1;
+    if (cudaMemsetAsync(c->sim_sizes, 0, sizeof(size_t) * (size_t)(nsinks + 1), st) != cudaSuccess) return ZCCL_E_CUDA;
+    int rc = zccl_compress(c, root, n, eb_mode, eb, rslot(0), slot, sz, stream);
+    if (rc != ZCCL_OK) return rc;
+    CopyBatcher cb;
+    for (int dist = 1; dist <= nsinks; dist <<= 1) {   // binomial tree: holders forward to rank + dist
+        for (int src = 0; src < dist; ++src) {
+            const int dst = src + dist;
+            if (dst > nsinks) break;
+            cb.add(rslot(src), rslot(dst), sz + src, sz + dst, slot);
+            if (cb.full() && (rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+        }
+        if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+    }
+    Batcher b;
+    for (int k = 0; k < nsinks; ++k) {
+        Job j{};
+        j.in_c = (const uint32_t*)rslot(k + 1); j.in_cap = slot; j.y = recv[k]; j.n = n;
+        b.add(j, tiles_of(n));
+        if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+    }
+    return flush_decode(c, b, st);
+}
+
+int zccl_sim_sizes(zccl_ctx* c, size_t* sizes, int capacity, void* stream)
+{
+    if (!c || !sizes || capacity < 0) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int cnt = c->sim_sizes_count < capacity ? c->sim_sizes_count : capacity;
+    if (cnt > 0 && cudaMemcpyAsync(sizes, c->sim_sizes, sizeof(size_t) * (size_t)cnt, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return ZCCL_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZCCL_E_CUDA;
+    return c->sim_sizes_count;
+}
+
+int zccl_compress_host(zccl_ctx* c, const float* x_host, size_t n, int eb_mode, float eb,
+                       void* out_host, size_t out_capacity, size_t* out_bytes_host, void* stream)
+{
+    if (!c || (!x_host && n) || !out_host || !out_bytes_host || n > c->max_elems) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n && cudaMemcpyAsync(c->stage_x, x_host, sizeof(float) * n, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZCCL_E_CUDA;
+    int rc = zccl_compress(c, c->stage_x, n, eb_mode, eb, c->stage_c, c->stage_c_cap, c->stage_bytes, stream);
+    if (rc != ZCCL_OK) return rc;
+    if (cudaMemcpyAsync(out_bytes_host, c->stage_bytes, sizeof(size_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZCCL_E_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZCCL_E_CUDA;
+    const size_t nbytes = *out_bytes_host;
+    if (nbytes > out_capacity) return ZCCL_E_CAPACITY;
+    if (nbytes && cudaMemcpyAsync(out_host, c->stage_c, nbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZCCL_E_CUDA;
+    return ZCCL_OK;
+}
+
+int zccl_decompress_host(zccl_ctx* c, const void* in_host, size_t in_bytes, float* y_host, size_t y_capacity_elems, void* stream)
+{
+    if (!c || !in_host || (!y_host && y_capacity_elems) || in_bytes > c->stage_c_cap) return ZCCL_E_ARG;
+    if (in_bytes < (size_t)kHeaderBytes) return ZCCL_E_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long n = 0;
+    std::memcpy(&n, (const uint8_t*)in_host + 8, 8);
+    if (n > c->max_elems || n > y_capacity_elems) return ZCCL_E_CAPACITY;
+    if (cudaMemcpyAsync(c->stage_c, in_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ZCCL_E_CUDA;
+    int rc = zccl_decompress(c, c->stage_c, in_bytes, c->stage_x, (size_t)n, stream);
+    if (rc != ZCCL_OK) return rc;
+    if (n && cudaMemcpyAsync(y_host, c->stage_x, sizeof(float) * (size_t)n, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZCCL_E_CUDA;
+    return ZCCL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,102 @@
+// Internal declarations shared by the kernel translation unit and the C boundary.  Not installed.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace zccl {
+
+constexpr uint32_t kMagic = 0x314C435Au;    // 'Z','C','L','1'
+constexpr uint32_t kVersion = 0x05000001u;  // version 1, dtype 0 (fp32), log2(block) = 5
+constexpr int kHeaderBytes = 32;
+constexpr int kHeaderWords = 8;
+constexpr int kBlock = 32;                  // elements per block = warp width
+constexpr int kTile = 4096;                 // elements per tile (Lorenzo restart unit, one index entry)
+constexpr int kBlocksPerTile = kTile / kBlock;
+constexpr int kThreads = 256;               // one CTA works on one tile at a time
+constexpr int kWarps = kThreads / 32;
+constexpr int kBlocksPerWarp = kBlocksPerTile / kWarps;   // 16 consecutive blocks per warp
+constexpr int kMaxJobs = 16;                // chunk-operations batched into one launch
+
+// Device status bits (zccl_status maps them to return codes).
+enum : uint32_t {
+    kStCapacity = 1u << 0,
+    kStRange = 1u << 1,
+    kStBadStream = 1u << 2,
+    kStTimeout = 1u << 3,
+    kStDegenerate = 1u << 4,
+    kStPrecision = 1u << 5,
+};
+
+// Resolved bound (device resident when the mode is value-range relative).
+struct Params {
+    float eb_abs;
+    float s;      // quantisation step
+    float r;      // fl32(1 / s)
+    int valid;    // 0: resolution failed (degenerate range); codec kernels then write nothing
+};
+
+// Scan / bookkeeping workspace owned by the context.
+struct Workspace {
+    unsigned long long* tile_state;  // one 64-bit {epoch:31 | inclusive:1 | words:32} per tile of a launch
+    uint32_t* ticket;                // next tile to hand out
+    uint32_t* done;                  // CTAs that have finished (the last one resets ticket/done, bumps epoch)
+    uint32_t* epoch;                 // launch counter that validates tile_state entries
+    uint32_t* status;                // device status bits
+    Params* params;                  // resolved bound for REL mode
+    uint32_t* minmax;                // two ordered-int keys: running min and max
+    uint32_t max_tiles;
+};
+
+// One chunk-operation.  Encoding jobs (compress, fused hop) and decoding jobs share the struct.
+struct Job {
+    const float* x;         // compress: input; fused: uncompressed local operand (or nullptr)
+    const uint32_t* in_c;   // decode / fused: compressed input stream
+    const uint32_t* in_c2;  // fused, two-compressed form: second stream (or nullptr)
+    uint32_t* out;          // encode: output stream
+    size_t* out_bytes;      // encode: receives stream length
+    float* y;               // decode: output; fused: optional uncompressed sum (or nullptr)
+    unsigned long long n;           // elements (decode: capacity of y in elements)
+    unsigned long long out_cap;     // encode: capacity of out in bytes
+    unsigned long long in_cap;      // bytes readable at in_c
+    unsigned long long in2_cap;     // bytes readable at in_c2
+    uint32_t tile_begin;    // first global tile number of this job within the launch
+    uint32_t flags;
+};
+
+struct JobBatch {
+    Job job[kMaxJobs];
+    int count;
+    uint32_t total_tiles;
+};
+
+struct CopyJob {
+    const uint32_t* src;
+    uint32_t* dst;
+    const size_t* bytes;   // device-resident length
+    size_t* bytes_out;     // optional: where to record the length at the destination
+    unsigned long long cap;
+};
+struct CopyBatch {
+    CopyJob job[kMaxJobs];
+    int count;
+};
+
+struct RangeBatch {
+    const float* x[kMaxJobs];
+    unsigned long long n[kMaxJobs];
+    int count;
+};
+
+enum EncodeMode { kEncodeRaw = 0, kEncodeFused = 1 };
+
+// Launchers (defined next to the kernels).
+cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_resolve(int eb_mode, float eb, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& ws, bool device_params,
+                          Params host_params, int sm_count, cudaStream_t st);
+cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_copy_raw(const float* src, float* dst, size_t n, int sm_count, cudaStream_t st);
+
+}  // namespace zccl

@@ -1,0 +1,208 @@
+"""Thin binding over the C-ABI library ``libzccl.so`` (declared in ``include/zccl.h``): argument marshalling only.
+PyTorch supplies device memory and streams; every step of the path runs in the library's CUDA kernels.  There is
+no CPU fallback: if the library is missing or no CUDA device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libzccl.so"
+
+OK, E_ARG, E_CUDA, E_CAPACITY, E_RANGE, E_BAD_STREAM, E_TIMEOUT, E_DEGENERATE, W_PRECISION = 0, -1, -2, -3, -4, -5, -6, -7, 1
+EB_ABS, EB_REL = 0, 1
+CONSISTENT_OWNER = 1
+TILE, BLOCK, HEADER_BYTES = 4096, 32, 32
+
+EXPORTS = [
+    "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_status", "zccl_strerror",
+    "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
+    "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_sizes",
+    "zccl_compress_host", "zccl_decompress_host",
+]
+
+_lib = None
+
+
+class ZcclError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        msg = lib().zccl_strerror(code).decode() if _lib is not None else str(code)
+        super().__init__(f"{what}: {msg} ({code})")
+        self.code = code
+
+
+def lib():
+    """Loads the shared library (no compute happens here; a GPU is not needed to load it)."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2502_18554_b200.build` "
+                               "(there is no CPU fallback)")
+        L = C.CDLL(str(LIB_PATH))
+        vp, sz = C.c_void_p, C.c_size_t
+        L.zccl_ctx_create.argtypes = [C.POINTER(vp), sz, C.c_int]
+        L.zccl_ctx_destroy.argtypes = [vp]
+        L.zccl_ctx_destroy.restype = None
+        L.zccl_compress_bound.argtypes = [sz]
+        L.zccl_compress_bound.restype = sz
+        L.zccl_status.argtypes = [vp, vp]
+        L.zccl_strerror.argtypes = [C.c_int]
+        L.zccl_strerror.restype = C.c_char_p
+        L.zccl_compress.argtypes = [vp, vp, sz, C.c_int, C.c_float, vp, sz, vp, vp]
+        L.zccl_decompress.argtypes = [vp, vp, sz, vp, sz, vp]
+        L.zccl_decompress_reduce_compress.argtypes = [vp, vp, sz, vp, vp, sz, sz, vp, sz, vp, vp, C.c_uint, vp]
+        L.zccl_sim_allreduce.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, C.c_uint, vp]
+        L.zccl_sim_allgather.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
+        L.zccl_sim_bcast.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
+        L.zccl_sim_sizes.argtypes = [vp, vp, C.c_int, vp]
+        L.zccl_compress_host.argtypes = [vp, vp, sz, C.c_int, C.c_float, vp, sz, vp, vp]
+        L.zccl_decompress_host.argtypes = [vp, vp, sz, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def compress_bound(n: int) -> int:
+    return int(lib().zccl_compress_bound(n))
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_ptr(t: torch.Tensor | None, dtype=None) -> int | None:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _check(rc: int, what: str):
+    if rc != OK:
+        raise ZcclError(rc, what)
+
+
+class Context:
+    """Owns the library context (scan workspace, status word, slots of the emulated ranks)."""
+
+    def __init__(self, max_elems: int, max_ranks: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("zccl needs a CUDA device (sm_100a); there is no CPU fallback")
+        torch.cuda.init()
+        torch.cuda.current_stream()   # make sure a CUDA context exists on the current device
+        h = C.c_void_p()
+        _check(lib().zccl_ctx_create(C.byref(h), max_elems, max_ranks), "zccl_ctx_create")
+        self._h = h
+        self.max_elems, self.max_ranks = max_elems, max_ranks
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().zccl_ctx_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- status
+    def status(self, stream=None) -> int:
+        return int(lib().zccl_status(self._h, _stream_ptr(stream)))
+
+    def check(self, stream=None, allow_warning: bool = True) -> int:
+        rc = self.status(stream)
+        if rc < 0 or (rc > 0 and not allow_warning):
+            raise ZcclError(rc, "device status")
+        return rc
+
+    # ---- codec
+    def compress(self, x: torch.Tensor, eb_mode: int, eb: float, out: torch.Tensor, out_bytes: torch.Tensor,
+                 stream=None, n: int | None = None):
+        """zccl_compress: x float32 [n] -> stream bytes in `out` (uint8), length in `out_bytes` (int64[1], device)."""
+        n = x.numel() if n is None else n
+        _check(lib().zccl_compress(self._h, _dev_ptr(x, torch.float32) if n else None, n, eb_mode, eb,
+                                   _dev_ptr(out, torch.uint8), out.numel(), _dev_ptr(out_bytes, torch.int64),
+                                   _stream_ptr(stream)), "zccl_compress")
+
+    def decompress(self, stream_bytes: torch.Tensor, y: torch.Tensor, in_bytes_max: int | None = None, stream=None):
+        """zccl_decompress: stream bytes (uint8) -> y float32; element count comes from the stream's header."""
+        cap = stream_bytes.numel() if in_bytes_max is None else in_bytes_max
+        _check(lib().zccl_decompress(self._h, _dev_ptr(stream_bytes, torch.uint8), cap,
+                                     _dev_ptr(y, torch.float32) if y.numel() else None, y.numel(),
+                                     _stream_ptr(stream)), "zccl_decompress")
+
+    def decompress_reduce_compress(self, in_c: torch.Tensor, n: int, out_c: torch.Tensor, out_bytes: torch.Tensor,
+                                   local: torch.Tensor | None = None, local_c: torch.Tensor | None = None,
+                                   raw_out: torch.Tensor | None = None, flags: int = 0, stream=None):
+        """zccl_decompress_reduce_compress: out_c = compress(decompress(in_c) + local) in one kernel."""
+        _check(lib().zccl_decompress_reduce_compress(
+            self._h, _dev_ptr(in_c, torch.uint8), in_c.numel(),
+            _dev_ptr(local, torch.float32), _dev_ptr(local_c, torch.uint8),
+            local_c.numel() if local_c is not None else 0, n,
+            _dev_ptr(out_c, torch.uint8), out_c.numel(), _dev_ptr(out_bytes, torch.int64),
+            _dev_ptr(raw_out, torch.float32), flags, _stream_ptr(stream)), "zccl_decompress_reduce_compress")
+
+    # ---- emulated collectives
+    @staticmethod
+    def _ptrs(tensors):
+        return (C.c_void_p * len(tensors))(*[_dev_ptr(t, torch.float32) for t in tensors])
+
+    def sim_allreduce(self, send, recv, eb_mode: int, eb: float, flags: int = 0, stream=None):
+        n = send[0].numel()
+        _check(lib().zccl_sim_allreduce(self._h, self._ptrs(send), self._ptrs(recv), len(send), n, eb_mode, eb, flags,
+                                        _stream_ptr(stream)), "zccl_sim_allreduce")
+
+    def sim_allgather(self, send, recv, eb_mode: int, eb: float, stream=None):
+        n = send[0].numel()
+        _check(lib().zccl_sim_allgather(self._h, self._ptrs(send), self._ptrs(recv), len(send), n, eb_mode, eb,
+                                        _stream_ptr(stream)), "zccl_sim_allgather")
+
+    def sim_bcast(self, root: torch.Tensor, recv, eb_mode: int, eb: float, stream=None):
+        _check(lib().zccl_sim_bcast(self._h, _dev_ptr(root, torch.float32), self._ptrs(recv), len(recv), root.numel(),
+                                    eb_mode, eb, _stream_ptr(stream)), "zccl_sim_bcast")
+
+    def sim_sizes(self, stream=None) -> list[int]:
+        cap = 2 * max(self.max_ranks, 1) ** 2 + 2
+        buf = (C.c_size_t * cap)()
+        cnt = lib().zccl_sim_sizes(self._h, buf, cap, _stream_ptr(stream))
+        if cnt < 0:
+            raise ZcclError(cnt, "zccl_sim_sizes")
+        return [int(buf[i]) for i in range(min(cnt, cap))]
+
+    # ---- host-buffer forms (pinned CPU tensors)
+    def compress_host(self, x_host: torch.Tensor, eb_mode: int, eb: float, out_host: torch.Tensor, stream=None) -> int:
+        nb = C.c_size_t(0)
+        _check(lib().zccl_compress_host(self._h, x_host.data_ptr(), x_host.numel(), eb_mode, eb, out_host.data_ptr(),
+                                        out_host.numel(), C.byref(nb), _stream_ptr(stream)), "zccl_compress_host")
+        return int(nb.value)
+
+    def decompress_host(self, in_host: torch.Tensor, in_bytes: int, y_host: torch.Tensor, stream=None):
+        _check(lib().zccl_decompress_host(self._h, in_host.data_ptr(), in_bytes, y_host.data_ptr(), y_host.numel(),
+                                          _stream_ptr(stream)), "zccl_decompress_host")
+
+
+# ---- convenience wrappers used by tests and examples (allocate with torch, call the entry points above)
+
+def compress_to_bytes(ctx: Context, x: torch.Tensor, eb_mode: int, eb: float, capacity: int | None = None):
+    """Returns (stream as a CUDA uint8 tensor trimmed to its length, device status)."""
+    cap = compress_bound(x.numel()) if capacity is None else capacity
+    out = torch.empty(max(cap, 1), dtype=torch.uint8, device=x.device)
+    nbytes = torch.zeros(1, dtype=torch.int64, device=x.device)
+    ctx.compress(x, eb_mode, eb, out[:cap] if cap else out[:0], nbytes)
+    rc = ctx.status()
+    return out[: int(nbytes.item())], rc
+
+
+def decompress_from_bytes(ctx: Context, stream_bytes: torch.Tensor, n: int):
+    y = torch.empty(n, dtype=torch.float32, device=stream_bytes.device)
+    ctx.decompress(stream_bytes, y)
+    rc = ctx.status()
+    return y, rc

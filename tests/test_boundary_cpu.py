@@ -1,0 +1,67 @@
+"""Host-side checks that need no GPU: the C-ABI library loads and exports every symbol the header declares, its
+pure host functions agree with the oracle, and argument errors the host can see are reported without CUDA."""
+import ctypes as C
+import re
+from pathlib import Path
+
+import pytest
+
+import oracle
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2502_18554_b200 import build, zccl
+    build.build()
+    return zccl.lib()
+
+
+def declared_symbols():
+    text = (ROOT / "include" / "zccl.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(zccl_[a-z_]+)\s*\(", text)))
+
+
+def test_header_symbols_are_exported(lib):
+    from paper_2502_18554_b200 import zccl
+    names = declared_symbols()
+    assert "zccl_compress" in names and "zccl_decompress_reduce_compress" in names and "zccl_sim_allreduce" in names
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in zccl.h but not exported"
+    assert sorted(zccl.EXPORTS) == [n for n in names]
+
+
+def test_compress_bound_matches_oracle(lib):
+    for n in [0, 1, 31, 32, 33, 4095, 4096, 4097, 8192, 10 ** 6 + 7, 2 ** 24, 2 ** 28 + 5]:
+        assert lib.zccl_compress_bound(n) == oracle.compress_bound(n)
+
+
+def test_strerror(lib):
+    from paper_2502_18554_b200 import zccl
+    assert lib.zccl_strerror(0) == b"ok"
+    for code in (zccl.E_ARG, zccl.E_CUDA, zccl.E_CAPACITY, zccl.E_RANGE, zccl.E_BAD_STREAM, zccl.E_TIMEOUT,
+                 zccl.E_DEGENERATE, zccl.W_PRECISION):
+        assert lib.zccl_strerror(code) not in (b"ok", b"unknown status")
+
+
+def test_null_context_is_rejected_without_cuda(lib):
+    from paper_2502_18554_b200 import zccl
+    assert lib.zccl_status(None, None) == zccl.E_ARG
+    assert lib.zccl_compress(None, None, 0, 0, 1.0, None, 0, None, None) == zccl.E_ARG
+    assert lib.zccl_decompress(None, None, 0, None, 0, None) == zccl.E_ARG
+    assert lib.zccl_ctx_create(None, 1, 0) == zccl.E_ARG
+    h = C.c_void_p()
+    assert lib.zccl_ctx_create(C.byref(h), 0, 0) == zccl.E_ARG
+    assert lib.zccl_ctx_create(C.byref(h), 10, 1000) == zccl.E_ARG
+    lib.zccl_ctx_destroy(None)
+
+
+def test_binding_refuses_to_run_without_gpu():
+    import torch
+    from paper_2502_18554_b200 import zccl
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    with pytest.raises(RuntimeError):
+        zccl.Context(1 << 20)
