@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the ZCCL hot path on B200: `python bench.py --gpus N --steps K --warmup W [--impl reference]`.
+
+One step = one pass of the whole hot path over one 64 MiB batch (a 256^3 fp32 Fourier-mode field, the paper's
+3-D scientific-field workload shape) at a value-range-relative bound of 1e-3:
+  compress (range pass + bound resolution + encode), decompress, fused decompress-add-recompress against a
+  second field, an emulated 8-rank ring Allreduce (each rank one eighth of the batch) and an emulated 8-rank ring
+  Allgather (each rank 1 MiB).
+`value` = uncompressed bytes that pass through a codec kernel per step / step time (GB/s), summed over ranks.
+With N > 1 every rank runs the same step on its own differently seeded batch (independent replicas; the path has no
+cross-GPU exchange).  `--impl reference` times the CPU oracle on the same step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+SIDE = 256
+N_ELEMS = SIDE ** 3                 # 2^24 elements = 64 MiB
+REL = 1e-3
+RANKS = 8
+AG_PER_RANK = 1 << 18               # allgather: 1 MiB per rank
+ROT = 4                             # rotating buffer sets, each larger than L2
+METRIC = "compress / decompress / fused decomp-reduce-comp GB/s (uncompressed bytes through the codec per step)"
+WORKLOAD = ("cfg1: 256^3 fp32 Fourier-mode field (64 MiB), REL 1e-3; step = compress + decompress + fused hop + "
+            "8-rank ring allreduce (8 MiB/rank) + 8-rank allgather (1 MiB/rank)")
+
+
+def step_units_bytes() -> dict:
+    """Uncompressed bytes entering an encoder or leaving a decoder, per op of one step."""
+    full = 4 * N_ELEMS
+    per_rank = full // RANKS
+    chunk = per_rank // RANKS
+    ar = RANKS * chunk + (RANKS - 1) * RANKS * chunk + RANKS * (RANKS - 1) * chunk
+    ag = RANKS * 4 * AG_PER_RANK + RANKS * (RANKS - 1) * 4 * AG_PER_RANK
+    return {"compress": full, "decompress": full, "fused": full, "allreduce": ar, "allgather": ag}
+
+
+def make_fields(rank: int):
+    from paper_2502_18554_b200 import fields
+    x = fields.fourier_field_3d(SIDE, seed=1 + 10 * rank)
+    loc = fields.fourier_field_3d(SIDE, seed=2 + 10 * rank)
+    return x, loc
+
+
+# --------------------------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in out.splitlines():
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_step(x, loc, sample_elems: int):
+    """The same step on the CPU oracle, on the first `sample_elems` elements of the batch."""
+    import oracle
+    xs, ls = x[:sample_elems], loc[:sample_elems]
+    st, _ = oracle.compress(xs, oracle.EB_REL, REL)
+    oracle.decompress(st)
+    oracle.drc(st, local=ls)
+    per = sample_elems // RANKS
+    oracle.sim_allreduce([xs[r * per:(r + 1) * per] for r in range(RANKS)], oracle.EB_REL, REL)
+    ag = min(AG_PER_RANK, per)
+    oracle.sim_allgather([xs[r * ag:(r + 1) * ag] for r in range(RANKS)], oracle.EB_REL, REL)
+    units = step_units_bytes()
+    scale = sample_elems / N_ELEMS
+    total = (units["compress"] + units["decompress"] + units["fused"] + units["allreduce"]) * scale
+    total += RANKS * 4 * ag + RANKS * (RANKS - 1) * 4 * ag
+    return total
+
+
+def run_oracle(x, loc, steps: int, warmup: int, sample_elems: int):
+    for _ in range(warmup):
+        oracle_step(x, loc, sample_elems)
+    t0 = time.perf_counter()
+    nbytes = 0
+    for _ in range(steps):
+        nbytes += oracle_step(x, loc, sample_elems)
+    dt = time.perf_counter() - t0
+    return nbytes / dt / 1e9, dt / steps * 1e3
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    x, loc = make_fields(0)
+    sample = N_ELEMS // 4
+    gbs, ms = run_oracle(x, loc, args.steps, max(args.warmup, 1), sample)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": {"workload": WORKLOAD},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                         "sample": f"first {sample} of {N_ELEMS} elements of the batch per step (one quarter)"},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------- CUDA arm
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_2502_18554_b200 import build, zccl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    z = zccl
+    ctx = z.Context(N_ELEMS, RANKS)
+
+    # ---- inputs: one batch per rank, copied into ROT rotating sets (distinct memory, > L2 each) by rolling it
+    x_h, loc_h = make_fields(rank)
+    shift = 4096 * 37
+    xs = [torch.from_numpy(np.roll(x_h, k * shift)).to(dev) for k in range(ROT)]
+    locs = [torch.from_numpy(np.roll(loc_h, k * shift)).to(dev) for k in range(ROT)]
+    cap = z.compress_bound(N_ELEMS)
+    cs = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(ROT)]
+    c2s = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(ROT)]
+    ys = [torch.empty(N_ELEMS, dtype=torch.float32, device=dev) for _ in range(ROT)]
+    ars = [torch.empty(N_ELEMS, dtype=torch.float32, device=dev) for _ in range(ROT)]
+    ags = [torch.empty(RANKS * RANKS * AG_PER_RANK, dtype=torch.float32, device=dev) for _ in range(ROT)]
+    nb1 = torch.zeros(1, dtype=torch.int64, device=dev)
+    nb2 = torch.zeros(1, dtype=torch.int64, device=dev)
+    per = N_ELEMS // RANKS
+    stream = torch.cuda.current_stream()
+
+    names = ["compress", "decompress", "fused", "allreduce", "allgather"]
+
+    def step(i: int, evs=None):
+        k = i % ROT
+        x, loc, c, c2, y, ar, ag = xs[k], locs[k], cs[k], c2s[k], ys[k], ars[k], ags[k]
+        if evs is not None:
+            evs[0].record(stream)
+        ctx.compress(x, z.EB_REL, REL, c, nb1)
+        if evs is not None:
+            evs[1].record(stream)
+        ctx.decompress(c, y)
+        if evs is not None:
+            evs[2].record(stream)
+        ctx.decompress_reduce_compress(c, N_ELEMS, c2, nb2, local=loc)
+        if evs is not None:
+            evs[3].record(stream)
+        ctx.sim_allreduce([x[r * per:(r + 1) * per] for r in range(RANKS)],
+                          [ar[r * per:(r + 1) * per] for r in range(RANKS)], z.EB_REL, REL)
+        if evs is not None:
+            evs[4].record(stream)
+        ctx.sim_allgather([x[r * AG_PER_RANK:(r + 1) * AG_PER_RANK] for r in range(RANKS)],
+                          [ag[r * RANKS * AG_PER_RANK:(r + 1) * RANKS * AG_PER_RANK] for r in range(RANKS)],
+                          z.EB_REL, REL)
+        if evs is not None:
+            evs[5].record(stream)
+
+    def fence():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    ctx.check()
+    ratio1 = 4 * N_ELEMS / int(nb1.item())
+    ratio2 = 4 * N_ELEMS / int(nb2.item())
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    fence()
+    sampler.start()
+    launches0 = z.launch_count()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i, evs[i])
+    t_end.record(stream)
+    fence()
+    launches = z.launch_count() - launches0
+    clocks = sampler.stop()
+    ctx.check()
+    ms_total = t_begin.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    units = step_units_bytes()
+    total_bytes = sum(units.values())
+    value = world * total_bytes / (ms_step * 1e-3) / 1e9
+
+    op_ms = {nm: statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps))
+             for j, nm in enumerate(names)}
+
+    # ---- roofline of the dominant kernel.  decompress and the fused hop are exactly one kernel launch per call,
+    # so their event brackets time that kernel alone; compress under a relative bound also holds the range pass,
+    # so the encoder kernel is additionally timed alone with the pre-resolved absolute bound.
+    peaks = {}
+    pk = ROOT / "MEASURED_PEAKS.json"
+    peak_src = "fallback"
+    peak = 6650.0
+    if pk.exists():
+        try:
+            peaks = json.loads(pk.read_text())
+            peak = float(peaks["hbm_gbs"]); peak_src = "measured"
+        except Exception:
+            pass
+    eb_abs = float(np.float32(REL) * (np.float32(x_h.max()) - np.float32(x_h.min())))
+    enc_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for i in range(args.steps):
+        k = i % ROT
+        enc_ev[i][0].record(stream)
+        ctx.compress(xs[k], z.EB_ABS, eb_abs, cs[k], nb1)
+        enc_ev[i][1].record(stream)
+    torch.cuda.synchronize()
+    enc_ms = statistics.mean(a.elapsed_time(b) for a, b in enc_ev)
+    in_b = 4 * N_ELEMS
+    c1_b = in_b / ratio1
+    c2_b = in_b / ratio2
+    kern = {
+        "encode(compress, ABS bound)": {"ms": enc_ms, "bytes": in_b + c1_b},
+        "decode(decompress)": {"ms": op_ms["decompress"], "bytes": c1_b + in_b},
+        "encode_fused(decompress-add-recompress)": {"ms": op_ms["fused"], "bytes": c1_b + in_b + c2_b},
+    }
+    for v in kern.values():
+        v["achieved_gbs"] = v["bytes"] / (v["ms"] * 1e-3) / 1e9
+        v["frac"] = v["achieved_gbs"] / peak
+        v["uncompressed_gbs"] = in_b / (v["ms"] * 1e-3) / 1e9
+    # the fused kernel also runs the 56 chunk hops of the allreduce: it carries the largest share of the step
+    dom = "encode_fused(decompress-add-recompress)"
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["achieved_gbs"], "peak": peak, "unit": "GB/s",
+                "frac": kern[dom]["frac"], "traffic": None, "peak_source": f"of {peak_src}",
+                "algorithmic_bytes_per_launch": kern[dom]["bytes"]}
+    tr = ROOT / "profiles" / "traffic.json"
+    if tr.exists():
+        try:
+            roofline["traffic"] = json.loads(tr.read_text()).get("encode_fused_bytes_per_launch_64MiB")
+        except Exception:
+            pass
+
+    # ---- end to end through the host-buffer entry points (pinned host memory; copies inside the timed region)
+    xh = torch.from_numpy(x_h).pin_memory()
+    oh = torch.empty(cap, dtype=torch.uint8).pin_memory()
+    yh = torch.empty(N_ELEMS, dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        nb = ctx.compress_host(xh, z.EB_REL, REL, oh)
+        ctx.decompress_host(oh, nb, yh)
+    fence()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        nb = ctx.compress_host(xh, z.EB_REL, REL, oh)
+        ctx.decompress_host(oh, nb, yh)
+    e1.record(stream)
+    fence()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_ms /= e2e_steps
+    e2e = {"value": world * 2 * in_b / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+           "what": "zccl_compress_host + zccl_decompress_host of the 64 MiB batch (uncompressed bytes per op / time)",
+           "ms_per_step": e2e_ms, "h2d_bytes_per_step": in_b + nb, "d2h_bytes_per_step": nb + 8 + in_b}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        sample = N_ELEMS // 4
+        reps = 4
+        gbs, ms = run_oracle(x_h, loc_h, reps, 1, sample)
+        cpu = {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "host_cores": os.cpu_count(),
+               "sample": f"{reps} steps on the first {sample} of {N_ELEMS} elements of the batch (one quarter), "
+                         f"{ms * reps / 1e3:.1f} s of CPU work"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": f"inputs and outputs rotate over {ROT} buffer sets, each above L2",
+                       "rel_bound": REL, "ratio_compress": ratio1, "ratio_fused_out": ratio2,
+                       "parallelism": f"{world} independent replicas" if world > 1 else "single GPU"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu,
+            "ops_ms": op_ms, "ops_uncompressed_gbs": {nm: units[nm] / (op_ms[nm] * 1e-3) / 1e9 for nm in names},
+            "kernels": kern,
+        }
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -78,6 +78,10 @@ size_t zccl_compress_bound(size_t n);
  */
 int zccl_status(zccl_ctx* ctx, void* stream);
 
+/* Number of kernels this library has launched in this process so far (for launch accounting in benchmarks;
+ * no paper counterpart).  Pure host function. */
+unsigned long long zccl_launch_count(void);
+
 /* Static description of a status code. */
 const char* zccl_strerror(int code);
 

@@ -159,6 +159,8 @@ extern "C" {
 
 size_t zccl_compress_bound(size_t n) { return bound_of(n); }
 
+unsigned long long zccl_launch_count(void) { return launch_count(); }
+
 const char* zccl_strerror(int code)
 {
     switch (code) {

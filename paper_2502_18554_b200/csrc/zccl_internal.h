@@ -97,6 +97,6 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
-cudaError_t launch_copy_raw(const float* src, float* dst, size_t n, int sm_count, cudaStream_t st);
+unsigned long long launch_count();
 
 }  // namespace zccl

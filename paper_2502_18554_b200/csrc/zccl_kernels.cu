@@ -562,10 +562,13 @@ __global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
 }
 
 int g_encode_ctas_per_sm = 0, g_decode_ctas_per_sm = 0;
+unsigned long long g_launches = 0;   // kernels launched by this library in this process
 
 }  // namespace
 
 // ------------------------------------------------------------------------------------------------ launchers
+
+unsigned long long launch_count() { return g_launches; }
 
 cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
@@ -575,12 +578,14 @@ cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count
     unsigned long long want = (nmax / 4 + 255) / 256;
     unsigned per = (unsigned)((sm_count * 8 + rb.count - 1) / rb.count);
     unsigned gx = (unsigned)(want < per ? (want ? want : 1) : per);
+    ++g_launches;
     range_kernel<<<dim3(gx, rb.count), 256, 0, st>>>(rb, ws);
     return cudaGetLastError();
 }
 
 cudaError_t launch_resolve(int eb_mode, float eb, const Workspace& ws, cudaStream_t st)
 {
+    ++g_launches;
     resolve_kernel<<<1, 32, 0, st>>>(eb_mode, eb, ws);
     return cudaGetLastError();
 }
@@ -597,6 +602,7 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
     }
     unsigned long long cap = (unsigned long long)sm_count * g_encode_ctas_per_sm;
     unsigned grid = (unsigned)(jb.total_tiles < cap ? jb.total_tiles : cap);
+    ++g_launches;
     if (mode == kEncodeRaw)
         encode_kernel<kEncodeRaw><<<grid, kThreads, 0, st>>>(jb, ws, host_params, device_params ? 1 : 0);
     else
@@ -614,6 +620,7 @@ cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count,
     }
     unsigned long long cap = (unsigned long long)sm_count * g_decode_ctas_per_sm;
     unsigned grid = (unsigned)(jb.total_tiles < cap ? jb.total_tiles : cap);
+    ++g_launches;
     decode_kernel<<<grid, kThreads, 0, st>>>(jb, ws);
     return cudaGetLastError();
 }
@@ -622,6 +629,7 @@ cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, 
 {
     if (cb.count <= 0) return cudaSuccess;
     unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
+    ++g_launches;
     copy_kernel<<<dim3(gx ? gx : 1, cb.count), 256, 0, st>>>(cb, ws);
     return cudaGetLastError();
 }

@@ -18,7 +18,7 @@ CONSISTENT_OWNER = 1
 TILE, BLOCK, HEADER_BYTES = 4096, 32, 32
 
 EXPORTS = [
-    "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_status", "zccl_strerror",
+    "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_sizes",
     "zccl_compress_host", "zccl_decompress_host",
@@ -48,6 +48,8 @@ def lib():
         L.zccl_ctx_destroy.restype = None
         L.zccl_compress_bound.argtypes = [sz]
         L.zccl_compress_bound.restype = sz
+        L.zccl_launch_count.argtypes = []
+        L.zccl_launch_count.restype = C.c_ulonglong
         L.zccl_status.argtypes = [vp, vp]
         L.zccl_strerror.argtypes = [C.c_int]
         L.zccl_strerror.restype = C.c_char_p
@@ -66,6 +68,10 @@ def lib():
 
 def compress_bound(n: int) -> int:
     return int(lib().zccl_compress_bound(n))
+
+
+def launch_count() -> int:
+    return int(lib().zccl_launch_count())
 
 
 def _stream_ptr(stream) -> int:
