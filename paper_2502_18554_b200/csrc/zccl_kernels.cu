@@ -1,10 +1,22 @@
 // fZ-light codec kernels for sm_100a: range reduction, bound resolution, encoder (plain and fused with a
 // decode + add front end), decoder, and compressed-chunk copy.
 //
-// Work decomposition: one CTA of 256 threads handles one 4096-element tile at a time; each of its 8 warps owns
-// 16 consecutive 32-element blocks, one element per lane, so a block's code length is a warp OR-reduction and
-// each bit plane is one ballot.  Tiles are handed out by an atomic ticket, so a tile's predecessors in the
-// placement scan (decoupled look-back over tile sizes) have always started before it.
+// Work decomposition.  One CTA of 256 threads handles one 4096-element tile at a time; each of its 8 warps owns
+// 16 consecutive 32-element blocks, one element per lane, so that a block's code length is one warp OR-reduction
+// and each bit plane is one ballot.  The kernels are bound by instruction issue (integer ALU pipe: 2
+// warp-instructions/clk/SM; shared memory and shuffles: 1), not by HBM, so the design minimises ALU and LSU
+// instructions per block:
+//   * tiles are staged in shared memory by 1-D bulk copies (cp.async.bulk + mbarrier), double buffered in the
+//     encoder, so no thread spends instructions or registers on global loads;
+//   * the common case runs in fp32 on the FMA pipe: codes are rounded with the 1.5*2^23 trick, deltas are float
+//     subtractions (exact below 2^23), magnitudes are read from the mantissa of |delta| + 2^23.  Tiles whose
+//     values leave the exactly representable range, ragged tails and unaligned inputs take an integer path
+//     that computes the same bits;
+//   * the encoder writes each block's words to a fixed slot and compacts while copying out, so quantisation and
+//     encoding are a single pass over a block; the decoder undoes the Lorenzo recurrence by a warp-local
+//     transposition through shared memory (16 consecutive elements per thread) instead of shuffle scans.
+// Tiles are handed out by an atomic ticket, so a tile's predecessors in the placement scan (decoupled look-back
+// over tile sizes) have always started before it.  Every wait is bounded and reports through the status word.
 #include "zccl_internal.h"
 
 namespace zccl {
@@ -12,7 +24,17 @@ namespace zccl {
 namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kSpinLimit = 1 << 20;   // polls of a predecessor's scan state before giving up (about a second)
+constexpr int kSpinLimit = 1 << 20;            // polls of a scan state or an mbarrier before giving up
+constexpr float kRoundMagic = 12582912.0f;     // 1.5 * 2^23: t + kRoundMagic has rint(t) in its low mantissa bits
+constexpr uint32_t kRoundMagicBits = 0x4B400000u;
+constexpr float kTwo23 = 8388608.0f;           // 2^23: |d| + 2^23 has the integer |d| in its mantissa
+constexpr float kGuardExact = 8.796093e12f;    // 2^43: sum of squares below it => every |x r| < 2^21.5
+constexpr float kGuardSmall = 1.0e9f;          // below 2^30: no |x r| can exceed 2^15
+constexpr int kSlotWords = 33;                 // sign word + up to 32 planes
+constexpr int kBlobStageWords = 2048 + 8;      // compressed tiles up to 8 KiB are staged by bulk copy
+constexpr int kFastDecodeMaxL = 18;
+
+// ------------------------------------------------------------------------------------------------ small helpers
 
 __device__ __forceinline__ uint32_t f2key(float f)
 {
@@ -28,7 +50,6 @@ __device__ __forceinline__ unsigned long long pack_state(uint32_t epoch, uint32_
 {
     return ((unsigned long long)epoch << 33) | ((unsigned long long)inclusive << 32) | words;
 }
-
 __device__ __forceinline__ unsigned long long ld_state(const unsigned long long* p)
 {
     unsigned long long v;
@@ -39,8 +60,52 @@ __device__ __forceinline__ void st_state(unsigned long long* p, unsigned long lo
 {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-
 __device__ __forceinline__ uint32_t ldg_u32(const uint32_t* p) { return __ldg(p); }
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait for a bulk copy to land; false after kSpinLimit polls.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity)
+{
+    for (int it = 0; it < kSpinLimit; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// 1-D bulk copy global -> this CTA's shared memory; addresses and size are multiples of 16 bytes.  The proxy
+// fence orders earlier ordinary accesses to the destination before the copy engine's writes.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar)
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
+{
+    int j = 0;
+#pragma unroll 1
+    for (int k = 1; k < jb.count; ++k)
+        if (jb.job[k].tile_begin <= ticket) j = k;
+    return j;
+}
 
 // ------------------------------------------------------------------------------------------------ range (REL)
 
@@ -135,356 +200,501 @@ __device__ __forceinline__ StreamInfo read_header(const uint32_t* in, unsigned l
     return h;
 }
 
-// ------------------------------------------------------------------------------------------------ tile decoder
+// ================================================================================================ DECODE SIDE
 
-// Decodes this warp's 16 blocks of tile `tile` into codes relative to the warp's first element:
-// q[i] = sum of the deltas from the warp's first block up to this lane (the caller adds the outlier and the sums
-// of the preceding warps).  Returns false, uniformly over the CTA, when the tile's blob is inconsistent.
-__device__ __forceinline__ bool decode_tile_warp(const uint32_t* __restrict__ in, unsigned long long cap_bytes,
-                                                 const StreamInfo& h, uint32_t tile, int warp, int lane,
-                                                 int32_t (&q)[kBlocksPerWarp], int32_t& outlier)
+// What a tile's index entry and code-length bytes say.  Uniform over the CTA (every warp reads the same words).
+struct TileDesc {
+    const uint32_t* blob;     // global: outlier word, code-length words, payload
+    uint32_t words;           // blob size
+    uint32_t nb, padw, len;
+    int32_t outlier;
+    bool ok;                  // sizes consistent with the index
+    bool fast;                // full tile whose codes stay exact in fp32 and whose blob fits the staging buffer
+    uint32_t lw;              // this lane's code-length word (blocks 4*lane .. 4*lane+3)
+    uint32_t o0, o1, o2, o3;  // payload offsets (words) of this lane's four blocks
+};
+
+__device__ __forceinline__ TileDesc describe_tile(const uint32_t* __restrict__ in, unsigned long long cap_bytes,
+                                                  const StreamInfo& h, uint32_t tile, int lane)
 {
+    TileDesc d;
+    d.ok = false; d.fast = false; d.blob = in; d.words = 0; d.outlier = 0; d.lw = 0; d.o0 = d.o1 = d.o2 = d.o3 = 0;
     const uint32_t* idx = in + kHeaderWords;
     const uint32_t w_end = ldg_u32(idx + tile);
     const uint32_t w_beg = tile ? ldg_u32(idx + tile - 1) : 0u;
     const unsigned long long blob0 = (unsigned long long)kHeaderWords + h.nT;   // in words
-    if (w_end < w_beg) return false;
-    if ((blob0 + w_end) * 4ull > cap_bytes) return false;
     const unsigned long long start = (unsigned long long)tile * kTile;
-    const uint32_t len = (uint32_t)((h.n - start < (unsigned long long)kTile) ? (h.n - start) : kTile);
-    const uint32_t nb = (len + kBlock - 1) / kBlock;
-    const uint32_t padw = (nb + 3) >> 2;
-    const uint32_t words = w_end - w_beg;
-    if (words < 1 + padw) return false;
-    const uint32_t* blob = in + blob0 + w_beg;
-    outlier = (int32_t)ldg_u32(blob);
+    d.len = (uint32_t)((h.n - start < (unsigned long long)kTile) ? (h.n - start) : kTile);
+    d.nb = (d.len + kBlock - 1) / kBlock;
+    d.padw = (d.nb + 3) >> 2;
+    if (w_end < w_beg) return d;
+    if ((blob0 + w_end) * 4ull > cap_bytes) return d;
+    d.words = w_end - w_beg;
+    if (d.words < 1 + d.padw) return d;
+    d.blob = in + blob0 + w_beg;
+    d.outlier = (int32_t)ldg_u32(d.blob);
 
     // code lengths: one word (4 blocks) per lane; sizes; warp-wide exclusive scan of the sizes
-    uint32_t lw = ((uint32_t)lane < padw) ? ldg_u32(blob + 1 + lane) : 0u;
+    const uint32_t lw = ((uint32_t)lane < d.padw) ? ldg_u32(d.blob + 1 + lane) : 0u;
     const uint32_t L0 = lw & 0xFF, L1 = (lw >> 8) & 0xFF, L2 = (lw >> 16) & 0xFF, L3 = lw >> 24;
     bool bad = (L0 > 31) | (L1 > 31) | (L2 > 31) | (L3 > 31);
-    // blocks at or beyond nb must have zero code length (they are padding of the code-length area)
-    const uint32_t b0 = 4u * lane;
-    if ((b0 + 0 >= nb && L0) || (b0 + 1 >= nb && L1) || (b0 + 2 >= nb && L2) || (b0 + 3 >= nb && L3)) bad = true;
+    const uint32_t b0 = 4u * lane;   // blocks at or beyond nb are padding of the code-length area: must be zero
+    if ((b0 + 0 >= d.nb && L0) || (b0 + 1 >= d.nb && L1) || (b0 + 2 >= d.nb && L2) || (b0 + 3 >= d.nb && L3)) bad = true;
     const uint32_t z0 = L0 ? L0 + 1 : 0, z1 = L1 ? L1 + 1 : 0, z2 = L2 ? L2 + 1 : 0, z3 = L3 ? L3 + 1 : 0;
     const uint32_t lane_sum = z0 + z1 + z2 + z3;
     uint32_t incl = lane_sum;
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        uint32_t t = __shfl_up_sync(kFull, incl, d);
-        if (lane >= d) incl += t;
+    for (int s = 1; s < 32; s <<= 1) {
+        uint32_t t = __shfl_up_sync(kFull, incl, s);
+        if (lane >= s) incl += t;
     }
     const uint32_t total = __shfl_sync(kFull, incl, 31);
     bad = __any_sync(kFull, bad);
-    if (bad || 1 + padw + total != words) return false;
-    const uint32_t o0 = incl - lane_sum, o1 = o0 + z0, o2 = o1 + z1, o3 = o2 + z2;
-    const uint32_t* payload = blob + 1 + padw;
+    if (bad || 1 + d.padw + total != d.words) return d;
+    d.ok = true;
+    d.lw = lw;
+    d.o0 = incl - lane_sum; d.o1 = d.o0 + z0; d.o2 = d.o1 + z1; d.o3 = d.o2 + z2;
 
-    // fetch: lane k of a block reads word k of the block's payload (sign word, then planes)
-    uint32_t word[kBlocksPerWarp];
-    uint32_t Ls[kBlocksPerWarp];
-#pragma unroll
+    // fp32 exactness: every partial sum of deltas is below sum_b 32 * 2^L_b; with the outlier it must stay < 2^24
+    const uint32_t Lmax = max(max(L0, L1), max(L2, L3));
+    uint32_t spread = 1u << 24;
+    if (Lmax <= (uint32_t)kFastDecodeMaxL) spread = (32u << L0) + (32u << L1) + (32u << L2) + (32u << L3);
+    spread = __reduce_add_sync(kFull, min(spread, 1u << 24));   // at most 32 * 2^24 = 2^29: no overflow
+    const uint32_t ao = (uint32_t)(d.outlier < 0 ? -d.outlier : d.outlier);
+    const bool exact = ao < (1u << 23) && spread < (1u << 23);
+    // staging copies the 16-byte-aligned cover of the blob; it must stay inside the readable bytes
+    const uintptr_t a_beg = (uintptr_t)d.blob & ~(uintptr_t)15;
+    const uintptr_t a_end = ((uintptr_t)(d.blob + d.words) + 15) & ~(uintptr_t)15;
+    const bool stageable = (a_end - a_beg) <= (uintptr_t)(kBlobStageWords * 4) &&
+                           (a_end - (uintptr_t)in) <= (uintptr_t)cap_bytes;
+    d.fast = exact && stageable && d.len == (uint32_t)kTile;
+    return d;
+}
+
+// Integer path: decodes this warp's 16 blocks straight from global memory into codes relative to the warp's first
+// element, one element per lane (q[i] = sum of deltas from the warp's first element; the caller adds the outlier
+// and the sums of the preceding warps).
+__device__ __noinline__ void decode_blocks_int(const TileDesc& d, int warp, int lane, int32_t* __restrict__ q)
+{
+    const uint32_t* payload = d.blob + 1 + d.padw;
+    int32_t carry = 0;
+#pragma unroll 1
     for (int i = 0; i < kBlocksPerWarp; ++i) {
         const int src = 4 * warp + (i >> 2);
-        const uint32_t lwi = __shfl_sync(kFull, lw, src);
+        const uint32_t lwi = __shfl_sync(kFull, d.lw, src);
         const uint32_t L = (lwi >> (8 * (i & 3))) & 0xFF;
-        const uint32_t osel = (i & 3) == 0 ? o0 : (i & 3) == 1 ? o1 : (i & 3) == 2 ? o2 : o3;
+        const uint32_t osel = (i & 3) == 0 ? d.o0 : (i & 3) == 1 ? d.o1 : (i & 3) == 2 ? d.o2 : d.o3;
         const uint32_t off = __shfl_sync(kFull, osel, src);
-        Ls[i] = L;
-        word[i] = (L && (uint32_t)lane <= L) ? ldg_u32(payload + off + lane) : 0u;
-    }
-    int32_t carry = 0;
-#pragma unroll
-    for (int i = 0; i < kBlocksPerWarp; ++i) {
-        const uint32_t L = Ls[i];
         int32_t v = 0;
         if (L) {   // uniform over the warp
-            const uint32_t sign = __shfl_sync(kFull, word[i], 0);
+            const uint32_t word = ((uint32_t)lane <= L) ? ldg_u32(payload + off + lane) : 0u;
+            const uint32_t sign = __shfl_sync(kFull, word, 0);
             uint32_t mag = 0;
             for (uint32_t k = 0; k < L; ++k) {
-                const uint32_t plane = __shfl_sync(kFull, word[i], k + 1);
+                const uint32_t plane = __shfl_sync(kFull, word, k + 1);
                 mag |= ((plane >> lane) & 1u) << k;
             }
             v = ((sign >> lane) & 1u) ? -(int32_t)mag : (int32_t)mag;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                int32_t t = __shfl_up_sync(kFull, v, d);
-                if (lane >= d) v += t;
+            for (int s = 1; s < 32; s <<= 1) {
+                int32_t t = __shfl_up_sync(kFull, v, s);
+                if (lane >= s) v += t;
             }
         }
         q[i] = carry + v;
         carry = __shfl_sync(kFull, q[i], 31);
     }
-    return true;
 }
 
-// ------------------------------------------------------------------------------------------------ encoder
+#define ZCCL_DEC_PLANE(k)                                        \
+    case (k) + 1:                                                \
+        if (pw[(k) + 1] & lanebit) mag += (float)(1u << (k));
 
-struct EncodeShared {
-    uint32_t stage[1 + kBlocksPerTile / 4 + kBlocksPerTile * kBlock];   // a tile's blob, worst case
-    uint32_t warp_words[kWarps];
-    int32_t warp_lastq[kWarps];
-    int32_t warp_sum[2][kWarps];
-    uint32_t ticket;
-    uint32_t excl;
-    uint32_t skip;
+// fp32 path: rebuilds this warp's 16 blocks of deltas from the staged blob and stores them, as exact floats, in
+// the warp's 512-word region `wbuf`, row i = block i, element j of a row at word j ^ ((i & 3) << 2) (so that the
+// 128-bit reads of decode_scan_f32 are free of bank conflicts).
+__device__ __forceinline__ void decode_blocks_f32(const uint32_t* __restrict__ payload, const uint32_t* __restrict__ tbl,
+                                                  float* __restrict__ wbuf, int lane)
+{
+    const uint32_t lanebit = 1u << lane;
+#pragma unroll 1
+    for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = 4 * g + u;
+            const uint32_t e = tbl[i];               // broadcast read: (offset << 8) | code length
+            const uint32_t L = e & 0xFF;
+            const uint32_t* pw = payload + (e >> 8);
+            float mag = 0.0f;
+            switch (L) {
+                ZCCL_DEC_PLANE(17) ZCCL_DEC_PLANE(16) ZCCL_DEC_PLANE(15) ZCCL_DEC_PLANE(14) ZCCL_DEC_PLANE(13)
+                ZCCL_DEC_PLANE(12) ZCCL_DEC_PLANE(11) ZCCL_DEC_PLANE(10) ZCCL_DEC_PLANE(9) ZCCL_DEC_PLANE(8)
+                ZCCL_DEC_PLANE(7) ZCCL_DEC_PLANE(6) ZCCL_DEC_PLANE(5) ZCCL_DEC_PLANE(4) ZCCL_DEC_PLANE(3)
+                ZCCL_DEC_PLANE(2) ZCCL_DEC_PLANE(1) ZCCL_DEC_PLANE(0)
+                    if (pw[0] & lanebit) mag = -mag;
+                default: break;
+            }
+            wbuf[32 * i + (lane ^ (u << 2))] = mag;
+        }
+    }
+}
+
+// Reads this thread's 16 consecutive deltas (elements 16*lane .. 16*lane+15 of the warp's 512) from `wbuf`,
+// forms their running sum and the warp-wide exclusive prefix.  On return v[k] = sum of the warp's deltas up to
+// and including this thread's element k; the return value is the warp's total.
+__device__ __forceinline__ float decode_scan_f32(const float* __restrict__ wbuf, int lane, float (&v)[16])
+{
+    const int sw = (lane >> 1) & 3;
+    const float4* row = reinterpret_cast<const float4*>(wbuf + 16 * lane);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const float4 f = row[c ^ sw];
+        v[4 * c + 0] = f.x; v[4 * c + 1] = f.y; v[4 * c + 2] = f.z; v[4 * c + 3] = f.w;
+    }
+    float run = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) { run = __fadd_rn(run, v[k]); v[k] = run; }
+    float incl = run;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+        const float t = __shfl_up_sync(kFull, incl, s);
+        if (lane >= s) incl = __fadd_rn(incl, t);
+    }
+    const float excl = __fsub_rn(incl, run);
+    const float total = __shfl_sync(kFull, incl, 31);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = __fadd_rn(v[k], excl);
+    return total;
+}
+
+// Writes the (offset, code length) table of this warp's 16 blocks from the lanes that hold them.
+__device__ __forceinline__ void write_block_table(const TileDesc& d, uint32_t* __restrict__ tbl, int warp, int lane)
+{
+    if ((lane >> 2) == warp) {
+        const int k = 4 * (lane & 3);
+        uint4 e;
+        e.x = (d.o0 << 8) | (d.lw & 0xFF);
+        e.y = (d.o1 << 8) | ((d.lw >> 8) & 0xFF);
+        e.z = (d.o2 << 8) | ((d.lw >> 16) & 0xFF);
+        e.w = (d.o3 << 8) | (d.lw >> 24);
+        *reinterpret_cast<uint4*>(tbl + k) = e;
+    }
+}
+
+struct DecodeShared {
+    alignas(16) uint32_t blob[kBlobStageWords];
+    alignas(16) float wbuf[kWarps][kBlocksPerWarp * kBlock];
+    alignas(16) uint32_t tbl[kWarps][kBlocksPerWarp];
+    float warp_total[2][kWarps];
+    int32_t warp_total_i[kWarps];
+    alignas(8) unsigned long long bar;
 };
 
-template <int MODE>
-__global__ void __launch_bounds__(kThreads, 3) encode_kernel(JobBatch jb, Workspace ws, Params hp, int use_dev_params)
+__global__ void __launch_bounds__(kThreads, 4) decode_kernel(JobBatch jb, Workspace ws)
 {
-    __shared__ EncodeShared sh;
+    __shared__ DecodeShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
     uint32_t status = 0;
+    uint32_t fills = 0;    // bulk copies completed on sh.bar (its phase parity)
+    uint32_t par = 0;      // parity of the warp_total double buffer
+    if (tid == 0) {
+        mbar_init(&sh.bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
 
-    Params prm = hp;
-    if (MODE == kEncodeRaw && use_dev_params) prm = *ws.params;
-
-    for (;;) {
-        __syncthreads();
-        if (tid == 0) sh.ticket = atomicAdd(ws.ticket, 1u);
-        __syncthreads();
-        const uint32_t ticket = sh.ticket;
-        if (ticket >= jb.total_tiles) break;
-        int j = 0;
-#pragma unroll 1
-        for (int k = 1; k < jb.count; ++k) if (jb.job[k].tile_begin <= ticket) j = k;
+    int cur_job = -1;
+    StreamInfo h;
+    h.ok = false; h.n = 0; h.nT = 0; h.s = 1.0f; h.eb_abs = 0.0f;
+    for (uint32_t g = blockIdx.x; g < jb.total_tiles; g += gridDim.x) {
+        const int j = find_job(jb, g);
         const Job& job = jb.job[j];
-        const uint32_t tile = ticket - job.tile_begin;
-        const unsigned long long n = job.n;
-        const uint32_t nT = (uint32_t)((n + kTile - 1) / kTile);
-        unsigned long long* my_state = ws.tile_state + ticket;
+        if (j != cur_job) { h = read_header(job.in_c, job.in_cap); cur_job = j; }
+        const uint32_t tile = g - job.tile_begin;
+        if (!h.ok) { status |= kStBadStream; continue; }
+        if (h.n > job.n) { status |= kStCapacity; continue; }
+        if (tile >= h.nT) continue;
+        const TileDesc d = describe_tile(job.in_c, job.in_cap, h, tile, lane);
+        if (!d.ok) { status |= kStBadStream; continue; }
+        float* __restrict__ y = job.y + (unsigned long long)tile * kTile;
 
-        bool tile_ok = true;
-        float s = prm.s, r = prm.r, eb_abs = prm.eb_abs;
-        StreamInfo h1, h2;
-        if (MODE == kEncodeFused) {
-            h1 = read_header(job.in_c, job.in_cap);
-            tile_ok = h1.ok && h1.n == n;
-            if (job.in_c2) {
-                h2 = read_header(job.in_c2, job.in2_cap);
-                tile_ok = tile_ok && h2.ok && h2.n == n && __float_as_uint(h2.s) == __float_as_uint(h1.s);
-            }
-            s = h1.s; eb_abs = h1.eb_abs;
-            r = __fdiv_rn(1.0f, s);
-            if (!tile_ok) status |= kStBadStream;
-        } else {
-            tile_ok = prm.valid != 0;
-        }
-
-        // a job with no elements still owns one ticket: it writes the header and the length
-        if (n == 0 || !tile_ok) {
+        if (d.fast) {
+            // stage the blob: the 16-byte aligned cover of [blob, blob + words)
+            const uintptr_t a_beg = (uintptr_t)d.blob & ~(uintptr_t)15;
+            const uintptr_t a_end = ((uintptr_t)(d.blob + d.words) + 15) & ~(uintptr_t)15;
+            const uint32_t shift = (uint32_t)(((uintptr_t)d.blob - a_beg) >> 2);
+            __syncthreads();   // the previous tile's readers of sh.blob are done
             if (tid == 0) {
-                st_state(my_state, pack_state(epoch, 1u, 0u));
-                if (tile == 0) {
-                    if (tile_ok && job.out_cap >= (unsigned)kHeaderBytes) {
-                        uint32_t* o = job.out;
-                        o[0] = kMagic; o[1] = kVersion; o[2] = 0; o[3] = 0;
-                        o[4] = __float_as_uint(eb_abs); o[5] = __float_as_uint(s); o[6] = kTile; o[7] = 0;
-                        *job.out_bytes = kHeaderBytes;
-                    } else {
-                        *job.out_bytes = 0;
-                    }
-                }
+                mbar_expect_tx(&sh.bar, (uint32_t)(a_end - a_beg));
+                bulk_load(sh.blob, (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar);
             }
-            continue;
-        }
-
-        const unsigned long long start = (unsigned long long)tile * kTile;
-        const uint32_t len = (uint32_t)((n - start < (unsigned long long)kTile) ? (n - start) : kTile);
-        const uint32_t nb = (len + kBlock - 1) / kBlock;
-        const uint32_t padw = (nb + 3) >> 2;
-        const unsigned long long last = n - 1;
-
-        // ---- values of this warp's 16 blocks, one element per lane; lanes past the end repeat the last element
-        float v[kBlocksPerWarp];
-        const unsigned long long e0 = start + (unsigned)(warp * kBlocksPerWarp * kBlock + lane);
-        if (MODE == kEncodeRaw) {
-            const float* __restrict__ x = job.x;
+            write_block_table(d, sh.tbl[warp], warp, lane);
+            __syncwarp();
+            const bool landed = mbar_wait(&sh.bar, fills & 1u);
+            ++fills;
+            if (!landed) status |= kStTimeout;   // carry on with whatever is staged: reads stay inside shared memory
+            decode_blocks_f32(sh.blob + shift + 1 + d.padw, sh.tbl[warp], sh.wbuf[warp], lane);
+            __syncwarp();
+            float v[16];
+            const float total = decode_scan_f32(sh.wbuf[warp], lane, v);
+            if (lane == 0) sh.warp_total[par][warp] = total;
+            __syncthreads();
+            float base = (float)d.outlier;
+            for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[par][w]);
+            par ^= 1u;
+            float4* dst = reinterpret_cast<float4*>(y + 512 * warp + 16 * lane);
+            const bool vec = (((uintptr_t)dst) & 15u) == 0;
 #pragma unroll
-            for (int i = 0; i < kBlocksPerWarp; ++i) {
-                unsigned long long e = e0 + (unsigned)(i * kBlock);
-                v[i] = __ldg(x + (e < last ? e : last));
+            for (int c = 0; c < 4; ++c) {
+                float4 o;
+                o.x = __fmul_rn(__fadd_rn(v[4 * c + 0], base), h.s);
+                o.y = __fmul_rn(__fadd_rn(v[4 * c + 1], base), h.s);
+                o.z = __fmul_rn(__fadd_rn(v[4 * c + 2], base), h.s);
+                o.w = __fmul_rn(__fadd_rn(v[4 * c + 3], base), h.s);
+                if (vec) dst[c] = o;
+                else {
+                    float* ds = reinterpret_cast<float*>(dst + c);
+                    ds[0] = o.x; ds[1] = o.y; ds[2] = o.z; ds[3] = o.w;
+                }
             }
         } else {
-            int32_t qa[kBlocksPerWarp], oa = 0;
-            bool ok = decode_tile_warp(job.in_c, job.in_cap, h1, tile, warp, lane, qa, oa);
-            int32_t qb[kBlocksPerWarp], ob = 0;
-            if (job.in_c2) ok = decode_tile_warp(job.in_c2, job.in2_cap, h2, tile, warp, lane, qb, ob) && ok;
-            if (lane == 31) {
-                sh.warp_sum[0][warp] = qa[kBlocksPerWarp - 1];
-                if (job.in_c2) sh.warp_sum[1][warp] = qb[kBlocksPerWarp - 1];
-            }
+            int32_t q[kBlocksPerWarp];
+            decode_blocks_int(d, warp, lane, q);
             __syncthreads();
-            if (!ok) {   // uniform over the CTA
-                status |= kStBadStream;
-                // keep the scan consistent for the tiles that follow: publish an empty tile, write nothing
-                if (tid == 0) st_state(my_state, pack_state(epoch, tile == 0 ? 1u : 0u, 0u));
-                if (tid == 0 && tile == nT - 1) *job.out_bytes = 0;
-                continue;
-            }
-            int32_t base_a = oa, base_b = ob;
-            for (int w = 0; w < warp; ++w) { base_a += sh.warp_sum[0][w]; if (job.in_c2) base_b += sh.warp_sum[1][w]; }
-            const float* __restrict__ loc = job.x;
+            if (lane == 31) sh.warp_total_i[warp] = q[kBlocksPerWarp - 1];
+            __syncthreads();
+            int32_t base = d.outlier;
+            for (int w = 0; w < warp; ++w) base += sh.warp_total_i[w];
+            const uint32_t e0 = (uint32_t)(warp * kBlocksPerWarp * kBlock + lane);
 #pragma unroll
             for (int i = 0; i < kBlocksPerWarp; ++i) {
-                unsigned long long e = e0 + (unsigned)(i * kBlock);
-                if (e > last) e = last;
-                const float xa = __fmul_rn(__int2float_rn(base_a + qa[i]), s);
-                float xb;
-                if (job.in_c2) xb = __fmul_rn(__int2float_rn(base_b + qb[i]), s);
-                else xb = __ldg(loc + e);
-                v[i] = __fadd_rn(xa, xb);
+                const uint32_t e = e0 + (uint32_t)(i * kBlock);
+                if (e < d.len) y[e] = __fmul_rn(__int2float_rn(base + q[i]), h.s);
             }
         }
+    }
+    if (status) atomicOr(ws.status, status);
+}
 
-        // ---- quantise (the multiplication), keep the largest |x * r| for the range / precision checks
-        int32_t q[kBlocksPerWarp];
-        float tmax = 0.0f;
+// ================================================================================================ ENCODE SIDE
+
+// Where a warp reads the values it encodes.  cur(g, u) / prev(g, u): element `lane` of the warp's block 4g + u
+// and the element before it (the tile's first element is its own predecessor: its delta is zero by definition).
+struct SrcStaged {          // tile staged in shared memory in element order, with one guard word in front
+    const float* xb;        // &tile[512 * warp + lane]
+    __device__ __forceinline__ float cur(int g, int u) const { return xb[32 * (4 * g + u)]; }
+    __device__ __forceinline__ float prev(int g, int u) const { return xb[32 * (4 * g + u) - 1]; }
+};
+struct SrcGlobal {          // straight from global memory, any alignment, ragged tails repeat the last element
+    const float* x;         // tile start
+    uint32_t e0;            // 512 * warp + lane
+    uint32_t last;          // len - 1
+    __device__ __forceinline__ float cur(int g, int u) const
+    {
+        const uint32_t e = e0 + 32u * (4 * g + u);
+        return __ldg(x + (e < last ? e : last));
+    }
+    __device__ __forceinline__ float prev(int g, int u) const
+    {
+        const uint32_t e = e0 + 32u * (4 * g + u);
+        const uint32_t ep = e ? e - 1 : 0;
+        return __ldg(x + (ep < last ? ep : last));
+    }
+};
+struct SrcSwizzled {        // the fused kernel's sum tile: per-warp region of 17 rows (row 0 = guard row); element j
+    const float* rows;      // of block i lives at rows[32 * (i + 1) + (j ^ ((i & 3) << 2))]
+    int co[4];              // lane's word within a row of block 4g + u
+    int po[4];              // predecessor's word relative to the same row (lane 0: last element of the row before)
+    __device__ __forceinline__ SrcSwizzled(const float* r, int lane) : rows(r)
+    {
 #pragma unroll
-        for (int i = 0; i < kBlocksPerWarp; ++i) {
-            const float t = __fmul_rn(v[i], r);
-            tmax = fmaxf(tmax, fabsf(t));
-            q[i] = __float2int_rn(t);
+        for (int u = 0; u < 4; ++u) {
+            co[u] = lane ^ (u << 2);
+            po[u] = lane ? ((lane - 1) ^ (u << 2)) : (-32 + (31 ^ (((u + 3) & 3) << 2)));
         }
-        if (!(tmax < 1073741824.0f)) status |= kStRange;
-        else if (tmax > 32768.5f) status |= kStPrecision;
+    }
+    __device__ __forceinline__ float cur(int g, int u) const { return rows[32 * (4 * g + u + 1) + co[u]]; }
+    __device__ __forceinline__ float prev(int g, int u) const { return rows[32 * (4 * g + u + 1) + po[u]]; }
+};
 
-        if (MODE == kEncodeFused && job.y != nullptr) {   // uncompressed copy of the sum for the chunk's owner
-            float* __restrict__ y = job.y;
-            const bool deq = (job.flags & 1u) != 0;
-#pragma unroll
-            for (int i = 0; i < kBlocksPerWarp; ++i) {
-                unsigned long long e = e0 + (unsigned)(i * kBlock);
-                if (e <= last) y[e] = deq ? __fmul_rn(__int2float_rn(q[i]), s) : v[i];
-            }
-        }
-
-        if (lane == 31) sh.warp_lastq[warp] = q[kBlocksPerWarp - 1];
-        __syncthreads();
-
-        // ---- 1-D Lorenzo deltas, code lengths
-        uint32_t mag[kBlocksPerWarp];
-        uint32_t sgn[kBlocksPerWarp];
-        uint32_t Ls[kBlocksPerWarp];
-        int32_t prev_last = (warp == 0) ? __shfl_sync(kFull, q[0], 0) : sh.warp_lastq[warp - 1];
-#pragma unroll
-        for (int i = 0; i < kBlocksPerWarp; ++i) {
-            const int32_t src = (lane == 31) ? prev_last : q[i];
-            const int32_t prev = __shfl_sync(kFull, src, (lane + 31) & 31);
-            const int32_t d = q[i] - prev;
-            prev_last = q[i];     // only lane 31's copy is consumed by the next block
-            const uint32_t a = (uint32_t)(d < 0 ? -d : d);
-            const uint32_t m = __reduce_or_sync(kFull, a);
-            uint32_t L = 32u - (uint32_t)__clz((int)m);
-            L = L > 31u ? 31u : L;
-            mag[i] = a;
-            sgn[i] = __ballot_sync(kFull, d < 0);
-            Ls[i] = L;
-        }
-
-        // ---- sizes: serial exclusive scan over this warp's 16 blocks (uniform), then across warps
-        uint32_t off[kBlocksPerWarp];
-        uint32_t wsum = 0;
-#pragma unroll
-        for (int i = 0; i < kBlocksPerWarp; ++i) { off[i] = wsum; wsum += Ls[i] ? Ls[i] + 1 : 0; }
-        if (lane == 0) sh.warp_words[warp] = wsum;
-        // code-length bytes of this warp's blocks: 4 words of the code-length area
-        if (lane < 4) {
-            uint32_t wv = 0;
-#pragma unroll
-            for (int i = 0; i < kBlocksPerWarp; ++i)
-                if ((i >> 2) == lane) wv |= Ls[i] << (8 * (i & 3));
-            const uint32_t widx = 4 * warp + lane;
-            if (widx < padw) sh.stage[1 + widx] = wv;
-        }
-        if (tid == 0) sh.stage[0] = (uint32_t)q[0];   // the outlier
-        __syncthreads();
-        uint32_t wbase = 1 + padw, total = 1 + padw;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const uint32_t ww = sh.warp_words[w];
-            if (w < warp) wbase += ww;
-            total += ww;
-        }
-        if (tid == 0) st_state(my_state, pack_state(epoch, tile == 0 ? 1u : 0u, total));
-
-        // ---- fixed-length encoding: sign word and one ballot per bit plane into the staged blob
-#pragma unroll
-        for (int i = 0; i < kBlocksPerWarp; ++i) {
-            const uint32_t L = Ls[i];
-            if (L) {   // uniform over the warp
-                uint32_t* dst = sh.stage + wbase + off[i];
-                uint32_t mine = sgn[i];
-                for (uint32_t k = 0; k < L; ++k) {
-                    const uint32_t plane = __ballot_sync(kFull, (mag[i] >> k) & 1u);
-                    if ((uint32_t)lane == k + 1) mine = plane;
-                }
-                if ((uint32_t)lane <= L) dst[lane] = mine;
-            }
-        }
-
-        // ---- placement: decoupled look-back over the preceding tiles of this job (warp 0)
-        if (warp == 0) {
-            uint32_t excl = 0, skip = 0;
-            if (tile != 0) {
-                long long pos = (long long)ticket - 1;
-                const long long lo = (long long)job.tile_begin;
-                int budget = kSpinLimit;
-                for (;;) {
-                    const long long at = pos - lane;
-                    unsigned long long st = pack_state(epoch, 1u, 0u);   // before the job's first tile: prefix 0
-                    if (at >= lo) st = ld_state(ws.tile_state + at);
-                    const bool valid = (uint32_t)(st >> 33) == epoch;
-                    const uint32_t vmask = __ballot_sync(kFull, valid);
-                    const uint32_t imask = __ballot_sync(kFull, valid && ((st >> 32) & 1ull));
-                    const int first = imask ? (__ffs((int)imask) - 1) : 31;
-                    const uint32_t need = (first == 31) ? kFull : ((2u << first) - 1u);
-                    if ((vmask & need) != need) {
-                        if (--budget == 0) { skip = 1; status |= kStTimeout; break; }
-                        __nanosleep(64);
-                        continue;
-                    }
-                    const uint32_t contrib = (lane <= first) ? (uint32_t)st : 0u;
-                    excl += __reduce_add_sync(kFull, contrib);
-                    if (imask) break;
-                    pos -= 32;
-                }
-                if (lane == 0) st_state(my_state, pack_state(epoch, 1u, excl + total));
-            }
-            if (lane == 0) { sh.excl = excl; sh.skip = skip; }
-        }
-        __syncthreads();
-
-        // ---- copy the staged blob to its place; index entry; header and length
-        const uint32_t excl = sh.excl;
-        const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
-        const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
-        if (!fits) status |= kStCapacity;
-        if (fits && !sh.skip) {
-            uint32_t* __restrict__ o = job.out + blob_word0;
-            for (uint32_t i = tid; i < total; i += kThreads) o[i] = sh.stage[i];
-            if (tid == 0) job.out[kHeaderWords + tile] = excl + total;
-        }
-        if (tile == 0 && tid < kHeaderWords) {
-            uint32_t hv;
-            switch (tid) {
-                case 0: hv = kMagic; break;
-                case 1: hv = kVersion; break;
-                case 2: hv = (uint32_t)n; break;
-                case 3: hv = (uint32_t)(n >> 32); break;
-                case 4: hv = __float_as_uint(eb_abs); break;
-                case 5: hv = __float_as_uint(s); break;
-                case 6: hv = kTile; break;
-                default: hv = nT; break;
-            }
-            job.out[tid] = hv;
-        }
-        if (tile == nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
+#define ZCCL_ENC_PLANE(k)                                                    \
+    case (k) + 1: {                                                          \
+        const uint32_t p_ = __ballot_sync(kFull, ab & (1u << (k)));          \
+        if (lane == 0) slot[(k) + 1] = p_;                                   \
     }
 
-    if (status) atomicOr(ws.status, status);
+// One pass over this warp's 16 blocks: quantise, 1-D Lorenzo delta, code length, sign word and bit planes into the
+// block's fixed slot.  Returns the warp's payload size in words; lane g (g < 4) ends up holding the code-length
+// word of blocks 4g..4g+3 in `my_lw`.  FAST: fp32 arithmetic, valid while every |x * r| < 2^21.5; the caller
+// checks `guard` (sum of squares of x * r) and reruns with FAST = false when it is too large.
+template <bool FAST, class Src>
+__device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint32_t* __restrict__ slots_w, int lane,
+                                                  uint32_t& my_lw, int32_t& q_first, float& guard, float& tmax)
+{
+    uint32_t wsum = 0;
+    float acc = 0.0f, tm = 0.0f;
+    my_lw = 0;
+#pragma unroll 1
+    for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
+        uint32_t lword = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float xv = src.cur(g, u), pv = src.prev(g, u);
+            const float t = __fmul_rn(xv, r), tp = __fmul_rn(pv, r);
+            uint32_t ab, sg, L;
+            if (FAST) {
+                acc = __fmaf_rn(t, t, acc);
+                acc = __fmaf_rn(tp, tp, acc);
+                const float c = __fadd_rn(t, kRoundMagic), cp = __fadd_rn(tp, kRoundMagic);
+                const float df = __fsub_rn(c, cp);
+                if (u == 0 && g == 0) q_first = (int32_t)(__float_as_uint(c) - kRoundMagicBits);
+                ab = __float_as_uint(__fadd_rn(fabsf(df), kTwo23));
+                const uint32_t m = __reduce_or_sync(kFull, ab) & 0x7FFFFFu;
+                L = 32u - (uint32_t)__clz((int)m);
+                sg = __ballot_sync(kFull, df < 0.0f);
+            } else {
+                tm = fmaxf(tm, fabsf(t));
+                const int32_t q = __float2int_rn(t), qp = __float2int_rn(tp);
+                const int32_t dd = q - qp;
+                if (u == 0 && g == 0) q_first = q;
+                ab = (uint32_t)(dd < 0 ? -dd : dd);
+                const uint32_t m = __reduce_or_sync(kFull, ab);
+                L = 32u - (uint32_t)__clz((int)m);
+                sg = __ballot_sync(kFull, dd < 0);
+            }
+            uint32_t* slot = slots_w + kSlotWords * (4 * g + u);
+            if (L) {   // uniform over the warp
+                if (lane == 0) slot[0] = sg;
+                switch (L) {
+                    default:
+                        if (!FAST) {
+                            for (uint32_t k = L - 1; k >= 23; --k) {
+                                const uint32_t p_ = __ballot_sync(kFull, ab & (1u << k));
+                                if (lane == 0) slot[k + 1] = p_;
+                            }
+                        }
+                    ZCCL_ENC_PLANE(22) ZCCL_ENC_PLANE(21) ZCCL_ENC_PLANE(20) ZCCL_ENC_PLANE(19) ZCCL_ENC_PLANE(18)
+                    ZCCL_ENC_PLANE(17) ZCCL_ENC_PLANE(16) ZCCL_ENC_PLANE(15) ZCCL_ENC_PLANE(14) ZCCL_ENC_PLANE(13)
+                    ZCCL_ENC_PLANE(12) ZCCL_ENC_PLANE(11) ZCCL_ENC_PLANE(10) ZCCL_ENC_PLANE(9) ZCCL_ENC_PLANE(8)
+                    ZCCL_ENC_PLANE(7) ZCCL_ENC_PLANE(6) ZCCL_ENC_PLANE(5) ZCCL_ENC_PLANE(4) ZCCL_ENC_PLANE(3)
+                    ZCCL_ENC_PLANE(2) ZCCL_ENC_PLANE(1) ZCCL_ENC_PLANE(0)
+                    break;
+                }
+                wsum += L + 1;
+            }
+            lword |= L << (8 * u);
+        }
+        if (lane == g) my_lw = lword;
+    }
+    guard = acc;
+    tmax = tm;
+    return wsum;
+}
+
+struct EncodeShared {
+    alignas(16) float xbuf[2][kTile + 8];                       // double-buffered input tiles (+ guard word)
+    alignas(16) uint32_t slots[kBlocksPerTile * kSlotWords];    // one fixed slot per block
+    uint32_t warp_words[kWarps];
+    uint32_t ticket[2];
+    uint32_t excl;
+    uint32_t skip;
+    alignas(8) unsigned long long bar[2];
+};
+
+struct FusedShared {
+    alignas(16) uint32_t blob[kBlobStageWords];
+    alignas(16) float ybuf[kWarps][(kBlocksPerWarp + 1) * kBlock];   // deltas, then sums (row 0 of a warp = guard)
+    alignas(16) uint32_t tbl[kWarps][kBlocksPerWarp];
+    alignas(16) uint32_t slots[kBlocksPerTile * kSlotWords];
+    float warp_total[kWarps];
+    int32_t warp_total_i[kWarps];
+    int32_t warp_total_i2[kWarps];
+    uint32_t warp_words[kWarps];
+    uint32_t ticket[2];
+    uint32_t excl;
+    uint32_t skip;
+    alignas(8) unsigned long long bar;
+};
+
+// A raw-mode tile can be staged by a bulk copy when it is full and starts on a 16-byte boundary.
+__device__ __forceinline__ bool stageable_raw(const Job& job, uint32_t tile)
+{
+    const unsigned long long start = (unsigned long long)tile * kTile;
+    return job.n - start >= (unsigned long long)kTile && (((uintptr_t)(job.x + start)) & 15u) == 0;
+}
+
+// Placement: decoupled look-back over the preceding tiles of this job, run by warp 0.  Returns the exclusive
+// prefix in words; sets `skip` when the bounded wait expired.
+__device__ __forceinline__ uint32_t look_back(const Workspace& ws, uint32_t ticket, uint32_t tile_begin, uint32_t epoch,
+                                              uint32_t total, int lane, uint32_t& skip, uint32_t& status)
+{
+    uint32_t excl = 0;
+    skip = 0;
+    long long pos = (long long)ticket - 1;
+    const long long lo = (long long)tile_begin;
+    int budget = kSpinLimit;
+    for (;;) {
+        const long long at = pos - lane;
+        unsigned long long st = pack_state(epoch, 1u, 0u);   // before the job's first tile: prefix 0
+        if (at >= lo) st = ld_state(ws.tile_state + at);
+        const bool valid = (uint32_t)(st >> 33) == epoch;
+        const uint32_t vmask = __ballot_sync(kFull, valid);
+        const uint32_t imask = __ballot_sync(kFull, valid && ((st >> 32) & 1ull));
+        const int first = imask ? (__ffs((int)imask) - 1) : 31;
+        const uint32_t need = (first == 31) ? kFull : ((2u << first) - 1u);
+        if ((vmask & need) != need) {
+            if (--budget == 0) { skip = 1; status |= kStTimeout; break; }
+            __nanosleep(40);
+            continue;
+        }
+        const uint32_t contrib = (lane <= first) ? (uint32_t)st : 0u;
+        excl += __reduce_add_sync(kFull, contrib);
+        if (imask) break;
+        pos -= 32;
+    }
+    if (lane == 0) st_state(ws.tile_state + ticket, pack_state(epoch, 1u, excl + total));
+    return excl;
+}
+
+// Copies this warp's blocks from their slots to the stream, compacting them; writes the warp's code-length words.
+__device__ __forceinline__ void copy_out_warp(uint32_t* __restrict__ blob_out, const uint32_t* __restrict__ slots_w,
+                                              uint32_t wbase, uint32_t my_lw, uint32_t padw, int warp, int lane)
+{
+    uint32_t off = wbase;
+#pragma unroll 1
+    for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
+        const uint32_t lword = __shfl_sync(kFull, my_lw, g);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t L = (lword >> (8 * u)) & 0xFF;
+            const uint32_t sz = L ? L + 1 : 0;
+            if ((uint32_t)lane < sz) blob_out[off + lane] = slots_w[kSlotWords * (4 * g + u) + lane];
+            off += sz;
+        }
+    }
+    if (lane < 4 && (uint32_t)(4 * warp + lane) < padw) blob_out[1 + 4 * warp + lane] = my_lw;
+}
+
+__device__ __forceinline__ void write_header(uint32_t* out, int tid, unsigned long long n, float eb_abs, float s, uint32_t nT)
+{
+    if (tid < kHeaderWords) {
+        uint32_t hv;
+        switch (tid) {
+            case 0: hv = kMagic; break;
+            case 1: hv = kVersion; break;
+            case 2: hv = (uint32_t)n; break;
+            case 3: hv = (uint32_t)(n >> 32); break;
+            case 4: hv = __float_as_uint(eb_abs); break;
+            case 5: hv = __float_as_uint(s); break;
+            case 6: hv = kTile; break;
+            default: hv = nT; break;
+        }
+        out[tid] = hv;
+    }
+}
+
+__device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoch, int tid)
+{
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -498,40 +708,397 @@ __global__ void __launch_bounds__(kThreads, 3) encode_kernel(JobBatch jb, Worksp
     }
 }
 
-// ------------------------------------------------------------------------------------------------ decoder
-
-__global__ void __launch_bounds__(kThreads, 3) decode_kernel(JobBatch jb, Workspace ws)
+// Sizes -> placement -> copy-out, shared by both encoders.  Called by all threads after the warp sizes are in
+// shared memory and a barrier has passed.
+template <class Shared>
+__device__ __forceinline__ void place_and_copy(Shared& sh, const Workspace& ws, const Job& job, uint32_t ticket, uint32_t tile,
+                                               uint32_t nT, uint32_t padw, uint32_t epoch, const uint32_t* slots_w,
+                                               uint32_t my_lw, int32_t q_first, float eb_abs, float s, int tid, int warp,
+                                               int lane, uint32_t& status)
 {
-    __shared__ int32_t s_warp_sum[kWarps];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t status = 0;
-    for (uint32_t g = blockIdx.x; g < jb.total_tiles; g += gridDim.x) {
-        int j = 0;
-#pragma unroll 1
-        for (int k = 1; k < jb.count; ++k) if (jb.job[k].tile_begin <= g) j = k;
-        const Job& job = jb.job[j];
-        const uint32_t tile = g - job.tile_begin;
-        const StreamInfo h = read_header(job.in_c, job.in_cap);
-        if (!h.ok) { status |= kStBadStream; continue; }
-        if (h.n > job.n) { status |= kStCapacity; continue; }
-        if (tile >= h.nT) continue;
-        int32_t q[kBlocksPerWarp], outlier = 0;
-        const bool ok = decode_tile_warp(job.in_c, job.in_cap, h, tile, warp, lane, q, outlier);
-        __syncthreads();   // previous iteration's readers of s_warp_sum are done
-        if (lane == 31) s_warp_sum[warp] = q[kBlocksPerWarp - 1];
-        __syncthreads();
-        if (!ok) { status |= kStBadStream; continue; }
-        int32_t base = outlier;
-        for (int w = 0; w < warp; ++w) base += s_warp_sum[w];
-        const unsigned long long e0 = (unsigned long long)tile * kTile + (unsigned)(warp * kBlocksPerWarp * kBlock + lane);
-        float* __restrict__ y = job.y;
+    uint32_t wbase = 1 + padw, total = 1 + padw;
 #pragma unroll
-        for (int i = 0; i < kBlocksPerWarp; ++i) {
-            const unsigned long long e = e0 + (unsigned)(i * kBlock);
-            if (e < h.n) y[e] = __fmul_rn(__int2float_rn(base + q[i]), h.s);
+    for (int w = 0; w < kWarps; ++w) {
+        const uint32_t ww = sh.warp_words[w];
+        if (w < warp) wbase += ww;
+        total += ww;
+    }
+    if (warp == 0) {
+        uint32_t excl = 0, skip = 0;
+        if (tile == 0) {
+            if (lane == 0) st_state(ws.tile_state + ticket, pack_state(epoch, 1u, total));
+        } else {
+            if (lane == 0) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
+            excl = look_back(ws, ticket, job.tile_begin, epoch, total, lane, skip, status);
+        }
+        if (lane == 0) { sh.excl = excl; sh.skip = skip; }
+    }
+    __syncthreads();   // exclusive prefix known
+
+    const uint32_t excl = sh.excl;
+    const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
+    const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
+    if (!fits) status |= kStCapacity;
+    if (fits && !sh.skip) {
+        uint32_t* blob_out = job.out + blob_word0;
+        copy_out_warp(blob_out, slots_w, wbase, my_lw, padw, warp, lane);
+        if (tid == 0) {
+            blob_out[0] = (uint32_t)q_first;
+            job.out[kHeaderWords + tile] = excl + total;
         }
     }
+    if (tile == 0) write_header(job.out, tid, job.n, eb_abs, s, nT);
+    if (tile == nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
+}
+
+// ------------------------------------------------------------------------------------------------ compress
+
+__global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Workspace ws, Params hp, int use_dev_params)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    EncodeShared& sh = *reinterpret_cast<EncodeShared*>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
+    uint32_t status = 0;
+    Params prm = hp;
+    if (use_dev_params) prm = *ws.params;
+    const float r = prm.r, s = prm.s, eb_abs = prm.eb_abs;
+
+    // prologue: first ticket, first bulk copy
+    if (tid == 0) {
+        mbar_init(&sh.bar[0], 1);
+        mbar_init(&sh.bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const uint32_t t0 = atomicAdd(ws.ticket, 1u);
+        sh.ticket[0] = t0;
+        if (t0 < jb.total_tiles && prm.valid) {
+            const Job& j0 = jb.job[find_job(jb, t0)];
+            const uint32_t tile0 = t0 - j0.tile_begin;
+            if (j0.n && stageable_raw(j0, tile0)) {
+                mbar_expect_tx(&sh.bar[0], kTile * 4);
+                bulk_load(&sh.xbuf[0][4], j0.x + (unsigned long long)tile0 * kTile, kTile * 4, &sh.bar[0]);
+            }
+        }
+    }
+    __syncthreads();
+    uint32_t fills0 = 0, fills1 = 0;   // completed bulk copies per buffer (phase parity of its mbarrier)
+    uint32_t p = 0;                    // buffer and ticket slot of the current tile
+    bool pending = false;              // thread 0: a bulk copy for the next tile is in flight
+
+    for (;;) {
+        const uint32_t ticket = sh.ticket[p];
+        if (ticket >= jb.total_tiles) break;
+        const int j = find_job(jb, ticket);
+        const Job& job = jb.job[j];
+        const uint32_t tile = ticket - job.tile_begin;
+        const unsigned long long n = job.n;
+        const uint32_t nT = (uint32_t)((n + kTile - 1) / kTile);
+        const bool staged = prm.valid && n && stageable_raw(job, tile);
+
+        // thread 0: draw the next ticket and start its bulk copy into the other buffer (its last readers
+        // finished before the barrier that ended the previous tile's encoding pass)
+        if (tid == 0) {
+            const uint32_t nt = atomicAdd(ws.ticket, 1u);
+            sh.ticket[p ^ 1u] = nt;
+            pending = false;
+            if (nt < jb.total_tiles && prm.valid) {
+                const Job& jn = jb.job[find_job(jb, nt)];
+                const uint32_t tn = nt - jn.tile_begin;
+                if (jn.n && stageable_raw(jn, tn)) {
+                    mbar_expect_tx(&sh.bar[p ^ 1u], kTile * 4);
+                    bulk_load(&sh.xbuf[p ^ 1u][4], jn.x + (unsigned long long)tn * kTile, kTile * 4, &sh.bar[p ^ 1u]);
+                    pending = true;
+                }
+            }
+        }
+
+        if (n == 0 || !prm.valid) {   // a job without elements still owns one ticket: header and length only
+            const bool hdr = prm.valid && job.out_cap >= (unsigned)kHeaderBytes;
+            if (tid == 0) {
+                st_state(ws.tile_state + ticket, pack_state(epoch, 1u, 0u));
+                if (tile == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
+            }
+            if (hdr && tile == 0) write_header(job.out, tid, 0, eb_abs, s, 0);
+            __syncthreads();
+            p ^= 1u;
+            continue;
+        }
+
+        const unsigned long long start = (unsigned long long)tile * kTile;
+        const uint32_t len = (uint32_t)((n - start < (unsigned long long)kTile) ? (n - start) : kTile);
+        const uint32_t nb = (len + kBlock - 1) / kBlock;
+        const uint32_t padw = (nb + 3) >> 2;
+
+        // ---- single pass over the warp's blocks: quantise, delta, code length, planes -> slots
+        uint32_t* slots_w = sh.slots + kSlotWords * kBlocksPerWarp * warp;
+        uint32_t my_lw = 0, wsum = 0;
+        int32_t q_first = 0;
+        float guard = 0.0f, tmax = 0.0f;
+        bool need_int = !staged;
+        if (staged) {
+            const uint32_t fl = p ? fills1 : fills0;
+            const bool landed = mbar_wait(&sh.bar[p], fl & 1u);
+            if (p) ++fills1; else ++fills0;
+            if (!landed) status |= kStTimeout;   // carry on with whatever is staged: the result is flagged invalid
+            float* xt = &sh.xbuf[p][4];
+            if (tid == 0) xt[-1] = xt[0];    // the tile's first element is its own predecessor
+            const SrcStaged src{xt + 512 * warp + lane};
+            wsum = encode_blocks<true>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+            need_int = __any_sync(kFull, !(guard < kGuardExact));
+            if (!need_int && __any_sync(kFull, guard >= kGuardSmall)) {   // codes beyond 2^15 raise the warning
+                float tm = 0.0f;
+#pragma unroll 1
+                for (int g = 0; g < 4; ++g)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) tm = fmaxf(tm, fabsf(__fmul_rn(src.cur(g, u), r)));
+                if (tm > 32768.5f) status |= kStPrecision;
+            }
+        }
+        if (need_int) {
+            const SrcGlobal src{job.x + start, (uint32_t)(512 * warp + lane), len - 1};
+            wsum = encode_blocks<false>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+            if (!(tmax < 1073741824.0f)) status |= kStRange;
+            else if (tmax > 32768.5f) status |= kStPrecision;
+        }
+        if (lane == 0) sh.warp_words[warp] = wsum;
+        __syncthreads();   // sizes of all warps; the staged tile has been consumed
+        place_and_copy(sh, ws, job, ticket, tile, nT, padw, epoch, slots_w, my_lw, q_first, eb_abs, s, tid, warp, lane, status);
+        p ^= 1u;
+    }
+
+    // never leave with a bulk copy in flight into this CTA's shared memory: every copy that was started has been
+    // waited for by the iteration that consumed it, except after an expired wait; then give it one more bounded wait
+    if (tid == 0 && (pending || (status & kStTimeout))) {
+        (void)mbar_wait(&sh.bar[0], (fills0 + 1u) & 1u);
+        (void)mbar_wait(&sh.bar[1], (fills1 + 1u) & 1u);
+    }
     if (status) atomicOr(ws.status, status);
+    finish_launch(ws, epoch, tid);
+}
+
+// ------------------------------------------------------------------------------------------------ fused hop
+
+// out = compress(decompress(in_c) + local) per tile, with no uncompressed intermediate in global memory.
+__global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, Workspace ws)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    FusedShared& sh = *reinterpret_cast<FusedShared*>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
+    uint32_t status = 0;
+    uint32_t fills = 0;
+    if (tid == 0) {
+        mbar_init(&sh.bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        sh.ticket[0] = atomicAdd(ws.ticket, 1u);
+    }
+    __syncthreads();
+    uint32_t p = 0;
+    int cur_job = -1;
+    StreamInfo h1, h2;
+    h1.ok = h2.ok = false; h1.n = h2.n = 0; h1.nT = h2.nT = 0; h1.s = h2.s = 1.0f; h1.eb_abs = h2.eb_abs = 0.0f;
+    bool job_ok = false;
+
+    for (;;) {
+        const uint32_t ticket = sh.ticket[p];
+        if (ticket >= jb.total_tiles) break;
+        const int j = find_job(jb, ticket);
+        const Job& job = jb.job[j];
+        const uint32_t tile = ticket - job.tile_begin;
+        const unsigned long long n = job.n;
+        const uint32_t nT = (uint32_t)((n + kTile - 1) / kTile);
+        if (j != cur_job) {
+            cur_job = j;
+            h1 = read_header(job.in_c, job.in_cap);
+            job_ok = h1.ok && h1.n == n;
+            if (job.in_c2) {
+                h2 = read_header(job.in_c2, job.in2_cap);
+                job_ok = job_ok && h2.ok && h2.n == n && __float_as_uint(h2.s) == __float_as_uint(h1.s);
+            }
+        }
+        const float s = h1.s, eb_abs = h1.eb_abs;
+        const float r = __fdiv_rn(1.0f, s);
+        if (tid == 0) sh.ticket[p ^ 1u] = atomicAdd(ws.ticket, 1u);
+
+        if (!job_ok || n == 0) {
+            if (!job_ok) status |= kStBadStream;
+            const bool hdr = job_ok && job.out_cap >= (unsigned)kHeaderBytes;
+            if (tid == 0) {
+                st_state(ws.tile_state + ticket, pack_state(epoch, 1u, 0u));
+                if (tile == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
+            }
+            if (hdr && tile == 0) write_header(job.out, tid, 0, eb_abs, s, 0);
+            __syncthreads();
+            p ^= 1u;
+            continue;
+        }
+
+        const unsigned long long start = (unsigned long long)tile * kTile;
+        const uint32_t len = (uint32_t)((n - start < (unsigned long long)kTile) ? (n - start) : kTile);
+        const uint32_t nb = (len + kBlock - 1) / kBlock;
+        const uint32_t padw = (nb + 3) >> 2;
+        const uint32_t last = len - 1;
+
+        const TileDesc d1 = describe_tile(job.in_c, job.in_cap, h1, tile, lane);
+        TileDesc d2 = d1;
+        if (job.in_c2) d2 = describe_tile(job.in_c2, job.in2_cap, h2, tile, lane);
+        if (!d1.ok || !d2.ok) {   // uniform: keep the scan consistent for the tiles that follow, write nothing
+            status |= kStBadStream;
+            if (tid == 0) {
+                st_state(ws.tile_state + ticket, pack_state(epoch, tile == 0 ? 1u : 0u, 0u));
+                if (tile == nT - 1) *job.out_bytes = 0;
+            }
+            __syncthreads();
+            p ^= 1u;
+            continue;
+        }
+
+        // ---- front end: decode + add, leaving the sums in this warp's rows of ybuf (swizzled), row 0 = guard
+        float* yrows = sh.ybuf[warp];
+        const float* __restrict__ loc = job.x ? job.x + start : nullptr;
+        float* __restrict__ yout = job.y ? job.y + start : nullptr;
+        const bool deq = (job.flags & 1u) != 0;
+        const bool fast_front = d1.fast && !job.in_c2;
+        if (fast_front) {
+            const uintptr_t a_beg = (uintptr_t)d1.blob & ~(uintptr_t)15;
+            const uintptr_t a_end = ((uintptr_t)(d1.blob + d1.words) + 15) & ~(uintptr_t)15;
+            const uint32_t shift = (uint32_t)(((uintptr_t)d1.blob - a_beg) >> 2);
+            if (tid == 0) {   // sh.blob's previous readers finished before the last barrier of the previous tile
+                mbar_expect_tx(&sh.bar, (uint32_t)(a_end - a_beg));
+                bulk_load(sh.blob, (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar);
+            }
+            // this thread's 16 consecutive elements of the local operand (128-bit loads when aligned)
+            float lv[16];
+            {
+                const float* lp = loc + 512 * warp + 16 * lane;
+                if ((((uintptr_t)lp) & 15u) == 0) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const float4 f = __ldg(reinterpret_cast<const float4*>(lp) + c);
+                        lv[4 * c] = f.x; lv[4 * c + 1] = f.y; lv[4 * c + 2] = f.z; lv[4 * c + 3] = f.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) lv[k] = __ldg(lp + k);
+                }
+            }
+            write_block_table(d1, sh.tbl[warp], warp, lane);
+            __syncwarp();
+            const bool landed = mbar_wait(&sh.bar, fills & 1u);
+            ++fills;
+            if (!landed) status |= kStTimeout;
+            decode_blocks_f32(sh.blob + shift + 1 + d1.padw, sh.tbl[warp], yrows + 32, lane);
+            __syncwarp();
+            float v[16];
+            const float total = decode_scan_f32(yrows + 32, lane, v);
+            if (lane == 0) sh.warp_total[warp] = total;
+            __syncthreads();   // warp totals
+            float base = (float)d1.outlier;
+            for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[w]);
+            // the element before this warp's first one is the last element of the previous warp: its code is `base`
+            if (lane == 0) {
+                float yprev;
+                if (warp == 0) yprev = __fadd_rn(__fmul_rn(__fadd_rn(v[0], base), s), lv[0]);
+                else yprev = __fadd_rn(__fmul_rn(base, s), __ldg(loc + 512 * warp - 1));
+                yrows[31 ^ 12] = yprev;   // guard row, element 31 under the swizzle of the row before row 0
+            }
+            const int sw = (lane >> 1) & 3;
+            float4* row = reinterpret_cast<float4*>(yrows + 32 + 16 * lane);
+            float4* gout = yout ? reinterpret_cast<float4*>(yout + 512 * warp + 16 * lane) : nullptr;
+            const bool gvec = (((uintptr_t)gout) & 15u) == 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float4 o;
+                o.x = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), lv[4 * c + 0]);
+                o.y = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), lv[4 * c + 1]);
+                o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), lv[4 * c + 2]);
+                o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), lv[4 * c + 3]);
+                row[c ^ sw] = o;
+                if (gout && !deq) {
+                    if (gvec) gout[c] = o;
+                    else { float* g = reinterpret_cast<float*>(gout + c); g[0] = o.x; g[1] = o.y; g[2] = o.z; g[3] = o.w; }
+                }
+            }
+            __syncwarp();
+        } else {
+            // integer front end, one element per lane; ragged tails repeat the last element
+            int32_t qa[kBlocksPerWarp], qb[kBlocksPerWarp];
+            decode_blocks_int(d1, warp, lane, qa);
+            if (job.in_c2) decode_blocks_int(d2, warp, lane, qb);
+            if (lane == 31) {
+                sh.warp_total_i[warp] = qa[kBlocksPerWarp - 1];
+                if (job.in_c2) sh.warp_total_i2[warp] = qb[kBlocksPerWarp - 1];
+            }
+            __syncthreads();   // warp totals
+            int32_t base_a = d1.outlier, base_b = d2.outlier;
+            for (int w = 0; w < warp; ++w) {
+                base_a += sh.warp_total_i[w];
+                if (job.in_c2) base_b += sh.warp_total_i2[w];
+            }
+            const uint32_t e0 = (uint32_t)(512 * warp + lane);
+#pragma unroll
+            for (int i = 0; i < kBlocksPerWarp; ++i) {
+                uint32_t e = e0 + 32u * i;
+                const bool inside = e <= last;
+                if (!inside) e = last;
+                const float xa = __fmul_rn(__int2float_rn(base_a + qa[i]), s);
+                const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b + qb[i]), s) : __ldg(loc + e);
+                const float yv = __fadd_rn(xa, xb);
+                yrows[32 * (i + 1) + (lane ^ ((i & 3) << 2))] = yv;
+                if (yout && !deq && inside) yout[e] = yv;
+            }
+            if (lane == 0) {
+                float yprev;
+                if (warp == 0) {
+                    yprev = yrows[32];   // own first element (row 1, lane 0, swizzle 0)
+                } else {
+                    const uint32_t ep = min((uint32_t)(512 * warp - 1), last);
+                    const float xa = __fmul_rn(__int2float_rn(base_a), s);
+                    const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b), s) : __ldg(loc + ep);
+                    yprev = __fadd_rn(xa, xb);
+                }
+                yrows[31 ^ 12] = yprev;
+            }
+            __syncwarp();
+        }
+
+        // ---- back end: encode the sums
+        uint32_t* slots_w = sh.slots + kSlotWords * kBlocksPerWarp * warp;
+        uint32_t my_lw = 0, wsum = 0;
+        int32_t q_first = 0;
+        float guard = 0.0f, tmax = 0.0f;
+        const SrcSwizzled src(yrows, lane);
+        wsum = encode_blocks<true>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+        const bool need_int = __any_sync(kFull, !(guard < kGuardExact));
+        if (need_int) {
+            wsum = encode_blocks<false>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+            if (!(tmax < 1073741824.0f)) status |= kStRange;
+            else if (tmax > 32768.5f) status |= kStPrecision;
+        } else if (__any_sync(kFull, guard >= kGuardSmall)) {
+            float tm = 0.0f;
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) tm = fmaxf(tm, fabsf(__fmul_rn(src.cur(g, u), r)));
+            if (tm > 32768.5f) status |= kStPrecision;
+        }
+        if (yout && deq) {   // owner's copy as the dequantised value float(q(y)) * s
+            const uint32_t e0 = (uint32_t)(512 * warp + lane);
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t e = e0 + 32u * (4 * g + u);
+                    if (e <= last) yout[e] = __fmul_rn(__int2float_rn(__float2int_rn(__fmul_rn(src.cur(g, u), r))), s);
+                }
+        }
+        if (lane == 0) sh.warp_words[warp] = wsum;
+        __syncthreads();   // sizes of all warps
+        place_and_copy(sh, ws, job, ticket, tile, nT, padw, epoch, slots_w, my_lw, q_first, eb_abs, s, tid, warp, lane, status);
+        p ^= 1u;
+    }
+    if (status) atomicOr(ws.status, status);
+    finish_launch(ws, epoch, tid);
 }
 
 // ------------------------------------------------------------------------------------------------ blob copy
@@ -561,7 +1128,7 @@ __global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
     if (tid == 0 && job.bytes_out) *job.bytes_out = (size_t)bytes;
 }
 
-int g_encode_ctas_per_sm = 0, g_decode_ctas_per_sm = 0;
+int g_raw_ctas_per_sm = 0, g_fused_ctas_per_sm = 0, g_decode_ctas_per_sm = 0;
 unsigned long long g_launches = 0;   // kernels launched by this library in this process
 
 }  // namespace
@@ -594,19 +1161,26 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
                           Params host_params, int sm_count, cudaStream_t st)
 {
     if (jb.total_tiles == 0) return cudaSuccess;
-    if (g_encode_ctas_per_sm == 0) {
+    if (g_raw_ctas_per_sm == 0) {
+        cudaError_t e = cudaFuncSetAttribute(encode_raw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)sizeof(EncodeShared));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(encode_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FusedShared));
+        if (e != cudaSuccess) return e;
         int a = 0, b = 0;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_kernel<kEncodeRaw>, kThreads, 0);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, encode_kernel<kEncodeFused>, kThreads, 0);
-        g_encode_ctas_per_sm = (a < b ? a : b) > 0 ? (a < b ? a : b) : 1;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_raw_kernel, kThreads, sizeof(EncodeShared));
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, encode_fused_kernel, kThreads, sizeof(FusedShared));
+        g_raw_ctas_per_sm = a > 0 ? a : 1;
+        g_fused_ctas_per_sm = b > 0 ? b : 1;
     }
-    unsigned long long cap = (unsigned long long)sm_count * g_encode_ctas_per_sm;
+    const int per_sm = mode == kEncodeRaw ? g_raw_ctas_per_sm : g_fused_ctas_per_sm;
+    unsigned long long cap = (unsigned long long)sm_count * per_sm;
     unsigned grid = (unsigned)(jb.total_tiles < cap ? jb.total_tiles : cap);
     ++g_launches;
     if (mode == kEncodeRaw)
-        encode_kernel<kEncodeRaw><<<grid, kThreads, 0, st>>>(jb, ws, host_params, device_params ? 1 : 0);
+        encode_raw_kernel<<<grid, kThreads, sizeof(EncodeShared), st>>>(jb, ws, host_params, device_params ? 1 : 0);
     else
-        encode_kernel<kEncodeFused><<<grid, kThreads, 0, st>>>(jb, ws, host_params, 0);
+        encode_fused_kernel<<<grid, kThreads, sizeof(FusedShared), st>>>(jb, ws);
     return cudaGetLastError();
 }
 
