@@ -38,7 +38,8 @@ def build(force: bool = False, verbose: bool = False, extra: list[str] | None = 
     if not force and not needs_build():
         return LIB
     tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-    cmd = [nvcc(), *NVCC_FLAGS, *(extra or []), "-o", str(tmp), *map(str, SOURCES)]
+    extra = list(extra or []) + os.environ.get("ZCCL_NVCC_EXTRA", "").split()
+    cmd = [nvcc(), *NVCC_FLAGS, *extra, "-o", str(tmp), *map(str, SOURCES)]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

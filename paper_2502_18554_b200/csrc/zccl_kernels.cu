@@ -15,8 +15,11 @@
 //   * the encoder writes each block's words to a fixed slot and compacts while copying out, so quantisation and
 //     encoding are a single pass over a block; the decoder undoes the Lorenzo recurrence by a warp-local
 //     transposition through shared memory (16 consecutive elements per thread) instead of shuffle scans.
-// Tiles are handed out by an atomic ticket, so a tile's predecessors in the placement scan (decoupled look-back
-// over tile sizes) have always started before it.  Every wait is bounded and reports through the status word.
+// Tiles are dealt round-robin to a grid that fits the device (CTA c takes tiles c, c + G, ...), so all CTAs move
+// through the stream in step, the next tile is known in advance (its bulk copy overlaps the current tile) and a
+// tile's predecessors in the placement scan (decoupled look-back over tile sizes) are at most one round behind.
+// The scan relies on the grid being resident at once; every wait is bounded and reports through the status word
+// instead of hanging if it is not.
 #include "zccl_internal.h"
 
 namespace zccl {
@@ -96,6 +99,39 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// Ballot of (v & mask) != 0 over the warp: one logic op with predicate output feeding the vote.
+__device__ __forceinline__ uint32_t ballot_and(uint32_t v, uint32_t mask)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b32 d, z;\n\t"
+        "mov.b32 z, 0;\n\t"
+        "setp.ne.u32 q, z, 0;\n\t"
+        "lop3.or.b32 d|p, %1, %2, z, 0xC0, q;\n\t"
+        "vote.sync.ballot.b32 %0, p, 0xffffffff;\n\t}"
+        : "=r"(r) : "r"(v), "r"(mask));
+    return r;
+}
+// acc += w when (word & bit) != 0: a logic op with predicate output and a predicated add, no branch.
+__device__ __forceinline__ void add_if_bit(float& acc, uint32_t word, uint32_t bit, float w)
+{
+    asm("{\n\t.reg .pred p, q;\n\t.reg .b32 d, z;\n\t"
+        "mov.b32 z, 0;\n\t"
+        "setp.ne.u32 q, z, 0;\n\t"
+        "lop3.or.b32 d|p, %1, %2, z, 0xC0, q;\n\t"
+        "@p add.rn.f32 %0, %0, %3;\n\t}"
+        : "+f"(acc) : "r"(word), "r"(bit), "f"(w));
+}
+__device__ __forceinline__ void neg_if_bit(float& acc, uint32_t word, uint32_t bit)
+{
+    asm("{\n\t.reg .pred p, q;\n\t.reg .b32 d, z;\n\t"
+        "mov.b32 z, 0;\n\t"
+        "setp.ne.u32 q, z, 0;\n\t"
+        "lop3.or.b32 d|p, %1, %2, z, 0xC0, q;\n\t"
+        "@p neg.f32 %0, %0;\n\t}"
+        : "+f"(acc) : "r"(word), "r"(bit));
 }
 
 __device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
@@ -274,7 +310,7 @@ __device__ __forceinline__ TileDesc describe_tile(const uint32_t* __restrict__ i
 // Integer path: decodes this warp's 16 blocks straight from global memory into codes relative to the warp's first
 // element, one element per lane (q[i] = sum of deltas from the warp's first element; the caller adds the outlier
 // and the sums of the preceding warps).
-__device__ __noinline__ void decode_blocks_int(const TileDesc& d, int warp, int lane, int32_t* __restrict__ q)
+__device__ __forceinline__ void decode_blocks_int(const TileDesc& d, int warp, int lane, int32_t* __restrict__ q)
 {
     const uint32_t* payload = d.blob + 1 + d.padw;
     int32_t carry = 0;
@@ -306,9 +342,8 @@ __device__ __noinline__ void decode_blocks_int(const TileDesc& d, int warp, int 
     }
 }
 
-#define ZCCL_DEC_PLANE(k)                                        \
-    case (k) + 1:                                                \
-        if (pw[(k) + 1] & lanebit) mag += (float)(1u << (k));
+#define ZCCL_DEC_PLANE(k) \
+    case (k) + 1: add_if_bit(mag, pw[(k) + 1], lanebit, (float)(1u << (k)));
 
 // fp32 path: rebuilds this warp's 16 blocks of deltas from the staged blob and stores them, as exact floats, in
 // the warp's 512-word region `wbuf`, row i = block i, element j of a row at word j ^ ((i & 3) << 2) (so that the
@@ -331,7 +366,7 @@ __device__ __forceinline__ void decode_blocks_f32(const uint32_t* __restrict__ p
                 ZCCL_DEC_PLANE(12) ZCCL_DEC_PLANE(11) ZCCL_DEC_PLANE(10) ZCCL_DEC_PLANE(9) ZCCL_DEC_PLANE(8)
                 ZCCL_DEC_PLANE(7) ZCCL_DEC_PLANE(6) ZCCL_DEC_PLANE(5) ZCCL_DEC_PLANE(4) ZCCL_DEC_PLANE(3)
                 ZCCL_DEC_PLANE(2) ZCCL_DEC_PLANE(1) ZCCL_DEC_PLANE(0)
-                    if (pw[0] & lanebit) mag = -mag;
+                    neg_if_bit(mag, pw[0], lanebit);
                 default: break;
             }
             wbuf[32 * i + (lane ^ (u << 2))] = mag;
@@ -517,15 +552,13 @@ struct SrcSwizzled {        // the fused kernel's sum tile: per-warp region of 1
     __device__ __forceinline__ float prev(int g, int u) const { return rows[32 * (4 * g + u + 1) + po[u]]; }
 };
 
-#define ZCCL_ENC_PLANE(k)                                                    \
-    case (k) + 1: {                                                          \
-        const uint32_t p_ = __ballot_sync(kFull, ab & (1u << (k)));          \
-        if (lane == 0) slot[(k) + 1] = p_;                                   \
-    }
+#define ZCCL_ENC_PLANE(k) \
+    case (k) + 1: slot[(k) + 1] = ballot_and(ab, 1u << (k));
 
-// One pass over this warp's 16 blocks: quantise, 1-D Lorenzo delta, code length, sign word and bit planes into the
-// block's fixed slot.  Returns the warp's payload size in words; lane g (g < 4) ends up holding the code-length
-// word of blocks 4g..4g+3 in `my_lw`.  FAST: fp32 arithmetic, valid while every |x * r| < 2^21.5; the caller
+// One pass over this warp's 16 blocks: quantise, 1-D Lorenzo delta, code length, sign word and bit planes, appended
+// to the warp's region of shared memory (every lane stores the same warp-uniform word: no predicate, one
+// wavefront).  Returns the warp's payload size in words; lane g (g < 4) ends up holding the code-length word of
+// blocks 4g..4g+3 in `my_lw`.  FAST: fp32 arithmetic, valid while every |x * r| < 2^21.5; the caller
 // checks `guard` (sum of squares of x * r) and reruns with FAST = false when it is too large.
 template <bool FAST, class Src>
 __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint32_t* __restrict__ slots_w, int lane,
@@ -562,16 +595,13 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
                 L = 32u - (uint32_t)__clz((int)m);
                 sg = __ballot_sync(kFull, dd < 0);
             }
-            uint32_t* slot = slots_w + kSlotWords * (4 * g + u);
             if (L) {   // uniform over the warp
-                if (lane == 0) slot[0] = sg;
+                uint32_t* slot = slots_w + wsum;
+                slot[0] = sg;
                 switch (L) {
                     default:
                         if (!FAST) {
-                            for (uint32_t k = L - 1; k >= 23; --k) {
-                                const uint32_t p_ = __ballot_sync(kFull, ab & (1u << k));
-                                if (lane == 0) slot[k + 1] = p_;
-                            }
+                            for (uint32_t k = L - 1; k >= 23; --k) slot[k + 1] = __ballot_sync(kFull, ab & (1u << k));
                         }
                     ZCCL_ENC_PLANE(22) ZCCL_ENC_PLANE(21) ZCCL_ENC_PLANE(20) ZCCL_ENC_PLANE(19) ZCCL_ENC_PLANE(18)
                     ZCCL_ENC_PLANE(17) ZCCL_ENC_PLANE(16) ZCCL_ENC_PLANE(15) ZCCL_ENC_PLANE(14) ZCCL_ENC_PLANE(13)
@@ -591,28 +621,30 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
     return wsum;
 }
 
+constexpr int kLookWindows = 32;   // windows of 32 scan states inspected per look-back iteration (4 per warp)
+struct LookShared {
+    uint32_t sum[2][kLookWindows];
+    uint32_t st[2][kLookWindows];     // 0: 32 aggregates, 1: reached an inclusive prefix, 2: met a state not yet published
+};
+
 struct EncodeShared {
-    alignas(16) float xbuf[2][kTile + 8];                       // double-buffered input tiles (+ guard word)
-    alignas(16) uint32_t slots[kBlocksPerTile * kSlotWords];    // one fixed slot per block
-    uint32_t warp_words[kWarps];
-    uint32_t ticket[2];
-    uint32_t excl;
-    uint32_t skip;
-    alignas(8) unsigned long long bar[2];
+    alignas(16) float xbuf[kTile + 8];                             // staged input tile (+ guard word in front)
+    alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];    // encoded tiles: current and awaiting placement
+    uint32_t warp_words[2][kWarps];
+    LookShared look;
+    alignas(8) unsigned long long bar;
 };
 
 struct FusedShared {
     alignas(16) uint32_t blob[kBlobStageWords];
     alignas(16) float ybuf[kWarps][(kBlocksPerWarp + 1) * kBlock];   // deltas, then sums (row 0 of a warp = guard)
     alignas(16) uint32_t tbl[kWarps][kBlocksPerWarp];
-    alignas(16) uint32_t slots[kBlocksPerTile * kSlotWords];
+    alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];
     float warp_total[kWarps];
     int32_t warp_total_i[kWarps];
     int32_t warp_total_i2[kWarps];
-    uint32_t warp_words[kWarps];
-    uint32_t ticket[2];
-    uint32_t excl;
-    uint32_t skip;
+    uint32_t warp_words[2][kWarps];
+    LookShared look;
     alignas(8) unsigned long long bar;
 };
 
@@ -623,56 +655,65 @@ __device__ __forceinline__ bool stageable_raw(const Job& job, uint32_t tile)
     return job.n - start >= (unsigned long long)kTile && (((uintptr_t)(job.x + start)) & 15u) == 0;
 }
 
-// Placement: decoupled look-back over the preceding tiles of this job, run by warp 0.  Returns the exclusive
-// prefix in words; sets `skip` when the bounded wait expired.
-__device__ __forceinline__ uint32_t look_back(const Workspace& ws, uint32_t ticket, uint32_t tile_begin, uint32_t epoch,
-                                              uint32_t total, int lane, uint32_t& skip, uint32_t& status)
+// Placement: decoupled look-back over the preceding tiles of this job, run by the whole CTA.  Each iteration
+// inspects the 1024 nearest predecessors (32 windows of 32 states, four per warp: more than a grid's worth of
+// tiles, so one iteration normally reaches an inclusive prefix); the windows are combined in order
+// until the first inclusive prefix.  Returns the exclusive prefix in words (same value in every thread); sets
+// `skip` when the bounded wait expired.
+
+__device__ __forceinline__ uint32_t look_back_cta(LookShared& ls, uint32_t& par, const Workspace& ws, uint32_t ticket,
+                                                  uint32_t tile_begin, uint32_t epoch, int warp, int lane, uint32_t& skip,
+                                                  uint32_t& status)
 {
     uint32_t excl = 0;
     skip = 0;
     long long pos = (long long)ticket - 1;
     const long long lo = (long long)tile_begin;
-    int budget = kSpinLimit;
+    int budget = kSpinLimit >> 4;
     for (;;) {
-        const long long at = pos - lane;
-        unsigned long long st = pack_state(epoch, 1u, 0u);   // before the job's first tile: prefix 0
-        if (at >= lo) st = ld_state(ws.tile_state + at);
-        const bool valid = (uint32_t)(st >> 33) == epoch;
-        const uint32_t vmask = __ballot_sync(kFull, valid);
-        const uint32_t imask = __ballot_sync(kFull, valid && ((st >> 32) & 1ull));
-        const int first = imask ? (__ffs((int)imask) - 1) : 31;
-        const uint32_t need = (first == 31) ? kFull : ((2u << first) - 1u);
-        if ((vmask & need) != need) {
-            if (--budget == 0) { skip = 1; status |= kStTimeout; break; }
-            __nanosleep(40);
-            continue;
+#pragma unroll
+        for (int hh = 0; hh < kLookWindows / kWarps; ++hh) {
+            const int w = warp + kWarps * hh;
+            const long long at = pos - 32 * w - lane;
+            unsigned long long st = pack_state(epoch, 1u, 0u);   // before the job's first tile: prefix 0
+            if (at >= lo) st = ld_state(ws.tile_state + at);
+            const bool valid = (uint32_t)(st >> 33) == epoch;
+            const uint32_t vmask = __ballot_sync(kFull, valid);
+            const uint32_t imask = __ballot_sync(kFull, valid && ((st >> 32) & 1ull));
+            const int first = imask ? (__ffs((int)imask) - 1) : 31;
+            const uint32_t need = (first == 31) ? kFull : ((2u << first) - 1u);
+            const uint32_t sum = __reduce_add_sync(kFull, (lane <= first) ? (uint32_t)st : 0u);
+            if (lane == 0) {
+                ls.sum[par][w] = sum;
+                ls.st[par][w] = ((vmask & need) != need) ? 2u : (imask ? 1u : 0u);
+            }
         }
-        const uint32_t contrib = (lane <= first) ? (uint32_t)st : 0u;
-        excl += __reduce_add_sync(kFull, contrib);
-        if (imask) break;
-        pos -= 32;
+        __syncthreads();
+        uint32_t acc = 0, res = 0;
+#pragma unroll 1
+        for (int w = 0; w < kLookWindows; ++w) {
+            const uint32_t t = ls.st[par][w];
+            if (t == 2u) { res = 2; break; }
+            acc += ls.sum[par][w];
+            if (t == 1u) { res = 1; break; }
+        }
+        par ^= 1u;
+        if (res == 1u) { excl += acc; break; }
+        if (res == 0u) { excl += acc; pos -= 32 * kLookWindows; continue; }
+        if (--budget == 0) { skip = 1; status |= kStTimeout; break; }   // uniform: every thread reads the same words
+        __nanosleep(64);
     }
-    if (lane == 0) st_state(ws.tile_state + ticket, pack_state(epoch, 1u, excl + total));
     return excl;
 }
 
-// Copies this warp's blocks from their slots to the stream, compacting them; writes the warp's code-length words.
+// Copies this warp's contiguous region to its place in the stream; writes the warp's code-length words.
 __device__ __forceinline__ void copy_out_warp(uint32_t* __restrict__ blob_out, const uint32_t* __restrict__ slots_w,
-                                              uint32_t wbase, uint32_t my_lw, uint32_t padw, int warp, int lane)
+                                              uint32_t wbase, uint32_t wsum, uint32_t my_lw, uint32_t padw, int warp, int lane)
 {
-    uint32_t off = wbase;
-#pragma unroll 1
-    for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
-        const uint32_t lword = __shfl_sync(kFull, my_lw, g);
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t L = (lword >> (8 * u)) & 0xFF;
-            const uint32_t sz = L ? L + 1 : 0;
-            if ((uint32_t)lane < sz) blob_out[off + lane] = slots_w[kSlotWords * (4 * g + u) + lane];
-            off += sz;
-        }
-    }
+    uint32_t* __restrict__ dst = blob_out + wbase;
+    for (uint32_t i = lane; i < wsum; i += 32) dst[i] = slots_w[i];
     if (lane < 4 && (uint32_t)(4 * warp + lane) < padw) blob_out[1 + 4 * warp + lane] = my_lw;
+    __syncwarp();
 }
 
 __device__ __forceinline__ void write_header(uint32_t* out, int tid, unsigned long long n, float eb_abs, float s, uint32_t nT)
@@ -699,8 +740,7 @@ __device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoc
     if (tid == 0) {
         __threadfence();
         const uint32_t prev = atomicAdd(ws.done, 1u);
-        if (prev == gridDim.x - 1) {   // every CTA has drawn its last ticket: re-arm for the next launch
-            *ws.ticket = 0;
+        if (prev == gridDim.x - 1) {   // every CTA is done with the scan states: re-arm for the next launch
             *ws.done = 0;
             uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
             *ws.epoch = e ? e : 1u;
@@ -708,47 +748,66 @@ __device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoc
     }
 }
 
-// Sizes -> placement -> copy-out, shared by both encoders.  Called by all threads after the warp sizes are in
-// shared memory and a barrier has passed.
-template <class Shared>
-__device__ __forceinline__ void place_and_copy(Shared& sh, const Workspace& ws, const Job& job, uint32_t ticket, uint32_t tile,
-                                               uint32_t nT, uint32_t padw, uint32_t epoch, const uint32_t* slots_w,
-                                               uint32_t my_lw, int32_t q_first, float eb_abs, float s, int tid, int warp,
-                                               int lane, uint32_t& status)
+// An encoded tile sitting in shared memory until its place in the stream is known.  Placement is deferred by one
+// tile: while a CTA encodes its next tile the sizes of the earlier tiles of all CTAs get published, so the
+// look-back of the deferred tile finds them without waiting.
+struct Pending {
+    bool valid;
+    int job;
+    uint32_t ticket, tile, nT, padw;
+    uint32_t buf;        // which half of the slots holds it
+    uint32_t wsum;       // this warp's payload words
+    uint32_t wbase;      // this warp's offset inside the blob
+    uint32_t total;      // blob words
+    uint32_t my_lw;      // lanes 0..3: this warp's code-length words
+    int32_t q_first;     // outlier (thread 0)
+    float eb_abs, s;
+};
+
+// After the barrier that follows a tile's encoding pass: this warp's offset and the blob size from the warps'
+// sizes, and the tile's size published to the scan (as an inclusive prefix for a job's first tile).
+__device__ __forceinline__ void announce(const uint32_t* warp_words, const Workspace& ws, uint32_t epoch, Pending& c, int tid, int warp)
 {
-    uint32_t wbase = 1 + padw, total = 1 + padw;
+    uint32_t wbase = 1 + c.padw, total = 1 + c.padw;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) {
-        const uint32_t ww = sh.warp_words[w];
+        const uint32_t ww = warp_words[w];
         if (w < warp) wbase += ww;
         total += ww;
     }
-    if (warp == 0) {
-        uint32_t excl = 0, skip = 0;
-        if (tile == 0) {
-            if (lane == 0) st_state(ws.tile_state + ticket, pack_state(epoch, 1u, total));
-        } else {
-            if (lane == 0) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
-            excl = look_back(ws, ticket, job.tile_begin, epoch, total, lane, skip, status);
-        }
-        if (lane == 0) { sh.excl = excl; sh.skip = skip; }
-    }
-    __syncthreads();   // exclusive prefix known
+    c.wbase = wbase;
+    c.total = total;
+    if (tid == 0) st_state(ws.tile_state + c.ticket, pack_state(epoch, c.tile == 0 ? 1u : 0u, total));
+}
 
-    const uint32_t excl = sh.excl;
-    const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
-    const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
+// Places a pending tile: exclusive prefix by look-back, then copy-out, index entry, header and stream length.
+__device__ __forceinline__ void place(const Pending& c, const JobBatch& jb, LookShared& look, uint32_t& look_par,
+                                      const uint32_t* slots_w, const Workspace& ws, uint32_t epoch, int tid, int warp, int lane,
+                                      uint32_t& status)
+{
+    const Job& job = jb.job[c.job];
+    uint32_t excl = 0, skip = 0;
+    if (c.tile != 0) {
+#ifdef ZCCL_DEBUG_NO_LOOKBACK
+        excl = c.tile * 700u;
+#else
+        excl = look_back_cta(look, look_par, ws, c.ticket, job.tile_begin, epoch, warp, lane, skip, status);
+#endif
+        if (tid == 0) st_state(ws.tile_state + c.ticket, pack_state(epoch, 1u, excl + c.total));
+    }
+    const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + c.nT + excl;
+    const bool fits = (blob_word0 + c.total) * 4ull <= job.out_cap;
     if (!fits) status |= kStCapacity;
-    if (fits && !sh.skip) {
+    if (fits && !skip) {
         uint32_t* blob_out = job.out + blob_word0;
-        copy_out_warp(blob_out, slots_w, wbase, my_lw, padw, warp, lane);
+        copy_out_warp(blob_out, slots_w, c.wbase, c.wsum, c.my_lw, c.padw, warp, lane);
         if (tid == 0) {
-            blob_out[0] = (uint32_t)q_first;
-            job.out[kHeaderWords + tile] = excl + total;
+            blob_out[0] = (uint32_t)c.q_first;
+            job.out[kHeaderWords + c.tile] = excl + c.total;
         }
     }
-    if (tile == 0) write_header(job.out, tid, job.n, eb_abs, s, nT);
-    if (tile == nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
+    if (c.tile == 0) write_header(job.out, tid, job.n, c.eb_abs, c.s, c.nT);
+    if (c.tile == c.nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + c.total) * 4ull);
 }
 
 // ------------------------------------------------------------------------------------------------ compress
@@ -759,35 +818,37 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     EncodeShared& sh = *reinterpret_cast<EncodeShared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
+    const uint32_t G = gridDim.x;
     uint32_t status = 0;
     Params prm = hp;
     if (use_dev_params) prm = *ws.params;
     const float r = prm.r, s = prm.s, eb_abs = prm.eb_abs;
+    float* const xt = &sh.xbuf[4];
 
-    // prologue: first ticket, first bulk copy
-    if (tid == 0) {
-        mbar_init(&sh.bar[0], 1);
-        mbar_init(&sh.bar[1], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        const uint32_t t0 = atomicAdd(ws.ticket, 1u);
-        sh.ticket[0] = t0;
-        if (t0 < jb.total_tiles && prm.valid) {
-            const Job& j0 = jb.job[find_job(jb, t0)];
-            const uint32_t tile0 = t0 - j0.tile_begin;
-            if (j0.n && stageable_raw(j0, tile0)) {
-                mbar_expect_tx(&sh.bar[0], kTile * 4);
-                bulk_load(&sh.xbuf[0][4], j0.x + (unsigned long long)tile0 * kTile, kTile * 4, &sh.bar[0]);
+    // thread 0 starts the bulk copy of tile `t` into the staging buffer when that tile can be staged
+    auto stage = [&](uint32_t t) {
+        if (t < jb.total_tiles && prm.valid) {
+            const Job& jn = jb.job[find_job(jb, t)];
+            const uint32_t tn = t - jn.tile_begin;
+            if (jn.n && stageable_raw(jn, tn)) {
+                mbar_expect_tx(&sh.bar, kTile * 4);
+                bulk_load(xt, jn.x + (unsigned long long)tn * kTile, kTile * 4, &sh.bar);
             }
         }
+    };
+    if (tid == 0) {
+        mbar_init(&sh.bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        stage(blockIdx.x);
     }
     __syncthreads();
-    uint32_t fills0 = 0, fills1 = 0;   // completed bulk copies per buffer (phase parity of its mbarrier)
-    uint32_t p = 0;                    // buffer and ticket slot of the current tile
-    bool pending = false;              // thread 0: a bulk copy for the next tile is in flight
+    uint32_t look_par = 0;
+    uint32_t fills = 0;    // completed bulk copies (phase parity of the mbarrier)
+    uint32_t p = 0;        // half of the slots the current tile is encoded into
+    Pending pend;
+    pend.valid = false;
 
-    for (;;) {
-        const uint32_t ticket = sh.ticket[p];
-        if (ticket >= jb.total_tiles) break;
+    for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += G) {
         const int j = find_job(jb, ticket);
         const Job& job = jb.job[j];
         const uint32_t tile = ticket - job.tile_begin;
@@ -795,53 +856,32 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         const uint32_t nT = (uint32_t)((n + kTile - 1) / kTile);
         const bool staged = prm.valid && n && stageable_raw(job, tile);
 
-        // thread 0: draw the next ticket and start its bulk copy into the other buffer (its last readers
-        // finished before the barrier that ended the previous tile's encoding pass)
-        if (tid == 0) {
-            const uint32_t nt = atomicAdd(ws.ticket, 1u);
-            sh.ticket[p ^ 1u] = nt;
-            pending = false;
-            if (nt < jb.total_tiles && prm.valid) {
-                const Job& jn = jb.job[find_job(jb, nt)];
-                const uint32_t tn = nt - jn.tile_begin;
-                if (jn.n && stageable_raw(jn, tn)) {
-                    mbar_expect_tx(&sh.bar[p ^ 1u], kTile * 4);
-                    bulk_load(&sh.xbuf[p ^ 1u][4], jn.x + (unsigned long long)tn * kTile, kTile * 4, &sh.bar[p ^ 1u]);
-                    pending = true;
-                }
-            }
-        }
-
-        if (n == 0 || !prm.valid) {   // a job without elements still owns one ticket: header and length only
+        if (n == 0 || !prm.valid) {   // a job without elements still owns one tile number: header and length only
             const bool hdr = prm.valid && job.out_cap >= (unsigned)kHeaderBytes;
             if (tid == 0) {
                 st_state(ws.tile_state + ticket, pack_state(epoch, 1u, 0u));
                 if (tile == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
+                stage(ticket + G);   // nothing was staged for this tile, and the buffer's last readers are past a barrier
             }
             if (hdr && tile == 0) write_header(job.out, tid, 0, eb_abs, s, 0);
-            __syncthreads();
-            p ^= 1u;
             continue;
         }
 
         const unsigned long long start = (unsigned long long)tile * kTile;
         const uint32_t len = (uint32_t)((n - start < (unsigned long long)kTile) ? (n - start) : kTile);
         const uint32_t nb = (len + kBlock - 1) / kBlock;
-        const uint32_t padw = (nb + 3) >> 2;
 
-        // ---- single pass over the warp's blocks: quantise, delta, code length, planes -> slots
-        uint32_t* slots_w = sh.slots + kSlotWords * kBlocksPerWarp * warp;
+        // ---- single pass over the warp's blocks: quantise, delta, code length, planes -> this warp's region
+        uint32_t* slots_w = sh.slots[p] + kSlotWords * kBlocksPerWarp * warp;
         uint32_t my_lw = 0, wsum = 0;
         int32_t q_first = 0;
         float guard = 0.0f, tmax = 0.0f;
         bool need_int = !staged;
         if (staged) {
-            const uint32_t fl = p ? fills1 : fills0;
-            const bool landed = mbar_wait(&sh.bar[p], fl & 1u);
-            if (p) ++fills1; else ++fills0;
+            const bool landed = mbar_wait(&sh.bar, fills & 1u);
+            ++fills;
             if (!landed) status |= kStTimeout;   // carry on with whatever is staged: the result is flagged invalid
-            float* xt = &sh.xbuf[p][4];
-            if (tid == 0) xt[-1] = xt[0];    // the tile's first element is its own predecessor
+            if (tid == 0) xt[-1] = xt[0];        // the tile's first element is its own predecessor
             const SrcStaged src{xt + 512 * warp + lane};
             wsum = encode_blocks<true>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
             need_int = __any_sync(kFull, !(guard < kGuardExact));
@@ -860,18 +900,25 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
             if (!(tmax < 1073741824.0f)) status |= kStRange;
             else if (tmax > 32768.5f) status |= kStPrecision;
         }
-        if (lane == 0) sh.warp_words[warp] = wsum;
-        __syncthreads();   // sizes of all warps; the staged tile has been consumed
-        place_and_copy(sh, ws, job, ticket, tile, nT, padw, epoch, slots_w, my_lw, q_first, eb_abs, s, tid, warp, lane, status);
+        if (lane == 0) sh.warp_words[p][warp] = wsum;
+        __syncthreads();   // sizes of all warps are visible; the staged tile has been consumed
+        if (tid == 0) stage(ticket + G);   // overlaps with the placement of the previous tile below
+
+        Pending cur;
+        cur.valid = true; cur.job = j; cur.ticket = ticket; cur.tile = tile; cur.nT = nT; cur.padw = (nb + 3) >> 2;
+        cur.buf = p; cur.wsum = wsum; cur.my_lw = my_lw; cur.q_first = q_first; cur.eb_abs = eb_abs; cur.s = s;
+        announce(sh.warp_words[p], ws, epoch, cur, tid, warp);
+        if (pend.valid)
+            place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
+        pend = cur;
         p ^= 1u;
     }
+    if (pend.valid)
+        place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
 
     // never leave with a bulk copy in flight into this CTA's shared memory: every copy that was started has been
     // waited for by the iteration that consumed it, except after an expired wait; then give it one more bounded wait
-    if (tid == 0 && (pending || (status & kStTimeout))) {
-        (void)mbar_wait(&sh.bar[0], (fills0 + 1u) & 1u);
-        (void)mbar_wait(&sh.bar[1], (fills1 + 1u) & 1u);
-    }
+    if (tid == 0 && (status & kStTimeout)) (void)mbar_wait(&sh.bar, (fills + 1u) & 1u);
     if (status) atomicOr(ws.status, status);
     finish_launch(ws, epoch, tid);
 }
@@ -890,18 +937,17 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     if (tid == 0) {
         mbar_init(&sh.bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        sh.ticket[0] = atomicAdd(ws.ticket, 1u);
     }
     __syncthreads();
-    uint32_t p = 0;
+    uint32_t look_par = 0, p = 0;
+    Pending pend;
+    pend.valid = false;
     int cur_job = -1;
     StreamInfo h1, h2;
     h1.ok = h2.ok = false; h1.n = h2.n = 0; h1.nT = h2.nT = 0; h1.s = h2.s = 1.0f; h1.eb_abs = h2.eb_abs = 0.0f;
     bool job_ok = false;
 
-    for (;;) {
-        const uint32_t ticket = sh.ticket[p];
-        if (ticket >= jb.total_tiles) break;
+    for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += gridDim.x) {
         const int j = find_job(jb, ticket);
         const Job& job = jb.job[j];
         const uint32_t tile = ticket - job.tile_begin;
@@ -918,7 +964,6 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
         const float s = h1.s, eb_abs = h1.eb_abs;
         const float r = __fdiv_rn(1.0f, s);
-        if (tid == 0) sh.ticket[p ^ 1u] = atomicAdd(ws.ticket, 1u);
 
         if (!job_ok || n == 0) {
             if (!job_ok) status |= kStBadStream;
@@ -929,7 +974,6 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             }
             if (hdr && tile == 0) write_header(job.out, tid, 0, eb_abs, s, 0);
             __syncthreads();
-            p ^= 1u;
             continue;
         }
 
@@ -949,7 +993,6 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 if (tile == nT - 1) *job.out_bytes = 0;
             }
             __syncthreads();
-            p ^= 1u;
             continue;
         }
 
@@ -1063,7 +1106,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
 
         // ---- back end: encode the sums
-        uint32_t* slots_w = sh.slots + kSlotWords * kBlocksPerWarp * warp;
+        uint32_t* slots_w = sh.slots[p] + kSlotWords * kBlocksPerWarp * warp;
         uint32_t my_lw = 0, wsum = 0;
         int32_t q_first = 0;
         float guard = 0.0f, tmax = 0.0f;
@@ -1092,11 +1135,19 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                     if (e <= last) yout[e] = __fmul_rn(__int2float_rn(__float2int_rn(__fmul_rn(src.cur(g, u), r))), s);
                 }
         }
-        if (lane == 0) sh.warp_words[warp] = wsum;
+        if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps
-        place_and_copy(sh, ws, job, ticket, tile, nT, padw, epoch, slots_w, my_lw, q_first, eb_abs, s, tid, warp, lane, status);
+        Pending cur;
+        cur.valid = true; cur.job = j; cur.ticket = ticket; cur.tile = tile; cur.nT = nT; cur.padw = padw;
+        cur.buf = p; cur.wsum = wsum; cur.my_lw = my_lw; cur.q_first = q_first; cur.eb_abs = eb_abs; cur.s = s;
+        announce(sh.warp_words[p], ws, epoch, cur, tid, warp);
+        if (pend.valid)
+            place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
+        pend = cur;
         p ^= 1u;
     }
+    if (pend.valid)
+        place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
     if (status) atomicOr(ws.status, status);
     finish_launch(ws, epoch, tid);
 }
