@@ -101,38 +101,75 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// Ballot of (v & mask) != 0 over the warp: one logic op with predicate output feeding the vote.
-__device__ __forceinline__ uint32_t ballot_and(uint32_t v, uint32_t mask)
-{
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b32 d, z;\n\t"
-        "mov.b32 z, 0;\n\t"
-        "setp.ne.u32 q, z, 0;\n\t"
-        "lop3.or.b32 d|p, %1, %2, z, 0xC0, q;\n\t"
-        "vote.sync.ballot.b32 %0, p, 0xffffffff;\n\t}"
-        : "=r"(r) : "r"(v), "r"(mask));
-    return r;
-}
-// acc += w when (word & bit) != 0: a logic op with predicate output and a predicated add, no branch.
-__device__ __forceinline__ void add_if_bit(float& acc, uint32_t word, uint32_t bit, float w)
-{
-    asm("{\n\t.reg .pred p, q;\n\t.reg .b32 d, z;\n\t"
-        "mov.b32 z, 0;\n\t"
-        "setp.ne.u32 q, z, 0;\n\t"
-        "lop3.or.b32 d|p, %1, %2, z, 0xC0, q;\n\t"
-        "@p add.rn.f32 %0, %0, %3;\n\t}"
-        : "+f"(acc) : "r"(word), "r"(bit), "f"(w));
-}
-__device__ __forceinline__ void neg_if_bit(float& acc, uint32_t word, uint32_t bit)
-{
-    asm("{\n\t.reg .pred p, q;\n\t.reg .b32 d, z;\n\t"
-        "mov.b32 z, 0;\n\t"
-        "setp.ne.u32 q, z, 0;\n\t"
-        "lop3.or.b32 d|p, %1, %2, z, 0xC0, q;\n\t"
-        "@p neg.f32 %0, %0;\n\t}"
-        : "+f"(acc) : "r"(word), "r"(bit));
-}
+// Per-block plane code.  The number of bit planes of a block is warp-uniform, so both coders jump (brx.idx.uni)
+// into a straight line of per-plane steps and fall through to plane 0: no compare tree, no per-plane branch.
+//   decoder: plane word (broadcast load from the staged blob) AND this lane's bit -> predicated add of 2^k; the sign
+//            word negates.  addr = shared-memory byte address of the block's payload (sign word first).
+//   encoder: (|delta| AND 2^k) != 0 -> ballot -> the same word stored by every lane at slot + 4 (k + 1); the sign
+//            word goes to slot + 0.  slot = shared-memory byte address.
+#define ZCCL_DEC_BLOCK_ASM(mag, L, addr, lanebit)                                  \
+    asm volatile("{\n\t"                                                              \
+                 ".reg .pred p;\n\t.reg .b32 w, d;\n\t"                                \
+                 "ts: .branchtargets T0, T1, T2, T3, T4, T5, T6, T7, T8, T9, T10, T11, T12, T13, T14, T15, T16, T17, T18, T19, T20, T21, T22, T23;\n\t"  \
+                 "brx.idx.uni %1, ts;\n\t"                                           \
+                 "T23: ld.shared.u32 w, [%2+92];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f4A800000;\n\t" \
+                 "T22: ld.shared.u32 w, [%2+88];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f4A000000;\n\t" \
+                 "T21: ld.shared.u32 w, [%2+84];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f49800000;\n\t" \
+                 "T20: ld.shared.u32 w, [%2+80];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f49000000;\n\t" \
+                 "T19: ld.shared.u32 w, [%2+76];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f48800000;\n\t" \
+                 "T18: ld.shared.u32 w, [%2+72];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f48000000;\n\t" \
+                 "T17: ld.shared.u32 w, [%2+68];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f47800000;\n\t" \
+                 "T16: ld.shared.u32 w, [%2+64];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f47000000;\n\t" \
+                 "T15: ld.shared.u32 w, [%2+60];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f46800000;\n\t" \
+                 "T14: ld.shared.u32 w, [%2+56];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f46000000;\n\t" \
+                 "T13: ld.shared.u32 w, [%2+52];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f45800000;\n\t" \
+                 "T12: ld.shared.u32 w, [%2+48];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f45000000;\n\t" \
+                 "T11: ld.shared.u32 w, [%2+44];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f44800000;\n\t" \
+                 "T10: ld.shared.u32 w, [%2+40];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f44000000;\n\t" \
+                 "T9: ld.shared.u32 w, [%2+36];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f43800000;\n\t" \
+                 "T8: ld.shared.u32 w, [%2+32];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f43000000;\n\t" \
+                 "T7: ld.shared.u32 w, [%2+28];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f42800000;\n\t" \
+                 "T6: ld.shared.u32 w, [%2+24];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f42000000;\n\t" \
+                 "T5: ld.shared.u32 w, [%2+20];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f41800000;\n\t" \
+                 "T4: ld.shared.u32 w, [%2+16];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f41000000;\n\t" \
+                 "T3: ld.shared.u32 w, [%2+12];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f40800000;\n\t" \
+                 "T2: ld.shared.u32 w, [%2+8];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f40000000;\n\t" \
+                 "T1: ld.shared.u32 w, [%2+4];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f3F800000;\n\t" \
+                 "ld.shared.u32 w, [%2];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p neg.f32 %0, %0;\n\t" \
+                 "T0:\n\t}"                                                          \
+                 : "+f"(mag) : "r"(L), "r"(addr), "r"(lanebit) : "memory")
+
+#define ZCCL_ENC_BLOCK_ASM(ab, L, sg, slot)                                        \
+    asm volatile("{\n\t"                                                              \
+                 ".reg .pred p;\n\t.reg .b32 w, d;\n\t"                                \
+                 "ts: .branchtargets T0, T1, T2, T3, T4, T5, T6, T7, T8, T9, T10, T11, T12, T13, T14, T15, T16, T17, T18, T19, T20, T21, T22, T23;\n\t"  \
+                 "brx.idx.uni %1, ts;\n\t"                                           \
+                 "T23: and.b32 d, %0, 4194304;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+92], w;\n\t" \
+                 "T22: and.b32 d, %0, 2097152;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+88], w;\n\t" \
+                 "T21: and.b32 d, %0, 1048576;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+84], w;\n\t" \
+                 "T20: and.b32 d, %0, 524288;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+80], w;\n\t" \
+                 "T19: and.b32 d, %0, 262144;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+76], w;\n\t" \
+                 "T18: and.b32 d, %0, 131072;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+72], w;\n\t" \
+                 "T17: and.b32 d, %0, 65536;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+68], w;\n\t" \
+                 "T16: and.b32 d, %0, 32768;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+64], w;\n\t" \
+                 "T15: and.b32 d, %0, 16384;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+60], w;\n\t" \
+                 "T14: and.b32 d, %0, 8192;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+56], w;\n\t" \
+                 "T13: and.b32 d, %0, 4096;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+52], w;\n\t" \
+                 "T12: and.b32 d, %0, 2048;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+48], w;\n\t" \
+                 "T11: and.b32 d, %0, 1024;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+44], w;\n\t" \
+                 "T10: and.b32 d, %0, 512;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+40], w;\n\t" \
+                 "T9: and.b32 d, %0, 256;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+36], w;\n\t" \
+                 "T8: and.b32 d, %0, 128;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+32], w;\n\t" \
+                 "T7: and.b32 d, %0, 64;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+28], w;\n\t" \
+                 "T6: and.b32 d, %0, 32;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+24], w;\n\t" \
+                 "T5: and.b32 d, %0, 16;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+20], w;\n\t" \
+                 "T4: and.b32 d, %0, 8;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+16], w;\n\t" \
+                 "T3: and.b32 d, %0, 4;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+12], w;\n\t" \
+                 "T2: and.b32 d, %0, 2;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+8], w;\n\t" \
+                 "T1: and.b32 d, %0, 1;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+4], w;\n\t" \
+                 "st.shared.u32 [%3], %2;\n\t"                                       \
+                 "T0:\n\t}"                                                          \
+                 :: "r"(ab), "r"(L), "r"(sg), "r"(slot) : "memory")
 
 __device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
 {
@@ -342,14 +379,10 @@ __device__ __forceinline__ void decode_blocks_int(const TileDesc& d, int warp, i
     }
 }
 
-#define ZCCL_DEC_PLANE(k) \
-    case (k) + 1: add_if_bit(mag, pw[(k) + 1], lanebit, (float)(1u << (k)));
-
 // fp32 path: rebuilds this warp's 16 blocks of deltas from the staged blob and stores them, as exact floats, in
 // the warp's 512-word region `wbuf`, row i = block i, element j of a row at word j ^ ((i & 3) << 2) (so that the
-// 128-bit reads of decode_scan_f32 are free of bank conflicts).
-__device__ __forceinline__ void decode_blocks_f32(const uint32_t* __restrict__ payload, const uint32_t* __restrict__ tbl,
-                                                  float* __restrict__ wbuf, int lane)
+// 128-bit reads of decode_scan_f32 are free of bank conflicts).  tbl: per block {code length, payload address}.
+__device__ __forceinline__ void decode_blocks_f32(const uint2* __restrict__ tbl, float* __restrict__ wbuf, int lane)
 {
     const uint32_t lanebit = 1u << lane;
 #pragma unroll 1
@@ -357,18 +390,9 @@ __device__ __forceinline__ void decode_blocks_f32(const uint32_t* __restrict__ p
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int i = 4 * g + u;
-            const uint32_t e = tbl[i];               // broadcast read: (offset << 8) | code length
-            const uint32_t L = e & 0xFF;
-            const uint32_t* pw = payload + (e >> 8);
+            const uint2 e = tbl[i];               // broadcast read: code length, shared address of the payload
             float mag = 0.0f;
-            switch (L) {
-                ZCCL_DEC_PLANE(17) ZCCL_DEC_PLANE(16) ZCCL_DEC_PLANE(15) ZCCL_DEC_PLANE(14) ZCCL_DEC_PLANE(13)
-                ZCCL_DEC_PLANE(12) ZCCL_DEC_PLANE(11) ZCCL_DEC_PLANE(10) ZCCL_DEC_PLANE(9) ZCCL_DEC_PLANE(8)
-                ZCCL_DEC_PLANE(7) ZCCL_DEC_PLANE(6) ZCCL_DEC_PLANE(5) ZCCL_DEC_PLANE(4) ZCCL_DEC_PLANE(3)
-                ZCCL_DEC_PLANE(2) ZCCL_DEC_PLANE(1) ZCCL_DEC_PLANE(0)
-                    neg_if_bit(mag, pw[0], lanebit);
-                default: break;
-            }
+            ZCCL_DEC_BLOCK_ASM(mag, e.x, e.y, lanebit);
             wbuf[32 * i + (lane ^ (u << 2))] = mag;
         }
     }
@@ -402,30 +426,28 @@ __device__ __forceinline__ float decode_scan_f32(const float* __restrict__ wbuf,
     return total;
 }
 
-// Writes the (offset, code length) table of this warp's 16 blocks from the lanes that hold them.
-__device__ __forceinline__ void write_block_table(const TileDesc& d, uint32_t* __restrict__ tbl, int warp, int lane)
+// Writes the table of this warp's 16 blocks, {code length, shared-memory byte address of the block's payload},
+// from the four lanes that hold their code-length word and offsets.
+__device__ __forceinline__ void write_block_table(const TileDesc& d, uint2* __restrict__ tbl, uint32_t payload_saddr,
+                                                  int warp, int lane)
 {
     if ((lane >> 2) == warp) {
-        const int k = 4 * (lane & 3);
-        uint4 e;
-        e.x = (d.o0 << 8) | (d.lw & 0xFF);
-        e.y = (d.o1 << 8) | ((d.lw >> 8) & 0xFF);
-        e.z = (d.o2 << 8) | ((d.lw >> 16) & 0xFF);
-        e.w = (d.o3 << 8) | (d.lw >> 24);
-        *reinterpret_cast<uint4*>(tbl + k) = e;
+        uint4* t4 = reinterpret_cast<uint4*>(tbl + 4 * (lane & 3));
+        t4[0] = make_uint4(d.lw & 0xFF, payload_saddr + 4 * d.o0, (d.lw >> 8) & 0xFF, payload_saddr + 4 * d.o1);
+        t4[1] = make_uint4((d.lw >> 16) & 0xFF, payload_saddr + 4 * d.o2, d.lw >> 24, payload_saddr + 4 * d.o3);
     }
 }
 
 struct DecodeShared {
     alignas(16) uint32_t blob[kBlobStageWords];
     alignas(16) float wbuf[kWarps][kBlocksPerWarp * kBlock];
-    alignas(16) uint32_t tbl[kWarps][kBlocksPerWarp];
+    alignas(16) uint2 tbl[kWarps][kBlocksPerWarp];
     float warp_total[2][kWarps];
     int32_t warp_total_i[kWarps];
     alignas(8) unsigned long long bar;
 };
 
-__global__ void __launch_bounds__(kThreads, 4) decode_kernel(JobBatch jb, Workspace ws)
+__global__ void __launch_bounds__(kThreads, 6) decode_kernel(JobBatch jb, Workspace ws)
 {
     __shared__ DecodeShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -463,12 +485,12 @@ __global__ void __launch_bounds__(kThreads, 4) decode_kernel(JobBatch jb, Worksp
                 mbar_expect_tx(&sh.bar, (uint32_t)(a_end - a_beg));
                 bulk_load(sh.blob, (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar);
             }
-            write_block_table(d, sh.tbl[warp], warp, lane);
+            write_block_table(d, sh.tbl[warp], smem_u32(sh.blob + shift + 1 + d.padw), warp, lane);
             __syncwarp();
             const bool landed = mbar_wait(&sh.bar, fills & 1u);
             ++fills;
             if (!landed) status |= kStTimeout;   // carry on with whatever is staged: reads stay inside shared memory
-            decode_blocks_f32(sh.blob + shift + 1 + d.padw, sh.tbl[warp], sh.wbuf[warp], lane);
+            decode_blocks_f32(sh.tbl[warp], sh.wbuf[warp], lane);
             __syncwarp();
             float v[16];
             const float total = decode_scan_f32(sh.wbuf[warp], lane, v);
@@ -552,9 +574,6 @@ struct SrcSwizzled {        // the fused kernel's sum tile: per-warp region of 1
     __device__ __forceinline__ float prev(int g, int u) const { return rows[32 * (4 * g + u + 1) + po[u]]; }
 };
 
-#define ZCCL_ENC_PLANE(k) \
-    case (k) + 1: slot[(k) + 1] = ballot_and(ab, 1u << (k));
-
 // One pass over this warp's 16 blocks: quantise, 1-D Lorenzo delta, code length, sign word and bit planes, appended
 // to the warp's region of shared memory (every lane stores the same warp-uniform word: no predicate, one
 // wavefront).  Returns the warp's payload size in words; lane g (g < 4) ends up holding the code-length word of
@@ -597,19 +616,11 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
             }
             if (L) {   // uniform over the warp
                 uint32_t* slot = slots_w + wsum;
-                slot[0] = sg;
-                switch (L) {
-                    default:
-                        if (!FAST) {
-                            for (uint32_t k = L - 1; k >= 23; --k) slot[k + 1] = __ballot_sync(kFull, ab & (1u << k));
-                        }
-                    ZCCL_ENC_PLANE(22) ZCCL_ENC_PLANE(21) ZCCL_ENC_PLANE(20) ZCCL_ENC_PLANE(19) ZCCL_ENC_PLANE(18)
-                    ZCCL_ENC_PLANE(17) ZCCL_ENC_PLANE(16) ZCCL_ENC_PLANE(15) ZCCL_ENC_PLANE(14) ZCCL_ENC_PLANE(13)
-                    ZCCL_ENC_PLANE(12) ZCCL_ENC_PLANE(11) ZCCL_ENC_PLANE(10) ZCCL_ENC_PLANE(9) ZCCL_ENC_PLANE(8)
-                    ZCCL_ENC_PLANE(7) ZCCL_ENC_PLANE(6) ZCCL_ENC_PLANE(5) ZCCL_ENC_PLANE(4) ZCCL_ENC_PLANE(3)
-                    ZCCL_ENC_PLANE(2) ZCCL_ENC_PLANE(1) ZCCL_ENC_PLANE(0)
-                    break;
+                uint32_t Lj = L;
+                if (!FAST) {   // planes beyond the jump table (integer path only)
+                    for (; Lj > 23; --Lj) slot[Lj] = __ballot_sync(kFull, ab & (1u << (Lj - 1)));
                 }
+                ZCCL_ENC_BLOCK_ASM(ab, Lj, sg, smem_u32(slot));
                 wsum += L + 1;
             }
             lword |= L << (8 * u);
@@ -621,7 +632,7 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
     return wsum;
 }
 
-constexpr int kLookWindows = 32;   // windows of 32 scan states inspected per look-back iteration (4 per warp)
+constexpr int kLookWindows = 16;   // windows of 32 scan states inspected per look-back iteration (2 per warp)
 struct LookShared {
     uint32_t sum[2][kLookWindows];
     uint32_t st[2][kLookWindows];     // 0: 32 aggregates, 1: reached an inclusive prefix, 2: met a state not yet published
@@ -638,7 +649,7 @@ struct EncodeShared {
 struct FusedShared {
     alignas(16) uint32_t blob[kBlobStageWords];
     alignas(16) float ybuf[kWarps][(kBlocksPerWarp + 1) * kBlock];   // deltas, then sums (row 0 of a warp = guard)
-    alignas(16) uint32_t tbl[kWarps][kBlocksPerWarp];
+    alignas(16) uint2 tbl[kWarps][kBlocksPerWarp];
     alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];
     float warp_total[kWarps];
     int32_t warp_total_i[kWarps];
@@ -656,8 +667,7 @@ __device__ __forceinline__ bool stageable_raw(const Job& job, uint32_t tile)
 }
 
 // Placement: decoupled look-back over the preceding tiles of this job, run by the whole CTA.  Each iteration
-// inspects the 1024 nearest predecessors (32 windows of 32 states, four per warp: more than a grid's worth of
-// tiles, so one iteration normally reaches an inclusive prefix); the windows are combined in order
+// inspects the 512 nearest predecessors (16 windows of 32 states, two per warp); the windows are combined in order
 // until the first inclusive prefix.  Returns the exclusive prefix in words (same value in every thread); sets
 // `skip` when the bounded wait expired.
 
@@ -689,14 +699,16 @@ __device__ __forceinline__ uint32_t look_back_cta(LookShared& ls, uint32_t& par,
             }
         }
         __syncthreads();
-        uint32_t acc = 0, res = 0;
-#pragma unroll 1
-        for (int w = 0; w < kLookWindows; ++w) {
-            const uint32_t t = ls.st[par][w];
-            if (t == 2u) { res = 2; break; }
-            acc += ls.sum[par][w];
-            if (t == 1u) { res = 1; break; }
-        }
+        // combine the windows in order (lane w holds window w): stop at the first inclusive prefix, fail on a
+        // window that met an unpublished state before it
+        const uint32_t wst = lane < kLookWindows ? ls.st[par][lane] : 0u;
+        const uint32_t wsm = lane < kLookWindows ? ls.sum[par][lane] : 0u;
+        const uint32_t m_incl = __ballot_sync(kFull, wst == 1u);
+        const uint32_t m_block = __ballot_sync(kFull, wst == 2u);
+        const int fw = m_incl ? (__ffs((int)m_incl) - 1) : (kLookWindows - 1);
+        const uint32_t upto = (2u << fw) - 1u;
+        const uint32_t acc = __reduce_add_sync(kFull, (lane <= fw) ? wsm : 0u);
+        const uint32_t res = (m_block & upto) ? 2u : (m_incl ? 1u : 0u);
         par ^= 1u;
         if (res == 1u) { excl += acc; break; }
         if (res == 0u) { excl += acc; pos -= 32 * kLookWindows; continue; }
@@ -1025,12 +1037,12 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                     for (int k = 0; k < 16; ++k) lv[k] = __ldg(lp + k);
                 }
             }
-            write_block_table(d1, sh.tbl[warp], warp, lane);
+            write_block_table(d1, sh.tbl[warp], smem_u32(sh.blob + shift + 1 + d1.padw), warp, lane);
             __syncwarp();
             const bool landed = mbar_wait(&sh.bar, fills & 1u);
             ++fills;
             if (!landed) status |= kStTimeout;
-            decode_blocks_f32(sh.blob + shift + 1 + d1.padw, sh.tbl[warp], yrows + 32, lane);
+            decode_blocks_f32(sh.tbl[warp], yrows + 32, lane);
             __syncwarp();
             float v[16];
             const float total = decode_scan_f32(yrows + 32, lane, v);
