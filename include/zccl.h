@@ -50,12 +50,14 @@ enum { ZCCL_OK = 0,
        ZCCL_E_BAD_STREAM = -5,  /* magic, version, sizes or index of a compressed stream are inconsistent */
        ZCCL_E_TIMEOUT = -6,     /* a bounded device-side wait in the placement scan expired */
        ZCCL_E_DEGENERATE = -7,  /* REL bound on an input whose range is zero (use ZCCL_EB_ABS) */
+       ZCCL_E_TOO_LARGE = -8,   /* more elements than the fixed scratch of zccl_compress_noalloc can place */
        ZCCL_W_PRECISION = 1 };  /* some |code| > 2^15: fp32 rounding may exceed eb_abs by about |x| * 1.8e-7 */
 
 /* Flags of the reduce hop and of zccl_sim_allreduce. */
 enum { ZCCL_CONSISTENT_OWNER = 1u };  /* owner's copy of a reduced chunk = dequantised value, not the raw sum */
 
-enum { ZCCL_TILE = 4096, ZCCL_BLOCK = 32, ZCCL_HEADER_BYTES = 32, ZCCL_MAX_RANKS = 64 };
+enum { ZCCL_TILE = 4096, ZCCL_BLOCK = 32, ZCCL_HEADER_BYTES = 32, ZCCL_MAX_RANKS = 64,
+       ZCCL_NOALLOC_MAX_ELEMS = 1 << 26 };  /* element limit of zccl_compress_noalloc (256 MiB of fp32) */
 
 /*
  * Context: look-back scan workspace for streams of up to `max_elems` elements, the device status word, the
@@ -129,6 +131,26 @@ int zccl_decompress_reduce_compress(zccl_ctx* ctx, const void* in_c, size_t in_b
                                     const float* local, const void* local_c, size_t local_c_bytes_max, size_t n,
                                     void* out_c, size_t out_capacity, size_t* out_bytes,
                                     float* raw_out, unsigned flags, void* stream);
+
+/*
+ * zccl_compress for callers that cannot allocate device memory (the paper has no counterpart: this is an addition
+ * of this library).  Work captured into a CUDA graph or running where an allocation would synchronise or is not
+ * allowed, plug-ins living inside a host application's fixed memory budget, and out-of-memory or teardown
+ * handlers cannot call zccl_ctx_create, because it calls cudaMalloc.  This entry point needs no context: its
+ * placement-scan workspace is a fixed array inside the library (about 129 KiB of device memory on every GPU that
+ * loads the library, until the process exits), and it calls no cudaMalloc, cudaFree or other allocating routine.
+ *   x, out, out_capacity, out_bytes [device], stream: as in zccl_compress;  eb_abs: absolute error bound
+ *   n: at most ZCCL_NOALLOC_MAX_ELEMS, else ZCCL_E_TOO_LARGE is returned and nothing is enqueued
+ * Produces the same bytes as zccl_compress(ctx, x, n, ZCCL_EB_ABS, eb_abs, ...).  There is no status word to read:
+ * if the device detects an error (capacity overrun, value out of range) *out_bytes is set to 0 and the contents of
+ * `out` are unspecified; the precision warning is not reported.
+ * The first call on a device looks up the array's device address and initialises it with one small asynchronous
+ * copy on `stream`; make that first call outside any stream capture.  All calls on a device share the array, which
+ * keeps the previous call's contents (each call re-arms what it needs): calls whose kernels could overlap on the
+ * GPU, for example on two streams, race and must be ordered by the caller.
+ */
+int zccl_compress_noalloc(const float* x, size_t n, float eb_abs, void* out, size_t out_capacity,
+                          size_t* out_bytes, void* stream);
 
 /*
  * Ring Allreduce (sum) over nranks rank buffers in this GPU's memory (Section 3.5: ring reduce-scatter in the

@@ -172,6 +172,7 @@ const char* zccl_strerror(int code)
         case ZCCL_E_BAD_STREAM: return "malformed compressed stream";
         case ZCCL_E_TIMEOUT: return "placement scan timed out";
         case ZCCL_E_DEGENERATE: return "degenerate value range or step";
+        case ZCCL_E_TOO_LARGE: return "more elements than the allocation-free entry point supports";
         case ZCCL_W_PRECISION: return "warning: codes beyond 2^15, bound may be exceeded by fp32 rounding";
         default: return "unknown status";
     }

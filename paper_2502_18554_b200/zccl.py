@@ -13,6 +13,8 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libzccl.so"
 
 OK, E_ARG, E_CUDA, E_CAPACITY, E_RANGE, E_BAD_STREAM, E_TIMEOUT, E_DEGENERATE, W_PRECISION = 0, -1, -2, -3, -4, -5, -6, -7, 1
+E_TOO_LARGE = -8
+NOALLOC_MAX_ELEMS = 1 << 26
 EB_ABS, EB_REL = 0, 1
 CONSISTENT_OWNER = 1
 TILE, BLOCK, HEADER_BYTES = 4096, 32, 32
@@ -21,7 +23,7 @@ EXPORTS = [
     "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_sizes",
-    "zccl_compress_host", "zccl_decompress_host",
+    "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc",
 ]
 
 _lib = None
@@ -62,6 +64,7 @@ def lib():
         L.zccl_sim_sizes.argtypes = [vp, vp, C.c_int, vp]
         L.zccl_compress_host.argtypes = [vp, vp, sz, C.c_int, C.c_float, vp, sz, vp, vp]
         L.zccl_decompress_host.argtypes = [vp, vp, sz, vp, sz, vp]
+        L.zccl_compress_noalloc.argtypes = [vp, sz, C.c_float, vp, sz, vp, vp]
         _lib = L
     return _lib
 
@@ -93,6 +96,17 @@ def _dev_ptr(t: torch.Tensor | None, dtype=None) -> int | None:
 def _check(rc: int, what: str):
     if rc != OK:
         raise ZcclError(rc, what)
+
+
+def compress_noalloc(x: torch.Tensor, eb_abs: float, out: torch.Tensor, out_bytes: torch.Tensor, stream=None,
+                     n: int | None = None) -> int:
+    """zccl_compress_noalloc: compression without a context, for callers that must not allocate device memory (its
+    scan workspace is a fixed array inside the library).  Returns the host-side status code instead of raising,
+    so that callers can tell ZCCL_E_TOO_LARGE from other errors."""
+    n = x.numel() if n is None else n
+    return int(lib().zccl_compress_noalloc(_dev_ptr(x, torch.float32) if x.numel() else None, n, eb_abs,
+                                           _dev_ptr(out, torch.uint8), out.numel(), _dev_ptr(out_bytes, torch.int64),
+                                           _stream_ptr(stream)))
 
 
 class Context:
