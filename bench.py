@@ -48,6 +48,22 @@ def step_units_bytes() -> dict:
     return {"compress": full, "decompress": full, "fused": full, "allreduce": ar, "allgather": ag}
 
 
+def max_over_ranks(value: float, device="cpu") -> float:
+    """Slowest rank's time: the job is as slow as its slowest replica."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_rank_step: float, world: int, ms_per_step: float) -> float:
+    """Aggregate throughput of `world` replicas that each process bytes_per_rank_step in ms_per_step."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
 def make_fields(rank: int):
     from paper_2502_18554_b200 import fields
     x = fields.fourier_field_3d(SIDE, seed=1 + 10 * rank)
@@ -155,12 +171,17 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    ref = args.impl == "reference"
+    if args.steps is None:
+        args.steps = 20 if ref else 1000    # the oracle needs about 0.4 s per step, the GPU under 1 ms
+    if args.warmup is None:
+        args.warmup = 2 if ref else 10
+    if ref:
         return reference_arm(args)
     if args.warmup < 3:
         args.warmup = 3
@@ -254,15 +275,11 @@ def main():
     launches = z.launch_count() - launches0
     clocks = sampler.stop()
     ctx.check()
-    ms_total = t_begin.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(t_begin.elapsed_time(t_end), dev)
     ms_step = ms_total / args.steps
     units = step_units_bytes()
     total_bytes = sum(units.values())
-    value = world * total_bytes / (ms_step * 1e-3) / 1e9
+    value = whole_job_gbs(total_bytes, world, ms_step)
 
     op_ms = {nm: statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps))
              for j, nm in enumerate(names)}
@@ -330,13 +347,8 @@ def main():
         ctx.decompress_host(oh, nb, yh)
     e1.record(stream)
     fence()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_ms /= e2e_steps
-    e2e = {"value": world * 2 * in_b / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dev) / e2e_steps
+    e2e = {"value": whole_job_gbs(2 * in_b, world, e2e_ms), "unit": "GB/s",
            "what": "zccl_compress_host + zccl_decompress_host of the 64 MiB batch (uncompressed bytes per op / time)",
            "ms_per_step": e2e_ms, "h2d_bytes_per_step": in_b + nb, "d2h_bytes_per_step": nb + 8 + in_b}
 

@@ -84,6 +84,14 @@ int zccl_status(zccl_ctx* ctx, void* stream);
  * no paper counterpart).  Pure host function. */
 unsigned long long zccl_launch_count(void);
 
+/*
+ * Test hook for the bounded waits of the placement scan (failure detection; no paper counterpart).  While set,
+ * the encoders do not publish the size of tile number `tile` of a launch, so the tiles after it find nothing to
+ * wait for: their look-back gives up after its poll limit (a fraction of a second), writes nothing for those tiles
+ * and records ZCCL_E_TIMEOUT; the context stays usable.  tile < 0 switches the hook off (the default).
+ */
+int zccl_debug_skip_publish(zccl_ctx* ctx, long long tile);
+
 /* Static description of a status code. */
 const char* zccl_strerror(int code);
 

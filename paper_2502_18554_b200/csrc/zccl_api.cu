@@ -210,6 +210,7 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
         c->ws.params = (Params*)(sm + 4);
         c->ws.minmax = sm + 8;
         c->ws.max_tiles = (uint32_t)max_tiles;
+        c->ws.skip_publish = 0xFFFFFFFFu;
         c->sim_sizes = (size_t*)(b + off_sizes);
         c->stage_bytes = c->sim_sizes + c->sim_sizes_cap;
         const uint32_t init[3] = {1u, 0xFFFFFFFFu, 0u};   // epoch, min key, max key
@@ -255,6 +256,13 @@ int zccl_status(zccl_ctx* c, void* stream)
     if (bits & kStRange) return ZCCL_E_RANGE;
     if (bits & kStCapacity) return ZCCL_E_CAPACITY;
     if (bits & kStPrecision) return ZCCL_W_PRECISION;
+    return ZCCL_OK;
+}
+
+int zccl_debug_skip_publish(zccl_ctx* c, long long tile)
+{
+    if (!c) return ZCCL_E_ARG;
+    c->ws.skip_publish = (tile < 0 || tile >= 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)tile;
     return ZCCL_OK;
 }
 

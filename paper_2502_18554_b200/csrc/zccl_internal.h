@@ -46,6 +46,7 @@ struct Workspace {
     Params* params;                  // resolved bound for REL mode
     uint32_t* minmax;                // two ordered-int keys: running min and max
     uint32_t max_tiles;
+    uint32_t skip_publish;           // test hook: tile number whose size is never published (0xFFFFFFFF = off)
 };
 
 // One chunk-operation.  Encoding jobs (compress, fused hop) and decoding jobs share the struct.

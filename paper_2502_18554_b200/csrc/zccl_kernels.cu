@@ -789,7 +789,8 @@ __device__ __forceinline__ void announce(const uint32_t* warp_words, const Works
     }
     c.wbase = wbase;
     c.total = total;
-    if (tid == 0) st_state(ws.tile_state + c.ticket, pack_state(epoch, c.tile == 0 ? 1u : 0u, total));
+    if (tid == 0 && c.ticket != ws.skip_publish)
+        st_state(ws.tile_state + c.ticket, pack_state(epoch, c.tile == 0 ? 1u : 0u, total));
 }
 
 // Places a pending tile: exclusive prefix by look-back, then copy-out, index entry, header and stream length.
@@ -805,7 +806,7 @@ __device__ __forceinline__ void place(const Pending& c, const JobBatch& jb, Look
 #else
         excl = look_back_cta(look, look_par, ws, c.ticket, job.tile_begin, epoch, warp, lane, skip, status);
 #endif
-        if (tid == 0) st_state(ws.tile_state + c.ticket, pack_state(epoch, 1u, excl + c.total));
+        if (tid == 0 && c.ticket != ws.skip_publish) st_state(ws.tile_state + c.ticket, pack_state(epoch, 1u, excl + c.total));
     }
     const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + c.nT + excl;
     const bool fits = (blob_word0 + c.total) * 4ull <= job.out_cap;

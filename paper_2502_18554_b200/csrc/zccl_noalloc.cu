@@ -57,6 +57,7 @@ Workspace workspace_at(unsigned char* base)
     ws.params = reinterpret_cast<Params*>(sm + 4);
     ws.minmax = sm + 8;
     ws.max_tiles = (uint32_t)kMaxTiles;
+    ws.skip_publish = 0xFFFFFFFFu;
     return ws;
 }
 

@@ -23,7 +23,7 @@ EXPORTS = [
     "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_sizes",
-    "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc",
+    "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
 ]
 
 _lib = None
@@ -65,6 +65,7 @@ def lib():
         L.zccl_compress_host.argtypes = [vp, vp, sz, C.c_int, C.c_float, vp, sz, vp, vp]
         L.zccl_decompress_host.argtypes = [vp, vp, sz, vp, sz, vp]
         L.zccl_compress_noalloc.argtypes = [vp, sz, C.c_float, vp, sz, vp, vp]
+        L.zccl_debug_skip_publish.argtypes = [vp, C.c_longlong]
         _lib = L
     return _lib
 
@@ -142,6 +143,10 @@ class Context:
         if rc < 0 or (rc > 0 and not allow_warning):
             raise ZcclError(rc, "device status")
         return rc
+
+    def debug_skip_publish(self, tile: int):
+        """Test hook: tile number whose size is never published to the placement scan (negative = off)."""
+        _check(lib().zccl_debug_skip_publish(self._h, tile), "zccl_debug_skip_publish")
 
     # ---- codec
     def compress(self, x: torch.Tensor, eb_mode: int, eb: float, out: torch.Tensor, out_bytes: torch.Tensor,

@@ -373,3 +373,23 @@ def test_host_buffer_forms(z, ctx):
     torch.cuda.synchronize()
     assert ctx.status() == z.OK
     assert_same_bits(yh.numpy(), oracle.decompress(want))
+
+
+def test_look_back_wait_is_bounded(z):
+    # a tile whose size is never published: the tiles after it give up after their poll limit, report a time-out
+    # and write nothing; no hang, and the context works again afterwards
+    ctx = z.Context(1 << 20, 0)
+    x = fields.smooth_1d(5 * 4096, seed=33)
+    dx = dev(x)
+    want, _ = oracle.compress(x, oracle.EB_REL, 1e-3)
+    out = torch.full((z.compress_bound(x.size) + 64,), 0x5A, dtype=torch.uint8, device="cuda")
+    nbytes = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx.debug_skip_publish(1)
+    ctx.compress(dx, z.EB_REL, 1e-3, out[: z.compress_bound(x.size)], nbytes)
+    assert ctx.status() == z.E_TIMEOUT
+    assert bool((out[z.compress_bound(x.size):] == 0x5A).all())
+    ctx.debug_skip_publish(-1)
+    ctx.compress(dx, z.EB_REL, 1e-3, out[: z.compress_bound(x.size)], nbytes)
+    assert ctx.status() == z.OK
+    assert np.array_equal(out[: int(nbytes.item())].cpu().numpy(), want)
+    ctx.close()
