@@ -101,75 +101,42 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// Per-block plane code.  The number of bit planes of a block is warp-uniform, so both coders jump (brx.idx.uni)
-// into a straight line of per-plane steps and fall through to plane 0: no compare tree, no per-plane branch.
-//   decoder: plane word (broadcast load from the staged blob) AND this lane's bit -> predicated add of 2^k; the sign
-//            word negates.  addr = shared-memory byte address of the block's payload (sign word first).
-//   encoder: (|delta| AND 2^k) != 0 -> ballot -> the same word stored by every lane at slot + 4 (k + 1); the sign
-//            word goes to slot + 0.  slot = shared-memory byte address.
-#define ZCCL_DEC_BLOCK_ASM(mag, L, addr, lanebit)                                  \
-    asm volatile("{\n\t"                                                              \
-                 ".reg .pred p;\n\t.reg .b32 w, d;\n\t"                                \
-                 "ts: .branchtargets T0, T1, T2, T3, T4, T5, T6, T7, T8, T9, T10, T11, T12, T13, T14, T15, T16, T17, T18, T19, T20, T21, T22, T23;\n\t"  \
-                 "brx.idx.uni %1, ts;\n\t"                                           \
-                 "T23: ld.shared.u32 w, [%2+92];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f4A800000;\n\t" \
-                 "T22: ld.shared.u32 w, [%2+88];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f4A000000;\n\t" \
-                 "T21: ld.shared.u32 w, [%2+84];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f49800000;\n\t" \
-                 "T20: ld.shared.u32 w, [%2+80];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f49000000;\n\t" \
-                 "T19: ld.shared.u32 w, [%2+76];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f48800000;\n\t" \
-                 "T18: ld.shared.u32 w, [%2+72];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f48000000;\n\t" \
-                 "T17: ld.shared.u32 w, [%2+68];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f47800000;\n\t" \
-                 "T16: ld.shared.u32 w, [%2+64];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f47000000;\n\t" \
-                 "T15: ld.shared.u32 w, [%2+60];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f46800000;\n\t" \
-                 "T14: ld.shared.u32 w, [%2+56];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f46000000;\n\t" \
-                 "T13: ld.shared.u32 w, [%2+52];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f45800000;\n\t" \
-                 "T12: ld.shared.u32 w, [%2+48];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f45000000;\n\t" \
-                 "T11: ld.shared.u32 w, [%2+44];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f44800000;\n\t" \
-                 "T10: ld.shared.u32 w, [%2+40];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f44000000;\n\t" \
-                 "T9: ld.shared.u32 w, [%2+36];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f43800000;\n\t" \
-                 "T8: ld.shared.u32 w, [%2+32];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f43000000;\n\t" \
-                 "T7: ld.shared.u32 w, [%2+28];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f42800000;\n\t" \
-                 "T6: ld.shared.u32 w, [%2+24];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f42000000;\n\t" \
-                 "T5: ld.shared.u32 w, [%2+20];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f41800000;\n\t" \
-                 "T4: ld.shared.u32 w, [%2+16];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f41000000;\n\t" \
-                 "T3: ld.shared.u32 w, [%2+12];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f40800000;\n\t" \
-                 "T2: ld.shared.u32 w, [%2+8];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f40000000;\n\t" \
-                 "T1: ld.shared.u32 w, [%2+4];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p add.rn.f32 %0, %0, 0f3F800000;\n\t" \
-                 "ld.shared.u32 w, [%2];\n\tand.b32 d, w, %3;\n\tsetp.ne.u32 p, d, 0;\n\t@p neg.f32 %0, %0;\n\t" \
-                 "T0:\n\t}"                                                          \
-                 : "+f"(mag) : "r"(L), "r"(addr), "r"(lanebit) : "memory")
-
-#define ZCCL_ENC_BLOCK_ASM(ab, L, sg, slot)                                        \
-    asm volatile("{\n\t"                                                              \
-                 ".reg .pred p;\n\t.reg .b32 w, d;\n\t"                                \
-                 "ts: .branchtargets T0, T1, T2, T3, T4, T5, T6, T7, T8, T9, T10, T11, T12, T13, T14, T15, T16, T17, T18, T19, T20, T21, T22, T23;\n\t"  \
-                 "brx.idx.uni %1, ts;\n\t"                                           \
-                 "T23: and.b32 d, %0, 4194304;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+92], w;\n\t" \
-                 "T22: and.b32 d, %0, 2097152;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+88], w;\n\t" \
-                 "T21: and.b32 d, %0, 1048576;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+84], w;\n\t" \
-                 "T20: and.b32 d, %0, 524288;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+80], w;\n\t" \
-                 "T19: and.b32 d, %0, 262144;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+76], w;\n\t" \
-                 "T18: and.b32 d, %0, 131072;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+72], w;\n\t" \
-                 "T17: and.b32 d, %0, 65536;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+68], w;\n\t" \
-                 "T16: and.b32 d, %0, 32768;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+64], w;\n\t" \
-                 "T15: and.b32 d, %0, 16384;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+60], w;\n\t" \
-                 "T14: and.b32 d, %0, 8192;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+56], w;\n\t" \
-                 "T13: and.b32 d, %0, 4096;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+52], w;\n\t" \
-                 "T12: and.b32 d, %0, 2048;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+48], w;\n\t" \
-                 "T11: and.b32 d, %0, 1024;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+44], w;\n\t" \
-                 "T10: and.b32 d, %0, 512;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+40], w;\n\t" \
-                 "T9: and.b32 d, %0, 256;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+36], w;\n\t" \
-                 "T8: and.b32 d, %0, 128;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+32], w;\n\t" \
-                 "T7: and.b32 d, %0, 64;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+28], w;\n\t" \
-                 "T6: and.b32 d, %0, 32;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+24], w;\n\t" \
-                 "T5: and.b32 d, %0, 16;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+20], w;\n\t" \
-                 "T4: and.b32 d, %0, 8;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+16], w;\n\t" \
-                 "T3: and.b32 d, %0, 4;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+12], w;\n\t" \
-                 "T2: and.b32 d, %0, 2;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+8], w;\n\t" \
-                 "T1: and.b32 d, %0, 1;\n\tsetp.ne.u32 p, d, 0;\n\tvote.sync.ballot.b32 w, p, 0xffffffff;\n\tst.shared.u32 [%3+4], w;\n\t" \
-                 "st.shared.u32 [%3], %2;\n\t"                                       \
-                 "T0:\n\t}"                                                          \
-                 :: "r"(ab), "r"(L), "r"(sg), "r"(slot) : "memory")
+// Bit planes by a 32 x 32 bit-matrix transpose across the warp.  Lane j holds the word of element j (bit k =
+// bit k of |delta_j|, bit 31 = its sign); after the transpose lane k holds plane k (bit j = that bit of element j)
+// and lane 31 the sign word.  Five butterfly stages exchange bit-index bit b with lane-index bit b (b = 4..0): one
+// shuffle plus a byte permute (strides 16, 8) or a rotate and a bit select (strides 4, 2, 1).  The transpose is
+// its own inverse, so the decoder uses the same routine.  Cost does not depend on the code length, and there is no
+// branch, so neighbouring blocks interleave.
+struct Xpose {
+    uint32_t sel16, sel8, m4, m2, m1, a4, a2, a1;
+    __device__ __forceinline__ explicit Xpose(int lane)
+    {
+        sel16 = (lane & 16) ? 0x3276u : 0x5410u;
+        sel8 = (lane & 8) ? 0x3715u : 0x6240u;
+        m4 = (lane & 4) ? 0xF0F0F0F0u : 0x0F0F0F0Fu;
+        m2 = (lane & 2) ? 0xCCCCCCCCu : 0x33333333u;
+        m1 = (lane & 1) ? 0xAAAAAAAAu : 0x55555555u;
+        a4 = (lane & 4) ? 28u : 4u;
+        a2 = (lane & 2) ? 30u : 2u;
+        a1 = (lane & 1) ? 31u : 1u;
+        // hide the values' origin from the compiler: it would otherwise recompute the selects at every use
+        asm volatile("" : "+r"(sel16), "+r"(sel8), "+r"(m4), "+r"(m2), "+r"(m1), "+r"(a4), "+r"(a2), "+r"(a1));
+    }
+    __device__ __forceinline__ uint32_t operator()(uint32_t x) const
+    {
+        uint32_t y = __shfl_xor_sync(kFull, x, 16);
+        x = __byte_perm(x, y, sel16);
+        y = __shfl_xor_sync(kFull, x, 8);
+        x = __byte_perm(x, y, sel8);
+        y = __shfl_xor_sync(kFull, x, 4);
+        x = (x & m4) | (__funnelshift_l(y, y, a4) & ~m4);
+        y = __shfl_xor_sync(kFull, x, 2);
+        x = (x & m2) | (__funnelshift_l(y, y, a2) & ~m2);
+        y = __shfl_xor_sync(kFull, x, 1);
+        x = (x & m1) | (__funnelshift_l(y, y, a1) & ~m1);
+        return x;
+    }
+};
 
 __device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
 {
@@ -382,18 +349,23 @@ __device__ __forceinline__ void decode_blocks_int(const TileDesc& d, int warp, i
 // fp32 path: rebuilds this warp's 16 blocks of deltas from the staged blob and stores them, as exact floats, in
 // the warp's 512-word region `wbuf`, row i = block i, element j of a row at word j ^ ((i & 3) << 2) (so that the
 // 128-bit reads of decode_scan_f32 are free of bank conflicts).  tbl: per block {code length, payload address}.
-__device__ __forceinline__ void decode_blocks_f32(const uint2* __restrict__ tbl, float* __restrict__ wbuf, int lane)
+__device__ __forceinline__ void decode_blocks_f32(const uint2* __restrict__ tbl, float* __restrict__ wbuf, int lane,
+                                                  const Xpose& xp)
 {
-    const uint32_t lanebit = 1u << lane;
+    const uint32_t widx = (uint32_t)(lane + 1) & 31u;   // lane k fetches plane k (word k + 1), lane 31 the sign word
 #pragma unroll 1
     for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int i = 4 * g + u;
             const uint2 e = tbl[i];               // broadcast read: code length, shared address of the payload
-            float mag = 0.0f;
-            ZCCL_DEC_BLOCK_ASM(mag, e.x, e.y, lanebit);
-            wbuf[32 * i + (lane ^ (u << 2))] = mag;
+            const uint32_t sz = e.x ? e.x + 1 : 0;
+            uint32_t w = 0;
+            if (widx < sz) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(e.y + 4 * widx) : "memory");
+            const uint32_t v = xp(w);             // bits 0..L-1: |delta| of this lane's element, bit 31: its sign
+            // exact fp32 value of the magnitude from its bits (|delta| < 2^23), then the sign bit on top
+            const float mag = __fsub_rn(__uint_as_float((v & 0x007FFFFFu) | 0x4B000000u), kTwo23);
+            wbuf[32 * i + (lane ^ (u << 2))] = __uint_as_float(__float_as_uint(mag) | (v & 0x80000000u));
         }
     }
 }
@@ -447,13 +419,14 @@ struct DecodeShared {
     alignas(8) unsigned long long bar;
 };
 
-__global__ void __launch_bounds__(kThreads, 6) decode_kernel(JobBatch jb, Workspace ws)
+__global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Workspace ws)
 {
     __shared__ DecodeShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t status = 0;
     uint32_t fills = 0;    // bulk copies completed on sh.bar (its phase parity)
     uint32_t par = 0;      // parity of the warp_total double buffer
+    const Xpose xp(lane);
     if (tid == 0) {
         mbar_init(&sh.bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -490,7 +463,7 @@ __global__ void __launch_bounds__(kThreads, 6) decode_kernel(JobBatch jb, Worksp
             const bool landed = mbar_wait(&sh.bar, fills & 1u);
             ++fills;
             if (!landed) status |= kStTimeout;   // carry on with whatever is staged: reads stay inside shared memory
-            decode_blocks_f32(sh.tbl[warp], sh.wbuf[warp], lane);
+            decode_blocks_f32(sh.tbl[warp], sh.wbuf[warp], lane, xp);
             __syncwarp();
             float v[16];
             const float total = decode_scan_f32(sh.wbuf[warp], lane, v);
@@ -575,17 +548,17 @@ struct SrcSwizzled {        // the fused kernel's sum tile: per-warp region of 1
 };
 
 // One pass over this warp's 16 blocks: quantise, 1-D Lorenzo delta, code length, sign word and bit planes, appended
-// to the warp's region of shared memory (every lane stores the same warp-uniform word: no predicate, one
-// wavefront).  Returns the warp's payload size in words; lane g (g < 4) ends up holding the code-length word of
-// blocks 4g..4g+3 in `my_lw`.  FAST: fp32 arithmetic, valid while every |x * r| < 2^21.5; the caller
-// checks `guard` (sum of squares of x * r) and reruns with FAST = false when it is too large.
+// to the warp's region of shared memory.  Returns the warp's payload size in words; lane g (g < 4) ends up holding
+// the code-length word of blocks 4g..4g+3 in `my_lw`.  FAST: fp32 arithmetic, valid while every |x * r| < 2^21.5;
+// the caller checks `guard` (sum of squares of x * r) and reruns with FAST = false when it is too large.
 template <bool FAST, class Src>
 __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint32_t* __restrict__ slots_w, int lane,
-                                                  uint32_t& my_lw, int32_t& q_first, float& guard, float& tmax)
+                                                  const Xpose& xp, uint32_t& my_lw, float& guard, float& tmax)
 {
     uint32_t wsum = 0;
     float acc = 0.0f, tm = 0.0f;
     my_lw = 0;
+    const uint32_t widx = (uint32_t)(lane + 1) & 31u;   // lane k stores plane k at word k + 1, lane 31 the sign word at 0
 #pragma unroll 1
     for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
         uint32_t lword = 0;
@@ -593,35 +566,35 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
         for (int u = 0; u < 4; ++u) {
             const float xv = src.cur(g, u), pv = src.prev(g, u);
             const float t = __fmul_rn(xv, r), tp = __fmul_rn(pv, r);
-            uint32_t ab, sg, L;
+            uint32_t L;
             if (FAST) {
                 acc = __fmaf_rn(t, t, acc);
                 acc = __fmaf_rn(tp, tp, acc);
                 const float c = __fadd_rn(t, kRoundMagic), cp = __fadd_rn(tp, kRoundMagic);
                 const float df = __fsub_rn(c, cp);
-                if (u == 0 && g == 0) q_first = (int32_t)(__float_as_uint(c) - kRoundMagicBits);
-                ab = __float_as_uint(__fadd_rn(fabsf(df), kTwo23));
+                const uint32_t ab = __float_as_uint(__fadd_rn(fabsf(df), kTwo23));
                 const uint32_t m = __reduce_or_sync(kFull, ab) & 0x7FFFFFu;
                 L = 32u - (uint32_t)__clz((int)m);
-                sg = __ballot_sync(kFull, df < 0.0f);
+                if (L) {   // uniform over the warp
+                    // magnitude in bits 0..22 (bits 23..30 hold exponent bits: never stored, L <= 23), sign in bit 31
+                    const uint32_t v = xp(ab | (__float_as_uint(df) & 0x80000000u));
+                    if (widx <= L) slots_w[wsum + widx] = v;
+                    wsum += L + 1;
+                }
             } else {
                 tm = fmaxf(tm, fabsf(t));
                 const int32_t q = __float2int_rn(t), qp = __float2int_rn(tp);
                 const int32_t dd = q - qp;
-                if (u == 0 && g == 0) q_first = q;
-                ab = (uint32_t)(dd < 0 ? -dd : dd);
+                const uint32_t ab = (uint32_t)(dd < 0 ? -dd : dd);
                 const uint32_t m = __reduce_or_sync(kFull, ab);
                 L = 32u - (uint32_t)__clz((int)m);
-                sg = __ballot_sync(kFull, dd < 0);
-            }
-            if (L) {   // uniform over the warp
-                uint32_t* slot = slots_w + wsum;
-                uint32_t Lj = L;
-                if (!FAST) {   // planes beyond the jump table (integer path only)
-                    for (; Lj > 23; --Lj) slot[Lj] = __ballot_sync(kFull, ab & (1u << (Lj - 1)));
+                const uint32_t sg = __ballot_sync(kFull, dd < 0);
+                if (L) {
+                    uint32_t* slot = slots_w + wsum;
+                    slot[0] = sg;   // every lane stores the same warp-uniform word
+                    for (uint32_t k = 0; k < L; ++k) slot[k + 1] = __ballot_sync(kFull, ab & (1u << k));
+                    wsum += L + 1;
                 }
-                ZCCL_ENC_BLOCK_ASM(ab, Lj, sg, smem_u32(slot));
-                wsum += L + 1;
             }
             lword |= L << (8 * u);
         }
@@ -632,10 +605,18 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
     return wsum;
 }
 
-constexpr int kLookWindows = 16;   // windows of 32 scan states inspected per look-back iteration (2 per warp)
+// The tile's outlier: the quantised code of its first element (thread 0 only needs it).
+template <bool FAST>
+__device__ __forceinline__ int32_t first_code(float x0, float r)
+{
+    const float t = __fmul_rn(x0, r);
+    if (FAST) return (int32_t)(__float_as_uint(__fadd_rn(t, kRoundMagic)) - kRoundMagicBits);
+    return __float2int_rn(t);
+}
+
 struct LookShared {
-    uint32_t sum[2][kLookWindows];
-    uint32_t st[2][kLookWindows];     // 0: 32 aggregates, 1: reached an inclusive prefix, 2: met a state not yet published
+    uint32_t part[2][kWarps];   // per-warp partial sums of tile sizes
+    uint32_t ok[2][kWarps];     // 1 if every state the warp inspected was published
 };
 
 struct EncodeShared {
@@ -666,56 +647,41 @@ __device__ __forceinline__ bool stageable_raw(const Job& job, uint32_t tile)
     return job.n - start >= (unsigned long long)kTile && (((uintptr_t)(job.x + start)) & 15u) == 0;
 }
 
-// Placement: decoupled look-back over the preceding tiles of this job, run by the whole CTA.  Each iteration
-// inspects the 512 nearest predecessors (16 windows of 32 states, two per warp); the windows are combined in order
-// until the first inclusive prefix.  Returns the exclusive prefix in words (same value in every thread); sets
-// `skip` when the bounded wait expired.
-
-__device__ __forceinline__ uint32_t look_back_cta(LookShared& ls, uint32_t& par, const Workspace& ws, uint32_t ticket,
-                                                  uint32_t tile_begin, uint32_t epoch, int warp, int lane, uint32_t& skip,
-                                                  uint32_t& status)
+// Placement: sum of the sizes of tiles [lo, hi) of the launch, run by the whole CTA (window w of 32 states is
+// inspected by warp w mod 8).  With round-robin tiles a CTA anchors the scan at its own previous tile, whose
+// inclusive prefix it knows, so it only ever needs plain sizes, at most one grid's worth of them, all fetched in one
+// round trip; nothing depends on another CTA having placed anything.  Returns the sum (same in every thread); sets
+// `skip` when a size stayed unpublished beyond the poll limit.
+__device__ __forceinline__ uint32_t sum_sizes_cta(LookShared& ls, uint32_t& par, const Workspace& ws, uint32_t lo, uint32_t hi,
+                                                  uint32_t epoch, int warp, int lane, uint32_t& skip, uint32_t& status)
 {
-    uint32_t excl = 0;
     skip = 0;
-    long long pos = (long long)ticket - 1;
-    const long long lo = (long long)tile_begin;
+    if (hi <= lo) return 0;
+    const uint32_t nwin = (hi - lo + 31u) >> 5;
     int budget = kSpinLimit >> 4;
     for (;;) {
-#pragma unroll
-        for (int hh = 0; hh < kLookWindows / kWarps; ++hh) {
-            const int w = warp + kWarps * hh;
-            const long long at = pos - 32 * w - lane;
-            unsigned long long st = pack_state(epoch, 1u, 0u);   // before the job's first tile: prefix 0
-            if (at >= lo) st = ld_state(ws.tile_state + at);
-            const bool valid = (uint32_t)(st >> 33) == epoch;
-            const uint32_t vmask = __ballot_sync(kFull, valid);
-            const uint32_t imask = __ballot_sync(kFull, valid && ((st >> 32) & 1ull));
-            const int first = imask ? (__ffs((int)imask) - 1) : 31;
-            const uint32_t need = (first == 31) ? kFull : ((2u << first) - 1u);
-            const uint32_t sum = __reduce_add_sync(kFull, (lane <= first) ? (uint32_t)st : 0u);
-            if (lane == 0) {
-                ls.sum[par][w] = sum;
-                ls.st[par][w] = ((vmask & need) != need) ? 2u : (imask ? 1u : 0u);
+        uint32_t sum = 0;
+        bool good = true;
+        for (uint32_t w = warp; w < nwin; w += kWarps) {
+            const uint32_t at = lo + 32u * w + lane;
+            if (at < hi) {
+                const unsigned long long st = ld_state(ws.tile_state + at);
+                if ((uint32_t)(st >> 33) == epoch) sum += (uint32_t)st;
+                else good = false;
             }
         }
+        sum = __reduce_add_sync(kFull, sum);
+        good = __all_sync(kFull, good);
+        if (lane == 0) { ls.part[par][warp] = sum; ls.ok[par][warp] = good ? 1u : 0u; }
         __syncthreads();
-        // combine the windows in order (lane w holds window w): stop at the first inclusive prefix, fail on a
-        // window that met an unpublished state before it
-        const uint32_t wst = lane < kLookWindows ? ls.st[par][lane] : 0u;
-        const uint32_t wsm = lane < kLookWindows ? ls.sum[par][lane] : 0u;
-        const uint32_t m_incl = __ballot_sync(kFull, wst == 1u);
-        const uint32_t m_block = __ballot_sync(kFull, wst == 2u);
-        const int fw = m_incl ? (__ffs((int)m_incl) - 1) : (kLookWindows - 1);
-        const uint32_t upto = (2u << fw) - 1u;
-        const uint32_t acc = __reduce_add_sync(kFull, (lane <= fw) ? wsm : 0u);
-        const uint32_t res = (m_block & upto) ? 2u : (m_incl ? 1u : 0u);
+        uint32_t total = 0, all_ok = 1;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { total += ls.part[par][w]; all_ok &= ls.ok[par][w]; }
         par ^= 1u;
-        if (res == 1u) { excl += acc; break; }
-        if (res == 0u) { excl += acc; pos -= 32 * kLookWindows; continue; }
-        if (--budget == 0) { skip = 1; status |= kStTimeout; break; }   // uniform: every thread reads the same words
+        if (all_ok) return total;
+        if (--budget == 0) { skip = 1; status |= kStTimeout; return 0; }   // uniform: every thread read the same words
         __nanosleep(64);
     }
-    return excl;
 }
 
 // Copies this warp's contiguous region to its place in the stream; writes the warp's code-length words.
@@ -761,66 +727,85 @@ __device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoc
 }
 
 // An encoded tile sitting in shared memory until its place in the stream is known.  Placement is deferred by one
-// tile: while a CTA encodes its next tile the sizes of the earlier tiles of all CTAs get published, so the
-// look-back of the deferred tile finds them without waiting.
+// tile: while a CTA encodes its next tile the sizes of the earlier tiles of all CTAs get published, so the scan of
+// the deferred tile finds them without waiting.
 struct Pending {
     bool valid;
     int job;
-    uint32_t ticket, tile, nT, padw;
-    uint32_t buf;        // which half of the slots holds it
+    uint32_t ticket;
+    uint32_t buf;        // which half of the slots (and of the warps' sizes) holds it
     uint32_t wsum;       // this warp's payload words
-    uint32_t wbase;      // this warp's offset inside the blob
-    uint32_t total;      // blob words
     uint32_t my_lw;      // lanes 0..3: this warp's code-length words
     int32_t q_first;     // outlier (thread 0)
-    float eb_abs, s;
 };
 
-// After the barrier that follows a tile's encoding pass: this warp's offset and the blob size from the warps'
-// sizes, and the tile's size published to the scan (as an inclusive prefix for a job's first tile).
-__device__ __forceinline__ void announce(const uint32_t* warp_words, const Workspace& ws, uint32_t epoch, Pending& c, int tid, int warp)
+// What a CTA remembers about the last tile it placed: the anchor of its next scan.
+struct Anchor {
+    int job;             // -1: none yet
+    uint32_t ticket;
+    uint32_t incl;       // inclusive prefix (words) of that tile within its job
+};
+
+// This warp's offset inside a tile's blob and the blob size, from the warps' payload sizes.
+__device__ __forceinline__ void blob_layout(const uint32_t* warp_words, uint32_t padw, int warp, uint32_t& wbase, uint32_t& total)
 {
-    uint32_t wbase = 1 + c.padw, total = 1 + c.padw;
+    wbase = 1 + padw;
+    total = 1 + padw;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) {
         const uint32_t ww = warp_words[w];
         if (w < warp) wbase += ww;
         total += ww;
     }
-    c.wbase = wbase;
-    c.total = total;
-    if (tid == 0 && c.ticket != ws.skip_publish)
-        st_state(ws.tile_state + c.ticket, pack_state(epoch, c.tile == 0 ? 1u : 0u, total));
 }
 
-// Places a pending tile: exclusive prefix by look-back, then copy-out, index entry, header and stream length.
-__device__ __forceinline__ void place(const Pending& c, const JobBatch& jb, LookShared& look, uint32_t& look_par,
-                                      const uint32_t* slots_w, const Workspace& ws, uint32_t epoch, int tid, int warp, int lane,
-                                      uint32_t& status)
+// After the barrier that follows a tile's encoding pass: the tile's size is published to the scan.
+__device__ __forceinline__ void announce(const uint32_t* warp_words, uint32_t padw, const Workspace& ws, uint32_t epoch,
+                                         uint32_t ticket, int tid)
+{
+    if (tid == 0 && ticket != ws.skip_publish) {
+        uint32_t total = 1 + padw;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) total += warp_words[w];
+        st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
+    }
+}
+
+// Places a pending tile: exclusive prefix = anchor + sizes of the tiles in between, then copy-out, index entry,
+// header and stream length.
+__device__ __forceinline__ void place(const Pending& c, Anchor& anchor, const JobBatch& jb, LookShared& look, uint32_t& look_par,
+                                      const uint32_t* warp_words, const uint32_t* slots_w, float eb_abs, float s,
+                                      const Workspace& ws, uint32_t epoch, int tid, int warp, int lane, uint32_t& status)
 {
     const Job& job = jb.job[c.job];
-    uint32_t excl = 0, skip = 0;
-    if (c.tile != 0) {
+    const uint32_t tile = c.ticket - job.tile_begin;
+    const unsigned long long start = (unsigned long long)tile * kTile;
+    const uint32_t nT = (uint32_t)((job.n + kTile - 1) / kTile);
+    const uint32_t len = (uint32_t)((job.n - start < (unsigned long long)kTile) ? (job.n - start) : kTile);
+    const uint32_t padw = (((len + kBlock - 1) / kBlock) + 3) >> 2;
+    uint32_t wbase, total;
+    blob_layout(warp_words, padw, warp, wbase, total);
+    uint32_t lo = job.tile_begin, base = 0, skip = 0;
+    if (anchor.job == c.job) { lo = anchor.ticket + 1; base = anchor.incl; }
 #ifdef ZCCL_DEBUG_NO_LOOKBACK
-        excl = c.tile * 700u;
+    const uint32_t excl = tile * 700u;
 #else
-        excl = look_back_cta(look, look_par, ws, c.ticket, job.tile_begin, epoch, warp, lane, skip, status);
+    const uint32_t excl = base + sum_sizes_cta(look, look_par, ws, lo, c.ticket, epoch, warp, lane, skip, status);
 #endif
-        if (tid == 0 && c.ticket != ws.skip_publish) st_state(ws.tile_state + c.ticket, pack_state(epoch, 1u, excl + c.total));
-    }
-    const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + c.nT + excl;
-    const bool fits = (blob_word0 + c.total) * 4ull <= job.out_cap;
+    anchor.job = c.job; anchor.ticket = c.ticket; anchor.incl = excl + total;
+    const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
+    const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
     if (!fits) status |= kStCapacity;
     if (fits && !skip) {
         uint32_t* blob_out = job.out + blob_word0;
-        copy_out_warp(blob_out, slots_w, c.wbase, c.wsum, c.my_lw, c.padw, warp, lane);
+        copy_out_warp(blob_out, slots_w, wbase, c.wsum, c.my_lw, padw, warp, lane);
         if (tid == 0) {
             blob_out[0] = (uint32_t)c.q_first;
-            job.out[kHeaderWords + c.tile] = excl + c.total;
+            job.out[kHeaderWords + tile] = excl + total;
         }
     }
-    if (c.tile == 0) write_header(job.out, tid, job.n, c.eb_abs, c.s, c.nT);
-    if (c.tile == c.nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + c.total) * 4ull);
+    if (tile == 0) write_header(job.out, tid, job.n, eb_abs, s, nT);
+    if (tile == nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
 }
 
 // ------------------------------------------------------------------------------------------------ compress
@@ -860,6 +845,9 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     uint32_t p = 0;        // half of the slots the current tile is encoded into
     Pending pend;
     pend.valid = false;
+    Anchor anchor;
+    anchor.job = -1; anchor.ticket = 0; anchor.incl = 0;
+    const Xpose xp(lane);
 
     for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += G) {
         const int j = find_job(jb, ticket);
@@ -872,7 +860,7 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         if (n == 0 || !prm.valid) {   // a job without elements still owns one tile number: header and length only
             const bool hdr = prm.valid && job.out_cap >= (unsigned)kHeaderBytes;
             if (tid == 0) {
-                st_state(ws.tile_state + ticket, pack_state(epoch, 1u, 0u));
+                st_state(ws.tile_state + ticket, pack_state(epoch, 0u, 0u));
                 if (tile == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
                 stage(ticket + G);   // nothing was staged for this tile, and the buffer's last readers are past a barrier
             }
@@ -896,7 +884,8 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
             if (!landed) status |= kStTimeout;   // carry on with whatever is staged: the result is flagged invalid
             if (tid == 0) xt[-1] = xt[0];        // the tile's first element is its own predecessor
             const SrcStaged src{xt + 512 * warp + lane};
-            wsum = encode_blocks<true>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+            wsum = encode_blocks<true>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
+            q_first = first_code<true>(src.cur(0, 0), r);
             need_int = __any_sync(kFull, !(guard < kGuardExact));
             if (!need_int && __any_sync(kFull, guard >= kGuardSmall)) {   // codes beyond 2^15 raise the warning
                 float tm = 0.0f;
@@ -909,7 +898,8 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         }
         if (need_int) {
             const SrcGlobal src{job.x + start, (uint32_t)(512 * warp + lane), len - 1};
-            wsum = encode_blocks<false>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+            wsum = encode_blocks<false>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
+            q_first = first_code<false>(src.cur(0, 0), r);
             if (!(tmax < 1073741824.0f)) status |= kStRange;
             else if (tmax > 32768.5f) status |= kStPrecision;
         }
@@ -917,17 +907,17 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         __syncthreads();   // sizes of all warps are visible; the staged tile has been consumed
         if (tid == 0) stage(ticket + G);   // overlaps with the placement of the previous tile below
 
-        Pending cur;
-        cur.valid = true; cur.job = j; cur.ticket = ticket; cur.tile = tile; cur.nT = nT; cur.padw = (nb + 3) >> 2;
-        cur.buf = p; cur.wsum = wsum; cur.my_lw = my_lw; cur.q_first = q_first; cur.eb_abs = eb_abs; cur.s = s;
-        announce(sh.warp_words[p], ws, epoch, cur, tid, warp);
+        announce(sh.warp_words[p], (nb + 3) >> 2, ws, epoch, ticket, tid);
         if (pend.valid)
-            place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
-        pend = cur;
+            place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
+                  sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, eb_abs, s, ws, epoch, tid, warp, lane, status);
+        pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
+        pend.q_first = q_first;
         p ^= 1u;
     }
     if (pend.valid)
-        place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
+        place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
+              sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, eb_abs, s, ws, epoch, tid, warp, lane, status);
 
     // never leave with a bulk copy in flight into this CTA's shared memory: every copy that was started has been
     // waited for by the iteration that consumed it, except after an expired wait; then give it one more bounded wait
@@ -953,8 +943,12 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     }
     __syncthreads();
     uint32_t look_par = 0, p = 0;
+    float pend_eb = 0.0f, pend_s = 1.0f;   // bound and step of the pending tile's job (header fields)
     Pending pend;
     pend.valid = false;
+    Anchor anchor;
+    anchor.job = -1; anchor.ticket = 0; anchor.incl = 0;
+    const Xpose xp(lane);
     int cur_job = -1;
     StreamInfo h1, h2;
     h1.ok = h2.ok = false; h1.n = h2.n = 0; h1.nT = h2.nT = 0; h1.s = h2.s = 1.0f; h1.eb_abs = h2.eb_abs = 0.0f;
@@ -982,7 +976,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             if (!job_ok) status |= kStBadStream;
             const bool hdr = job_ok && job.out_cap >= (unsigned)kHeaderBytes;
             if (tid == 0) {
-                st_state(ws.tile_state + ticket, pack_state(epoch, 1u, 0u));
+                st_state(ws.tile_state + ticket, pack_state(epoch, 0u, 0u));
                 if (tile == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
             }
             if (hdr && tile == 0) write_header(job.out, tid, 0, eb_abs, s, 0);
@@ -1002,7 +996,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         if (!d1.ok || !d2.ok) {   // uniform: keep the scan consistent for the tiles that follow, write nothing
             status |= kStBadStream;
             if (tid == 0) {
-                st_state(ws.tile_state + ticket, pack_state(epoch, tile == 0 ? 1u : 0u, 0u));
+                st_state(ws.tile_state + ticket, pack_state(epoch, 0u, 0u));
                 if (tile == nT - 1) *job.out_bytes = 0;
             }
             __syncthreads();
@@ -1043,7 +1037,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             const bool landed = mbar_wait(&sh.bar, fills & 1u);
             ++fills;
             if (!landed) status |= kStTimeout;
-            decode_blocks_f32(sh.tbl[warp], yrows + 32, lane);
+            decode_blocks_f32(sh.tbl[warp], yrows + 32, lane, xp);
             __syncwarp();
             float v[16];
             const float total = decode_scan_f32(yrows + 32, lane, v);
@@ -1124,10 +1118,12 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         int32_t q_first = 0;
         float guard = 0.0f, tmax = 0.0f;
         const SrcSwizzled src(yrows, lane);
-        wsum = encode_blocks<true>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+        wsum = encode_blocks<true>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
+            q_first = first_code<true>(src.cur(0, 0), r);
         const bool need_int = __any_sync(kFull, !(guard < kGuardExact));
         if (need_int) {
-            wsum = encode_blocks<false>(src, r, slots_w, lane, my_lw, q_first, guard, tmax);
+            wsum = encode_blocks<false>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
+            q_first = first_code<false>(src.cur(0, 0), r);
             if (!(tmax < 1073741824.0f)) status |= kStRange;
             else if (tmax > 32768.5f) status |= kStPrecision;
         } else if (__any_sync(kFull, guard >= kGuardSmall)) {
@@ -1150,17 +1146,18 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps
-        Pending cur;
-        cur.valid = true; cur.job = j; cur.ticket = ticket; cur.tile = tile; cur.nT = nT; cur.padw = padw;
-        cur.buf = p; cur.wsum = wsum; cur.my_lw = my_lw; cur.q_first = q_first; cur.eb_abs = eb_abs; cur.s = s;
-        announce(sh.warp_words[p], ws, epoch, cur, tid, warp);
+        announce(sh.warp_words[p], padw, ws, epoch, ticket, tid);
         if (pend.valid)
-            place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
-        pend = cur;
+            place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
+                  sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, pend_eb, pend_s, ws, epoch, tid, warp, lane, status);
+        pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
+        pend.q_first = q_first;
+        pend_eb = eb_abs; pend_s = s;
         p ^= 1u;
     }
     if (pend.valid)
-        place(pend, jb, sh.look, look_par, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, ws, epoch, tid, warp, lane, status);
+        place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
+              sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, pend_eb, pend_s, ws, epoch, tid, warp, lane, status);
     if (status) atomicOr(ws.status, status);
     finish_launch(ws, epoch, tid);
 }
