@@ -410,98 +410,229 @@ __device__ __forceinline__ void write_block_table(const TileDesc& d, uint2* __re
     }
 }
 
+// Where a tile's blob is, as known from the index alone (no access to the blob itself).
+struct BlobSpan {
+    uint32_t w_beg, w_end;   // index entries: blob = words [w_beg, w_end) of the blob area
+    uint32_t staged;         // 1: its 16-byte-aligned cover was requested by a bulk copy
+};
+
+// The 16-byte-aligned cover of a blob can be staged when it fits the staging buffer and lies inside the readable
+// bytes of the stream.
+__device__ __forceinline__ bool blob_stageable(const uint32_t* in, unsigned long long cap_bytes, uint32_t nT, uint32_t w_beg,
+                                               uint32_t w_end, uintptr_t& a_beg, uint32_t& bytes)
+{
+    if (w_end <= w_beg) return false;
+    const unsigned long long blob0 = (unsigned long long)kHeaderWords + nT;
+    if ((blob0 + w_end) * 4ull > cap_bytes) return false;
+    const uintptr_t b = (uintptr_t)(in + blob0 + w_beg), e = (uintptr_t)(in + blob0 + w_end);
+    a_beg = b & ~(uintptr_t)15;
+    const uintptr_t a_end = (e + 15) & ~(uintptr_t)15;
+    bytes = (uint32_t)(a_end - a_beg);
+    return (a_end - a_beg) <= (uintptr_t)(kBlobStageWords * 4) && (a_end - (uintptr_t)in) <= (uintptr_t)cap_bytes;
+}
+
 struct DecodeShared {
-    alignas(16) uint32_t blob[kBlobStageWords];
+    alignas(16) uint32_t blob[2][kBlobStageWords];            // staged blobs: current tile and the next one
     alignas(16) float wbuf[kWarps][kBlocksPerWarp * kBlock];
-    alignas(16) uint2 tbl[kWarps][kBlocksPerWarp];
+    alignas(16) uint2 tbl[kBlocksPerTile];                    // per block {code length, shared address of its payload}
+    BlobSpan span[2];
+    uint32_t sz_part[4];                                      // describe: payload words of blocks 32w .. 32w+31
+    uint32_t spread_part[4];
     float warp_total[2][kWarps];
     int32_t warp_total_i[kWarps];
-    alignas(8) unsigned long long bar;
+    alignas(8) unsigned long long bar[2];
 };
+
+// Cooperative description of a staged full tile: thread b (b < 128) owns block b.  Builds the block table, checks
+// the code lengths against the blob size and decides whether the tile's codes stay exact in fp32.
+// Two barriers.  Returns 0: inconsistent blob, 1: take the fp32 path, 2: consistent but needs the integer path.
+__device__ __forceinline__ int describe_staged(DecodeShared& sh, const uint32_t* sb, uint32_t words, int tid, int lane, int warp)
+{
+    constexpr uint32_t padw = kBlocksPerTile / 4;
+    bool good = true;
+    uint32_t L = 0, sz = 0, incl = 0;
+    if (tid < kBlocksPerTile) {
+        L = reinterpret_cast<const unsigned char*>(sb + 1)[tid];
+        good = L <= 31u;
+        sz = L ? L + 1 : 0;
+        incl = sz;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(kFull, incl, d);
+            if (lane >= d) incl += t;
+        }
+        const uint32_t spread = __reduce_add_sync(kFull, L <= (uint32_t)kFastDecodeMaxL ? (32u << L) : (1u << 24));
+        if (lane == 31) { sh.sz_part[warp] = incl; sh.spread_part[warp] = spread; }
+    }
+    __syncthreads();
+    uint32_t total = 0, spread = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const uint32_t pw = sh.sz_part[w];
+        if (w < warp) incl += pw;
+        total += pw;
+        spread += min(sh.spread_part[w], 1u << 24);
+    }
+    if (tid < kBlocksPerTile) sh.tbl[tid] = make_uint2(L, smem_u32(sb + 1 + padw) + 4 * (incl - sz));
+    good = good && (1 + padw + total == words);
+    const int all_good = __syncthreads_and(good ? 1 : 0);
+    if (!all_good) return 0;
+    const int32_t outlier = (int32_t)sb[0];
+    const uint32_t ao = (uint32_t)(outlier < 0 ? -outlier : outlier);
+    return (ao < (1u << 23) && spread < (1u << 23)) ? 1 : 2;
+}
 
 __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Workspace ws)
 {
     __shared__ DecodeShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t G = gridDim.x;
     uint32_t status = 0;
-    uint32_t fills = 0;    // bulk copies completed on sh.bar (its phase parity)
-    uint32_t par = 0;      // parity of the warp_total double buffer
+    uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed per staging buffer (phase parity of its mbarrier)
+    uint32_t par = 0;                  // parity of the warp_total double buffer
+    uint32_t p = 0;                    // staging buffer of the current tile
     const Xpose xp(lane);
-    if (tid == 0) {
-        mbar_init(&sh.bar, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
 
     int cur_job = -1;
     StreamInfo h;
     h.ok = false; h.n = 0; h.nT = 0; h.s = 1.0f; h.eb_abs = 0.0f;
-    for (uint32_t g = blockIdx.x; g < jb.total_tiles; g += gridDim.x) {
+
+    // thread 0 runs ahead of the CTA: it holds the index entries of the tile after next in registers and turns the
+    // next tile's entries into a bulk copy, so that no warp waits on a chain of global loads
+    uint32_t n_beg = 0, n_end = 0;       // index entries of tile g + G (valid when n_job >= 0)
+    int n_job = -1;
+    auto fetch_span = [&](uint32_t t, int& job_out, uint32_t& b, uint32_t& e) {   // thread 0: entries of tile number t
+        job_out = -1;
+        if (t >= jb.total_tiles) return;
+        const int jj = find_job(jb, t);
+        const Job& jq = jb.job[jj];
+        const StreamInfo hq = (jj == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
+        const uint32_t tl = t - jq.tile_begin;
+        if (!hq.ok || hq.n > jq.n || tl >= hq.nT) return;
+        const uint32_t* idx = jq.in_c + kHeaderWords;
+        e = ldg_u32(idx + tl);
+        b = tl ? ldg_u32(idx + tl - 1) : 0u;
+        job_out = jj;
+    };
+    auto stage_span = [&](uint32_t t, int jj, uint32_t b, uint32_t e, uint32_t buf) {   // thread 0: request tile t's blob
+        BlobSpan sp;
+        sp.w_beg = b; sp.w_end = e; sp.staged = 0;
+        if (jj >= 0) {
+            const Job& jq = jb.job[jj];
+            const StreamInfo hq = (jj == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
+            const uint32_t tl = t - jq.tile_begin;
+            const unsigned long long start = (unsigned long long)tl * kTile;
+            uintptr_t a_beg = 0;
+            uint32_t bytes = 0;
+            if (hq.ok && hq.n - start >= (unsigned long long)kTile &&
+                blob_stageable(jq.in_c, jq.in_cap, hq.nT, b, e, a_beg, bytes)) {
+                mbar_expect_tx(&sh.bar[buf], bytes);
+                bulk_load(sh.blob[buf], (const void*)a_beg, bytes, &sh.bar[buf]);
+                sp.staged = 1;
+            }
+        }
+        sh.span[buf] = sp;
+    };
+
+    if (tid == 0) {
+        mbar_init(&sh.bar[0], 1);
+        mbar_init(&sh.bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        int j0;
+        uint32_t b0 = 0, e0 = 0;
+        fetch_span(blockIdx.x, j0, b0, e0);
+        stage_span(blockIdx.x, j0, b0, e0, 0);
+        fetch_span(blockIdx.x + G, n_job, n_beg, n_end);
+    }
+    __syncthreads();
+
+    for (uint32_t g = blockIdx.x; g < jb.total_tiles; g += G) {
         const int j = find_job(jb, g);
         const Job& job = jb.job[j];
         if (j != cur_job) { h = read_header(job.in_c, job.in_cap); cur_job = j; }
         const uint32_t tile = g - job.tile_begin;
-        if (!h.ok) { status |= kStBadStream; continue; }
-        if (h.n > job.n) { status |= kStCapacity; continue; }
-        if (tile >= h.nT) continue;
-        const TileDesc d = describe_tile(job.in_c, job.in_cap, h, tile, lane);
-        if (!d.ok) { status |= kStBadStream; continue; }
-        float* __restrict__ y = job.y + (unsigned long long)tile * kTile;
 
-        if (d.fast) {
-            // stage the blob: the 16-byte aligned cover of [blob, blob + words)
-            const uintptr_t a_beg = (uintptr_t)d.blob & ~(uintptr_t)15;
-            const uintptr_t a_end = ((uintptr_t)(d.blob + d.words) + 15) & ~(uintptr_t)15;
-            const uint32_t shift = (uint32_t)(((uintptr_t)d.blob - a_beg) >> 2);
-            __syncthreads();   // the previous tile's readers of sh.blob are done
-            if (tid == 0) {
-                mbar_expect_tx(&sh.bar, (uint32_t)(a_end - a_beg));
-                bulk_load(sh.blob, (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar);
-            }
-            write_block_table(d, sh.tbl[warp], smem_u32(sh.blob + shift + 1 + d.padw), warp, lane);
-            __syncwarp();
-            const bool landed = mbar_wait(&sh.bar, fills & 1u);
-            ++fills;
-            if (!landed) status |= kStTimeout;   // carry on with whatever is staged: reads stay inside shared memory
-            decode_blocks_f32(sh.tbl[warp], sh.wbuf[warp], lane, xp);
-            __syncwarp();
-            float v[16];
-            const float total = decode_scan_f32(sh.wbuf[warp], lane, v);
-            if (lane == 0) sh.warp_total[par][warp] = total;
-            __syncthreads();
-            float base = (float)d.outlier;
-            for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[par][w]);
-            par ^= 1u;
-            float4* dst = reinterpret_cast<float4*>(y + 512 * warp + 16 * lane);
-            const bool vec = (((uintptr_t)dst) & 15u) == 0;
+        // thread 0: request the next tile's blob into the other buffer (its readers finished before the last barrier
+        // of the previous iteration), then fetch the index entries of the tile after it
+        if (tid == 0) {
+            stage_span(g + G, n_job, n_beg, n_end, p ^ 1u);
+            fetch_span(g + 2 * G, n_job, n_beg, n_end);
+        }
+        const BlobSpan sp = sh.span[p];
+        if (sp.staged) {   // a copy was requested for this tile: always consume it, whatever happens next
+            const uint32_t fl = p ? fills1 : fills0;
+            if (!mbar_wait(&sh.bar[p], fl & 1u)) status |= kStTimeout;
+            if (p) ++fills1; else ++fills0;
+        }
+        bool skip_tile = false;
+        if (!h.ok) { status |= kStBadStream; skip_tile = true; }
+        else if (h.n > job.n) { status |= kStCapacity; skip_tile = true; }
+        else if (tile >= h.nT) skip_tile = true;
+
+        int mode = 2;   // 1: fp32 path from the staged blob, 2: integer path from global memory
+        if (!skip_tile && sp.staged) {
+            const unsigned long long blob0 = (unsigned long long)kHeaderWords + h.nT;
+            const uint32_t shift = (uint32_t)(((uintptr_t)(job.in_c + blob0 + sp.w_beg) & 15u) >> 2);
+            const uint32_t* sb = sh.blob[p] + shift;
+            mode = describe_staged(sh, sb, sp.w_end - sp.w_beg, tid, lane, warp);
+            if (mode == 0) { status |= kStBadStream; skip_tile = true; }
+            if (mode == 1) {
+                float* __restrict__ y = job.y + (unsigned long long)tile * kTile;
+                decode_blocks_f32(sh.tbl + kBlocksPerWarp * warp, sh.wbuf[warp], lane, xp);
+                __syncwarp();
+                float v[16];
+                const float total = decode_scan_f32(sh.wbuf[warp], lane, v);
+                if (lane == 0) sh.warp_total[par][warp] = total;
+                const float outlier = (float)(int32_t)sb[0];
+                __syncthreads();
+                float base = outlier;
+                for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[par][w]);
+                par ^= 1u;
+                float4* dst = reinterpret_cast<float4*>(y + 512 * warp + 16 * lane);
+                const bool vec = (((uintptr_t)dst) & 15u) == 0;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                float4 o;
-                o.x = __fmul_rn(__fadd_rn(v[4 * c + 0], base), h.s);
-                o.y = __fmul_rn(__fadd_rn(v[4 * c + 1], base), h.s);
-                o.z = __fmul_rn(__fadd_rn(v[4 * c + 2], base), h.s);
-                o.w = __fmul_rn(__fadd_rn(v[4 * c + 3], base), h.s);
-                if (vec) dst[c] = o;
-                else {
-                    float* ds = reinterpret_cast<float*>(dst + c);
-                    ds[0] = o.x; ds[1] = o.y; ds[2] = o.z; ds[3] = o.w;
+                for (int c = 0; c < 4; ++c) {
+                    float4 o;
+                    o.x = __fmul_rn(__fadd_rn(v[4 * c + 0], base), h.s);
+                    o.y = __fmul_rn(__fadd_rn(v[4 * c + 1], base), h.s);
+                    o.z = __fmul_rn(__fadd_rn(v[4 * c + 2], base), h.s);
+                    o.w = __fmul_rn(__fadd_rn(v[4 * c + 3], base), h.s);
+                    if (vec) dst[c] = o;
+                    else {
+                        float* ds = reinterpret_cast<float*>(dst + c);
+                        ds[0] = o.x; ds[1] = o.y; ds[2] = o.z; ds[3] = o.w;
+                    }
                 }
             }
-        } else {
-            int32_t q[kBlocksPerWarp];
-            decode_blocks_int(d, warp, lane, q);
-            __syncthreads();
-            if (lane == 31) sh.warp_total_i[warp] = q[kBlocksPerWarp - 1];
-            __syncthreads();
-            int32_t base = d.outlier;
-            for (int w = 0; w < warp; ++w) base += sh.warp_total_i[w];
-            const uint32_t e0 = (uint32_t)(warp * kBlocksPerWarp * kBlock + lane);
+        }
+        if (!skip_tile && mode == 2) {
+            const TileDesc d = describe_tile(job.in_c, job.in_cap, h, tile, lane);
+            if (!d.ok) status |= kStBadStream;
+            else {
+                float* __restrict__ y = job.y + (unsigned long long)tile * kTile;
+                int32_t q[kBlocksPerWarp];
+                decode_blocks_int(d, warp, lane, q);
+                __syncthreads();
+                if (lane == 31) sh.warp_total_i[warp] = q[kBlocksPerWarp - 1];
+                __syncthreads();
+                int32_t base = d.outlier;
+                for (int w = 0; w < warp; ++w) base += sh.warp_total_i[w];
+                const uint32_t e0 = (uint32_t)(warp * kBlocksPerWarp * kBlock + lane);
 #pragma unroll
-            for (int i = 0; i < kBlocksPerWarp; ++i) {
-                const uint32_t e = e0 + (uint32_t)(i * kBlock);
-                if (e < d.len) y[e] = __fmul_rn(__int2float_rn(base + q[i]), h.s);
+                for (int i = 0; i < kBlocksPerWarp; ++i) {
+                    const uint32_t e = e0 + (uint32_t)(i * kBlock);
+                    if (e < d.len) y[e] = __fmul_rn(__int2float_rn(base + q[i]), h.s);
+                }
             }
         }
+        __syncthreads();   // the staged blob, the table and the span of this tile may be overwritten from here on
+        p ^= 1u;
+    }
+    // a copy requested for a tile beyond the last one is never started (stage_span checks the tile number); after an
+    // expired wait give the outstanding copies one more bounded wait before leaving
+    if (tid == 0 && (status & kStTimeout)) {
+        (void)mbar_wait(&sh.bar[0], (fills0 + 1u) & 1u);
+        (void)mbar_wait(&sh.bar[1], (fills1 + 1u) & 1u);
     }
     if (status) atomicOr(ws.status, status);
 }
