@@ -398,7 +398,7 @@ __device__ __forceinline__ float decode_scan_f32(const float* __restrict__ wbuf,
     return total;
 }
 
-// Writes the table of this warp's 16 blocks, {code length, shared-memory byte address of the block's payload},
+// (integer path helper) Writes the table of this warp's 16 blocks, {code length, shared address of the payload},
 // from the four lanes that hold their code-length word and offsets.
 __device__ __forceinline__ void write_block_table(const TileDesc& d, uint2* __restrict__ tbl, uint32_t payload_saddr,
                                                   int warp, int lane)
@@ -431,6 +431,52 @@ __device__ __forceinline__ bool blob_stageable(const uint32_t* in, unsigned long
     return (a_end - a_beg) <= (uintptr_t)(kBlobStageWords * 4) && (a_end - (uintptr_t)in) <= (uintptr_t)cap_bytes;
 }
 
+// Thread 0 of a CTA runs ahead of the others: it keeps the index entries of the tile after next in registers and
+// turns the next tile's entries into a bulk copy of its blob, so that no warp waits on a chain of global loads.
+// Shared needs: blob[2][kBlobStageWords], span[2], bar[2].
+struct StagePipe {
+    uint32_t n_beg = 0, n_end = 0;   // index entries of the next tile (valid when n_job >= 0)
+    int n_job = -1;
+
+    // index entries of tile number t of the launch
+    __device__ __forceinline__ void fetch(const JobBatch& jb, uint32_t t, int cur_job, const StreamInfo& h)
+    {
+        n_job = -1;
+        if (t >= jb.total_tiles) return;
+        const int jj = find_job(jb, t);
+        const Job& jq = jb.job[jj];
+        const StreamInfo hq = (jj == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
+        const uint32_t tl = t - jq.tile_begin;
+        if (!hq.ok || hq.n > jq.n || tl >= hq.nT) return;
+        const uint32_t* idx = jq.in_c + kHeaderWords;
+        n_end = ldg_u32(idx + tl);
+        n_beg = tl ? ldg_u32(idx + tl - 1) : 0u;
+        n_job = jj;
+    }
+    // request the blob of tile t (whose entries were fetched before) into staging buffer `buf`
+    template <class Shared>
+    __device__ __forceinline__ void stage(Shared& sh, const JobBatch& jb, uint32_t t, int cur_job, const StreamInfo& h, uint32_t buf)
+    {
+        BlobSpan sp;
+        sp.w_beg = n_beg; sp.w_end = n_end; sp.staged = 0;
+        if (n_job >= 0) {
+            const Job& jq = jb.job[n_job];
+            const StreamInfo hq = (n_job == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
+            const uint32_t tl = t - jq.tile_begin;
+            const unsigned long long start = (unsigned long long)tl * kTile;
+            uintptr_t a_beg = 0;
+            uint32_t bytes = 0;
+            if (hq.ok && !jq.in_c2 && hq.n - start >= (unsigned long long)kTile &&
+                blob_stageable(jq.in_c, jq.in_cap, hq.nT, n_beg, n_end, a_beg, bytes)) {
+                mbar_expect_tx(&sh.bar[buf], bytes);
+                bulk_load(sh.blob[buf], (const void*)a_beg, bytes, &sh.bar[buf]);
+                sp.staged = 1;
+            }
+        }
+        sh.span[buf] = sp;
+    }
+};
+
 struct DecodeShared {
     alignas(16) uint32_t blob[2][kBlobStageWords];            // staged blobs: current tile and the next one
     alignas(16) float wbuf[kWarps][kBlocksPerWarp * kBlock];
@@ -446,7 +492,8 @@ struct DecodeShared {
 // Cooperative description of a staged full tile: thread b (b < 128) owns block b.  Builds the block table, checks
 // the code lengths against the blob size and decides whether the tile's codes stay exact in fp32.
 // Two barriers.  Returns 0: inconsistent blob, 1: take the fp32 path, 2: consistent but needs the integer path.
-__device__ __forceinline__ int describe_staged(DecodeShared& sh, const uint32_t* sb, uint32_t words, int tid, int lane, int warp)
+template <class Shared>
+__device__ __forceinline__ int describe_staged(Shared& sh, const uint32_t* sb, uint32_t words, int tid, int lane, int warp)
 {
     constexpr uint32_t padw = kBlocksPerTile / 4;
     bool good = true;
@@ -497,52 +544,14 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
     StreamInfo h;
     h.ok = false; h.n = 0; h.nT = 0; h.s = 1.0f; h.eb_abs = 0.0f;
 
-    // thread 0 runs ahead of the CTA: it holds the index entries of the tile after next in registers and turns the
-    // next tile's entries into a bulk copy, so that no warp waits on a chain of global loads
-    uint32_t n_beg = 0, n_end = 0;       // index entries of tile g + G (valid when n_job >= 0)
-    int n_job = -1;
-    auto fetch_span = [&](uint32_t t, int& job_out, uint32_t& b, uint32_t& e) {   // thread 0: entries of tile number t
-        job_out = -1;
-        if (t >= jb.total_tiles) return;
-        const int jj = find_job(jb, t);
-        const Job& jq = jb.job[jj];
-        const StreamInfo hq = (jj == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
-        const uint32_t tl = t - jq.tile_begin;
-        if (!hq.ok || hq.n > jq.n || tl >= hq.nT) return;
-        const uint32_t* idx = jq.in_c + kHeaderWords;
-        e = ldg_u32(idx + tl);
-        b = tl ? ldg_u32(idx + tl - 1) : 0u;
-        job_out = jj;
-    };
-    auto stage_span = [&](uint32_t t, int jj, uint32_t b, uint32_t e, uint32_t buf) {   // thread 0: request tile t's blob
-        BlobSpan sp;
-        sp.w_beg = b; sp.w_end = e; sp.staged = 0;
-        if (jj >= 0) {
-            const Job& jq = jb.job[jj];
-            const StreamInfo hq = (jj == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
-            const uint32_t tl = t - jq.tile_begin;
-            const unsigned long long start = (unsigned long long)tl * kTile;
-            uintptr_t a_beg = 0;
-            uint32_t bytes = 0;
-            if (hq.ok && hq.n - start >= (unsigned long long)kTile &&
-                blob_stageable(jq.in_c, jq.in_cap, hq.nT, b, e, a_beg, bytes)) {
-                mbar_expect_tx(&sh.bar[buf], bytes);
-                bulk_load(sh.blob[buf], (const void*)a_beg, bytes, &sh.bar[buf]);
-                sp.staged = 1;
-            }
-        }
-        sh.span[buf] = sp;
-    };
-
+    StagePipe pipe;   // thread 0 only
     if (tid == 0) {
         mbar_init(&sh.bar[0], 1);
         mbar_init(&sh.bar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        int j0;
-        uint32_t b0 = 0, e0 = 0;
-        fetch_span(blockIdx.x, j0, b0, e0);
-        stage_span(blockIdx.x, j0, b0, e0, 0);
-        fetch_span(blockIdx.x + G, n_job, n_beg, n_end);
+        pipe.fetch(jb, blockIdx.x, cur_job, h);
+        pipe.stage(sh, jb, blockIdx.x, cur_job, h, 0);
+        pipe.fetch(jb, blockIdx.x + G, cur_job, h);
     }
     __syncthreads();
 
@@ -555,8 +564,8 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
         // thread 0: request the next tile's blob into the other buffer (its readers finished before the last barrier
         // of the previous iteration), then fetch the index entries of the tile after it
         if (tid == 0) {
-            stage_span(g + G, n_job, n_beg, n_end, p ^ 1u);
-            fetch_span(g + 2 * G, n_job, n_beg, n_end);
+            pipe.stage(sh, jb, g + G, cur_job, h, p ^ 1u);
+            pipe.fetch(jb, g + 2 * G, cur_job, h);
         }
         const BlobSpan sp = sh.span[p];
         if (sp.staged) {   // a copy was requested for this tile: always consume it, whatever happens next
@@ -759,16 +768,19 @@ struct EncodeShared {
 };
 
 struct FusedShared {
-    alignas(16) uint32_t blob[kBlobStageWords];
+    alignas(16) uint32_t blob[2][kBlobStageWords];                   // staged blobs: current tile and the next one
     alignas(16) float ybuf[kWarps][(kBlocksPerWarp + 1) * kBlock];   // deltas, then sums (row 0 of a warp = guard)
-    alignas(16) uint2 tbl[kWarps][kBlocksPerWarp];
+    alignas(16) uint2 tbl[kBlocksPerTile];
     alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];
+    BlobSpan span[2];
+    uint32_t sz_part[4];
+    uint32_t spread_part[4];
     float warp_total[kWarps];
     int32_t warp_total_i[kWarps];
     int32_t warp_total_i2[kWarps];
     uint32_t warp_words[2][kWarps];
     LookShared look;
-    alignas(8) unsigned long long bar;
+    alignas(8) unsigned long long bar[2];
 };
 
 // A raw-mode tile can be staged by a bulk copy when it is full and starts on a 16-byte boundary.
@@ -1066,14 +1078,11 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     FusedShared& sh = *reinterpret_cast<FusedShared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
+    const uint32_t G = gridDim.x;
     uint32_t status = 0;
-    uint32_t fills = 0;
-    if (tid == 0) {
-        mbar_init(&sh.bar, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-    uint32_t look_par = 0, p = 0;
+    uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed per staging buffer
+    uint32_t look_par = 0;
+    uint32_t p = 0;                    // half of the slots and staging buffer of the current tile
     float pend_eb = 0.0f, pend_s = 1.0f;   // bound and step of the pending tile's job (header fields)
     Pending pend;
     pend.valid = false;
@@ -1085,7 +1094,18 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     h1.ok = h2.ok = false; h1.n = h2.n = 0; h1.nT = h2.nT = 0; h1.s = h2.s = 1.0f; h1.eb_abs = h2.eb_abs = 0.0f;
     bool job_ok = false;
 
-    for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += gridDim.x) {
+    StagePipe pipe;   // thread 0 only
+    if (tid == 0) {
+        mbar_init(&sh.bar[0], 1);
+        mbar_init(&sh.bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        pipe.fetch(jb, blockIdx.x, cur_job, h1);
+        pipe.stage(sh, jb, blockIdx.x, cur_job, h1, 0);
+        pipe.fetch(jb, blockIdx.x + G, cur_job, h1);
+    }
+    __syncthreads();
+
+    for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += G, p ^= 1u) {
         const int j = find_job(jb, ticket);
         const Job& job = jb.job[j];
         const uint32_t tile = ticket - job.tile_begin;
@@ -1102,6 +1122,19 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
         const float s = h1.s, eb_abs = h1.eb_abs;
         const float r = __fdiv_rn(1.0f, s);
+
+        // thread 0: request the next tile's blob into the other staging buffer (its readers finished before the last
+        // barrier of the previous iteration), then fetch the index entries of the tile after it
+        if (tid == 0) {
+            pipe.stage(sh, jb, ticket + G, cur_job, h1, p ^ 1u);
+            pipe.fetch(jb, ticket + 2 * G, cur_job, h1);
+        }
+        const BlobSpan sp = sh.span[p];
+        if (sp.staged) {   // a copy was requested for this tile: always consume it, whatever happens next
+            const uint32_t fl = p ? fills1 : fills0;
+            if (!mbar_wait(&sh.bar[p], fl & 1u)) status |= kStTimeout;
+            if (p) ++fills1; else ++fills0;
+        }
 
         if (!job_ok || n == 0) {
             if (!job_ok) status |= kStBadStream;
@@ -1120,11 +1153,113 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         const uint32_t nb = (len + kBlock - 1) / kBlock;
         const uint32_t padw = (nb + 3) >> 2;
         const uint32_t last = len - 1;
+        float* yrows = sh.ybuf[warp];
+        const float* __restrict__ loc = job.x ? job.x + start : nullptr;
+        float* __restrict__ yout = job.y ? job.y + start : nullptr;
+        const bool deq = (job.flags & 1u) != 0;
 
-        const TileDesc d1 = describe_tile(job.in_c, job.in_cap, h1, tile, lane);
-        TileDesc d2 = d1;
-        if (job.in_c2) d2 = describe_tile(job.in_c2, job.in2_cap, h2, tile, lane);
-        if (!d1.ok || !d2.ok) {   // uniform: keep the scan consistent for the tiles that follow, write nothing
+        // ---- front end: decode + add, leaving the sums in this warp's rows of ybuf (swizzled), row 0 = guard
+        int mode = 2;   // 1: fp32 front end from the staged blob, 2: integer front end from global memory
+        bool bad_tile = false;
+        if (sp.staged) {
+            // this thread's 16 consecutive elements of the local operand are needed after the scan: pull their lines
+            // towards L2 now, load them (128-bit when aligned) when they are used
+            const float* lp = loc + 512 * warp + 16 * lane;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(lp));
+            const unsigned long long blob0 = (unsigned long long)kHeaderWords + h1.nT;
+            const uint32_t shift = (uint32_t)(((uintptr_t)(job.in_c + blob0 + sp.w_beg) & 15u) >> 2);
+            const uint32_t* sb = sh.blob[p] + shift;
+            mode = describe_staged(sh, sb, sp.w_end - sp.w_beg, tid, lane, warp);
+            if (mode == 0) bad_tile = true;
+            if (mode == 1) {
+                decode_blocks_f32(sh.tbl + kBlocksPerWarp * warp, yrows + 32, lane, xp);
+                __syncwarp();
+                float v[16];
+                const float total = decode_scan_f32(yrows + 32, lane, v);
+                if (lane == 0) sh.warp_total[warp] = total;
+                const float outlier = (float)(int32_t)sb[0];
+                __syncthreads();   // warp totals
+                float base = outlier;
+                for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[w]);
+                // the element before this warp's first one is the last element of the previous warp: its code is `base`
+                if (lane == 0) {
+                    float yprev;
+                    if (warp == 0) yprev = __fadd_rn(__fmul_rn(__fadd_rn(v[0], base), s), __ldg(loc));
+                    else yprev = __fadd_rn(__fmul_rn(base, s), __ldg(loc + 512 * warp - 1));
+                    yrows[31 ^ 12] = yprev;   // guard row, element 31 under the swizzle of the row before row 0
+                }
+                const int sw = (lane >> 1) & 3;
+                float4* row = reinterpret_cast<float4*>(yrows + 32 + 16 * lane);
+                float4* gout = yout ? reinterpret_cast<float4*>(yout + 512 * warp + 16 * lane) : nullptr;
+                const bool gvec = (((uintptr_t)gout) & 15u) == 0;
+                const bool lvec = (((uintptr_t)lp) & 15u) == 0;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    float4 l;
+                    if (lvec) l = __ldg(reinterpret_cast<const float4*>(lp) + c);
+                    else { l.x = __ldg(lp + 4 * c); l.y = __ldg(lp + 4 * c + 1); l.z = __ldg(lp + 4 * c + 2); l.w = __ldg(lp + 4 * c + 3); }
+                    float4 o;
+                    o.x = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), l.x);
+                    o.y = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), l.y);
+                    o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), l.z);
+                    o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), l.w);
+                    row[c ^ sw] = o;
+                    if (gout && !deq) {
+                        if (gvec) gout[c] = o;
+                        else { float* g = reinterpret_cast<float*>(gout + c); g[0] = o.x; g[1] = o.y; g[2] = o.z; g[3] = o.w; }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        if (!bad_tile && mode == 2) {
+            // integer front end, one element per lane; ragged tails repeat the last element
+            const TileDesc d1 = describe_tile(job.in_c, job.in_cap, h1, tile, lane);
+            TileDesc d2 = d1;
+            if (job.in_c2) d2 = describe_tile(job.in_c2, job.in2_cap, h2, tile, lane);
+            if (!d1.ok || !d2.ok) bad_tile = true;
+            else {
+                int32_t qa[kBlocksPerWarp], qb[kBlocksPerWarp];
+                decode_blocks_int(d1, warp, lane, qa);
+                if (job.in_c2) decode_blocks_int(d2, warp, lane, qb);
+                if (lane == 31) {
+                    sh.warp_total_i[warp] = qa[kBlocksPerWarp - 1];
+                    if (job.in_c2) sh.warp_total_i2[warp] = qb[kBlocksPerWarp - 1];
+                }
+                __syncthreads();   // warp totals
+                int32_t base_a = d1.outlier, base_b = d2.outlier;
+                for (int w = 0; w < warp; ++w) {
+                    base_a += sh.warp_total_i[w];
+                    if (job.in_c2) base_b += sh.warp_total_i2[w];
+                }
+                const uint32_t e0 = (uint32_t)(512 * warp + lane);
+#pragma unroll
+                for (int i = 0; i < kBlocksPerWarp; ++i) {
+                    uint32_t e = e0 + 32u * i;
+                    const bool inside = e <= last;
+                    if (!inside) e = last;
+                    const float xa = __fmul_rn(__int2float_rn(base_a + qa[i]), s);
+                    const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b + qb[i]), s) : __ldg(loc + e);
+                    const float yv = __fadd_rn(xa, xb);
+                    yrows[32 * (i + 1) + (lane ^ ((i & 3) << 2))] = yv;
+                    if (yout && !deq && inside) yout[e] = yv;
+                }
+                if (lane == 0) {
+                    float yprev;
+                    if (warp == 0) {
+                        yprev = yrows[32];   // own first element (row 1, lane 0, swizzle 0)
+                    } else {
+                        const uint32_t ep = min((uint32_t)(512 * warp - 1), last);
+                        const float xa = __fmul_rn(__int2float_rn(base_a), s);
+                        const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b), s) : __ldg(loc + ep);
+                        yprev = __fadd_rn(xa, xb);
+                    }
+                    yrows[31 ^ 12] = yprev;
+                }
+                __syncwarp();
+            }
+        }
+        if (bad_tile) {   // uniform: keep the scan consistent for the tiles that follow, write nothing
             status |= kStBadStream;
             if (tid == 0) {
                 st_state(ws.tile_state + ticket, pack_state(epoch, 0u, 0u));
@@ -1134,115 +1269,6 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             continue;
         }
 
-        // ---- front end: decode + add, leaving the sums in this warp's rows of ybuf (swizzled), row 0 = guard
-        float* yrows = sh.ybuf[warp];
-        const float* __restrict__ loc = job.x ? job.x + start : nullptr;
-        float* __restrict__ yout = job.y ? job.y + start : nullptr;
-        const bool deq = (job.flags & 1u) != 0;
-        const bool fast_front = d1.fast && !job.in_c2;
-        if (fast_front) {
-            const uintptr_t a_beg = (uintptr_t)d1.blob & ~(uintptr_t)15;
-            const uintptr_t a_end = ((uintptr_t)(d1.blob + d1.words) + 15) & ~(uintptr_t)15;
-            const uint32_t shift = (uint32_t)(((uintptr_t)d1.blob - a_beg) >> 2);
-            if (tid == 0) {   // sh.blob's previous readers finished before the last barrier of the previous tile
-                mbar_expect_tx(&sh.bar, (uint32_t)(a_end - a_beg));
-                bulk_load(sh.blob, (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar);
-            }
-            // this thread's 16 consecutive elements of the local operand (128-bit loads when aligned)
-            float lv[16];
-            {
-                const float* lp = loc + 512 * warp + 16 * lane;
-                if ((((uintptr_t)lp) & 15u) == 0) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const float4 f = __ldg(reinterpret_cast<const float4*>(lp) + c);
-                        lv[4 * c] = f.x; lv[4 * c + 1] = f.y; lv[4 * c + 2] = f.z; lv[4 * c + 3] = f.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) lv[k] = __ldg(lp + k);
-                }
-            }
-            write_block_table(d1, sh.tbl[warp], smem_u32(sh.blob + shift + 1 + d1.padw), warp, lane);
-            __syncwarp();
-            const bool landed = mbar_wait(&sh.bar, fills & 1u);
-            ++fills;
-            if (!landed) status |= kStTimeout;
-            decode_blocks_f32(sh.tbl[warp], yrows + 32, lane, xp);
-            __syncwarp();
-            float v[16];
-            const float total = decode_scan_f32(yrows + 32, lane, v);
-            if (lane == 0) sh.warp_total[warp] = total;
-            __syncthreads();   // warp totals
-            float base = (float)d1.outlier;
-            for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[w]);
-            // the element before this warp's first one is the last element of the previous warp: its code is `base`
-            if (lane == 0) {
-                float yprev;
-                if (warp == 0) yprev = __fadd_rn(__fmul_rn(__fadd_rn(v[0], base), s), lv[0]);
-                else yprev = __fadd_rn(__fmul_rn(base, s), __ldg(loc + 512 * warp - 1));
-                yrows[31 ^ 12] = yprev;   // guard row, element 31 under the swizzle of the row before row 0
-            }
-            const int sw = (lane >> 1) & 3;
-            float4* row = reinterpret_cast<float4*>(yrows + 32 + 16 * lane);
-            float4* gout = yout ? reinterpret_cast<float4*>(yout + 512 * warp + 16 * lane) : nullptr;
-            const bool gvec = (((uintptr_t)gout) & 15u) == 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                float4 o;
-                o.x = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), lv[4 * c + 0]);
-                o.y = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), lv[4 * c + 1]);
-                o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), lv[4 * c + 2]);
-                o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), lv[4 * c + 3]);
-                row[c ^ sw] = o;
-                if (gout && !deq) {
-                    if (gvec) gout[c] = o;
-                    else { float* g = reinterpret_cast<float*>(gout + c); g[0] = o.x; g[1] = o.y; g[2] = o.z; g[3] = o.w; }
-                }
-            }
-            __syncwarp();
-        } else {
-            // integer front end, one element per lane; ragged tails repeat the last element
-            int32_t qa[kBlocksPerWarp], qb[kBlocksPerWarp];
-            decode_blocks_int(d1, warp, lane, qa);
-            if (job.in_c2) decode_blocks_int(d2, warp, lane, qb);
-            if (lane == 31) {
-                sh.warp_total_i[warp] = qa[kBlocksPerWarp - 1];
-                if (job.in_c2) sh.warp_total_i2[warp] = qb[kBlocksPerWarp - 1];
-            }
-            __syncthreads();   // warp totals
-            int32_t base_a = d1.outlier, base_b = d2.outlier;
-            for (int w = 0; w < warp; ++w) {
-                base_a += sh.warp_total_i[w];
-                if (job.in_c2) base_b += sh.warp_total_i2[w];
-            }
-            const uint32_t e0 = (uint32_t)(512 * warp + lane);
-#pragma unroll
-            for (int i = 0; i < kBlocksPerWarp; ++i) {
-                uint32_t e = e0 + 32u * i;
-                const bool inside = e <= last;
-                if (!inside) e = last;
-                const float xa = __fmul_rn(__int2float_rn(base_a + qa[i]), s);
-                const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b + qb[i]), s) : __ldg(loc + e);
-                const float yv = __fadd_rn(xa, xb);
-                yrows[32 * (i + 1) + (lane ^ ((i & 3) << 2))] = yv;
-                if (yout && !deq && inside) yout[e] = yv;
-            }
-            if (lane == 0) {
-                float yprev;
-                if (warp == 0) {
-                    yprev = yrows[32];   // own first element (row 1, lane 0, swizzle 0)
-                } else {
-                    const uint32_t ep = min((uint32_t)(512 * warp - 1), last);
-                    const float xa = __fmul_rn(__int2float_rn(base_a), s);
-                    const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b), s) : __ldg(loc + ep);
-                    yprev = __fadd_rn(xa, xb);
-                }
-                yrows[31 ^ 12] = yprev;
-            }
-            __syncwarp();
-        }
-
         // ---- back end: encode the sums
         uint32_t* slots_w = sh.slots[p] + kSlotWords * kBlocksPerWarp * warp;
         uint32_t my_lw = 0, wsum = 0;
@@ -1250,7 +1276,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         float guard = 0.0f, tmax = 0.0f;
         const SrcSwizzled src(yrows, lane);
         wsum = encode_blocks<true>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
-            q_first = first_code<true>(src.cur(0, 0), r);
+        q_first = first_code<true>(src.cur(0, 0), r);
         const bool need_int = __any_sync(kFull, !(guard < kGuardExact));
         if (need_int) {
             wsum = encode_blocks<false>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
@@ -1284,11 +1310,14 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
         pend.q_first = q_first;
         pend_eb = eb_abs; pend_s = s;
-        p ^= 1u;
     }
     if (pend.valid)
         place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
               sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, pend_eb, pend_s, ws, epoch, tid, warp, lane, status);
+    if (tid == 0 && (status & kStTimeout)) {
+        (void)mbar_wait(&sh.bar[0], (fills0 + 1u) & 1u);
+        (void)mbar_wait(&sh.bar[1], (fills1 + 1u) & 1u);
+    }
     if (status) atomicOr(ws.status, status);
     finish_launch(ws, epoch, tid);
 }
