@@ -3,23 +3,24 @@
 //
 // Work decomposition.  One CTA of 256 threads handles one 4096-element tile at a time; each of its 8 warps owns
 // 16 consecutive 32-element blocks, one element per lane, so that a block's code length is one warp OR-reduction
-// and each bit plane is one ballot.  The kernels are bound by instruction issue (integer ALU pipe: 2
-// warp-instructions/clk/SM; shared memory and shuffles: 1), not by HBM, so the design minimises ALU and LSU
-// instructions per block:
-//   * tiles are staged in shared memory by 1-D bulk copies (cp.async.bulk + mbarrier), double buffered in the
-//     encoder, so no thread spends instructions or registers on global loads;
+// and its bit planes come out of a 32 x 32 bit-matrix transpose across the warp.  The kernels are bound by
+// instruction issue (integer ALU pipe: 2 warp-instructions/clk/SM; shared memory and shuffles: 1), not by HBM, so
+// the design minimises instructions per block:
+//   * tiles (encoder) and compressed blobs (decoder, fused hop) are staged in shared memory by 1-D bulk copies
+//     (cp.async.bulk + mbarrier), requested one tile ahead, so no thread spends instructions or registers on
+//     global loads and no warp waits on a chain of them;
 //   * the common case runs in fp32 on the FMA pipe: codes are rounded with the 1.5*2^23 trick, deltas are float
 //     subtractions (exact below 2^23), magnitudes are read from the mantissa of |delta| + 2^23.  Tiles whose
 //     values leave the exactly representable range, ragged tails and unaligned inputs take an integer path
 //     that computes the same bits;
-//   * the encoder writes each block's words to a fixed slot and compacts while copying out, so quantisation and
-//     encoding are a single pass over a block; the decoder undoes the Lorenzo recurrence by a warp-local
-//     transposition through shared memory (16 consecutive elements per thread) instead of shuffle scans.
+//   * the encoder appends each block's words to its warp's region of shared memory in a single pass over the
+//     block; the decoder undoes the Lorenzo recurrence by a warp-local transposition through shared memory
+//     (16 consecutive elements per thread) instead of shuffle scans.
 // Tiles are dealt round-robin to a grid that fits the device (CTA c takes tiles c, c + G, ...), so all CTAs move
-// through the stream in step, the next tile is known in advance (its bulk copy overlaps the current tile) and a
-// tile's predecessors in the placement scan (decoupled look-back over tile sizes) are at most one round behind.
-// The scan relies on the grid being resident at once; every wait is bounded and reports through the status word
-// instead of hanging if it is not.
+// through the stream in step and the next tile is known in advance.  Placement (prefix sum of tile sizes) is
+// anchored at a CTA's own previous tile and deferred by one tile, so it only ever sums sizes that are already
+// published.  The scan relies on the grid being resident at once; every wait is bounded and reports through the
+// status word instead of hanging if it is not.
 #include "zccl_internal.h"
 
 namespace zccl {
@@ -398,18 +399,6 @@ __device__ __forceinline__ float decode_scan_f32(const float* __restrict__ wbuf,
     return total;
 }
 
-// (integer path helper) Writes the table of this warp's 16 blocks, {code length, shared address of the payload},
-// from the four lanes that hold their code-length word and offsets.
-__device__ __forceinline__ void write_block_table(const TileDesc& d, uint2* __restrict__ tbl, uint32_t payload_saddr,
-                                                  int warp, int lane)
-{
-    if ((lane >> 2) == warp) {
-        uint4* t4 = reinterpret_cast<uint4*>(tbl + 4 * (lane & 3));
-        t4[0] = make_uint4(d.lw & 0xFF, payload_saddr + 4 * d.o0, (d.lw >> 8) & 0xFF, payload_saddr + 4 * d.o1);
-        t4[1] = make_uint4((d.lw >> 16) & 0xFF, payload_saddr + 4 * d.o2, d.lw >> 24, payload_saddr + 4 * d.o3);
-    }
-}
-
 // Where a tile's blob is, as known from the index alone (no access to the blob itself).
 struct BlobSpan {
     uint32_t w_beg, w_end;   // index entries: blob = words [w_beg, w_end) of the blob area
@@ -634,7 +623,8 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
                 }
             }
         }
-        __syncthreads();   // the staged blob, the table and the span of this tile may be overwritten from here on
+        // no barrier here: everything the next iteration overwrites (the other staging buffer, the block table, the
+        // partial sums) was last read before a barrier of this iteration that every thread has passed
         p ^= 1u;
     }
     // a copy requested for a tile beyond the last one is never started (stage_span checks the tile number); after an
@@ -930,11 +920,7 @@ __device__ __forceinline__ void place(const Pending& c, Anchor& anchor, const Jo
     blob_layout(warp_words, padw, warp, wbase, total);
     uint32_t lo = job.tile_begin, base = 0, skip = 0;
     if (anchor.job == c.job) { lo = anchor.ticket + 1; base = anchor.incl; }
-#ifdef ZCCL_DEBUG_NO_LOOKBACK
-    const uint32_t excl = tile * 700u;
-#else
     const uint32_t excl = base + sum_sizes_cta(look, look_par, ws, lo, c.ticket, epoch, warp, lane, skip, status);
-#endif
     anchor.job = c.job; anchor.ticket = c.ticket; anchor.incl = excl + total;
     const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
     const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
@@ -997,7 +983,6 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         const Job& job = jb.job[j];
         const uint32_t tile = ticket - job.tile_begin;
         const unsigned long long n = job.n;
-        const uint32_t nT = (uint32_t)((n + kTile - 1) / kTile);
         const bool staged = prm.valid && n && stageable_raw(job, tile);
 
         if (n == 0 || !prm.valid) {   // a job without elements still owns one tile number: header and length only
