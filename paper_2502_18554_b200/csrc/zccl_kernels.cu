@@ -623,8 +623,7 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
                 }
             }
         }
-        // no barrier here: everything the next iteration overwrites (the other staging buffer, the block table, the
-        // partial sums) was last read before a barrier of this iteration that every thread has passed
+        __syncthreads();   // keeps the warps of a CTA in step (measured faster than letting them drift apart)
         p ^= 1u;
     }
     // a copy requested for a tile beyond the last one is never started (stage_span checks the tile number); after an
