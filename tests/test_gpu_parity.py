@@ -255,6 +255,26 @@ def test_fused_hop_fourier_and_gradient(z, ctx):
     assert rc == wrc and np.array_equal(got, want)
 
 
+def test_fused_hop_wide_code_lengths(z, ctx):
+    # noisy operands at a tight bound: encoded tiles larger than the shared-memory regions of the encoder, which
+    # then encodes them again straight into the stream; mixed with smooth tiles that take the ordinary route
+    rng = np.random.default_rng(12)
+    n = 9 * 4096 + 100
+    a = fields.smooth_1d(n, seed=3)
+    b = fields.smooth_1d(n, seed=4)
+    b[2 * 4096: 5 * 4096] += rng.normal(0, 0.5, 3 * 4096).astype(f32)
+    a[7 * 4096:] += rng.normal(0, 0.5, n - 7 * 4096).astype(f32)
+    ea, s, r = oracle.resolve(oracle.EB_ABS, 2e-6)
+    sa, _ = oracle.compress_core(a, ea, s, r)
+    want, wrc, wraw = oracle.drc(sa, local=b, want_raw=True)
+    got, rc, raw = _drc_gpu(z, ctx, sa, n, local=b, raw=True)
+    assert rc == wrc
+    assert np.array_equal(got, want)
+    assert_same_bits(raw, wraw)
+    st, rc2 = gpu_compress(z, ctx, a, z.EB_ABS, 2e-6)
+    assert np.array_equal(st, sa)
+
+
 def test_fused_hop_rejects_mismatch(z, ctx):
     a = fields.smooth_1d(9000, seed=1)
     sa, _ = oracle.compress(a, oracle.EB_ABS, 1e-3)
