@@ -676,10 +676,32 @@ struct SrcSwizzled {        // the fused kernel's sum tile: per-warp region of 1
     __device__ __forceinline__ float prev(int g, int u) const { return rows[32 * (4 * g + u + 1) + po[u]]; }
 };
 
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Per-lane constants of the packed store: with four blocks per transpose lane 8u + b ends up with plane b of
+// block u (b = 7: its sign word).
+struct PackLane {
+    uint32_t sh8;   // 8 * (lane / 8): position of this lane's block in a word of four per-block bytes
+    uint32_t wp;    // word of the block's slot this lane stores: 0 = sign word, b + 1 = plane b
+    __device__ __forceinline__ explicit PackLane(int lane)
+    {
+        sh8 = 8u * ((uint32_t)lane >> 3);
+        wp = ((uint32_t)(lane & 7) + 1u) & 7u;
+        asm volatile("" : "+r"(sh8), "+r"(wp));
+    }
+};
+
 // One pass over this warp's 16 blocks: quantise, 1-D Lorenzo delta, code length, sign word and bit planes, appended
 // to the warp's region of shared memory.  Returns the warp's payload size in words; lane g (g < 4) ends up holding
 // the code-length word of blocks 4g..4g+3 in `my_lw`.  FAST: fp32 arithmetic, valid while every |x * r| < 2^21.5;
-// the caller checks `guard` (sum of squares of x * r) and reruns with FAST = false when it is too large.
+// the caller checks `guard` (sum of squares of x * r over the warp's elements and the one before them) and reruns
+// with FAST = false when it is too large.  FAST handles four blocks per bit-matrix transpose while their code
+// lengths are at most 7 (sign + 7 magnitude bits of four elements share a word), else one block per transpose.
 template <bool FAST, class Src>
 __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint32_t* __restrict__ slots_w, int lane,
                                                   const Xpose& xp, uint32_t& my_lw, float& guard, float& tmax)
@@ -688,35 +710,62 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
     float acc = 0.0f, tm = 0.0f;
     my_lw = 0;
     const uint32_t widx = (uint32_t)(lane + 1) & 31u;   // lane k stores plane k at word k + 1, lane 31 the sign word at 0
+    const PackLane pk(lane);
+    if (FAST) {   // the element before the warp's first one belongs to nobody else's sum
+        const float tp0 = __fmul_rn(src.prev(0, 0), r);
+        if (lane == 0) acc = __fmul_rn(tp0, tp0);
+    }
 #pragma unroll 1
     for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
         uint32_t lword = 0;
+        if (FAST) {
+            uint32_t ab[4], db[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const float xv = src.cur(g, u), pv = src.prev(g, u);
-            const float t = __fmul_rn(xv, r), tp = __fmul_rn(pv, r);
-            uint32_t L;
-            if (FAST) {
+            for (int u = 0; u < 4; ++u) {
+                const float t = __fmul_rn(src.cur(g, u), r), tp = __fmul_rn(src.prev(g, u), r);
                 acc = __fmaf_rn(t, t, acc);
-                acc = __fmaf_rn(tp, tp, acc);
-                const float c = __fadd_rn(t, kRoundMagic), cp = __fadd_rn(tp, kRoundMagic);
-                const float df = __fsub_rn(c, cp);
-                const uint32_t ab = __float_as_uint(__fadd_rn(fabsf(df), kTwo23));
-                const uint32_t m = __reduce_or_sync(kFull, ab) & 0x7FFFFFu;
-                L = 32u - (uint32_t)__clz((int)m);
-                if (L) {   // uniform over the warp
-                    // magnitude in bits 0..22 (bits 23..30 hold exponent bits: never stored, L <= 23), sign in bit 31
-                    const uint32_t v = xp(ab | (__float_as_uint(df) & 0x80000000u));
-                    if (widx <= L) slots_w[wsum + widx] = v;
-                    wsum += L + 1;
-                }
+                const float df = __fsub_rn(__fadd_rn(t, kRoundMagic), __fadd_rn(tp, kRoundMagic));
+                // magnitude in bits 0..22 (bits 23..30 hold exponent bits: never stored, L <= 23)
+                ab[u] = __float_as_uint(__fadd_rn(fabsf(df), kTwo23));
+                db[u] = __float_as_uint(df);
+            }
+            const uint32_t wide = ((ab[0] | ab[1] | ab[2]) | ab[3]) & 0x7FFF80u;
+            if (!__any_sync(kFull, wide != 0)) {
+                // byte u of the word: bits 0..6 = |delta| of this lane's element of block u, bit 7 = its sign
+                const uint32_t mg = prmt(prmt(ab[0], ab[1], 0x0040u), prmt(ab[2], ab[3], 0x0040u), 0x5410u);
+                const uint32_t sg = prmt(prmt(db[0], db[1], 0x00FBu), prmt(db[2], db[3], 0x00FBu), 0x5410u);
+                const uint32_t v = xp(mg | (sg & 0x80808080u));
+                const uint32_t ors = __reduce_or_sync(kFull, mg);                       // byte u: OR of block u's magnitudes
+                const uint32_t l_mine = 32u - (uint32_t)__clz((int)((ors >> pk.sh8) & 0xFFu));
+                lword = __reduce_or_sync(kFull, l_mine << pk.sh8);                      // byte u: code length of block u
+                const uint32_t nword = lword + (((lword + 0x7F7F7F7Fu) >> 7) & 0x01010101u);   // byte u: slot size of block u
+                const uint32_t pref = nword * 0x01010100u;                              // byte u: slots of blocks before u
+                const uint32_t n_mine = (nword >> pk.sh8) & 0xFFu;
+                if (pk.wp < n_mine) slots_w[wsum + ((pref >> pk.sh8) & 0xFFu) + pk.wp] = v;
+                wsum += (nword * 0x01010101u) >> 24;
             } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t m = __reduce_or_sync(kFull, ab[u]) & 0x7FFFFFu;
+                    const uint32_t L = 32u - (uint32_t)__clz((int)m);
+                    if (L) {   // uniform over the warp
+                        const uint32_t v = xp(ab[u] | (db[u] & 0x80000000u));
+                        if (widx <= L) slots_w[wsum + widx] = v;
+                        wsum += L + 1;
+                    }
+                    lword |= L << (8 * u);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float t = __fmul_rn(src.cur(g, u), r), tp = __fmul_rn(src.prev(g, u), r);
                 tm = fmaxf(tm, fabsf(t));
                 const int32_t q = __float2int_rn(t), qp = __float2int_rn(tp);
                 const int32_t dd = q - qp;
                 const uint32_t ab = (uint32_t)(dd < 0 ? -dd : dd);
                 const uint32_t m = __reduce_or_sync(kFull, ab);
-                L = 32u - (uint32_t)__clz((int)m);
+                const uint32_t L = 32u - (uint32_t)__clz((int)m);
                 const uint32_t sg = __ballot_sync(kFull, dd < 0);
                 if (L) {
                     uint32_t* slot = slots_w + wsum;
@@ -724,8 +773,8 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
                     for (uint32_t k = 0; k < L; ++k) slot[k + 1] = __ballot_sync(kFull, ab & (1u << k));
                     wsum += L + 1;
                 }
+                lword |= L << (8 * u);
             }
-            lword |= L << (8 * u);
         }
         if (lane == g) my_lw = lword;
     }
@@ -748,11 +797,20 @@ struct LookShared {
     uint32_t ok[2][kWarps];     // 1 if every state the warp inspected was published
 };
 
+// Placement split in two.  Everything about a pending tile that is the same for all threads (scan of the sizes,
+// layout of the warps' regions, capacity check, index entry, outlier, header, stream length) is done once, by warp 0,
+// which leaves the result here; after a barrier each warp only copies its own region.
+struct PlanShared {
+    uint32_t* blob_out;       // where the pending tile's blob starts in the stream (nullptr: do not copy)
+    uint32_t wbase[kWarps];   // each warp's first word inside the blob
+    uint32_t padw;            // code-length words of the blob
+};
+
 struct EncodeShared {
     alignas(16) float xbuf[kTile + 8];                             // staged input tile (+ guard word in front)
     alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];    // encoded tiles: current and awaiting placement
     uint32_t warp_words[2][kWarps];
-    LookShared look;
+    PlanShared plan;
     alignas(8) unsigned long long bar;
 };
 
@@ -936,6 +994,97 @@ __device__ __forceinline__ void place(const Pending& c, Anchor& anchor, const Jo
     if (tile == nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
 }
 
+// Sum of the sizes of tiles [lo, hi) of the launch, by one warp: all states are fetched in one round trip.
+__device__ __forceinline__ uint32_t sum_sizes_warp(const Workspace& ws, uint32_t lo, uint32_t hi, uint32_t epoch, int lane,
+                                                   uint32_t& skip, uint32_t& status)
+{
+    skip = 0;
+    if (hi <= lo) return 0;
+    int budget = kSpinLimit >> 4;
+    for (;;) {
+        uint32_t sum = 0;
+        bool good = true;
+        for (uint32_t base = lo; base < hi; base += 256) {
+            unsigned long long st[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t at = base + 32u * k + lane;
+                st[k] = (at < hi) ? ld_state(ws.tile_state + at) : pack_state(epoch, 0u, 0u);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if ((uint32_t)(st[k] >> 33) == epoch) sum += (uint32_t)st[k];
+                else good = false;
+            }
+        }
+        sum = __reduce_add_sync(kFull, sum);
+        if (__all_sync(kFull, good)) return sum;
+        if (--budget == 0) { skip = 1; status |= kStTimeout; return 0; }
+        __nanosleep(64);
+    }
+}
+
+// Warp 0, after the barrier that follows a tile's encoding pass: publishes the size of the tile just encoded
+// (`ticket`, sizes in `cur_words`) and plans the pending one (sizes in `pend_words`).
+__device__ __forceinline__ void announce_and_plan(PlanShared& plan, const uint32_t* cur_words, uint32_t cur_padw, uint32_t ticket,
+                                                  bool have_cur, const Pending& c, const uint32_t* pend_words, Anchor& anchor,
+                                                  const JobBatch& jb, float eb_abs, float s, const Workspace& ws,
+                                                  uint32_t epoch, int lane, uint32_t& status)
+{
+    if (have_cur) {
+        const uint32_t ww = lane < kWarps ? cur_words[lane] : 0u;
+        const uint32_t total = 1 + cur_padw + __reduce_add_sync(kFull, ww);
+        if (lane == 0 && ticket != ws.skip_publish) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
+    }
+    if (!c.valid) return;
+    const Job& job = jb.job[c.job];
+    const uint32_t tile = c.ticket - job.tile_begin;
+    const unsigned long long start = (unsigned long long)tile * kTile;
+    const uint32_t nT = (uint32_t)((job.n + kTile - 1) / kTile);
+    const uint32_t len = (uint32_t)((job.n - start < (unsigned long long)kTile) ? (job.n - start) : kTile);
+    const uint32_t padw = (((len + kBlock - 1) / kBlock) + 3) >> 2;
+    // exclusive scan of the warps' sizes across lanes 0..7
+    const uint32_t ww = lane < kWarps ? pend_words[lane] : 0u;
+    uint32_t inc = ww;
+#pragma unroll
+    for (int d = 1; d < kWarps; d <<= 1) {
+        const uint32_t up = __shfl_up_sync(kFull, inc, d);
+        if (lane >= d) inc += up;
+    }
+    const uint32_t total = 1 + padw + __shfl_sync(kFull, inc, kWarps - 1);
+    uint32_t lo = job.tile_begin, base = 0, skip = 0;
+    if (anchor.job == c.job) { lo = anchor.ticket + 1; base = anchor.incl; }
+    const uint32_t excl = base + sum_sizes_warp(ws, lo, c.ticket, epoch, lane, skip, status);
+    anchor.job = c.job; anchor.ticket = c.ticket; anchor.incl = excl + total;
+    const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
+    const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
+    if (!fits) status |= kStCapacity;
+    const bool go = fits && !skip;
+    uint32_t* blob_out = job.out + blob_word0;
+    if (lane < kWarps) plan.wbase[lane] = 1 + padw + inc - ww;
+    if (lane == 0) {
+        plan.blob_out = go ? blob_out : nullptr;
+        plan.padw = padw;
+        if (go) {
+            blob_out[0] = (uint32_t)c.q_first;
+            job.out[kHeaderWords + tile] = excl + total;
+        }
+        if (tile == nT - 1) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
+    }
+    if (tile == 0) write_header(job.out, lane, job.n, eb_abs, s, nT);
+}
+
+// Every warp, after the barrier that follows the plan: copy its own region of the pending tile.
+__device__ __forceinline__ void copy_planned(const PlanShared& plan, const Pending& c, const uint32_t* __restrict__ slots_w,
+                                             int warp, int lane)
+{
+    uint32_t* __restrict__ blob_out = plan.blob_out;
+    if (blob_out == nullptr) return;
+    uint32_t* __restrict__ dst = blob_out + plan.wbase[warp];
+    for (uint32_t i = lane; i < c.wsum; i += 32) dst[i] = slots_w[i];
+    if (lane < 4 && (uint32_t)(4 * warp + lane) < plan.padw) blob_out[1 + 4 * warp + lane] = c.my_lw;
+}
+
 // ------------------------------------------------------------------------------------------------ compress
 
 __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Workspace ws, Params hp, int use_dev_params)
@@ -968,7 +1117,6 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         stage(blockIdx.x);
     }
     __syncthreads();
-    uint32_t look_par = 0;
     uint32_t fills = 0;    // completed bulk copies (phase parity of the mbarrier)
     uint32_t p = 0;        // half of the slots the current tile is encoded into
     Pending pend;
@@ -1032,19 +1180,27 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps are visible; the staged tile has been consumed
-        if (tid == 0) stage(ticket + G);   // overlaps with the placement of the previous tile below
-
-        announce(sh.warp_words[p], (nb + 3) >> 2, ws, epoch, ticket, tid);
-        if (pend.valid)
-            place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
-                  sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, eb_abs, s, ws, epoch, tid, warp, lane, status);
+        if (warp == 0) {
+            if (lane == 0) stage(ticket + G);   // overlaps with the placement of the previous tile below
+            announce_and_plan(sh.plan, sh.warp_words[p], (nb + 3) >> 2, ticket, true, pend, sh.warp_words[pend.buf], anchor, jb,
+                              eb_abs, s, ws, epoch, lane, status);
+        }
+        if (pend.valid) {
+            __syncthreads();   // the plan is visible
+            copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+        }
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
         pend.q_first = q_first;
         p ^= 1u;
     }
-    if (pend.valid)
-        place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
-              sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, eb_abs, s, ws, epoch, tid, warp, lane, status);
+    if (pend.valid) {
+        __syncthreads();
+        if (warp == 0)
+            announce_and_plan(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, jb, eb_abs, s, ws, epoch,
+                              lane, status);
+        __syncthreads();
+        copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+    }
 
     // never leave with a bulk copy in flight into this CTA's shared memory: every copy that was started has been
     // waited for by the iteration that consumed it, except after an expired wait; then give it one more bounded wait
