@@ -139,6 +139,26 @@ struct Xpose {
     }
 };
 
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Per-lane constants of the packed store: with four blocks per transpose lane 8u + b ends up with plane b of
+// block u (b = 7: its sign word).
+struct PackLane {
+    uint32_t sh8;   // 8 * (lane / 8): position of this lane's block in a word of four per-block bytes
+    uint32_t wp;    // word of the block's slot this lane stores: 0 = sign word, b + 1 = plane b
+    __device__ __forceinline__ explicit PackLane(int lane)
+    {
+        sh8 = 8u * ((uint32_t)lane >> 3);
+        wp = ((uint32_t)(lane & 7) + 1u) & 7u;
+        asm volatile("" : "+r"(sh8), "+r"(wp));
+    }
+};
+
 __device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
 {
     int j = 0;
@@ -354,19 +374,38 @@ __device__ __forceinline__ void decode_blocks_f32(const uint2* __restrict__ tbl,
                                                   const Xpose& xp)
 {
     const uint32_t widx = (uint32_t)(lane + 1) & 31u;   // lane k fetches plane k (word k + 1), lane 31 the sign word
+    const PackLane pk(lane);
+    const uint2* my_tbl = tbl + (lane >> 3);
 #pragma unroll 1
     for (int g = 0; g < kBlocksPerWarp / 4; ++g) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int i = 4 * g + u;
-            const uint2 e = tbl[i];               // broadcast read: code length, shared address of the payload
-            const uint32_t sz = e.x ? e.x + 1 : 0;
+        const uint2 em = my_tbl[4 * g];           // entry of block 4g + lane / 8: code length, shared address of the payload
+        if (!__any_sync(kFull, em.x > 7u)) {
+            // four blocks per transpose: lane 8u + b fetches plane b of block u (b = 7: its sign word)
+            const uint32_t n = em.x ? em.x + 1 : 0;
             uint32_t w = 0;
-            if (widx < sz) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(e.y + 4 * widx) : "memory");
-            const uint32_t v = xp(w);             // bits 0..L-1: |delta| of this lane's element, bit 31: its sign
-            // exact fp32 value of the magnitude from its bits (|delta| < 2^23), then the sign bit on top
-            const float mag = __fsub_rn(__uint_as_float((v & 0x007FFFFFu) | 0x4B000000u), kTwo23);
-            wbuf[32 * i + (lane ^ (u << 2))] = __uint_as_float(__float_as_uint(mag) | (v & 0x80000000u));
+            if (pk.wp < n) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(em.y + 4 * pk.wp) : "memory");
+            const uint32_t v = xp(w);             // byte u: bits 0..6 = |delta| of this lane's element of block u, bit 7 = sign
+            const uint32_t vm = v & 0x7F7F7F7Fu;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = 4 * g + u;
+                const float mag = __fsub_rn(__uint_as_float(prmt(vm, 0x4B000000u, 0x7540u | (uint32_t)u)), kTwo23);
+                const uint32_t sg = prmt(v, v, (0x8u | (uint32_t)u) << 12);   // byte 3 = sign of byte u, replicated
+                wbuf[32 * i + (lane ^ (u << 2))] = __uint_as_float(__float_as_uint(mag) | (sg & 0x80000000u));
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = 4 * g + u;
+                const uint2 e = tbl[i];           // broadcast read
+                const uint32_t sz = e.x ? e.x + 1 : 0;
+                uint32_t w = 0;
+                if (widx < sz) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(e.y + 4 * widx) : "memory");
+                const uint32_t v = xp(w);         // bits 0..L-1: |delta| of this lane's element, bit 31: its sign
+                // exact fp32 value of the magnitude from its bits (|delta| < 2^23), then the sign bit on top
+                const float mag = __fsub_rn(__uint_as_float((v & 0x007FFFFFu) | 0x4B000000u), kTwo23);
+                wbuf[32 * i + (lane ^ (u << 2))] = __uint_as_float(__float_as_uint(mag) | (v & 0x80000000u));
+            }
         }
     }
 }
@@ -674,26 +713,6 @@ struct SrcSwizzled {        // the fused kernel's sum tile: per-warp region of 1
     }
     __device__ __forceinline__ float cur(int g, int u) const { return rows[32 * (4 * g + u + 1) + co[u]]; }
     __device__ __forceinline__ float prev(int g, int u) const { return rows[32 * (4 * g + u + 1) + po[u]]; }
-};
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
-{
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-// Per-lane constants of the packed store: with four blocks per transpose lane 8u + b ends up with plane b of
-// block u (b = 7: its sign word).
-struct PackLane {
-    uint32_t sh8;   // 8 * (lane / 8): position of this lane's block in a word of four per-block bytes
-    uint32_t wp;    // word of the block's slot this lane stores: 0 = sign word, b + 1 = plane b
-    __device__ __forceinline__ explicit PackLane(int lane)
-    {
-        sh8 = 8u * ((uint32_t)lane >> 3);
-        wp = ((uint32_t)(lane & 7) + 1u) & 7u;
-        asm volatile("" : "+r"(sh8), "+r"(wp));
-    }
 };
 
 // One pass over this warp's 16 blocks: quantise, 1-D Lorenzo delta, code length, sign word and bit planes, appended
