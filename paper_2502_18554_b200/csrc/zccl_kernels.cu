@@ -102,6 +102,12 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Asks for a 16-byte-aligned range of global memory to be brought into L2 (no destination, nothing to wait for).
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+
 // Bit planes by a 32 x 32 bit-matrix transpose across the warp.  Lane j holds the word of element j (bit k =
 // bit k of |delta_j|, bit 31 = its sign); after the transpose lane k holds plane k (bit j = that bit of element j)
 // and lane 31 the sign word.  Five butterfly stages exchange bit-index bit b with lane-index bit b (b = 4..0): one
@@ -499,6 +505,8 @@ struct StagePipe {
                 mbar_expect_tx(&sh.bar[buf], bytes);
                 bulk_load(sh.blob[buf], (const void*)a_beg, bytes, &sh.bar[buf]);
                 sp.staged = 1;
+                // the fused kernel adds a local operand to this tile: have it in L2 by then
+                if (jq.x && (((uintptr_t)(jq.x + start)) & 15u) == 0) bulk_prefetch_l2(jq.x + start, kTile * 4);
             }
         }
         sh.span[buf] = sp;
@@ -811,11 +819,6 @@ __device__ __forceinline__ int32_t first_code(float x0, float r)
     return __float2int_rn(t);
 }
 
-struct LookShared {
-    uint32_t part[2][kWarps];   // per-warp partial sums of tile sizes
-    uint32_t ok[2][kWarps];     // 1 if every state the warp inspected was published
-};
-
 // Placement split in two.  Everything about a pending tile that is the same for all threads (scan of the sizes,
 // layout of the warps' regions, capacity check, index entry, outlier, header, stream length) is done once, by warp 0,
 // which leaves the result here; after a barrier each warp only copies its own region.
@@ -845,7 +848,7 @@ struct FusedShared {
     int32_t warp_total_i[kWarps];
     int32_t warp_total_i2[kWarps];
     uint32_t warp_words[2][kWarps];
-    LookShared look;
+    PlanShared plan;
     alignas(8) unsigned long long bar[2];
 };
 
@@ -854,53 +857,6 @@ __device__ __forceinline__ bool stageable_raw(const Job& job, uint32_t tile)
 {
     const unsigned long long start = (unsigned long long)tile * kTile;
     return job.n - start >= (unsigned long long)kTile && (((uintptr_t)(job.x + start)) & 15u) == 0;
-}
-
-// Placement: sum of the sizes of tiles [lo, hi) of the launch, run by the whole CTA (window w of 32 states is
-// inspected by warp w mod 8).  With round-robin tiles a CTA anchors the scan at its own previous tile, whose
-// inclusive prefix it knows, so it only ever needs plain sizes, at most one grid's worth of them, all fetched in one
-// round trip; nothing depends on another CTA having placed anything.  Returns the sum (same in every thread); sets
-// `skip` when a size stayed unpublished beyond the poll limit.
-__device__ __forceinline__ uint32_t sum_sizes_cta(LookShared& ls, uint32_t& par, const Workspace& ws, uint32_t lo, uint32_t hi,
-                                                  uint32_t epoch, int warp, int lane, uint32_t& skip, uint32_t& status)
-{
-    skip = 0;
-    if (hi <= lo) return 0;
-    const uint32_t nwin = (hi - lo + 31u) >> 5;
-    int budget = kSpinLimit >> 4;
-    for (;;) {
-        uint32_t sum = 0;
-        bool good = true;
-        for (uint32_t w = warp; w < nwin; w += kWarps) {
-            const uint32_t at = lo + 32u * w + lane;
-            if (at < hi) {
-                const unsigned long long st = ld_state(ws.tile_state + at);
-                if ((uint32_t)(st >> 33) == epoch) sum += (uint32_t)st;
-                else good = false;
-            }
-        }
-        sum = __reduce_add_sync(kFull, sum);
-        good = __all_sync(kFull, good);
-        if (lane == 0) { ls.part[par][warp] = sum; ls.ok[par][warp] = good ? 1u : 0u; }
-        __syncthreads();
-        uint32_t total = 0, all_ok = 1;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) { total += ls.part[par][w]; all_ok &= ls.ok[par][w]; }
-        par ^= 1u;
-        if (all_ok) return total;
-        if (--budget == 0) { skip = 1; status |= kStTimeout; return 0; }   // uniform: every thread read the same words
-        __nanosleep(64);
-    }
-}
-
-// Copies this warp's contiguous region to its place in the stream; writes the warp's code-length words.
-__device__ __forceinline__ void copy_out_warp(uint32_t* __restrict__ blob_out, const uint32_t* __restrict__ slots_w,
-                                              uint32_t wbase, uint32_t wsum, uint32_t my_lw, uint32_t padw, int warp, int lane)
-{
-    uint32_t* __restrict__ dst = blob_out + wbase;
-    for (uint32_t i = lane; i < wsum; i += 32) dst[i] = slots_w[i];
-    if (lane < 4 && (uint32_t)(4 * warp + lane) < padw) blob_out[1 + 4 * warp + lane] = my_lw;
-    __syncwarp();
 }
 
 __device__ __forceinline__ void write_header(uint32_t* out, int tid, unsigned long long n, float eb_abs, float s, uint32_t nT)
@@ -954,64 +910,6 @@ struct Anchor {
     uint32_t ticket;
     uint32_t incl;       // inclusive prefix (words) of that tile within its job
 };
-
-// This warp's offset inside a tile's blob and the blob size, from the warps' payload sizes.
-__device__ __forceinline__ void blob_layout(const uint32_t* warp_words, uint32_t padw, int warp, uint32_t& wbase, uint32_t& total)
-{
-    wbase = 1 + padw;
-    total = 1 + padw;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        const uint32_t ww = warp_words[w];
-        if (w < warp) wbase += ww;
-        total += ww;
-    }
-}
-
-// After the barrier that follows a tile's encoding pass: the tile's size is published to the scan.
-__device__ __forceinline__ void announce(const uint32_t* warp_words, uint32_t padw, const Workspace& ws, uint32_t epoch,
-                                         uint32_t ticket, int tid)
-{
-    if (tid == 0 && ticket != ws.skip_publish) {
-        uint32_t total = 1 + padw;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) total += warp_words[w];
-        st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
-    }
-}
-
-// Places a pending tile: exclusive prefix = anchor + sizes of the tiles in between, then copy-out, index entry,
-// header and stream length.
-__device__ __forceinline__ void place(const Pending& c, Anchor& anchor, const JobBatch& jb, LookShared& look, uint32_t& look_par,
-                                      const uint32_t* warp_words, const uint32_t* slots_w, float eb_abs, float s,
-                                      const Workspace& ws, uint32_t epoch, int tid, int warp, int lane, uint32_t& status)
-{
-    const Job& job = jb.job[c.job];
-    const uint32_t tile = c.ticket - job.tile_begin;
-    const unsigned long long start = (unsigned long long)tile * kTile;
-    const uint32_t nT = (uint32_t)((job.n + kTile - 1) / kTile);
-    const uint32_t len = (uint32_t)((job.n - start < (unsigned long long)kTile) ? (job.n - start) : kTile);
-    const uint32_t padw = (((len + kBlock - 1) / kBlock) + 3) >> 2;
-    uint32_t wbase, total;
-    blob_layout(warp_words, padw, warp, wbase, total);
-    uint32_t lo = job.tile_begin, base = 0, skip = 0;
-    if (anchor.job == c.job) { lo = anchor.ticket + 1; base = anchor.incl; }
-    const uint32_t excl = base + sum_sizes_cta(look, look_par, ws, lo, c.ticket, epoch, warp, lane, skip, status);
-    anchor.job = c.job; anchor.ticket = c.ticket; anchor.incl = excl + total;
-    const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
-    const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
-    if (!fits) status |= kStCapacity;
-    if (fits && !skip) {
-        uint32_t* blob_out = job.out + blob_word0;
-        copy_out_warp(blob_out, slots_w, wbase, c.wsum, c.my_lw, padw, warp, lane);
-        if (tid == 0) {
-            blob_out[0] = (uint32_t)c.q_first;
-            job.out[kHeaderWords + tile] = excl + total;
-        }
-    }
-    if (tile == 0) write_header(job.out, tid, job.n, eb_abs, s, nT);
-    if (tile == nT - 1 && tid == 0) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
-}
 
 // Sum of the sizes of tiles [lo, hi) of the launch, by one warp: all states are fetched in one round trip.
 __device__ __forceinline__ uint32_t sum_sizes_warp(const Workspace& ws, uint32_t lo, uint32_t hi, uint32_t epoch, int lane,
@@ -1240,7 +1138,6 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     const uint32_t G = gridDim.x;
     uint32_t status = 0;
     uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed per staging buffer
-    uint32_t look_par = 0;
     uint32_t p = 0;                    // half of the slots and staging buffer of the current tile
     float pend_eb = 0.0f, pend_s = 1.0f;   // bound and step of the pending tile's job (header fields)
     Pending pend;
@@ -1252,6 +1149,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     StreamInfo h1, h2;
     h1.ok = h2.ok = false; h1.n = h2.n = 0; h1.nT = h2.nT = 0; h1.s = h2.s = 1.0f; h1.eb_abs = h2.eb_abs = 0.0f;
     bool job_ok = false;
+    float r = 1.0f;   // reciprocal of the current job's step
 
     StagePipe pipe;   // thread 0 only
     if (tid == 0) {
@@ -1278,9 +1176,9 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 h2 = read_header(job.in_c2, job.in2_cap);
                 job_ok = job_ok && h2.ok && h2.n == n && __float_as_uint(h2.s) == __float_as_uint(h1.s);
             }
+            r = __fdiv_rn(1.0f, h1.s);
         }
         const float s = h1.s, eb_abs = h1.eb_abs;
-        const float r = __fdiv_rn(1.0f, s);
 
         // thread 0: request the next tile's blob into the other staging buffer (its readers finished before the last
         // barrier of the previous iteration), then fetch the index entries of the tile after it
@@ -1324,7 +1222,6 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             // this thread's 16 consecutive elements of the local operand are needed after the scan: pull their lines
             // towards L2 now, load them (128-bit when aligned) when they are used
             const float* lp = loc + 512 * warp + 16 * lane;
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(lp));
             const unsigned long long blob0 = (unsigned long long)kHeaderWords + h1.nT;
             const uint32_t shift = (uint32_t)(((uintptr_t)(job.in_c + blob0 + sp.w_beg) & 15u) >> 2);
             const uint32_t* sb = sh.blob[p] + shift;
@@ -1350,22 +1247,35 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 const int sw = (lane >> 1) & 3;
                 float4* row = reinterpret_cast<float4*>(yrows + 32 + 16 * lane);
                 float4* gout = yout ? reinterpret_cast<float4*>(yout + 512 * warp + 16 * lane) : nullptr;
-                const bool gvec = (((uintptr_t)gout) & 15u) == 0;
-                const bool lvec = (((uintptr_t)lp) & 15u) == 0;
+                // alignment and the presence of an uncompressed output are the same for every thread of the launch's job
+                const bool lvec = (((uintptr_t)loc) & 15u) == 0;
+                const bool store = gout != nullptr && !deq;
+                const bool gvec = (((uintptr_t)yout) & 15u) == 0;
+                if (lvec && (!store || gvec)) {
+                    float4 l[4];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    float4 l;
-                    if (lvec) l = __ldg(reinterpret_cast<const float4*>(lp) + c);
-                    else { l.x = __ldg(lp + 4 * c); l.y = __ldg(lp + 4 * c + 1); l.z = __ldg(lp + 4 * c + 2); l.w = __ldg(lp + 4 * c + 3); }
-                    float4 o;
-                    o.x = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), l.x);
-                    o.y = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), l.y);
-                    o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), l.z);
-                    o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), l.w);
-                    row[c ^ sw] = o;
-                    if (gout && !deq) {
-                        if (gvec) gout[c] = o;
-                        else { float* g = reinterpret_cast<float*>(gout + c); g[0] = o.x; g[1] = o.y; g[2] = o.z; g[3] = o.w; }
+                    for (int c = 0; c < 4; ++c) l[c] = __ldg(reinterpret_cast<const float4*>(lp) + c);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float4 o;
+                        o.x = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), l[c].x);
+                        o.y = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), l[c].y);
+                        o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), l[c].z);
+                        o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), l[c].w);
+                        row[c ^ sw] = o;
+                        if (store) gout[c] = o;
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float4 l, o;
+                        l.x = __ldg(lp + 4 * c); l.y = __ldg(lp + 4 * c + 1); l.z = __ldg(lp + 4 * c + 2); l.w = __ldg(lp + 4 * c + 3);
+                        o.x = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), l.x);
+                        o.y = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), l.y);
+                        o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), l.z);
+                        o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), l.w);
+                        row[c ^ sw] = o;
+                        if (store) { float* g = reinterpret_cast<float*>(gout + c); g[0] = o.x; g[1] = o.y; g[2] = o.z; g[3] = o.w; }
                     }
                 }
                 __syncwarp();
@@ -1462,17 +1372,25 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps
-        announce(sh.warp_words[p], padw, ws, epoch, ticket, tid);
-        if (pend.valid)
-            place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
-                  sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, pend_eb, pend_s, ws, epoch, tid, warp, lane, status);
+        if (warp == 0)
+            announce_and_plan(sh.plan, sh.warp_words[p], padw, ticket, true, pend, sh.warp_words[pend.buf], anchor, jb, pend_eb, pend_s,
+                              ws, epoch, lane, status);
+        if (pend.valid) {
+            __syncthreads();   // the plan is visible
+            copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+        }
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
         pend.q_first = q_first;
         pend_eb = eb_abs; pend_s = s;
     }
-    if (pend.valid)
-        place(pend, anchor, jb, sh.look, look_par, sh.warp_words[pend.buf],
-              sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, pend_eb, pend_s, ws, epoch, tid, warp, lane, status);
+    if (pend.valid) {
+        __syncthreads();
+        if (warp == 0)
+            announce_and_plan(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, jb, pend_eb, pend_s, ws, epoch,
+                              lane, status);
+        __syncthreads();
+        copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+    }
     if (tid == 0 && (status & kStTimeout)) {
         (void)mbar_wait(&sh.bar[0], (fills0 + 1u) & 1u);
         (void)mbar_wait(&sh.bar[1], (fills1 + 1u) & 1u);
