@@ -1151,16 +1151,29 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     bool job_ok = false;
     float r = 1.0f;   // reciprocal of the current job's step
 
-    StagePipe pipe;   // thread 0 only
+    // The first thread of warp 1 requests the blobs: it does so while warp 0 plans a placement, when the other
+    // warps have nothing to do.
+    StagePipe pipe;   // thread 32 only
     if (tid == 0) {
         mbar_init(&sh.bar[0], 1);
         mbar_init(&sh.bar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 32) {
         pipe.fetch(jb, blockIdx.x, cur_job, h1);
         pipe.stage(sh, jb, blockIdx.x, cur_job, h1, 0);
         pipe.fetch(jb, blockIdx.x + G, cur_job, h1);
     }
     __syncthreads();
+    // requests the next tile's blob into the other staging buffer (its readers finished before the last barrier), then
+    // fetches the index entries of the tile after it; a barrier follows before the span is read
+    auto stage_next = [&](uint32_t ticket) {
+        if (tid == 32) {
+            pipe.stage(sh, jb, ticket + G, cur_job, h1, p ^ 1u);
+            pipe.fetch(jb, ticket + 2 * G, cur_job, h1);
+        }
+    };
 
     for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += G, p ^= 1u) {
         const int j = find_job(jb, ticket);
@@ -1180,12 +1193,6 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
         const float s = h1.s, eb_abs = h1.eb_abs;
 
-        // thread 0: request the next tile's blob into the other staging buffer (its readers finished before the last
-        // barrier of the previous iteration), then fetch the index entries of the tile after it
-        if (tid == 0) {
-            pipe.stage(sh, jb, ticket + G, cur_job, h1, p ^ 1u);
-            pipe.fetch(jb, ticket + 2 * G, cur_job, h1);
-        }
         const BlobSpan sp = sh.span[p];
         if (sp.staged) {   // a copy was requested for this tile: always consume it, whatever happens next
             const uint32_t fl = p ? fills1 : fills0;
@@ -1201,6 +1208,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 if (tile == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
             }
             if (hdr && tile == 0) write_header(job.out, tid, 0, eb_abs, s, 0);
+            stage_next(ticket);
             __syncthreads();
             continue;
         }
@@ -1334,6 +1342,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 st_state(ws.tile_state + ticket, pack_state(epoch, 0u, 0u));
                 if (tile == nT - 1) *job.out_bytes = 0;
             }
+            stage_next(ticket);
             __syncthreads();
             continue;
         }
@@ -1375,8 +1384,9 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         if (warp == 0)
             announce_and_plan(sh.plan, sh.warp_words[p], padw, ticket, true, pend, sh.warp_words[pend.buf], anchor, jb, pend_eb, pend_s,
                               ws, epoch, lane, status);
+        stage_next(ticket);
+        __syncthreads();   // the plan and the next tile's span are visible
         if (pend.valid) {
-            __syncthreads();   // the plan is visible
             copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
         }
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
