@@ -1238,6 +1238,8 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             if (mode == 1) {
                 decode_blocks_f32(sh.tbl + kBlocksPerWarp * warp, yrows + 32, lane, xp);
                 __syncwarp();
+                // lane 0 needs the local operand's element before the warp's first one after the barrier below
+                const float lprev = (lane == 0 && warp != 0) ? __ldg(loc + 512 * warp - 1) : 0.0f;
                 float v[16];
                 const float total = decode_scan_f32(yrows + 32, lane, v);
                 if (lane == 0) sh.warp_total[warp] = total;
@@ -1249,7 +1251,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 if (lane == 0) {
                     float yprev;
                     if (warp == 0) yprev = __fadd_rn(__fmul_rn(__fadd_rn(v[0], base), s), __ldg(loc));
-                    else yprev = __fadd_rn(__fmul_rn(base, s), __ldg(loc + 512 * warp - 1));
+                    else yprev = __fadd_rn(__fmul_rn(base, s), lprev);
                     yrows[31 ^ 12] = yprev;   // guard row, element 31 under the swizzle of the row before row 0
                 }
                 const int sw = (lane >> 1) & 3;
