@@ -518,48 +518,45 @@ struct DecodeShared {
     alignas(16) float wbuf[kWarps][kBlocksPerWarp * kBlock];
     alignas(16) uint2 tbl[kBlocksPerTile];                    // per block {code length, shared address of its payload}
     BlobSpan span[2];
-    uint32_t sz_part[4];                                      // describe: payload words of blocks 32w .. 32w+31
-    uint32_t spread_part[4];
     float warp_total[2][kWarps];
     int32_t warp_total_i[kWarps];
     alignas(8) unsigned long long bar[2];
 };
 
-// Cooperative description of a staged full tile: thread b (b < 128) owns block b.  Builds the block table, checks
-// the code lengths against the blob size and decides whether the tile's codes stay exact in fp32.
-// Two barriers.  Returns 0: inconsistent blob, 1: take the fp32 path, 2: consistent but needs the integer path.
-template <class Shared>
-__device__ __forceinline__ int describe_staged(Shared& sh, const uint32_t* sb, uint32_t words, int tid, int lane, int warp)
+// Description of a staged full tile, by every warp on its own (no barrier): lane l reads the code lengths of blocks
+// 4l .. 4l+3, a warp-wide scan gives every block's payload offset, and the lanes that hold the warp's own 16 blocks
+// write their entries of the block table {code length, shared address of the payload}.  Checks the code lengths
+// against the blob size and decides whether the tile's codes stay exact in fp32.  Every warp reaches the same
+// verdict.  Returns 0: inconsistent blob, 1: take the fp32 path, 2: consistent but needs the integer path.
+__device__ __forceinline__ int describe_staged(uint2* __restrict__ tbl, const uint32_t* sb, uint32_t words, int lane, int warp)
 {
     constexpr uint32_t padw = kBlocksPerTile / 4;
-    bool good = true;
-    uint32_t L = 0, sz = 0, incl = 0;
-    if (tid < kBlocksPerTile) {
-        L = reinterpret_cast<const unsigned char*>(sb + 1)[tid];
-        good = L <= 31u;
-        sz = L ? L + 1 : 0;
-        incl = sz;
+    const uint32_t lw = sb[1 + lane];
+    const uint32_t L0 = lw & 0xFFu, L1 = (lw >> 8) & 0xFFu, L2 = (lw >> 16) & 0xFFu, L3 = lw >> 24;
+    const bool bad = ((lw & 0xE0E0E0E0u) != 0u);   // a code length above 31
+    const uint32_t z0 = L0 ? L0 + 1 : 0, z1 = L1 ? L1 + 1 : 0, z2 = L2 ? L2 + 1 : 0, z3 = L3 ? L3 + 1 : 0;
+    const uint32_t lane_sum = z0 + z1 + z2 + z3;
+    uint32_t incl = lane_sum;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t t = __shfl_up_sync(kFull, incl, d);
-            if (lane >= d) incl += t;
-        }
-        const uint32_t spread = __reduce_add_sync(kFull, L <= (uint32_t)kFastDecodeMaxL ? (32u << L) : (1u << 24));
-        if (lane == 31) { sh.sz_part[warp] = incl; sh.spread_part[warp] = spread; }
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(kFull, incl, d);
+        if (lane >= d) incl += t;
     }
-    __syncthreads();
-    uint32_t total = 0, spread = 0;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-        const uint32_t pw = sh.sz_part[w];
-        if (w < warp) incl += pw;
-        total += pw;
-        spread += min(sh.spread_part[w], 1u << 24);
+    const uint32_t total = __shfl_sync(kFull, incl, 31);
+    const uint32_t Lmax = max(max(L0, L1), max(L2, L3));
+    uint32_t spread = 1u << 24;
+    if (Lmax <= (uint32_t)kFastDecodeMaxL) spread = (32u << L0) + (32u << L1) + (32u << L2) + (32u << L3);
+    spread = __reduce_add_sync(kFull, min(spread, 1u << 24));   // at most 32 * 2^24 = 2^29: no overflow
+    if (__any_sync(kFull, bad) || 1 + padw + total != words) return 0;
+    if ((lane >> 2) == warp) {   // this lane's four blocks are blocks 4 (lane & 3) .. of the warp
+        const uint32_t a0 = smem_u32(sb + 1 + padw) + 4 * (incl - lane_sum);
+        uint2* e = tbl + kBlocksPerWarp * warp + 4 * (lane & 3);
+        e[0] = make_uint2(L0, a0);
+        e[1] = make_uint2(L1, a0 + 4 * z0);
+        e[2] = make_uint2(L2, a0 + 4 * (z0 + z1));
+        e[3] = make_uint2(L3, a0 + 4 * (z0 + z1 + z2));
     }
-    if (tid < kBlocksPerTile) sh.tbl[tid] = make_uint2(L, smem_u32(sb + 1 + padw) + 4 * (incl - sz));
-    good = good && (1 + padw + total == words);
-    const int all_good = __syncthreads_and(good ? 1 : 0);
-    if (!all_good) return 0;
+    __syncwarp();
     const int32_t outlier = (int32_t)sb[0];
     const uint32_t ao = (uint32_t)(outlier < 0 ? -outlier : outlier);
     return (ao < (1u << 23) && spread < (1u << 23)) ? 1 : 2;
@@ -619,7 +616,7 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
             const unsigned long long blob0 = (unsigned long long)kHeaderWords + h.nT;
             const uint32_t shift = (uint32_t)(((uintptr_t)(job.in_c + blob0 + sp.w_beg) & 15u) >> 2);
             const uint32_t* sb = sh.blob[p] + shift;
-            mode = describe_staged(sh, sb, sp.w_end - sp.w_beg, tid, lane, warp);
+            mode = describe_staged(sh.tbl, sb, sp.w_end - sp.w_beg, lane, warp);
             if (mode == 0) { status |= kStBadStream; skip_tile = true; }
             if (mode == 1) {
                 float* __restrict__ y = job.y + (unsigned long long)tile * kTile;
@@ -842,8 +839,6 @@ struct FusedShared {
     alignas(16) uint2 tbl[kBlocksPerTile];
     alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];
     BlobSpan span[2];
-    uint32_t sz_part[4];
-    uint32_t spread_part[4];
     float warp_total[kWarps];
     int32_t warp_total_i[kWarps];
     int32_t warp_total_i2[kWarps];
@@ -1233,7 +1228,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             const unsigned long long blob0 = (unsigned long long)kHeaderWords + h1.nT;
             const uint32_t shift = (uint32_t)(((uintptr_t)(job.in_c + blob0 + sp.w_beg) & 15u) >> 2);
             const uint32_t* sb = sh.blob[p] + shift;
-            mode = describe_staged(sh, sb, sp.w_end - sp.w_beg, tid, lane, warp);
+            mode = describe_staged(sh.tbl, sb, sp.w_end - sp.w_beg, lane, warp);
             if (mode == 0) bad_tile = true;
             if (mode == 1) {
                 decode_blocks_f32(sh.tbl + kBlocksPerWarp * warp, yrows + 32, lane, xp);
