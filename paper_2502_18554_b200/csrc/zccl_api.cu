@@ -381,19 +381,17 @@ int zccl_sim_allreduce(zccl_ctx* c, const float* const* send, float* const* recv
         uint8_t* t = cur; cur = nxt; nxt = t;
     }
 
-    // allgather stage: N-1 forwarding hops of compressed chunks between per-rank slots
-    const size_t* own_sz = hop_sz + (size_t)(N - 1) * N;   // rank r owns chunk (r+1) mod N in cur[r]
-    CopyBatcher cb;
-    for (int h = 0; h + 1 < N; ++h) {
+    // allgather stage: N-1 forwarding hops of compressed chunks between per-rank slots, all in one launch.  Rank r
+    // owns chunk (r+1) mod N in cur[r]; hop h hands it to rank r+1+h.
+    const size_t* own_sz = hop_sz + (size_t)(N - 1) * N;
+    {
+        ChainBatch cb{};
+        cb.slots = gs0; cb.sizes = g_sz; cb.slot_bytes = slot; cb.N = N; cb.hops = N - 1; cb.count = N;
         for (int r = 0; r < N; ++r) {
-            const int from = (r - 1 + N) % N;
-            const int ch = ((r - h) % N + N) % N;
-            const uint8_t* src = h == 0 ? cur + (size_t)from * slot : gslot(from, ch);
-            const size_t* sz = h == 0 ? own_sz + from : g_sz + (size_t)from * N + ch;
-            cb.add(src, gslot(r, ch), sz, g_sz + (size_t)r * N + ch, slot);
-            if (cb.full() && (rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+            ChainJob& j = cb.job[r];
+            j.src0 = (const uint32_t*)(cur + (size_t)r * slot); j.bytes = own_sz + r; j.first_rank = (r + 1) % N; j.chunk = (r + 1) % N;
         }
-        if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+        if ((rc = cuda_rc(launch_copy_chain(cb, c->ws, c->sm_count, st))) != ZCCL_OK) return rc;
     }
     // every rank decompresses the chunks it does not own
     for (int r = 0; r < N; ++r) {
@@ -440,16 +438,14 @@ int zccl_sim_allgather(zccl_ctx* c, const float* const* send, float* const* recv
     }
     if ((rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
 
-    CopyBatcher cb;
-    for (int h = 0; h + 1 < N; ++h) {   // forward compressed bytes around the ring
+    if (N > 1) {   // forward compressed bytes around the ring: hop h hands rank r's contribution to rank r+1+h
+        ChainBatch cb{};
+        cb.slots = c->arena; cb.sizes = g_sz; cb.slot_bytes = slot; cb.N = N; cb.hops = N - 1; cb.count = N;
         for (int r = 0; r < N; ++r) {
-            const int from = (r - 1 + N) % N;
-            const int src = ((r - 1 - h) % N + N) % N;
-            const size_t* sz = h == 0 ? own_sz + from : g_sz + (size_t)from * N + src;
-            cb.add(gslot(from, src), gslot(r, src), sz, g_sz + (size_t)r * N + src, slot);
-            if (cb.full() && (rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+            ChainJob& j = cb.job[r];
+            j.src0 = (const uint32_t*)gslot(r, r); j.bytes = own_sz + r; j.first_rank = (r + 1) % N; j.chunk = r;
         }
-        if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+        if ((rc = cuda_rc(launch_copy_chain(cb, c->ws, c->sm_count, st))) != ZCCL_OK) return rc;
     }
     for (int r = 0; r < N; ++r) {
         for (int src = 0; src < N; ++src) {

@@ -83,6 +83,25 @@ struct CopyBatch {
     int count;
 };
 
+// All forwarding hops of a ring Allgather stage in one launch.  Chain c carries one compressed chunk from its
+// first holder around the ring: hop h copies it from where hop h - 1 left it to the slot of rank
+// (first_rank + h) mod N.  Slots are laid out regularly: rank r keeps chunk c at slots + (r * N + c) * slot_bytes
+// and its length at sizes[r * N + c].
+constexpr int kMaxChains = 64;
+struct ChainJob {
+    const uint32_t* src0;   // where the chunk is before the first hop
+    const size_t* bytes;    // its device-resident length
+    int first_rank;         // receiver of the first hop
+    int chunk;
+};
+struct ChainBatch {
+    ChainJob job[kMaxChains];
+    unsigned char* slots;
+    size_t* sizes;
+    unsigned long long slot_bytes;
+    int N, hops, count;
+};
+
 struct RangeBatch {
     const float* x[kMaxJobs];
     unsigned long long n[kMaxJobs];
@@ -98,6 +117,7 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
 unsigned long long launch_count();
 
 }  // namespace zccl
