@@ -133,6 +133,13 @@ struct CopyBatcher {
     {
         CopyJob& j = cb.job[cb.count++];
         j.src = (const uint32_t*)src; j.dst = (uint32_t*)dst; j.bytes = bytes; j.bytes_out = bytes_out; j.cap = cap;
+        j.fixed_bytes = 0;
+    }
+    void add_fixed(const void* src, void* dst, size_t nbytes)   // a copy whose length the host knows
+    {
+        CopyJob& j = cb.job[cb.count++];
+        j.src = (const uint32_t*)src; j.dst = (uint32_t*)dst; j.bytes = nullptr; j.bytes_out = nullptr; j.cap = nbytes;
+        j.fixed_bytes = nbytes;
     }
     bool full() const { return cb.count == kMaxJobs; }
 };
@@ -447,13 +454,17 @@ int zccl_sim_allgather(zccl_ctx* c, const float* const* send, float* const* recv
         }
         if ((rc = cuda_rc(launch_copy_chain(cb, c->ws, c->sm_count, st))) != ZCCL_OK) return rc;
     }
+    {   // own contributions stay uncompressed: one launch copies them all
+        CopyBatcher cb;
+        for (int r = 0; r < N; ++r) {
+            cb.add_fixed(send[r], recv[r] + (size_t)r * n, sizeof(float) * n);
+            if (cb.full() && (rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+        }
+        if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+    }
     for (int r = 0; r < N; ++r) {
         for (int src = 0; src < N; ++src) {
-            if (src == r) {   // own contribution stays uncompressed
-                if (cudaMemcpyAsync(recv[r] + (size_t)src * n, send[r], sizeof(float) * n, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-                    return ZCCL_E_CUDA;
-                continue;
-            }
+            if (src == r) continue;
             Job j{};
             j.in_c = (const uint32_t*)gslot(r, src); j.in_cap = slot; j.y = recv[r] + (size_t)src * n; j.n = n;
             b.add(j, tiles_of(n));

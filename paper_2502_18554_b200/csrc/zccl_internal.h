@@ -16,7 +16,7 @@ constexpr int kBlocksPerTile = kTile / kBlock;
 constexpr int kThreads = 256;               // one CTA works on one tile at a time
 constexpr int kWarps = kThreads / 32;
 constexpr int kBlocksPerWarp = kBlocksPerTile / kWarps;   // 16 consecutive blocks per warp
-constexpr int kMaxJobs = 16;                // chunk-operations batched into one launch
+constexpr int kMaxJobs = 64;                // chunk-operations per launch (8 ranks x 7 chunks of a ring stage fit one launch)
 
 // Device status bits (zccl_status maps them to return codes).
 enum : uint32_t {
@@ -74,9 +74,10 @@ struct JobBatch {
 struct CopyJob {
     const uint32_t* src;
     uint32_t* dst;
-    const size_t* bytes;   // device-resident length
+    const size_t* bytes;   // device-resident length (nullptr: the length is `fixed_bytes`)
     size_t* bytes_out;     // optional: where to record the length at the destination
     unsigned long long cap;
+    unsigned long long fixed_bytes;
 };
 struct CopyBatch {
     CopyJob job[kMaxJobs];

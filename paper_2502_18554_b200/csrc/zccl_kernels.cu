@@ -165,13 +165,17 @@ struct PackLane {
     }
 };
 
+// The job that owns tile number `ticket` of the launch: the last one whose first tile is not beyond it.
 __device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
 {
-    int j = 0;
+    int lo = 0, hi = jb.count;
 #pragma unroll 1
-    for (int k = 1; k < jb.count; ++k)
-        if (jb.job[k].tile_begin <= ticket) j = k;
-    return j;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (jb.job[mid].tile_begin <= ticket) lo = mid;
+        else hi = mid;
+    }
+    return lo;
 }
 
 // ------------------------------------------------------------------------------------------------ range (REL)
@@ -1412,7 +1416,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
 __global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
 {
     const CopyJob& job = cb.job[blockIdx.y];
-    const unsigned long long bytes = *job.bytes;
+    const unsigned long long bytes = job.bytes ? *job.bytes : job.fixed_bytes;
     if (bytes > job.cap) {
         if (threadIdx.x == 0 && blockIdx.x == 0) { atomicOr(ws.status, kStCapacity); if (job.bytes_out) *job.bytes_out = 0; }
         return;
