@@ -1096,8 +1096,8 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps are visible; the staged tile has been consumed
+        if (tid == 32) stage(ticket + G);   // by warp 1, while warp 0 plans the placement of the previous tile
         if (warp == 0) {
-            if (lane == 0) stage(ticket + G);   // overlaps with the placement of the previous tile below
             announce_and_plan(sh.plan, sh.warp_words[p], (nb + 3) >> 2, ticket, true, pend, sh.warp_words[pend.buf], anchor, jb,
                               eb_abs, s, ws, epoch, lane, status);
         }
