@@ -885,7 +885,12 @@ __device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoc
         if (prev == gridDim.x - 1) {   // every CTA is done with the scan states: re-arm for the next launch
             *ws.done = 0;
             uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
-            *ws.epoch = e ? e : 1u;
+            if (e == 0) {   // the counter wraps (once in 2^31 launches): no state of an earlier launch may look current again
+                for (uint32_t t = 0; t < ws.max_tiles; ++t) st_state(ws.tile_state + t, 0ull);
+                __threadfence();
+                e = 1u;
+            }
+            *ws.epoch = e;
         }
     }
 }
