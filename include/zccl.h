@@ -92,6 +92,14 @@ unsigned long long zccl_launch_count(void);
  */
 int zccl_debug_skip_publish(zccl_ctx* ctx, long long tile);
 
+/*
+ * Test hook for the launch counter that validates the scan states (no paper counterpart): sets it to `value`
+ * (1 .. 2^31 - 1) on `stream`, so that a test can run the launches on both sides of its wrap-around, where every
+ * scan state is cleared.  Must not overlap with other work on the context.  Returns ZCCL_E_ARG for a value
+ * outside the range, ZCCL_E_CUDA if the copy cannot be queued.
+ */
+int zccl_debug_set_launch_counter(zccl_ctx* ctx, unsigned int value, void* stream);
+
 /* Static description of a status code. */
 const char* zccl_strerror(int code);
 

@@ -58,6 +58,10 @@ def lib():
         L.zo_sim_allgather.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
                                        C.c_void_p]
         L.zo_sim_bcast.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32, szp]
+        L.zo_sim_reduce_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
+                                            C.c_void_p]
+        L.zo_sim_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
+                                     C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -200,3 +204,37 @@ def sim_bcast(root, nsinks: int, eb_mode: int, eb: float, T: int = DEFAULT_TILE)
     if rc < 0:
         raise OracleError(rc, "sim_bcast")
     return recv, rc, sb.value
+
+
+def chunk_span(n: int, N: int, c: int):
+    """Offset and length of chunk c when n elements are split into N chunks of ceil(n / N) (the last ones shorter)."""
+    m = (n + N - 1) // N
+    off = min(c * m, n)
+    return off, min(m, n - off)
+
+
+def sim_reduce_scatter(send, eb_mode: int, eb: float, T: int = DEFAULT_TILE):
+    """Ring Reduce-scatter: recv[r] = chunk r of the sum.  Returns (recv, rc, hop_bytes[(N-1) x N])."""
+    send = [_f32(a) for a in send]
+    N, n = len(send), send[0].size
+    recv = [np.zeros(chunk_span(n, N, r)[1], np.float32) for r in range(N)]
+    hop = np.zeros(max(N - 1, 1) * N, dtype=np.uintp)
+    rc = lib().zo_sim_reduce_scatter(_ptr_array(send), _ptr_array(recv), N, n, eb_mode, eb, T, _ptr(hop))
+    if rc < 0:
+        raise OracleError(rc, "sim_reduce_scatter")
+    return recv, rc, hop.reshape(max(N - 1, 1), N)
+
+
+def sim_scatter(root, N: int, eb_mode: int, eb: float, T: int = DEFAULT_TILE):
+    """Binomial-tree Scatter of N chunks held by rank 0.  Returns (recv, rc, sizes[N], round_bytes)."""
+    root = _f32(root)
+    assert root.size % N == 0
+    n = root.size // N
+    recv = [np.zeros(n, np.float32) for _ in range(N)]
+    sizes = np.zeros(N, dtype=np.uintp)
+    rounds = np.zeros(32, dtype=np.uintp)
+    rc = lib().zo_sim_scatter(_ptr(root), _ptr_array(recv), N, n, eb_mode, eb, T, _ptr(sizes), _ptr(rounds))
+    if rc < 0:
+        raise OracleError(rc, "sim_scatter")
+    nrounds = max(N - 1, 0).bit_length()
+    return recv, rc, sizes, rounds[:nrounds]

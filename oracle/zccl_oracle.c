@@ -502,3 +502,94 @@ int zo_sim_bcast(const float *root, float *const *recv, int nsinks, size_t n, in
     if (rc < 0) return rc;
     return warn ? ZO_W_PRECISION : ZO_OK;
 }
+
+/* Ring Reduce-scatter in the collective computation framework (Section 3.1.2; first stage of the Allreduce of
+ * Section 3.1.3), as a collective of its own: rank r ends with chunk r of the element-wise sum, uncompressed.
+ * Chunk c starts at rank c+1 (compressed there), travels c+1 -> c+2 -> ... -> c, and every receiver decompresses,
+ * adds its own chunk c and, unless it is the last one, compresses the partial sum again: N-1 compressions per
+ * chunk, the last rank keeps the sum it formed.  recv[r] holds the elements of chunk r.
+ * hop_bytes (optional, (N-1)*N entries): hop_bytes[k*N + r] = compressed bytes rank r sent in step k. */
+int zo_sim_reduce_scatter(const float *const *send, float *const *recv, int N, size_t n, int eb_mode, float eb,
+                          uint32_t T, size_t *hop_bytes)
+{
+    if (N < 1) return ZO_E_ARG;
+    float eb_abs, s, r;
+    int rc = resolve_over_ranks(send, N, n, eb_mode, eb, &eb_abs, &s, &r);
+    if (rc != ZO_OK) return rc;
+    size_t m = (n + (size_t)N - 1) / (size_t)N;
+    size_t cap = zo_compress_bound(m, T);
+    int warn = 0;
+    if (N == 1) { memcpy(recv[0], send[0], sizeof(float) * n); return ZO_OK; }
+    uint8_t **cur = (uint8_t **)calloc((size_t)N, sizeof(uint8_t *));
+    uint8_t **nxt = (uint8_t **)calloc((size_t)N, sizeof(uint8_t *));
+    size_t *cur_b = (size_t *)calloc((size_t)N, sizeof(size_t));
+    size_t *nxt_b = (size_t *)calloc((size_t)N, sizeof(size_t));
+    for (int k = 0; k < N; ++k) { cur[k] = (uint8_t *)malloc(cap); nxt[k] = (uint8_t *)malloc(cap); }
+
+    for (int rk = 0; rk < N && rc >= 0; ++rk) {          /* step 0: rank rk compresses chunk rk-1 */
+        int c = (rk - 1 + N) % N;
+        size_t off, len; chunk_span(n, N, c, &off, &len);
+        rc = zo_compress_core(send[rk] + off, len, eb_abs, s, r, T, cur[rk], cap, &cur_b[rk]);
+        if (rc == ZO_W_PRECISION) warn = 1;
+        if (hop_bytes) hop_bytes[rk] = cur_b[rk];
+    }
+    for (int k = 0; k + 1 < N && rc >= 0; ++k) {           /* step k+1: rank rk receives chunk rk-k-2 from rk-1 */
+        int last = (k == N - 2);
+        for (int rk = 0; rk < N && rc >= 0; ++rk) {
+            int from = (rk - 1 + N) % N;
+            int c = ((rk - k - 2) % N + N) % N;
+            size_t off, len; chunk_span(n, N, c, &off, &len);
+            rc = zo_drc(cur[from], cur_b[from], send[rk] + off, NULL, 0, len, nxt[rk], cap, &nxt_b[rk],
+                        last ? recv[rk] : NULL, 0u);
+            if (rc == ZO_W_PRECISION) warn = 1;
+            if (hop_bytes && rc >= 0 && !last) hop_bytes[(size_t)(k + 1) * (size_t)N + (size_t)rk] = nxt_b[rk];
+        }
+        for (int rk = 0; rk < N; ++rk) { uint8_t *tp = cur[rk]; cur[rk] = nxt[rk]; nxt[rk] = tp; size_t tb = cur_b[rk]; cur_b[rk] = nxt_b[rk]; nxt_b[rk] = tb; }
+    }
+    for (int k = 0; k < N; ++k) { free(cur[k]); free(nxt[k]); }
+    free(cur); free(nxt); free(cur_b); free(nxt_b);
+    if (rc < 0) return rc;
+    return warn ? ZO_W_PRECISION : ZO_OK;
+}
+
+/* Scatter in the data movement framework over the binomial tree (Section 4.4): the root (rank 0) holds N chunks of
+ * n elements, compresses chunks 1..N-1 once each, the tree forwards compressed bytes only (in the round with
+ * distance d = the largest power of two below N, then d/2, ..., 1, every holder h hands the chunks h+d .. h+2d-1
+ * to rank h+d), every rank decompresses its own chunk; the root keeps chunk 0 as it is.  recv[r] holds n elements.
+ * sizes (optional, N entries; sizes[0] = 0): compressed bytes of each chunk.
+ * round_bytes (optional, one entry per round, at most 32): bytes that cross the tree's links in that round. */
+int zo_sim_scatter(const float *root, float *const *recv, int N, size_t n, int eb_mode, float eb, uint32_t T,
+                   size_t *sizes, size_t *round_bytes)
+{
+    if (N < 1) return ZO_E_ARG;
+    float eb_abs, s, r;
+    int rc = zo_resolve(eb_mode, eb, root, (size_t)N * n, &eb_abs, &s, &r);
+    if (rc != ZO_OK) return rc;
+    size_t cap = zo_compress_bound(n, T);
+    int warn = 0;
+    uint8_t *st = (uint8_t *)malloc(cap);
+    size_t *sb = (size_t *)calloc((size_t)N, sizeof(size_t));
+    memcpy(recv[0], root, sizeof(float) * n);
+    for (int c = 1; c < N && rc >= 0; ++c) {
+        rc = zo_compress_core(root + (size_t)c * n, n, eb_abs, s, r, T, st, cap, &sb[c]);
+        if (rc == ZO_W_PRECISION) warn = 1;
+        if (rc >= 0) {
+            int rc2 = zo_decompress(st, sb[c], recv[c], n, NULL);
+            if (rc2 != ZO_OK) rc = rc2;
+        }
+    }
+    if (sizes) for (int c = 0; c < N; ++c) sizes[c] = sb[c];
+    if (round_bytes) {
+        int d = 1, round = 0;
+        while (2 * d < N) d *= 2;
+        for (; d >= 1 && N > 1; d /= 2, ++round) {
+            size_t moved = 0;
+            for (int h = 0; h < N; h += 2 * d)              /* holders of this round */
+                for (int c = h + d; c < h + 2 * d && c < N; ++c) moved += sb[c];
+            round_bytes[round] = moved;
+        }
+    }
+    free(st); free(sb);
+    if (rc < 0) return rc;
+    return warn ? ZO_W_PRECISION : ZO_OK;
+}

@@ -15,6 +15,7 @@ struct zccl_ctx {
     int sm_count = 0;
     size_t max_elems = 0;
     int max_ranks = 0;
+    uint32_t debug_epoch = 0;
     Workspace ws{};
     void* small_block = nullptr;     // tile states + counters + params + sizes
     uint8_t* arena = nullptr;        // compressed-chunk slots of the emulated ranks
@@ -271,6 +272,13 @@ int zccl_debug_skip_publish(zccl_ctx* c, long long tile)
     if (!c) return ZCCL_E_ARG;
     c->ws.skip_publish = (tile < 0 || tile >= 0xFFFFFFFFll) ? 0xFFFFFFFFu : (uint32_t)tile;
     return ZCCL_OK;
+}
+
+int zccl_debug_set_launch_counter(zccl_ctx* c, unsigned int value, void* stream)
+{
+    if (!c || value == 0 || value > 0x7FFFFFFFu) return ZCCL_E_ARG;
+    c->debug_epoch = value;   // the source of an asynchronous copy must outlive the call
+    return cuda_rc(cudaMemcpyAsync(c->ws.epoch, &c->debug_epoch, sizeof(uint32_t), cudaMemcpyHostToDevice, (cudaStream_t)stream));
 }
 
 int zccl_compress(zccl_ctx* c, const float* x, size_t n, int eb_mode, float eb,

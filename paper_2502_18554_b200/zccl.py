@@ -24,6 +24,7 @@ EXPORTS = [
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_sizes",
     "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
+    "zccl_debug_set_launch_counter",
 ]
 
 _lib = None
@@ -66,6 +67,7 @@ def lib():
         L.zccl_decompress_host.argtypes = [vp, vp, sz, vp, sz, vp]
         L.zccl_compress_noalloc.argtypes = [vp, sz, C.c_float, vp, sz, vp, vp]
         L.zccl_debug_skip_publish.argtypes = [vp, C.c_longlong]
+        L.zccl_debug_set_launch_counter.argtypes = [vp, C.c_uint, vp]
         _lib = L
     return _lib
 
@@ -147,6 +149,10 @@ class Context:
     def debug_skip_publish(self, tile: int):
         """Test hook: tile number whose size is never published to the placement scan (negative = off)."""
         _check(lib().zccl_debug_skip_publish(self._h, tile), "zccl_debug_skip_publish")
+
+    def debug_set_launch_counter(self, value: int, stream=None):
+        """Test hook: sets the launch counter that validates the placement scan's states."""
+        _check(lib().zccl_debug_set_launch_counter(self._h, value, _stream_ptr(stream)), "zccl_debug_set_launch_counter")
 
     # ---- codec
     def compress(self, x: torch.Tensor, eb_mode: int, eb: float, out: torch.Tensor, out_bytes: torch.Tensor,

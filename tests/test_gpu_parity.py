@@ -413,3 +413,28 @@ def test_look_back_wait_is_bounded(z):
     assert ctx.status() == z.OK
     assert np.array_equal(out[: int(nbytes.item())].cpu().numpy(), want)
     ctx.close()
+
+
+def test_launch_counter_wraps_cleanly(z):
+    # the scan states are validated by a launch counter: run compress, fused hop and decompress on both sides of its
+    # wrap-around (states of earlier launches must not look current afterwards)
+    ctx = z.Context(1 << 20, 0)
+    x = fields.smooth_1d(37 * 4096 + 123, seed=35)
+    loc = fields.smooth_1d(x.size, seed=36)
+    dx, dl = dev(x), dev(loc)
+    want, wrc = oracle.compress(x, oracle.EB_REL, 1e-3)
+    want2, wrc2 = oracle.drc(want, local=loc)
+    cap = z.compress_bound(x.size)
+    ctx.debug_set_launch_counter(0x7FFFFFFF - 2)
+    for _ in range(3):   # counters 2^31 - 3, 2^31 - 2, 2^31 - 1 for the encoder launches, then 1, 2, ...
+        out = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+        nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+        ctx.compress(dx, z.EB_REL, 1e-3, out, nb)
+        assert ctx.status() == wrc
+        assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+        out2 = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+        nb2 = torch.zeros(1, dtype=torch.int64, device="cuda")
+        ctx.decompress_reduce_compress(out[: int(nb.item())], x.size, out2, nb2, local=dl)
+        assert ctx.status() == wrc2
+        assert np.array_equal(out2[: int(nb2.item())].cpu().numpy(), want2)
+    ctx.close()

@@ -160,3 +160,129 @@ def test_bcast_compresses_once():
     for y in recv:
         assert np.array_equal(y, oracle.decompress(st))
         assert np.abs(y.astype(np.float64) - x.astype(np.float64)).max() <= float(ea)
+
+
+# ---------------------------------------------------------------- Reduce-scatter and Scatter as collectives of their own
+
+def mailbox_ring_reduce_scatter(send, compress, decompress, add):
+    """Independent statement of the ring Reduce-scatter that leaves chunk r on rank r: every rank owns one mailbox,
+    in every step each rank hands its partial sum to its right neighbour, who adds its own piece of that chunk."""
+    N, n = len(send), send[0].size
+    m = -(-n // N)
+    span = lambda c: slice(min(c * m, n), min((c + 1) * m, n))
+    chunk_at = [(r - 1) % N for r in range(N)]                     # the chunk whose partial sum rank r holds
+    box = [compress(send[r][span(chunk_at[r])]) for r in range(N)]
+    out = [None] * N
+    for step in range(N - 1):
+        got = [(chunk_at[(r - 1) % N], box[(r - 1) % N]) for r in range(N)]
+        for r in range(N):
+            c, stream = got[r]
+            y = add(decompress(stream), send[r][span(c)])
+            chunk_at[r] = c
+            if step == N - 2:
+                assert c == r
+                out[r] = y
+            else:
+                box[r] = compress(y)
+    return out
+
+
+@pytest.mark.parametrize("N,n", [(2, 1000), (3, 10_001), (4, 4096 * 4), (8, 8 * 5000 + 3), (5, 4096 * 5 + 1), (8, 11)])
+def test_reduce_scatter_matches_independent_schedule(N, n):
+    send = [fields.smooth_1d(n, seed=60 + r) for r in range(N)]
+    ea, s, r_ = oracle.resolve(oracle.EB_ABS, 1e-3)
+    got, rc, hop = oracle.sim_reduce_scatter(send, oracle.EB_ABS, 1e-3)
+    want = mailbox_ring_reduce_scatter(
+        send,
+        compress=lambda x: oracle.compress_core(x, ea, s, r_)[0],
+        decompress=oracle.decompress,
+        add=lambda a, b: (a + b).astype(f32))
+    for r in range(N):
+        assert got[r].size == oracle.chunk_span(n, N, r)[1]
+        assert np.array_equal(got[r].view(np.uint32), want[r].view(np.uint32))
+
+
+def test_reduce_scatter_lossless_on_grid_is_the_textbook_sum():
+    # inputs on a power-of-two grid whose partial sums stay on it: every compression is lossless, so the result is
+    # the exact sum (computed in fp64), chunk by chunk
+    N, n = 8, 8 * 4096 + 77
+    eb, s = find_power_of_two_step_bound(-6)
+    send = fields.on_grid_ranks(N, n, float(s), seed=5)
+    got, rc, hop = oracle.sim_reduce_scatter(send, oracle.EB_ABS, eb)
+    exact = np.sum(np.stack(send).astype(np.float64), axis=0)
+    for r in range(N):
+        off, ln = oracle.chunk_span(n, N, r)
+        assert np.array_equal(got[r].astype(np.float64), exact[off:off + ln])
+
+
+def test_reduce_scatter_error_chain_and_traffic():
+    # Eq. 2: chunk r went through N-1 compressions of partial sums, each within the bound
+    N, n = 8, 8 * 6000
+    send = [fields.smooth_1d(n, seed=80 + r) for r in range(N)]
+    got, rc, hop = oracle.sim_reduce_scatter(send, oracle.EB_REL, 1e-3)
+    ea, _, _ = oracle.resolve(oracle.EB_REL, 1e-3, np.concatenate(send))
+    exact = np.sum(np.stack(send).astype(np.float64), axis=0)
+    mag = np.sum(np.abs(np.stack(send).astype(np.float64)), axis=0)
+    for r in range(N):
+        off, ln = oracle.chunk_span(n, N, r)
+        err = np.abs(got[r].astype(np.float64) - exact[off:off + ln])
+        assert np.all(err <= (N - 1) * float(ea) + N * 2.0 ** -24 * mag[off:off + ln])
+    # every step moves one compressed chunk per rank, each well below the uncompressed chunk
+    assert hop.shape == (N - 1, N) and np.all(hop > 0) and np.all(hop < 4 * (n // N) / 2)
+
+
+def test_reduce_scatter_two_ranks_by_hand():
+    # N = 2: rank r receives the other rank's compressed chunk r and adds its own, nothing else happens
+    n = 2 * 700
+    a, b = fields.smooth_1d(n, seed=91), fields.smooth_1d(n, seed=92)
+    ea, s, r_ = oracle.resolve(oracle.EB_ABS, 2e-3)
+    got, rc, hop = oracle.sim_reduce_scatter([a, b], oracle.EB_ABS, 2e-3)
+    lo, hi = slice(0, 700), slice(700, 1400)
+    want0 = (oracle.decompress(oracle.compress_core(b[lo], ea, s, r_)[0]) + a[lo]).astype(f32)
+    want1 = (oracle.decompress(oracle.compress_core(a[hi], ea, s, r_)[0]) + b[hi]).astype(f32)
+    assert np.array_equal(got[0].view(np.uint32), want0.view(np.uint32))
+    assert np.array_equal(got[1].view(np.uint32), want1.view(np.uint32))
+
+
+def binomial_scatter_rounds(N):
+    """Textbook binomial scatter from rank 0: per round the list of (sender, receiver, chunks handed over)."""
+    rounds = []
+    d = 1
+    while 2 * d < N:
+        d *= 2
+    holders = {0: list(range(N))}
+    while d >= 1 and N > 1:
+        moves = []
+        for h in sorted(holders):
+            give = [c for c in holders[h] if c >= h + d]
+            if give:
+                moves.append((h, h + d, give))
+        for h, to, give in moves:
+            holders[h] = [c for c in holders[h] if c < h + d]
+            holders[to] = give
+        rounds.append(moves)
+        d //= 2
+    for r in range(N):
+        assert holders[r] == [r]
+    return rounds
+
+
+@pytest.mark.parametrize("N,n", [(1, 300), (2, 1000), (3, 5000), (5, 4096 + 7), (8, 3 * 4096), (13, 777)])
+def test_scatter_compress_once_and_tree_traffic(N, n):
+    root = fields.smooth_1d(N * n, seed=70 + N)
+    got, rc, sizes, rounds = oracle.sim_scatter(root, N, oracle.EB_REL, 1e-3)
+    ea, s, r_ = oracle.resolve(oracle.EB_REL, 1e-3, root)
+    assert np.array_equal(got[0].view(np.uint32), root[:n].view(np.uint32))      # the root keeps its chunk as it is
+    assert sizes[0] == 0
+    for c in range(1, N):
+        stream, _ = oracle.compress_core(root[c * n:(c + 1) * n], ea, s, r_)       # compressed once, with the bound of the whole buffer
+        assert sizes[c] == stream.size
+        assert np.array_equal(got[c].view(np.uint32), oracle.decompress(stream).view(np.uint32))
+        assert np.max(np.abs(got[c].astype(np.float64) - root[c * n:(c + 1) * n].astype(np.float64))) <= float(ea)
+    tree = binomial_scatter_rounds(N)
+    assert len(rounds) == len(tree)
+    for moved, moves in zip(rounds, tree):
+        assert moved == sum(int(sizes[c]) for _, _, give in moves for c in give)
+    # every chunk but the root's crosses at least one link; the first round carries about half of them
+    if N > 1:
+        assert sum(int(v) for v in rounds) >= int(np.sum(sizes))
