@@ -205,10 +205,35 @@ int zccl_sim_bcast(zccl_ctx* ctx, const float* root, float* const* recv, int nsi
                    int eb_mode, float eb, void* stream);
 
 /*
+ * Ring Reduce-scatter (sum) as a collective of its own (Section 3.1.2; the first stage of the Allreduce of
+ * Section 3.5 with the ring shifted so that rank r ends with chunk r): chunk c is compressed by rank c+1, travels
+ * c+1 -> c+2 -> ... -> c, every receiver runs the fused hop with its own piece of chunk c, and the last one keeps
+ * the uncompressed sum.  Chunks as for zccl_sim_allreduce.
+ *   send [host]  nranks device pointers, each n_per_rank floats (read only)
+ *   recv [host]  nranks device pointers; recv[r] receives the elements of chunk r (at most ceil(n_per_rank / nranks))
+ * Needs a context created with max_ranks >= nranks and max_elems >= n_per_rank.
+ */
+int zccl_sim_reduce_scatter(zccl_ctx* ctx, const float* const* send, float* const* recv, int nranks,
+                            size_t n_per_rank, int eb_mode, float eb, void* stream);
+
+/*
+ * Scatter over a binomial tree in the data movement framework (Section 4.4): rank 0 holds nranks chunks of
+ * n_per_rank elements, compresses chunks 1..nranks-1 once each (one bound for the whole buffer; with ZCCL_EB_REL
+ * eb times its range), the tree forwards compressed bytes only (in the round with distance d = the largest power
+ * of two below nranks, then d/2, ..., 1, holder h hands the chunks h+d .. h+2d-1 to rank h+d), and every rank
+ * decompresses its own chunk; chunk 0 is copied as it is.
+ *   root [device] nranks * n_per_rank floats;  recv [host] nranks device pointers, each n_per_rank floats
+ * Needs a context with max_ranks >= nranks and max_elems >= nranks * n_per_rank.
+ */
+int zccl_sim_scatter(zccl_ctx* ctx, const float* root, float* const* recv, int nranks, size_t n_per_rank,
+                     int eb_mode, float eb, void* stream);
+
+/*
  * Compressed sizes of the last zccl_sim_* call, for reporting ratios (the paper's compressed_sizes array,
  * Section 3.5.1).  Synchronises `stream`.  sizes [host] receives up to `capacity` entries and the call returns how
  * many there are: allreduce nranks*nranks (entry k*nranks + r = bytes rank r produced at step k, k = 0 the
- * initial compression), allgather nranks, bcast 1.  Negative on error.
+ * initial compression), allgather nranks, bcast 1, reduce_scatter (nranks-1)*nranks (as for allreduce), scatter
+ * nranks (entry c = bytes of chunk c, 0 for the root's own).  Negative on error.
  */
 int zccl_sim_sizes(zccl_ctx* ctx, size_t* sizes, int capacity, void* stream);
 

@@ -517,6 +517,124 @@ int zccl_sim_bcast(zccl_ctx* c, const float* root, float* const* recv, int nsink
     return flush_decode(c, b, st);
 }
 
+int zccl_sim_reduce_scatter(zccl_ctx* c, const float* const* send, float* const* recv, int N,
+                            size_t n, int eb_mode, float eb, void* stream)
+{
+    if (!c || !send || !recv || N < 1 || N > c->max_ranks || !eb_ok(eb_mode, eb) || n > c->max_elems) return ZCCL_E_ARG;
+    for (int r = 0; r < N; ++r) if (!send[r] || !recv[r]) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t m = (n + (size_t)N - 1) / (size_t)N;
+    const size_t slot = align_up(bound_of(m), 256);
+    if (2 * (size_t)N * slot > c->arena_bytes) return ZCCL_E_ARG;
+    uint8_t* cur = c->arena;
+    uint8_t* nxt = c->arena + (size_t)N * slot;
+    size_t* hop_sz = c->sim_sizes;                       // [N-1][N]: step k, rank r; one more row for the last hop's unused stream
+    c->sim_sizes_count = (N - 1) * N;
+    if (cudaMemsetAsync(c->sim_sizes, 0, sizeof(size_t) * (size_t)N * N, st) != cudaSuccess) return ZCCL_E_CUDA;
+    if (N == 1) {
+        size_t off, len; chunk_span(n, N, 0, off, len);
+        return cuda_rc(cudaMemcpyAsync(recv[0], send[0], sizeof(float) * len, cudaMemcpyDeviceToDevice, st));
+    }
+
+    Params hp{};
+    bool dev = false;
+    RangeList rl;
+    for (int r = 0; r < N; ++r) { rl.x.push_back(send[r]); rl.n.push_back(n); }
+    int rc = resolve_bound(c, rl, eb_mode, eb, hp, dev, st);
+    if (rc != ZCCL_OK) return rc;
+
+    Batcher b;
+    for (int r = 0; r < N; ++r) {   // step 0: rank r compresses chunk r-1
+        size_t off, len; chunk_span(n, N, (r - 1 + N) % N, off, len);
+        Job j{};
+        j.x = send[r] + off; j.n = len; j.out = (uint32_t*)(cur + (size_t)r * slot); j.out_cap = slot;
+        j.out_bytes = hop_sz + r;
+        b.add(j, tiles_of(len));
+        if (b.full() && (rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+    }
+    if ((rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+    for (int k = 0; k + 1 < N; ++k) {   // step k+1: rank r takes chunk r-k-2 from rank r-1; the last step keeps the sum
+        const bool last = (k == N - 2);
+        for (int r = 0; r < N; ++r) {
+            const int from = (r - 1 + N) % N;
+            const int ch = ((r - k - 2) % N + N) % N;
+            size_t off, len; chunk_span(n, N, ch, off, len);
+            Job j{};
+            j.in_c = (const uint32_t*)(cur + (size_t)from * slot); j.in_cap = slot;
+            j.x = send[r] + off; j.n = len;
+            j.out = (uint32_t*)(nxt + (size_t)r * slot); j.out_cap = slot;
+            j.out_bytes = hop_sz + (size_t)(k + 1) * N + r;   // the last step's stream is produced but not part of the collective
+            j.y = last ? recv[r] : nullptr;
+            j.flags = 0;
+            b.add(j, tiles_of(len));
+            if (b.full() && (rc = flush_encode(c, b, kEncodeFused, false, hp, st)) != ZCCL_OK) return rc;
+        }
+        if ((rc = flush_encode(c, b, kEncodeFused, false, hp, st)) != ZCCL_OK) return rc;
+        uint8_t* t = cur; cur = nxt; nxt = t;
+    }
+    return ZCCL_OK;
+}
+
+int zccl_sim_scatter(zccl_ctx* c, const float* root, float* const* recv, int N, size_t n,
+                     int eb_mode, float eb, void* stream)
+{
+    if (!c || (!root && n) || !recv || N < 1 || N > c->max_ranks || !eb_ok(eb_mode, eb) || n * (size_t)N > c->max_elems)
+        return ZCCL_E_ARG;
+    for (int r = 0; r < N; ++r) if (!recv[r]) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t slot = align_up(bound_of(n), 256);
+    if ((size_t)N * N * slot > c->arena_bytes) return ZCCL_E_ARG;
+    auto gslot = [&](int r, int ch) { return c->arena + ((size_t)r * N + ch) * slot; };
+    size_t* own_sz = c->sim_sizes;                     // [N]: bytes of chunk c as compressed by the root
+    size_t* g_sz = c->sim_sizes + N;                   // [N][N]: rank r, chunk c
+    c->sim_sizes_count = N;
+    if (cudaMemsetAsync(c->sim_sizes, 0, sizeof(size_t) * ((size_t)N * N + N), st) != cudaSuccess) return ZCCL_E_CUDA;
+
+    Params hp{};
+    bool dev = false;
+    RangeList rl;
+    rl.x.push_back(root); rl.n.push_back(n * (size_t)N);
+    int rc = resolve_bound(c, rl, eb_mode, eb, hp, dev, st);
+    if (rc != ZCCL_OK) return rc;
+
+    Batcher b;
+    for (int ch = 1; ch < N; ++ch) {   // the root compresses every foreign chunk once
+        Job j{};
+        j.x = root + (size_t)ch * n; j.n = n; j.out = (uint32_t*)gslot(0, ch); j.out_cap = slot; j.out_bytes = own_sz + ch;
+        b.add(j, tiles_of(n));
+        if (b.full() && (rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+    }
+    if ((rc = flush_encode(c, b, kEncodeRaw, dev, hp, st)) != ZCCL_OK) return rc;
+
+    if (N > 1) {   // tree forwarding: chunk ch moves to holder h + d in every round whose distance d it is beyond
+        int top = 1;
+        while (2 * top < N) top *= 2;
+        ChainBatch cb{};
+        cb.slots = c->arena; cb.sizes = g_sz; cb.slot_bytes = slot; cb.N = N; cb.hops = -1; cb.count = 0;
+        for (int ch = 1; ch < N; ++ch) {
+            ChainJob& j = cb.job[cb.count++];
+            j.src0 = (const uint32_t*)gslot(0, ch); j.bytes = own_sz + ch; j.first_rank = 0; j.chunk = ch;
+            j.path = 0; j.hops = 0;
+            int h = 0;
+            for (int d = top; d >= 1; d /= 2)
+                if (ch >= h + d) { h += d; j.path |= (unsigned long long)h << (8 * j.hops); ++j.hops; }
+        }
+        if ((rc = cuda_rc(launch_copy_chain(cb, c->ws, c->sm_count, st))) != ZCCL_OK) return rc;
+    }
+    {   // the root keeps its own chunk as it is
+        CopyBatcher cb;
+        cb.add_fixed(root, recv[0], sizeof(float) * n);
+        if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
+    }
+    for (int r = 1; r < N; ++r) {
+        Job j{};
+        j.in_c = (const uint32_t*)gslot(r, r); j.in_cap = slot; j.y = recv[r]; j.n = n;
+        b.add(j, tiles_of(n));
+        if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+    }
+    return flush_decode(c, b, st);
+}
+
 int zccl_sim_sizes(zccl_ctx* c, size_t* sizes, int capacity, void* stream)
 {
     if (!c || !sizes || capacity < 0) return ZCCL_E_ARG;

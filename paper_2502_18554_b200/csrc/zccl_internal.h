@@ -92,15 +92,17 @@ constexpr int kMaxChains = 64;
 struct ChainJob {
     const uint32_t* src0;   // where the chunk is before the first hop
     const size_t* bytes;    // its device-resident length
-    int first_rank;         // receiver of the first hop
+    int first_rank;         // ring: receiver of the first hop (hop h goes to rank first_rank + h mod N)
     int chunk;
+    unsigned long long path;   // tree: receiver of hop h in bits 8h .. 8h+7 (at most 8 hops)
+    int hops;                  // tree: hops of this chain
 };
 struct ChainBatch {
     ChainJob job[kMaxChains];
     unsigned char* slots;
     size_t* sizes;
     unsigned long long slot_bytes;
-    int N, hops, count;
+    int N, hops, count;   // hops < 0: every chain follows its own path
 };
 
 struct RangeBatch {

@@ -1452,32 +1452,31 @@ __global__ void __launch_bounds__(256) copy_chain_kernel(ChainBatch cb, Workspac
     const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     const unsigned long long nth = (unsigned long long)gridDim.x * blockDim.x;
     const bool fits = bytes <= cb.slot_bytes;
+    const bool ring = cb.hops >= 0;
+    const int hops = ring ? cb.hops : job.hops;
+    auto rank_of = [&](int h) { return ring ? (job.first_rank + h) % cb.N : (int)((job.path >> (8 * h)) & 0xFFu); };
     if (tid == 0) {
         if (!fits) atomicOr(ws.status, kStCapacity);
-        for (int h = 0; h < cb.hops; ++h) {
-            const int r = (job.first_rank + h) % cb.N;
-            cb.sizes[(size_t)r * cb.N + job.chunk] = fits ? (size_t)bytes : 0;
-        }
+        for (int h = 0; h < hops; ++h)
+            cb.sizes[(size_t)rank_of(h) * cb.N + job.chunk] = fits ? (size_t)bytes : 0;
     }
     if (!fits) return;
     const unsigned long long words = bytes >> 2;
     const unsigned long long nv = ((((uintptr_t)job.src0) & 15u) == 0) ? (words >> 2) : 0;   // slots are 256-byte aligned
     for (unsigned long long i = tid; i < nv; i += nth) {
         uint4 v = __ldg(reinterpret_cast<const uint4*>(job.src0) + i);
-        for (int h = 0; h < cb.hops; ++h) {
-            const int r = (job.first_rank + h) % cb.N;
-            uint4* d = reinterpret_cast<uint4*>(cb.slots + ((size_t)r * cb.N + job.chunk) * cb.slot_bytes) + i;
+        for (int h = 0; h < hops; ++h) {
+            uint4* d = reinterpret_cast<uint4*>(cb.slots + ((size_t)rank_of(h) * cb.N + job.chunk) * cb.slot_bytes) + i;
             *d = v;
-            if (h + 1 < cb.hops) asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(d) : "memory");
+            if (h + 1 < hops) asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(d) : "memory");
         }
     }
     for (unsigned long long i = (nv << 2) + tid; i < words; i += nth) {
         uint32_t v = __ldg(job.src0 + i);
-        for (int h = 0; h < cb.hops; ++h) {
-            const int r = (job.first_rank + h) % cb.N;
-            uint32_t* d = reinterpret_cast<uint32_t*>(cb.slots + ((size_t)r * cb.N + job.chunk) * cb.slot_bytes) + i;
+        for (int h = 0; h < hops; ++h) {
+            uint32_t* d = reinterpret_cast<uint32_t*>(cb.slots + ((size_t)rank_of(h) * cb.N + job.chunk) * cb.slot_bytes) + i;
             *d = v;
-            if (h + 1 < cb.hops) asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(d) : "memory");
+            if (h + 1 < hops) asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(d) : "memory");
         }
     }
 }
@@ -1564,7 +1563,7 @@ cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, 
 
 cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
-    if (cb.count <= 0 || cb.hops <= 0) return cudaSuccess;
+    if (cb.count <= 0 || cb.hops == 0) return cudaSuccess;
     unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
     ++g_launches;
     copy_chain_kernel<<<dim3(gx ? gx : 1, cb.count), 256, 0, st>>>(cb, ws);

@@ -22,7 +22,8 @@ TILE, BLOCK, HEADER_BYTES = 4096, 32, 32
 EXPORTS = [
     "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
-    "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_sizes",
+    "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_reduce_scatter", "zccl_sim_scatter",
+    "zccl_sim_sizes",
     "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
     "zccl_debug_set_launch_counter",
 ]
@@ -61,6 +62,8 @@ def lib():
         L.zccl_decompress_reduce_compress.argtypes = [vp, vp, sz, vp, vp, sz, sz, vp, sz, vp, vp, C.c_uint, vp]
         L.zccl_sim_allreduce.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, C.c_uint, vp]
         L.zccl_sim_allgather.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
+        L.zccl_sim_reduce_scatter.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
+        L.zccl_sim_scatter.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
         L.zccl_sim_bcast.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
         L.zccl_sim_sizes.argtypes = [vp, vp, C.c_int, vp]
         L.zccl_compress_host.argtypes = [vp, vp, sz, C.c_int, C.c_float, vp, sz, vp, vp]
@@ -199,6 +202,18 @@ class Context:
     def sim_bcast(self, root: torch.Tensor, recv, eb_mode: int, eb: float, stream=None):
         _check(lib().zccl_sim_bcast(self._h, _dev_ptr(root, torch.float32), self._ptrs(recv), len(recv), root.numel(),
                                     eb_mode, eb, _stream_ptr(stream)), "zccl_sim_bcast")
+
+    def sim_reduce_scatter(self, send, recv, eb_mode: int, eb: float, stream=None):
+        """zccl_sim_reduce_scatter: recv[r] receives chunk r of the sum of the send buffers."""
+        n = send[0].numel()
+        _check(lib().zccl_sim_reduce_scatter(self._h, self._ptrs(send), self._ptrs(recv), len(send), n, eb_mode, eb,
+                                             _stream_ptr(stream)), "zccl_sim_reduce_scatter")
+
+    def sim_scatter(self, root: torch.Tensor, recv, eb_mode: int, eb: float, stream=None):
+        """zccl_sim_scatter: root holds len(recv) chunks; recv[r] receives chunk r."""
+        N = len(recv)
+        _check(lib().zccl_sim_scatter(self._h, _dev_ptr(root, torch.float32), self._ptrs(recv), N, root.numel() // N,
+                                      eb_mode, eb, _stream_ptr(stream)), "zccl_sim_scatter")
 
     def sim_sizes(self, stream=None) -> list[int]:
         cap = 2 * max(self.max_ranks, 1) ** 2 + 2

@@ -438,3 +438,51 @@ def test_launch_counter_wraps_cleanly(z):
         assert ctx.status() == wrc2
         assert np.array_equal(out2[: int(nb2.item())].cpu().numpy(), want2)
     ctx.close()
+
+
+@pytest.mark.parametrize("N,n", [(2, 1000), (3, 10_001), (8, 8 * 4096 * 3), (8, 8 * 5000 + 3), (8, 11), (5, 4096 * 5 + 1),
+                                 (1, 5000)])
+def test_reduce_scatter_matches_oracle(z, ctx, N, n):
+    send = [fields.smooth_1d(n, seed=60 + r) for r in range(N)]
+    want, wrc, whop = oracle.sim_reduce_scatter(send, oracle.EB_REL, 1e-3)
+    d_send = [dev(a) for a in send]
+    guard = 8   # elements after each receive buffer that must stay untouched
+    d_recv = [torch.full((want[r].size + guard,), 7.0, dtype=torch.float32, device="cuda") for r in range(N)]
+    ctx.sim_reduce_scatter(d_send, d_recv, z.EB_REL, 1e-3)
+    assert ctx.status() == wrc
+    for r in range(N):
+        got = d_recv[r].cpu().numpy()
+        assert_same_bits(got[: want[r].size], want[r])
+        assert np.all(got[want[r].size:] == 7.0)
+    if N > 1:
+        assert np.array_equal(np.array(ctx.sim_sizes()).reshape(N - 1, N), whop)
+
+
+def test_reduce_scatter_lossless_on_grid(z, ctx):
+    from _util import find_power_of_two_step_bound
+    eb, s = find_power_of_two_step_bound(-6)
+    N, n = 8, 8 * 4096 + 77
+    send = fields.on_grid_ranks(N, n, float(s), seed=5)
+    exact = np.sum(np.stack(send).astype(np.float64), axis=0)
+    d_recv = [torch.zeros(oracle.chunk_span(n, N, r)[1], dtype=torch.float32, device="cuda") for r in range(N)]
+    ctx.sim_reduce_scatter([dev(a) for a in send], d_recv, z.EB_ABS, eb)
+    assert ctx.status() == z.OK
+    for r in range(N):
+        off, ln = oracle.chunk_span(n, N, r)
+        assert np.array_equal(d_recv[r].cpu().numpy().astype(np.float64), exact[off:off + ln])
+
+
+@pytest.mark.parametrize("N,n", [(1, 300), (2, 1000), (3, 5000), (5, 4096 + 7), (8, 3 * 4096), (13, 777), (16, 4096)])
+def test_scatter_matches_oracle(z, N, n):
+    c = z.Context(max(N * n, 4096), max(N, 2))
+    root = fields.smooth_1d(N * n, seed=70 + N)
+    want, wrc, wsizes, _ = oracle.sim_scatter(root, N, oracle.EB_REL, 1e-3)
+    d_recv = [torch.full((n + 8,), 7.0, dtype=torch.float32, device="cuda") for _ in range(N)]
+    c.sim_scatter(dev(root), d_recv, z.EB_REL, 1e-3)
+    assert c.status() == wrc
+    for r in range(N):
+        got = d_recv[r].cpu().numpy()
+        assert_same_bits(got[:n], want[r])
+        assert np.all(got[n:] == 7.0)
+    assert np.array_equal(np.array(c.sim_sizes()), wsizes)
+    c.close()
