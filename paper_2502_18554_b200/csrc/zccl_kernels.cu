@@ -3,9 +3,10 @@
 //
 // Work decomposition.  One CTA of 256 threads handles one 4096-element tile at a time; each of its 8 warps owns
 // 16 consecutive 32-element blocks, one element per lane, so that a block's code length is one warp OR-reduction
-// and its bit planes come out of a 32 x 32 bit-matrix transpose across the warp.  The kernels are bound by
-// instruction issue (integer ALU pipe: 2 warp-instructions/clk/SM; shared memory and shuffles: 1), not by HBM, so
-// the design minimises instructions per block:
+// and its bit planes come out of a 32 x 32 bit-matrix transpose across the warp (one transpose serves four blocks
+// while their code lengths fit 7 bits).  The kernels are bound by instruction issue (integer ALU pipe:
+// 2 warp-instructions/clk/SM; shared memory and shuffles: 1) and by the latency of each tile's chain of phases, not
+// by HBM, so the design minimises instructions per block and keeps barriers and one-thread work off that chain:
 //   * tiles (encoder) and compressed blobs (decoder, fused hop) are staged in shared memory by 1-D bulk copies
 //     (cp.async.bulk + mbarrier), requested one tile ahead, so no thread spends instructions or registers on
 //     global loads and no warp waits on a chain of them;
@@ -19,8 +20,10 @@
 // Tiles are dealt round-robin to a grid that fits the device (CTA c takes tiles c, c + G, ...), so all CTAs move
 // through the stream in step and the next tile is known in advance.  Placement (prefix sum of tile sizes) is
 // anchored at a CTA's own previous tile and deferred by one tile, so it only ever sums sizes that are already
-// published.  The scan relies on the grid being resident at once; every wait is bounded and reports through the
-// status word instead of hanging if it is not.
+// published; warp 0 plans a placement once for the CTA (scan, layout, capacity check, index entry), warp 1 requests
+// the next tile meanwhile, and after one barrier every warp copies its own share.  The scan relies on the grid
+// being resident at once; every wait is bounded and reports through the status word instead of hanging if it is
+// not.
 #include "zccl_internal.h"
 
 namespace zccl {
