@@ -830,6 +830,9 @@ struct PlanShared {
     uint32_t* blob_out;       // where the pending tile's blob starts in the stream (nullptr: do not copy)
     uint32_t wbase[kWarps];   // each warp's first word inside the blob
     uint32_t padw;            // code-length words of the blob
+    uint32_t part[kWarps];    // scan: sum of the sizes warp w fetched (warps 1..7)
+    uint32_t ok[kWarps];      // scan: 1 if every state that warp saw was published
+    alignas(8) unsigned long long scanbar;   // warps 1..7 arrive once their shares are written
 };
 
 struct EncodeShared {
@@ -948,19 +951,70 @@ __device__ __forceinline__ uint32_t sum_sizes_warp(const Workspace& ws, uint32_t
     }
 }
 
-// Warp 0, after the barrier that follows a tile's encoding pass: publishes the size of the tile just encoded
-// (`ticket`, sizes in `cur_words`) and plans the pending one (sizes in `pend_words`).
-__device__ __forceinline__ void announce_and_plan(PlanShared& plan, const uint32_t* cur_words, uint32_t cur_padw, uint32_t ticket,
-                                                  bool have_cur, const Pending& c, const uint32_t* pend_words, Anchor& anchor,
-                                                  const JobBatch& jb, float eb_abs, float s, const Workspace& ws,
-                                                  uint32_t epoch, int lane, uint32_t& status)
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar)
 {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// First tile of the scan that places a tile of job `job_index`, given the tile this CTA placed last.
+__device__ __forceinline__ uint32_t scan_begin(const Anchor& a, int job_index, const JobBatch& jb)
+{
+    return a.job == job_index ? a.ticket + 1 : jb.job[job_index].tile_begin;
+}
+
+// Warps 1..7, while warp 0 publishes and lays out: each fetches its share of the sizes of tiles [lo, hi) (window k
+// of 32 tiles belongs to warp 1 + k mod 7, all loads of a warp in flight together), leaves the sum for warp 0 and
+// arrives on the hand-off barrier.  One round trip to L2 for the whole scan.
+__device__ __forceinline__ void scan_share(PlanShared& plan, const Workspace& ws, uint32_t lo, uint32_t hi, uint32_t epoch,
+                                           int warp, int lane)
+{
+    uint32_t sum = 0;
+    bool good = true;
+    if (hi > lo) {
+        const uint32_t nwin = (hi - lo + 31u) >> 5;
+#pragma unroll 4
+        for (uint32_t w = (uint32_t)warp - 1u; w < nwin; w += kWarps - 1) {
+            const uint32_t at = lo + 32u * w + (uint32_t)lane;
+            if (at < hi) {
+                const unsigned long long st = ld_state(ws.tile_state + at);
+                if ((uint32_t)(st >> 33) == epoch) sum += (uint32_t)st;
+                else good = false;
+            }
+        }
+    }
+    sum = __reduce_add_sync(kFull, sum);
+    good = __all_sync(kFull, good);
+    if (lane == 0) {
+        plan.part[warp] = sum;
+        plan.ok[warp] = good ? 1u : 0u;
+        mbar_arrive(&plan.scanbar);
+    }
+}
+
+// What warp 0 keeps of a plan for the stores it does once the other warps have been released.
+struct Planned {
+    uint32_t* blob_out;
+    uint32_t incl;
+    bool go;
+};
+
+// Warp 0, after the barrier that follows a tile's encoding pass: publishes the size of the tile just encoded
+// (`ticket`, sizes in `cur_words`) and plans the pending one (sizes in `pend_words`): layout of the warps' regions,
+// then the scan's sum from the other warps' shares (`shared_scan`; a blocking scan of its own when a size was not
+// published yet, or when there are no shares), capacity check.
+__device__ __forceinline__ Planned announce_and_plan(PlanShared& plan, const uint32_t* cur_words, uint32_t cur_padw, uint32_t ticket,
+                                                     bool have_cur, const Pending& c, const uint32_t* pend_words, Anchor& anchor,
+                                                     bool shared_scan, uint32_t scan_parity, const JobBatch& jb,
+                                                     const Workspace& ws, uint32_t epoch, int lane, uint32_t& status)
+{
+    Planned d;
+    d.blob_out = nullptr; d.incl = 0; d.go = false;
     if (have_cur) {
         const uint32_t ww = lane < kWarps ? cur_words[lane] : 0u;
         const uint32_t total = 1 + cur_padw + __reduce_add_sync(kFull, ww);
         if (lane == 0 && ticket != ws.skip_publish) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
     }
-    if (!c.valid) return;
+    if (!c.valid) return d;
     const Job& job = jb.job[c.job];
     const uint32_t tile = c.ticket - job.tile_begin;
     const unsigned long long start = (unsigned long long)tile * kTile;
@@ -971,29 +1025,51 @@ __device__ __forceinline__ void announce_and_plan(PlanShared& plan, const uint32
     const uint32_t ww = lane < kWarps ? pend_words[lane] : 0u;
     uint32_t inc = ww;
 #pragma unroll
-    for (int d = 1; d < kWarps; d <<= 1) {
-        const uint32_t up = __shfl_up_sync(kFull, inc, d);
-        if (lane >= d) inc += up;
+    for (int k = 1; k < kWarps; k <<= 1) {
+        const uint32_t up = __shfl_up_sync(kFull, inc, k);
+        if (lane >= k) inc += up;
     }
     const uint32_t total = 1 + padw + __shfl_sync(kFull, inc, kWarps - 1);
-    uint32_t lo = job.tile_begin, base = 0, skip = 0;
-    if (anchor.job == c.job) { lo = anchor.ticket + 1; base = anchor.incl; }
-    const uint32_t excl = base + sum_sizes_warp(ws, lo, c.ticket, epoch, lane, skip, status);
-    anchor.job = c.job; anchor.ticket = c.ticket; anchor.incl = excl + total;
+    const uint32_t lo = scan_begin(anchor, c.job, jb);
+    const uint32_t base = anchor.job == c.job ? anchor.incl : 0u;
+    uint32_t skip = 0, between = 0;
+    bool have = false;
+    if (shared_scan) {
+        if (!mbar_wait(&plan.scanbar, scan_parity)) status |= kStTimeout;
+        const uint32_t ps = (lane >= 1 && lane < kWarps) ? plan.part[lane] : 0u;
+        const uint32_t ok = (lane >= 1 && lane < kWarps) ? plan.ok[lane] : 1u;
+        between = __reduce_add_sync(kFull, ps);
+        have = __all_sync(kFull, ok != 0u);
+    }
+    if (!have) between = sum_sizes_warp(ws, lo, c.ticket, epoch, lane, skip, status);
+    const uint32_t excl = base + between;
+    anchor.incl = excl + total;
+    d.incl = excl + total;
     const unsigned long long blob_word0 = (unsigned long long)kHeaderWords + nT + excl;
     const bool fits = (blob_word0 + total) * 4ull <= job.out_cap;
     if (!fits) status |= kStCapacity;
-    const bool go = fits && !skip;
-    uint32_t* blob_out = job.out + blob_word0;
+    d.go = fits && !skip;
+    d.blob_out = job.out + blob_word0;
     if (lane < kWarps) plan.wbase[lane] = 1 + padw + inc - ww;
     if (lane == 0) {
-        plan.blob_out = go ? blob_out : nullptr;
+        plan.blob_out = d.go ? d.blob_out : nullptr;
         plan.padw = padw;
-        if (go) {
-            blob_out[0] = (uint32_t)c.q_first;
-            job.out[kHeaderWords + tile] = excl + total;
+    }
+    return d;
+}
+
+// Warp 0, once the other warps are copying: outlier, index entry, stream length, header of the tile just planned.
+__device__ __forceinline__ void finish_plan(const Planned& d, const Pending& c, const JobBatch& jb, float eb_abs, float s, int lane)
+{
+    const Job& job = jb.job[c.job];
+    const uint32_t tile = c.ticket - job.tile_begin;
+    const uint32_t nT = (uint32_t)((job.n + kTile - 1) / kTile);
+    if (lane == 0) {
+        if (d.go) {
+            d.blob_out[0] = (uint32_t)c.q_first;
+            job.out[kHeaderWords + tile] = d.incl;
         }
-        if (tile == nT - 1) *job.out_bytes = (size_t)((blob_word0 + total) * 4ull);
+        if (tile == nT - 1) *job.out_bytes = (size_t)(((unsigned long long)kHeaderWords + nT + d.incl) * 4ull);
     }
     if (tile == 0) write_header(job.out, lane, job.n, eb_abs, s, nT);
 }
@@ -1007,6 +1083,30 @@ __device__ __forceinline__ void copy_planned(const PlanShared& plan, const Pendi
     uint32_t* __restrict__ dst = blob_out + plan.wbase[warp];
     for (uint32_t i = lane; i < c.wsum; i += 32) dst[i] = slots_w[i];
     if (lane < 4 && (uint32_t)(4 * warp + lane) < plan.padw) blob_out[1 + 4 * warp + lane] = c.my_lw;
+}
+
+// First half of the placement of a pending tile, by the whole CTA, after the barrier that made the current tile's
+// sizes visible (have_cur) or at the end of the launch: warps 1..7 fetch the scan's sizes while warp 0 publishes
+// and lays out, then warp 0 completes the plan.  The caller follows with a barrier, copy_planned by every warp and
+// finish_plan by warp 0.  Uniform over the CTA.
+__device__ __forceinline__ Planned plan_pending(PlanShared& plan, const uint32_t* cur_words, uint32_t cur_padw, uint32_t ticket,
+                                                bool have_cur, const Pending& c, const uint32_t* pend_words, Anchor& anchor,
+                                                uint32_t& scan_parity, const JobBatch& jb, const Workspace& ws, uint32_t epoch,
+                                                int warp, int lane, uint32_t& status)
+{
+    Planned pl;
+    pl.blob_out = nullptr; pl.incl = 0; pl.go = false;
+    if (warp == 0) {
+        pl = announce_and_plan(plan, cur_words, cur_padw, ticket, have_cur, c, pend_words, anchor, c.valid, scan_parity, jb, ws,
+                               epoch, lane, status);
+    } else if (c.valid) {
+        scan_share(plan, ws, scan_begin(anchor, c.job, jb), c.ticket, epoch, warp, lane);
+    }
+    if (c.valid) {
+        scan_parity ^= 1u;
+        anchor.job = c.job; anchor.ticket = c.ticket;   // every warp tracks which tile was placed last; warp 0 also its prefix
+    }
+    return pl;
 }
 
 // ------------------------------------------------------------------------------------------------ compress
@@ -1037,10 +1137,12 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     };
     if (tid == 0) {
         mbar_init(&sh.bar, 1);
+        mbar_init(&sh.plan.scanbar, kWarps - 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         stage(blockIdx.x);
     }
     __syncthreads();
+    uint32_t scan_par = 0;   // phase parity of the scan's hand-off barrier
     uint32_t fills = 0;    // completed bulk copies (phase parity of the mbarrier)
     uint32_t p = 0;        // half of the slots the current tile is encoded into
     Pending pend;
@@ -1104,14 +1206,13 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps are visible; the staged tile has been consumed
-        if (tid == 32) stage(ticket + G);   // by warp 1, while warp 0 plans the placement of the previous tile
-        if (warp == 0) {
-            announce_and_plan(sh.plan, sh.warp_words[p], (nb + 3) >> 2, ticket, true, pend, sh.warp_words[pend.buf], anchor, jb,
-                              eb_abs, s, ws, epoch, lane, status);
-        }
+        const Planned pl = plan_pending(sh.plan, sh.warp_words[p], (nb + 3) >> 2, ticket, true, pend, sh.warp_words[pend.buf], anchor,
+                                        scan_par, jb, ws, epoch, warp, lane, status);
+        if (tid == 32) stage(ticket + G);   // by warp 1, while warp 0 completes the plan
         if (pend.valid) {
             __syncthreads();   // the plan is visible
             copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+            if (warp == 0) finish_plan(pl, pend, jb, eb_abs, s, lane);
         }
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
         pend.q_first = q_first;
@@ -1119,11 +1220,11 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     }
     if (pend.valid) {
         __syncthreads();
-        if (warp == 0)
-            announce_and_plan(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, jb, eb_abs, s, ws, epoch,
-                              lane, status);
+        const Planned pl = plan_pending(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, scan_par, jb, ws, epoch,
+                                        warp, lane, status);
         __syncthreads();
         copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+        if (warp == 0) finish_plan(pl, pend, jb, eb_abs, s, lane);
     }
 
     // never leave with a bulk copy in flight into this CTA's shared memory: every copy that was started has been
@@ -1164,9 +1265,11 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     if (tid == 0) {
         mbar_init(&sh.bar[0], 1);
         mbar_init(&sh.bar[1], 1);
+        mbar_init(&sh.plan.scanbar, kWarps - 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    uint32_t scan_par = 0;   // phase parity of the scan's hand-off barrier
     if (tid == 32) {
         pipe.fetch(jb, blockIdx.x, cur_job, h1);
         pipe.stage(sh, jb, blockIdx.x, cur_job, h1, 0);
@@ -1390,13 +1493,13 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps
-        if (warp == 0)
-            announce_and_plan(sh.plan, sh.warp_words[p], padw, ticket, true, pend, sh.warp_words[pend.buf], anchor, jb, pend_eb, pend_s,
-                              ws, epoch, lane, status);
+        const Planned pl = plan_pending(sh.plan, sh.warp_words[p], padw, ticket, true, pend, sh.warp_words[pend.buf], anchor, scan_par,
+                                        jb, ws, epoch, warp, lane, status);
         stage_next(ticket);
         __syncthreads();   // the plan and the next tile's span are visible
         if (pend.valid) {
             copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+            if (warp == 0) finish_plan(pl, pend, jb, pend_eb, pend_s, lane);
         }
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
         pend.q_first = q_first;
@@ -1404,11 +1507,11 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     }
     if (pend.valid) {
         __syncthreads();
-        if (warp == 0)
-            announce_and_plan(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, jb, pend_eb, pend_s, ws, epoch,
-                              lane, status);
+        const Planned pl = plan_pending(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, scan_par, jb, ws, epoch,
+                                        warp, lane, status);
         __syncthreads();
         copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+        if (warp == 0) finish_plan(pl, pend, jb, pend_eb, pend_s, lane);
     }
     if (tid == 0 && (status & kStTimeout)) {
         (void)mbar_wait(&sh.bar[0], (fills0 + 1u) & 1u);
