@@ -840,6 +840,7 @@ struct EncodeShared {
     alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];    // encoded tiles: current and awaiting placement
     uint32_t warp_words[2][kWarps];
     PlanShared plan;
+    uint32_t next_ticket;                                          // number of the tile after the current one
     alignas(8) unsigned long long bar;
 };
 
@@ -882,7 +883,7 @@ __device__ __forceinline__ void write_header(uint32_t* out, int tid, unsigned lo
     }
 }
 
-__device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoch, int tid)
+__device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoch, int tid, uint32_t* tile_counter = nullptr)
 {
     __syncthreads();
     if (tid == 0) {
@@ -890,6 +891,7 @@ __device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoc
         const uint32_t prev = atomicAdd(ws.done, 1u);
         if (prev == gridDim.x - 1) {   // every CTA is done with the scan states: re-arm for the next launch
             *ws.done = 0;
+            if (tile_counter) *tile_counter = 0;
             uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
             if (e == 0) {   // the counter wraps (once in 2^31 launches): no state of an earlier launch may look current again
                 for (uint32_t t = 0; t < ws.max_tiles; ++t) st_state(ws.tile_state + t, 0ull);
@@ -1117,7 +1119,6 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     EncodeShared& sh = *reinterpret_cast<EncodeShared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
-    const uint32_t G = gridDim.x;
     uint32_t status = 0;
     Params prm = hp;
     if (use_dev_params) prm = *ws.params;
@@ -1135,11 +1136,19 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
             }
         }
     };
+    // Tiles are handed out in order by a device-wide counter, one tile ahead of the encoding (the thread that
+    // requests a tile's input takes its number): a CTA that gets fewer issue slots than its neighbours simply takes
+    // fewer tiles, and every tile before a given one was taken earlier than it.
+    auto take_next = [&]() {
+        const uint32_t t = atomicAdd(ws.ticket, 1u);
+        sh.next_ticket = t;
+        stage(t);
+    };
     if (tid == 0) {
         mbar_init(&sh.bar, 1);
         mbar_init(&sh.plan.scanbar, kWarps - 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        stage(blockIdx.x);
+        take_next();
     }
     __syncthreads();
     uint32_t scan_par = 0;   // phase parity of the scan's hand-off barrier
@@ -1151,7 +1160,9 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     anchor.job = -1; anchor.ticket = 0; anchor.incl = 0;
     const Xpose xp(lane);
 
-    for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += G) {
+    for (;;) {
+        const uint32_t ticket = sh.next_ticket;   // written before the last barrier
+        if (ticket >= jb.total_tiles) break;
         const int j = find_job(jb, ticket);
         const Job& job = jb.job[j];
         const uint32_t tile = ticket - job.tile_begin;
@@ -1160,12 +1171,14 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
 
         if (n == 0 || !prm.valid) {   // a job without elements still owns one tile number: header and length only
             const bool hdr = prm.valid && job.out_cap >= (unsigned)kHeaderBytes;
+            __syncthreads();   // every thread has read this tile's number
             if (tid == 0) {
                 st_state(ws.tile_state + ticket, pack_state(epoch, 0u, 0u));
                 if (tile == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
-                stage(ticket + G);   // nothing was staged for this tile, and the buffer's last readers are past a barrier
+                take_next();   // nothing was staged for this tile, and the buffer's last readers are past a barrier
             }
             if (hdr && tile == 0) write_header(job.out, tid, 0, eb_abs, s, 0);
+            __syncthreads();   // the next tile's number is visible
             continue;
         }
 
@@ -1208,9 +1221,9 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         __syncthreads();   // sizes of all warps are visible; the staged tile has been consumed
         const Planned pl = plan_pending(sh.plan, sh.warp_words[p], (nb + 3) >> 2, ticket, true, pend, sh.warp_words[pend.buf], anchor,
                                         scan_par, jb, ws, epoch, warp, lane, status);
-        if (tid == 32) stage(ticket + G);   // by warp 1, while warp 0 completes the plan
+        if (tid == 32) take_next();   // by warp 1, while warp 0 completes the plan
+        __syncthreads();   // the plan and the next tile's number are visible
         if (pend.valid) {
-            __syncthreads();   // the plan is visible
             copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
             if (warp == 0) finish_plan(pl, pend, jb, eb_abs, s, lane);
         }
@@ -1231,7 +1244,7 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     // waited for by the iteration that consumed it, except after an expired wait; then give it one more bounded wait
     if (tid == 0 && (status & kStTimeout)) (void)mbar_wait(&sh.bar, (fills + 1u) & 1u);
     if (status) atomicOr(ws.status, status);
-    finish_launch(ws, epoch, tid);
+    finish_launch(ws, epoch, tid, ws.ticket);
 }
 
 // ------------------------------------------------------------------------------------------------ fused hop
