@@ -60,6 +60,7 @@ def lib():
         L.zo_sim_bcast.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32, szp]
         L.zo_sim_reduce_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
                                             C.c_void_p]
+        L.zo_quality.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.zo_sim_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
                                      C.c_void_p, C.c_void_p]
         _lib = L
@@ -238,3 +239,14 @@ def sim_scatter(root, N: int, eb_mode: int, eb: float, T: int = DEFAULT_TILE):
         raise OracleError(rc, "sim_scatter")
     nrounds = max(N - 1, 0).bit_length()
     return recv, rc, sizes, rounds[:nrounds]
+
+
+def quality(x, y):
+    """Quality of the reconstruction y of x: dict with max_abs_err, mse, nrmse, psnr, min, max (fp64)."""
+    x, y = _f32(x), _f32(y)
+    assert x.size == y.size
+    out = np.zeros(6, dtype=np.float64)
+    rc = lib().zo_quality(_ptr(x), _ptr(y), x.size, _ptr(out))
+    if rc < 0:
+        raise OracleError(rc, "quality")
+    return dict(max_abs_err=out[0], mse=out[1], nrmse=out[2], psnr=out[3], min=out[4], max=out[5])

@@ -593,3 +593,33 @@ int zo_sim_scatter(const float *root, float *const *recv, int N, size_t n, int e
     if (rc < 0) return rc;
     return warn ? ZO_W_PRECISION : ZO_OK;
 }
+
+/* Quality of a reconstruction y of x (Section 4.1: the paper reports NRMSE and PSNR next to the bit rate
+ * 32 / ratio; the definitions are the usual ones): everything in fp64, elements taken in order.
+ *   out[0] = max |x_i - y_i|          out[1] = MSE = mean (x_i - y_i)^2
+ *   out[2] = NRMSE = sqrt(MSE) / (max x - min x)      out[3] = PSNR = 20 log10((max x - min x) / sqrt(MSE)) dB
+ *   out[4] = min x                    out[5] = max x
+ * A constant x has no range: NRMSE and PSNR are then NaN; an exact reconstruction has PSNR = +inf. */
+int zo_quality(const float *x, const float *y, size_t n, double *out)
+{
+    if (n == 0) return ZO_E_ARG;
+    double maxerr = 0.0, sumsq = 0.0, lo = (double)x[0], hi = (double)x[0];
+    for (size_t i = 0; i < n; ++i) {
+        double d = (double)x[i] - (double)y[i];
+        double a = fabs(d);
+        if (a > maxerr) maxerr = a;
+        sumsq += d * d;
+        if ((double)x[i] < lo) lo = (double)x[i];
+        if ((double)x[i] > hi) hi = (double)x[i];
+    }
+    double mse = sumsq / (double)n;
+    double range = hi - lo;
+    out[0] = maxerr; out[1] = mse; out[4] = lo; out[5] = hi;
+    if (range > 0.0) {
+        out[2] = sqrt(mse) / range;
+        out[3] = mse > 0.0 ? 20.0 * log10(range / sqrt(mse)) : (double)INFINITY;
+    } else {
+        out[2] = (double)NAN; out[3] = (double)NAN;
+    }
+    return ZO_OK;
+}
