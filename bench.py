@@ -329,6 +329,29 @@ def main():
                 "algorithmic_bytes_per_launch": kern[dom]["bytes"]}
     roofline["traffic"] = DRAM_TRAFFIC_FUSED_64MIB
 
+    # ---- quality of the reconstruction (Section 4.1: NRMSE, PSNR, bit rate), and the metrics kernel's own roofline
+    # (it reads both arrays once: 8 bytes per element, nothing else)
+    qout = torch.zeros(6, dtype=torch.float64, device=dev)
+    for k in range(ROT):
+        ctx.compress(xs[k], z.EB_REL, REL, cs[k], nb1)
+        ctx.decompress(cs[k], ys[k])
+    q_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for i in range(args.steps):
+        k = (i + 1) % ROT if i + 1 < args.steps else 0   # the last launch looks at the batch the ratios are quoted on
+        q_ev[i][0].record(stream)
+        ctx.quality(xs[k], ys[k], qout)
+        q_ev[i][1].record(stream)
+    torch.cuda.synchronize()
+    q_ms = statistics.mean(a.elapsed_time(b) for a, b in q_ev)
+    qv = qout.cpu().numpy()
+    quality = {"max_abs_err": float(qv[0]), "nrmse": float(qv[2]), "psnr_db": float(qv[3]), "bit_rate": 32.0 / ratio1,
+               "eb_abs": eb_abs}
+    kern["quality(metrics)"] = {"ms": q_ms, "bytes": 2.0 * in_b}
+    kq = kern["quality(metrics)"]
+    kq["achieved_gbs"] = kq["bytes"] / (kq["ms"] * 1e-3) / 1e9
+    kq["frac"] = kq["achieved_gbs"] / peak
+    kq["uncompressed_gbs"] = in_b / (kq["ms"] * 1e-3) / 1e9
+
     # ---- end to end through the host-buffer entry points (pinned host memory; copies inside the timed region)
     xh = torch.from_numpy(x_h).pin_memory()
     oh = torch.empty(cap, dtype=torch.uint8).pin_memory()
@@ -373,7 +396,7 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
             "ops_ms": op_ms, "ops_uncompressed_gbs": {nm: units[nm] / (op_ms[nm] * 1e-3) / 1e9 for nm in names},
-            "kernels": kern,
+            "kernels": kern, "quality": quality,
         }
         print(json.dumps(line))
     ctx.close()

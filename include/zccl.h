@@ -238,6 +238,18 @@ int zccl_sim_scatter(zccl_ctx* ctx, const float* root, float* const* recv, int n
 int zccl_sim_sizes(zccl_ctx* ctx, size_t* sizes, int capacity, void* stream);
 
 /*
+ * Quality of a reconstruction y of x (Section 4.1: NRMSE and PSNR, reported next to the bit rate 32 / ratio),
+ * computed in fp64 on the device.
+ *   x, y [device] n floats (n >= 1, n <= max_elems of the context)
+ *   out  [device] 6 doubles: max |x - y|, MSE = mean (x - y)^2, NRMSE = sqrt(MSE) / (max x - min x),
+ *                 PSNR = 20 log10((max x - min x) / sqrt(MSE)) in dB, min x, max x.
+ * A constant x gives NaN for NRMSE and PSNR; an exact reconstruction gives PSNR = +inf.  Sums are formed per
+ * thread, per CTA and then over the CTAs in a fixed order, so the result does not vary from run to run.
+ * Returns ZCCL_E_ARG for a null pointer, n == 0 or n beyond the context's max_elems.
+ */
+int zccl_quality(zccl_ctx* ctx, const float* x, const float* y, size_t n, double* out, void* stream);
+
+/*
  * Host-buffer convenience forms: copy the input from host memory into a staging area of the context, run the
  * device path, copy the result back, all enqueued on `stream` (pinned host memory makes the copies asynchronous).
  * They exist so that end-to-end cost including PCIe transfers can be measured through this boundary.

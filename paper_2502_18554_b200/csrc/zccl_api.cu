@@ -16,6 +16,8 @@ struct zccl_ctx {
     size_t max_elems = 0;
     int max_ranks = 0;
     uint32_t debug_epoch = 0;
+    double* quality_partials = nullptr;   // device: per-CTA partial results of zccl_quality
+    uint32_t* quality_counter = nullptr;
     Workspace ws{};
     void* small_block = nullptr;     // tile states + counters + params + sizes
     uint8_t* arena = nullptr;        // compressed-chunk slots of the emulated ranks
@@ -204,7 +206,8 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
     const size_t off_state = 0;
     const size_t off_small = align_up(off_state + 8 * max_tiles, 256);
     const size_t off_sizes = off_small + 256;
-    const size_t small_bytes = off_sizes + sizeof(size_t) * (size_t)(c->sim_sizes_cap + 1);
+    const size_t off_quality = align_up(off_sizes + sizeof(size_t) * (size_t)(c->sim_sizes_cap + 1), 256);
+    const size_t small_bytes = off_quality + sizeof(double) * 4 * (size_t)kQualityCtas + 256;
     bool ok = cudaMalloc(&c->small_block, small_bytes) == cudaSuccess;
     if (ok) ok = cudaMemset(c->small_block, 0, small_bytes) == cudaSuccess;
     if (ok) {
@@ -221,6 +224,8 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
         c->ws.skip_publish = 0xFFFFFFFFu;
         c->sim_sizes = (size_t*)(b + off_sizes);
         c->stage_bytes = c->sim_sizes + c->sim_sizes_cap;
+        c->quality_partials = (double*)(b + off_quality);
+        c->quality_counter = (uint32_t*)(b + off_quality + sizeof(double) * 4 * (size_t)kQualityCtas);
         const uint32_t init[3] = {1u, 0xFFFFFFFFu, 0u};   // epoch, min key, max key
         ok = cudaMemcpy(c->ws.epoch, &init[0], 4, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->ws.minmax, &init[1], 8, cudaMemcpyHostToDevice) == cudaSuccess;
@@ -633,6 +638,13 @@ int zccl_sim_scatter(zccl_ctx* c, const float* root, float* const* recv, int N, 
         if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
     }
     return flush_decode(c, b, st);
+}
+
+int zccl_quality(zccl_ctx* c, const float* x, const float* y, size_t n, double* out, void* stream)
+{
+    if (!c || !x || !y || !out || n == 0 || n > c->max_elems) return ZCCL_E_ARG;
+    if (((uintptr_t)x & 3u) || ((uintptr_t)y & 3u) || ((uintptr_t)out & 7u)) return ZCCL_E_ARG;
+    return cuda_rc(launch_quality(x, y, n, out, c->quality_partials, c->quality_counter, c->sm_count, (cudaStream_t)stream));
 }
 
 int zccl_sim_sizes(zccl_ctx* c, size_t* sizes, int capacity, void* stream)

@@ -120,6 +120,11 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
+// quality metrics: `partials` holds 4 doubles per CTA of the launch (at most kQualityCtas), `counter` one word that
+// is zero between launches
+constexpr int kQualityCtas = 1024;
+cudaError_t launch_quality(const float* x, const float* y, unsigned long long n, double* out, double* partials,
+                           uint32_t* counter, int sm_count, cudaStream_t st);
 cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
 unsigned long long launch_count();
 

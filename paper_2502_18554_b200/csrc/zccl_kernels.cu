@@ -1600,6 +1600,119 @@ __global__ void __launch_bounds__(256) copy_chain_kernel(ChainBatch cb, Workspac
     }
 }
 
+// ------------------------------------------------------------------------------------------------ quality metrics
+
+// max |x - y|, sum (x - y)^2, min x, max x.  The results are those of fp64 arithmetic, but the per-element work is
+// done in fp32 with error-free transformations (fp64 instructions are an order of magnitude more expensive here):
+// d = x - y together with its rounding error (the error is zero whenever x and y are within a factor of two of
+// each other, which a reconstruction always is); d^2 as an exact fp32 pair (product and fused-multiply-add
+// residual); the sum as a compensated fp32 pair.  A group of elements in which some difference is not an fp32
+// number takes the fp64 path.  128-bit loads, per-thread accumulators, warp shuffles, one partial per CTA, and the
+// last CTA to finish combines the partials in CTA order and writes the six results.
+__global__ void __launch_bounds__(256) quality_kernel(const float* __restrict__ x, const float* __restrict__ y, unsigned long long n,
+                                                      double* __restrict__ out, double* __restrict__ partials, uint32_t* counter)
+{
+    __shared__ double red[4][8];
+    __shared__ uint32_t is_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000), emax = 0.0f;
+    float sh = 0.0f, sl = 0.0f;     // compensated sum of squares of the differences that are fp32 numbers
+    double dmax = 0.0, dsum = 0.0;  // the others
+    auto take = [&](float a, float b) {
+        lo = fminf(lo, a);
+        hi = fmaxf(hi, a);
+        const float d = __fsub_rn(a, b);
+        const float bb = __fsub_rn(d, a);                                                     // TwoSum of a and -b
+        const float err = __fsub_rn(__fsub_rn(a, __fsub_rn(d, bb)), __fadd_rn(b, bb));
+        if (err == 0.0f) {
+            emax = fmaxf(emax, fabsf(d));
+            const float p = __fmul_rn(d, d), e = __fmaf_rn(d, d, -p);                         // d * d = p + e exactly
+            const float t = __fadd_rn(sh, p), z = __fsub_rn(t, sh);
+            sl = __fadd_rn(sl, __fadd_rn(__fadd_rn(__fsub_rn(sh, __fsub_rn(t, z)), __fsub_rn(p, z)), e));
+            sh = t;
+        } else {
+            const double dd = (double)a - (double)b;
+            dmax = fmax(dmax, fabs(dd));
+            dsum += dd * dd;
+        }
+    };
+    const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + tid;
+    const unsigned long long nth = (unsigned long long)gridDim.x * blockDim.x;
+    unsigned long long done = 0;
+    if (((((uintptr_t)x) | ((uintptr_t)y)) & 15u) == 0) {
+        const unsigned long long nv = n >> 2;
+        const float4* x4 = reinterpret_cast<const float4*>(x);
+        const float4* y4 = reinterpret_cast<const float4*>(y);
+        unsigned long long i = gtid;
+        for (; i + nth < nv; i += 2 * nth) {   // two independent pairs of loads in flight
+            const float4 a0 = __ldg(x4 + i), b0 = __ldg(y4 + i), a1 = __ldg(x4 + i + nth), b1 = __ldg(y4 + i + nth);
+            take(a0.x, b0.x); take(a0.y, b0.y); take(a0.z, b0.z); take(a0.w, b0.w);
+            take(a1.x, b1.x); take(a1.y, b1.y); take(a1.z, b1.z); take(a1.w, b1.w);
+        }
+        for (; i < nv; i += nth) {
+            const float4 a = __ldg(x4 + i), b = __ldg(y4 + i);
+            take(a.x, b.x); take(a.y, b.y); take(a.z, b.z); take(a.w, b.w);
+        }
+        done = nv << 2;
+    }
+    for (unsigned long long i = done + gtid; i < n; i += nth) take(__ldg(x + i), __ldg(y + i));
+    double maxerr = fmax(dmax, (double)emax), sumsq = dsum + ((double)sh + (double)sl);
+    double dlo = (double)lo, dhi = (double)hi;
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        maxerr = fmax(maxerr, __shfl_xor_sync(kFull, maxerr, d));
+        sumsq += __shfl_xor_sync(kFull, sumsq, d);
+        dlo = fmin(dlo, __shfl_xor_sync(kFull, dlo, d));
+        dhi = fmax(dhi, __shfl_xor_sync(kFull, dhi, d));
+    }
+    if (lane == 0) { red[0][warp] = maxerr; red[1][warp] = sumsq; red[2][warp] = dlo; red[3][warp] = dhi; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 8; ++w) {
+            maxerr = fmax(maxerr, red[0][w]); sumsq += red[1][w]; dlo = fmin(dlo, red[2][w]); dhi = fmax(dhi, red[3][w]);
+        }
+        double* mine = partials + 4ull * blockIdx.x;
+        mine[0] = maxerr; mine[1] = sumsq; mine[2] = dlo; mine[3] = dhi;
+        __threadfence();
+        is_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1u : 0u;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    // the last CTA: every thread takes the partials of CTAs tid, tid + 256, ... in that order, then the same tree as
+    // above: a fixed order of additions whatever order the CTAs finished in
+    __threadfence();
+    maxerr = 0.0; sumsq = 0.0; dlo = __longlong_as_double(0x7FF0000000000000ll); dhi = __longlong_as_double(0xFFF0000000000000ull);
+    for (unsigned b = tid; b < gridDim.x; b += 256) {
+        const volatile double* pb = partials + 4ull * b;
+        maxerr = fmax(maxerr, pb[0]); sumsq += pb[1]; dlo = fmin(dlo, pb[2]); dhi = fmax(dhi, pb[3]);
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        maxerr = fmax(maxerr, __shfl_xor_sync(kFull, maxerr, d));
+        sumsq += __shfl_xor_sync(kFull, sumsq, d);
+        dlo = fmin(dlo, __shfl_xor_sync(kFull, dlo, d));
+        dhi = fmax(dhi, __shfl_xor_sync(kFull, dhi, d));
+    }
+    __syncthreads();   // the first round's values in `red` have been read
+    if (lane == 0) { red[0][warp] = maxerr; red[1][warp] = sumsq; red[2][warp] = dlo; red[3][warp] = dhi; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 8; ++w) {
+            maxerr = fmax(maxerr, red[0][w]); sumsq += red[1][w]; dlo = fmin(dlo, red[2][w]); dhi = fmax(dhi, red[3][w]);
+        }
+        const double mse = sumsq / (double)n, range = dhi - dlo;
+        out[0] = maxerr; out[1] = mse; out[4] = dlo; out[5] = dhi;
+        if (range > 0.0) {
+            out[2] = sqrt(mse) / range;
+            out[3] = mse > 0.0 ? 20.0 * log10(range / sqrt(mse)) : __longlong_as_double(0x7FF0000000000000ll);
+        } else {
+            out[2] = __longlong_as_double(0x7FF8000000000000ll);
+            out[3] = __longlong_as_double(0x7FF8000000000000ll);
+        }
+        *counter = 0;
+    }
+}
+
 int g_raw_ctas_per_sm = 0, g_fused_ctas_per_sm = 0, g_decode_ctas_per_sm = 0;
 unsigned long long g_launches = 0;   // kernels launched by this library in this process
 
@@ -1677,6 +1790,18 @@ cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, 
     unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
     ++g_launches;
     copy_kernel<<<dim3(gx ? gx : 1, cb.count), 256, 0, st>>>(cb, ws);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quality(const float* x, const float* y, unsigned long long n, double* out, double* partials,
+                           uint32_t* counter, int sm_count, cudaStream_t st)
+{
+    unsigned long long want = (n / 4 + 255) / 256;
+    unsigned long long cap = (unsigned long long)sm_count * 6;
+    if (cap > (unsigned long long)kQualityCtas) cap = kQualityCtas;
+    const unsigned grid = (unsigned)(want < cap ? (want ? want : 1) : cap);
+    ++g_launches;
+    quality_kernel<<<grid, 256, 0, st>>>(x, y, n, out, partials, counter);
     return cudaGetLastError();
 }
 

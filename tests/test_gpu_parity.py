@@ -486,3 +486,52 @@ def test_scatter_matches_oracle(z, N, n):
         assert np.all(got[n:] == 7.0)
     assert np.array_equal(np.array(c.sim_sizes()), wsizes)
     c.close()
+
+
+def _quality(ctx, x, y):
+    out = torch.zeros(6, dtype=torch.float64, device="cuda")
+    ctx.quality(x, y, out)
+    v = out.cpu().numpy()
+    return dict(max_abs_err=v[0], mse=v[1], nrmse=v[2], psnr=v[3], min=v[4], max=v[5])
+
+
+@pytest.mark.parametrize("n", [1, 5, 4099, 1 << 20, (1 << 22) - 3])
+def test_quality_matches_oracle(z, ctx, n):
+    # exact for the extrema and the largest error (fp64 differences of fp32 values are exact); the sum of squares is
+    # formed in another order than the oracle's, so MSE and what derives from it agree to fp64 summation accuracy:
+    # n terms of one sign, relative error at most n * 2^-53 < 1e-9
+    import math
+    x = fields.smooth_1d(n, seed=50)
+    rng = np.random.default_rng(n)
+    y = (x + rng.normal(0, 1e-3, n)).astype(f32)
+    want = oracle.quality(x, y)
+    dx, dy = dev(x), dev(y)
+    got = _quality(ctx, dx, dy)
+    assert got["max_abs_err"] == want["max_abs_err"] and got["min"] == want["min"] and got["max"] == want["max"]
+    assert math.isclose(got["mse"], want["mse"], rel_tol=1e-9)
+    if n > 1:
+        assert math.isclose(got["nrmse"], want["nrmse"], rel_tol=1e-9) and math.isclose(got["psnr"], want["psnr"], rel_tol=1e-9)
+    else:
+        assert math.isnan(got["nrmse"]) and math.isnan(want["nrmse"])
+    again = _quality(ctx, dx, dy)                              # same bits on a second run
+    assert np.array_equal(np.array(list(again.values())), np.array(list(got.values())), equal_nan=True)
+    got_u = _quality(ctx, dev(np.concatenate([[0], x]).astype(f32))[1:], dev(np.concatenate([[0], y]).astype(f32))[1:])
+    assert got_u["max_abs_err"] == want["max_abs_err"] and math.isclose(got_u["mse"], want["mse"], rel_tol=1e-9)   # unaligned
+
+
+def test_quality_of_a_compressed_field(z, ctx):
+    import math
+    x = fields.fourier_field_3d(128, seed=4)
+    dx = dev(x)
+    out = torch.empty(z.compress_bound(x.size), dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx.compress(dx, z.EB_REL, 1e-3, out, nb)
+    y = torch.empty_like(dx)
+    ctx.decompress(out[: int(nb.item())], y)
+    q = _quality(ctx, dx, y)
+    ea, s, _ = oracle.resolve(oracle.EB_REL, 1e-3, x)
+    assert q["max_abs_err"] <= float(ea)
+    assert q["nrmse"] < 1e-3 and q["psnr"] > 60.0
+    assert _quality(ctx, dx, dx)["psnr"] == math.inf
+    want = oracle.quality(x, y.cpu().numpy())
+    assert q["max_abs_err"] == want["max_abs_err"] and math.isclose(q["mse"], want["mse"], rel_tol=1e-9)
