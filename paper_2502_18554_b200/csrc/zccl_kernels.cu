@@ -830,8 +830,13 @@ struct PlanShared {
     uint32_t* blob_out;       // where the pending tile's blob starts in the stream (nullptr: do not copy)
     uint32_t wbase[kWarps];   // each warp's first word inside the blob
     uint32_t padw;            // code-length words of the blob
-    uint32_t part[kWarps];    // scan: sum of the sizes warp w fetched (warps 1..7)
-    uint32_t ok[kWarps];      // scan: 1 if every state that warp saw was published
+    // what warp 0 worked out ahead of the barrier (laid_out != 0) and picks up again after it
+    uint32_t laid_out, total, nT, lo, base;
+};
+// Hand-off of the scan's sizes from warps 1..7 to warp 0.
+struct ScanShared {
+    uint32_t part[kWarps];    // sum of the sizes warp w fetched
+    uint32_t ok[kWarps];      // 1 if every state that warp saw was published
     alignas(8) unsigned long long scanbar;   // warps 1..7 arrive once their shares are written
 };
 
@@ -839,7 +844,8 @@ struct EncodeShared {
     alignas(16) float xbuf[kTile + 8];                             // staged input tile (+ guard word in front)
     alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];    // encoded tiles: current and awaiting placement
     uint32_t warp_words[2][kWarps];
-    PlanShared plan;
+    PlanShared plan[2];                                            // placements alternate between the two cells
+    ScanShared scan;
     uint32_t next_ticket;                                          // number of the tile after the current one
     alignas(8) unsigned long long bar;
 };
@@ -854,7 +860,8 @@ struct FusedShared {
     int32_t warp_total_i[kWarps];
     int32_t warp_total_i2[kWarps];
     uint32_t warp_words[2][kWarps];
-    PlanShared plan;
+    PlanShared plan[2];                                              // placements alternate between the two cells
+    ScanShared scan;
     alignas(8) unsigned long long bar[2];
 };
 
@@ -967,7 +974,7 @@ __device__ __forceinline__ uint32_t scan_begin(const Anchor& a, int job_index, c
 // Warps 1..7, while warp 0 publishes and lays out: each fetches its share of the sizes of tiles [lo, hi) (window k
 // of 32 tiles belongs to warp 1 + k mod 7, all loads of a warp in flight together), leaves the sum for warp 0 and
 // arrives on the hand-off barrier.  One round trip to L2 for the whole scan.
-__device__ __forceinline__ void scan_share(PlanShared& plan, const Workspace& ws, uint32_t lo, uint32_t hi, uint32_t epoch,
+__device__ __forceinline__ void scan_share(ScanShared& plan, const Workspace& ws, uint32_t lo, uint32_t hi, uint32_t epoch,
                                            int warp, int lane)
 {
     uint32_t sum = 0;
@@ -1000,23 +1007,11 @@ struct Planned {
     bool go;
 };
 
-// Warp 0, after the barrier that follows a tile's encoding pass: publishes the size of the tile just encoded
-// (`ticket`, sizes in `cur_words`) and plans the pending one (sizes in `pend_words`): layout of the warps' regions,
-// then the scan's sum from the other warps' shares (`shared_scan`; a blocking scan of its own when a size was not
-// published yet, or when there are no shares), capacity check.
-__device__ __forceinline__ Planned announce_and_plan(PlanShared& plan, const uint32_t* cur_words, uint32_t cur_padw, uint32_t ticket,
-                                                     bool have_cur, const Pending& c, const uint32_t* pend_words, Anchor& anchor,
-                                                     bool shared_scan, uint32_t scan_parity, const JobBatch& jb,
-                                                     const Workspace& ws, uint32_t epoch, int lane, uint32_t& status)
+// Warp 0, any time after the pending tile was encoded (the encoder does it while it waits for the next input
+// tile): everything about its placement that does not depend on the other CTAs' sizes.
+__device__ __forceinline__ void lay_out_pending(PlanShared& plan, const Pending& c, const uint32_t* pend_words, const Anchor& anchor,
+                                                const JobBatch& jb, int lane)
 {
-    Planned d;
-    d.blob_out = nullptr; d.incl = 0; d.go = false;
-    if (have_cur) {
-        const uint32_t ww = lane < kWarps ? cur_words[lane] : 0u;
-        const uint32_t total = 1 + cur_padw + __reduce_add_sync(kFull, ww);
-        if (lane == 0 && ticket != ws.skip_publish) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
-    }
-    if (!c.valid) return d;
     const Job& job = jb.job[c.job];
     const uint32_t tile = c.ticket - job.tile_begin;
     const unsigned long long start = (unsigned long long)tile * kTile;
@@ -1032,14 +1027,43 @@ __device__ __forceinline__ Planned announce_and_plan(PlanShared& plan, const uin
         if (lane >= k) inc += up;
     }
     const uint32_t total = 1 + padw + __shfl_sync(kFull, inc, kWarps - 1);
-    const uint32_t lo = scan_begin(anchor, c.job, jb);
-    const uint32_t base = anchor.job == c.job ? anchor.incl : 0u;
+    if (lane < kWarps) plan.wbase[lane] = 1 + padw + inc - ww;
+    if (lane == 0) {
+        plan.padw = padw;
+        plan.total = total; plan.nT = nT;
+        plan.lo = scan_begin(anchor, c.job, jb);
+        plan.base = anchor.job == c.job ? anchor.incl : 0u;
+        plan.laid_out = 1u;
+    }
+    __syncwarp();
+}
+
+// Warp 0, after the barrier that follows a tile's encoding pass: publishes the size of the tile just encoded
+// (`ticket`, sizes in `cur_words`) and completes the plan of the pending one: the scan's sum from the other warps'
+// shares (`shared_scan`; a blocking scan of its own when a size was not published yet, or when there are no
+// shares), capacity check, target address.
+__device__ __forceinline__ Planned announce_and_plan(PlanShared& plan, ScanShared& scan, const uint32_t* cur_words, uint32_t cur_padw,
+                                                     uint32_t ticket, bool have_cur, const Pending& c, const uint32_t* pend_words,
+                                                     Anchor& anchor, bool shared_scan, uint32_t scan_parity, const JobBatch& jb,
+                                                     const Workspace& ws, uint32_t epoch, int lane, uint32_t& status)
+{
+    Planned d;
+    d.blob_out = nullptr; d.incl = 0; d.go = false;
+    if (have_cur) {
+        const uint32_t ww = lane < kWarps ? cur_words[lane] : 0u;
+        const uint32_t total = 1 + cur_padw + __reduce_add_sync(kFull, ww);
+        if (lane == 0 && ticket != ws.skip_publish) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
+    }
+    if (!c.valid) return d;
+    if (!plan.laid_out) lay_out_pending(plan, c, pend_words, anchor, jb, lane);
+    const uint32_t total = plan.total, nT = plan.nT, lo = plan.lo, base = plan.base;
+    const Job& job = jb.job[c.job];
     uint32_t skip = 0, between = 0;
     bool have = false;
     if (shared_scan) {
-        if (!mbar_wait(&plan.scanbar, scan_parity)) status |= kStTimeout;
-        const uint32_t ps = (lane >= 1 && lane < kWarps) ? plan.part[lane] : 0u;
-        const uint32_t ok = (lane >= 1 && lane < kWarps) ? plan.ok[lane] : 1u;
+        if (!mbar_wait(&scan.scanbar, scan_parity)) status |= kStTimeout;
+        const uint32_t ps = (lane >= 1 && lane < kWarps) ? scan.part[lane] : 0u;
+        const uint32_t ok = (lane >= 1 && lane < kWarps) ? scan.ok[lane] : 1u;
         between = __reduce_add_sync(kFull, ps);
         have = __all_sync(kFull, ok != 0u);
     }
@@ -1052,10 +1076,10 @@ __device__ __forceinline__ Planned announce_and_plan(PlanShared& plan, const uin
     if (!fits) status |= kStCapacity;
     d.go = fits && !skip;
     d.blob_out = job.out + blob_word0;
-    if (lane < kWarps) plan.wbase[lane] = 1 + padw + inc - ww;
+    __syncwarp();
     if (lane == 0) {
         plan.blob_out = d.go ? d.blob_out : nullptr;
-        plan.padw = padw;
+        plan.laid_out = 0u;   // the next tile planned in this cell starts afresh
     }
     return d;
 }
@@ -1091,18 +1115,18 @@ __device__ __forceinline__ void copy_planned(const PlanShared& plan, const Pendi
 // sizes visible (have_cur) or at the end of the launch: warps 1..7 fetch the scan's sizes while warp 0 publishes
 // and lays out, then warp 0 completes the plan.  The caller follows with a barrier, copy_planned by every warp and
 // finish_plan by warp 0.  Uniform over the CTA.
-__device__ __forceinline__ Planned plan_pending(PlanShared& plan, const uint32_t* cur_words, uint32_t cur_padw, uint32_t ticket,
-                                                bool have_cur, const Pending& c, const uint32_t* pend_words, Anchor& anchor,
-                                                uint32_t& scan_parity, const JobBatch& jb, const Workspace& ws, uint32_t epoch,
-                                                int warp, int lane, uint32_t& status)
+__device__ __forceinline__ Planned plan_pending(PlanShared& plan, ScanShared& scan, const uint32_t* cur_words, uint32_t cur_padw,
+                                                uint32_t ticket, bool have_cur, const Pending& c, const uint32_t* pend_words,
+                                                Anchor& anchor, uint32_t& scan_parity, const JobBatch& jb, const Workspace& ws,
+                                                uint32_t epoch, int warp, int lane, uint32_t& status)
 {
     Planned pl;
     pl.blob_out = nullptr; pl.incl = 0; pl.go = false;
     if (warp == 0) {
-        pl = announce_and_plan(plan, cur_words, cur_padw, ticket, have_cur, c, pend_words, anchor, c.valid, scan_parity, jb, ws,
+        pl = announce_and_plan(plan, scan, cur_words, cur_padw, ticket, have_cur, c, pend_words, anchor, c.valid, scan_parity, jb, ws,
                                epoch, lane, status);
     } else if (c.valid) {
-        scan_share(plan, ws, scan_begin(anchor, c.job, jb), c.ticket, epoch, warp, lane);
+        scan_share(scan, ws, scan_begin(anchor, c.job, jb), c.ticket, epoch, warp, lane);
     }
     if (c.valid) {
         scan_parity ^= 1u;
@@ -1146,7 +1170,8 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     };
     if (tid == 0) {
         mbar_init(&sh.bar, 1);
-        mbar_init(&sh.plan.scanbar, kWarps - 1);
+        mbar_init(&sh.scan.scanbar, kWarps - 1);
+        sh.plan[0].laid_out = 0u; sh.plan[1].laid_out = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         take_next();
     }
@@ -1192,6 +1217,9 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         int32_t q_first = 0;
         float guard = 0.0f, tmax = 0.0f;
         bool need_int = !staged;
+        // while the input tile is on its way, warp 0 lays out the pending tile (its cell of the plan is free: the
+        // placement before it used the other one)
+        if (warp == 0 && pend.valid) lay_out_pending(sh.plan[scan_par], pend, sh.warp_words[pend.buf], anchor, jb, lane);
         if (staged) {
             const bool landed = mbar_wait(&sh.bar, fills & 1u);
             ++fills;
@@ -1219,12 +1247,13 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps are visible; the staged tile has been consumed
-        const Planned pl = plan_pending(sh.plan, sh.warp_words[p], (nb + 3) >> 2, ticket, true, pend, sh.warp_words[pend.buf], anchor,
-                                        scan_par, jb, ws, epoch, warp, lane, status);
+        PlanShared& cell = sh.plan[scan_par];
+        const Planned pl = plan_pending(cell, sh.scan, sh.warp_words[p], (nb + 3) >> 2, ticket, true, pend, sh.warp_words[pend.buf],
+                                        anchor, scan_par, jb, ws, epoch, warp, lane, status);
         if (tid == 32) take_next();   // by warp 1, while warp 0 completes the plan
         __syncthreads();   // the plan and the next tile's number are visible
         if (pend.valid) {
-            copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+            copy_planned(cell, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
             if (warp == 0) finish_plan(pl, pend, jb, eb_abs, s, lane);
         }
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
@@ -1233,10 +1262,11 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     }
     if (pend.valid) {
         __syncthreads();
-        const Planned pl = plan_pending(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, scan_par, jb, ws, epoch,
-                                        warp, lane, status);
+        PlanShared& cell = sh.plan[scan_par];
+        const Planned pl = plan_pending(cell, sh.scan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, scan_par, jb, ws,
+                                        epoch, warp, lane, status);
         __syncthreads();
-        copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+        copy_planned(cell, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
         if (warp == 0) finish_plan(pl, pend, jb, eb_abs, s, lane);
     }
 
@@ -1278,7 +1308,8 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     if (tid == 0) {
         mbar_init(&sh.bar[0], 1);
         mbar_init(&sh.bar[1], 1);
-        mbar_init(&sh.plan.scanbar, kWarps - 1);
+        mbar_init(&sh.scan.scanbar, kWarps - 1);
+        sh.plan[0].laid_out = 0u; sh.plan[1].laid_out = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -1506,12 +1537,13 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         }
         if (lane == 0) sh.warp_words[p][warp] = wsum;
         __syncthreads();   // sizes of all warps
-        const Planned pl = plan_pending(sh.plan, sh.warp_words[p], padw, ticket, true, pend, sh.warp_words[pend.buf], anchor, scan_par,
-                                        jb, ws, epoch, warp, lane, status);
+        PlanShared& cell = sh.plan[scan_par];
+        const Planned pl = plan_pending(cell, sh.scan, sh.warp_words[p], padw, ticket, true, pend, sh.warp_words[pend.buf], anchor,
+                                        scan_par, jb, ws, epoch, warp, lane, status);
         stage_next(ticket);
         __syncthreads();   // the plan and the next tile's span are visible
         if (pend.valid) {
-            copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+            copy_planned(cell, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
             if (warp == 0) finish_plan(pl, pend, jb, pend_eb, pend_s, lane);
         }
         pend.valid = true; pend.job = j; pend.ticket = ticket; pend.buf = p; pend.wsum = wsum; pend.my_lw = my_lw;
@@ -1520,10 +1552,11 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     }
     if (pend.valid) {
         __syncthreads();
-        const Planned pl = plan_pending(sh.plan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, scan_par, jb, ws, epoch,
-                                        warp, lane, status);
+        PlanShared& cell = sh.plan[scan_par];
+        const Planned pl = plan_pending(cell, sh.scan, nullptr, 0, 0, false, pend, sh.warp_words[pend.buf], anchor, scan_par, jb, ws,
+                                        epoch, warp, lane, status);
         __syncthreads();
-        copy_planned(sh.plan, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
+        copy_planned(cell, pend, sh.slots[pend.buf] + kSlotWords * kBlocksPerWarp * warp, warp, lane);
         if (warp == 0) finish_plan(pl, pend, jb, pend_eb, pend_s, lane);
     }
     if (tid == 0 && (status & kStTimeout)) {
