@@ -19,6 +19,7 @@ _LIB = _HERE / "libzccl_oracle.so"
 OK, E_ARG, E_CAPACITY, E_RANGE, E_BAD_STREAM, E_DEGENERATE, W_PRECISION = 0, -1, -3, -4, -5, -7, 1
 EB_ABS, EB_REL = 0, 1
 FLAG_CONSISTENT_OWNER = 1
+OP_SUM, OP_MAX, OP_MIN, OP_AVG = 0, 2, 4, 6   # reduce operation, or-ed into flags
 DEFAULT_TILE = 4096
 HEADER_BYTES = 32
 

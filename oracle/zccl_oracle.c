@@ -49,6 +49,12 @@
 #define ZO_EB_REL 1
 
 #define ZO_FLAG_CONSISTENT_OWNER 1u
+/* reduce operation of the collective computation framework (Section 3.2: Sum, Average, Max, Min), bits 1..2 */
+#define ZO_OP_MASK 6u
+#define ZO_OP_SUM 0u
+#define ZO_OP_MAX 2u
+#define ZO_OP_MIN 4u
+#define ZO_OP_AVG 6u   /* Sum on every hop; the collective divides the result by the number of ranks at the end */
 
 #define ZO_MAGIC   0x314C435Au /* bytes 'Z','C','L','1' */
 #define ZO_VERSION 0x05000001u
@@ -313,7 +319,8 @@ int zo_decompress(const uint8_t *in, size_t in_bytes, float *y, size_t cap_elems
 
 /* ---------------------------------------------------------------- reduce-scatter hop (Section 3.1.2, Eq. 2) */
 
-/* out_c = compress( decompress(in_c) + local ), written as exactly that composition.  Exactly one of `local`
+/* out_c = compress( decompress(in_c) (+) local ), written as exactly that composition; (+) is the addition unless
+ * flags select Max or Min (the larger / the smaller of the two, the decoded operand kept when they compare equal).  Exactly one of `local`
  * (uncompressed fp32 chunk: the paper's form) and `local_c` (a second compressed chunk) is non-NULL.  The bound
  * and step are those of in_c's header (one bound for the whole collective).  raw_out, if given, receives the
  * fp32 sum y, or float(q(y))*s when ZO_FLAG_CONSISTENT_OWNER is set. */
@@ -343,7 +350,12 @@ int zo_drc(const uint8_t *in_c, size_t in_bytes, const float *local, const uint8
         if (rc != ZO_OK) { free(a); free(b); return rc; }
         local = b;
     }
-    for (size_t i = 0; i < m; ++i) a[i] = a[i] + local[i];   /* decoded partial on the left, one fp32 add */
+    unsigned op = flags & ZO_OP_MASK;
+    for (size_t i = 0; i < m; ++i) {   /* decoded partial on the left, one fp32 operation */
+        if (op == ZO_OP_MAX) a[i] = (a[i] < local[i]) ? local[i] : a[i];
+        else if (op == ZO_OP_MIN) a[i] = (local[i] < a[i]) ? local[i] : a[i];
+        else a[i] = a[i] + local[i];
+    }
     rc = zo_compress_core(a, m, eb_abs, s, r, T, out_c, cap, out_bytes);
     if (rc >= 0 && raw_out) {
         if (flags & ZO_FLAG_CONSISTENT_OWNER) {
@@ -443,6 +455,9 @@ int zo_sim_allreduce(const float *const *send, float *const *recv, int N, size_t
             if (rc2 != ZO_OK) rc = rc2;
         }
     }
+    if ((flags & ZO_OP_MASK) == ZO_OP_AVG && rc >= 0)   /* Average = Sum / N, one fp32 division per element */
+        for (int rk = 0; rk < N; ++rk)
+            for (size_t i = 0; i < n; ++i) recv[rk][i] = recv[rk][i] / (float)N;
     for (int k = 0; k < N; ++k) { free(cur[k]); free(nxt[k]); }
     free(cur); free(nxt); free(cur_b); free(nxt_b);
     if (rc < 0) return rc;

@@ -286,3 +286,70 @@ def test_scatter_compress_once_and_tree_traffic(N, n):
     # every chunk but the root's crosses at least one link; the first round carries about half of them
     if N > 1:
         assert sum(int(v) for v in rounds) >= int(np.sum(sizes))
+
+
+# ---------------------------------------------------------------- other reduce operations (Section 3.2: Average, Max, Min)
+
+@pytest.mark.parametrize("op,fn", [(oracle.OP_MAX, np.maximum), (oracle.OP_MIN, np.minimum)])
+def test_hop_max_min_is_the_composition(op, fn):
+    # the fused hop with Max / Min is compress(max(decompress(in), local)): composition of pinned primitives
+    n = 3 * 4096 + 50
+    a, b = fields.smooth_1d(n, seed=11), fields.smooth_1d(n, seed=12)
+    st, _ = oracle.compress(a, oracle.EB_REL, 1e-3)
+    ea, s, r_ = oracle.resolve(oracle.EB_REL, 1e-3, a)
+    got, rc, raw = oracle.drc(st, local=b, flags=op, want_raw=True)
+    want_raw = fn(oracle.decompress(st), b).astype(f32)
+    assert np.array_equal(raw.view(np.uint32), want_raw.view(np.uint32))
+    assert np.array_equal(got, oracle.compress_core(want_raw, ea, s, r_)[0])
+
+
+@pytest.mark.parametrize("op,fn", [(oracle.OP_MAX, np.max), (oracle.OP_MIN, np.min)])
+@pytest.mark.parametrize("N", [2, 3, 8])
+def test_allreduce_max_min_lossless_on_grid_and_bound(op, fn, N):
+    # on the quantisation grid every compression is exact: the result is the exact element-wise extremum
+    eb, s = find_power_of_two_step_bound(-7)
+    n = 2 * 4096 + 33
+    send = fields.on_grid_ranks(N, n, float(s), seed=17)
+    got, rc = oracle.sim_allreduce(send, oracle.EB_ABS, eb, flags=op)
+    exact = fn(np.stack(send), axis=0)
+    for r in range(N):
+        assert np.array_equal(got[r], exact)
+    # off the grid: the extremum is 1-Lipschitz in each operand, so every compression on a chunk's path adds at most
+    # the bound (N-1 compressions before the owner's copy, one more for the copies the other ranks decompress)
+    send = [fields.smooth_1d(n, seed=200 + r) for r in range(N)]
+    got, rc = oracle.sim_allreduce(send, oracle.EB_REL, 1e-3, flags=op)
+    ea, _, _ = oracle.resolve(oracle.EB_REL, 1e-3, np.concatenate(send))
+    exact = fn(np.stack(send).astype(np.float64), axis=0)
+    for r in range(N):
+        assert np.max(np.abs(got[r].astype(np.float64) - exact)) <= N * float(ea)
+
+
+def test_allreduce_average_is_sum_over_n():
+    N, n = 8, 8 * 1000 + 5
+    send = [fields.smooth_1d(n, seed=300 + r) for r in range(N)]
+    s_, _ = oracle.sim_allreduce(send, oracle.EB_REL, 1e-3)
+    a_, _ = oracle.sim_allreduce(send, oracle.EB_REL, 1e-3, flags=oracle.OP_AVG)
+    for r in range(N):
+        assert np.array_equal(a_[r].view(np.uint32), (s_[r] / f32(N)).astype(f32).view(np.uint32))
+    # Corollary 2: the error of the average is the error of the sum divided by N
+    ea, _, _ = oracle.resolve(oracle.EB_REL, 1e-3, np.concatenate(send))
+    exact = np.mean(np.stack(send).astype(np.float64), axis=0)
+    assert np.max(np.abs(a_[0].astype(np.float64) - exact)) <= float(ea) * (1 + 1e-3)
+
+
+def test_max_error_variance_is_reported_against_theorem_2():
+    # Theorem 2 models the error of Max / Min over n ranks as N(0, (2 - (n+2)/2^n) sigma^2), sigma^2 the variance of
+    # one compression's error.  Measured on independent random inputs, reported with a loose check only: the model
+    # assumes that each comparison picks the compressed operand with probability 1/2.
+    N, n = 8, 8 * 8192
+    rng = np.random.default_rng(5)
+    send = [rng.normal(0, 1, n).astype(f32) for _ in range(N)]
+    eb = 1e-2
+    got, rc = oracle.sim_allreduce(send, oracle.EB_ABS, eb, flags=oracle.OP_MAX)
+    ea, s, _ = oracle.resolve(oracle.EB_ABS, eb)
+    exact = np.max(np.stack(send).astype(np.float64), axis=0)
+    var = float(np.var(got[0].astype(np.float64) - exact))
+    sigma2 = float(s) ** 2 / 12                       # uniform quantisation error of one compression
+    model = (2 - (N + 2) / 2 ** N) * sigma2
+    print(f"Max over {N} ranks: error variance {var:.3e}, one compression {sigma2:.3e}, Theorem 2 {model:.3e}")
+    assert 0.5 * sigma2 < var < 1.5 * N * sigma2
