@@ -55,6 +55,10 @@ enum { ZCCL_OK = 0,
 
 /* Flags of the reduce hop and of zccl_sim_allreduce. */
 enum { ZCCL_CONSISTENT_OWNER = 1u };  /* owner's copy of a reduced chunk = dequantised value, not the raw sum */
+/* Reduce operation of the collective computation framework (Section 3.2: Sum, Average, Max, Min), or-ed into `flags`.
+ * Max and Min keep the decoded operand when the two compare equal.  Average is a Sum on every hop; the Allreduce
+ * divides every rank's result by the number of ranks at the end (one fp32 division per element). */
+enum { ZCCL_OP_SUM = 0u, ZCCL_OP_MAX = 2u, ZCCL_OP_MIN = 4u, ZCCL_OP_AVG = 6u, ZCCL_OP_MASK = 6u };
 
 enum { ZCCL_TILE = 4096, ZCCL_BLOCK = 32, ZCCL_HEADER_BYTES = 32, ZCCL_MAX_RANKS = 64,
        ZCCL_NOALLOC_MAX_ELEMS = 1 << 26 };  /* element limit of zccl_compress_noalloc (256 MiB of fp32) */
@@ -134,6 +138,7 @@ int zccl_decompress(zccl_ctx* ctx, const void* in, size_t in_bytes_max,
  * One reduce-scatter hop of the collective computation framework (Section 3.1.2; error chain of Eq. 2):
  * out_c = compress( decompress(in_c) + local ), in one kernel, with no uncompressed intermediate in memory.
  * y_i = fl32( fl32(float(q_i) * s) + local_i ), the decoded operand on the left; bound and step are in_c's.
+ * With ZCCL_OP_MAX / ZCCL_OP_MIN in flags the addition becomes the larger / the smaller of the two operands.
  *   in_c [device]      received compressed chunk (at most in_bytes_max bytes are read)
  *   local [device]     this rank's uncompressed chunk, n floats (the paper's form), or NULL
  *   local_c [device]   instead of `local`: a second compressed chunk of the same n and step (at most

@@ -424,7 +424,20 @@ int zccl_sim_allreduce(zccl_ctx* c, const float* const* send, float* const* recv
             if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
         }
     }
-    return flush_decode(c, b, st);
+    if ((rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+    if ((flags & ZCCL_OP_MASK) == ZCCL_OP_AVG) {   // Average = Sum / N: one division per element of every rank's result
+        ScaleBatch sb{};
+        sb.n = n; sb.divisor = (float)N; sb.count = 0;
+        for (int r = 0; r < N; ++r) {
+            sb.y[sb.count++] = recv[r];
+            if (sb.count == kMaxJobs) {
+                if (launch_scale(sb, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
+                sb.count = 0;
+            }
+        }
+        if (launch_scale(sb, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
+    }
+    return ZCCL_OK;
 }
 
 int zccl_sim_allgather(zccl_ctx* c, const float* const* send, float* const* recv, int N,

@@ -105,6 +105,14 @@ struct ChainBatch {
     int N, hops, count;   // hops < 0: every chain follows its own path
 };
 
+// Average: every rank's result divided by the number of ranks (one fp32 division per element), grid.y = buffer.
+struct ScaleBatch {
+    float* y[kMaxJobs];
+    unsigned long long n;
+    float divisor;
+    int count;
+};
+
 struct RangeBatch {
     const float* x[kMaxJobs];
     unsigned long long n[kMaxJobs];
@@ -119,6 +127,7 @@ cudaError_t launch_resolve(int eb_mode, float eb, const Workspace& ws, cudaStrea
 cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& ws, bool device_params,
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st);
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
 // quality metrics: `partials` holds 4 doubles per CTA of the launch (at most kQualityCtas), `counter` one word that
 // is zero between launches

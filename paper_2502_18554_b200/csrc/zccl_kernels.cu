@@ -1376,6 +1376,13 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         const float* __restrict__ loc = job.x ? job.x + start : nullptr;
         float* __restrict__ yout = job.y ? job.y + start : nullptr;
         const bool deq = (job.flags & 1u) != 0;
+        // reduce operation (bits 1..2 of the flags): 0 = sum, 1 = max, 2 = min, 3 = average (a sum on every hop);
+        // of two operands that compare equal Max and Min keep the decoded one
+        const uint32_t op = (job.flags >> 1) & 3u;
+        const bool summing = op == 0u || op == 3u;
+        auto combine = [&](float a, float b) {
+            return op == 1u ? ((a < b) ? b : a) : op == 2u ? ((b < a) ? b : a) : __fadd_rn(a, b);
+        };
 
         // ---- front end: decode + add, leaving the sums in this warp's rows of ybuf (swizzled), row 0 = guard
         int mode = 2;   // 1: fp32 front end from the staged blob, 2: integer front end from global memory
@@ -1404,8 +1411,8 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 // the element before this warp's first one is the last element of the previous warp: its code is `base`
                 if (lane == 0) {
                     float yprev;
-                    if (warp == 0) yprev = __fadd_rn(__fmul_rn(__fadd_rn(v[0], base), s), __ldg(loc));
-                    else yprev = __fadd_rn(__fmul_rn(base, s), lprev);
+                    if (warp == 0) yprev = combine(__fmul_rn(__fadd_rn(v[0], base), s), __ldg(loc));
+                    else yprev = combine(__fmul_rn(base, s), lprev);
                     yrows[31 ^ 12] = yprev;   // guard row, element 31 under the swizzle of the row before row 0
                 }
                 const int sw = (lane >> 1) & 3;
@@ -1415,7 +1422,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 const bool lvec = (((uintptr_t)loc) & 15u) == 0;
                 const bool store = gout != nullptr && !deq;
                 const bool gvec = (((uintptr_t)yout) & 15u) == 0;
-                if (lvec && (!store || gvec)) {
+                if (summing && lvec && (!store || gvec)) {
                     float4 l[4];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) l[c] = __ldg(reinterpret_cast<const float4*>(lp) + c);
@@ -1434,10 +1441,10 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                     for (int c = 0; c < 4; ++c) {
                         float4 l, o;
                         l.x = __ldg(lp + 4 * c); l.y = __ldg(lp + 4 * c + 1); l.z = __ldg(lp + 4 * c + 2); l.w = __ldg(lp + 4 * c + 3);
-                        o.x = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), l.x);
-                        o.y = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), l.y);
-                        o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), l.z);
-                        o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), l.w);
+                        o.x = combine(__fmul_rn(__fadd_rn(v[4 * c + 0], base), s), l.x);
+                        o.y = combine(__fmul_rn(__fadd_rn(v[4 * c + 1], base), s), l.y);
+                        o.z = combine(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), l.z);
+                        o.w = combine(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), l.w);
                         row[c ^ sw] = o;
                         if (store) { float* g = reinterpret_cast<float*>(gout + c); g[0] = o.x; g[1] = o.y; g[2] = o.z; g[3] = o.w; }
                     }
@@ -1473,7 +1480,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                     if (!inside) e = last;
                     const float xa = __fmul_rn(__int2float_rn(base_a + qa[i]), s);
                     const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b + qb[i]), s) : __ldg(loc + e);
-                    const float yv = __fadd_rn(xa, xb);
+                    const float yv = combine(xa, xb);
                     yrows[32 * (i + 1) + (lane ^ ((i & 3) << 2))] = yv;
                     if (yout && !deq && inside) yout[e] = yv;
                 }
@@ -1485,7 +1492,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                         const uint32_t ep = min((uint32_t)(512 * warp - 1), last);
                         const float xa = __fmul_rn(__int2float_rn(base_a), s);
                         const float xb = job.in_c2 ? __fmul_rn(__int2float_rn(base_b), s) : __ldg(loc + ep);
-                        yprev = __fadd_rn(xa, xb);
+                        yprev = combine(xa, xb);
                     }
                     yrows[31 ^ 12] = yprev;
                 }
@@ -1631,6 +1638,15 @@ __global__ void __launch_bounds__(256) copy_chain_kernel(ChainBatch cb, Workspac
             if (h + 1 < hops) asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(d) : "memory");
         }
     }
+}
+
+// y = y / divisor, element by element (Average = Sum / N at the end of the Allreduce).
+__global__ void __launch_bounds__(256) scale_kernel(ScaleBatch sb)
+{
+    float* __restrict__ y = sb.y[blockIdx.y];
+    const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned long long nth = (unsigned long long)gridDim.x * blockDim.x;
+    for (unsigned long long i = tid; i < sb.n; i += nth) y[i] = __fdiv_rn(y[i], sb.divisor);
 }
 
 // ------------------------------------------------------------------------------------------------ quality metrics
@@ -1823,6 +1839,17 @@ cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, 
     unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
     ++g_launches;
     copy_kernel<<<dim3(gx ? gx : 1, cb.count), 256, 0, st>>>(cb, ws);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st)
+{
+    if (sb.count <= 0 || sb.n == 0) return cudaSuccess;
+    unsigned long long want = (sb.n + 255) / 256;
+    unsigned per = (unsigned)((sm_count * 8 + sb.count - 1) / sb.count);
+    unsigned gx = (unsigned)(want < per ? want : per);
+    ++g_launches;
+    scale_kernel<<<dim3(gx ? gx : 1, sb.count), 256, 0, st>>>(sb);
     return cudaGetLastError();
 }
 

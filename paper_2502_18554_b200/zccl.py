@@ -17,6 +17,7 @@ E_TOO_LARGE = -8
 NOALLOC_MAX_ELEMS = 1 << 26
 EB_ABS, EB_REL = 0, 1
 CONSISTENT_OWNER = 1
+OP_SUM, OP_MAX, OP_MIN, OP_AVG = 0, 2, 4, 6   # reduce operation, or-ed into flags
 TILE, BLOCK, HEADER_BYTES = 4096, 32, 32
 
 EXPORTS = [

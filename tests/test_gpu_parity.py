@@ -535,3 +535,33 @@ def test_quality_of_a_compressed_field(z, ctx):
     assert _quality(ctx, dx, dx)["psnr"] == math.inf
     want = oracle.quality(x, y.cpu().numpy())
     assert q["max_abs_err"] == want["max_abs_err"] and math.isclose(q["mse"], want["mse"], rel_tol=1e-9)
+
+
+@pytest.mark.parametrize("op", ["max", "min"])
+@pytest.mark.parametrize("n", [4096 * 3 + 50, 4096 * 40, 777])
+def test_fused_hop_max_min_matches_oracle(z, ctx, op, n):
+    zop, oop = (z.OP_MAX, oracle.OP_MAX) if op == "max" else (z.OP_MIN, oracle.OP_MIN)
+    a, b = fields.smooth_1d(n, seed=11), fields.smooth_1d(n, seed=12)
+    st, _ = oracle.compress(a, oracle.EB_REL, 1e-3)
+    want, wrc, wraw = oracle.drc(st, local=b, flags=oop, want_raw=True)
+    out = torch.empty(z.compress_bound(n), dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    raw = torch.empty(n, dtype=torch.float32, device="cuda")
+    ctx.decompress_reduce_compress(dev(st), n, out, nb, local=dev(b), raw_out=raw, flags=zop)
+    assert ctx.status() == wrc
+    assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+    assert_same_bits(raw.cpu().numpy(), wraw)
+
+
+@pytest.mark.parametrize("op", ["max", "min", "avg"])
+@pytest.mark.parametrize("N,n", [(3, 10_001), (8, 8 * 4096 * 2 + 5)])
+def test_allreduce_other_operations_match_oracle(z, ctx, op, N, n):
+    zop = dict(max=z.OP_MAX, min=z.OP_MIN, avg=z.OP_AVG)[op]
+    oop = dict(max=oracle.OP_MAX, min=oracle.OP_MIN, avg=oracle.OP_AVG)[op]
+    send = [fields.smooth_1d(n, seed=210 + r) for r in range(N)]
+    want, wrc, whop = oracle.sim_allreduce(send, oracle.EB_REL, 1e-3, flags=oop, want_hop_bytes=True)
+    got, rc, sizes = _run_allreduce(z, ctx, send, z.EB_REL, 1e-3, flags=zop)
+    assert rc == wrc
+    for r in range(N):
+        assert_same_bits(got[r], want[r])
+    assert np.array_equal(sizes.reshape(N, N), whop)
