@@ -565,3 +565,28 @@ def test_allreduce_other_operations_match_oracle(z, ctx, op, N, n):
     for r in range(N):
         assert_same_bits(got[r], want[r])
     assert np.array_equal(sizes.reshape(N, N), whop)
+
+
+def test_collectives_with_more_jobs_than_a_launch_holds(z):
+    # 12 ranks: 132 decode jobs per collective, more than the 64 chunk-operations one launch takes, so the batches are
+    # cut in the middle of a rank's chunks; tile counts per chunk differ (ragged last chunk)
+    N, n = 12, 12 * 3000 + 7
+    c = z.Context(1 << 20, N)
+    send = [fields.smooth_1d(n, seed=400 + r) for r in range(N)]
+    want, wrc, whop = oracle.sim_allreduce(send, oracle.EB_REL, 1e-3, want_hop_bytes=True)
+    d_send = [dev(a) for a in send]
+    d_recv = [torch.zeros_like(t) for t in d_send]
+    c.sim_allreduce(d_send, d_recv, z.EB_REL, 1e-3)
+    assert c.status() == wrc
+    for r in range(N):
+        assert_same_bits(d_recv[r].cpu().numpy(), want[r])
+    assert np.array_equal(np.array(c.sim_sizes()).reshape(N, N), whop)
+    m = 5000
+    send = [fields.smooth_1d(m, seed=500 + r) for r in range(N)]
+    want, wrc, wsizes = oracle.sim_allgather(send, oracle.EB_REL, 1e-3)
+    d_recv = [torch.zeros(N * m, dtype=torch.float32, device="cuda") for _ in range(N)]
+    c.sim_allgather([dev(a) for a in send], d_recv, z.EB_REL, 1e-3)
+    assert c.status() == wrc
+    for r in range(N):
+        assert_same_bits(d_recv[r].cpu().numpy(), want[r])
+    c.close()
