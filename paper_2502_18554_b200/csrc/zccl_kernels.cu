@@ -833,11 +833,12 @@ struct PlanShared {
     // what warp 0 worked out ahead of the barrier (laid_out != 0) and picks up again after it
     uint32_t laid_out, total, nT, lo, base;
 };
-// Hand-off of the scan's sizes from warps 1..7 to warp 0.
+// Hand-off of the scan's sizes from warps 2..7 to warp 0 (warp 1 requests the next tile's input meanwhile).
+constexpr int kScanFirstWarp = 2, kScanWarps = kWarps - kScanFirstWarp;
 struct ScanShared {
     uint32_t part[kWarps];    // sum of the sizes warp w fetched
     uint32_t ok[kWarps];      // 1 if every state that warp saw was published
-    alignas(8) unsigned long long scanbar;   // warps 1..7 arrive once their shares are written
+    alignas(8) unsigned long long scanbar;   // the scanning warps arrive once their shares are written
 };
 
 struct EncodeShared {
@@ -971,8 +972,8 @@ __device__ __forceinline__ uint32_t scan_begin(const Anchor& a, int job_index, c
     return a.job == job_index ? a.ticket + 1 : jb.job[job_index].tile_begin;
 }
 
-// Warps 1..7, while warp 0 publishes and lays out: each fetches its share of the sizes of tiles [lo, hi) (window k
-// of 32 tiles belongs to warp 1 + k mod 7, all loads of a warp in flight together), leaves the sum for warp 0 and
+// Warps 2..7, while warp 0 publishes and lays out: each fetches its share of the sizes of tiles [lo, hi) (window k
+// of 32 tiles belongs to warp 2 + k mod 6, all loads of a warp in flight together), leaves the sum for warp 0 and
 // arrives on the hand-off barrier.  One round trip to L2 for the whole scan.
 __device__ __forceinline__ void scan_share(ScanShared& plan, const Workspace& ws, uint32_t lo, uint32_t hi, uint32_t epoch,
                                            int warp, int lane)
@@ -982,7 +983,7 @@ __device__ __forceinline__ void scan_share(ScanShared& plan, const Workspace& ws
     if (hi > lo) {
         const uint32_t nwin = (hi - lo + 31u) >> 5;
 #pragma unroll 4
-        for (uint32_t w = (uint32_t)warp - 1u; w < nwin; w += kWarps - 1) {
+        for (uint32_t w = (uint32_t)(warp - kScanFirstWarp); w < nwin; w += kScanWarps) {
             const uint32_t at = lo + 32u * w + (uint32_t)lane;
             if (at < hi) {
                 const unsigned long long st = ld_state(ws.tile_state + at);
@@ -1062,8 +1063,8 @@ __device__ __forceinline__ Planned announce_and_plan(PlanShared& plan, ScanShare
     bool have = false;
     if (shared_scan) {
         if (!mbar_wait(&scan.scanbar, scan_parity)) status |= kStTimeout;
-        const uint32_t ps = (lane >= 1 && lane < kWarps) ? scan.part[lane] : 0u;
-        const uint32_t ok = (lane >= 1 && lane < kWarps) ? scan.ok[lane] : 1u;
+        const uint32_t ps = (lane >= kScanFirstWarp && lane < kWarps) ? scan.part[lane] : 0u;
+        const uint32_t ok = (lane >= kScanFirstWarp && lane < kWarps) ? scan.ok[lane] : 1u;
         between = __reduce_add_sync(kFull, ps);
         have = __all_sync(kFull, ok != 0u);
     }
@@ -1125,7 +1126,7 @@ __device__ __forceinline__ Planned plan_pending(PlanShared& plan, ScanShared& sc
     if (warp == 0) {
         pl = announce_and_plan(plan, scan, cur_words, cur_padw, ticket, have_cur, c, pend_words, anchor, c.valid, scan_parity, jb, ws,
                                epoch, lane, status);
-    } else if (c.valid) {
+    } else if (c.valid && warp >= kScanFirstWarp) {
         scan_share(scan, ws, scan_begin(anchor, c.job, jb), c.ticket, epoch, warp, lane);
     }
     if (c.valid) {
@@ -1170,7 +1171,7 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
     };
     if (tid == 0) {
         mbar_init(&sh.bar, 1);
-        mbar_init(&sh.scan.scanbar, kWarps - 1);
+        mbar_init(&sh.scan.scanbar, kScanWarps);
         sh.plan[0].laid_out = 0u; sh.plan[1].laid_out = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         take_next();
@@ -1308,7 +1309,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     if (tid == 0) {
         mbar_init(&sh.bar[0], 1);
         mbar_init(&sh.bar[1], 1);
-        mbar_init(&sh.scan.scanbar, kWarps - 1);
+        mbar_init(&sh.scan.scanbar, kScanWarps);
         sh.plan[0].laid_out = 0u; sh.plan[1].laid_out = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
