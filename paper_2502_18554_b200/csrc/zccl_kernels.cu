@@ -426,7 +426,9 @@ __device__ __forceinline__ void decode_blocks_f32(const uint2* __restrict__ tbl,
 // Reads this thread's 16 consecutive deltas (elements 16*lane .. 16*lane+15 of the warp's 512) from `wbuf`,
 // forms their running sum and the warp-wide exclusive prefix.  On return v[k] = sum of the warp's deltas up to
 // and including this thread's element k; the return value is the warp's total.
-__device__ __forceinline__ float decode_scan_f32(const float* __restrict__ wbuf, int lane, float (&v)[16])
+// `excl` receives the sum of the warp's deltas before this thread's first element: v[k] is then only the running sum
+// inside the thread, and the caller adds excl (plus whatever comes before the warp) once, in one addition per element.
+__device__ __forceinline__ float decode_scan_f32(const float* __restrict__ wbuf, int lane, float (&v)[16], float& excl)
 {
     const int sw = (lane >> 1) & 3;
     const float4* row = reinterpret_cast<const float4*>(wbuf + 16 * lane);
@@ -444,11 +446,8 @@ __device__ __forceinline__ float decode_scan_f32(const float* __restrict__ wbuf,
         const float t = __shfl_up_sync(kFull, incl, s);
         if (lane >= s) incl = __fadd_rn(incl, t);
     }
-    const float excl = __fsub_rn(incl, run);
-    const float total = __shfl_sync(kFull, incl, 31);
-#pragma unroll
-    for (int k = 0; k < 16; ++k) v[k] = __fadd_rn(v[k], excl);
-    return total;
+    excl = __fsub_rn(incl, run);
+    return __shfl_sync(kFull, incl, 31);
 }
 
 // Where a tile's blob is, as known from the index alone (no access to the blob itself).
@@ -630,12 +629,14 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
                 decode_blocks_f32(sh.tbl + kBlocksPerWarp * warp, sh.wbuf[warp], lane, xp);
                 __syncwarp();
                 float v[16];
-                const float total = decode_scan_f32(sh.wbuf[warp], lane, v);
+                float before;
+                const float total = decode_scan_f32(sh.wbuf[warp], lane, v, before);
                 if (lane == 0) sh.warp_total[par][warp] = total;
                 const float outlier = (float)(int32_t)sb[0];
                 __syncthreads();
                 float base = outlier;
                 for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[par][w]);
+                base = __fadd_rn(base, before);   // all of these are integers below 2^24: any order of addition is exact
                 par ^= 1u;
                 float4* dst = reinterpret_cast<float4*>(y + 512 * warp + 16 * lane);
                 const bool vec = (((uintptr_t)dst) & 15u) == 0;
@@ -1403,7 +1404,8 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 // lane 0 needs the local operand's element before the warp's first one after the barrier below
                 const float lprev = (lane == 0 && warp != 0) ? __ldg(loc + 512 * warp - 1) : 0.0f;
                 float v[16];
-                const float total = decode_scan_f32(yrows + 32, lane, v);
+                float before;
+                const float total = decode_scan_f32(yrows + 32, lane, v, before);
                 if (lane == 0) sh.warp_total[warp] = total;
                 const float outlier = (float)(int32_t)sb[0];
                 __syncthreads();   // warp totals
@@ -1416,6 +1418,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                     else yprev = combine(__fmul_rn(base, s), lprev);
                     yrows[31 ^ 12] = yprev;   // guard row, element 31 under the swizzle of the row before row 0
                 }
+                base = __fadd_rn(base, before);   // integers below 2^24: any order of addition is exact
                 const int sw = (lane >> 1) & 3;
                 float4* row = reinterpret_cast<float4*>(yrows + 32 + 16 * lane);
                 float4* gout = yout ? reinterpret_cast<float4*>(yout + 512 * warp + 16 * lane) : nullptr;
