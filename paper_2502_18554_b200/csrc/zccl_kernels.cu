@@ -17,11 +17,12 @@
 //   * the encoder appends each block's words to its warp's region of shared memory in a single pass over the
 //     block; the decoder undoes the Lorenzo recurrence by a warp-local transposition through shared memory
 //     (16 consecutive elements per thread) instead of shuffle scans.
-// Tiles are dealt round-robin to a grid that fits the device (CTA c takes tiles c, c + G, ...), so all CTAs move
-// through the stream in step and the next tile is known in advance.  Placement (prefix sum of tile sizes) is
-// anchored at a CTA's own previous tile and deferred by one tile, so it only ever sums sizes that are already
-// published; warp 0 plans a placement once for the CTA (scan, layout, capacity check, index entry), warp 1 requests
-// the next tile meanwhile, and after one barrier every warp copies its own share.  The scan relies on the grid
+// The grid fits the device.  Decoder and fused hop deal tiles round-robin (CTA c takes tiles c, c + G, ...), so the
+// next tiles are known in advance; the encoder hands them out in order through a device-wide counter, one tile
+// ahead, so that a CTA which gets fewer issue slots takes fewer tiles.  Placement (prefix sum of tile sizes) is
+// anchored at the tile a CTA placed last and deferred by one tile, so it only ever sums sizes that are already
+// published; warp 0 plans a placement once for the CTA (layout, capacity check, index entry), warps 2..7 fetch the
+// sizes for it, warp 1 requests the next tile meanwhile, and after one barrier every warp copies its own share.  The scan relies on the grid
 // being resident at once; every wait is bounded and reports through the status word instead of hanging if it is
 // not.
 #include "zccl_internal.h"
@@ -1114,7 +1115,7 @@ __device__ __forceinline__ void copy_planned(const PlanShared& plan, const Pendi
 }
 
 // First half of the placement of a pending tile, by the whole CTA, after the barrier that made the current tile's
-// sizes visible (have_cur) or at the end of the launch: warps 1..7 fetch the scan's sizes while warp 0 publishes
+// sizes visible (have_cur) or at the end of the launch: warps 2..7 fetch the scan's sizes while warp 0 publishes
 // and lays out, then warp 0 completes the plan.  The caller follows with a barrier, copy_planned by every warp and
 // finish_plan by warp 0.  Uniform over the CTA.
 __device__ __forceinline__ Planned plan_pending(PlanShared& plan, ScanShared& scan, const uint32_t* cur_words, uint32_t cur_padw,
