@@ -590,3 +590,52 @@ def test_collectives_with_more_jobs_than_a_launch_holds(z):
     for r in range(N):
         assert_same_bits(d_recv[r].cpu().numpy(), want[r])
     c.close()
+
+
+def test_step_replayed_from_a_cuda_graph(z):
+    # every entry point only enqueues work on its stream, so a whole step (relative-bound compress with its range
+    # pass, decompress, fused hop, ring Allreduce) can be captured once and replayed: same bytes as the oracle
+    c = z.Context(1 << 20, 4)
+    n, N = 4 * 4096 * 3 + 40, 4
+    x, loc = fields.smooth_1d(n, seed=61), fields.smooth_1d(n, seed=62)
+    send = [fields.smooth_1d(n, seed=63 + r) for r in range(N)]
+    dx, dl = dev(x), dev(loc)
+    d_send = [dev(a) for a in send]
+    d_recv = [torch.zeros_like(t) for t in d_send]
+    cap = z.compress_bound(n)
+    out = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    out2 = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    nb2 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    y = torch.zeros(n, dtype=torch.float32, device="cuda")
+
+    def step():
+        c.compress(dx, z.EB_REL, 1e-3, out, nb)
+        c.decompress(out, y)
+        c.decompress_reduce_compress(out, n, out2, nb2, local=dl)
+        c.sim_allreduce(d_send, d_recv, z.EB_REL, 1e-3)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                   # first calls set kernel attributes: outside the capture
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            step()
+    torch.cuda.synchronize()
+    want, wrc = oracle.compress(x, oracle.EB_REL, 1e-3)
+    want2, _ = oracle.drc(want, local=loc)
+    want3, _ = oracle.sim_allreduce(send, oracle.EB_REL, 1e-3)
+    for _ in range(3):
+        for t in (out, out2, y, nb, nb2, *d_recv):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert c.status() == wrc
+        assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+        assert_same_bits(y.cpu().numpy(), oracle.decompress(want))
+        assert np.array_equal(out2[: int(nb2.item())].cpu().numpy(), want2)
+        for r in range(N):
+            assert_same_bits(d_recv[r].cpu().numpy(), want3[r])
+    c.close()
