@@ -486,12 +486,17 @@ struct StagePipe {
         if (t >= jb.total_tiles) return;
         const int jj = find_job(jb, t);
         const Job& jq = jb.job[jj];
-        const StreamInfo hq = (jj == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
         const uint32_t tl = t - jq.tile_begin;
-        if (!hq.ok || hq.n > jq.n || tl >= hq.nT) return;
+        // the index entries do not depend on the header's contents, only on their being inside the readable bytes:
+        // ask for them first, so that they travel together with the header instead of after it
         const uint32_t* idx = jq.in_c + kHeaderWords;
-        n_end = ldg_u32(idx + tl);
-        n_beg = tl ? ldg_u32(idx + tl - 1) : 0u;
+        const bool inside = ((unsigned long long)kHeaderWords + tl + 1ull) * 4ull <= jq.in_cap;
+        const uint32_t e_end = inside ? ldg_u32(idx + tl) : 0u;
+        const uint32_t e_beg = (inside && tl) ? ldg_u32(idx + tl - 1) : 0u;
+        const StreamInfo hq = (jj == cur_job) ? h : read_header(jq.in_c, jq.in_cap);
+        if (!hq.ok || hq.n > jq.n || tl >= hq.nT) return;   // a valid header guarantees that the whole index is readable
+        n_end = e_end;
+        n_beg = e_beg;
         n_job = jj;
     }
     // request the blob of tile t (whose entries were fetched before) into staging buffer `buf`
