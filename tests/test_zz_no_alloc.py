@@ -66,3 +66,32 @@ def test_noalloc_rejects_what_it_cannot_place(z):
     assert z.compress_noalloc(y, 1e-4, big, nbytes) == z.OK
     torch.cuda.synchronize()
     assert int(nbytes.item()) > 32
+
+
+def test_noalloc_inside_a_captured_graph(z):
+    # the case the entry point exists for: after one call outside any capture (which resolves the array's address),
+    # a call is captured into a CUDA graph and replayed; every replay produces the context entry point's bytes
+    ctx = z.Context(1 << 20, 0)
+    x = fields.smooth_1d(150_000 + 5, seed=15)
+    eb = 1e-3
+    dx = torch.from_numpy(x).cuda()
+    want = _reference_stream(z, ctx, dx, eb)
+    cap = z.compress_bound(x.size)
+    out = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    nbytes = torch.zeros(1, dtype=torch.int64, device="cuda")
+    assert z.compress_noalloc(dx, eb, out, nbytes) == z.OK          # first call: outside the capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            assert z.compress_noalloc(dx, eb, out, nbytes) == z.OK
+    torch.cuda.synchronize()
+    for _ in range(3):
+        out.zero_()
+        nbytes.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(out[: int(nbytes.item())].cpu().numpy(), want)
+    ctx.close()
