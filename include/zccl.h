@@ -255,6 +255,20 @@ int zccl_sim_sizes(zccl_ctx* ctx, size_t* sizes, int capacity, void* stream);
 int zccl_quality(zccl_ctx* ctx, const float* x, const float* y, size_t n, double* out, void* stream);
 
 /*
+ * The two per-rank steps of a real ring that are not a codec call (Section 3.2: the error bound is resolved once
+ * per collective, over the data of all ranks; Corollary 2: Average = Sum / N).
+ *   zccl_range: minmax [device, 2 floats] <- (min, max) of x [device, n floats]; (+inf, -inf) when n == 0.  A
+ *               rank combines these with its peers' (min of minima, max of maxima), forms
+ *               eb_abs = fl32(eb * fl32(max - min)) and passes it to the codec calls as ZCCL_EB_ABS; that is the
+ *               bound a ZCCL_EB_REL call over the concatenated data would resolve.
+ *   zccl_scale: y [device, n floats] <- y / divisor, one IEEE fp32 division per element.
+ * Both enqueue on `stream` and return at once.  ZCCL_E_ARG for null or misaligned pointers, n beyond the
+ * context's max_elems (range), a divisor that is not a positive finite number (scale).
+ */
+int zccl_range(zccl_ctx* ctx, const float* x, size_t n, float* minmax, void* stream);
+int zccl_scale(zccl_ctx* ctx, float* y, size_t n, float divisor, void* stream);
+
+/*
  * Host-buffer convenience forms: copy the input from host memory into a staging area of the context, run the
  * device path, copy the result back, all enqueued on `stream` (pinned host memory makes the copies asynchronous).
  * They exist so that end-to-end cost including PCIe transfers can be measured through this boundary.

@@ -660,6 +660,28 @@ int zccl_quality(zccl_ctx* c, const float* x, const float* y, size_t n, double* 
     return cuda_rc(launch_quality(x, y, n, out, c->quality_partials, c->quality_counter, c->sm_count, (cudaStream_t)stream));
 }
 
+int zccl_range(zccl_ctx* c, const float* x, size_t n, float* minmax, void* stream)
+{
+    if (!c || (!x && n) || !minmax || n > c->max_elems) return ZCCL_E_ARG;
+    if (((uintptr_t)x & 3u) || ((uintptr_t)minmax & 3u)) return ZCCL_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n) {
+        RangeBatch rb{};
+        rb.x[0] = x; rb.n[0] = n; rb.count = 1;
+        if (launch_range(rb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
+    }
+    return cuda_rc(launch_export_range(c->ws, minmax, st));
+}
+
+int zccl_scale(zccl_ctx* c, float* y, size_t n, float divisor, void* stream)
+{
+    if (!c || (!y && n) || ((uintptr_t)y & 3u) || !(divisor > 0.0f) || !std::isfinite(divisor)) return ZCCL_E_ARG;
+    if (n == 0) return ZCCL_OK;
+    ScaleBatch sb{};
+    sb.y[0] = y; sb.n = n; sb.divisor = divisor; sb.count = 1;
+    return cuda_rc(launch_scale(sb, c->sm_count, (cudaStream_t)stream));
+}
+
 int zccl_sim_sizes(zccl_ctx* c, size_t* sizes, int capacity, void* stream)
 {
     if (!c || !sizes || capacity < 0) return ZCCL_E_ARG;

@@ -124,6 +124,7 @@ enum EncodeMode { kEncodeRaw = 0, kEncodeFused = 1 };
 // Launchers (defined next to the kernels).
 cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_resolve(int eb_mode, float eb, const Workspace& ws, cudaStream_t st);
+cudaError_t launch_export_range(const Workspace& ws, float* out, cudaStream_t st);
 cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& ws, bool device_params,
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);

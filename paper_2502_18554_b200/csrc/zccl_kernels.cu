@@ -249,6 +249,20 @@ __global__ void resolve_kernel(int eb_mode, float eb, Workspace ws)
     if (!p.valid) atomicOr(ws.status, kStDegenerate);
 }
 
+// Hands the minimum and maximum collected by range_kernel to the caller (out[0] = min, out[1] = max; +inf, -inf
+// when nothing was scanned) and re-arms the keys.  A rank of a real ring combines these with its peers' before it
+// resolves the bound (Section 3.2: one bound per collective).
+__global__ void export_range_kernel(Workspace ws, float* out)
+{
+    if (threadIdx.x || blockIdx.x) return;
+    const uint32_t kmin = ws.minmax[0], kmax = ws.minmax[1];
+    const bool any = kmin <= kmax;
+    out[0] = any ? key2f(kmin) : __int_as_float(0x7F800000);
+    out[1] = any ? key2f(kmax) : __int_as_float(0xFF800000);
+    ws.minmax[0] = 0xFFFFFFFFu;
+    ws.minmax[1] = 0u;
+}
+
 // ------------------------------------------------------------------------------------------------ stream header
 
 struct StreamInfo {
@@ -1798,6 +1812,13 @@ cudaError_t launch_resolve(int eb_mode, float eb, const Workspace& ws, cudaStrea
 {
     ++g_launches;
     resolve_kernel<<<1, 32, 0, st>>>(eb_mode, eb, ws);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_export_range(const Workspace& ws, float* out, cudaStream_t st)
+{
+    ++g_launches;
+    export_range_kernel<<<1, 32, 0, st>>>(ws, out);
     return cudaGetLastError();
 }
 

@@ -639,3 +639,26 @@ def test_step_replayed_from_a_cuda_graph(z):
         for r in range(N):
             assert_same_bits(d_recv[r].cpu().numpy(), want3[r])
     c.close()
+
+
+def test_range_and_scale_steps_of_a_real_rank(z, ctx):
+    """zccl_range against numpy's min and max (any order of comparisons gives the same two values) and zccl_scale
+    against one fp32 division per element."""
+    for n in (1, 5, 4097, 1_000_003):
+        a = fields.smooth_1d(n, seed=n % 97)
+        x = dev(a)
+        mm = torch.zeros(2, dtype=torch.float32, device="cuda")
+        ctx.range(x, mm)
+        got = mm.cpu().numpy()
+        assert got[0] == a.min() and got[1] == a.max()
+        y = x.clone()
+        ctx.scale(y, 7.0)
+        np.testing.assert_array_equal(y.cpu().numpy(), a / np.float32(7.0))
+    mm = torch.zeros(2, dtype=torch.float32, device="cuda")
+    ctx.range(torch.zeros(0, dtype=torch.float32, device="cuda"), mm)
+    assert mm.cpu().numpy().tolist() == [np.inf, -np.inf]
+    # the keys are re-armed: a second call sees only its own data
+    ctx.range(torch.full((10,), 3.0, device="cuda"), mm)
+    assert mm.cpu().numpy().tolist() == [3.0, 3.0]
+    with pytest.raises(z.ZcclError):
+        ctx.scale(torch.ones(4, device="cuda"), 0.0)

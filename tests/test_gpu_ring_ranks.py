@@ -1,0 +1,102 @@
+"""The real-rank collectives with the CUDA codec: several processes share the one GPU of the test box, each with its
+own context, and exchange the compressed streams through host memory (gloo), so no kernel of one rank ever waits
+for another rank's.  Every rank's result must equal, bit for bit, what the oracle's emulated ring computes for it
+(Sections 3.1.1, 3.1.2, 3.2)."""
+import os
+import sys
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = Path(__file__).resolve().parent.parent
+pytestmark = pytest.mark.gpu
+
+
+def _inputs(world, n):
+    from paper_2502_18554_b200 import fields
+    return [fields.smooth_1d(n, seed=60 + r) * np.float32(1 + 0.5 * r) for r in range(world)]
+
+
+def _worker(rank, world, port, n, segments, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, str(ROOT))
+    try:
+        from paper_2502_18554_b200 import ring, zccl as z
+        torch.cuda.set_device(0)
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+        dev = torch.device("cuda:0")
+        xs = _inputs(world, n)
+        x = torch.from_numpy(xs[rank].copy()).to(dev)
+        R = ring.Ring(n * world, segments=segments)
+        assert isinstance(R.codec, ring.DeviceCodec)
+        res = {}
+        out = torch.zeros(n, device=dev)
+        R.allreduce(x, out, z.EB_REL, 1e-3)
+        res["allreduce"] = out.cpu().numpy()
+        out = torch.zeros(n, device=dev)
+        R.allreduce(x, out, z.EB_ABS, 2e-3, flags=z.OP_AVG)
+        res["allreduce_avg"] = out.cpu().numpy()
+        out = torch.zeros(n, device=dev)
+        R.allreduce(x, out, z.EB_REL, 1e-3, flags=z.OP_MAX)
+        res["allreduce_max"] = out.cpu().numpy()
+        out = torch.zeros(ring.chunk_span(n, world, rank)[1], device=dev)
+        R.reduce_scatter(x, out, z.EB_REL, 1e-3)
+        res["reduce_scatter"] = out.cpu().numpy()
+        out = torch.zeros(world * n, device=dev)
+        R.allgather(x, out, z.EB_REL, 1e-2)
+        res["allgather"] = out.cpu().numpy()
+        xb = x.clone() if rank == 0 else torch.zeros(n, device=dev)
+        R.bcast(xb, 0, z.EB_REL, 1e-4)
+        res["bcast"] = xb.cpu().numpy()
+        res["launches"] = z.launch_count()
+        q.put((rank, res, None))
+        dist.barrier()
+        dist.destroy_process_group()
+    except Exception as e:
+        import traceback
+        q.put((rank, None, traceback.format_exc()))
+        raise e
+
+
+def _run(world, n, segments):
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29650 + (os.getpid() * 3 + world * 17 + segments) % 300
+    procs = [ctx.Process(target=_worker, args=(r, world, port, n, segments, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = {}
+    for _ in range(world):
+        rank, res, err = q.get(timeout=600)
+        assert err is None, err
+        got[rank] = res
+    for p in procs:
+        p.join(120)
+        assert p.exitcode == 0
+    return got
+
+
+@pytest.mark.parametrize("world,n,segments", [(2, 100000, 1), (3, 70001, 2), (4, 5, 1)])
+def test_cuda_ranks_match_the_oracle_ring(world, n, segments):
+    import oracle
+    got = _run(world, n, segments)
+    xs = _inputs(world, n)
+    for key, mode, eb, flags in (("allreduce", oracle.EB_REL, 1e-3, 0), ("allreduce_avg", oracle.EB_ABS, 2e-3, oracle.OP_AVG),
+                                 ("allreduce_max", oracle.EB_REL, 1e-3, oracle.OP_MAX)):
+        exp, _ = oracle.sim_allreduce(xs, mode, eb, flags=flags)
+        for r in range(world):
+            np.testing.assert_array_equal(got[r][key], exp[r], err_msg=f"{key} rank {r}")
+    exp, _, _ = oracle.sim_reduce_scatter(xs, oracle.EB_REL, 1e-3)
+    for r in range(world):
+        np.testing.assert_array_equal(got[r]["reduce_scatter"], exp[r])
+    exp, _, _ = oracle.sim_allgather(xs, oracle.EB_REL, 1e-2)
+    for r in range(world):
+        np.testing.assert_array_equal(got[r]["allgather"], exp[r])
+    exp, _, _ = oracle.sim_bcast(xs[0], world - 1, oracle.EB_REL, 1e-4)
+    for r in range(world):
+        np.testing.assert_array_equal(got[r]["bcast"], xs[0] if r == 0 else exp[0])
+    assert all(got[r]["launches"] > 0 for r in range(world))      # the CUDA path ran in every rank
