@@ -87,28 +87,51 @@ class DeviceCodec:
         return self.ctx.check()
 
 
+class _Msg:
+    """The outstanding work of one posted group.  With NCCL a wait makes the current stream wait, and two streams
+    may each have to (the codec's and the one messages are issued from); elsewhere a wait blocks the host and is
+    taken once."""
+
+    def __init__(self, works, stream_side: bool):
+        self.works, self.stream_side, self.done = works, stream_side, False
+
+    def wait(self):
+        if self.stream_side or not self.done:
+            for w in self.works:
+                w.wait()
+            self.done = True
+
+
 class _Link:
     """Point-to-point transport inside one process group.  NCCL moves device memory; any other backend is given
     the bytes in host memory."""
 
-    def __init__(self, group, device: torch.device):
+    def __init__(self, group, device: torch.device, transport: str = "auto"):
         self.group = group
         self.rank = dist.get_rank(group)
         self.N = dist.get_world_size(group)
-        self.direct = dist.get_backend(group) == "nccl"
-        if self.direct and device.type != "cuda":
-            raise ValueError("an NCCL group needs a codec on a CUDA device")
+        nccl = dist.get_backend(group) == "nccl"
+        if transport not in ("auto", "direct", "host"):
+            raise ValueError("transport must be auto, direct or host")
+        # direct: the backend is handed the codec's own buffers and payloads stay in flight while the codec works;
+        # host: payloads are copied to host memory and each message is waited for.  NCCL needs direct, a backend
+        # that moves host memory only can be direct when the codec's buffers are host memory too.
+        self.direct = nccl or transport == "direct" if transport != "host" else False
+        if nccl and (device.type != "cuda" or transport == "host"):
+            raise ValueError("an NCCL group needs the direct transport and a codec on a CUDA device")
+        if self.direct and not nccl and device.type != "cpu":
+            raise ValueError("this backend moves host memory only: use transport='host'")
         self.msg_device = device if self.direct else torch.device("cpu")
         # messages are issued from a stream of their own, so that a send waits for the piece it carries (the host
         # has seen that piece's event) and not for whatever else the codec stream has queued behind it
-        self.comm_stream = torch.cuda.Stream(device) if self.direct else None
+        self.comm_stream = torch.cuda.Stream(device) if nccl else None
 
     def peer(self, r: int) -> int:
         r %= self.N
         return dist.get_global_rank(self.group, r) if self.group is not None else r
 
     def issuing(self):
-        return torch.cuda.stream(self.comm_stream) if self.direct else contextlib.nullcontext()
+        return torch.cuda.stream(self.comm_stream) if self.comm_stream is not None else contextlib.nullcontext()
 
     def post(self, send, dst, recv, src):
         """One send (to dst) and one receive (from src) as a single group, either of which may be absent: a ring
@@ -118,7 +141,7 @@ class _Link:
             ops.append(dist.P2POp(dist.isend, send, self.peer(dst), self.group))
         if src is not None:
             ops.append(dist.P2POp(dist.irecv, recv, self.peer(src), self.group))
-        return dist.batch_isend_irecv(ops) if ops else []
+        return [_Msg(dist.batch_isend_irecv(ops), self.comm_stream is not None)] if ops else []
 
     @staticmethod
     def wait(reqs):
@@ -161,13 +184,14 @@ class Ring:
 
     max_elems: largest array a collective will be given (sizes the codec's workspace).
     group:     process group (default: the world); its backend decides the transport.
-    segments:  pieces per ring chunk (see the module text)."""
+    segments:  pieces per ring chunk (see the module text).
+    transport: "auto" (direct for NCCL, through host memory otherwise), "direct" or "host"."""
 
-    def __init__(self, max_elems: int, group=None, codec=None, segments: int = 1):
+    def __init__(self, max_elems: int, group=None, codec=None, segments: int = 1, transport: str = "auto"):
         if segments < 1:
             raise ValueError("segments must be at least 1")
         self.codec = codec if codec is not None else DeviceCodec(max_elems)
-        self.link = _Link(group, self.codec.device)
+        self.link = _Link(group, self.codec.device, transport)
         self.rank, self.N = self.link.rank, self.link.N
         self.S = segments
         self.max_elems = max_elems

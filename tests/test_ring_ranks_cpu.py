@@ -61,7 +61,7 @@ def _inputs(world, n):
     return [fields.smooth_1d(n, seed=40 + r) * np.float32(1 + r) for r in range(world)]
 
 
-def _worker(rank, world, port, n, segments, q):
+def _worker(rank, world, port, n, segments, transport, q):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     sys.path.insert(0, str(ROOT))
     try:
@@ -70,7 +70,7 @@ def _worker(rank, world, port, n, segments, q):
         dist.init_process_group("gloo", rank=rank, world_size=world)
         xs = _inputs(world, n)
         x = torch.from_numpy(xs[rank].copy())
-        R = ring.Ring(n * world, codec=HostCodec(), segments=segments)
+        R = ring.Ring(n * world, codec=HostCodec(), segments=segments, transport=transport)
         res = {}
         out = torch.zeros(n)
         R.allreduce(x, out, z.EB_REL, 1e-3)
@@ -97,11 +97,11 @@ def _worker(rank, world, port, n, segments, q):
         raise e
 
 
-def _run(world, n, segments):
+def _run(world, n, segments, transport):
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    port = 29700 + (os.getpid() * 7 + world * 13 + segments) % 900
-    procs = [ctx.Process(target=_worker, args=(r, world, port, n, segments, q)) for r in range(world)]
+    port = 29700 + (os.getpid() * 7 + world * 13 + segments * 3 + len(transport)) % 900
+    procs = [ctx.Process(target=_worker, args=(r, world, port, n, segments, transport, q)) for r in range(world)]
     for p in procs:
         p.start()
     got = {}
@@ -115,11 +115,14 @@ def _run(world, n, segments):
     return got
 
 
-@pytest.mark.parametrize("world,n,segments", [(2, 20000, 1), (3, 20000, 2), (4, 9001, 3), (3, 2, 1)])
-def test_real_rank_collectives_match_the_emulated_ones(world, n, segments):
+@pytest.mark.parametrize("world,n,segments,transport", [(2, 20000, 1, "host"), (3, 20000, 2, "host"), (4, 9001, 3, "direct"),
+                                                       (3, 2, 1, "host"), (2, 30000, 2, "direct"), (3, 20000, 1, "direct")])
+def test_real_rank_collectives_match_the_emulated_ones(world, n, segments, transport):
+    """"direct" keeps the payload messages in flight behind the codec steps and waits for each where its data is
+    needed (the bookkeeping an NCCL group runs with); "host" waits for every message where it is posted."""
     import oracle
     from paper_2502_18554_b200 import ring, zccl as z
-    got = _run(world, n, segments)
+    got = _run(world, n, segments, transport)
     xs = _inputs(world, n)
 
     exp, _ = oracle.sim_allreduce(xs, oracle.EB_REL, 1e-3)
