@@ -170,6 +170,178 @@ def reference_arm(args):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------------------------- per-config table
+
+L2_BYTES = 126 << 20
+
+
+def _timed(fn, sets: int, warmup: int = 10, iters: int = 10):
+    """Mean and best device time (us) of one call fn(set index), over `iters` timed replays after `warmup`.  One
+    replay is a CUDA graph of `sets` calls, one per buffer set, so that the device never waits for the host between
+    calls (the entry points only enqueue); its time is divided by `sets`."""
+    import torch
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(sets):
+            fn(i)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(sets):
+            fn(i)
+    for _ in range(warmup):
+        g.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(iters):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3 / sets)
+    return statistics.mean(ts), min(ts)
+
+
+def _codec_row(z, ctx, name, x_h, mode, eb, with_oracle: bool, loc_h=None):
+    """Compress and decompress (and, with loc_h, the fused hop) of one array: time, GB/s of uncompressed bytes,
+    ratio; inputs and outputs rotate over enough copies to exceed L2 several times (arrays of 256 MiB and more are
+    used in place)."""
+    import torch
+    n = x_h.size
+    nbytes = 4 * n
+    sets = 1 if nbytes >= (256 << 20) else max(2, min(32, -(-4 * L2_BYTES // max(3 * nbytes // 2, 1))))
+    cap = z.compress_bound(n)
+    xs = [torch.from_numpy(x_h).cuda() for _ in range(sets)]
+    outs = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    ys = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(sets)]
+    sz = torch.zeros(1, dtype=torch.int64, device="cuda")
+    c_mean, c_best = _timed(lambda i: ctx.compress(xs[i], mode, eb, outs[i], sz), sets)
+    rc = ctx.check()
+    cbytes = int(sz.item())
+    d_mean, d_best = _timed(lambda i: ctx.decompress(outs[i][:cbytes], ys[i]), sets)
+    ctx.check()
+    err = float((ys[0].double() - xs[0].double()).abs().max().item())
+    row = {"config": name, "n": n, "bytes": nbytes, "bound": ("REL " if mode == z.EB_REL else "ABS ") + f"{eb:g}",
+           "ratio": round(nbytes / cbytes, 3), "status": rc, "max_abs_err": err, "buffer_sets": sets,
+           "compress_us_mean": round(c_mean, 2), "compress_us_best": round(c_best, 2),
+           "compress_gbs": round(nbytes / c_mean / 1e3, 1),
+           "decompress_us_mean": round(d_mean, 2), "decompress_us_best": round(d_best, 2),
+           "decompress_gbs": round(nbytes / d_mean / 1e3, 1)}
+    if loc_h is not None:
+        locs = [torch.from_numpy(loc_h).cuda() for _ in range(sets)]
+        fouts = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+        f_mean, f_best = _timed(lambda i: ctx.decompress_reduce_compress(outs[i][:cbytes], n, fouts[i], sz,
+                                                                         local=locs[i]), sets)
+        ctx.check()
+        row.update({"fused_us_mean": round(f_mean, 2), "fused_us_best": round(f_best, 2),
+                    "fused_gbs": round(nbytes / f_mean / 1e3, 1), "fused_out_ratio": round(nbytes / int(sz.item()), 3)})
+        del locs, fouts
+    if with_oracle:
+        import oracle
+        best_c = best_d = float("inf")
+        for _ in range(1 if nbytes >= (1 << 30) else 3):
+            t0 = time.perf_counter()
+            st, _ = oracle.compress(x_h, oracle.EB_REL if mode == z.EB_REL else oracle.EB_ABS, eb)
+            t1 = time.perf_counter()
+            oracle.decompress(st)
+            t2 = time.perf_counter()
+            best_c, best_d = min(best_c, t1 - t0), min(best_d, t2 - t1)
+        row["oracle_compress_gbs"] = round(nbytes / best_c / 1e9, 3)
+        row["oracle_decompress_gbs"] = round(nbytes / best_d / 1e9, 3)
+        row["oracle_threads"] = 1
+    del xs, outs, ys
+    torch.cuda.empty_cache()
+    return row
+
+
+def config_table(args):
+    """Timings of the survey's configurations 0-4 (10 warm-up + 10 timed calls each, mean and best): one JSON line
+    per row on stdout.  Not part of the default run."""
+    import torch
+    from paper_2502_18554_b200 import build, fields, zccl as z
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --table needs a CUDA device")
+    build.build()
+    if not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+    orc = not args.no_cpu_baseline
+    emit = lambda row: print(json.dumps(row), flush=True)
+    emit({"table": "configs 0-4", "host_cores": os.cpu_count(),
+          "protocol": "10 warm-up + 10 timed CUDA-graph replays of one call per buffer set, CUDA events, per call"})
+    big = z.Context(1 << 29, 1)
+
+    emit(_codec_row(z, big, "cfg0", fields.smooth_1d(1 << 20, seed=0), z.EB_REL, 1e-3, orc))
+    x1, loc1 = fields.fourier_field_3d(SIDE, seed=1), fields.fourier_field_3d(SIDE, seed=2)
+    for eb in (1e-2, 1e-3, 1e-4):
+        emit(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, orc and eb == 1e-3, loc1))
+    emit(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, orc))
+
+    # cfg4: message sizes 4 KiB ... 1 GiB in steps of x4, and 2 GiB; prefixes of one cfg0-style field
+    x4 = fields.smooth_1d(1 << 29, seed=0)
+    for log2b in list(range(12, 31, 2)) + [31]:
+        for eb in ((1e-2, 1e-3, 1e-4) if log2b in (20, 26) else (1e-3,)):
+            emit(_codec_row(z, big, f"cfg4 2^{log2b} B", x4[: 1 << (log2b - 2)], z.EB_REL, eb, False))
+    big.close()
+    torch.cuda.empty_cache()
+
+    # cfg4 collectives: 8-rank Allgather and Bcast per message size (per-rank size up to 64 MiB)
+    N = RANKS
+    ctx = z.Context(1 << 27, N)
+    for log2b in range(12, 27, 2):
+        n = 1 << (log2b - 2)
+        send = [torch.from_numpy(x4[r * n:(r + 1) * n]).cuda() for r in range(N)]
+        recv = [torch.empty(N * n, dtype=torch.float32, device="cuda") for _ in range(N)]
+        ag_mean, ag_best = _timed(lambda i: ctx.sim_allgather(send, recv, z.EB_REL, REL), 1)
+        sizes = ctx.sim_sizes()
+        brecv = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(N)]
+        bc_mean, bc_best = _timed(lambda i: ctx.sim_bcast(send[0], brecv, z.EB_REL, REL), 1)
+        ctx.check()
+        emit({"config": f"cfg4 collectives 2^{log2b} B per rank", "ranks": N, "bound": "REL 0.001",
+              "allgather_us_mean": round(ag_mean, 2), "allgather_us_best": round(ag_best, 2),
+              "allgather_gbs": round((N * 4 * n + N * (N - 1) * 4 * n) / ag_mean / 1e3, 1),
+              "allgather_ratio": round(N * 4 * n / sum(sizes[:N]), 3),
+              "bcast_us_mean": round(bc_mean, 2), "bcast_us_best": round(bc_best, 2),
+              "bcast_gbs": round((4 * n + N * 4 * n) / bc_mean / 1e3, 1)})
+        del send, recv, brecv
+    del x4
+    torch.cuda.empty_cache()
+
+    # cfg2: 8 ranks x 2^24, REL 1e-3 of the global range
+    send_h = fields.rank_fields(N, 1 << 24, base_seed=100)
+    send = [torch.from_numpy(a).cuda() for a in send_h]
+    recv = [torch.empty(1 << 24, dtype=torch.float32, device="cuda") for _ in range(N)]
+    ar_mean, ar_best = _timed(lambda i: ctx.sim_allreduce(send, recv, z.EB_REL, REL), 1)
+    rc = ctx.check()
+    sizes = ctx.sim_sizes()
+    exact = torch.zeros(1 << 24, dtype=torch.float64, device="cuda")
+    for t in send:
+        exact += t.double()
+    err = max(float((r.double() - exact).abs().max().item()) for r in recv)
+    lo = min(float(t.min().item()) for t in send)
+    hi = max(float(t.max().item()) for t in send)
+    chunk_bytes = 4 * (1 << 21)
+    per_step = [round(N * chunk_bytes / sum(sizes[k * N:(k + 1) * N]), 3) for k in range(N)]
+    units = N * chunk_bytes + 2 * (N - 1) * N * chunk_bytes
+    row = {"config": "cfg2", "ranks": N, "n_per_rank": 1 << 24, "bound": "REL 0.001", "status": rc,
+           "allreduce_us_mean": round(ar_mean, 1), "allreduce_us_best": round(ar_best, 1),
+           "allreduce_codec_gbs": round(units / ar_mean / 1e3, 1),
+           "allreduce_algbw_gbs": round(4 * (1 << 24) / ar_mean / 1e3, 1),
+           "ratio_per_step": per_step, "max_abs_err_vs_fp64_sum": err, "eb_abs": REL * (hi - lo),
+           "err_over_eb": round(err / (REL * (hi - lo)), 3)}
+    if orc:
+        import oracle
+        t0 = time.perf_counter()
+        oracle.sim_allreduce(send_h, oracle.EB_REL, REL)
+        dt = time.perf_counter() - t0
+        row["oracle_allreduce_s"] = round(dt, 2)
+        row["oracle_codec_gbs"] = round(units / dt / 1e9, 3)
+    emit(row)
+
+
 # --------------------------------------------------------------------------------------------- CUDA arm
 
 def main():
@@ -180,7 +352,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eagerly launched steps instead of CUDA graph replays")
+    ap.add_argument("--table", action="store_true",
+                    help="time configurations 0-4 one by one (one JSON line per row) instead of the benchmark step")
     args = ap.parse_args()
+    if args.table:
+        return config_table(args)
     ref = args.impl == "reference"
     if args.steps is None:
         args.steps = 20 if ref else 1000    # the oracle needs about 0.4 s per step, the GPU under 1 ms
