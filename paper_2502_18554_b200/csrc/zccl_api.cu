@@ -100,15 +100,18 @@ int resolve_bound(zccl_ctx* c, const RangeList& rl, int mode, float eb, Params& 
     rb.count = 0;
     for (size_t i = 0; i < rl.x.size(); ++i) {
         if (rl.n[i] == 0) continue;
-        rb.x[rb.count] = rl.x[i];
-        rb.n[rb.count] = rl.n[i];
-        if (++rb.count == kMaxJobs) {
+        if (rb.count == kMaxJobs) {     // a full batch with more to come: collect only
+            rb.finish = kRangeOnly;
             if (launch_range(rb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
             rb.count = 0;
         }
+        rb.x[rb.count] = rl.x[i];
+        rb.n[rb.count] = rl.n[i];
+        ++rb.count;
     }
-    if (rb.count && launch_range(rb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
-    if (launch_resolve(mode, eb, c->ws, st) != cudaSuccess) return ZCCL_E_CUDA;
+    rb.finish = kRangeResolve;          // the last launch also turns (min, max, eb) into the bound
+    rb.eb = eb;
+    if (launch_range(rb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
     hp = Params{0.f, 1.f, 1.f, 1};
     on_device = true;
     return ZCCL_OK;
@@ -665,12 +668,11 @@ int zccl_range(zccl_ctx* c, const float* x, size_t n, float* minmax, void* strea
     if (!c || (!x && n) || !minmax || n > c->max_elems) return ZCCL_E_ARG;
     if (((uintptr_t)x & 3u) || ((uintptr_t)minmax & 3u)) return ZCCL_E_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    if (n) {
-        RangeBatch rb{};
-        rb.x[0] = x; rb.n[0] = n; rb.count = 1;
-        if (launch_range(rb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
-    }
-    return cuda_rc(launch_export_range(c->ws, minmax, st));
+    RangeBatch rb{};
+    rb.x[0] = x; rb.n[0] = n; rb.count = 1;
+    rb.finish = kRangeExport;
+    rb.out = minmax;
+    return cuda_rc(launch_range(rb, c->ws, c->sm_count, st));
 }
 
 int zccl_scale(zccl_ctx* c, float* y, size_t n, float divisor, void* stream)

@@ -113,18 +113,22 @@ struct ScaleBatch {
     int count;
 };
 
+// What the last CTA of a range launch does with the collected minimum and maximum.
+enum RangeFinish { kRangeOnly = 0, kRangeResolve = 1, kRangeExport = 2 };
+
 struct RangeBatch {
     const float* x[kMaxJobs];
     unsigned long long n[kMaxJobs];
     int count;
+    int finish;     // RangeFinish
+    float eb;       // kRangeResolve: the relative bound
+    float* out;     // kRangeExport: receives (min, max)
 };
 
 enum EncodeMode { kEncodeRaw = 0, kEncodeFused = 1 };
 
 // Launchers (defined next to the kernels).
 cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count, cudaStream_t st);
-cudaError_t launch_resolve(int eb_mode, float eb, const Workspace& ws, cudaStream_t st);
-cudaError_t launch_export_range(const Workspace& ws, float* out, cudaStream_t st);
 cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& ws, bool device_params,
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);

@@ -184,6 +184,47 @@ __device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
 
 // ------------------------------------------------------------------------------------------------ range (REL)
 
+// eb -> (eb_abs, s, r), the reading used throughout: eb_abs = eb * (max - min); step shrunk by 1 - 2^-6;
+// r by one IEEE division.  Consumes and re-arms the min/max keys.  One thread.
+__device__ void resolve_params(float eb, const Workspace& ws)
+{
+    Params p;
+    p.valid = 1;
+    const uint32_t kmin = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 0);
+    const uint32_t kmax = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 1);
+    float range = 0.0f;
+    if (kmin <= kmax) range = __fsub_rn(key2f(kmax), key2f(kmin));
+    if (!(range > 0.0f) || !isfinite(range)) p.valid = 0;
+    const float ea = __fmul_rn(eb, range);
+    ws.minmax[0] = 0xFFFFFFFFu;
+    ws.minmax[1] = 0u;
+    const float ebq = __fmul_rn(ea, 0.984375f);
+    const float s = __fmul_rn(ebq, 2.0f);
+    if (!(s > 0.0f) || !isfinite(s)) p.valid = 0;
+    const float r = __fdiv_rn(1.0f, s);
+    if (!isfinite(r)) p.valid = 0;
+    p.eb_abs = ea; p.s = s; p.r = r;
+    *ws.params = p;
+    if (!p.valid) atomicOr(ws.status, kStDegenerate);
+}
+
+// Hands the minimum and maximum to the caller (out[0] = min, out[1] = max; +inf, -inf when nothing was scanned)
+// and re-arms the keys.  A rank of a real ring combines these with its peers' before it resolves the bound
+// (Section 3.2: one bound per collective).  One thread.
+__device__ void export_range(const Workspace& ws, float* out)
+{
+    const uint32_t kmin = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 0);
+    const uint32_t kmax = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 1);
+    const bool any = kmin <= kmax;
+    out[0] = any ? key2f(kmin) : __int_as_float(0x7F800000);
+    out[1] = any ? key2f(kmax) : __int_as_float(0xFF800000);
+    ws.minmax[0] = 0xFFFFFFFFu;
+    ws.minmax[1] = 0u;
+}
+
+// Minimum and maximum of up to kMaxJobs arrays into the workspace's two ordered keys.  With rb.finish set, the
+// last CTA of the launch to get there turns the keys into the bound (kRangeResolve) or hands them out
+// (kRangeExport), so that a relative bound costs one launch in front of the encoder.
 __global__ void __launch_bounds__(256) range_kernel(RangeBatch rb, Workspace ws)
 {
     float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
@@ -192,13 +233,22 @@ __global__ void __launch_bounds__(256) range_kernel(RangeBatch rb, Workspace ws)
     const unsigned long long n = rb.n[j];
     const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     const unsigned long long nthreads = (unsigned long long)gridDim.x * blockDim.x;
-    // peel to a 16-byte boundary, then 128-bit loads
+    // peel to a 16-byte boundary, then 128-bit loads, four of them in flight per thread
     unsigned long long head = ((16u - (unsigned)((uintptr_t)x & 15u)) & 15u) >> 2;
     if (head > n) head = n;
     if (tid < head) { float v = x[tid]; lo = fminf(lo, v); hi = fmaxf(hi, v); }
     const unsigned long long nvec = (n - head) >> 2;
     const float4* xv = reinterpret_cast<const float4*>(x + head);
-    for (unsigned long long i = tid; i < nvec; i += nthreads) {
+    unsigned long long i = tid;
+    for (; i + 3 * nthreads < nvec; i += 4 * nthreads) {
+        const float4 a = __ldg(xv + i), b = __ldg(xv + i + nthreads), c = __ldg(xv + i + 2 * nthreads),
+                     d = __ldg(xv + i + 3 * nthreads);
+        lo = fminf(fminf(fminf(lo, a.x), fminf(a.y, fminf(a.z, a.w))), fminf(fminf(b.x, b.y), fminf(b.z, b.w)));
+        hi = fmaxf(fmaxf(fmaxf(hi, a.x), fmaxf(a.y, fmaxf(a.z, a.w))), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
+        lo = fminf(fminf(fminf(lo, c.x), fminf(c.y, fminf(c.z, c.w))), fminf(fminf(d.x, d.y), fminf(d.z, d.w)));
+        hi = fmaxf(fmaxf(fmaxf(hi, c.x), fmaxf(c.y, fmaxf(c.z, c.w))), fmaxf(fmaxf(d.x, d.y), fmaxf(d.z, d.w)));
+    }
+    for (; i < nvec; i += nthreads) {
         float4 v = __ldg(xv + i);
         lo = fminf(fminf(lo, v.x), fminf(v.y, fminf(v.z, v.w)));
         hi = fmaxf(fmaxf(hi, v.x), fmaxf(v.y, fmaxf(v.z, v.w)));
@@ -219,48 +269,16 @@ __global__ void __launch_bounds__(256) range_kernel(RangeBatch rb, Workspace ws)
             atomicMin(&ws.minmax[0], f2key(lo));
             atomicMax(&ws.minmax[1], f2key(hi));
         }
+        if (rb.finish != kRangeOnly) {
+            __threadfence();
+            if (atomicAdd(ws.done, 1u) == gridDim.x * gridDim.y - 1u) {   // every CTA's keys are in
+                __threadfence();
+                *ws.done = 0;
+                if (rb.finish == kRangeResolve) resolve_params(rb.eb, ws);
+                else export_range(ws, rb.out);
+            }
+        }
     }
-}
-
-// eb -> (eb_abs, s, r), the reading used throughout: eb_abs = eb * (max - min); step shrunk by 1 - 2^-6;
-// r by one IEEE division.  Consumes and re-arms the min/max keys.
-__global__ void resolve_kernel(int eb_mode, float eb, Workspace ws)
-{
-    if (threadIdx.x || blockIdx.x) return;
-    Params p;
-    p.valid = 1;
-    float ea = eb;
-    if (eb_mode == 1) {
-        const uint32_t kmin = ws.minmax[0], kmax = ws.minmax[1];
-        float range = 0.0f;
-        if (kmin <= kmax) range = __fsub_rn(key2f(kmax), key2f(kmin));
-        if (!(range > 0.0f) || !isfinite(range)) p.valid = 0;
-        ea = __fmul_rn(eb, range);
-        ws.minmax[0] = 0xFFFFFFFFu;
-        ws.minmax[1] = 0u;
-    }
-    const float ebq = __fmul_rn(ea, 0.984375f);
-    const float s = __fmul_rn(ebq, 2.0f);
-    if (!(s > 0.0f) || !isfinite(s)) p.valid = 0;
-    const float r = __fdiv_rn(1.0f, s);
-    if (!isfinite(r)) p.valid = 0;
-    p.eb_abs = ea; p.s = s; p.r = r;
-    *ws.params = p;
-    if (!p.valid) atomicOr(ws.status, kStDegenerate);
-}
-
-// Hands the minimum and maximum collected by range_kernel to the caller (out[0] = min, out[1] = max; +inf, -inf
-// when nothing was scanned) and re-arms the keys.  A rank of a real ring combines these with its peers' before it
-// resolves the bound (Section 3.2: one bound per collective).
-__global__ void export_range_kernel(Workspace ws, float* out)
-{
-    if (threadIdx.x || blockIdx.x) return;
-    const uint32_t kmin = ws.minmax[0], kmax = ws.minmax[1];
-    const bool any = kmin <= kmax;
-    out[0] = any ? key2f(kmin) : __int_as_float(0x7F800000);
-    out[1] = any ? key2f(kmax) : __int_as_float(0xFF800000);
-    ws.minmax[0] = 0xFFFFFFFFu;
-    ws.minmax[1] = 0u;
 }
 
 // ------------------------------------------------------------------------------------------------ stream header
@@ -1805,20 +1823,6 @@ cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count
     unsigned gx = (unsigned)(want < per ? (want ? want : 1) : per);
     ++g_launches;
     range_kernel<<<dim3(gx, rb.count), 256, 0, st>>>(rb, ws);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_resolve(int eb_mode, float eb, const Workspace& ws, cudaStream_t st)
-{
-    ++g_launches;
-    resolve_kernel<<<1, 32, 0, st>>>(eb_mode, eb, ws);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_export_range(const Workspace& ws, float* out, cudaStream_t st)
-{
-    ++g_launches;
-    export_range_kernel<<<1, 32, 0, st>>>(ws, out);
     return cudaGetLastError();
 }
 
