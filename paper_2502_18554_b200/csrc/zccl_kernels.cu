@@ -439,6 +439,25 @@ __device__ __forceinline__ void decode_blocks_f32(const uint2* __restrict__ tbl,
                 const uint32_t sg = prmt(v, v, (0x8u | (uint32_t)u) << 12);   // byte 3 = sign of byte u, replicated
                 wbuf[32 * i + (lane ^ (u << 2))] = __uint_as_float(__float_as_uint(mag) | (sg & 0x80000000u));
             }
+        } else if (!__any_sync(kFull, em.x > 15u)) {
+            // two blocks per transpose: lane 16u + b fetches plane b of block 2h + u (b = 15: its sign word)
+            const uint32_t wp2 = ((uint32_t)lane + 1u) & 15u;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint2 e = tbl[4 * g + 2 * h + (lane >> 4)];
+                const uint32_t n = e.x ? e.x + 1 : 0;
+                uint32_t w = 0;
+                if (wp2 < n) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(e.y + 4 * wp2) : "memory");
+                const uint32_t v = xp(w);   // half u: bits 0..14 = |delta| of this lane's element of block 2h + u, bit 15 = sign
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int b4 = 2 * h + u, i = 4 * g + b4;
+                    const uint32_t m = u ? (v >> 16) & 0x7FFFu : v & 0x7FFFu;
+                    const float mag = __fsub_rn(__uint_as_float(m | 0x4B000000u), kTwo23);
+                    const uint32_t sg = u ? v : v << 16;
+                    wbuf[32 * i + (lane ^ (b4 << 2))] = __uint_as_float(__float_as_uint(mag) | (sg & 0x80000000u));
+                }
+            }
         } else {
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -799,7 +818,7 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
                 ab[u] = __float_as_uint(__fadd_rn(fabsf(df), kTwo23));
                 db[u] = __float_as_uint(df);
             }
-            const uint32_t wide = ((ab[0] | ab[1] | ab[2]) | ab[3]) & 0x7FFF80u;
+            const uint32_t wide = ((ab[0] | ab[1] | ab[2]) | ab[3]) & 0x7FFF80u;   // magnitude bits above bit 6
             if (!__any_sync(kFull, wide != 0)) {
                 // byte u of the word: bits 0..6 = |delta| of this lane's element of block u, bit 7 = its sign
                 const uint32_t mg = prmt(prmt(ab[0], ab[1], 0x0040u), prmt(ab[2], ab[3], 0x0040u), 0x5410u);
@@ -813,6 +832,25 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
                 const uint32_t n_mine = (nword >> pk.sh8) & 0xFFu;
                 if (pk.wp < n_mine) slots_w[wsum + ((pref >> pk.sh8) & 0xFFu) + pk.wp] = v;
                 wsum += (nword * 0x01010101u) >> 24;
+            } else if (!__any_sync(kFull, (wide & 0x7F8000u) != 0)) {
+                // two blocks per transpose while their code lengths are at most 15: half u of the word holds
+                // |delta| of this lane's element of block 2h + u in bits 0..14 and its sign in bit 15, so lane
+                // 16u + b ends up with plane b of that block (b = 15: its sign word)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t mg = prmt(ab[2 * h], ab[2 * h + 1], 0x5410u);
+                    const uint32_t sg = prmt(db[2 * h], db[2 * h + 1], 0xF0B0u);
+                    const uint32_t v = xp(mg | (sg & 0x80008000u));
+                    const uint32_t ors = __reduce_or_sync(kFull, mg);
+                    const uint32_t L0 = 32u - (uint32_t)__clz((int)(ors & 0x7FFFu));
+                    const uint32_t L1 = 32u - (uint32_t)__clz((int)(ors >> 16));
+                    const uint32_t n0 = L0 ? L0 + 1u : 0u, n1 = L1 ? L1 + 1u : 0u;
+                    const uint32_t wp2 = ((uint32_t)lane + 1u) & 15u;
+                    const bool hi = lane >= 16;
+                    if (wp2 < (hi ? n1 : n0)) slots_w[wsum + (hi ? n0 : 0u) + wp2] = v;
+                    wsum += n0 + n1;
+                    lword |= (L0 | (L1 << 8)) << (16 * h);
+                }
             } else {
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {

@@ -130,6 +130,40 @@ def test_all_code_lengths_occur(z, ctx):
     assert_same_bits(y, oracle.decompress(want))
 
 
+def _mixed_length_field(seed, nblocks, lmax):
+    """Blocks whose code lengths are drawn independently from 0..lmax (amplitude 2^(L-1) around a common level), so
+    that neighbouring blocks of every pair and every group of four differ in length."""
+    rng = np.random.default_rng(seed)
+    ea, s, r = oracle.resolve(oracle.EB_ABS, 0.5)
+    q = np.zeros(nblocks * 32, np.int64)
+    for b in range(nblocks):
+        L = int(rng.integers(0, lmax + 1))
+        if L:
+            q[32 * b: 32 * b + 32] = rng.integers(-(2 ** (L - 1)), 2 ** (L - 1) + 1, 32)
+        elif b:
+            q[32 * b: 32 * b + 32] = q[32 * b - 1]           # a constant block continues the last value
+    return (q.astype(np.float64) * float(s)).astype(f32)
+
+
+@pytest.mark.parametrize("lmax", [7, 9, 15, 17, 22])
+def test_neighbouring_blocks_of_different_code_lengths(z, ctx, lmax):
+    # the encoder and the decoder handle four, two or one block per bit-matrix transpose depending on the longest
+    # code of a group of four; every mixture of lengths inside a group must give the oracle's bytes and values
+    x = _mixed_length_field(100 + lmax, 5 * 128 + 37, lmax)
+    want, wrc = oracle.compress(x, oracle.EB_ABS, 0.5)
+    got, rc = gpu_compress(z, ctx, x, z.EB_ABS, 0.5)
+    assert rc == wrc
+    assert np.array_equal(got, want)
+    y, _ = gpu_decompress(z, ctx, want, x.size)
+    assert_same_bits(y, oracle.decompress(want))
+    b = _mixed_length_field(200 + lmax, 5 * 128 + 37, max(lmax - 2, 1))
+    fw, frc, fraw = oracle.drc(want, local=b, want_raw=True)
+    fg, grc, graw = _drc_gpu(z, ctx, want, x.size, local=b, raw=True)
+    assert grc == frc
+    assert np.array_equal(fg, fw)
+    assert_same_bits(graw, fraw)
+
+
 def test_adversarial_ties_and_denormals(z, ctx):
     ea, s, r = oracle.resolve(oracle.EB_ABS, 1e-3)
     k = np.arange(-3000, 3000, dtype=np.float64)
