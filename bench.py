@@ -269,29 +269,34 @@ def config_table(args):
         import oracle
         oracle.build()
     orc = not args.no_cpu_baseline
+    want = set(args.rows.split(","))
     emit = lambda row: print(json.dumps(row), flush=True)
     emit({"table": "configs 0-4", "host_cores": os.cpu_count(),
           "protocol": "10 warm-up + 10 timed CUDA-graph replays of one call per buffer set, CUDA events, per call"})
     big = z.Context(1 << 29, 1)
 
-    emit(_codec_row(z, big, "cfg0", fields.smooth_1d(1 << 20, seed=0), z.EB_REL, 1e-3, orc))
-    x1, loc1 = fields.fourier_field_3d(SIDE, seed=1), fields.fourier_field_3d(SIDE, seed=2)
-    for eb in (1e-2, 1e-3, 1e-4):
-        emit(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, orc and eb == 1e-3, loc1))
-    emit(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, orc))
+    if "cfg0" in want:
+        emit(_codec_row(z, big, "cfg0", fields.smooth_1d(1 << 20, seed=0), z.EB_REL, 1e-3, orc))
+    if "cfg1" in want:
+        x1, loc1 = fields.fourier_field_3d(SIDE, seed=1), fields.fourier_field_3d(SIDE, seed=2)
+        for eb in (1e-2, 1e-3, 1e-4):
+            emit(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, orc and eb == 1e-3, loc1))
+    if "cfg3" in want:
+        emit(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, orc))
 
     # cfg4: message sizes 4 KiB ... 1 GiB in steps of x4, and 2 GiB; prefixes of one cfg0-style field
-    x4 = fields.smooth_1d(1 << 29, seed=0)
-    for log2b in list(range(12, 31, 2)) + [31]:
-        for eb in ((1e-2, 1e-3, 1e-4) if log2b in (20, 26) else (1e-3,)):
-            emit(_codec_row(z, big, f"cfg4 2^{log2b} B", x4[: 1 << (log2b - 2)], z.EB_REL, eb, False))
+    x4 = fields.smooth_1d(1 << 29 if "cfg4" in want else 1 << 27, seed=0) if want & {"cfg4", "collectives"} else None
+    if "cfg4" in want:
+        for log2b in list(range(12, 31, 2)) + [31]:
+            for eb in ((1e-2, 1e-3, 1e-4) if log2b in (20, 26) else (1e-3,)):
+                emit(_codec_row(z, big, f"cfg4 2^{log2b} B", x4[: 1 << (log2b - 2)], z.EB_REL, eb, False))
     big.close()
     torch.cuda.empty_cache()
 
     # cfg4 collectives: 8-rank Allgather and Bcast per message size (per-rank size up to 64 MiB)
     N = RANKS
     ctx = z.Context(1 << 27, N)
-    for log2b in range(12, 27, 2):
+    for log2b in range(12, 27, 2) if "collectives" in want else ():
         n = 1 << (log2b - 2)
         send = [torch.from_numpy(x4[r * n:(r + 1) * n]).cuda() for r in range(N)]
         recv = [torch.empty(N * n, dtype=torch.float32, device="cuda") for _ in range(N)]
@@ -310,6 +315,8 @@ def config_table(args):
     del x4
     torch.cuda.empty_cache()
 
+    if "cfg2" not in want:
+        return
     # cfg2: 8 ranks x 2^24, REL 1e-3 of the global range
     send_h = fields.rank_fields(N, 1 << 24, base_seed=100)
     send = [torch.from_numpy(a).cuda() for a in send_h]
@@ -354,6 +361,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eagerly launched steps instead of CUDA graph replays")
     ap.add_argument("--table", action="store_true",
                     help="time configurations 0-4 one by one (one JSON line per row) instead of the benchmark step")
+    ap.add_argument("--rows", default="cfg0,cfg1,cfg2,cfg3,cfg4,collectives",
+                    help="with --table: which groups of rows to run (comma-separated)")
     args = ap.parse_args()
     if args.table:
         return config_table(args)
