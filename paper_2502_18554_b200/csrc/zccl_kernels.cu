@@ -27,6 +27,8 @@
 // not.
 #include "zccl_internal.h"
 
+#include <cstdlib>
+
 namespace zccl {
 
 namespace {
@@ -182,6 +184,17 @@ __device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
     return lo;
 }
 
+// Programmatic dependent launch: every kernel of the library is launched with stream serialisation relaxed, so that
+// its CTAs are dispatched while the kernel in front of it on the stream drains, and waits here, before it touches
+// memory, until that kernel has completed and its writes are visible.  Only then does it let the kernel behind it
+// start to launch, so at most one waiting grid is resident at a time.  Without the launch attribute both
+// instructions do nothing.
+__device__ __forceinline__ void pdl_enter()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------------------------------------------------ range (REL)
 
 // eb -> (eb_abs, s, r), the reading used throughout: eb_abs = eb * (max - min); step shrunk by 1 - 2^-6;
@@ -227,6 +240,7 @@ __device__ void export_range(const Workspace& ws, float* out)
 // (kRangeExport), so that a relative bound costs one launch in front of the encoder.
 __global__ void __launch_bounds__(256) range_kernel(RangeBatch rb, Workspace ws)
 {
+    pdl_enter();
     float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
     const int j = blockIdx.y;
     const float* x = rb.x[j];
@@ -627,6 +641,7 @@ __device__ __forceinline__ int describe_staged(uint2* __restrict__ tbl, const ui
 
 __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Workspace ws)
 {
+    pdl_enter();
     __shared__ DecodeShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t G = gridDim.x;
@@ -1217,6 +1232,7 @@ __device__ __forceinline__ Planned plan_pending(PlanShared& plan, ScanShared& sc
 
 __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Workspace ws, Params hp, int use_dev_params)
 {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     EncodeShared& sh = *reinterpret_cast<EncodeShared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1360,6 +1376,7 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
 // out = compress(decompress(in_c) + local) per tile, with no uncompressed intermediate in global memory.
 __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, Workspace ws)
 {
+    pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     FusedShared& sh = *reinterpret_cast<FusedShared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1659,6 +1676,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
 // One forwarding hop of compressed bytes whose length lives on the device (grid.y = job).
 __global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
 {
+    pdl_enter();
     const CopyJob& job = cb.job[blockIdx.y];
     const unsigned long long bytes = job.bytes ? *job.bytes : job.fixed_bytes;
     if (bytes > job.cap) {
@@ -1686,6 +1704,7 @@ __global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
 // synchronisation is needed) and stores it into the next rank's slot.
 __global__ void __launch_bounds__(256) copy_chain_kernel(ChainBatch cb, Workspace ws)
 {
+    pdl_enter();
     const ChainJob& job = cb.job[blockIdx.y];
     const unsigned long long bytes = *job.bytes;
     const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -1723,6 +1742,7 @@ __global__ void __launch_bounds__(256) copy_chain_kernel(ChainBatch cb, Workspac
 // y = y / divisor, element by element (Average = Sum / N at the end of the Allreduce).
 __global__ void __launch_bounds__(256) scale_kernel(ScaleBatch sb)
 {
+    pdl_enter();
     float* __restrict__ y = sb.y[blockIdx.y];
     const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     const unsigned long long nth = (unsigned long long)gridDim.x * blockDim.x;
@@ -1741,6 +1761,7 @@ __global__ void __launch_bounds__(256) scale_kernel(ScaleBatch sb)
 __global__ void __launch_bounds__(256) quality_kernel(const float* __restrict__ x, const float* __restrict__ y, unsigned long long n,
                                                       double* __restrict__ out, double* __restrict__ partials, uint32_t* counter)
 {
+    pdl_enter();
     __shared__ double red[4][8];
     __shared__ uint32_t is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1851,6 +1872,34 @@ unsigned long long g_launches = 0;   // kernels launched by this library in this
 
 unsigned long long launch_count() { return g_launches; }
 
+// Launch with programmatic stream serialisation (see pdl_enter); ZCCL_PDL=0 in the environment turns it off.
+// EARLY = false keeps a kernel fully serialised behind its predecessor.  The fused hop needs that: its tiles are
+// dealt round-robin over a grid that must be resident as a whole (a CTA's scan waits for tiles of other CTAs), and
+// CTAs dispatched onto SMs that still run another kernel's CTAs do not all fit (the SM keeps that kernel's
+// shared-memory configuration), which left part of the grid waiting behind the resident part.  The other kernels
+// make no such assumption: tiles handed out by a counter, or CTAs that never wait for one another.
+static bool pdl_enabled()
+{
+    static const bool on = [] { const char* e = getenv("ZCCL_PDL"); return !(e && e[0] == '0'); }();
+    return on;
+}
+
+template <bool EARLY = true, class... KArgs, class... Args>
+static cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = (EARLY && pdl_enabled()) ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
     if (rb.count <= 0) return cudaSuccess;
@@ -1860,8 +1909,7 @@ cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count
     unsigned per = (unsigned)((sm_count * 8 + rb.count - 1) / rb.count);
     unsigned gx = (unsigned)(want < per ? (want ? want : 1) : per);
     ++g_launches;
-    range_kernel<<<dim3(gx, rb.count), 256, 0, st>>>(rb, ws);
-    return cudaGetLastError();
+    return launch_k(range_kernel, dim3(gx, rb.count), dim3(256), 0, st, rb, ws);
 }
 
 cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& ws, bool device_params,
@@ -1885,10 +1933,9 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
     unsigned grid = (unsigned)(jb.total_tiles < cap ? jb.total_tiles : cap);
     ++g_launches;
     if (mode == kEncodeRaw)
-        encode_raw_kernel<<<grid, kThreads, sizeof(EncodeShared), st>>>(jb, ws, host_params, device_params ? 1 : 0);
+        return launch_k(encode_raw_kernel, dim3(grid), dim3(kThreads), sizeof(EncodeShared), st, jb, ws, host_params, device_params ? 1 : 0);
     else
-        encode_fused_kernel<<<grid, kThreads, sizeof(FusedShared), st>>>(jb, ws);
-    return cudaGetLastError();
+        return launch_k<false>(encode_fused_kernel, dim3(grid), dim3(kThreads), sizeof(FusedShared), st, jb, ws);
 }
 
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
@@ -1902,8 +1949,7 @@ cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count,
     unsigned long long cap = (unsigned long long)sm_count * g_decode_ctas_per_sm;
     unsigned grid = (unsigned)(jb.total_tiles < cap ? jb.total_tiles : cap);
     ++g_launches;
-    decode_kernel<<<grid, kThreads, 0, st>>>(jb, ws);
-    return cudaGetLastError();
+    return launch_k(decode_kernel, dim3(grid), dim3(kThreads), 0, st, jb, ws);
 }
 
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st)
@@ -1911,8 +1957,7 @@ cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, 
     if (cb.count <= 0) return cudaSuccess;
     unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
     ++g_launches;
-    copy_kernel<<<dim3(gx ? gx : 1, cb.count), 256, 0, st>>>(cb, ws);
-    return cudaGetLastError();
+    return launch_k(copy_kernel, dim3(gx ? gx : 1, cb.count), dim3(256), 0, st, cb, ws);
 }
 
 cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st)
@@ -1922,8 +1967,7 @@ cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st)
     unsigned per = (unsigned)((sm_count * 8 + sb.count - 1) / sb.count);
     unsigned gx = (unsigned)(want < per ? want : per);
     ++g_launches;
-    scale_kernel<<<dim3(gx ? gx : 1, sb.count), 256, 0, st>>>(sb);
-    return cudaGetLastError();
+    return launch_k(scale_kernel, dim3(gx ? gx : 1, sb.count), dim3(256), 0, st, sb);
 }
 
 cudaError_t launch_quality(const float* x, const float* y, unsigned long long n, double* out, double* partials,
@@ -1934,8 +1978,7 @@ cudaError_t launch_quality(const float* x, const float* y, unsigned long long n,
     if (cap > (unsigned long long)kQualityCtas) cap = kQualityCtas;
     const unsigned grid = (unsigned)(want < cap ? (want ? want : 1) : cap);
     ++g_launches;
-    quality_kernel<<<grid, 256, 0, st>>>(x, y, n, out, partials, counter);
-    return cudaGetLastError();
+    return launch_k(quality_kernel, dim3(grid), dim3(256), 0, st, x, y, n, out, partials, counter);
 }
 
 cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st)
@@ -1943,8 +1986,7 @@ cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_
     if (cb.count <= 0 || cb.hops == 0) return cudaSuccess;
     unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
     ++g_launches;
-    copy_chain_kernel<<<dim3(gx ? gx : 1, cb.count), 256, 0, st>>>(cb, ws);
-    return cudaGetLastError();
+    return launch_k(copy_chain_kernel, dim3(gx ? gx : 1, cb.count), dim3(256), 0, st, cb, ws);
 }
 
 }  // namespace zccl
