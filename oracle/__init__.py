@@ -62,6 +62,7 @@ def lib():
         L.zo_sim_reduce_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
                                             C.c_void_p]
         L.zo_quality.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.zo_stream_stats.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
         L.zo_sim_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
                                      C.c_void_p, C.c_void_p]
         _lib = L
@@ -251,3 +252,13 @@ def quality(x, y):
     if rc < 0:
         raise OracleError(rc, "quality")
     return dict(max_abs_err=out[0], mse=out[1], nrmse=out[2], psnr=out[3], min=out[4], max=out[5])
+
+
+def stream_stats(stream):
+    """Code-length histogram of a stream: uint64[33], entry L = blocks stored with code length L, entry 32 = blocks."""
+    st = np.ascontiguousarray(stream, dtype=np.uint8)
+    hist = np.zeros(33, dtype=np.uint64)
+    rc = lib().zo_stream_stats(_ptr(st), st.size, _ptr(hist))
+    if rc != OK:
+        raise OracleError(rc, "stream_stats")
+    return hist

@@ -638,3 +638,34 @@ int zo_quality(const float *x, const float *y, size_t n, double *out)
     }
     return ZO_OK;
 }
+
+/* Code-length statistics of a stream (Section 4.1, the table of compression ratios and percentages of constant
+ * blocks: a block whose code length is 0 is a constant block and costs one byte).  hist[L], L = 0..31, receives the
+ * number of 32-element blocks stored with code length L; hist[32] the number of blocks.  The walk is that of the
+ * decompressor: chunk starts from the sizes at the front, code-length bytes behind each tile's outlier. */
+int zo_stream_stats(const uint8_t *in, size_t in_bytes, uint64_t *hist)
+{
+    uint64_t n; float eb_abs, s; uint32_t T, nT; size_t total;
+    int rc = zo_stream_info(in, in_bytes, &n, &eb_abs, &s, &T, &nT, &total);
+    if (rc != ZO_OK) return rc;
+    for (int k = 0; k <= 32; ++k) hist[k] = 0;
+    size_t blob0 = ZO_HEADER + 4 * (size_t)nT;
+    uint32_t prev_words = 0;
+    for (size_t t = 0; t < nT; ++t) {
+        uint32_t w = get_u32(in + ZO_HEADER + 4 * t);
+        if (w < prev_words) return ZO_E_BAD_STREAM;
+        size_t start = t * (size_t)T;
+        size_t len = (n - start < T) ? (size_t)(n - start) : T;
+        size_t nb = (len + ZO_BLOCK - 1) / ZO_BLOCK;
+        size_t pos = blob0 + 4 * (size_t)prev_words;
+        if (pos + 4 + pad4(nb) > blob0 + 4 * (size_t)w) return ZO_E_BAD_STREAM;
+        for (size_t b = 0; b < nb; ++b) {
+            unsigned L = in[pos + 4 + b];
+            if (L > 31) return ZO_E_BAD_STREAM;
+            hist[L] += 1;
+            hist[32] += 1;
+        }
+        prev_words = w;
+    }
+    return ZO_OK;
+}

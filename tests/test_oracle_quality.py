@@ -68,3 +68,63 @@ def test_uniform_quantisation_error_statistics():
     assert 0.5 < q["mse"] / (float(s) ** 2 / 12) < 1.5
     assert 0.5 * rel / math.sqrt(3) < q["nrmse"] < 1.05 * rel / math.sqrt(3)
     assert math.isclose(q["psnr"], -20 * math.log10(q["nrmse"]), rel_tol=1e-12)
+
+
+# ----------------------------------------------------------------------------- code-length statistics of a stream
+
+def _brute_force_hist(x, ea_s_r, T):
+    """Histogram of code lengths straight from the definition: quantise, deltas inside each tile (the first element
+    of a tile has none), bit length of the largest magnitude of every block of 32."""
+    _, s, r = ea_s_r
+    q, _ = oracle.quantise(x, r)
+    q = q.astype(np.int64)
+    hist = np.zeros(33, np.uint64)
+    for t0 in range(0, q.size, T):
+        qt = q[t0:t0 + T]
+        d = np.diff(qt, prepend=qt[:1])
+        for b0 in range(0, d.size, 32):
+            L = int(np.abs(d[b0:b0 + 32]).max()).bit_length()
+            hist[L] += 1
+            hist[32] += 1
+    return hist
+
+
+def test_stream_stats_constant_field_is_all_constant_blocks():
+    # Section 3.3: code length 0 = constant block, stored as its one byte; a constant array has nothing else
+    x = np.full(3 * 4096 + 100, 2.5, np.float32)
+    st, _ = oracle.compress(x, oracle.EB_ABS, 1e-3)
+    h = oracle.stream_stats(st)
+    nblk = 3 * 128 + 4
+    assert h[0] == nblk and h[32] == nblk and h[1:32].sum() == 0
+
+
+def test_stream_stats_match_brute_force_and_stream_size():
+    for T in (4096, 5120):
+        for seed, n, eb in ((1, 20000, 1e-3), (2, 4096 * 3, 1e-2), (3, 5000, 1e-5)):
+            x = fields.smooth_1d(n, seed=seed)
+            x[n // 2: n // 2 + 700] += np.random.default_rng(seed).normal(0, 0.3, 700).astype(np.float32)
+            st, _ = oracle.compress(x, oracle.EB_REL, eb, T)
+            h = oracle.stream_stats(st)
+            want = _brute_force_hist(x, oracle.resolve(oracle.EB_REL, eb, x), T)
+            assert np.array_equal(h, want)
+            # the histogram fixes the stream's length: header, one index entry and one outlier per tile, the padded
+            # code-length bytes, a sign word and L plane words per non-constant block
+            nT = -(-n // T)
+            size = 32 + 4 * nT
+            for t in range(nT):
+                nb = -(-min(T, n - t * T) // 32)
+                size += 4 + ((nb + 3) & ~3)
+            size += sum(4 * (1 + L) * int(h[L]) for L in range(1, 32))
+            assert size == st.size
+
+
+def test_stream_stats_rejects_a_damaged_stream():
+    x = fields.smooth_1d(9000, seed=5)
+    st, _ = oracle.compress(x, oracle.EB_ABS, 1e-3)
+    bad = st.copy()
+    bad[0] ^= 0xFF
+    try:
+        oracle.stream_stats(bad)
+        assert False, "a stream without the magic word must be refused"
+    except oracle.OracleError as e:
+        assert e.code == oracle.E_BAD_STREAM
