@@ -224,8 +224,14 @@ def _codec_row(z, ctx, name, x_h, mode, eb, with_oracle: bool, loc_h=None):
     d_mean, d_best = _timed(lambda i: ctx.decompress(outs[i][:cbytes], ys[i]), sets)
     ctx.check()
     err = float((ys[0].double() - xs[0].double()).abs().max().item())
+    hist = torch.zeros(33, dtype=torch.int64, device="cuda")
+    ctx.stream_stats(outs[0][:cbytes], hist)
+    ctx.check()
+    hh = hist.cpu().numpy().astype(np.float64)
     row = {"config": name, "n": n, "bytes": nbytes, "bound": ("REL " if mode == z.EB_REL else "ABS ") + f"{eb:g}",
            "ratio": round(nbytes / cbytes, 3), "status": rc, "max_abs_err": err, "buffer_sets": sets,
+           "constant_block_pct": round(100.0 * hh[0] / max(hh[32], 1.0), 2),
+           "mean_code_length": round(float((hh[:32] * np.arange(32)).sum() / max(hh[32], 1.0)), 3),
            "compress_us_mean": round(c_mean, 2), "compress_us_best": round(c_best, 2),
            "compress_gbs": round(nbytes / c_mean / 1e3, 1),
            "decompress_us_mean": round(d_mean, 2), "decompress_us_best": round(d_best, 2),
@@ -573,8 +579,13 @@ def main():
     torch.cuda.synchronize()
     q_ms = statistics.mean(a.elapsed_time(b) for a, b in q_ev)
     qv = qout.cpu().numpy()
+    hist = torch.zeros(33, dtype=torch.int64, device=dev)
+    ctx.stream_stats(cs[0], hist)     # the stream of the batch the ratios are quoted on (length from its header)
+    ctx.check()
+    hh = hist.cpu().numpy().astype(np.float64)
     quality = {"max_abs_err": float(qv[0]), "nrmse": float(qv[2]), "psnr_db": float(qv[3]), "bit_rate": 32.0 / ratio1,
-               "eb_abs": eb_abs}
+               "eb_abs": eb_abs, "constant_block_pct": 100.0 * hh[0] / max(hh[32], 1.0),
+               "mean_code_length": float((hh[:32] * np.arange(32)).sum() / max(hh[32], 1.0))}
     kern["quality(metrics)"] = {"ms": q_ms, "bytes": 2.0 * in_b}
     kq = kern["quality(metrics)"]
     kq["achieved_gbs"] = kq["bytes"] / (kq["ms"] * 1e-3) / 1e9

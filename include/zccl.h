@@ -255,6 +255,19 @@ int zccl_sim_sizes(zccl_ctx* ctx, size_t* sizes, int capacity, void* stream);
 int zccl_quality(zccl_ctx* ctx, const float* x, const float* y, size_t n, double* out, void* stream);
 
 /*
+ * Code-length statistics of a stream (Section 4.1 reports the percentage of constant blocks next to the ratio: a
+ * block whose code length is 0 is a constant block and is stored as its one code-length byte).
+ *   in   [device] stream, in_bytes_max readable bytes (4-byte aligned)
+ *   hist [device] 33 x unsigned long long: hist[L], L = 0..31 = number of 32-element blocks stored with code length
+ *        L; hist[32] = number of blocks.  Constant-block share = hist[0] / hist[32]; mean code length =
+ *        sum L hist[L] / hist[32].
+ * Enqueues on `stream`.  A stream that does not parse (magic, version, tile size, index beyond in_bytes_max, a code
+ * length above 31) sets ZCCL_E_BAD_STREAM in the device status and leaves hist incomplete.  ZCCL_E_ARG for null or
+ * misaligned pointers, ZCCL_E_CAPACITY when in_bytes_max is smaller than a header.
+ */
+int zccl_stream_stats(zccl_ctx* ctx, const void* in, size_t in_bytes_max, unsigned long long* hist, void* stream);
+
+/*
  * The two per-rank steps of a real ring that are not a codec call (Section 3.2: the error bound is resolved once
  * per collective, over the data of all ranks; Corollary 2: Average = Sum / N).
  *   zccl_range: minmax [device, 2 floats] <- (min, max) of x [device, n floats]; (+inf, -inf) when n == 0.  A

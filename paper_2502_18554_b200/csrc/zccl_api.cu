@@ -663,6 +663,15 @@ int zccl_quality(zccl_ctx* c, const float* x, const float* y, size_t n, double* 
     return cuda_rc(launch_quality(x, y, n, out, c->quality_partials, c->quality_counter, c->sm_count, (cudaStream_t)stream));
 }
 
+int zccl_stream_stats(zccl_ctx* c, const void* in, size_t in_bytes_max, unsigned long long* hist, void* stream)
+{
+    if (!c || !in || !hist || ((uintptr_t)in & 3u) || ((uintptr_t)hist & 7u)) return ZCCL_E_ARG;
+    if (in_bytes_max < (size_t)kHeaderBytes) return ZCCL_E_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(hist, 0, sizeof(unsigned long long) * 33, st) != cudaSuccess) return ZCCL_E_CUDA;
+    return cuda_rc(launch_stream_stats((const uint32_t*)in, in_bytes_max, hist, c->ws, c->sm_count, st));
+}
+
 int zccl_range(zccl_ctx* c, const float* x, size_t n, float* minmax, void* stream)
 {
     if (!c || (!x && n) || !minmax || n > c->max_elems) return ZCCL_E_ARG;

@@ -1752,6 +1752,51 @@ __global__ void __launch_bounds__(256) scale_kernel(ScaleBatch sb)
     for (unsigned long long i = tid; i < sb.n; i += nth) y[i] = __fdiv_rn(y[i], sb.divisor);
 }
 
+// ------------------------------------------------------------------------------------------------ stream statistics
+
+// Histogram of the code lengths of a stream (hist[L], L = 0..31: blocks stored with code length L; hist[32]: blocks),
+// from which the share of constant blocks (L = 0) and the mean code length follow.  One warp per tile: it finds the
+// tile's blob through the index, reads the code-length bytes behind the outlier (a word of four per lane) and
+// counts them in shared memory; every CTA adds its counts to the result at the end.
+__global__ void __launch_bounds__(256) stream_stats_kernel(const uint32_t* __restrict__ in, unsigned long long cap_bytes,
+                                                           unsigned long long* __restrict__ hist, Workspace ws)
+{
+    pdl_enter();
+    __shared__ unsigned int cnt[33];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid < 33) cnt[tid] = 0;
+    __syncthreads();
+    const StreamInfo h = read_header(in, cap_bytes);
+    bool bad = !h.ok;
+    if (h.ok) {
+        const unsigned long long blob0 = (unsigned long long)kHeaderWords + h.nT;
+        const uint32_t total_w = h.nT ? ldg_u32(in + kHeaderWords + h.nT - 1) : 0;
+        if ((blob0 + total_w) * 4ull > cap_bytes) bad = true;
+        const unsigned long long warps = (unsigned long long)gridDim.x * kWarps;
+        for (unsigned long long t = (unsigned long long)blockIdx.x * kWarps + warp; !bad && t < h.nT; t += warps) {
+            const uint32_t w_beg = t ? ldg_u32(in + kHeaderWords + t - 1) : 0, w_end = ldg_u32(in + kHeaderWords + t);
+            const unsigned long long left = h.n - t * kTile;
+            const uint32_t nb = (uint32_t)(((left < (unsigned long long)kTile ? left : (unsigned long long)kTile) + kBlock - 1) / kBlock);
+            const uint32_t lw = (nb + 3) >> 2;                         // words of code-length bytes
+            if (w_end < w_beg || w_end > total_w || w_end - w_beg < 1 + lw) { bad = true; break; }
+            if ((uint32_t)lane < lw) {
+                const uint32_t word = ldg_u32(in + blob0 + w_beg + 1 + lane);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (4u * lane + k < nb) {
+                        const uint32_t L = (word >> (8 * k)) & 0xFFu;
+                        if (L > 31u) bad = true;
+                        else { atomicAdd(&cnt[L], 1u); atomicAdd(&cnt[32], 1u); }
+                    }
+                }
+            }
+        }
+    }
+    if (__any_sync(kFull, bad) && lane == 0) atomicOr(ws.status, kStBadStream);
+    __syncthreads();
+    if (tid < 33 && cnt[tid]) atomicAdd(hist + tid, (unsigned long long)cnt[tid]);
+}
+
 // ------------------------------------------------------------------------------------------------ quality metrics
 
 // max |x - y|, sum (x - y)^2, min x, max x.  The results are those of fp64 arithmetic, but the per-element work is
@@ -1982,6 +2027,13 @@ cudaError_t launch_quality(const float* x, const float* y, unsigned long long n,
     const unsigned grid = (unsigned)(want < cap ? (want ? want : 1) : cap);
     ++g_launches;
     return launch_k(quality_kernel, dim3(grid), dim3(256), 0, st, x, y, n, out, partials, counter);
+}
+
+cudaError_t launch_stream_stats(const uint32_t* in, unsigned long long cap_bytes, unsigned long long* hist, const Workspace& ws,
+                                int sm_count, cudaStream_t st)
+{
+    ++g_launches;
+    return launch_k(stream_stats_kernel, dim3((unsigned)sm_count * 2), dim3(256), 0, st, in, cap_bytes, hist, ws);
 }
 
 cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st)

@@ -24,7 +24,7 @@ EXPORTS = [
     "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_reduce_scatter", "zccl_sim_scatter",
-    "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_scale",
+    "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_scale", "zccl_stream_stats",
     "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
     "zccl_debug_set_launch_counter",
 ]
@@ -67,6 +67,7 @@ def lib():
         L.zccl_sim_scatter.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
         L.zccl_quality.argtypes = [vp, vp, vp, sz, vp, vp]
         L.zccl_range.argtypes = [vp, vp, sz, vp, vp]
+        L.zccl_stream_stats.argtypes = [vp, vp, sz, vp, vp]
         L.zccl_scale.argtypes = [vp, vp, sz, C.c_float, vp]
         L.zccl_sim_bcast.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
         L.zccl_sim_sizes.argtypes = [vp, vp, C.c_int, vp]
@@ -223,6 +224,11 @@ class Context:
         """zccl_quality: out (float64[6], device) <- max |x - y|, MSE, NRMSE, PSNR, min x, max x."""
         _check(lib().zccl_quality(self._h, _dev_ptr(x, torch.float32), _dev_ptr(y, torch.float32), x.numel(),
                                   _dev_ptr(out, torch.float64), _stream_ptr(stream)), "zccl_quality")
+
+    def stream_stats(self, stream_bytes: torch.Tensor, hist: torch.Tensor, stream=None):
+        """zccl_stream_stats: hist (int64[33], device) <- blocks per code length 0..31, then the number of blocks."""
+        _check(lib().zccl_stream_stats(self._h, _dev_ptr(stream_bytes, torch.uint8), stream_bytes.numel(),
+                                       _dev_ptr(hist, torch.int64), _stream_ptr(stream)), "zccl_stream_stats")
 
     def range(self, x: torch.Tensor, minmax: torch.Tensor, stream=None):
         """zccl_range: minmax (float32[2], device) <- (min x, max x)."""

@@ -696,3 +696,38 @@ def test_range_and_scale_steps_of_a_real_rank(z, ctx):
     assert mm.cpu().numpy().tolist() == [3.0, 3.0]
     with pytest.raises(z.ZcclError):
         ctx.scale(torch.ones(4, device="cuda"), 0.0)
+
+
+@pytest.mark.parametrize("n,eb", [(1, 1e-3), (37, 1e-3), (4096 * 5 + 77, 1e-2), (300_000, 1e-3), (300_000, 1e-5)])
+def test_stream_stats_match_oracle(z, ctx, n, eb):
+    x = fields.smooth_1d(n, seed=n % 89)
+    if n > 1000:
+        x[n // 3: n // 3 + 900] += np.random.default_rng(n).normal(0, 0.2, 900).astype(f32)
+    st, _ = oracle.compress(x, oracle.EB_ABS, eb)
+    hist = torch.full((33,), -1, dtype=torch.int64, device="cuda")
+    ctx.stream_stats(dev(st), hist)
+    assert ctx.status() == z.OK
+    assert np.array_equal(hist.cpu().numpy().astype(np.uint64), oracle.stream_stats(st))
+
+
+def test_stream_stats_constant_and_damaged(z, ctx):
+    x = np.full(10_000, -3.0, f32)
+    st, _ = oracle.compress(x, oracle.EB_ABS, 1e-2)
+    hist = torch.zeros(33, dtype=torch.int64, device="cuda")
+    ctx.stream_stats(dev(st), hist)
+    assert ctx.status() == z.OK
+    h = hist.cpu().numpy()
+    assert h[0] == h[32] == -(-10_000 // 32) and h[1:32].sum() == 0
+    bad = st.copy()
+    bad[32 + 4 * 3 - 1] = 0xFF                     # last index entry far beyond the stream
+    ctx.stream_stats(dev(bad), hist)
+    assert ctx.status() == z.E_BAD_STREAM
+    y = x.copy()
+    y[5000] = 4.0
+    st2, _ = oracle.compress(y, oracle.EB_ABS, 1e-2)
+    bad2 = st2.copy()
+    nT = 3
+    first_L = 32 + 4 * nT + 4                      # first tile: outlier word, then the code-length bytes
+    bad2[first_L] = 77
+    ctx.stream_stats(dev(bad2), hist)
+    assert ctx.status() == z.E_BAD_STREAM
