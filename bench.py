@@ -263,6 +263,31 @@ def _codec_row(z, ctx, name, x_h, mode, eb, with_oracle: bool, loc_h=None):
     return row
 
 
+def _tiled_row(z, ctx, name, x_h, mode, eb, tile):
+    """Compress and decompress through the plain kernels for another tile size (same protocol as _codec_row)."""
+    import torch
+    n = x_h.size
+    nbytes = 4 * n
+    sets = max(2, min(32, -(-4 * L2_BYTES // max(3 * nbytes // 2, 1))))
+    cap = z.compress_bound_tiled(n, tile)
+    xs = [torch.from_numpy(x_h).cuda() for _ in range(sets)]
+    outs = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    ys = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(sets)]
+    sz = torch.zeros(1, dtype=torch.int64, device="cuda")
+    c_mean, c_best = _timed(lambda i: ctx.compress_tiled(xs[i], mode, eb, tile, outs[i], sz), sets)
+    rc = ctx.check()
+    cbytes = int(sz.item())
+    d_mean, d_best = _timed(lambda i: ctx.decompress_tiled(outs[i][:cbytes], tile, ys[i]), sets)
+    ctx.check()
+    return {"config": name, "tile": tile, "n": n, "bytes": nbytes, "bound": ("REL " if mode == z.EB_REL else "ABS ") + f"{eb:g}",
+            "ratio": round(nbytes / cbytes, 3), "status": rc, "buffer_sets": sets,
+            "max_abs_err": float((ys[0].double() - xs[0].double()).abs().max().item()),
+            "compress_us_mean": round(c_mean, 2), "compress_us_best": round(c_best, 2),
+            "compress_gbs": round(nbytes / c_mean / 1e3, 1),
+            "decompress_us_mean": round(d_mean, 2), "decompress_us_best": round(d_best, 2),
+            "decompress_gbs": round(nbytes / d_mean / 1e3, 1)}
+
+
 def config_table(args):
     """Timings of the survey's configurations 0-4 (10 warm-up + 10 timed calls each, mean and best): one JSON line
     per row on stdout.  Not part of the default run."""
@@ -287,6 +312,7 @@ def config_table(args):
         x1, loc1 = fields.fourier_field_3d(SIDE, seed=1), fields.fourier_field_3d(SIDE, seed=2)
         for eb in (1e-2, 1e-3, 1e-4):
             emit(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, orc and eb == 1e-3, loc1))
+        emit(_tiled_row(z, big, "cfg1, tile of 5120 (plain kernels)", x1, z.EB_REL, 1e-3, 5120))
     if "cfg3" in want:
         emit(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, orc))
 

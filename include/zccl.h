@@ -255,6 +255,21 @@ int zccl_sim_sizes(zccl_ctx* ctx, size_t* sizes, int capacity, void* stream);
 int zccl_quality(zccl_ctx* ctx, const float* x, const float* y, size_t n, double* out, void* stream);
 
 /*
+ * Other tile sizes.  The tile (elements per Lorenzo restart and per index entry) is a header field of the stream;
+ * Section 3.5.2 cuts the data into chunks of 5120 points.  The entry points above are built around 4096; these two
+ * take any tile size that is a multiple of 32 between 1024 and 8192, through plain kernels (three launches to
+ * compress, one to decompress) that produce and accept exactly the streams the format defines for that tile size.
+ * Arguments, asynchrony and error reporting are those of zccl_compress and zccl_decompress; a stream whose header
+ * names another tile size than `tile` sets ZCCL_E_BAD_STREAM.  ZCCL_E_ARG also for a tile size outside the range.
+ * zccl_compress_bound_tiled returns 0 for such a tile size.
+ */
+size_t zccl_compress_bound_tiled(size_t n, unsigned tile);
+int zccl_compress_tiled(zccl_ctx* ctx, const float* x, size_t n, int eb_mode, float eb, unsigned tile,
+                        void* out, size_t out_capacity, size_t* out_bytes /*device*/, void* stream);
+int zccl_decompress_tiled(zccl_ctx* ctx, const void* in, size_t in_bytes_max, unsigned tile,
+                          float* y, size_t y_capacity_elems, void* stream);
+
+/*
  * Code-length statistics of a stream (Section 4.1 reports the percentage of constant blocks next to the ratio: a
  * block whose code length is 0 is a constant block and is stored as its one code-length byte).
  *   in   [device] stream, in_bytes_max readable bytes (4-byte aligned)

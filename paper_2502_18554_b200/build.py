@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libzccl.so"
-SOURCES = [CSRC / "zccl_kernels.cu", CSRC / "zccl_api.cu", CSRC / "zccl_noalloc.cu"]
+SOURCES = [CSRC / "zccl_kernels.cu", CSRC / "zccl_api.cu", CSRC / "zccl_noalloc.cu", CSRC / "zccl_generic.cu"]
 HEADERS = [CSRC / "zccl_internal.h", PKG.parent / "include" / "zccl.h"]
 
 NVCC_FLAGS = [

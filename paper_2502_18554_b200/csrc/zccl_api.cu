@@ -16,6 +16,8 @@ struct zccl_ctx {
     size_t max_elems = 0;
     int max_ranks = 0;
     uint32_t debug_epoch = 0;
+    uint32_t* gen_sizes = nullptr;        // device: tile sizes (and, behind them, the go flag) of zccl_compress_tiled
+    size_t gen_tiles = 0;
     double* quality_partials = nullptr;   // device: per-CTA partial results of zccl_quality
     uint32_t* quality_counter = nullptr;
     Workspace ws{};
@@ -238,6 +240,10 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
         ok = cudaMalloc((void**)&c->arena, c->arena_bytes) == cudaSuccess;
     }
     if (ok) {
+        c->gen_tiles = (max_elems + kGenericMinTile - 1) / kGenericMinTile + 1;
+        ok = cudaMalloc((void**)&c->gen_sizes, sizeof(uint32_t) * (c->gen_tiles + 1)) == cudaSuccess;
+    }
+    if (ok) {
         c->stage_c_cap = align_up(bound_of(max_elems), 256);
         ok = cudaMalloc((void**)&c->stage_x, sizeof(float) * max_elems) == cudaSuccess &&
              cudaMalloc((void**)&c->stage_c, c->stage_c_cap) == cudaSuccess;
@@ -252,6 +258,7 @@ void zccl_ctx_destroy(zccl_ctx* c)
     if (!c) return;
     cudaDeviceSynchronize();
     if (c->small_block) cudaFree(c->small_block);
+    if (c->gen_sizes) cudaFree(c->gen_sizes);
     if (c->arena) cudaFree(c->arena);
     if (c->stage_x) cudaFree(c->stage_x);
     if (c->stage_c) cudaFree(c->stage_c);
@@ -661,6 +668,53 @@ int zccl_quality(zccl_ctx* c, const float* x, const float* y, size_t n, double* 
     if (!c || !x || !y || !out || n == 0 || n > c->max_elems) return ZCCL_E_ARG;
     if (((uintptr_t)x & 3u) || ((uintptr_t)y & 3u) || ((uintptr_t)out & 7u)) return ZCCL_E_ARG;
     return cuda_rc(launch_quality(x, y, n, out, c->quality_partials, c->quality_counter, c->sm_count, (cudaStream_t)stream));
+}
+
+static bool tile_ok(unsigned tile)
+{
+    return tile >= (unsigned)kGenericMinTile && tile <= (unsigned)kGenericMaxTile && tile % (unsigned)kBlock == 0;
+}
+
+size_t zccl_compress_bound_tiled(size_t n, unsigned tile)
+{
+    if (!tile_ok(tile)) return 0;
+    const size_t nT = (n + tile - 1) / tile;
+    size_t total = kHeaderBytes + 4 * nT;
+    if (nT == 0) return total;
+    const size_t full = nT - 1, bpt = tile / kBlock;
+    total += full * (4 + ((bpt + 3) & ~(size_t)3) + bpt * 128);
+    const size_t nb = (n - full * tile + kBlock - 1) / kBlock;
+    total += 4 + ((nb + 3) & ~(size_t)3) + nb * 128;
+    return total;
+}
+
+int zccl_compress_tiled(zccl_ctx* c, const float* x, size_t n, int eb_mode, float eb, unsigned tile,
+                        void* out, size_t out_capacity, size_t* out_bytes, void* stream)
+{
+    if (!c || (!x && n) || !out || !out_bytes || !eb_ok(eb_mode, eb) || n > c->max_elems || !tile_ok(tile)) return ZCCL_E_ARG;
+    if (((uintptr_t)x & 3u) || ((uintptr_t)out & 3u)) return ZCCL_E_ARG;
+    const size_t nT = (n + tile - 1) / tile;
+    if (nT > c->gen_tiles) return ZCCL_E_ARG;
+    if (out_capacity < kHeaderBytes + 4 * nT) return ZCCL_E_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    Params hp{};
+    bool dev = false;
+    RangeList rl;
+    rl.x.push_back(x); rl.n.push_back(n);
+    int rc = resolve_bound(c, rl, eb_mode, eb, hp, dev, st);
+    if (rc != ZCCL_OK) return rc;
+    return cuda_rc(launch_generic_encode(x, n, tile, hp, dev, c->gen_sizes, c->gen_sizes + c->gen_tiles, (uint32_t*)out,
+                                         out_capacity, out_bytes, c->ws, c->sm_count, st));
+}
+
+int zccl_decompress_tiled(zccl_ctx* c, const void* in, size_t in_bytes_max, unsigned tile, float* y, size_t y_capacity_elems,
+                          void* stream)
+{
+    if (!c || !in || (!y && y_capacity_elems) || !tile_ok(tile)) return ZCCL_E_ARG;
+    if (((uintptr_t)in & 3u) || ((uintptr_t)y & 3u)) return ZCCL_E_ARG;
+    if (in_bytes_max < (size_t)kHeaderBytes) return ZCCL_E_CAPACITY;
+    return cuda_rc(launch_generic_decode((const uint32_t*)in, in_bytes_max, tile, y, y_capacity_elems, c->ws, c->sm_count,
+                                         (cudaStream_t)stream));
 }
 
 int zccl_stream_stats(zccl_ctx* c, const void* in, size_t in_bytes_max, unsigned long long* hist, void* stream)

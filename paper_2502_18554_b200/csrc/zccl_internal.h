@@ -16,6 +16,8 @@ constexpr int kBlocksPerTile = kTile / kBlock;
 constexpr int kThreads = 256;               // one CTA works on one tile at a time
 constexpr int kWarps = kThreads / 32;
 constexpr int kBlocksPerWarp = kBlocksPerTile / kWarps;   // 16 consecutive blocks per warp
+constexpr int kGenericMinTile = 1024;       // tile sizes the plain kernels of zccl_generic.cu accept (multiples of 32)
+constexpr int kGenericMaxTile = 8192;
 constexpr int kMaxJobs = 64;                // chunk-operations per launch (8 ranks x 7 chunks of a ring stage fit one launch)
 
 // Device status bits (zccl_status maps them to return codes).
@@ -133,6 +135,11 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st);
+cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* sizes,
+                                  uint32_t* go, uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws,
+                                  int sm_count, cudaStream_t st);
+cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, float* y, unsigned long long y_cap,
+                                  const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_stream_stats(const uint32_t* in, unsigned long long cap_bytes, unsigned long long* hist, const Workspace& ws,
                                 int sm_count, cudaStream_t st);
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);

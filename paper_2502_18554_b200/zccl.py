@@ -25,6 +25,7 @@ EXPORTS = [
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_reduce_scatter", "zccl_sim_scatter",
     "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_scale", "zccl_stream_stats",
+    "zccl_compress_bound_tiled", "zccl_compress_tiled", "zccl_decompress_tiled",
     "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
     "zccl_debug_set_launch_counter",
 ]
@@ -68,6 +69,10 @@ def lib():
         L.zccl_quality.argtypes = [vp, vp, vp, sz, vp, vp]
         L.zccl_range.argtypes = [vp, vp, sz, vp, vp]
         L.zccl_stream_stats.argtypes = [vp, vp, sz, vp, vp]
+        L.zccl_compress_bound_tiled.argtypes = [sz, C.c_uint]
+        L.zccl_compress_bound_tiled.restype = sz
+        L.zccl_compress_tiled.argtypes = [vp, vp, sz, C.c_int, C.c_float, C.c_uint, vp, sz, vp, vp]
+        L.zccl_decompress_tiled.argtypes = [vp, vp, sz, C.c_uint, vp, sz, vp]
         L.zccl_scale.argtypes = [vp, vp, sz, C.c_float, vp]
         L.zccl_sim_bcast.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
         L.zccl_sim_sizes.argtypes = [vp, vp, C.c_int, vp]
@@ -82,6 +87,10 @@ def lib():
 
 def compress_bound(n: int) -> int:
     return int(lib().zccl_compress_bound(n))
+
+
+def compress_bound_tiled(n: int, tile: int) -> int:
+    return int(lib().zccl_compress_bound_tiled(n, tile))
 
 
 def launch_count() -> int:
@@ -224,6 +233,20 @@ class Context:
         """zccl_quality: out (float64[6], device) <- max |x - y|, MSE, NRMSE, PSNR, min x, max x."""
         _check(lib().zccl_quality(self._h, _dev_ptr(x, torch.float32), _dev_ptr(y, torch.float32), x.numel(),
                                   _dev_ptr(out, torch.float64), _stream_ptr(stream)), "zccl_quality")
+
+    def compress_tiled(self, x: torch.Tensor, eb_mode: int, eb: float, tile: int, out: torch.Tensor, out_bytes: torch.Tensor,
+                       stream=None):
+        """zccl_compress_tiled: as compress, for a tile size other than 4096 (multiple of 32 in 1024..8192)."""
+        n = x.numel()
+        _check(lib().zccl_compress_tiled(self._h, _dev_ptr(x, torch.float32) if n else None, n, eb_mode, eb, tile,
+                                         _dev_ptr(out, torch.uint8), out.numel(), _dev_ptr(out_bytes, torch.int64),
+                                         _stream_ptr(stream)), "zccl_compress_tiled")
+
+    def decompress_tiled(self, stream_bytes: torch.Tensor, tile: int, y: torch.Tensor, stream=None):
+        """zccl_decompress_tiled: as decompress, for a stream of tile size `tile`."""
+        _check(lib().zccl_decompress_tiled(self._h, _dev_ptr(stream_bytes, torch.uint8), stream_bytes.numel(), tile,
+                                           _dev_ptr(y, torch.float32) if y.numel() else None, y.numel(),
+                                           _stream_ptr(stream)), "zccl_decompress_tiled")
 
     def stream_stats(self, stream_bytes: torch.Tensor, hist: torch.Tensor, stream=None):
         """zccl_stream_stats: hist (int64[33], device) <- blocks per code length 0..31, then the number of blocks."""

@@ -65,3 +65,15 @@ def test_binding_refuses_to_run_without_gpu():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError):
         zccl.Context(1 << 20)
+
+
+def test_compress_bound_for_other_tile_sizes_is_the_oracles():
+    """Pure host arithmetic of the library (no GPU involved) against the oracle's worst case: every block at 31 bits
+    plus its sign word, per tile an outlier, the padded code-length bytes and an index entry."""
+    import oracle
+    from paper_2502_18554_b200 import zccl
+    for T in (1024, 4096, 5120, 8192):
+        for n in (0, 1, 31, 32, 33, T - 1, T, T + 1, 7 * T + 100, 1 << 24):
+            assert zccl.compress_bound_tiled(n, T) == oracle.compress_bound(n, T)
+    assert zccl.compress_bound_tiled(1000, 5000) == 0 and zccl.compress_bound_tiled(1000, 512) == 0
+    assert zccl.compress_bound_tiled(12345, 4096) == zccl.compress_bound(12345)

@@ -731,3 +731,69 @@ def test_stream_stats_constant_and_damaged(z, ctx):
     bad2[first_L] = 77
     ctx.stream_stats(dev(bad2), hist)
     assert ctx.status() == z.E_BAD_STREAM
+
+
+# ----------------------------------------------------------------------------- other tile sizes (plain kernels)
+
+def _tiled_case(z, ctx, x, mode, eb, T):
+    want, wrc = oracle.compress(x, mode, eb, T)
+    out = torch.full((z.compress_bound_tiled(x.size, T) + 64,), 0xCD, dtype=torch.uint8, device="cuda")
+    cap = out.numel() - 64
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx.compress_tiled(dev(x), mode, eb, T, out[:cap], nb)
+    assert ctx.status() == wrc
+    got = out[: int(nb.item())].cpu().numpy()
+    assert got.size == want.size and np.array_equal(got, want)
+    assert bool((out[cap:] == 0xCD).all())
+    y = torch.full((x.size + 16,), 7.0, dtype=torch.float32, device="cuda")
+    ctx.decompress_tiled(dev(want), T, y[: x.size])
+    assert ctx.status() == z.OK
+    assert_same_bits(y[: x.size].cpu().numpy(), oracle.decompress(want))
+    assert bool((y[x.size:] == 7.0).all())
+    return want
+
+
+@pytest.mark.parametrize("T", [5120, 1024, 8192, 4096, 4128])
+@pytest.mark.parametrize("n", [1, 33, 5119, 5120, 5121, 3 * 5120 + 77, 200_001])
+def test_other_tile_sizes_match_oracle(z, ctx, T, n):
+    # Section 3.5.2: chunks of 5120 points; the tile size is a header field, the oracle takes any
+    x = fields.smooth_1d(n, seed=T % 97 + n % 13)
+    if n > 3000:
+        x[n // 2: n // 2 + 1500] += np.random.default_rng(n).normal(0, 0.4, 1500).astype(f32)
+    _tiled_case(z, ctx, x, z.EB_REL if n > 1 else z.EB_ABS, 1e-3, T)
+    _tiled_case(z, ctx, x, z.EB_ABS, 3e-6, T)       # long codes, precision warning on the larger arrays
+
+
+def test_tile_4096_streams_of_both_routes_are_the_same(z, ctx):
+    x = fields.fourier_field_3d(64, seed=5)
+    a = _tiled_case(z, ctx, x, z.EB_REL, 1e-3, 4096)
+    b, _ = gpu_compress(z, ctx, x, z.EB_REL, 1e-3)
+    assert np.array_equal(a, b)
+
+
+def test_other_tile_sizes_errors(z, ctx):
+    x = fields.smooth_1d(30_000, seed=8)
+    want, _ = oracle.compress(x, oracle.EB_REL, 1e-3, 5120)
+    out = torch.full((want.size + 64,), 0xCD, dtype=torch.uint8, device="cuda")
+    nb = torch.ones(1, dtype=torch.int64, device="cuda")
+    ctx.compress_tiled(dev(x), z.EB_REL, 1e-3, 5120, out[: want.size - 8], nb)      # too small: nothing is written
+    assert ctx.status() == z.E_CAPACITY
+    assert int(nb.item()) == 0 and bool((out == 0xCD).all())
+    with pytest.raises(z.ZcclError):
+        ctx.compress_tiled(dev(x), z.EB_REL, 1e-3, 5000, out, nb)                   # not a multiple of 32
+    with pytest.raises(z.ZcclError):
+        ctx.compress_tiled(dev(x), z.EB_REL, 1e-3, 512, out, nb)                    # below the supported range
+    y = torch.zeros(x.size, dtype=torch.float32, device="cuda")
+    ctx.decompress_tiled(dev(want), 4096, y)                                        # the header says 5120
+    assert ctx.status() == z.E_BAD_STREAM
+    ctx.decompress(dev(want), y)                                                    # the tuned decoder is for 4096
+    assert ctx.status() == z.E_BAD_STREAM
+    ctx.decompress_tiled(dev(want), 5120, y[:100])                                  # output too small
+    assert ctx.status() == z.E_CAPACITY
+    bad = want.copy()
+    bad[32 + 4 * 6 + 4] = 40                                                        # a code length above 31
+    ctx.decompress_tiled(dev(bad), 5120, y)
+    assert ctx.status() == z.E_BAD_STREAM
+    const = np.full(9000, 1.25, f32)
+    ctx.compress_tiled(dev(const), z.EB_REL, 1e-3, 5120, out, nb)                   # no range to relate the bound to
+    assert ctx.status() == z.E_DEGENERATE and int(nb.item()) == 0
