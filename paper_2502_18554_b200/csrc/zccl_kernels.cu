@@ -713,8 +713,11 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
                 for (int w = 0; w < warp; ++w) base = __fadd_rn(base, sh.warp_total[par][w]);
                 base = __fadd_rn(base, before);   // all of these are integers below 2^24: any order of addition is exact
                 par ^= 1u;
-                float4* dst = reinterpret_cast<float4*>(y + 512 * warp + 16 * lane);
-                const bool vec = (((uintptr_t)dst) & 15u) == 0;
+                // A thread holds 16 consecutive elements; stored from there, a 128-bit store would touch 32 separate
+                // 64-byte pieces and be replayed.  The values go back through the warp's rows instead (same swizzle as
+                // the deltas), so that store c of the warp writes 512 consecutive bytes.
+                float4* wrow = reinterpret_cast<float4*>(sh.wbuf[warp]);
+                const int sw = (lane >> 1) & 3;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     float4 o;
@@ -722,9 +725,18 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
                     o.y = __fmul_rn(__fadd_rn(v[4 * c + 1], base), h.s);
                     o.z = __fmul_rn(__fadd_rn(v[4 * c + 2], base), h.s);
                     o.w = __fmul_rn(__fadd_rn(v[4 * c + 3], base), h.s);
-                    if (vec) dst[c] = o;
+                    wrow[4 * lane + (c ^ sw)] = o;
+                }
+                __syncwarp();
+                float4* dst = reinterpret_cast<float4*>(y + 512 * warp);
+                const bool vec = (((uintptr_t)dst) & 15u) == 0;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int f = 32 * c + lane, t = f >> 2;           // float4 number f of the warp's 128: thread t's
+                    const float4 o = wrow[4 * t + ((f & 3) ^ ((t >> 1) & 3))];
+                    if (vec) dst[f] = o;
                     else {
-                        float* ds = reinterpret_cast<float*>(dst + c);
+                        float* ds = reinterpret_cast<float*>(dst + f);
                         ds[0] = o.x; ds[1] = o.y; ds[2] = o.z; ds[3] = o.w;
                     }
                 }
@@ -1523,9 +1535,20 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                 const bool store = gout != nullptr && !deq;
                 const bool gvec = (((uintptr_t)yout) & 15u) == 0;
                 if (summing && lvec && (!store || gvec)) {
+                    // Global accesses are made warp-contiguous (access c of the warp covers 512 consecutive bytes)
+                    // and the 16 consecutive elements a thread works on are exchanged through the warp's rows, whose
+                    // deltas the scan has consumed: a 128-bit access with the lanes 64 bytes apart is replayed.
+                    float4* row_w = reinterpret_cast<float4*>(yrows + 32);
+                    const float4* lw = reinterpret_cast<const float4*>(loc + 512 * warp);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int f = 32 * c + lane, t = f >> 2;
+                        row_w[4 * t + ((f & 3) ^ ((t >> 1) & 3))] = __ldg(lw + f);
+                    }
+                    __syncwarp();
                     float4 l[4];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) l[c] = __ldg(reinterpret_cast<const float4*>(lp) + c);
+                    for (int c = 0; c < 4; ++c) l[c] = row[c ^ sw];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         float4 o;
@@ -1534,7 +1557,15 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
                         o.z = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 2], base), s), l[c].z);
                         o.w = __fadd_rn(__fmul_rn(__fadd_rn(v[4 * c + 3], base), s), l[c].w);
                         row[c ^ sw] = o;
-                        if (store) gout[c] = o;
+                    }
+                    if (store) {
+                        __syncwarp();
+                        float4* gw = reinterpret_cast<float4*>(yout + 512 * warp);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int f = 32 * c + lane, t = f >> 2;
+                            gw[f] = row_w[4 * t + ((f & 3) ^ ((t >> 1) & 3))];
+                        }
                     }
                 } else {
 #pragma unroll
