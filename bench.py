@@ -289,7 +289,7 @@ def _tiled_row(z, ctx, name, x_h, mode, eb, tile):
 
 
 def config_table(args):
-    """Timings of the survey's configurations 0-4 (10 warm-up + 10 timed calls each, mean and best): one JSON line
+    """Timings of the workload configurations 0-4 (10 warm-up + 10 timed calls each, mean and best): one JSON line
     per row on stdout.  Not part of the default run."""
     import torch
     from paper_2502_18554_b200 import build, fields, zccl as z
