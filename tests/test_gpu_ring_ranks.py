@@ -80,7 +80,7 @@ def _run(world, n, segments):
     return got
 
 
-@pytest.mark.parametrize("world,n,segments", [(2, 100000, 1), (3, 70001, 2), (4, 5, 1)])
+@pytest.mark.parametrize("world,n,segments", [(2, 100000, 1), (3, 70001, 2), (4, 5, 1), (2, 9000, 4)])
 def test_cuda_ranks_match_the_oracle_ring(world, n, segments):
     import oracle
     got = _run(world, n, segments)

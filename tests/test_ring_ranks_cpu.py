@@ -116,7 +116,8 @@ def _run(world, n, segments, transport):
 
 
 @pytest.mark.parametrize("world,n,segments,transport", [(2, 20000, 1, "host"), (3, 20000, 2, "host"), (4, 9001, 3, "direct"),
-                                                       (3, 2, 1, "host"), (2, 30000, 2, "direct"), (3, 20000, 1, "direct")])
+                                                       (3, 2, 1, "host"), (2, 30000, 2, "direct"), (3, 20000, 1, "direct"),
+                                                       (2, 5000, 8, "direct")])     # more pieces than tiles: empty pieces travel too
 def test_real_rank_collectives_match_the_emulated_ones(world, n, segments, transport):
     """"direct" keeps the payload messages in flight behind the codec steps and waits for each where its data is
     needed (the bookkeeping an NCCL group runs with); "host" waits for every message where it is posted."""
