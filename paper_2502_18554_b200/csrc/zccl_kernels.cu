@@ -430,8 +430,8 @@ __device__ __forceinline__ void decode_blocks_int(const TileDesc& d, int warp, i
 // fp32 path: rebuilds this warp's 16 blocks of deltas from the staged blob and stores them, as exact floats, in
 // the warp's 512-word region `wbuf`, row i = block i, element j of a row at word j ^ ((i & 3) << 2) (so that the
 // 128-bit reads of decode_scan_f32 are free of bank conflicts).  tbl: per block {code length, payload address}.
-// UNROLL: the fused hop unrolls the loop over the groups of four (fewer instructions, 75 -> 73 us); the decoder,
-// at its 46 registers, is faster with the loop kept.
+// UNROLL: the fused hop unrolls the loop over the groups of four completely (fewer instructions, 75 -> 73 us); the
+// decoder, at its 48 registers, is fastest with two groups per iteration (35.2 -> 34.4 us; 35.2 again with four).
 template <int UNROLL>
 __device__ __forceinline__ void decode_blocks_f32(const uint2* __restrict__ tbl, float* __restrict__ wbuf, int lane,
                                                   const Xpose& xp)
@@ -701,7 +701,7 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
             if (mode == 0) { status |= kStBadStream; skip_tile = true; }
             if (mode == 1) {
                 float* __restrict__ y = job.y + (unsigned long long)tile * kTile;
-                decode_blocks_f32<1>(sh.tbl + kBlocksPerWarp * warp, sh.wbuf[warp], lane, xp);
+                decode_blocks_f32<2>(sh.tbl + kBlocksPerWarp * warp, sh.wbuf[warp], lane, xp);
                 __syncwarp();
                 float v[16];
                 float before;
