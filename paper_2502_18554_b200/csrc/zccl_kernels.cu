@@ -821,7 +821,7 @@ struct SrcSwizzled {        // the fused kernel's sum tile: per-warp region of 1
 // the caller checks `guard` (sum of squares of x * r over the warp's elements and the one before them) and reruns
 // with FAST = false when it is too large.  FAST handles four blocks per bit-matrix transpose while their code
 // lengths are at most 7 (sign + 7 magnitude bits of four elements share a word), else one block per transpose.
-template <bool FAST, class Src>
+template <bool FAST, int UNROLL = 4, class Src>
 __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint32_t* __restrict__ slots_w, int lane,
                                                   const Xpose& xp, uint32_t& my_lw, float& guard, float& tmax)
 {
@@ -834,8 +834,8 @@ __device__ __forceinline__ uint32_t encode_blocks(const Src& src, float r, uint3
         const float tp0 = __fmul_rn(src.prev(0, 0), r);
         if (lane == 0) acc = __fmul_rn(tp0, tp0);
     }
-#pragma unroll
-    for (int g = 0; g < kBlocksPerWarp / 4; ++g) {   // unrolled: constant offsets, 5 % fewer instructions
+#pragma unroll UNROLL
+    for (int g = 0; g < kBlocksPerWarp / 4; ++g) {   // unrolled by default: constant offsets, 5 % fewer instructions
         uint32_t lword = 0;
         if (FAST) {
             uint32_t ab[4], db[4];
@@ -958,11 +958,14 @@ struct EncodeShared {
     alignas(8) unsigned long long bar;
 };
 
-struct FusedShared {
-    alignas(16) uint32_t blob[2][kBlobStageWords];                   // staged blobs: current tile and the next one
+// COMPACT: the kernel instance for launches whose tiles all fit the device at once, one tile per CTA: nothing is
+// double buffered, which leaves room for one more CTA per SM.
+template <bool COMPACT>
+struct FusedSharedT {
+    alignas(16) uint32_t blob[COMPACT ? 1 : 2][kBlobStageWords];     // staged blobs: current tile and the next one
     alignas(16) float ybuf[kWarps][(kBlocksPerWarp + 1) * kBlock];   // deltas, then sums (row 0 of a warp = guard)
     alignas(16) uint2 tbl[kBlocksPerTile];
-    alignas(16) uint32_t slots[2][kBlocksPerTile * kSlotWords];
+    alignas(16) uint32_t slots[COMPACT ? 1 : 2][kBlocksPerTile * kSlotWords];
     BlobSpan span[2];
     float warp_total[kWarps];
     int32_t warp_total_i[kWarps];
@@ -972,6 +975,8 @@ struct FusedShared {
     ScanShared scan;
     alignas(8) unsigned long long bar[2];
 };
+using FusedShared = FusedSharedT<false>;
+using FusedSharedCompact = FusedSharedT<true>;
 
 // A raw-mode tile can be staged by a bulk copy when it is full and starts on a 16-byte boundary.
 __device__ __forceinline__ bool stageable_raw(const Job& job, uint32_t tile)
@@ -1389,11 +1394,13 @@ __global__ void __launch_bounds__(kThreads, 4) encode_raw_kernel(JobBatch jb, Wo
 // ------------------------------------------------------------------------------------------------ fused hop
 
 // out = compress(decompress(in_c) + local) per tile, with no uncompressed intermediate in global memory.
-__global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, Workspace ws)
+template <bool COMPACT>
+__global__ void __launch_bounds__(kThreads, COMPACT ? 4 : 3) encode_fused_kernel(JobBatch jb, Workspace ws)
 {
     pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    FusedShared& sh = *reinterpret_cast<FusedShared*>(smem_raw);
+    using Shared = FusedSharedT<COMPACT>;
+    Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
     const uint32_t G = gridDim.x;
@@ -1427,19 +1434,19 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
     if (tid == 32) {
         pipe.fetch(jb, blockIdx.x, cur_job, h1);
         pipe.stage(sh, jb, blockIdx.x, cur_job, h1, 0);
-        pipe.fetch(jb, blockIdx.x + G, cur_job, h1);
+        if (!COMPACT) pipe.fetch(jb, blockIdx.x + G, cur_job, h1);
     }
     __syncthreads();
     // requests the next tile's blob into the other staging buffer (its readers finished before the last barrier), then
     // fetches the index entries of the tile after it; a barrier follows before the span is read
     auto stage_next = [&](uint32_t ticket) {
-        if (tid == 32) {
+        if (!COMPACT && tid == 32) {   // a compact launch has one tile per CTA: nothing comes next
             pipe.stage(sh, jb, ticket + G, cur_job, h1, p ^ 1u);
             pipe.fetch(jb, ticket + 2 * G, cur_job, h1);
         }
     };
 
-    for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += G, p ^= 1u) {
+    for (uint32_t ticket = blockIdx.x; ticket < jb.total_tiles; ticket += G, p ^= (COMPACT ? 0u : 1u)) {
         const int j = find_job(jb, ticket);
         const Job& job = jb.job[j];
         const uint32_t tile = ticket - job.tile_begin;
@@ -1507,7 +1514,7 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
             mode = describe_staged(sh.tbl, sb, sp.w_end - sp.w_beg, lane, warp);
             if (mode == 0) bad_tile = true;
             if (mode == 1) {
-                decode_blocks_f32<4>(sh.tbl + kBlocksPerWarp * warp, yrows + 32, lane, xp);
+                decode_blocks_f32<(COMPACT ? 1 : 4)>(sh.tbl + kBlocksPerWarp * warp, yrows + 32, lane, xp);
                 __syncwarp();
                 // lane 0 needs the local operand's element before the warp's first one after the barrier below
                 const float lprev = (lane == 0 && warp != 0) ? __ldg(loc + 512 * warp - 1) : 0.0f;
@@ -1647,11 +1654,11 @@ __global__ void __launch_bounds__(kThreads, 3) encode_fused_kernel(JobBatch jb, 
         int32_t q_first = 0;
         float guard = 0.0f, tmax = 0.0f;
         const SrcSwizzled src(yrows, lane);
-        wsum = encode_blocks<true>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
+        wsum = encode_blocks<true, (COMPACT ? 1 : 4)>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
         q_first = first_code<true>(src.cur(0, 0), r);
         const bool need_int = __any_sync(kFull, !(guard < kGuardExact));
         if (need_int) {
-            wsum = encode_blocks<false>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
+            wsum = encode_blocks<false, (COMPACT ? 1 : 4)>(src, r, slots_w, lane, xp, my_lw, guard, tmax);
             q_first = first_code<false>(src.cur(0, 0), r);
             if (!(tmax < 1073741824.0f)) status |= kStRange;
             else if (tmax > 32768.5f) status |= kStPrecision;
@@ -1942,7 +1949,7 @@ __global__ void __launch_bounds__(256) quality_kernel(const float* __restrict__ 
     }
 }
 
-int g_raw_ctas_per_sm = 0, g_fused_ctas_per_sm = 0, g_decode_ctas_per_sm = 0;
+int g_raw_ctas_per_sm = 0, g_fused_ctas_per_sm = 0, g_decode_ctas_per_sm = 0, g_compact_ctas_per_sm = 0;
 unsigned long long g_launches = 0;   // kernels launched by this library in this process
 
 }  // namespace
@@ -1957,6 +1964,15 @@ unsigned long long launch_count() { return g_launches; }
 // CTAs dispatched onto SMs that still run another kernel's CTAs do not all fit (the SM keeps that kernel's
 // shared-memory configuration), which left part of the grid waiting behind the resident part.  The other kernels
 // make no such assumption: tiles handed out by a counter, or CTAs that never wait for one another.
+// ZCCL_COMPACT in the environment: 0 never use the compact instance of the fused kernel, 1 (default) use it for
+// launches that exceed the persistent instance's resident CTAs but fit the compact one's, 2 use it whenever the
+// tiles fit (measured: a little faster up to 128 tiles, slower at 256).
+static int compact_mode()
+{
+    static const int m = [] { const char* e = getenv("ZCCL_COMPACT"); return e ? atoi(e) : 1; }();
+    return m;
+}
+
 static bool pdl_enabled()
 {
     static const bool on = [] { const char* e = getenv("ZCCL_PDL"); return !(e && e[0] == '0'); }();
@@ -1999,13 +2015,17 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
         cudaError_t e = cudaFuncSetAttribute(encode_raw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)sizeof(EncodeShared));
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(encode_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FusedShared));
+        e = cudaFuncSetAttribute(encode_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FusedShared));
         if (e != cudaSuccess) return e;
-        int a = 0, b = 0;
+        e = cudaFuncSetAttribute(encode_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FusedSharedCompact));
+        if (e != cudaSuccess) return e;
+        int a = 0, b = 0, c = 0;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_raw_kernel, kThreads, sizeof(EncodeShared));
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, encode_fused_kernel, kThreads, sizeof(FusedShared));
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, encode_fused_kernel<false>, kThreads, sizeof(FusedShared));
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c, encode_fused_kernel<true>, kThreads, sizeof(FusedSharedCompact));
         g_raw_ctas_per_sm = a > 0 ? a : 1;
         g_fused_ctas_per_sm = b > 0 ? b : 1;
+        g_compact_ctas_per_sm = c > 0 ? c : 1;
     }
     const int per_sm = mode == kEncodeRaw ? g_raw_ctas_per_sm : g_fused_ctas_per_sm;
     unsigned long long cap = (unsigned long long)sm_count * per_sm;
@@ -2013,8 +2033,12 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
     ++g_launches;
     if (mode == kEncodeRaw)
         return launch_k(encode_raw_kernel, dim3(grid), dim3(kThreads), sizeof(EncodeShared), st, jb, ws, host_params, device_params ? 1 : 0);
-    else
-        return launch_k<false>(encode_fused_kernel, dim3(grid), dim3(kThreads), sizeof(FusedShared), st, jb, ws);
+    // a fused launch whose tiles fit the device at once, but not at the persistent kernel's occupancy, runs as one
+    // tile per CTA on the compact instance (no second wave of tiles behind the first)
+    const unsigned long long compact_cap = (unsigned long long)sm_count * g_compact_ctas_per_sm;
+    if ((jb.total_tiles > cap || compact_mode() == 2) && jb.total_tiles <= compact_cap && compact_mode() != 0)
+        return launch_k<false>(encode_fused_kernel<true>, dim3((unsigned)jb.total_tiles), dim3(kThreads), sizeof(FusedSharedCompact), st, jb, ws);
+    return launch_k<false>(encode_fused_kernel<false>, dim3(grid), dim3(kThreads), sizeof(FusedShared), st, jb, ws);
 }
 
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)

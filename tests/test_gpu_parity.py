@@ -797,3 +797,38 @@ def test_other_tile_sizes_errors(z, ctx):
     const = np.full(9000, 1.25, f32)
     ctx.compress_tiled(dev(const), z.EB_REL, 1e-3, 5120, out, nb)                   # no range to relate the bound to
     assert ctx.status() == z.E_DEGENERATE and int(nb.item()) == 0
+
+
+# ----------------------------------------------------------------------------- one-wave launches of the fused hop
+
+def test_fused_hop_launches_that_fit_the_device_at_once(z, ctx):
+    """A fused launch of more tiles than the persistent kernel holds at once (3 CTAs per SM) but not more than the
+    compact instance does (4 per SM) runs as one tile per CTA; the streams must not depend on which instance ran."""
+    props = torch.cuda.get_device_properties(0)
+    sms = props.multi_processor_count
+    for tiles in (3 * sms + 1, 3 * sms + sms // 2, 4 * sms):
+        n = tiles * 4096 - 1000                      # ragged last tile
+        if n > ctx.max_elems:
+            pytest.skip("context too small for this device")
+        a = fields.smooth_1d(n, seed=tiles % 50)
+        b = fields.smooth_1d(n, seed=tiles % 50 + 1)
+        sa, _ = oracle.compress(a, oracle.EB_REL, 1e-3)
+        want, wrc, wraw = oracle.drc(sa, local=b, want_raw=True)
+        got, rc, raw = _drc_gpu(z, ctx, sa, n, local=b, raw=True)
+        assert rc == wrc
+        assert np.array_equal(got, want)
+        assert_same_bits(raw, wraw)
+
+
+def test_allreduce_whose_hops_fit_the_device_at_once(z):
+    """8 ranks x 8 MiB: every reduce-scatter hop is 8 jobs of 64 tiles = 512 tiles in one launch."""
+    N, n = 8, 1 << 21
+    c = z.Context(n, N)
+    send = fields.rank_fields(N, n, base_seed=300, kind="smooth")
+    want, wrc = oracle.sim_allreduce(send, oracle.EB_REL, 1e-3)
+    recv = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(N)]
+    c.sim_allreduce([dev(a) for a in send], recv, z.EB_REL, 1e-3)
+    assert c.status() == wrc
+    for r in range(N):
+        assert_same_bits(recv[r].cpu().numpy(), want[r])
+    c.close()
