@@ -1844,7 +1844,7 @@ __global__ void __launch_bounds__(256) stream_stats_kernel(const uint32_t* __res
 // residual); the sum as a compensated fp32 pair.  A group of elements in which some difference is not an fp32
 // number takes the fp64 path.  128-bit loads, per-thread accumulators, warp shuffles, one partial per CTA, and the
 // last CTA to finish combines the partials in CTA order and writes the six results.
-__global__ void __launch_bounds__(256) quality_kernel(const float* __restrict__ x, const float* __restrict__ y, unsigned long long n,
+__global__ void __launch_bounds__(256, 4) quality_kernel(const float* __restrict__ x, const float* __restrict__ y, unsigned long long n,
                                                       double* __restrict__ out, double* __restrict__ partials, uint32_t* counter)
 {
     pdl_enter();
@@ -1852,9 +1852,13 @@ __global__ void __launch_bounds__(256) quality_kernel(const float* __restrict__ 
     __shared__ uint32_t is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000), emax = 0.0f;
-    float sh = 0.0f, sl = 0.0f;     // compensated sum of squares of the differences that are fp32 numbers
+    // compensated sums of squares of the differences that are fp32 numbers: eight independent ones (one per element
+    // of the two 128-bit loads in flight), so that consecutive elements do not wait for each other's additions
+    float sh8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, sl8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     double dmax = 0.0, dsum = 0.0;  // the others
-    auto take = [&](float a, float b) {
+    auto take = [&](float a, float b, int k) {
+        float& sh = sh8[k];
+        float& sl = sl8[k];
         lo = fminf(lo, a);
         hi = fmaxf(hi, a);
         const float d = __fsub_rn(a, b);
@@ -1882,17 +1886,20 @@ __global__ void __launch_bounds__(256) quality_kernel(const float* __restrict__ 
         unsigned long long i = gtid;
         for (; i + nth < nv; i += 2 * nth) {   // two independent pairs of loads in flight
             const float4 a0 = __ldg(x4 + i), b0 = __ldg(y4 + i), a1 = __ldg(x4 + i + nth), b1 = __ldg(y4 + i + nth);
-            take(a0.x, b0.x); take(a0.y, b0.y); take(a0.z, b0.z); take(a0.w, b0.w);
-            take(a1.x, b1.x); take(a1.y, b1.y); take(a1.z, b1.z); take(a1.w, b1.w);
+            take(a0.x, b0.x, 0); take(a0.y, b0.y, 1); take(a0.z, b0.z, 2); take(a0.w, b0.w, 3);
+            take(a1.x, b1.x, 4); take(a1.y, b1.y, 5); take(a1.z, b1.z, 6); take(a1.w, b1.w, 7);
         }
         for (; i < nv; i += nth) {
             const float4 a = __ldg(x4 + i), b = __ldg(y4 + i);
-            take(a.x, b.x); take(a.y, b.y); take(a.z, b.z); take(a.w, b.w);
+            take(a.x, b.x, 0); take(a.y, b.y, 1); take(a.z, b.z, 2); take(a.w, b.w, 3);
         }
         done = nv << 2;
     }
-    for (unsigned long long i = done + gtid; i < n; i += nth) take(__ldg(x + i), __ldg(y + i));
-    double maxerr = fmax(dmax, (double)emax), sumsq = dsum + ((double)sh + (double)sl);
+    for (unsigned long long i = done + gtid; i < n; i += nth) take(__ldg(x + i), __ldg(y + i), 0);
+    double sumsq = dsum;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) sumsq += (double)sh8[k] + (double)sl8[k];   // fixed order
+    double maxerr = fmax(dmax, (double)emax);
     double dlo = (double)lo, dhi = (double)hi;
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
@@ -2077,7 +2084,13 @@ cudaError_t launch_quality(const float* x, const float* y, unsigned long long n,
                            uint32_t* counter, int sm_count, cudaStream_t st)
 {
     unsigned long long want = (n / 4 + 255) / 256;
-    unsigned long long cap = (unsigned long long)sm_count * 6;
+    static int per_sm = 0;     // one wave of resident CTAs, each striding over the arrays
+    if (per_sm == 0) {
+        int a = 0;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, quality_kernel, 256, 0);
+        per_sm = a > 0 ? a : 1;
+    }
+    unsigned long long cap = (unsigned long long)sm_count * per_sm;
     if (cap > (unsigned long long)kQualityCtas) cap = kQualityCtas;
     const unsigned grid = (unsigned)(want < cap ? (want ? want : 1) : cap);
     ++g_launches;
