@@ -548,10 +548,10 @@ struct StagePipe {
     int n_job = -1;
 
     // index entries of tile number t of the launch
-    __device__ __forceinline__ void fetch(const JobBatch& jb, uint32_t t, int cur_job, const StreamInfo& h)
+    __device__ __forceinline__ void fetch(const JobBatch& jb, uint32_t t, int cur_job, const StreamInfo& h, uint32_t limit = 0xFFFFFFFFu)
     {
         n_job = -1;
-        if (t >= jb.total_tiles) return;
+        if (t >= jb.total_tiles || t >= limit) return;   // limit: end of the CTA's own range of tiles
         const int jj = find_job(jb, t);
         const Job& jq = jb.job[jj];
         const uint32_t tl = t - jq.tile_begin;
@@ -647,7 +647,12 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
     pdl_enter();
     __shared__ DecodeShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t G = gridDim.x;
+    // every CTA takes a run of consecutive tiles: their blobs and index entries are neighbours in the stream, and in a
+    // launch of many short jobs (the chunks of a ring) a CTA stays inside one job instead of changing it with every tile
+    // (the first `rem` CTAs take one tile more than the others, as dealing them round-robin would give them)
+    const uint32_t quo = jb.total_tiles / gridDim.x, rem = jb.total_tiles % gridDim.x;
+    const uint32_t g0 = blockIdx.x * quo + (blockIdx.x < rem ? blockIdx.x : rem);
+    const uint32_t g1 = g0 + quo + (blockIdx.x < rem ? 1u : 0u);
     uint32_t status = 0;
     uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed per staging buffer (phase parity of its mbarrier)
     uint32_t par = 0;                  // parity of the warp_total double buffer
@@ -663,13 +668,13 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
         mbar_init(&sh.bar[0], 1);
         mbar_init(&sh.bar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        pipe.fetch(jb, blockIdx.x, cur_job, h);
-        pipe.stage(sh, jb, blockIdx.x, cur_job, h, 0);
-        pipe.fetch(jb, blockIdx.x + G, cur_job, h);
+        pipe.fetch(jb, g0, cur_job, h, g1);
+        pipe.stage(sh, jb, g0, cur_job, h, 0);
+        pipe.fetch(jb, g0 + 1, cur_job, h, g1);
     }
     __syncthreads();
 
-    for (uint32_t g = blockIdx.x; g < jb.total_tiles; g += G) {
+    for (uint32_t g = g0; g < g1; ++g) {
         const int j = find_job(jb, g);
         const Job& job = jb.job[j];
         if (j != cur_job) { h = read_header(job.in_c, job.in_cap); cur_job = j; }
@@ -678,8 +683,8 @@ __global__ void __launch_bounds__(kThreads, 5) decode_kernel(JobBatch jb, Worksp
         // thread 0: request the next tile's blob into the other buffer (its readers finished before the last barrier
         // of the previous iteration), then fetch the index entries of the tile after it
         if (tid == 0) {
-            pipe.stage(sh, jb, g + G, cur_job, h, p ^ 1u);
-            pipe.fetch(jb, g + 2 * G, cur_job, h);
+            pipe.stage(sh, jb, g + 1, cur_job, h, p ^ 1u);
+            pipe.fetch(jb, g + 2, cur_job, h, g1);
         }
         const BlobSpan sp = sh.span[p];
         if (sp.staged) {   // a copy was requested for this tile: always consume it, whatever happens next
