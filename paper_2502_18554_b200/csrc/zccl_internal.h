@@ -41,6 +41,7 @@ struct Params {
 // Scan / bookkeeping workspace owned by the context.
 struct Workspace {
     unsigned long long* tile_state;  // one 64-bit {epoch:31 | inclusive:1 | words:32} per tile of a launch
+    unsigned long long* group_state; // the same per group of 32 consecutive tiles of a job: group_slots(max_tiles) entries
     uint32_t* ticket;                // next tile to hand out
     uint32_t* done;                  // CTAs that have finished (the last one resets ticket/done, bumps epoch)
     uint32_t* epoch;                 // launch counter that validates tile_state entries
@@ -50,6 +51,9 @@ struct Workspace {
     uint32_t max_tiles;
     uint32_t skip_publish;           // test hook: tile number whose size is never published (0xFFFFFFFF = off)
 };
+
+// Groups of 32 tiles never span jobs, so a launch needs at most one slot per 32 tiles plus one per job.
+__host__ __device__ constexpr unsigned long long group_slots(unsigned long long max_tiles) { return max_tiles / 32 + kMaxJobs + 2; }
 
 // One chunk-operation.  Encoding jobs (compress, fused hop) and decoding jobs share the struct.
 struct Job {
@@ -133,6 +137,8 @@ enum EncodeMode { kEncodeRaw = 0, kEncodeFused = 1 };
 cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& ws, bool device_params,
                           Params host_params, int sm_count, cudaStream_t st);
+cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool device_params, Params host_params, int sm_count,
+                                cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st);
 cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* sizes,
