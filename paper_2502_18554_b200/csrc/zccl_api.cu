@@ -210,7 +210,8 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
     c->sim_sizes_cap = 2 * (max_ranks > 1 ? max_ranks * max_ranks : 1) + 2;
     const size_t off_state = 0;
     const size_t off_group = off_state + 8 * max_tiles;
-    const size_t off_small = align_up(off_group + 8 * (size_t)group_slots(max_tiles), 256);
+    const size_t off_acc = off_group + 8 * (size_t)group_slots(max_tiles);
+    const size_t off_small = align_up(off_acc + 8 * (size_t)group_slots(max_tiles), 256);
     const size_t off_sizes = off_small + 256;
     const size_t off_quality = align_up(off_sizes + sizeof(size_t) * (size_t)(c->sim_sizes_cap + 1), 256);
     const size_t small_bytes = off_quality + sizeof(double) * 4 * (size_t)kQualityCtas + 256;
@@ -220,6 +221,7 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
         uint8_t* b = (uint8_t*)c->small_block;
         c->ws.tile_state = (unsigned long long*)(b + off_state);
         c->ws.group_state = (unsigned long long*)(b + off_group);
+        c->ws.group_acc = (unsigned long long*)(b + off_acc);
         uint32_t* sm = (uint32_t*)(b + off_small);
         c->ws.ticket = sm + 0;
         c->ws.done = sm + 1;

@@ -26,11 +26,13 @@
 // Every wait is bounded and reports through the status word instead of hanging.
 #include "zccl_device.cuh"
 
+#include <cuda.h>
+#include <cstring>
 #include <mutex>
 
 namespace zccl {
 #ifdef ZCCL_TRACE
-__device__ unsigned long long g_trace[16];
+__device__ unsigned long long g_trace[32];
 __device__ unsigned long long g_rec[4096 * 8];
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long v; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(v)); return v; }
 #define TR_DECL unsigned long long tr_t0 = clock64(), tr_acc[8] = {0,0,0,0,0,0,0,0}; const unsigned long long tr_g0 = gtime()
@@ -97,12 +99,17 @@ __device__ __forceinline__ void bit_transpose(uint32_t (&w)[N])
 // ------------------------------------------------------------------------------------------------ stages
 
 // A stage holds one round: row t = the 32 floats of block t (128 bytes), its 16-byte chunk c stored at chunk
-// position c ^ (t & 7) of the row.
+// position c ^ (t & 7) of the row, so that the lanes' 128-bit reads of their own rows fall into different banks.
+// That is the 128-byte swizzle of the tensor copy engine: a full round of an array that starts on a 16-byte boundary
+// is brought in by ONE tiled tensor copy (32 rows x 32 floats of the array seen as rows of 32 floats; issued by one
+// lane, completion on the stage's mbarrier).  Besides costing no instructions, this keeps the load/store path free:
+// with the input streamed through it (16-byte asynchronous copies were tried first), every latency-critical load
+// of the placement (the states of other tiles) queued up behind kilobytes of input and took microseconds.  Stages
+// must start on a 1024-byte boundary (the swizzle works on address bits).  Other rounds (ragged ends, unaligned
+// arrays) are loaded element by element, positions beyond the tile's end repeating its last element (so that the
+// padding of the last block has zero deltas).
 __device__ __forceinline__ uint32_t stage_chunk_byte(uint32_t row, uint32_t chunk) { return row * 128u + ((chunk ^ (row & 7u)) << 4); }
 
-// Brings elements [e0, e0 + 1024) of a tile that has `len` elements at xt into a stage.  Full rounds that start on
-// a 16-byte boundary are copied asynchronously (the caller commits and waits); others element by element, positions
-// beyond the tile's end repeating its last element (so that the padding of the last block has zero deltas).
 __device__ __noinline__ void load_round_ragged(float* stage, const float* __restrict__ xt, uint32_t e0, uint32_t len, int lane)
 {
     const uint32_t last = len - 1;
@@ -113,19 +120,13 @@ __device__ __noinline__ void load_round_ragged(float* stage, const float* __rest
         *reinterpret_cast<float*>(reinterpret_cast<char*>(stage) + stage_chunk_byte(k, (uint32_t)lane >> 2) + 4 * (lane & 3)) = v;
     }
 }
-// lane_off0 / lane_off1: this lane's byte offset inside the four rows its copies go to, for even / odd copy numbers
-__device__ __forceinline__ void load_round(float* stage, const float* __restrict__ xt, uint32_t e0, uint32_t len, int lane, uint32_t lane_off0,
-                                           uint32_t lane_off1)
+// Tiled tensor copy of rows [row0, row0 + 32) of the array behind `map` into a stage (one thread).
+__device__ __forceinline__ void tensor_load_round(float* stage, unsigned long long* bar, const CUtensorMap* map, uint32_t row0)
 {
-    const float* src = xt + e0;
-    if (e0 + (uint32_t)kRound <= len && (((uintptr_t)src) & 15u) == 0) {
-        const uint32_t sb = smem_u32(stage);
-        const char* g = reinterpret_cast<const char*>(src) + 16 * lane;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) cp_async16(sb + 512u * k + ((k & 1) ? lane_off1 : lane_off0), g + 512 * k);
-    } else {
-        load_round_ragged(stage, xt, e0, len, lane);
-    }
+    mbar_expect_tx(bar, kRound * 4);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(stage)), "l"(map), "r"(0), "r"((int)row0), "r"(smem_u32(bar)) : "memory");
 }
 
 // The last element of a row of a stage (the element in front of the next row's block).
@@ -317,6 +318,7 @@ struct LookBack {
     uint32_t first;             // first tile of its group (launch numbering)
     uint32_t gslot0;            // slot of the state of the job's first group
     uint32_t g;                 // the tile's group within the job
+    uint32_t gsize;             // tiles of that group
     uint32_t grel;              // groups of the job in front of it that are not summed yet
     uint32_t sum_a, sum_b;      // sizes of the tiles of its group in front of it; of the groups summed so far
     bool a_done, b_done, closes_group;
@@ -338,21 +340,43 @@ __device__ __forceinline__ void look_back_begin(LookBack& lb, uint32_t ticket, u
     lb.a_done = (tile & 31u) == 0;
     lb.b_done = lb.g == 0;
     lb.closes_group = (tile & 31u) == 31u || tile + 1 == tiles_in_job;
+    lb.gsize = tiles_in_job - (lb.g << 5) < 32u ? tiles_in_job - (lb.g << 5) : 32u;
 }
 
-// A tile's size, published as soon as it is known.
-__device__ __forceinline__ void publish_size(const Workspace& ws, uint32_t ticket, uint32_t total, uint32_t epoch, int lane)
+// A tile's size, published as soon as it is known (one thread): its own state, and its share of its group's
+// accumulator {tiles:24 | words:40}.  The tile whose addition completes the group publishes the group's size, so a
+// group's size never waits for anybody's position.  Split in two, so that the caller can do other work while the
+// addition is on its way.
+constexpr unsigned long long kAccWordsMask = (1ull << 40) - 1ull;
+__device__ __forceinline__ unsigned long long publish_size_issue(const Workspace& ws, const LookBack& lb)
 {
-    if (lane == 0 && ticket != ws.skip_publish) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
+    if (lb.ticket == ws.skip_publish) return ~0ull;
+    const unsigned long long old = atomicAdd(ws.group_acc + lb.gslot0 + lb.g, (1ull << 40) | (unsigned long long)lb.total);
+    return old;
+}
+__device__ __forceinline__ void publish_size_finish(const Workspace& ws, const LookBack& lb, unsigned long long old, uint32_t epoch)
+{
+    if (old == ~0ull) return;
+#ifdef ZCCL_TRACE
+    if ((uint32_t)(old >> 40) + 1u == lb.gsize) atomicAdd(&g_trace[16], 1ull);
+    if ((uint32_t)(old >> 40) + 1u > lb.gsize) atomicAdd(&g_trace[20], 1ull);
+#endif
+    if ((uint32_t)(old >> 40) + 1u == lb.gsize)
+        st_state(ws.group_state + lb.gslot0 + lb.g, pack_state(epoch, 0u, (uint32_t)(old & kAccWordsMask) + lb.total));
+}
+__device__ __forceinline__ void publish_tile_state(const Workspace& ws, uint32_t ticket, uint32_t total, uint32_t epoch)
+{
+    if (ticket != ws.skip_publish) st_state(ws.tile_state + ticket, pack_state(epoch, 0u, total));
 }
 
-// What the search publishes as it goes, by the tile that closes a group: the group's size once the tiles in front
-// are summed, the group's inclusive prefix once the position is known.
-__device__ __forceinline__ void look_back_publish(const Workspace& ws, const LookBack& lb, bool a_was_done, uint32_t epoch, int lane)
+// The tile that closes a group publishes the group's inclusive prefix once its own position is known.
+__device__ __forceinline__ void look_back_publish(const Workspace& ws, const LookBack& lb, uint32_t epoch, int lane)
 {
-    if (!lb.closes_group || lane != 0 || lb.ticket == ws.skip_publish) return;
-    if (look_back_done(lb)) st_state(ws.group_state + lb.gslot0 + lb.g, pack_state(epoch, 1u, lb.sum_a + lb.sum_b + lb.total));
-    else if (lb.a_done && !a_was_done) st_state(ws.group_state + lb.gslot0 + lb.g, pack_state(epoch, 0u, lb.sum_a + lb.total));
+    if (!lb.closes_group || lane != 0 || lb.ticket == ws.skip_publish || !look_back_done(lb)) return;
+#ifdef ZCCL_TRACE
+    atomicAdd(&g_trace[19], 1ull);
+#endif
+    st_state(ws.group_state + lb.gslot0 + lb.g, pack_state(epoch, 1u, lb.sum_a + lb.sum_b + lb.total));
 }
 
 // One trip: NW windows of group states plus the window of the own group, issued together.
@@ -376,7 +400,7 @@ __device__ __forceinline__ void look_back_issue(const Workspace& ws, const LookB
 template <int NW>
 __device__ __forceinline__ bool look_back_eval(const Workspace& ws, LookBack& lb, uint32_t epoch, int lane, const LookBackTrip<NW>& tr)
 {
-    const bool a_was_done = lb.a_done, was_done = look_back_done(lb);
+    const bool was_done = look_back_done(lb);
     bool stuck = false;
     if (!lb.a_done) {
         const bool ready = (uint32_t)(tr.tile_st >> 33) == epoch;   // lanes beyond the group's first tile hold a ready zero
@@ -404,7 +428,7 @@ __device__ __forceinline__ bool look_back_eval(const Workspace& ws, LookBack& lb
             }
         }
     }
-    if (!was_done) look_back_publish(ws, lb, a_was_done, epoch, lane);
+    if (!was_done) look_back_publish(ws, lb, epoch, lane);
     return !(stuck || b_stuck);
 }
 // Runs the search to its end.  false: a state was not published within the poll limit (the time-out is recorded;
@@ -417,10 +441,18 @@ __device__ __forceinline__ bool look_back_finish(const Workspace& ws, LookBack& 
     while (!look_back_done(lb)) {
         LookBackTrip<kGroupWindows> tr;
         look_back_issue(ws, lb, epoch, lane, tr);
+#ifdef ZCCL_TRACE
+        if (lane == 0) atomicAdd(&g_trace[14], 1ull);
+#endif
         if (!look_back_eval(ws, lb, epoch, lane, tr)) {
+#ifdef ZCCL_TRACE
+            if (lane == 0) { atomicAdd(&g_trace[15], 1ull); if (!lb.a_done) atomicAdd(&g_trace[17], 1ull); if (!lb.b_done) atomicAdd(&g_trace[18], 1ull); }
+#endif
             if (--budget == 0) { status |= kStTimeout; return false; }
+#ifndef ZCCL_EXP_NOSLEEP
             __nanosleep(sleep_ns);
-            if (sleep_ns < 1600u) sleep_ns *= 2u;
+            if (sleep_ns < 400u) sleep_ns *= 2u;
+#endif
         }
     }
     return true;
@@ -429,10 +461,13 @@ __device__ __forceinline__ bool look_back_finish(const Workspace& ws, LookBack& 
 __device__ __forceinline__ bool place_tile(const Workspace& ws, uint32_t ticket, int job_index, uint32_t tile_begin, uint32_t tiles_in_job,
                                            uint32_t total, uint32_t epoch, int lane, uint32_t& excl, uint32_t& status)
 {
-    publish_size(ws, ticket, total, epoch, lane);
     LookBack lb;
     look_back_begin(lb, ticket, total, job_index, tile_begin, tiles_in_job);
-    if (look_back_done(lb)) look_back_publish(ws, lb, true, epoch, lane);   // a group of one tile at the job's start
+    if (lane == 0) {
+        publish_tile_state(ws, ticket, total, epoch);
+        publish_size_finish(ws, lb, publish_size_issue(ws, lb), epoch);
+    }
+    if (look_back_done(lb)) look_back_publish(ws, lb, epoch, lane);   // the job's first tile
     const bool ok = look_back_finish(ws, lb, epoch, lane, status);
     excl = look_back_result(lb);
     return ok;
@@ -476,9 +511,18 @@ __device__ __noinline__ uint32_t flush_tile(const JobBatch* jb, Workspace ws, in
 {
     const Job& jp = jb->job[job];
     uint32_t st = 0;
+#ifdef ZCCL_TRACE
+    const long long c0 = clock64();
+#endif
     const bool placed = look_back_finish(ws, lb, epoch, lane, st);
+#ifdef ZCCL_TRACE
+    const long long c1 = clock64();
+#endif
     emit_tile(jp, lb.ticket - jp.tile_begin, blob, dir ? blob_words - 1u : 0u, dir ? -1 : 1, lb.total, look_back_result(lb), placed, eb_abs,
               s, lane, st);
+#ifdef ZCCL_TRACE
+    if (lane == 0) { atomicAdd(&g_trace[21], (unsigned long long)(c1 - c0)); atomicAdd(&g_trace[22], (unsigned long long)(clock64() - c1)); atomicAdd(&g_trace[23], 1ull); }
+#endif
     return st;
 }
 
@@ -558,10 +602,17 @@ __device__ __noinline__ uint32_t encode_tile_general(const float* __restrict__ x
 // placement until the warp has encoded the next one (by then the tiles in front of it have published their sizes, so
 // the look-back does not wait).  The two share the area from its two ends: one blob grows upwards from word 0, the
 // other downwards from the last word, alternating, so that only their sum is limited.
-constexpr int kEncBlobWords = 1536;
-struct EncWarpShared {
-    alignas(16) float stage[2][kRound];
-    alignas(16) uint32_t blob[kEncBlobWords];
+constexpr int kEncBlobWords = 2556;
+struct alignas(1024) EncWarpShared {
+    float stage[2][kRound];                 // each on a 1024-byte boundary
+    uint32_t blob[kEncBlobWords];
+    alignas(8) unsigned long long bar[2];   // completion of the tensor copies into each stage
+};
+static_assert(sizeof(EncWarpShared) == 18 * 1024, "a warp's share of the shared memory");
+
+// One tensor map per job of a launch: the job's input seen as rows of 32 floats.
+struct alignas(64) TileMaps {
+    CUtensorMap m[kMaxJobs];
 };
 
 // A tile of the launch as a warp sees it.
@@ -571,21 +622,49 @@ struct TileInfo {
     uint32_t tiles;     // tiles of the job
     uint32_t len;       // elements (0: a job without elements, or no valid bound: header and length only)
     const float* xt;    // the tile's first element
+    bool mapped;        // the job's input has a tensor map (16-byte aligned, at least one row)
 };
 
-__global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(const __grid_constant__ JobBatch jb, Workspace ws, Params hp, int use_dev_params)
+__global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps, Workspace ws, Params hp,
+                                                                               int use_dev_params)
 {
     pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    EncWarpShared& sh = reinterpret_cast<EncWarpShared*>(smem_raw)[warp];
+    EncWarpShared& sh = reinterpret_cast<EncWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
     const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
     uint32_t status = 0;
     Params prm = hp;
     if (use_dev_params) prm = *ws.params;
     const float r = prm.r, s = prm.s, eb_abs = prm.eb_abs;
-    const uint32_t rl = (uint32_t)lane >> 3, lc = (uint32_t)lane & 7u;
-    const uint32_t lane_off0 = rl * 128u + ((lc ^ rl) << 4), lane_off1 = rl * 128u + ((lc ^ (rl | 4u)) << 4);
+    if (lane == 0) {
+        mbar_init(&sh.bar[0], 1);
+        mbar_init(&sh.bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    uint32_t fills0 = 0, fills1 = 0;      // bulk rounds completed per stage (phase parity of its mbarrier)
+    bool bulk0 = false, bulk1 = false;    // the round on its way into each stage comes by bulk copies
+    // asks for the round that starts at element e0 of a tile into stage `buf` (nothing for a tile without elements)
+    auto request = [&](uint32_t buf, const TileInfo& ti, uint32_t e0) {
+        bool bulk = false;
+        if (ti.len) {
+            if (ti.mapped && e0 + (uint32_t)kRound <= ti.len) {
+                if (lane == 0) tensor_load_round(sh.stage[buf], &sh.bar[buf], &maps.m[ti.job], ti.tile * (uint32_t)kBlocksPerTile + (e0 >> 5));
+                bulk = true;
+            } else load_round_ragged(sh.stage[buf], ti.xt, e0, ti.len, lane);
+        }
+        if (buf) bulk1 = bulk; else bulk0 = bulk;
+    };
+    // waits for the round in stage `buf`
+    auto arrive = [&](uint32_t buf) {
+        if (buf ? bulk1 : bulk0) {
+            if (!mbar_wait(&sh.bar[buf], (buf ? fills1 : fills0) & 1u)) status |= kStTimeout;
+            if (buf) ++fills1; else ++fills0;
+        }
+        if (buf) bulk1 = false; else bulk0 = false;
+        __syncwarp();
+    };
 
     // the job of the tile looked up last: consecutive look-ups mostly stay inside it
     int cj = -1;
@@ -594,7 +673,7 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
     unsigned long long cj_n = 0;
     auto locate = [&](uint32_t t) {
         TileInfo ti;
-        ti.job = -1; ti.tile = 0; ti.tiles = 1; ti.len = 0; ti.xt = nullptr;
+        ti.job = -1; ti.tile = 0; ti.tiles = 1; ti.len = 0; ti.xt = nullptr; ti.mapped = false;
         if (t >= jb.total_tiles) return ti;
         if (t - cj_begin >= cj_count) {
             cj = find_job(jb, t);
@@ -611,6 +690,7 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
         if (cj_n && prm.valid) {
             ti.len = (uint32_t)((cj_n - start < (unsigned long long)kTile) ? (cj_n - start) : kTile);
             ti.xt = cj_x + start;
+            ti.mapped = (((uintptr_t)cj_x) & 15u) == 0;
         }
         return ti;
     };
@@ -634,8 +714,7 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
 #endif
     TileInfo cur = locate(ticket);
     uint32_t p = 0;   // stage that holds (or will hold) the round about to be encoded
-    if (cur.len) load_round(sh.stage[p], cur.xt, 0, cur.len, lane, lane_off0, lane_off1);
-    cp_async_commit();
+    request(p, cur, 0);
 
     while (cur.job >= 0) {
         const uint32_t tile_begin = ticket - cur.tile;
@@ -653,7 +732,7 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
         if (lane == 0) next_raw = atomicAdd(ws.ticket, 1u);
         uint32_t next = 0;
         TileInfo nxt;
-        nxt.job = -1; nxt.tile = 0; nxt.tiles = 1; nxt.len = 0; nxt.xt = nullptr;
+        nxt.job = -1; nxt.tile = 0; nxt.tiles = 1; nxt.len = 0; nxt.xt = nullptr; nxt.mapped = false;
 
         EncodeCarry cy;
         cy.pay_used = 0; cy.wide = false;
@@ -668,19 +747,17 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
             if (last_round) {
                 next = __shfl_sync(kFull, next_raw, 0);
                 nxt = locate(next);
-                if (nxt.len) load_round(sh.stage[p ^ 1u], nxt.xt, 0, nxt.len, lane, lane_off0, lane_off1);
+                request(p ^ 1u, nxt, 0);
             } else {
-                load_round(sh.stage[p ^ 1u], xt, (rd + 1) * kRound, len, lane, lane_off0, lane_off1);
+                request(p ^ 1u, cur, (rd + 1) * kRound);
             }
-            cp_async_commit();
-            if (rounds == 0) { cp_async_wait<1>(); break; }
+            if (rounds == 0) break;
             // one window of the waiting tile's look-back rides along with this round
             const bool looking = pend.valid && !look_back_done(pend.lb);
             LookBackTrip<1> trip;
             if (looking) look_back_issue(ws, pend.lb, epoch, lane, trip);
             TR_MARK(1);   // request of the next round
-            cp_async_wait<1>();
-            __syncwarp();   // the round's copies of all lanes have landed
+            arrive(p);   // the round has landed
             TR_MARK(2);   // wait for this round's data
             const float* st = sh.stage[p];
             const char* row = reinterpret_cast<const char*>(st) + 128 * lane;
@@ -709,12 +786,10 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
             if (rc != 0) {
                 general = true;
                 if (!last_round) {   // hand over to the next tile: its first round goes where this tile's next round was asked into
-                    cp_async_wait<0>();
-                    __syncwarp();
+                    arrive(p);   // this tile's next round, asked for above and not needed any more
                     next = __shfl_sync(kFull, next_raw, 0);
                     nxt = locate(next);
-                    if (nxt.len) load_round(sh.stage[p], nxt.xt, 0, nxt.len, lane, lane_off0, lane_off1);
-                    cp_async_commit();
+                    request(p, nxt, 0);
                 }
                 break;
             }
@@ -735,8 +810,15 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
         } else {
             if (lane == 0) sh.blob[org] = (uint32_t)q_first;
             const uint32_t total = 1u + padw + cy.pay_used;
-            publish_size(ws, ticket, total, epoch, lane);
+            LookBack lb_cur;
+            look_back_begin(lb_cur, ticket, total, cur.job, tile_begin, cur.tiles);
+            unsigned long long acc_old = ~0ull;
+            if (lane == 0) {
+                publish_tile_state(ws, ticket, total, epoch);
+                acc_old = publish_size_issue(ws, lb_cur);
+            }
             __syncwarp();   // the blob's words, written by all lanes, are visible to all
+            if (lane == 0) publish_size_finish(ws, lb_cur, acc_old, epoch);   // before any wait: others may need the group's size
             TR_MARK(5);   // publish
 #ifdef ZCCL_TRACE
             if (tr_ntiles < 3) tr_tile_end[tr_ntiles] = gtime();
@@ -744,8 +826,11 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
 #endif
             if (pend.valid) flush_pending();
             pend.valid = true; pend.job = cur.job; pend.dir = dir;
-            look_back_begin(pend.lb, ticket, total, cur.job, tile_begin, cur.tiles);
-            if (look_back_done(pend.lb)) look_back_publish(ws, pend.lb, true, epoch, lane);   // a group of one tile at the job's start
+            pend.lb = lb_cur;
+            if (look_back_done(pend.lb)) look_back_publish(ws, pend.lb, epoch, lane);   // the job's first tile
+#ifdef ZCCL_EXP_NODEFER
+            flush_pending();
+#endif
             TR_MARK(6);   // flush of the waiting tile
         }
         cur = nxt;
@@ -757,19 +842,22 @@ __global__ void __launch_bounds__(kCodecThreads, 16 / kCodecWarps) enc_kernel(co
 #ifdef ZCCL_TRACE
     if (lane == 0) { unsigned long long* rec = g_rec + 8 * (blockIdx.x * kCodecWarps + warp); rec[0] = tr_g0; rec[1] = tr_tile_end[0]; rec[2] = tr_tile_end[1]; rec[3] = tr_tile_end[2]; rec[4] = gtime(); rec[5] = tr_ntiles; rec[6] = tr_first_ticket; }
 #endif
-    cp_async_wait<0>();
     if (status) atomicOr(ws.status, status);
-    finish_launch(ws, epoch, tid, ws.ticket);
+    finish_launch(ws, epoch, tid, ws.ticket, (jb.total_tiles >> 5) + (uint32_t)jb.count + 1u);
 }
 
 // Per-device launch set-up (shared-memory attribute, resident CTAs per SM), done once per device under a lock.
 constexpr int kMaxDevices = 64;
+constexpr size_t kEncSmemBytes = sizeof(EncWarpShared) * kCodecWarps + 1024;   // + room to reach a 1024-byte boundary
 struct DeviceSetup {
     bool ready = false;
     int enc_ctas = 1;
 };
 DeviceSetup g_dev[kMaxDevices];
 std::mutex g_dev_mu;
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;   // the driver's cuTensorMapEncodeTiled, looked up through the runtime
 
 cudaError_t device_setup(const DeviceSetup** out)
 {
@@ -778,12 +866,20 @@ cudaError_t device_setup(const DeviceSetup** out)
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(g_dev_mu);
+    if (!g_encode_tiled) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+        if (e != cudaSuccess) return e;
+        if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+        g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    }
     DeviceSetup& d = g_dev[dev];
     if (!d.ready) {
-        e = cudaFuncSetAttribute(enc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(sizeof(EncWarpShared) * kCodecWarps));
+        e = cudaFuncSetAttribute(enc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEncSmemBytes);
         if (e != cudaSuccess) return e;
         int a = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, enc_kernel, kCodecThreads, sizeof(EncWarpShared) * kCodecWarps);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, enc_kernel, kCodecThreads, kEncSmemBytes);
         if (e != cudaSuccess) return e;
         d.enc_ctas = a > 0 ? a : 1;
         d.ready = true;
@@ -792,13 +888,28 @@ cudaError_t device_setup(const DeviceSetup** out)
     return cudaSuccess;
 }
 
+// The array x of n floats as rows of 32 floats, copied in tiles of 32 rows with the 128-byte swizzle.  Arrays that
+// do not start on a 16-byte boundary or have no full row get no map (the kernels load them element by element).
+cudaError_t make_row_map(CUtensorMap* map, const float* x, unsigned long long n)
+{
+    if ((((uintptr_t)x) & 15u) != 0 || n < (unsigned long long)kBlock) return cudaSuccess;
+    const cuuint64_t dims[2] = {(cuuint64_t)kBlock, (cuuint64_t)(n / kBlock)};
+    const cuuint64_t strides[1] = {(cuuint64_t)kBlock * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlock, 32u};
+    const cuuint32_t estr[2] = {1u, 1u};
+    const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(x), dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 }  // namespace
 
 #ifdef ZCCL_TRACE
 extern "C" int zccl_debug_rec(unsigned long long* out, int n) { return cudaMemcpyFromSymbol(out, g_rec, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -1; }
 extern "C" int zccl_debug_trace(unsigned long long* out16)
 {
-    unsigned long long z[16] = {};
+    unsigned long long z[32] = {};
     z[9] = z[11] = ~0ull;
     if (cudaMemcpyFromSymbol(out16, g_trace, sizeof(z)) != cudaSuccess) return -1;
     return cudaMemcpyToSymbol(g_trace, z, sizeof(z)) == cudaSuccess ? 0 : -1;
@@ -811,14 +922,17 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
     const DeviceSetup* d = nullptr;
     cudaError_t e = device_setup(&d);
     if (e != cudaSuccess) return e;
+    TileMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    for (int j = 0; j < jb.count; ++j)
+        if ((e = make_row_map(&maps.m[j], jb.job[j].x, jb.job[j].n)) != cudaSuccess) return e;
     const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     unsigned long long cap = (unsigned long long)sm_count * d->enc_ctas;
 #ifdef ZCCL_TRACE
-    if (const char* e = getenv("ZCCL_EXP_CTAS")) cap = (unsigned long long)sm_count * atoi(e);
+    if (const char* ev = getenv("ZCCL_EXP_CTAS")) cap = (unsigned long long)sm_count * atoi(ev);
 #endif
     const unsigned grid = (unsigned)(want < cap ? want : cap);
-    return launch_k(enc_kernel, dim3(grid), dim3(kCodecThreads), sizeof(EncWarpShared) * kCodecWarps, st, jb, ws, host_params,
-                    device_params ? 1 : 0);
+    return launch_k(enc_kernel, dim3(grid), dim3(kCodecThreads), kEncSmemBytes, st, jb, maps, ws, host_params, device_params ? 1 : 0);
 }
 
 }  // namespace zccl

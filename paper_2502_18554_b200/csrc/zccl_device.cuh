@@ -161,7 +161,8 @@ __device__ __forceinline__ void write_header(uint32_t* out, int tid, unsigned lo
     }
 }
 
-__device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoch, int tid, uint32_t* tile_counter = nullptr)
+__device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoch, int tid, uint32_t* tile_counter = nullptr,
+                                              uint32_t groups_used = 0)
 {
     __syncthreads();
     if (tid == 0) {
@@ -170,6 +171,7 @@ __device__ __forceinline__ void finish_launch(const Workspace& ws, uint32_t epoc
         if (prev == gridDim.x - 1) {   // every CTA is done with the scan states: re-arm for the next launch
             *ws.done = 0;
             if (tile_counter) *tile_counter = 0;
+            for (uint32_t g = 0; g < groups_used; ++g) ws.group_acc[g] = 0ull;   // the group accumulators of this launch
             uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
             if (e == 0) {   // the counter wraps (once in 2^31 launches): no state of an earlier launch may look current again
                 for (uint32_t t = 0; t < ws.max_tiles; ++t) st_state(ws.tile_state + t, 0ull);

@@ -42,6 +42,7 @@ struct Params {
 struct Workspace {
     unsigned long long* tile_state;  // one 64-bit {epoch:31 | inclusive:1 | words:32} per tile of a launch
     unsigned long long* group_state; // the same per group of 32 consecutive tiles of a job: group_slots(max_tiles) entries
+    unsigned long long* group_acc;   // per group {tiles published:24 | their words:40}, zero between launches
     uint32_t* ticket;                // next tile to hand out
     uint32_t* done;                  // CTAs that have finished (the last one resets ticket/done, bumps epoch)
     uint32_t* epoch;                 // launch counter that validates tile_state entries

@@ -20,7 +20,7 @@ namespace {
 
 constexpr size_t kMaxElems = (size_t)ZCCL_NOALLOC_MAX_ELEMS;
 constexpr size_t kMaxTiles = kMaxElems / kTile + 1;
-constexpr size_t kStateBytes = ((kMaxTiles + (size_t)group_slots(kMaxTiles)) * 8 + 255) / 256 * 256;
+constexpr size_t kStateBytes = ((kMaxTiles + 2 * (size_t)group_slots(kMaxTiles)) * 8 + 255) / 256 * 256;
 constexpr size_t kScratchBytes = kStateBytes + 256;   // scan states, then counters / status / parameter block
 
 // Scratch shared by every call on a device (about 129 KiB, held by each GPU that loads the library until exit).
@@ -50,6 +50,7 @@ Workspace workspace_at(unsigned char* base)
     Workspace ws{};
     ws.tile_state = reinterpret_cast<unsigned long long*>(base);
     ws.group_state = ws.tile_state + kMaxTiles;
+    ws.group_acc = ws.group_state + group_slots(kMaxTiles);
     uint32_t* sm = reinterpret_cast<uint32_t*>(base + kStateBytes);
     ws.ticket = sm + 0;
     ws.done = sm + 1;
