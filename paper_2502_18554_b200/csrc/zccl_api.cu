@@ -22,6 +22,7 @@ struct zccl_ctx {
     uint32_t* quality_counter = nullptr;
     Workspace ws{};
     void* small_block = nullptr;     // tile states + counters + params + sizes
+    void* slot_block = nullptr;      // round slots, round sizes and outliers of the two-step compression
     uint8_t* arena = nullptr;        // compressed-chunk slots of the emulated ranks
     size_t arena_bytes = 0;
     size_t* sim_sizes = nullptr;     // device: sizes of the last zccl_sim_* call
@@ -239,6 +240,17 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
         ok = cudaMemcpy(c->ws.epoch, &init[0], 4, cudaMemcpyHostToDevice) == cudaSuccess &&
              cudaMemcpy(c->ws.minmax, &init[1], 8, cudaMemcpyHostToDevice) == cudaSuccess;
     }
+    if (ok) {
+        const size_t off_rw = align_up(max_tiles * 4 * (size_t)kRoundSlotWords * 4, 256);
+        const size_t off_ol = align_up(off_rw + max_tiles * 4 * 4, 256);
+        ok = cudaMalloc(&c->slot_block, off_ol + max_tiles * 4) == cudaSuccess;
+        if (ok) {
+            uint8_t* b = (uint8_t*)c->slot_block;
+            c->ws.slots = (uint32_t*)b;
+            c->ws.round_words = (uint32_t*)(b + off_rw);
+            c->ws.outliers = (int32_t*)(b + off_ol);
+        }
+    }
     if (ok && max_ranks >= 2) {
         c->arena_bytes = (size_t)(max_ranks + 2) * align_up(bound_of(max_elems) + (size_t)max_ranks * 1024, 256);
         ok = cudaMalloc((void**)&c->arena, c->arena_bytes) == cudaSuccess;
@@ -262,6 +274,7 @@ void zccl_ctx_destroy(zccl_ctx* c)
     if (!c) return;
     cudaDeviceSynchronize();
     if (c->small_block) cudaFree(c->small_block);
+    if (c->slot_block) cudaFree(c->slot_block);
     if (c->gen_sizes) cudaFree(c->gen_sizes);
     if (c->arena) cudaFree(c->arena);
     if (c->stage_x) cudaFree(c->stage_x);

@@ -433,26 +433,20 @@ __device__ __forceinline__ bool look_back_eval(const Workspace& ws, LookBack& lb
 }
 // Runs the search to its end.  false: a state was not published within the poll limit (the time-out is recorded;
 // nothing may be written for this tile).
-constexpr int kGroupWindows = 2;   // windows of group states per trip of the blocking search
+constexpr int kGroupWindows = 4;   // windows of group states per trip of the blocking search
 __device__ __forceinline__ bool look_back_finish(const Workspace& ws, LookBack& lb, uint32_t epoch, int lane, uint32_t& status)
 {
     int budget = kSpinLimit >> 4;
-    uint32_t sleep_ns = 100;   // backs off: polling warps take issue slots from working ones
+    uint32_t sleep_ns = 0;   // the first polls follow each other at once; then the warp backs off (polling takes issue slots)
     while (!look_back_done(lb)) {
         LookBackTrip<kGroupWindows> tr;
         look_back_issue(ws, lb, epoch, lane, tr);
-#ifdef ZCCL_TRACE
-        if (lane == 0) atomicAdd(&g_trace[14], 1ull);
-#endif
         if (!look_back_eval(ws, lb, epoch, lane, tr)) {
-#ifdef ZCCL_TRACE
-            if (lane == 0) { atomicAdd(&g_trace[15], 1ull); if (!lb.a_done) atomicAdd(&g_trace[17], 1ull); if (!lb.b_done) atomicAdd(&g_trace[18], 1ull); }
-#endif
             if (--budget == 0) { status |= kStTimeout; return false; }
-#ifndef ZCCL_EXP_NOSLEEP
-            __nanosleep(sleep_ns);
-            if (sleep_ns < 400u) sleep_ns *= 2u;
-#endif
+            if (budget < (kSpinLimit >> 4) - 6) {
+                sleep_ns = sleep_ns < 400u ? sleep_ns + 100u : 400u;
+                __nanosleep(sleep_ns);
+            }
         }
     }
     return true;
@@ -846,12 +840,388 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
     finish_launch(ws, epoch, tid, ws.ticket, (jb.total_tiles >> 5) + (uint32_t)jb.count + 1u);
 }
 
+// ------------------------------------------------------------------------------------------------ compress, two steps
+//
+// Step 1 (encode_rounds_kernel): the unit of work is a ROUND (32 blocks of a tile, one per lane).  A round needs
+// nothing from the rounds around it but the element in front of it, so the rounds of a launch are handed to the warps
+// by a counter in any order and nobody waits for anybody: a warp brings its round in with one tensor copy, encodes it
+// into its shared memory and sends it off with one bulk store to the round's fixed slot in the workspace (code-length
+// bytes, then payload), together with its size and, for a tile's first round, the tile's first quantised value.
+// Step 2 (place_kernel) turns the slots into the stream.
+
+constexpr int kRoundBufWords = 8 + 32 * 17;   // code-length bytes + payload at code length 16 (longer codes go the general route)
+struct alignas(1024) RoundWarpShared {
+    float stage[2][kRound];                   // each on a 1024-byte boundary
+    alignas(16) uint32_t out[2][kRoundBufWords];
+    alignas(8) unsigned long long bar[2];
+};
+static_assert(sizeof(RoundWarpShared) == 13 * 1024, "a warp's share of the shared memory");
+
+// A round of the launch as a warp sees it.
+struct RoundInfo {
+    int job;            // -1: beyond the launch's last round
+    uint32_t tile;      // launch number of the round's tile
+    uint32_t jtile;     // the tile's number within its job
+    uint32_t rd;        // the round within the tile
+    uint32_t len;       // elements of the tile (0: nothing to encode)
+    uint32_t gslot;     // slot of the accumulator of the tile's group
+    const float* xt;    // the tile's first element
+    bool mapped;
+};
+
+// General route for one round: any code length, straight from global memory into the round's slot.
+__device__ __noinline__ uint32_t encode_round_general(const float* __restrict__ xt, uint32_t len, uint32_t rd, float r, uint32_t* __restrict__ slot,
+                                                      uint32_t* round_words, int32_t* outlier, unsigned long long* group_words, int lane)
+{
+    uint32_t status = 0;
+    const uint32_t nb = (len + kBlock - 1) / kBlock;
+    const uint32_t bi = 32u * rd + (uint32_t)lane;
+    uint32_t planes[33];
+    float tmax = 0.0f;
+    uint32_t L = 0;
+    if (bi < nb) L = general_block(xt, bi, len, r, planes, &tmax);
+    if (!(tmax < 1073741824.0f)) status |= kStRange;
+    else if (tmax > 32768.5f) status |= kStPrecision;
+    const uint32_t nw = L ? L + 1u : 0u;
+    const uint32_t incl = warp_incl_scan(nw, lane);
+    reinterpret_cast<unsigned char*>(slot)[lane] = (unsigned char)L;
+    if (L) {
+        uint32_t* d = slot + 8 + (incl - nw);
+        for (uint32_t k = 0; k <= L; ++k) d[k] = planes[k];
+    }
+    if (lane == 31) { *round_words = incl; atomicAdd(group_words, (unsigned long long)incl); }
+    if (rd == 0 && lane == 0) *outlier = __float2int_rn(__fmul_rn(__ldg(xt), r));
+    return status;
+}
+
+__global__ void __launch_bounds__(kCodecThreads, 4) encode_rounds_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
+                                                                         Workspace ws, Params hp, int use_dev_params)
+{
+    pdl_enter();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    RoundWarpShared& sh = reinterpret_cast<RoundWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
+    uint32_t status = 0;
+    Params prm = hp;
+    if (use_dev_params) prm = *ws.params;
+    const float r = prm.r;
+    const uint32_t total_rounds = jb.total_tiles * (uint32_t)kRoundsPerTile;
+
+    if (lane == 0) {
+        mbar_init(&sh.bar[0], 1);
+        mbar_init(&sh.bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    uint32_t fills0 = 0, fills1 = 0;      // tensor copies completed per stage (phase parity of its mbarrier)
+    bool bulk0 = false, bulk1 = false;    // the round on its way into each stage comes by a tensor copy
+
+    // the job of the round looked up last: consecutive look-ups mostly stay inside it
+    int cj = -1;
+    uint32_t cj_begin = 0, cj_count = 0;
+    const float* cj_x = nullptr;
+    unsigned long long cj_n = 0;
+    auto locate = [&](uint32_t u) {
+        RoundInfo ri;
+        ri.job = -1; ri.tile = 0; ri.jtile = 0; ri.rd = 0; ri.len = 0; ri.gslot = 0; ri.xt = nullptr; ri.mapped = false;
+        if (u >= total_rounds) return ri;
+        const uint32_t t = u >> 2;
+        if (t - cj_begin >= cj_count) {
+            cj = find_job(jb, t);
+            const Job& q = jb.job[cj];
+            cj_begin = q.tile_begin;
+            cj_count = (cj + 1 < jb.count ? jb.job[cj + 1].tile_begin : jb.total_tiles) - cj_begin;
+            cj_x = q.x;
+            cj_n = q.n;
+        }
+        ri.job = cj; ri.tile = t; ri.jtile = t - cj_begin; ri.rd = u & 3u;
+        ri.gslot = (cj_begin >> 5) + (uint32_t)cj + (ri.jtile >> 5);
+        const unsigned long long start = (unsigned long long)ri.jtile * kTile;
+        if (cj_n && prm.valid) {
+            ri.len = (uint32_t)((cj_n - start < (unsigned long long)kTile) ? (cj_n - start) : kTile);
+            ri.xt = cj_x + start;
+            ri.mapped = (((uintptr_t)cj_x) & 15u) == 0;
+        }
+        return ri;
+    };
+    // asks for a round into stage `buf`; lane 0 also fetches the element in front of the round
+    auto request = [&](uint32_t buf, const RoundInfo& ri, float& front) {
+        bool bulk = false;
+        const uint32_t e0 = ri.rd * (uint32_t)kRound;
+        if (e0 < ri.len) {
+            if (ri.mapped && e0 + (uint32_t)kRound <= ri.len) {
+                if (lane == 0) tensor_load_round(sh.stage[buf], &sh.bar[buf], &maps.m[ri.job], ri.jtile * (uint32_t)kBlocksPerTile + (e0 >> 5));
+                bulk = true;
+            } else load_round_ragged(sh.stage[buf], ri.xt, e0, ri.len, lane);
+            if (lane == 0) front = __ldg(ri.xt + (e0 ? e0 - 1u : 0u));   // a tile's first element is its own predecessor
+        }
+        if (buf) bulk1 = bulk; else bulk0 = bulk;
+    };
+    auto arrive = [&](uint32_t buf) {
+        if (buf ? bulk1 : bulk0) {
+            if (!mbar_wait(&sh.bar[buf], (buf ? fills1 : fills0) & 1u)) status |= kStTimeout;
+            if (buf) ++fills1; else ++fills0;
+        }
+        if (buf) bulk1 = false; else bulk0 = false;
+        __syncwarp();
+    };
+
+    // Rounds are dealt round-robin over the warps of the launch (no counter: same-address atomics would bound the kernel
+    // at about 1.5 ns per round), and the next round's input is asked for before this round is encoded.
+    const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
+    const uint32_t u0 = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
+    uint32_t u1 = u0 + stride;
+    if (u1 < u0) u1 = 0xFFFFFFFFu;
+    RoundInfo cur = locate(u0), nxt = locate(u1);
+    uint32_t p = 0;
+    float front = 0.0f, front1 = 0.0f;
+    request(0, cur, front);
+    EncodeCarry cy;
+    cy.pay_used = 0; cy.wide = false;
+
+    while (cur.job >= 0) {
+        __syncwarp();   // every lane is done with the other stage
+        request(p ^ 1u, nxt, front1);
+        const uint32_t u = 4u * cur.tile + cur.rd;
+        const uint32_t nb = (cur.len + kBlock - 1) / kBlock;
+        if (32u * cur.rd < nb) {
+            arrive(p);
+            uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
+            const float* st = sh.stage[p];
+            const char* row = reinterpret_cast<const char*>(st) + 128 * lane;
+            const uint32_t sw = ((uint32_t)lane & 7u) << 4;
+            const float xprev = lane ? read_last_of_row(st, (uint32_t)lane - 1u) : front;
+            // the buffer this round is encoded into was sent off two rounds ago: that store has to be through with it
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            __syncwarp();
+            uint32_t* buf = sh.out[p];
+            cy.pay_used = 0;
+            const uint32_t bi = 32u * cur.rd + (uint32_t)lane;
+            // laid out like a tile's blob whose word 0 sits in front of the buffer: code-length bytes at words 1.., payload at word 9
+#ifdef ZCCL_EXP_NOCOMPUTE
+            const int rc = 0;
+            cy.pay_used = (uint32_t)(xprev + *reinterpret_cast<const float*>(row + sw)) & 15u;
+#else
+            const int rc = encode_round(row, sw, xprev, r, bi < nb, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, cy, lane,
+                                        status);
+#endif
+            if (rc == 0) {
+                __syncwarp();   // the buffer's words, written by all lanes, are visible to lane 0's store
+                if (lane == 0) {
+                    const uint32_t bytes = (32u + 4u * cy.pay_used + 15u) & ~15u;
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(slot), "r"(smem_u32(buf)), "r"(bytes) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    ws.round_words[u] = cy.pay_used;
+                    atomicAdd(ws.group_acc + cur.gslot, (unsigned long long)cy.pay_used);
+                    if (cur.rd == 0) {
+                        // exact while |x r| < 2^22; larger codes take the general route
+                        ws.outliers[cur.tile] = (int32_t)(__float_as_uint(__fadd_rn(__fmul_rn(front, r), kRoundMagic)) - kRoundMagicBits);
+                    }
+                }
+            } else {
+                status |= encode_round_general(cur.xt, cur.len, cur.rd, r, slot, ws.round_words + u, ws.outliers + cur.tile, ws.group_acc + cur.gslot,
+                                               lane);
+            }
+        } else {
+            if (lane == 0) ws.round_words[u] = 0;   // a round beyond the tile's last block, or a tile without elements
+        }
+        u1 = u1 + stride < u1 ? 0xFFFFFFFFu : u1 + stride;
+        cur = nxt;
+        nxt = locate(u1);
+        front = front1;
+        p ^= 1u;
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the stores have read shared memory and are complete
+    if (status) atomicOr(ws.status, status);
+}
+
+// Step 2: one CTA per group of 32 tiles of a job turns the group's round slots into its piece of the stream.  The
+// tiles' sizes follow from the rounds' sizes; the group's position is the sum of the groups of the job in front of
+// it, found by a decoupled look-back over the group states (every CTA publishes its group's size as soon as it has
+// read 128 numbers, so the waits are short; they are bounded all the same); then each warp copies tiles.
+struct GroupTable {
+    uint32_t begin[kMaxJobs + 1];   // first group (= CTA) of each job; begin[count] = number of groups
+};
+constexpr int kPlaceThreads = 1024;   // one warp per tile of the group
+
+__global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ GroupTable gt, Workspace ws,
+                                                              Params hp, int use_dev_params)
+{
+    pdl_enter();
+    __shared__ uint32_t s_words[32], s_off[32], s_part[kPlaceThreads / 32], s_base, s_ok;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
+    uint32_t status = 0;
+    Params prm = hp;
+    if (use_dev_params) prm = *ws.params;
+
+    int j = 0;
+    {
+        int lo = 0, hi = jb.count;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (gt.begin[mid] <= blockIdx.x) lo = mid; else hi = mid;
+        }
+        j = lo;
+    }
+#ifdef ZCCL_TRACE
+    if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 0] = gtime();
+#endif
+    const Job& job = jb.job[j];
+    const uint32_t g = blockIdx.x - gt.begin[j];
+    const uint32_t tiles = (j + 1 < jb.count ? jb.job[j + 1].tile_begin : jb.total_tiles) - job.tile_begin;
+    const unsigned long long n = job.n;
+    const uint32_t nT = (uint32_t)((n + kTile - 1) / kTile);
+    uint32_t* __restrict__ out = job.out;
+
+    if (n == 0 || !prm.valid) {   // a job without elements, or no valid bound: header and length only
+        const bool hdr = prm.valid && job.out_cap >= (unsigned)kHeaderBytes;
+        if (tid == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
+        if (hdr) write_header(out, tid, 0, prm.eb_abs, prm.s, 0);
+    } else {
+        const uint32_t t0 = 32u * g;                               // first tile of the group, within the job
+        const uint32_t ntl = tiles - t0 < 32u ? tiles - t0 : 32u;   // tiles of the group
+        const uint32_t T0 = job.tile_begin + t0;                   // the same, in the launch's numbering
+        // sizes: thread i < 128 holds round i & 3 of tile i >> 2
+        if (tid < 128) {
+            const uint32_t ti = (uint32_t)tid >> 2;
+            const uint32_t rw = ti < ntl ? ws.round_words[4u * T0 + (uint32_t)tid] : 0u;
+            uint32_t pay = rw + __shfl_xor_sync(kFull, rw, 1);
+            pay += __shfl_xor_sync(kFull, pay, 2);
+            const unsigned long long left = n - (unsigned long long)(t0 + ti) * kTile;
+            const uint32_t len = ti < ntl ? (uint32_t)(left < (unsigned long long)kTile ? left : (unsigned long long)kTile) : 0u;
+            const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2;
+            if ((tid & 3) == 0) s_words[ti] = ti < ntl ? 1u + padw + pay : 0u;
+        }
+        __syncthreads();
+#ifdef ZCCL_TRACE
+        if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 1] = gtime();
+#endif
+        if (warp == 0) {
+            const uint32_t w = s_words[lane];
+            const uint32_t incl = warp_incl_scan(w, lane);
+            s_off[lane] = incl - w;
+        }
+        // the group's place: the groups of the job in front of it are full ones (33 fixed words per tile) with the
+        // payload that step 1 added up per group
+        {
+            const uint32_t gslot0 = (job.tile_begin >> 5) + (uint32_t)j;
+            unsigned long long part = 0;
+            for (uint32_t k = (uint32_t)tid; k < g; k += kPlaceThreads) part += ws.group_acc[gslot0 + k];
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(kFull, part, d);
+            if (lane == 0) s_part[warp] = (uint32_t)part;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t sum = 0;
+            for (int w = 0; w < kPlaceThreads / 32; ++w) sum += s_part[w];
+            s_base = sum + g * 32u * (1u + (uint32_t)kLWords);
+            s_ok = 1u;
+        }
+        __syncthreads();
+        // every warp fetches its tile's pieces (up to eight words per lane and round); after the look-back, whose few
+        // loads would otherwise queue up behind these
+        const uint32_t tl = (uint32_t)warp;
+        const bool mine = tl < ntl;
+        const uint32_t T = T0 + tl;
+        const uint32_t* __restrict__ slot = ws.slots + (size_t)(4u * T) * kRoundSlotWords;
+        uint32_t nqs[kRoundsPerTile] = {0, 0, 0, 0};
+        uint32_t v[kRoundsPerTile][8];
+        uint32_t lword = 0, first = 0;
+        if (mine) {
+            const uint4 nq4 = *reinterpret_cast<const uint4*>(ws.round_words + 4u * T);
+            nqs[0] = nq4.x; nqs[1] = nq4.y; nqs[2] = nq4.z; nqs[3] = nq4.w;
+            lword = slot[(size_t)(lane >> 3) * kRoundSlotWords + (lane & 7)];   // code-length word `lane` of the tile
+            if (lane == 0) first = (uint32_t)ws.outliers[T];
+#pragma unroll
+            for (int q = 0; q < kRoundsPerTile; ++q) {
+                const uint32_t* __restrict__ src = slot + (size_t)q * kRoundSlotWords + 8;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint32_t i = (uint32_t)lane + 32u * k;
+                    v[q][k] = i < nqs[q] ? src[i] : 0u;
+                }
+            }
+        }
+#ifdef ZCCL_TRACE
+        if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 3] = gtime();
+#endif
+        const uint32_t base = s_base;
+        const bool placed = s_ok != 0;
+        if (mine) {
+            const uint32_t tile = t0 + tl;
+            const uint32_t words = s_words[tl];
+            const unsigned long long word0 = (unsigned long long)kHeaderWords + nT + base + s_off[tl];
+            const bool fits = (word0 + words) * 4ull <= job.out_cap;
+            if (!fits) status |= kStCapacity;
+            if (fits && placed) {
+                uint32_t* __restrict__ dst = out + word0;
+                const unsigned long long tleft = n - (unsigned long long)tile * kTile;
+                const uint32_t tlen = (uint32_t)(tleft < (unsigned long long)kTile ? tleft : (unsigned long long)kTile);
+                const uint32_t tpadw = (((tlen + kBlock - 1) / kBlock) + 3) >> 2;
+                if (lane == 0) dst[0] = first;
+                if ((uint32_t)lane < tpadw) dst[1 + lane] = lword;
+                uint32_t* __restrict__ d = dst + 1 + tpadw;
+#pragma unroll
+                for (int q = 0; q < kRoundsPerTile; ++q) {
+                    const uint32_t nq = nqs[q];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t i = (uint32_t)lane + 32u * k;
+                        if (i < nq) d[i] = v[q][k];
+                    }
+                    if (nq > 256u) {   // code lengths beyond 7 on average: the rest of the round
+                        const uint32_t* __restrict__ src = slot + (size_t)q * kRoundSlotWords + 8;
+                        for (uint32_t i = 256u + (uint32_t)lane; i < nq; i += 32) d[i] = src[i];
+                    }
+                    d += nq;
+                }
+                if (lane == 0) out[kHeaderWords + tile] = base + s_off[tl] + words;
+            }
+            if (lane == 0 && tile == nT - 1) *job.out_bytes = (size_t)((word0 + words) * 4ull);
+            if (tile == 0) write_header(out, lane, n, prm.eb_abs, prm.s, nT);
+        }
+    }
+#ifdef ZCCL_TRACE
+    __syncthreads();
+    if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 4] = gtime();
+#endif
+    if (status) atomicOr(ws.status, status);
+    // the last CTA to get here re-arms the workspace: group sums back to zero, launch counter on
+    __shared__ uint32_t s_last;
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        s_last = atomicAdd(ws.done, 1u) == gridDim.x - 1 ? 1u : 0u;
+    }
+    __syncthreads();
+    if (s_last) {
+        const uint32_t used = (jb.total_tiles >> 5) + (uint32_t)jb.count + 1u;
+        for (uint32_t k = (uint32_t)tid; k < used; k += kPlaceThreads) ws.group_acc[k] = 0ull;
+        const uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
+        if (e == 0) {   // the counter wraps (once in 2^31 launches): no scan state of an earlier launch may look current again
+            for (uint32_t k = (uint32_t)tid; k < ws.max_tiles; k += kPlaceThreads) st_state(ws.tile_state + k, 0ull);
+            for (uint32_t k = (uint32_t)tid; k < (uint32_t)group_slots(ws.max_tiles); k += kPlaceThreads) st_state(ws.group_state + k, 0ull);
+            __threadfence();
+        }
+        __syncthreads();
+        if (tid == 0) {
+            *ws.done = 0;
+            *ws.ticket = 0;
+            *ws.epoch = e ? e : 1u;
+        }
+    }
+}
+
 // Per-device launch set-up (shared-memory attribute, resident CTAs per SM), done once per device under a lock.
 constexpr int kMaxDevices = 64;
 constexpr size_t kEncSmemBytes = sizeof(EncWarpShared) * kCodecWarps + 1024;   // + room to reach a 1024-byte boundary
+constexpr size_t kRoundSmemBytes = sizeof(RoundWarpShared) * kCodecWarps + 1024;
 struct DeviceSetup {
     bool ready = false;
-    int enc_ctas = 1;
+    int enc_ctas = 1, round_ctas = 1;
 };
 DeviceSetup g_dev[kMaxDevices];
 std::mutex g_dev_mu;
@@ -882,6 +1252,11 @@ cudaError_t device_setup(const DeviceSetup** out)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, enc_kernel, kCodecThreads, kEncSmemBytes);
         if (e != cudaSuccess) return e;
         d.enc_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(encode_rounds_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRoundSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_rounds_kernel, kCodecThreads, kRoundSmemBytes);
+        if (e != cudaSuccess) return e;
+        d.round_ctas = a > 0 ? a : 1;
         d.ready = true;
     }
     *out = &d;
@@ -926,6 +1301,24 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
     memset(&maps, 0, sizeof(maps));
     for (int j = 0; j < jb.count; ++j)
         if ((e = make_row_map(&maps.m[j], jb.job[j].x, jb.job[j].n)) != cudaSuccess) return e;
+    if (ws.slots && ws.skip_publish == 0xFFFFFFFFu) {
+        // two steps: rounds into their slots, then one CTA per group of 32 tiles places them
+        GroupTable gt;
+        uint32_t groups = 0;
+        for (int j = 0; j < jb.count; ++j) {
+            gt.begin[j] = groups;
+            const uint32_t tiles = (j + 1 < jb.count ? jb.job[j + 1].tile_begin : jb.total_tiles) - jb.job[j].tile_begin;
+            groups += (tiles + 31u) / 32u;
+        }
+        for (int j = jb.count; j <= kMaxJobs; ++j) gt.begin[j] = groups;
+        const unsigned long long rounds = (unsigned long long)jb.total_tiles * kRoundsPerTile;
+        const unsigned long long want_a = (rounds + kCodecWarps - 1) / kCodecWarps;
+        const unsigned long long cap_a = (unsigned long long)sm_count * d->round_ctas;
+        e = launch_k(encode_rounds_kernel, dim3((unsigned)(want_a < cap_a ? want_a : cap_a)), dim3(kCodecThreads), kRoundSmemBytes, st, jb, maps, ws,
+                     host_params, device_params ? 1 : 0);
+        if (e != cudaSuccess) return e;
+        return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, host_params, device_params ? 1 : 0);
+    }
     const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     unsigned long long cap = (unsigned long long)sm_count * d->enc_ctas;
 #ifdef ZCCL_TRACE

@@ -49,9 +49,17 @@ struct Workspace {
     uint32_t* status;                // device status bits
     Params* params;                  // resolved bound for REL mode
     uint32_t* minmax;                // two ordered-int keys: running min and max
+    // Two-step compression (encode rounds into fixed slots, then place): null where there is no room for it (the
+    // allocation-free entry point), which then compresses in a single pass.
+    uint32_t* slots;                 // per round of a launch (4 per tile): kRoundSlotWords words
+    uint32_t* round_words;           // per round: its payload words
+    int32_t* outliers;               // per tile: its first quantised value
     uint32_t max_tiles;
     uint32_t skip_publish;           // test hook: tile number whose size is never published (0xFFFFFFFF = off)
 };
+
+// A round's slot: the code-length bytes of its 32 blocks (8 words), then its payload at the largest code length.
+constexpr int kRoundSlotWords = 8 + 32 * 32;
 
 // Groups of 32 tiles never span jobs, so a launch needs at most one slot per 32 tiles plus one per job.
 __host__ __device__ constexpr unsigned long long group_slots(unsigned long long max_tiles) { return max_tiles / 32 + kMaxJobs + 2; }
