@@ -1215,13 +1215,310 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
     }
 }
 
+// ------------------------------------------------------------------------------------------------ decompress
+//
+// A warp decodes a tile of its own in four rounds, lane l of a round taking block 32 * round + l: the block's sign
+// word and planes come out of the tile's blob (staged in shared memory by a bulk copy, one tile ahead), the block's
+// sum of deltas follows from population counts of the planes, a shuffle scan of those sums gives every block the
+// code in front of it, and the lane then walks its 32 elements: inverse bit-matrix transpose, magnitude, sign,
+// running code, one multiplication; the values go into the lane's row of a swizzled stage, which one tiled tensor
+// store (or, for ragged ends and unaligned arrays, a loop of coalesced stores) moves to the output.
+
+// What a tile's code-length bytes say, found by every lane alike: 0 = inconsistent with the blob's size (or a code
+// length above 31, or a non-zero padding byte), 1 = consistent and every code of the tile stays below 2^23 in
+// magnitude (fp32 arithmetic is exact), 2 = consistent, integer arithmetic needed.  blob: the tile's words.
+__device__ __forceinline__ int describe_blob(const uint32_t* blob, uint32_t words, uint32_t nb, int lane)
+{
+    const uint32_t padw = (nb + 3) >> 2;
+    if (words < 1u + padw) return 0;
+    const uint32_t lw = (uint32_t)lane < padw ? blob[1 + lane] : 0u;
+    const uint32_t L0 = lw & 0xFFu, L1 = (lw >> 8) & 0xFFu, L2 = (lw >> 16) & 0xFFu, L3 = lw >> 24;
+    bool bad = (lw & 0xE0E0E0E0u) != 0u;   // a code length above 31
+    const uint32_t b0 = 4u * (uint32_t)lane;   // blocks at or beyond nb are padding of the code-length area: must be zero
+    if ((b0 + 0 >= nb && L0) || (b0 + 1 >= nb && L1) || (b0 + 2 >= nb && L2) || (b0 + 3 >= nb && L3)) bad = true;
+    const uint32_t sizes = (L0 ? L0 + 1 : 0) + (L1 ? L1 + 1 : 0) + (L2 ? L2 + 1 : 0) + (L3 ? L3 + 1 : 0);
+    const uint32_t total = __reduce_add_sync(kFull, sizes);
+    // every partial sum of deltas is below sum_b 32 * 2^L_b; with the outlier it must stay below 2^24
+    const uint32_t Lmax = max(max(L0, L1), max(L2, L3));
+    uint32_t spread = 1u << 24;
+    if (Lmax <= 18u) spread = (32u << L0) + (32u << L1) + (32u << L2) + (32u << L3);
+    spread = __reduce_add_sync(kFull, min(spread, 1u << 24));   // at most 32 * 2^24 = 2^29: no overflow
+    if (__any_sync(kFull, bad) || 1u + padw + total != words) return 0;
+    const int32_t outlier = (int32_t)blob[0];
+    const uint32_t ao = (uint32_t)(outlier < 0 ? -outlier : outlier);
+    return (ao < (1u << 23) && spread < (1u << 23)) ? 1 : 2;
+}
+
+// A block's sign word and planes (payload words pay[0 .. L]) as N-bit packed words ready for the inverse transpose,
+// N = 8, 16 or 32 (code lengths up to N), and the block's sum of deltas.
+template <int N>
+__device__ __forceinline__ int32_t load_planes(const uint32_t* pay, uint32_t L, uint32_t& sign, uint32_t (&w)[N])
+{
+    sign = L ? pay[0] : 0u;
+    int32_t total = 0;
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+        w[k] = (uint32_t)k < L ? pay[1 + k] : 0u;
+        // elements with the bit set count 2^k each, negative ones with the opposite sign
+        total += (__popc(w[k]) - 2 * __popc(w[k] & sign)) << k;
+    }
+    return total;
+}
+
+// The lane's 32 elements from the transposed words (word i, field h = magnitude of element N h + i), written as
+// values into the lane's row of a stage.  F32: codes are exact in fp32 (`code` runs in float); otherwise integers.
+template <int N, bool F32>
+__device__ __forceinline__ void expand_block(uint32_t (&w)[N], uint32_t sign, int32_t code_in_front, float s, char* row, uint32_t sw)
+{
+    float runf = (float)code_in_front;
+    int32_t runi = code_in_front;
+    constexpr int kFields = 32 / N;   // elements per word
+#pragma unroll 1
+    for (int h = 0; h < kFields; ++h) {
+#pragma unroll
+        for (int q = 0; q < N / 4; ++q) {
+            float o[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int i = 4 * q + e;
+                const uint32_t mag = N == 32 ? w[i] : (w[i] & ((1u << (N & 31)) - 1u));
+                if (N != 32) w[i] >>= (N & 31);
+                const uint32_t neg = (sign >> i) & 1u;
+                if (F32) {
+                    // the magnitude as an exact float from its bits, the sign on top
+                    const float m = __fsub_rn(__uint_as_float(mag | 0x4B000000u), kTwo23);
+                    runf = __fadd_rn(runf, __uint_as_float(__float_as_uint(m) | (neg << 31)));
+                    o[e] = __fmul_rn(runf, s);
+                } else {
+                    runi += neg ? -(int32_t)mag : (int32_t)mag;
+                    o[e] = __fmul_rn(__int2float_rn(runi), s);
+                }
+            }
+            *reinterpret_cast<float4*>(row + ((16u * (uint32_t)(h * (N / 4) + q)) ^ sw)) = make_float4(o[0], o[1], o[2], o[3]);
+        }
+        sign >>= (N & 31);
+    }
+}
+
+constexpr int kDecBlobWords = 1024 + 8;   // staged blobs: up to 4 KiB plus the slack of the 16-byte-aligned cover
+struct alignas(1024) DecWarpShared {
+    float out[2][kRound];                  // each on a 1024-byte boundary
+    alignas(16) uint32_t blob[2][kDecBlobWords];
+    alignas(8) unsigned long long bar[2];
+};
+static_assert(sizeof(DecWarpShared) == 17 * 1024, "a warp's share of the shared memory");
+
+// Where a tile's blob is, as known from the index alone.
+struct BlobRef {
+    const uint32_t* ptr;    // nullptr: no blob (tile beyond the stream, or a stream that does not parse)
+    uint32_t words;
+    bool staged;            // a bulk copy of its 16-byte-aligned cover is on its way
+};
+
+// Tiled tensor store of a stage to rows [row0, row0 + 32) of the array behind `map` (one thread).
+__device__ __forceinline__ void tensor_store_round(const CUtensorMap* map, uint32_t row0, const float* stage)
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(0), "r"((int)row0), "r"(smem_u32(stage)) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// The same for ragged ends and unaligned arrays: `count` elements of the stage, coalesced.
+__device__ __noinline__ void store_round_ragged(float* __restrict__ y, const float* stage, uint32_t count, int lane)
+{
+#pragma unroll 4
+    for (int k = 0; k < 32; ++k) {
+        const uint32_t e = 32u * k + (uint32_t)lane;
+        if (e < count) y[e] = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(stage) + stage_chunk_byte(k, (uint32_t)lane >> 2) + 4 * (lane & 3));
+    }
+}
+
+// One round of a tile: blocks 32 rd + lane.  blob: the tile's words (shared or global memory); pay_off: payload words
+// of the rounds before; code: the code in front of the round.  Leaves the values in the stage.
+template <bool F32>
+__device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t& pay_off, int32_t& code, float s,
+                                             float* stage, int lane)
+{
+    const uint32_t bi = 32u * rd + (uint32_t)lane;
+    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
+    const uint32_t nw = L ? L + 1u : 0u;
+    const uint32_t incl = warp_incl_scan(nw, lane);
+    const uint32_t* pay = blob + 1 + padw + pay_off + (incl - nw);
+    pay_off += __shfl_sync(kFull, incl, 31);
+    char* row = reinterpret_cast<char*>(stage) + 128 * lane;
+    const uint32_t sw = ((uint32_t)lane & 7u) << 4;
+    // The block's sum of deltas first, so that the scan over the lanes gives the code in front of every block before
+    // any element is expanded.  The lanes of a warp mostly share one width class.
+    uint32_t sign;
+    int32_t total;
+    const unsigned wide = __ballot_sync(kFull, L > 8u), wider = __ballot_sync(kFull, L > 16u);
+    if (!wide) {
+        uint32_t w[8];
+        total = load_planes<8>(pay, L, sign, w);
+        int32_t inc = total;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int32_t v = __shfl_up_sync(kFull, inc, d);
+            if (lane >= d) inc += v;
+        }
+        bit_transpose<8>(w);
+        expand_block<8, F32>(w, sign, code + inc - total, s, row, sw);
+        code += __shfl_sync(kFull, inc, 31);
+    } else if (!wider) {
+        uint32_t w[16];
+        total = load_planes<16>(pay, L, sign, w);
+        int32_t inc = total;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int32_t v = __shfl_up_sync(kFull, inc, d);
+            if (lane >= d) inc += v;
+        }
+        bit_transpose<16>(w);
+        expand_block<16, F32>(w, sign, code + inc - total, s, row, sw);
+        code += __shfl_sync(kFull, inc, 31);
+    } else {
+        uint32_t w[32];
+        total = load_planes<32>(pay, L, sign, w);
+        int32_t inc = total;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int32_t v = __shfl_up_sync(kFull, inc, d);
+            if (lane >= d) inc += v;
+        }
+        bit_transpose<32>(w);
+        expand_block<32, false>(w, sign, code + inc - total, s, row, sw);
+        code += __shfl_sync(kFull, inc, 31);
+    }
+}
+
+__global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
+                                                                        Workspace ws)
+{
+    pdl_enter();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    DecWarpShared& sh = reinterpret_cast<DecWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
+    uint32_t status = 0;
+    if (lane == 0) {
+        mbar_init(&sh.bar[0], 1);
+        mbar_init(&sh.bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed per blob buffer (phase parity of its mbarrier)
+
+    // the job of the tile looked up last, with its stream's header
+    int cj = -1;
+    uint32_t cj_begin = 0, cj_count = 0;
+    StreamInfo h;
+    h.ok = false; h.n = 0; h.nT = 0; h.s = 1.0f; h.eb_abs = 0.0f;
+    auto enter_job = [&](uint32_t t) {
+        if (t - cj_begin >= cj_count) {
+            cj = find_job(jb, t);
+            const Job& q = jb.job[cj];
+            cj_begin = q.tile_begin;
+            cj_count = (cj + 1 < jb.count ? jb.job[cj + 1].tile_begin : jb.total_tiles) - cj_begin;
+            h = read_header(q.in_c, q.in_cap);
+        }
+    };
+    // The blob of tile t of the launch, from the index alone; its 16-byte-aligned cover is requested into blob buffer
+    // `buf` when it fits there and lies inside the readable bytes.  Uniform over the warp.
+    auto request = [&](uint32_t t, uint32_t buf) {
+        BlobRef br;
+        br.ptr = nullptr; br.words = 0; br.staged = false;
+        if (t >= jb.total_tiles) return br;
+        enter_job(t);
+        const Job& q = jb.job[cj];
+        const uint32_t tile = t - cj_begin;
+        if (!h.ok || h.n > q.n || tile >= h.nT) return br;
+        const uint32_t* idx = q.in_c + kHeaderWords;
+        const uint32_t w_end = ldg_u32(idx + tile), w_beg = tile ? ldg_u32(idx + tile - 1) : 0u;
+        const unsigned long long blob0 = (unsigned long long)kHeaderWords + h.nT;
+        if (w_end <= w_beg || (blob0 + w_end) * 4ull > q.in_cap) { br.words = 0xFFFFFFFFu; return br; }   // marks a damaged index
+        br.ptr = q.in_c + blob0 + w_beg;
+        br.words = w_end - w_beg;
+        const uintptr_t b = (uintptr_t)br.ptr, e = (uintptr_t)(br.ptr + br.words);
+        const uintptr_t a_beg = b & ~(uintptr_t)15, a_end = (e + 15) & ~(uintptr_t)15;
+        if (a_end - a_beg <= (uintptr_t)(kDecBlobWords * 4) && a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {
+            if (lane == 0) {
+                mbar_expect_tx(&sh.bar[buf], (uint32_t)(a_end - a_beg));
+                bulk_load(sh.blob[buf], (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar[buf]);
+            }
+            br.staged = true;
+        }
+        return br;
+    };
+
+    const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
+    uint32_t t = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
+    uint32_t p = 0;    // blob buffer of the current tile
+    uint32_t so = 0;   // output stage to use next
+    BlobRef cur = request(t, 0);
+    while (t < jb.total_tiles) {
+        // the current tile's facts, before the look-up of the next tile moves on to another job
+        enter_job(t);
+        const Job& job = jb.job[cj];
+        const uint32_t tile = t - cj_begin;
+        const StreamInfo hc = h;
+        const int jcur = cj;
+        const bool job_bad = !hc.ok, too_small = hc.ok && hc.n > job.n;
+        __syncwarp();   // every lane is done with the other blob buffer
+        const uint32_t tn = t + stride < t ? 0xFFFFFFFFu : t + stride;
+        const BlobRef nxt = request(tn, p ^ 1u);
+        if (cur.staged) {
+            if (!mbar_wait(&sh.bar[p], (p ? fills1 : fills0) & 1u)) status |= kStTimeout;
+            if (p) ++fills1; else ++fills0;
+        }
+        if (job_bad) status |= kStBadStream;
+        else if (too_small) status |= kStCapacity;
+        else if (cur.words == 0xFFFFFFFFu) status |= kStBadStream;
+        else if (cur.ptr) {
+            const unsigned long long start = (unsigned long long)tile * kTile;
+            const uint32_t len = (uint32_t)((hc.n - start < (unsigned long long)kTile) ? (hc.n - start) : kTile);
+            const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2;
+            const uint32_t* blob = cur.staged ? sh.blob[p] + ((((uintptr_t)cur.ptr) & 15u) >> 2) : cur.ptr;
+            const int mode = describe_blob(blob, cur.words, nb, lane);
+            if (mode == 0) status |= kStBadStream;
+            else {
+                float* __restrict__ y = job.y + start;
+                const bool mapped = (((uintptr_t)job.y) & 15u) == 0;
+                uint32_t pay_off = 0;
+                int32_t code = (int32_t)blob[0];
+                const uint32_t rounds = (nb + 31) >> 5;
+                for (uint32_t rd = 0; rd < rounds; ++rd) {
+                    // the stage about to be written was handed to a tensor store two rounds ago
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                    float* stage = sh.out[so];
+                    if (mode == 1) decode_round<true>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
+                    else decode_round<false>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
+                    __syncwarp();   // the stage's rows, written by all lanes, are visible
+                    const uint32_t e0 = rd * (uint32_t)kRound;
+                    if (mapped && e0 + (uint32_t)kRound <= len) {
+                        if (lane == 0) tensor_store_round(&maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), stage);
+                        so ^= 1u;
+                    } else {
+                        store_round_ragged(y + e0, stage, len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound, lane);
+                    }
+                }
+            }
+        }
+        cur = nxt;
+        t = tn;
+        p ^= 1u;
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (status) atomicOr(ws.status, status);
+}
+
 // Per-device launch set-up (shared-memory attribute, resident CTAs per SM), done once per device under a lock.
 constexpr int kMaxDevices = 64;
 constexpr size_t kEncSmemBytes = sizeof(EncWarpShared) * kCodecWarps + 1024;   // + room to reach a 1024-byte boundary
 constexpr size_t kRoundSmemBytes = sizeof(RoundWarpShared) * kCodecWarps + 1024;
+constexpr size_t kDecSmemBytes = sizeof(DecWarpShared) * kCodecWarps + 1024;
 struct DeviceSetup {
     bool ready = false;
-    int enc_ctas = 1, round_ctas = 1;
+    int enc_ctas = 1, round_ctas = 1, dec_ctas = 1;
 };
 DeviceSetup g_dev[kMaxDevices];
 std::mutex g_dev_mu;
@@ -1257,6 +1554,11 @@ cudaError_t device_setup(const DeviceSetup** out)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_rounds_kernel, kCodecThreads, kRoundSmemBytes);
         if (e != cudaSuccess) return e;
         d.round_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(decode_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_kernel, kCodecThreads, kDecSmemBytes);
+        if (e != cudaSuccess) return e;
+        d.dec_ctas = a > 0 ? a : 1;
         d.ready = true;
     }
     *out = &d;
@@ -1279,6 +1581,20 @@ cudaError_t make_row_map(CUtensorMap* map, const float* x, unsigned long long n)
 }
 
 }  // namespace
+
+cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    const DeviceSetup* d = nullptr;
+    cudaError_t e = device_setup(&d);
+    if (e != cudaSuccess) return e;
+    TileMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    for (int j = 0; j < jb.count; ++j)
+        if ((e = make_row_map(&maps.m[j], jb.job[j].y, jb.job[j].n)) != cudaSuccess) return e;
+    const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
+    const unsigned long long cap = (unsigned long long)sm_count * d->dec_ctas;
+    return launch_k(decode_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kDecSmemBytes, st, jb, maps, ws);
+}
 
 #ifdef ZCCL_TRACE
 extern "C" int zccl_debug_rec(unsigned long long* out, int n) { return cudaMemcpyFromSymbol(out, g_rec, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -1; }

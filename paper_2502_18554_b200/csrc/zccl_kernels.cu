@@ -1871,6 +1871,10 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
     if (jb.total_tiles == 0) return cudaSuccess;
+    if (lanes_engine()) {
+        ++g_launches;
+        return launch_decode_lanes(jb, ws, sm_count, st);
+    }
     if (g_decode_ctas_per_sm == 0) {
         int a = 0;
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_kernel, kThreads, 0);
