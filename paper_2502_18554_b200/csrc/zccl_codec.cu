@@ -894,6 +894,54 @@ __device__ __noinline__ uint32_t encode_round_general(const float* __restrict__ 
     return status;
 }
 
+// The same for a round whose values sit in a stage (the hop's sums): block `lane` of the round from the lane's row.
+__device__ __noinline__ uint32_t encode_round_general_staged(const float* stage, float xprev, bool active, uint32_t rd, float r,
+                                                             uint32_t* __restrict__ slot, uint32_t* round_words, int32_t* outlier,
+                                                             unsigned long long* group_words, int lane)
+{
+    uint32_t status = 0;
+    const char* row = reinterpret_cast<const char*>(stage) + 128 * lane;
+    const uint32_t sw = ((uint32_t)lane & 7u) << 4;
+    uint32_t m[32];
+    uint32_t sg = 0, ob = 0;
+    const float tp = __fmul_rn(xprev, r);
+    float tm = fabsf(tp);
+    uint32_t qp = (uint32_t)__float2int_rn(tp);
+    const int32_t q0 = __float2int_rn(__fmul_rn(*reinterpret_cast<const float*>(row + sw), r));
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const float x = *reinterpret_cast<const float*>(row + ((16u * (uint32_t)(j >> 2)) ^ sw) + 4 * (j & 3));
+        const float tt = __fmul_rn(x, r);
+        tm = fmaxf(tm, fabsf(tt));
+        const uint32_t q = (uint32_t)__float2int_rn(tt);
+        const int32_t dd = (int32_t)(q - qp);
+        qp = q;
+        const uint32_t sm = (uint32_t)(dd >> 31);
+        m[j] = (((uint32_t)dd ^ sm) - sm) & 0x7FFFFFFFu;
+        ob |= m[j];
+        sg = __funnelshift_l((uint32_t)dd, sg, 1);
+    }
+    uint32_t L = active ? code_length(ob) : 0u;
+    if (active) {
+        if (!(tm < 1073741824.0f)) status |= kStRange;
+        else if (tm > 32768.5f) status |= kStPrecision;
+    }
+    bit_transpose<32>(m);
+    const uint32_t nw = L ? L + 1u : 0u;
+    const uint32_t incl = warp_incl_scan(nw, lane);
+    reinterpret_cast<unsigned char*>(slot)[lane] = (unsigned char)L;
+    if (L) {
+        uint32_t* d = slot + 8 + (incl - nw);
+        d[0] = __brev(sg);
+#pragma unroll
+        for (int k = 0; k < 31; ++k)
+            if ((uint32_t)k < L) d[1 + k] = m[k];
+    }
+    if (lane == 31) { *round_words = incl; atomicAdd(group_words, (unsigned long long)incl); }
+    if (rd == 0 && lane == 0) *outlier = q0;
+    return status;
+}
+
 __global__ void __launch_bounds__(kCodecThreads, 4) encode_rounds_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
                                                                          Workspace ws, Params hp, int use_dev_params)
 {
@@ -1046,7 +1094,7 @@ struct GroupTable {
 constexpr int kPlaceThreads = 1024;   // one warp per tile of the group
 
 __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ GroupTable gt, Workspace ws,
-                                                              Params hp, int use_dev_params)
+                                                              Params hp, int use_dev_params, int from_stream)
 {
     pdl_enter();
     __shared__ uint32_t s_words[32], s_off[32], s_part[kPlaceThreads / 32], s_base, s_ok;
@@ -1069,6 +1117,15 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
     if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 0] = gtime();
 #endif
     const Job& job = jb.job[j];
+    if (from_stream) {   // a hop: bound and step are the incoming stream's, and the job counts only if its streams agree with it
+        const StreamInfo h1 = read_header(job.in_c, job.in_cap);
+        bool ok = h1.ok && h1.n == job.n;
+        if (job.in_c2) {
+            const StreamInfo h2 = read_header(job.in_c2, job.in2_cap);
+            ok = ok && h2.ok && h2.n == job.n && __float_as_uint(h2.s) == __float_as_uint(h1.s);
+        }
+        prm.eb_abs = h1.eb_abs; prm.s = h1.s; prm.valid = ok ? 1 : 0;
+    }
     const uint32_t g = blockIdx.x - gt.begin[j];
     const uint32_t tiles = (j + 1 < jb.count ? jb.job[j + 1].tile_begin : jb.total_tiles) - job.tile_begin;
     const unsigned long long n = job.n;
@@ -1267,8 +1324,17 @@ __device__ __forceinline__ int32_t load_planes(const uint32_t* pay, uint32_t L, 
 
 // The lane's 32 elements from the transposed words (word i, field h = magnitude of element N h + i), written as
 // values into the lane's row of a stage.  F32: codes are exact in fp32 (`code` runs in float); otherwise integers.
-template <int N, bool F32>
-__device__ __forceinline__ void expand_block(uint32_t (&w)[N], uint32_t sign, int32_t code_in_front, float s, char* row, uint32_t sw)
+// Reduce operation of the hop: 0 = sum, 1 = max, 2 = min, 3 = average (a sum on every hop); of two operands that
+// compare equal Max and Min keep the decoded one.
+__device__ __forceinline__ float combine(uint32_t op, float a, float b)
+{
+    return op == 1u ? ((a < b) ? b : a) : op == 2u ? ((b < a) ? b : a) : __fadd_rn(a, b);
+}
+// MODE 0: plain decoding; 1: every value is added to the operand in the same place of the row `loc`; 2: combined with
+// it by the operation `op`.
+template <int N, bool F32, int MODE>
+__device__ __forceinline__ void expand_block(uint32_t (&w)[N], uint32_t sign, int32_t code_in_front, float s, char* row, uint32_t sw,
+                                             const char* loc, uint32_t op)
 {
     float runf = (float)code_in_front;
     int32_t runi = code_in_front;
@@ -1294,7 +1360,13 @@ __device__ __forceinline__ void expand_block(uint32_t (&w)[N], uint32_t sign, in
                     o[e] = __fmul_rn(__int2float_rn(runi), s);
                 }
             }
-            *reinterpret_cast<float4*>(row + ((16u * (uint32_t)(h * (N / 4) + q)) ^ sw)) = make_float4(o[0], o[1], o[2], o[3]);
+            const uint32_t at = (16u * (uint32_t)(h * (N / 4) + q)) ^ sw;
+            if (MODE != 0) {
+                const float4 l = *reinterpret_cast<const float4*>(loc + at);
+                if (MODE == 1) { o[0] = __fadd_rn(o[0], l.x); o[1] = __fadd_rn(o[1], l.y); o[2] = __fadd_rn(o[2], l.z); o[3] = __fadd_rn(o[3], l.w); }
+                else { o[0] = combine(op, o[0], l.x); o[1] = combine(op, o[1], l.y); o[2] = combine(op, o[2], l.z); o[3] = combine(op, o[3], l.w); }
+            }
+            *reinterpret_cast<float4*>(row + at) = make_float4(o[0], o[1], o[2], o[3]);
         }
         sign >>= (N & 31);
     }
@@ -1335,9 +1407,10 @@ __device__ __noinline__ void store_round_ragged(float* __restrict__ y, const flo
 
 // One round of a tile: blocks 32 rd + lane.  blob: the tile's words (shared or global memory); pay_off: payload words
 // of the rounds before; code: the code in front of the round.  Leaves the values in the stage.
-template <bool F32>
+// MODE, loc_stage, op: see expand_block (loc_stage: the stage that holds the operand's round; may be `stage` itself).
+template <bool F32, int MODE>
 __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t& pay_off, int32_t& code, float s,
-                                             float* stage, int lane)
+                                             float* stage, int lane, const float* loc_stage = nullptr, uint32_t op = 0)
 {
     const uint32_t bi = 32u * rd + (uint32_t)lane;
     const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
@@ -1346,6 +1419,7 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
     const uint32_t* pay = blob + 1 + padw + pay_off + (incl - nw);
     pay_off += __shfl_sync(kFull, incl, 31);
     char* row = reinterpret_cast<char*>(stage) + 128 * lane;
+    const char* loc = reinterpret_cast<const char*>(loc_stage) + 128 * lane;
     const uint32_t sw = ((uint32_t)lane & 7u) << 4;
     // The block's sum of deltas first, so that the scan over the lanes gives the code in front of every block before
     // any element is expanded.  The lanes of a warp mostly share one width class.
@@ -1362,7 +1436,7 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
             if (lane >= d) inc += v;
         }
         bit_transpose<8>(w);
-        expand_block<8, F32>(w, sign, code + inc - total, s, row, sw);
+        expand_block<8, F32, MODE>(w, sign, code + inc - total, s, row, sw, loc, op);
         code += __shfl_sync(kFull, inc, 31);
     } else if (!wider) {
         uint32_t w[16];
@@ -1374,7 +1448,7 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
             if (lane >= d) inc += v;
         }
         bit_transpose<16>(w);
-        expand_block<16, F32>(w, sign, code + inc - total, s, row, sw);
+        expand_block<16, F32, MODE>(w, sign, code + inc - total, s, row, sw, loc, op);
         code += __shfl_sync(kFull, inc, 31);
     } else {
         uint32_t w[32];
@@ -1386,7 +1460,7 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
             if (lane >= d) inc += v;
         }
         bit_transpose<32>(w);
-        expand_block<32, false>(w, sign, code + inc - total, s, row, sw);
+        expand_block<32, false, MODE>(w, sign, code + inc - total, s, row, sw, loc, op);
         code += __shfl_sync(kFull, inc, 31);
     }
 }
@@ -1490,8 +1564,8 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                     float* stage = sh.out[so];
-                    if (mode == 1) decode_round<true>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
-                    else decode_round<false>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
+                    if (mode == 1) decode_round<true, 0>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
+                    else decode_round<false, 0>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
                     __syncwarp();   // the stage's rows, written by all lanes, are visible
                     const uint32_t e0 = rd * (uint32_t)kRound;
                     if (mapped && e0 + (uint32_t)kRound <= len) {
@@ -1511,14 +1585,276 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
     if (status) atomicOr(ws.status, status);
 }
 
+// ------------------------------------------------------------------------------------------------ fused hop
+//
+// out = compress(decompress(in_c) (+) local), tile by tile, with no uncompressed intermediate in global memory: a
+// warp decodes a round of the incoming tile straight onto the local operand's round (tensor copy, one round ahead;
+// or a second compressed stream, decoded first), leaves the combined values in a stage, and encodes that stage like
+// a round of the compressor: into a buffer, off to the round's slot by a bulk store.  The place kernel finishes the
+// stream.  An uncompressed copy of the result, when asked for, leaves the stage by a tensor store.
+
+__device__ __forceinline__ uint32_t cj_begin_of(const JobBatch& jb, int j) { return jb.job[j].tile_begin; }
+
+struct alignas(1024) HopWarpShared {
+    float loc[2][kRound];                  // the operand's rounds; each on a 1024-byte boundary
+    float ys[kRound];                      // decoded (+) operand
+    alignas(16) uint32_t blob[2][kDecBlobWords];
+    alignas(16) uint32_t out[2][kRoundBufWords];
+    alignas(8) unsigned long long bar_loc[2], bar_blob[2];
+};
+static_assert(sizeof(HopWarpShared) == 25 * 1024, "a warp's share of the shared memory");
+
+// The owner's copy as the dequantised value float(q(y)) * s: `count` elements of the stage, coalesced.
+__device__ __noinline__ void store_round_dequantised(float* __restrict__ y, const float* stage, uint32_t count, float r, float s, int lane)
+{
+#pragma unroll 4
+    for (int k = 0; k < 32; ++k) {
+        const uint32_t e = 32u * k + (uint32_t)lane;
+        const float v = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(stage) + stage_chunk_byte(k, (uint32_t)lane >> 2) + 4 * (lane & 3));
+        if (e < count) y[e] = __fmul_rn(__int2float_rn(__float2int_rn(__fmul_rn(v, r))), s);
+    }
+}
+
+__global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps loc_maps,
+                                                                     const __grid_constant__ TileMaps raw_maps, Workspace ws)
+{
+    pdl_enter();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    HopWarpShared& sh = reinterpret_cast<HopWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
+    uint32_t status = 0;
+    if (lane == 0) {
+        mbar_init(&sh.bar_loc[0], 1); mbar_init(&sh.bar_loc[1], 1);
+        mbar_init(&sh.bar_blob[0], 1); mbar_init(&sh.bar_blob[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    uint32_t lfill0 = 0, lfill1 = 0, bfill0 = 0, bfill1 = 0;   // completed copies per buffer (phase parities)
+    bool lbulk0 = false, lbulk1 = false;
+
+    // the job of the tile looked up last, with its streams' headers
+    int cj = -1;
+    uint32_t cj_begin = 0, cj_count = 0;
+    StreamInfo h1, h2;
+    h1.ok = h2.ok = false; h1.n = h2.n = 0; h1.nT = h2.nT = 0; h1.s = h2.s = 1.0f; h1.eb_abs = h2.eb_abs = 0.0f;
+    bool job_ok = false;
+    auto enter_job = [&](uint32_t t) {
+        if (t - cj_begin >= cj_count) {
+            cj = find_job(jb, t);
+            const Job& q = jb.job[cj];
+            cj_begin = q.tile_begin;
+            cj_count = (cj + 1 < jb.count ? jb.job[cj + 1].tile_begin : jb.total_tiles) - cj_begin;
+            h1 = read_header(q.in_c, q.in_cap);
+            job_ok = h1.ok && h1.n == q.n;
+            if (q.in_c2) {
+                h2 = read_header(q.in_c2, q.in2_cap);
+                job_ok = job_ok && h2.ok && h2.n == q.n && __float_as_uint(h2.s) == __float_as_uint(h1.s);
+            }
+        }
+    };
+    // a tile's blob out of one of the job's streams, from the index alone (ptr = nullptr, words = ~0: damaged index)
+    auto blob_of = [&](const uint32_t* in, unsigned long long cap, uint32_t nT, uint32_t tile) {
+        BlobRef br;
+        br.ptr = nullptr; br.words = 0xFFFFFFFFu; br.staged = false;
+        const uint32_t* idx = in + kHeaderWords;
+        const uint32_t w_end = ldg_u32(idx + tile), w_beg = tile ? ldg_u32(idx + tile - 1) : 0u;
+        const unsigned long long blob0 = (unsigned long long)kHeaderWords + nT;
+        if (w_end <= w_beg || (blob0 + w_end) * 4ull > cap) return br;
+        br.ptr = in + blob0 + w_beg;
+        br.words = w_end - w_beg;
+        return br;
+    };
+    // the incoming blob of tile t of the launch; its cover is requested into blob buffer `buf` when it fits
+    auto request_blob = [&](uint32_t t, uint32_t buf) {
+        BlobRef br;
+        br.ptr = nullptr; br.words = 0; br.staged = false;
+        if (t >= jb.total_tiles) return br;
+        enter_job(t);
+        const Job& q = jb.job[cj];
+        const uint32_t tile = t - cj_begin;
+        if (!job_ok || q.n == 0 || tile >= h1.nT) return br;
+        br = blob_of(q.in_c, q.in_cap, h1.nT, tile);
+        if (!br.ptr) return br;
+        const uintptr_t b = (uintptr_t)br.ptr, e = (uintptr_t)(br.ptr + br.words);
+        const uintptr_t a_beg = b & ~(uintptr_t)15, a_end = (e + 15) & ~(uintptr_t)15;
+        if (a_end - a_beg <= (uintptr_t)(kDecBlobWords * 4) && a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {
+            if (lane == 0) {
+                mbar_expect_tx(&sh.bar_blob[buf], (uint32_t)(a_end - a_beg));
+                bulk_load(sh.blob[buf], (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar_blob[buf]);
+            }
+            br.staged = true;
+        }
+        return br;
+    };
+    // round rd of the uncompressed operand of tile `tile` of the current job into operand stage `buf`
+    auto request_loc = [&](int job_index, uint32_t tile, uint32_t rd, uint32_t buf) {
+        bool bulk = false;
+        const Job& q = jb.job[job_index];
+        if (q.x) {
+            const unsigned long long start = (unsigned long long)tile * kTile;
+            const uint32_t len = (uint32_t)((q.n - start < (unsigned long long)kTile) ? (q.n - start) : kTile);
+            const uint32_t e0 = rd * (uint32_t)kRound;
+            if (e0 < len) {
+                if ((((uintptr_t)q.x) & 15u) == 0 && e0 + (uint32_t)kRound <= len) {
+                    if (lane == 0) tensor_load_round(sh.loc[buf], &sh.bar_loc[buf], &loc_maps.m[job_index], tile * (uint32_t)kBlocksPerTile + (e0 >> 5));
+                    bulk = true;
+                } else load_round_ragged(sh.loc[buf], q.x + start, e0, len, lane);
+            }
+        }
+        if (buf) lbulk1 = bulk; else lbulk0 = bulk;
+    };
+    auto arrive_loc = [&](uint32_t buf) {
+        if (buf ? lbulk1 : lbulk0) {
+            if (!mbar_wait(&sh.bar_loc[buf], (buf ? lfill1 : lfill0) & 1u)) status |= kStTimeout;
+            if (buf) ++lfill1; else ++lfill0;
+        }
+        if (buf) lbulk1 = false; else lbulk0 = false;
+        __syncwarp();
+    };
+
+    const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
+    uint32_t t = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
+    uint32_t pb = 0, pl = 0, po = 0;   // blob buffer, operand stage and output buffer in turn
+    BlobRef cur = request_blob(t, 0);
+    if (t < jb.total_tiles && job_ok && jb.job[cj].n) request_loc(cj, t - cj_begin, 0, 0);
+    EncodeCarry cy;
+    cy.pay_used = 0; cy.wide = false;
+
+    while (t < jb.total_tiles) {
+        // the current tile's facts, before the look-up of the next tile moves on to another job
+        enter_job(t);
+        const int jcur = cj;
+        const Job& job = jb.job[jcur];
+        const uint32_t tile = t - cj_begin;
+        const StreamInfo hc1 = h1, hc2 = h2;
+        const bool ok = job_ok;
+        const unsigned long long n = job.n;
+        const float s = hc1.s, r = __fdiv_rn(1.0f, hc1.s);
+        const unsigned long long start = (unsigned long long)tile * kTile;
+        const uint32_t len = (ok && n) ? (uint32_t)((n - start < (unsigned long long)kTile) ? (n - start) : kTile) : 0u;
+        const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2, rounds = (nb + 31) >> 5;
+        const uint32_t op = (job.flags >> 1) & 3u;
+        const bool summing = op == 0u || op == 3u, deq = (job.flags & 1u) != 0;
+        if (!ok) status |= kStBadStream;
+
+        __syncwarp();   // every lane is done with the other blob buffer
+        const uint32_t tn = t + stride < t ? 0xFFFFFFFFu : t + stride;
+        const BlobRef nxt = request_blob(tn, pb ^ 1u);   // moves the job look-up on to the next tile
+        const bool next_has_operand = tn < jb.total_tiles && job_ok && jb.job[cj].n != 0;
+        const int njob = cj;
+        const uint32_t ntile = tn - cj_begin;
+        if (cur.staged) {
+            if (!mbar_wait(&sh.bar_blob[pb], (pb ? bfill1 : bfill0) & 1u)) status |= kStTimeout;
+            if (pb) ++bfill1; else ++bfill0;
+        }
+
+        // what the two blobs say
+        const uint32_t* blob1 = nullptr;
+        const uint32_t* blob2 = nullptr;
+        int mode1 = 0, mode2 = 1;
+        if (len) {
+            if (cur.ptr) {
+                blob1 = cur.staged ? sh.blob[pb] + ((((uintptr_t)cur.ptr) & 15u) >> 2) : cur.ptr;
+                mode1 = describe_blob(blob1, cur.words, nb, lane);
+            }
+            if (job.in_c2) {
+                const BlobRef b2 = blob_of(job.in_c2, job.in2_cap, hc2.nT, tile);
+                blob2 = b2.ptr;
+                mode2 = b2.ptr ? describe_blob(b2.ptr, b2.words, nb, lane) : 0;
+            }
+            if (mode1 == 0 || mode2 == 0) status |= kStBadStream;
+        }
+        const bool good = len != 0 && mode1 != 0 && mode2 != 0;
+
+        uint32_t pay1 = 0, pay2 = 0;
+        int32_t code1 = good ? (int32_t)blob1[0] : 0, code2 = (good && blob2) ? (int32_t)blob2[0] : 0;
+        float carry_y = 0.0f;
+        for (uint32_t rd = 0; rd < rounds; ++rd) {
+            __syncwarp();   // every lane is done with the other operand stage
+            if (rd + 1 < rounds) request_loc(jcur, tile, rd + 1, pl ^ 1u);
+            else if (next_has_operand) request_loc(njob, ntile, 0, pl ^ 1u);
+            else { if (pl) lbulk0 = false; else lbulk1 = false; }
+            arrive_loc(pl);
+            const uint32_t u = 4u * t + rd;
+            if (!good) {
+                if (lane == 0) ws.round_words[u] = 0;
+            } else {
+                float* loc = sh.loc[pl];
+                if (blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
+                    if (mode2 == 1) decode_round<true, 0>(blob2, padw, nb, rd, pay2, code2, s, loc, lane);
+                    else decode_round<false, 0>(blob2, padw, nb, rd, pay2, code2, s, loc, lane);
+                    __syncwarp();
+                }
+                // the stage and the buffer about to be written were handed to the copy engine one and two rounds ago
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
+                if (mode1 == 1) {
+                    if (summing) decode_round<true, 1>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
+                    else decode_round<true, 2>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
+                } else {
+                    if (summing) decode_round<false, 1>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
+                    else decode_round<false, 2>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
+                }
+                __syncwarp();   // the stage's rows, written by all lanes, are visible
+                const float* ys = sh.ys;
+                const char* row = reinterpret_cast<const char*>(ys) + 128 * lane;
+                const uint32_t sw = ((uint32_t)lane & 7u) << 4;
+                const float y0 = ys[0];
+                const float xprev = lane ? read_last_of_row(ys, (uint32_t)lane - 1u) : (rd ? carry_y : y0);
+                carry_y = read_last_of_row(ys, 31);
+                const uint32_t e0 = rd * (uint32_t)kRound;
+                if (job.y) {
+                    const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
+                    if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
+                    else if ((((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
+                        if (lane == 0) tensor_store_round(&raw_maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), ys);
+                    } else store_round_ragged(job.y + start + e0, ys, count, lane);
+                }
+                uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
+                uint32_t* buf = sh.out[po];
+                cy.pay_used = 0;
+                const uint32_t bi = 32u * rd + (uint32_t)lane;
+                const int rc = encode_round(row, sw, xprev, r, bi < nb, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, cy, lane,
+                                            status);
+                const uint32_t gslot = (cj_begin_of(jb, jcur) >> 5) + (uint32_t)jcur + (tile >> 5);
+                if (rc == 0) {
+                    __syncwarp();   // the buffer's words, written by all lanes, are visible to lane 0's store
+                    if (lane == 0) {
+                        const uint32_t bytes = (32u + 4u * cy.pay_used + 15u) & ~15u;
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(slot), "r"(smem_u32(buf)), "r"(bytes) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                        ws.round_words[u] = cy.pay_used;
+                        atomicAdd(ws.group_acc + gslot, (unsigned long long)cy.pay_used);
+                        // exact while |y r| < 2^22; larger codes take the general route
+                        if (rd == 0) ws.outliers[t] = (int32_t)(__float_as_uint(__fadd_rn(__fmul_rn(y0, r), kRoundMagic)) - kRoundMagicBits);
+                    }
+                    po ^= 1u;
+                } else {
+                    status |= encode_round_general_staged(ys, xprev, bi < nb, rd, r, slot, ws.round_words + u, ws.outliers + t, ws.group_acc + gslot, lane);
+                }
+            }
+            pl ^= 1u;
+        }
+        if (rounds == 0 && next_has_operand) request_loc(njob, ntile, 0, pl);
+        if ((uint32_t)lane >= rounds && lane < kRoundsPerTile) ws.round_words[4u * t + (uint32_t)lane] = 0;   // rounds the tile does not have
+        cur = nxt;
+        t = tn;
+        pb ^= 1u;
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (status) atomicOr(ws.status, status);
+}
+
 // Per-device launch set-up (shared-memory attribute, resident CTAs per SM), done once per device under a lock.
 constexpr int kMaxDevices = 64;
 constexpr size_t kEncSmemBytes = sizeof(EncWarpShared) * kCodecWarps + 1024;   // + room to reach a 1024-byte boundary
 constexpr size_t kRoundSmemBytes = sizeof(RoundWarpShared) * kCodecWarps + 1024;
 constexpr size_t kDecSmemBytes = sizeof(DecWarpShared) * kCodecWarps + 1024;
+constexpr size_t kHopSmemBytes = sizeof(HopWarpShared) * kCodecWarps + 1024;
 struct DeviceSetup {
     bool ready = false;
-    int enc_ctas = 1, round_ctas = 1, dec_ctas = 1;
+    int enc_ctas = 1, round_ctas = 1, dec_ctas = 1, hop_ctas = 1;
 };
 DeviceSetup g_dev[kMaxDevices];
 std::mutex g_dev_mu;
@@ -1559,6 +1895,11 @@ cudaError_t device_setup(const DeviceSetup** out)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_kernel, kCodecThreads, kDecSmemBytes);
         if (e != cudaSuccess) return e;
         d.dec_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(hop_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, hop_tiles_kernel, kCodecThreads, kHopSmemBytes);
+        if (e != cudaSuccess) return e;
+        d.hop_ctas = a > 0 ? a : 1;
         d.ready = true;
     }
     *out = &d;
@@ -1581,6 +1922,43 @@ cudaError_t make_row_map(CUtensorMap* map, const float* x, unsigned long long n)
 }
 
 }  // namespace
+
+// one CTA of the place kernel per group of 32 tiles of every job
+uint32_t group_table(const JobBatch& jb, GroupTable& gt)
+{
+    uint32_t groups = 0;
+    for (int j = 0; j < jb.count; ++j) {
+        gt.begin[j] = groups;
+        const uint32_t tiles = (j + 1 < jb.count ? jb.job[j + 1].tile_begin : jb.total_tiles) - jb.job[j].tile_begin;
+        groups += (tiles + 31u) / 32u;
+    }
+    for (int j = jb.count; j <= kMaxJobs; ++j) gt.begin[j] = groups;
+    return groups;
+}
+
+cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    const DeviceSetup* d = nullptr;
+    cudaError_t e = device_setup(&d);
+    if (e != cudaSuccess) return e;
+    if (!ws.slots) return cudaErrorInvalidValue;
+    static TileMaps loc_maps, raw_maps;   // too large for the stack of some callers; guarded by the lock below
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    memset(&loc_maps, 0, sizeof(loc_maps));
+    memset(&raw_maps, 0, sizeof(raw_maps));
+    for (int j = 0; j < jb.count; ++j) {
+        if (jb.job[j].x && (e = make_row_map(&loc_maps.m[j], jb.job[j].x, jb.job[j].n)) != cudaSuccess) return e;
+        if (jb.job[j].y && (e = make_row_map(&raw_maps.m[j], jb.job[j].y, jb.job[j].n)) != cudaSuccess) return e;
+    }
+    GroupTable gt;
+    const uint32_t groups = group_table(jb, gt);
+    const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
+    const unsigned long long cap = (unsigned long long)sm_count * d->hop_ctas;
+    e = launch_k(hop_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kHopSmemBytes, st, jb, loc_maps, raw_maps, ws);
+    if (e != cudaSuccess) return e;
+    return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
+}
 
 cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
@@ -1620,20 +1998,14 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
     if (ws.slots && ws.skip_publish == 0xFFFFFFFFu) {
         // two steps: rounds into their slots, then one CTA per group of 32 tiles places them
         GroupTable gt;
-        uint32_t groups = 0;
-        for (int j = 0; j < jb.count; ++j) {
-            gt.begin[j] = groups;
-            const uint32_t tiles = (j + 1 < jb.count ? jb.job[j + 1].tile_begin : jb.total_tiles) - jb.job[j].tile_begin;
-            groups += (tiles + 31u) / 32u;
-        }
-        for (int j = jb.count; j <= kMaxJobs; ++j) gt.begin[j] = groups;
+        const uint32_t groups = group_table(jb, gt);
         const unsigned long long rounds = (unsigned long long)jb.total_tiles * kRoundsPerTile;
         const unsigned long long want_a = (rounds + kCodecWarps - 1) / kCodecWarps;
         const unsigned long long cap_a = (unsigned long long)sm_count * d->round_ctas;
         e = launch_k(encode_rounds_kernel, dim3((unsigned)(want_a < cap_a ? want_a : cap_a)), dim3(kCodecThreads), kRoundSmemBytes, st, jb, maps, ws,
                      host_params, device_params ? 1 : 0);
         if (e != cudaSuccess) return e;
-        return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, host_params, device_params ? 1 : 0);
+        return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, host_params, device_params ? 1 : 0, 0);
     }
     const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     unsigned long long cap = (unsigned long long)sm_count * d->enc_ctas;

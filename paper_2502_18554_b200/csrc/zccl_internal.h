@@ -148,6 +148,7 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
                           Params host_params, int sm_count, cudaStream_t st);
 cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool device_params, Params host_params, int sm_count,
                                 cudaStream_t st);
+cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st);

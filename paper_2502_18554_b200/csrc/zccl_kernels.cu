@@ -1835,8 +1835,12 @@ cudaError_t launch_encode(const JobBatch& jb, EncodeMode mode, const Workspace& 
 {
     if (jb.total_tiles == 0) return cudaSuccess;
     if (mode == kEncodeRaw && lanes_engine()) {
-        ++g_launches;
+        g_launches += ws.slots ? 2 : 1;
         return launch_encode_lanes(jb, ws, device_params, host_params, sm_count, st);
+    }
+    if (mode == kEncodeFused && lanes_engine() && ws.slots) {
+        g_launches += 2;
+        return launch_hop_lanes(jb, ws, sm_count, st);
     }
     if (g_raw_ctas_per_sm == 0) {
         cudaError_t e = cudaFuncSetAttribute(encode_raw_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
