@@ -1323,52 +1323,94 @@ __device__ __forceinline__ int32_t load_planes(const uint32_t* pay, uint32_t L, 
 }
 
 // The lane's 32 elements from the transposed words (word i, field h = magnitude of element N h + i), written as
-// values into the lane's row of a stage.  F32: codes are exact in fp32 (`code` runs in float); otherwise integers.
-// Reduce operation of the hop: 0 = sum, 1 = max, 2 = min, 3 = average (a sum on every hop); of two operands that
-// compare equal Max and Min keep the decoded one.
-__device__ __forceinline__ float combine(uint32_t op, float a, float b)
+// values into the lane's row of a stage.  Codes are exact in fp32 (the caller checked): the magnitude is read as a
+// float from its bits, gets its sign, joins the running code, and one multiplication makes the value.  MODE 0:
+// plain decoding; MODE 1: every value is added to the operand in the same place of the row `loc`.
+template <int N, int MODE>
+__device__ __forceinline__ void expand_block(const uint32_t (&w)[N], uint32_t sign, int32_t code_in_front, float s, char* row, uint32_t sw,
+                                             const char* loc)
 {
-    return op == 1u ? ((a < b) ? b : a) : op == 2u ? ((b < a) ? b : a) : __fadd_rn(a, b);
-}
-// MODE 0: plain decoding; 1: every value is added to the operand in the same place of the row `loc`; 2: combined with
-// it by the operation `op`.
-template <int N, bool F32, int MODE>
-__device__ __forceinline__ void expand_block(uint32_t (&w)[N], uint32_t sign, int32_t code_in_front, float s, char* row, uint32_t sw,
-                                             const char* loc, uint32_t op)
-{
-    float runf = (float)code_in_front;
-    int32_t runi = code_in_front;
-    constexpr int kFields = 32 / N;   // elements per word
+    float run = (float)code_in_front;
+    uint32_t sel = N == 8 ? 0x7650u : 0x7610u;   // byte (pair) h of a word under the exponent of 2^23
 #pragma unroll 1
-    for (int h = 0; h < kFields; ++h) {
+    for (int h = 0; h < 32 / N; ++h) {
 #pragma unroll
         for (int q = 0; q < N / 4; ++q) {
             float o[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int i = 4 * q + e;
-                const uint32_t mag = N == 32 ? w[i] : (w[i] & ((1u << (N & 31)) - 1u));
-                if (N != 32) w[i] >>= (N & 31);
-                const uint32_t neg = (sign >> i) & 1u;
-                if (F32) {
-                    // the magnitude as an exact float from its bits, the sign on top
-                    const float m = __fsub_rn(__uint_as_float(mag | 0x4B000000u), kTwo23);
-                    runf = __fadd_rn(runf, __uint_as_float(__float_as_uint(m) | (neg << 31)));
-                    o[e] = __fmul_rn(runf, s);
-                } else {
-                    runi += neg ? -(int32_t)mag : (int32_t)mag;
-                    o[e] = __fmul_rn(__int2float_rn(runi), s);
-                }
+                const float m = __fsub_rn(__uint_as_float(prmt(w[i], 0x4B000000u, sel)), kTwo23);
+                const uint32_t sbit = (sign << (31 - i)) & 0x80000000u;
+                run = __fadd_rn(run, __uint_as_float(__float_as_uint(m) | sbit));
+                o[e] = __fmul_rn(run, s);
             }
             const uint32_t at = (16u * (uint32_t)(h * (N / 4) + q)) ^ sw;
-            if (MODE != 0) {
+            if (MODE == 1) {
                 const float4 l = *reinterpret_cast<const float4*>(loc + at);
-                if (MODE == 1) { o[0] = __fadd_rn(o[0], l.x); o[1] = __fadd_rn(o[1], l.y); o[2] = __fadd_rn(o[2], l.z); o[3] = __fadd_rn(o[3], l.w); }
-                else { o[0] = combine(op, o[0], l.x); o[1] = combine(op, o[1], l.y); o[2] = combine(op, o[2], l.z); o[3] = combine(op, o[3], l.w); }
+                o[0] = __fadd_rn(o[0], l.x); o[1] = __fadd_rn(o[1], l.y); o[2] = __fadd_rn(o[2], l.z); o[3] = __fadd_rn(o[3], l.w);
             }
             *reinterpret_cast<float4*>(row + at) = make_float4(o[0], o[1], o[2], o[3]);
         }
-        sign >>= (N & 31);
+        sign >>= N;
+        sel += N == 8 ? 0x0001u : 0x0022u;
+    }
+}
+
+// Reduce operation of the hop: 0 = sum, 1 = max, 2 = min, 3 = average (a sum on every hop); of two operands that
+// compare equal Max and Min keep the decoded one.
+__device__ __forceinline__ float combine(uint32_t op, float a, float b)
+{
+    return op == 1u ? ((a < b) ? b : a) : op == 2u ? ((b < a) ? b : a) : __fadd_rn(a, b);
+}
+
+// Where a tile's blob is, as known from the index alone.
+struct BlobRef {
+    const uint32_t* ptr;    // nullptr: no blob (tile beyond the stream, or a stream that does not parse)
+    uint32_t words;
+    bool staged;            // a bulk copy of its 16-byte-aligned cover is on its way
+};
+
+// One round of a tile (blocks 32 rd + lane) by the general route: any code length, integer arithmetic, any reduce
+// operation.  blob: the tile's words (shared or global memory); pay_off: payload words of the rounds before; code:
+// the code in front of the round; loc_stage: the stage with the operand's round, or nullptr.  Leaves the values in
+// `stage`.  Compact rather than fast: the rounds that come here are rare.
+__device__ __noinline__ void decode_round_general(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t* pay_off_io, int32_t* code_io,
+                                                  float s, float* stage, int lane, const float* loc_stage, uint32_t op)
+{
+    const uint32_t bi = 32u * rd + (uint32_t)lane;
+    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
+    const uint32_t nw = L ? L + 1u : 0u;
+    const uint32_t incl = warp_incl_scan(nw, lane);
+    const uint32_t* pay = blob + 1 + padw + *pay_off_io + (incl - nw);
+    *pay_off_io += __shfl_sync(kFull, incl, 31);
+    const uint32_t sign = L ? pay[0] : 0u;
+    uint32_t w[32];
+    int32_t total = 0;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+        w[k] = (uint32_t)k < L ? pay[1 + k] : 0u;
+        total += (__popc(w[k]) - 2 * __popc(w[k] & sign)) << k;
+    }
+    int32_t inc = total;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int32_t v = __shfl_up_sync(kFull, inc, d);
+        if (lane >= d) inc += v;
+    }
+    bit_transpose<32>(w);
+    int32_t run = *code_io + inc - total;
+    *code_io += __shfl_sync(kFull, inc, 31);
+    char* row = reinterpret_cast<char*>(stage) + 128 * lane;
+    const char* loc = reinterpret_cast<const char*>(loc_stage) + 128 * lane;
+    const uint32_t sw = ((uint32_t)lane & 7u) << 4;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        run += ((sign >> j) & 1u) ? -(int32_t)w[j] : (int32_t)w[j];
+        float v = __fmul_rn(__int2float_rn(run), s);
+        const uint32_t at = ((16u * (uint32_t)(j >> 2)) ^ sw) + 4u * (j & 3);
+        if (loc_stage) v = combine(op, v, *reinterpret_cast<const float*>(loc + at));
+        *reinterpret_cast<float*>(row + at) = v;
     }
 }
 
@@ -1379,13 +1421,6 @@ struct alignas(1024) DecWarpShared {
     alignas(8) unsigned long long bar[2];
 };
 static_assert(sizeof(DecWarpShared) == 17 * 1024, "a warp's share of the shared memory");
-
-// Where a tile's blob is, as known from the index alone.
-struct BlobRef {
-    const uint32_t* ptr;    // nullptr: no blob (tile beyond the stream, or a stream that does not parse)
-    uint32_t words;
-    bool staged;            // a bulk copy of its 16-byte-aligned cover is on its way
-};
 
 // Tiled tensor store of a stage to rows [row0, row0 + 32) of the array behind `map` (one thread).
 __device__ __forceinline__ void tensor_store_round(const CUtensorMap* map, uint32_t row0, const float* stage)
@@ -1405,15 +1440,19 @@ __device__ __noinline__ void store_round_ragged(float* __restrict__ y, const flo
     }
 }
 
-// One round of a tile: blocks 32 rd + lane.  blob: the tile's words (shared or global memory); pay_off: payload words
-// of the rounds before; code: the code in front of the round.  Leaves the values in the stage.
-// MODE, loc_stage, op: see expand_block (loc_stage: the stage that holds the operand's round; may be `stage` itself).
-template <bool F32, int MODE>
+// One round of a tile whose codes are exact in fp32: blocks 32 rd + lane.  Arguments as for decode_round_general;
+// MODE as for expand_block.  The lanes of a warp mostly share one width class; a round with a code length above 16
+// takes the general route.
+template <int MODE>
 __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t& pay_off, int32_t& code, float s,
-                                             float* stage, int lane, const float* loc_stage = nullptr, uint32_t op = 0)
+                                             float* stage, int lane, const float* loc_stage = nullptr)
 {
     const uint32_t bi = 32u * rd + (uint32_t)lane;
     const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
+    if (__any_sync(kFull, L > 16u)) {
+        decode_round_general(blob, padw, nb, rd, &pay_off, &code, s, stage, lane, loc_stage, 0u);
+        return;
+    }
     const uint32_t nw = L ? L + 1u : 0u;
     const uint32_t incl = warp_incl_scan(nw, lane);
     const uint32_t* pay = blob + 1 + padw + pay_off + (incl - nw);
@@ -1422,11 +1461,10 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
     const char* loc = reinterpret_cast<const char*>(loc_stage) + 128 * lane;
     const uint32_t sw = ((uint32_t)lane & 7u) << 4;
     // The block's sum of deltas first, so that the scan over the lanes gives the code in front of every block before
-    // any element is expanded.  The lanes of a warp mostly share one width class.
+    // any element is expanded.
     uint32_t sign;
     int32_t total;
-    const unsigned wide = __ballot_sync(kFull, L > 8u), wider = __ballot_sync(kFull, L > 16u);
-    if (!wide) {
+    if (!__any_sync(kFull, L > 8u)) {
         uint32_t w[8];
         total = load_planes<8>(pay, L, sign, w);
         int32_t inc = total;
@@ -1436,9 +1474,9 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
             if (lane >= d) inc += v;
         }
         bit_transpose<8>(w);
-        expand_block<8, F32, MODE>(w, sign, code + inc - total, s, row, sw, loc, op);
+        expand_block<8, MODE>(w, sign, code + inc - total, s, row, sw, loc);
         code += __shfl_sync(kFull, inc, 31);
-    } else if (!wider) {
+    } else {
         uint32_t w[16];
         total = load_planes<16>(pay, L, sign, w);
         int32_t inc = total;
@@ -1448,19 +1486,7 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
             if (lane >= d) inc += v;
         }
         bit_transpose<16>(w);
-        expand_block<16, F32, MODE>(w, sign, code + inc - total, s, row, sw, loc, op);
-        code += __shfl_sync(kFull, inc, 31);
-    } else {
-        uint32_t w[32];
-        total = load_planes<32>(pay, L, sign, w);
-        int32_t inc = total;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int32_t v = __shfl_up_sync(kFull, inc, d);
-            if (lane >= d) inc += v;
-        }
-        bit_transpose<32>(w);
-        expand_block<32, false, MODE>(w, sign, code + inc - total, s, row, sw, loc, op);
+        expand_block<16, MODE>(w, sign, code + inc - total, s, row, sw, loc);
         code += __shfl_sync(kFull, inc, 31);
     }
 }
@@ -1564,8 +1590,8 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                     float* stage = sh.out[so];
-                    if (mode == 1) decode_round<true, 0>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
-                    else decode_round<false, 0>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
+                    if (mode == 1) decode_round<0>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
+                    else decode_round_general(blob, padw, nb, rd, &pay_off, &code, hc.s, stage, lane, nullptr, 0u);
                     __syncwarp();   // the stage's rows, written by all lanes, are visible
                     const uint32_t e0 = rd * (uint32_t)kRound;
                     if (mapped && e0 + (uint32_t)kRound <= len) {
@@ -1593,16 +1619,30 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
 // a round of the compressor: into a buffer, off to the round's slot by a bulk store.  The place kernel finishes the
 // stream.  An uncompressed copy of the result, when asked for, leaves the stage by a tensor store.
 
+// Out-of-line copies for the hop, whose kernel holds a decoder and an encoder: inlined, the compiler multiplied their
+// code along the kernel's branches until instruction fetch bounded it (four times the size, 15 % slower).
+template <int MODE>
+__device__ __noinline__ void decode_round_call(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t* pay_off, int32_t* code, float s,
+                                               float* stage, int lane, const float* loc_stage)
+{
+    decode_round<MODE>(blob, padw, nb, rd, *pay_off, *code, s, stage, lane, loc_stage);
+}
+__device__ __noinline__ int encode_round_call(const char* row, uint32_t sw, float xprev, float r, bool active, uint32_t* buf, EncodeCarry* cy, int lane,
+                                              uint32_t* status)
+{
+    // laid out like a tile's blob whose word 0 sits in front of the buffer: code-length bytes at words 1.., payload at word 9
+    return encode_round(row, sw, xprev, r, active, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, *cy, lane, *status);
+}
+
 __device__ __forceinline__ uint32_t cj_begin_of(const JobBatch& jb, int j) { return jb.job[j].tile_begin; }
 
 struct alignas(1024) HopWarpShared {
-    float loc[2][kRound];                  // the operand's rounds; each on a 1024-byte boundary
-    float ys[kRound];                      // decoded (+) operand
-    alignas(16) uint32_t blob[2][kDecBlobWords];
-    alignas(16) uint32_t out[2][kRoundBufWords];
-    alignas(8) unsigned long long bar_loc[2], bar_blob[2];
+    float loc[2][kRound];                  // the operand's rounds, replaced in place by the combined values; 1024-byte boundaries
+    alignas(16) uint32_t blob[kDecBlobWords];
+    alignas(16) uint32_t out[kRoundBufWords];
+    alignas(8) unsigned long long bar_loc[2], bar_blob;
 };
-static_assert(sizeof(HopWarpShared) == 25 * 1024, "a warp's share of the shared memory");
+static_assert(sizeof(HopWarpShared) == 15 * 1024, "a warp's share of the shared memory");
 
 // The owner's copy as the dequantised value float(q(y)) * s: `count` elements of the stage, coalesced.
 __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, const float* stage, uint32_t count, float r, float s, int lane)
@@ -1615,7 +1655,7 @@ __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, cons
     }
 }
 
-__global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps loc_maps,
+__global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps loc_maps,
                                                                      const __grid_constant__ TileMaps raw_maps, Workspace ws)
 {
     pdl_enter();
@@ -1625,11 +1665,11 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
     uint32_t status = 0;
     if (lane == 0) {
         mbar_init(&sh.bar_loc[0], 1); mbar_init(&sh.bar_loc[1], 1);
-        mbar_init(&sh.bar_blob[0], 1); mbar_init(&sh.bar_blob[1], 1);
+        mbar_init(&sh.bar_blob, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    uint32_t lfill0 = 0, lfill1 = 0, bfill0 = 0, bfill1 = 0;   // completed copies per buffer (phase parities)
+    uint32_t lfill0 = 0, lfill1 = 0, bfill = 0;   // completed copies per buffer (phase parities)
     bool lbulk0 = false, lbulk1 = false;
 
     // the job of the tile looked up last, with its streams' headers
@@ -1664,8 +1704,8 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
         br.words = w_end - w_beg;
         return br;
     };
-    // the incoming blob of tile t of the launch; its cover is requested into blob buffer `buf` when it fits
-    auto request_blob = [&](uint32_t t, uint32_t buf) {
+    // the incoming blob of tile t of the launch; its cover is requested into the blob buffer when it fits
+    auto request_blob = [&](uint32_t t) {
         BlobRef br;
         br.ptr = nullptr; br.words = 0; br.staged = false;
         if (t >= jb.total_tiles) return br;
@@ -1679,8 +1719,8 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
         const uintptr_t a_beg = b & ~(uintptr_t)15, a_end = (e + 15) & ~(uintptr_t)15;
         if (a_end - a_beg <= (uintptr_t)(kDecBlobWords * 4) && a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {
             if (lane == 0) {
-                mbar_expect_tx(&sh.bar_blob[buf], (uint32_t)(a_end - a_beg));
-                bulk_load(sh.blob[buf], (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar_blob[buf]);
+                mbar_expect_tx(&sh.bar_blob, (uint32_t)(a_end - a_beg));
+                bulk_load(sh.blob, (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar_blob);
             }
             br.staged = true;
         }
@@ -1714,8 +1754,8 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
 
     const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
     uint32_t t = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
-    uint32_t pb = 0, pl = 0, po = 0;   // blob buffer, operand stage and output buffer in turn
-    BlobRef cur = request_blob(t, 0);
+    uint32_t pl = 0;   // operand stage in turn
+    BlobRef cur = request_blob(t);
     if (t < jb.total_tiles && job_ok && jb.job[cj].n) request_loc(cj, t - cj_begin, 0, 0);
     EncodeCarry cy;
     cy.pay_used = 0; cy.wide = false;
@@ -1737,15 +1777,10 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
         const bool summing = op == 0u || op == 3u, deq = (job.flags & 1u) != 0;
         if (!ok) status |= kStBadStream;
 
-        __syncwarp();   // every lane is done with the other blob buffer
         const uint32_t tn = t + stride < t ? 0xFFFFFFFFu : t + stride;
-        const BlobRef nxt = request_blob(tn, pb ^ 1u);   // moves the job look-up on to the next tile
-        const bool next_has_operand = tn < jb.total_tiles && job_ok && jb.job[cj].n != 0;
-        const int njob = cj;
-        const uint32_t ntile = tn - cj_begin;
         if (cur.staged) {
-            if (!mbar_wait(&sh.bar_blob[pb], (pb ? bfill1 : bfill0) & 1u)) status |= kStTimeout;
-            if (pb) ++bfill1; else ++bfill0;
+            if (!mbar_wait(&sh.bar_blob, bfill & 1u)) status |= kStTimeout;
+            ++bfill;
         }
 
         // what the two blobs say
@@ -1754,7 +1789,7 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
         int mode1 = 0, mode2 = 1;
         if (len) {
             if (cur.ptr) {
-                blob1 = cur.staged ? sh.blob[pb] + ((((uintptr_t)cur.ptr) & 15u) >> 2) : cur.ptr;
+                blob1 = cur.staged ? sh.blob + ((((uintptr_t)cur.ptr) & 15u) >> 2) : cur.ptr;
                 mode1 = describe_blob(blob1, cur.words, nb, lane);
             }
             if (job.in_c2) {
@@ -1769,53 +1804,63 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
         uint32_t pay1 = 0, pay2 = 0;
         int32_t code1 = good ? (int32_t)blob1[0] : 0, code2 = (good && blob2) ? (int32_t)blob2[0] : 0;
         float carry_y = 0.0f;
+        // The next tile's blob goes into the one blob buffer as soon as this tile's last round is decoded; that look-up
+        // moves the job on, so the next tile's facts are kept from there.
+        BlobRef nxt;
+        nxt.ptr = nullptr; nxt.words = 0; nxt.staged = false;
+        bool next_has_operand = false, next_known = false;
+        int njob = 0;
+        uint32_t ntile = 0;
+        auto look_ahead = [&]() {
+            __syncwarp();   // every lane is done with the blob buffer
+            nxt = request_blob(tn);
+            next_has_operand = tn < jb.total_tiles && job_ok && jb.job[cj].n != 0;
+            njob = cj;
+            ntile = tn - cj_begin;
+            next_known = true;
+        };
+        if (rounds == 0 || !good) look_ahead();
         for (uint32_t rd = 0; rd < rounds; ++rd) {
-            __syncwarp();   // every lane is done with the other operand stage
-            if (rd + 1 < rounds) request_loc(jcur, tile, rd + 1, pl ^ 1u);
-            else if (next_has_operand) request_loc(njob, ntile, 0, pl ^ 1u);
-            else { if (pl) lbulk0 = false; else lbulk1 = false; }
-            arrive_loc(pl);
+            // the copy engine is through with what it was handed in the round before: the other operand stage (an
+            // uncompressed copy of the result left from there) and the output buffer
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            __syncwarp();
+            float* loc = sh.loc[pl];
             const uint32_t u = 4u * t + rd;
             if (!good) {
+                if (rd + 1 < rounds) request_loc(jcur, tile, rd + 1, pl ^ 1u);
+                else if (next_has_operand) request_loc(njob, ntile, 0, pl ^ 1u);
+                else { if (pl) lbulk0 = false; else lbulk1 = false; }
+                arrive_loc(pl);
                 if (lane == 0) ws.round_words[u] = 0;
             } else {
-                float* loc = sh.loc[pl];
+                if (rd + 1 < rounds) request_loc(jcur, tile, rd + 1, pl ^ 1u);
+                arrive_loc(pl);
                 if (blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
-                    if (mode2 == 1) decode_round<true, 0>(blob2, padw, nb, rd, pay2, code2, s, loc, lane);
-                    else decode_round<false, 0>(blob2, padw, nb, rd, pay2, code2, s, loc, lane);
+                    if (mode2 == 1) decode_round_call<0>(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr);
+                    else decode_round_general(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr, 0u);
                     __syncwarp();
                 }
-                // the stage and the buffer about to be written were handed to the copy engine one and two rounds ago
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                __syncwarp();
-                if (mode1 == 1) {
-                    if (summing) decode_round<true, 1>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
-                    else decode_round<true, 2>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
-                } else {
-                    if (summing) decode_round<false, 1>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
-                    else decode_round<false, 2>(blob1, padw, nb, rd, pay1, code1, s, sh.ys, lane, loc, op);
+                if (mode1 == 1 && summing) decode_round_call<1>(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc);
+                else decode_round_general(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc, op);
+                if (rd + 1 == rounds) {   // the blob is decoded: the next tile's may come, and its first operand round
+                    look_ahead();
+                    if (next_has_operand) request_loc(njob, ntile, 0, pl ^ 1u);
+                    else { if (pl) lbulk0 = false; else lbulk1 = false; }
                 }
                 __syncwarp();   // the stage's rows, written by all lanes, are visible
-                const float* ys = sh.ys;
+                const float* ys = loc;
                 const char* row = reinterpret_cast<const char*>(ys) + 128 * lane;
                 const uint32_t sw = ((uint32_t)lane & 7u) << 4;
                 const float y0 = ys[0];
                 const float xprev = lane ? read_last_of_row(ys, (uint32_t)lane - 1u) : (rd ? carry_y : y0);
                 carry_y = read_last_of_row(ys, 31);
                 const uint32_t e0 = rd * (uint32_t)kRound;
-                if (job.y) {
-                    const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
-                    if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
-                    else if ((((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
-                        if (lane == 0) tensor_store_round(&raw_maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), ys);
-                    } else store_round_ragged(job.y + start + e0, ys, count, lane);
-                }
                 uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
-                uint32_t* buf = sh.out[po];
+                uint32_t* buf = sh.out;
                 cy.pay_used = 0;
                 const uint32_t bi = 32u * rd + (uint32_t)lane;
-                const int rc = encode_round(row, sw, xprev, r, bi < nb, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, cy, lane,
-                                            status);
+                const int rc = encode_round_call(row, sw, xprev, r, bi < nb, buf, &cy, lane, &status);
                 const uint32_t gslot = (cj_begin_of(jb, jcur) >> 5) + (uint32_t)jcur + (tile >> 5);
                 if (rc == 0) {
                     __syncwarp();   // the buffer's words, written by all lanes, are visible to lane 0's store
@@ -1829,18 +1874,24 @@ __global__ void __launch_bounds__(kCodecThreads, 2) hop_tiles_kernel(const __gri
                         // exact while |y r| < 2^22; larger codes take the general route
                         if (rd == 0) ws.outliers[t] = (int32_t)(__float_as_uint(__fadd_rn(__fmul_rn(y0, r), kRoundMagic)) - kRoundMagicBits);
                     }
-                    po ^= 1u;
                 } else {
                     status |= encode_round_general_staged(ys, xprev, bi < nb, rd, r, slot, ws.round_words + u, ws.outliers + t, ws.group_acc + gslot, lane);
+                }
+                if (job.y) {
+                    const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
+                    if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
+                    else if ((((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
+                        if (lane == 0) tensor_store_round(&raw_maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), ys);
+                    } else store_round_ragged(job.y + start + e0, ys, count, lane);
                 }
             }
             pl ^= 1u;
         }
         if (rounds == 0 && next_has_operand) request_loc(njob, ntile, 0, pl);
         if ((uint32_t)lane >= rounds && lane < kRoundsPerTile) ws.round_words[4u * t + (uint32_t)lane] = 0;   // rounds the tile does not have
+        (void)next_known;
         cur = nxt;
         t = tn;
-        pb ^= 1u;
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (status) atomicOr(ws.status, status);
