@@ -32,6 +32,9 @@
 
 namespace zccl {
 #ifdef ZCCL_TRACE
+#ifndef ZCCL_TRACE_PLACE
+#define ZCCL_TRACE_PLACE 0
+#endif
 __device__ unsigned long long g_trace[32];
 __device__ unsigned long long g_rec[4096 * 8];
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long v; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(v)); return v; }
@@ -1096,10 +1099,10 @@ constexpr int kPlaceThreads = 1024;   // one warp per tile of the group
 __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ GroupTable gt, Workspace ws,
                                                               Params hp, int use_dev_params, int from_stream)
 {
-    pdl_enter();
-    __shared__ uint32_t s_words[32], s_off[32], s_part[kPlaceThreads / 32], s_base, s_ok;
+    // What this kernel reads before it waits for step 1 is older than step 1's launch: job table, the incoming
+    // streams' headers, the resolved bound.
+    __shared__ uint32_t s_words[32], s_part[kPlaceThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
     uint32_t status = 0;
     Params prm = hp;
     if (use_dev_params) prm = *ws.params;
@@ -1114,7 +1117,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         j = lo;
     }
 #ifdef ZCCL_TRACE
-    if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 0] = gtime();
+    if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 0] = gtime();
 #endif
     const Job& job = jb.job[j];
     if (from_stream) {   // a hop: bound and step are the incoming stream's, and the job counts only if its streams agree with it
@@ -1126,6 +1129,11 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         }
         prm.eb_abs = h1.eb_abs; prm.s = h1.s; prm.valid = ok ? 1 : 0;
     }
+    pdl_enter();
+#ifdef ZCCL_TRACE
+    if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 1] = gtime();
+#endif
+    const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
     const uint32_t g = blockIdx.x - gt.begin[j];
     const uint32_t tiles = (j + 1 < jb.count ? jb.job[j + 1].tile_begin : jb.total_tiles) - job.tile_begin;
     const unsigned long long n = job.n;
@@ -1140,77 +1148,55 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         const uint32_t t0 = 32u * g;                               // first tile of the group, within the job
         const uint32_t ntl = tiles - t0 < 32u ? tiles - t0 : 32u;   // tiles of the group
         const uint32_t T0 = job.tile_begin + t0;                   // the same, in the launch's numbering
-        // sizes: thread i < 128 holds round i & 3 of tile i >> 2
-        if (tid < 128) {
-            const uint32_t ti = (uint32_t)tid >> 2;
-            const uint32_t rw = ti < ntl ? ws.round_words[4u * T0 + (uint32_t)tid] : 0u;
-            uint32_t pay = rw + __shfl_xor_sync(kFull, rw, 1);
-            pay += __shfl_xor_sync(kFull, pay, 2);
-            const unsigned long long left = n - (unsigned long long)(t0 + ti) * kTile;
-            const uint32_t len = ti < ntl ? (uint32_t)(left < (unsigned long long)kTile ? left : (unsigned long long)kTile) : 0u;
-            const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2;
-            if ((tid & 3) == 0) s_words[ti] = ti < ntl ? 1u + padw + pay : 0u;
-        }
-        __syncthreads();
-#ifdef ZCCL_TRACE
-        if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 1] = gtime();
-#endif
-        if (warp == 0) {
-            const uint32_t w = s_words[lane];
-            const uint32_t incl = warp_incl_scan(w, lane);
-            s_off[lane] = incl - w;
-        }
-        // the group's place: the groups of the job in front of it are full ones (33 fixed words per tile) with the
-        // payload that step 1 added up per group
-        {
-            const uint32_t gslot0 = (job.tile_begin >> 5) + (uint32_t)j;
-            unsigned long long part = 0;
-            for (uint32_t k = (uint32_t)tid; k < g; k += kPlaceThreads) part += ws.group_acc[gslot0 + k];
-#pragma unroll
-            for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(kFull, part, d);
-            if (lane == 0) s_part[warp] = (uint32_t)part;
-        }
-        __syncthreads();
-        if (tid == 0) {
-            uint32_t sum = 0;
-            for (int w = 0; w < kPlaceThreads / 32; ++w) sum += s_part[w];
-            s_base = sum + g * 32u * (1u + (uint32_t)kLWords);
-            s_ok = 1u;
-        }
-        __syncthreads();
-        // every warp fetches its tile's pieces (up to eight words per lane and round); after the look-back, whose few
-        // loads would otherwise queue up behind these
+        // One round trip: every warp asks for all that belongs to its tile at once (round sizes, first value, its lane's
+        // code-length word, eight payload words per lane and round whatever the sizes turn out to be) and for its share of
+        // the sums of the groups in front.
         const uint32_t tl = (uint32_t)warp;
         const bool mine = tl < ntl;
-        const uint32_t T = T0 + tl;
+        const uint32_t T = T0 + (mine ? tl : 0u);
         const uint32_t* __restrict__ slot = ws.slots + (size_t)(4u * T) * kRoundSlotWords;
-        uint32_t nqs[kRoundsPerTile] = {0, 0, 0, 0};
+        const uint4 nq4 = *reinterpret_cast<const uint4*>(ws.round_words + 4u * T);
+        const uint32_t lword = slot[(size_t)(lane >> 3) * kRoundSlotWords + (lane & 7)];   // code-length word `lane` of the tile
+        const uint32_t first = (uint32_t)ws.outliers[T];
         uint32_t v[kRoundsPerTile][8];
-        uint32_t lword = 0, first = 0;
-        if (mine) {
-            const uint4 nq4 = *reinterpret_cast<const uint4*>(ws.round_words + 4u * T);
-            nqs[0] = nq4.x; nqs[1] = nq4.y; nqs[2] = nq4.z; nqs[3] = nq4.w;
-            lword = slot[(size_t)(lane >> 3) * kRoundSlotWords + (lane & 7)];   // code-length word `lane` of the tile
-            if (lane == 0) first = (uint32_t)ws.outliers[T];
 #pragma unroll
-            for (int q = 0; q < kRoundsPerTile; ++q) {
-                const uint32_t* __restrict__ src = slot + (size_t)q * kRoundSlotWords + 8;
+        for (int q = 0; q < kRoundsPerTile; ++q) {
+            const uint32_t* __restrict__ src = slot + (size_t)q * kRoundSlotWords + 8;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const uint32_t i = (uint32_t)lane + 32u * k;
-                    v[q][k] = i < nqs[q] ? src[i] : 0u;
-                }
+            for (int k = 0; k < 8; ++k) v[q][k] = src[lane + 32 * k];
+        }
+        unsigned long long part = 0;
+        {
+            const uint32_t gslot0 = (job.tile_begin >> 5) + (uint32_t)j;
+            for (uint32_t k = (uint32_t)tid; k < g; k += kPlaceThreads) part += ws.group_acc[gslot0 + k];
+        }
+        const uint32_t nqs[kRoundsPerTile] = {nq4.x, nq4.y, nq4.z, nq4.w};
+        {
+            const unsigned long long left = n - (unsigned long long)(t0 + (mine ? tl : 0u)) * kTile;
+            const uint32_t len = (uint32_t)(left < (unsigned long long)kTile ? left : (unsigned long long)kTile);
+            const uint32_t padw = (((len + kBlock - 1) / kBlock) + 3) >> 2;
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) part += __shfl_xor_sync(kFull, part, d);
+            if (lane == 0) {
+                s_words[warp] = mine ? 1u + padw + nq4.x + nq4.y + nq4.z + nq4.w : 0u;
+                s_part[warp] = (uint32_t)part;
             }
         }
+        __syncthreads();
+        // the group's place: the groups of the job in front of it are full ones (33 fixed words per tile) with the
+        // payload that step 1 added up per group; the tile's place inside the group: the tiles in front of it
 #ifdef ZCCL_TRACE
-        if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 3] = gtime();
+        if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 3] = gtime();
 #endif
-        const uint32_t base = s_base;
-        const bool placed = s_ok != 0;
+        const uint32_t wl = s_words[lane];
+        const uint32_t incl = warp_incl_scan(wl, lane);
+        const uint32_t my_off = __shfl_sync(kFull, incl - wl, warp);
+        const uint32_t base = __reduce_add_sync(kFull, s_part[lane]) + g * 32u * (1u + (uint32_t)kLWords);
+        const bool placed = true;
         if (mine) {
             const uint32_t tile = t0 + tl;
             const uint32_t words = s_words[tl];
-            const unsigned long long word0 = (unsigned long long)kHeaderWords + nT + base + s_off[tl];
+            const unsigned long long word0 = (unsigned long long)kHeaderWords + nT + base + my_off;
             const bool fits = (word0 + words) * 4ull <= job.out_cap;
             if (!fits) status |= kStCapacity;
             if (fits && placed) {
@@ -1235,7 +1221,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
                     }
                     d += nq;
                 }
-                if (lane == 0) out[kHeaderWords + tile] = base + s_off[tl] + words;
+                if (lane == 0) out[kHeaderWords + tile] = base + my_off + words;
             }
             if (lane == 0 && tile == nT - 1) *job.out_bytes = (size_t)((word0 + words) * 4ull);
             if (tile == 0) write_header(out, lane, n, prm.eb_abs, prm.s, nT);
@@ -1243,7 +1229,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
     }
 #ifdef ZCCL_TRACE
     __syncthreads();
-    if (tid == 0 && blockIdx.x < 512) g_rec[8 * blockIdx.x + 4] = gtime();
+    if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 4] = gtime();
 #endif
     if (status) atomicOr(ws.status, status);
     // the last CTA to get here re-arms the workspace: group sums back to zero, launch counter on
@@ -1634,6 +1620,25 @@ __device__ __noinline__ int encode_round_call(const char* row, uint32_t sw, floa
     return encode_round(row, sw, xprev, r, active, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, *cy, lane, *status);
 }
 
+// Advances (pay_off, code) over round e of a tile without expanding it: the blocks' sizes from their code lengths,
+// their sums of deltas from population counts of their planes.  Lets a warp start in the middle of a tile.
+__device__ __noinline__ void skip_round(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t e, uint32_t* pay_off, int32_t* code, int lane)
+{
+    const uint32_t bi = 32u * e + (uint32_t)lane;
+    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
+    const uint32_t nw = L ? L + 1u : 0u;
+    const uint32_t incl = warp_incl_scan(nw, lane);
+    const uint32_t* pay = blob + 1 + padw + *pay_off + (incl - nw);
+    const uint32_t sign = L ? pay[0] : 0u;
+    int32_t total = 0;
+    for (uint32_t k = 0; k < L; ++k) {
+        const uint32_t w = pay[1 + k];
+        total += (__popc(w) - 2 * __popc(w & sign)) << k;
+    }
+    *pay_off += __shfl_sync(kFull, incl, 31);
+    *code += (int32_t)__reduce_add_sync(kFull, total);
+}
+
 __device__ __forceinline__ uint32_t cj_begin_of(const JobBatch& jb, int j) { return jb.job[j].tile_begin; }
 
 struct alignas(1024) HopWarpShared {
@@ -1656,9 +1661,17 @@ __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, cons
 }
 
 __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps loc_maps,
-                                                                     const __grid_constant__ TileMaps raw_maps, Workspace ws)
+                                                                     const __grid_constant__ TileMaps raw_maps, Workspace ws, uint32_t split_shift)
 {
+    // split_shift 0: a warp's unit of work is a tile; 1: two rounds; 2: a round (small launches: more warps at work, and
+    // none of them walks four rounds in a row)
+#ifdef ZCCL_TRACE
+    unsigned long long tr0 = gtime(), tr_cnt = 0, tr_blob = 0, tr_dec = 0, tr_enc = 0;
+#endif
     pdl_enter();
+#ifdef ZCCL_TRACE
+    const unsigned long long tr1 = gtime();
+#endif
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     HopWarpShared& sh = reinterpret_cast<HopWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
@@ -1753,14 +1766,16 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
     };
 
     const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
-    uint32_t t = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
+    const uint32_t total_units = jb.total_tiles << split_shift, rd_mask = (1u << split_shift) - 1u;
+    uint32_t un = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;   // unit: tile un >> split_shift, from round un & rd_mask on
     uint32_t pl = 0;   // operand stage in turn
-    BlobRef cur = request_blob(t);
-    if (t < jb.total_tiles && job_ok && jb.job[cj].n) request_loc(cj, t - cj_begin, 0, 0);
+    BlobRef cur = request_blob(un < total_units ? un >> split_shift : 0xFFFFFFFFu);
+    if (un < total_units && job_ok && jb.job[cj].n) request_loc(cj, (un >> split_shift) - cj_begin, (un & rd_mask) * (4u >> split_shift), 0);
     EncodeCarry cy;
     cy.pay_used = 0; cy.wide = false;
 
-    while (t < jb.total_tiles) {
+    while (un < total_units) {
+        const uint32_t t = un >> split_shift, rd_first = (un & rd_mask) * (4u >> split_shift);
         // the current tile's facts, before the look-up of the next tile moves on to another job
         enter_job(t);
         const int jcur = cj;
@@ -1777,12 +1792,18 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
         const bool summing = op == 0u || op == 3u, deq = (job.flags & 1u) != 0;
         if (!ok) status |= kStBadStream;
 
-        const uint32_t tn = t + stride < t ? 0xFFFFFFFFu : t + stride;
+        const uint32_t unn = (un + stride < un || un + stride >= total_units) ? 0xFFFFFFFFu : un + stride;
+        const uint32_t tn = unn == 0xFFFFFFFFu ? 0xFFFFFFFFu : unn >> split_shift, nrd = (unn & rd_mask) * (4u >> split_shift);
+        const uint32_t rd_end = rd_first + (4u >> split_shift);
+        const uint32_t rd_stop = rd_first >= rounds ? rd_first : (rd_end < rounds ? rd_end : rounds);   // rounds [rd_first, rd_stop)
         if (cur.staged) {
             if (!mbar_wait(&sh.bar_blob, bfill & 1u)) status |= kStTimeout;
             ++bfill;
         }
 
+#ifdef ZCCL_TRACE
+        if (tr_cnt == 0) tr_blob = gtime();
+#endif
         // what the two blobs say
         const uint32_t* blob1 = nullptr;
         const uint32_t* blob2 = nullptr;
@@ -1819,8 +1840,18 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
             ntile = tn - cj_begin;
             next_known = true;
         };
-        if (rounds == 0 || !good) look_ahead();
-        for (uint32_t rd = 0; rd < rounds; ++rd) {
+        if (rd_first >= rd_stop || !good) look_ahead();
+        if (good && rd_first != 0 && rd_first < rd_stop) {
+            // a unit that starts inside its tile: sizes and codes of the rounds in front, and the value in front of it
+            for (uint32_t e = 0; e < rd_first; ++e) {
+                skip_round(blob1, padw, nb, e, &pay1, &code1, lane);
+                if (blob2) skip_round(blob2, padw, nb, e, &pay2, &code2, lane);
+            }
+            const float xa = __fmul_rn(__int2float_rn(code1), s);
+            const float xb = blob2 ? __fmul_rn(__int2float_rn(code2), s) : __ldg(job.x + start + rd_first * (uint32_t)kRound - 1u);
+            carry_y = combine(op, xa, xb);
+        }
+        for (uint32_t rd = rd_first; rd < rd_stop; ++rd) {
             // the copy engine is through with what it was handed in the round before: the other operand stage (an
             // uncompressed copy of the result left from there) and the output buffer
             if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -1828,13 +1859,13 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
             float* loc = sh.loc[pl];
             const uint32_t u = 4u * t + rd;
             if (!good) {
-                if (rd + 1 < rounds) request_loc(jcur, tile, rd + 1, pl ^ 1u);
-                else if (next_has_operand) request_loc(njob, ntile, 0, pl ^ 1u);
+                if (rd + 1 < rd_stop) request_loc(jcur, tile, rd + 1, pl ^ 1u);
+                else if (next_has_operand) request_loc(njob, ntile, nrd, pl ^ 1u);
                 else { if (pl) lbulk0 = false; else lbulk1 = false; }
                 arrive_loc(pl);
                 if (lane == 0) ws.round_words[u] = 0;
             } else {
-                if (rd + 1 < rounds) request_loc(jcur, tile, rd + 1, pl ^ 1u);
+                if (rd + 1 < rd_stop) request_loc(jcur, tile, rd + 1, pl ^ 1u);
                 arrive_loc(pl);
                 if (blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
                     if (mode2 == 1) decode_round_call<0>(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr);
@@ -1843,17 +1874,20 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
                 }
                 if (mode1 == 1 && summing) decode_round_call<1>(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc);
                 else decode_round_general(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc, op);
-                if (rd + 1 == rounds) {   // the blob is decoded: the next tile's may come, and its first operand round
+                if (rd + 1 == rd_stop) {   // the blob is decoded: the next unit's may come, and its first operand round
                     look_ahead();
-                    if (next_has_operand) request_loc(njob, ntile, 0, pl ^ 1u);
+                    if (next_has_operand) request_loc(njob, ntile, nrd, pl ^ 1u);
                     else { if (pl) lbulk0 = false; else lbulk1 = false; }
                 }
                 __syncwarp();   // the stage's rows, written by all lanes, are visible
+#ifdef ZCCL_TRACE
+                if (tr_cnt == 0) tr_dec = gtime();
+#endif
                 const float* ys = loc;
                 const char* row = reinterpret_cast<const char*>(ys) + 128 * lane;
                 const uint32_t sw = ((uint32_t)lane & 7u) << 4;
                 const float y0 = ys[0];
-                const float xprev = lane ? read_last_of_row(ys, (uint32_t)lane - 1u) : (rd ? carry_y : y0);
+                const float xprev = lane ? read_last_of_row(ys, (uint32_t)lane - 1u) : (rd ? carry_y : y0);   // carry_y: the value in front of the round
                 carry_y = read_last_of_row(ys, 31);
                 const uint32_t e0 = rd * (uint32_t)kRound;
                 uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
@@ -1877,6 +1911,10 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
                 } else {
                     status |= encode_round_general_staged(ys, xprev, bi < nb, rd, r, slot, ws.round_words + u, ws.outliers + t, ws.group_acc + gslot, lane);
                 }
+#ifdef ZCCL_TRACE
+                if (tr_cnt == 0) tr_enc = gtime();
+                ++tr_cnt;
+#endif
                 if (job.y) {
                     const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
                     if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
@@ -1887,13 +1925,17 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
             }
             pl ^= 1u;
         }
-        if (rounds == 0 && next_has_operand) request_loc(njob, ntile, 0, pl);
-        if ((uint32_t)lane >= rounds && lane < kRoundsPerTile) ws.round_words[4u * t + (uint32_t)lane] = 0;   // rounds the tile does not have
+        if (rd_first >= rd_stop && next_has_operand) request_loc(njob, ntile, nrd, pl);
+        // rounds the tile does not have
+        if ((uint32_t)lane >= rd_first && (uint32_t)lane < rd_end && (uint32_t)lane >= rounds) ws.round_words[4u * t + (uint32_t)lane] = 0;
         (void)next_known;
         cur = nxt;
-        t = tn;
+        un = unn;
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+#ifdef ZCCL_TRACE
+    if (lane == 0) { unsigned long long* rec = g_rec + 8 * (blockIdx.x * kCodecWarps + warp); if (blockIdx.x * kCodecWarps + warp < 4096) { rec[0] = tr0; rec[1] = tr1; rec[2] = tr_blob; rec[3] = tr_dec; rec[4] = tr_enc; rec[5] = gtime(); rec[6] = tr_cnt; } }
+#endif
     if (status) atomicOr(ws.status, status);
 }
 
@@ -2004,9 +2046,13 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     }
     GroupTable gt;
     const uint32_t groups = group_table(jb, gt);
-    const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     const unsigned long long cap = (unsigned long long)sm_count * d->hop_ctas;
-    e = launch_k(hop_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kHopSmemBytes, st, jb, loc_maps, raw_maps, ws);
+    // launches that would leave warps idle with a tile per warp (a ring's hops) hand out rounds instead
+    const unsigned long long warps = cap * kCodecWarps;
+    const uint32_t split_shift = 4ull * jb.total_tiles <= warps ? 2u : 2ull * jb.total_tiles <= warps ? 1u : 0u;
+    const unsigned long long want = ((((unsigned long long)jb.total_tiles) << split_shift) + kCodecWarps - 1) / kCodecWarps;
+    e = launch_k(hop_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kHopSmemBytes, st, jb, loc_maps, raw_maps, ws,
+                 split_shift);
     if (e != cudaSuccess) return e;
     return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
 }
