@@ -1,29 +1,43 @@
 // fZ-light codec kernels for sm_100a: encoder, decoder and the fused decode + reduce + encode hop.
 //
-// Work decomposition: ONE LANE OWNS ONE 32-ELEMENT BLOCK.  A warp works on a 4096-element tile of its own in four
-// rounds of 32 blocks (1024 elements); lane l of a round holds the 32 consecutive elements of block l in registers.
-// Everything the format asks of a block then happens inside one thread, with no shuffle, vote or barrier:
+// Work decomposition: ONE LANE OWNS ONE 32-ELEMENT BLOCK.  A warp works on a round of 32 blocks (1024 elements,
+// a quarter of a tile); lane l holds the 32 consecutive elements of block l in registers.  Everything the format
+// asks of a block then happens inside one thread, with no shuffle, vote or barrier:
 //   * quantise and 1-D Lorenzo delta: fp32 on the FMA pipe (t + 1.5 * 2^23 rounds to nearest even, deltas of two
 //     such values are exact, |delta| + 2^23 has the magnitude in its mantissa);
 //   * code length: OR of the 32 magnitudes, one count-leading-zeros;
-//   * bit planes: the magnitudes are packed four (code lengths up to 8), two (up to 16) or one to a word and an
-//     in-register bit-matrix transpose (3, 4 or 5 stages of shift + bit-select pairs) turns them into plane words;
+//   * bit planes: the magnitudes are packed four (code lengths up to 8), two (up to 16) or one to a word by byte
+//     permutes and an in-register bit-matrix transpose (3, 4 or 5 stages of shift + bit-select pairs) turns them
+//     into plane words; the decoder runs the same transpose backwards and gets the block's delta sum from
+//     population counts of the planes;
 //   * sign word: one funnel shift per element.
-// A warp needs its neighbours only for the prefix sum of the blocks' sizes (one shuffle scan per round) and, when it
-// decodes, of the blocks' delta sums.  Warps never wait for each other inside a CTA: there is no __syncthreads in
-// the tile loops.
+// A warp needs its neighbours only for the prefix sum of the blocks' sizes and, when it decodes, of the blocks'
+// delta sums (one shuffle scan per round each).  Warps never wait for each other: there is no __syncthreads and no
+// inter-CTA wait in the round loops.  The loops over a block's elements are rolled on purpose: the unrolled forms
+// were bound by instruction fetch.
 //
 // Memory.  A lane wants 128 consecutive bytes per block while global accesses must be contiguous across the warp,
-// so rounds go through shared memory: the warp copies 4 KiB with 16-byte asynchronous copies (cp.async, no
-// registers, one round ahead) into a stage whose 16-byte chunks are XOR-swizzled by the row number, so that the
-// copy, the lanes' 128-bit row reads and (decoder) the row writes are all free of bank conflicts.  A tile's blob is
-// assembled in the warp's shared memory and moved to the stream once its position is known.
+// so rounds go through shared memory.  The array is described to the copy engine as rows of 32 floats (one tensor
+// map per chunk-operation, built on the host); one tiled tensor copy brings a round's 32 rows into a 4 KiB stage
+// in the 128-byte swizzle (16-byte chunk c of row t at c ^ (t & 7)), one round ahead, completion on an mbarrier;
+// the lanes' 128-bit row reads and (decoder) row writes are free of bank conflicts; decoded rounds leave by a
+// tensor store.  Ragged or misaligned rounds take plain loads and stores into the same layout.  Compressed bytes
+// move with untiled bulk copies.
 //
-// Placement.  Tiles are handed out in order by a device-wide counter, so every tile before a given one is already
-// owned by a running warp.  A warp publishes its tile's size as soon as it is known and finds its position by a
-// decoupled look-back over the 8-byte states of the tiles in front of it (32 at a time, one per lane), stopping at
-// the first one that carries an inclusive prefix; states are validated by a launch counter instead of being cleared.
-// Every wait is bounded and reports through the status word instead of hanging.
+// Compression takes two launches and no waits:
+//   1. encode_rounds_kernel: rounds are dealt round-robin to the warps of the grid; each is encoded into a fixed
+//      slot of the workspace (code-length bytes, then the payload), its payload size recorded, and added to the
+//      sum of its group of 32 tiles;
+//   2. place_kernel: one CTA per group turns the group sums in front of it and its own rounds' sizes into stream
+//      positions, writes index entries, outliers and code lengths and moves the payloads from the slots.
+// The fused hop (hop_tiles_kernel) is the same first step with a decoder in front: the incoming round is decoded
+// in place onto the stage that holds the local operand, reduced, optionally stored, and re-encoded from the stage.
+// The slots cost a write and a read of the compressed bytes, mostly absorbed by L2; in exchange no warp ever waits
+// for another, so nothing depends on which CTAs are resident together.
+//
+// A single-pass encoder (enc_kernel: a warp per tile, positions by a two-level decoupled look-back over per-tile and
+// per-group states, every wait bounded and reported through the status word) remains for contexts without slots:
+// the allocation-free entry point.
 #include "zccl_device.cuh"
 
 #include <cuda.h>
@@ -31,21 +45,6 @@
 #include <mutex>
 
 namespace zccl {
-#ifdef ZCCL_TRACE
-#ifndef ZCCL_TRACE_PLACE
-#define ZCCL_TRACE_PLACE 0
-#endif
-__device__ unsigned long long g_trace[32];
-__device__ unsigned long long g_rec[4096 * 8];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long v; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(v)); return v; }
-#define TR_DECL unsigned long long tr_t0 = clock64(), tr_acc[8] = {0,0,0,0,0,0,0,0}; const unsigned long long tr_g0 = gtime()
-#define TR_MARK(k) do { const unsigned long long tr_now = clock64(); tr_acc[k] += tr_now - tr_t0; tr_t0 = tr_now; } while (0)
-#define TR_FLUSH do { if (lane == 0) { for (int k = 0; k < 8; ++k) atomicAdd(&g_trace[k], tr_acc[k]); atomicAdd(&g_trace[8], 1ull); const unsigned long long g1 = gtime(); atomicMin(&g_trace[9], tr_g0); atomicMax(&g_trace[10], tr_g0); atomicMin(&g_trace[11], g1); atomicMax(&g_trace[12], g1); atomicAdd(&g_trace[13], g1 - tr_g0); } } while (0)
-#else
-#define TR_DECL
-#define TR_MARK(k)
-#define TR_FLUSH
-#endif
 namespace {
 
 constexpr int kCodecWarps = 4;                        // warps per CTA, each with tiles of its own
@@ -53,21 +52,8 @@ constexpr int kCodecThreads = 32 * kCodecWarps;
 constexpr int kRound = 32 * kBlock;                   // elements per round: one block per lane
 constexpr int kRoundsPerTile = kTile / kRound;
 constexpr int kLWords = kBlocksPerTile / 4;           // code-length words of a full tile
-constexpr int kBlobHeadWords = 1 + kLWords;           // outlier + code lengths
-constexpr int kMaxPayWords = kBlocksPerTile * 32;     // every block at code length 31: sign word + 31 planes
 
 // ------------------------------------------------------------------------------------------------ small pieces
-
-__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* g)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(g) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
-{
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane)
 {
@@ -360,10 +346,6 @@ __device__ __forceinline__ unsigned long long publish_size_issue(const Workspace
 __device__ __forceinline__ void publish_size_finish(const Workspace& ws, const LookBack& lb, unsigned long long old, uint32_t epoch)
 {
     if (old == ~0ull) return;
-#ifdef ZCCL_TRACE
-    if ((uint32_t)(old >> 40) + 1u == lb.gsize) atomicAdd(&g_trace[16], 1ull);
-    if ((uint32_t)(old >> 40) + 1u > lb.gsize) atomicAdd(&g_trace[20], 1ull);
-#endif
     if ((uint32_t)(old >> 40) + 1u == lb.gsize)
         st_state(ws.group_state + lb.gslot0 + lb.g, pack_state(epoch, 0u, (uint32_t)(old & kAccWordsMask) + lb.total));
 }
@@ -376,9 +358,6 @@ __device__ __forceinline__ void publish_tile_state(const Workspace& ws, uint32_t
 __device__ __forceinline__ void look_back_publish(const Workspace& ws, const LookBack& lb, uint32_t epoch, int lane)
 {
     if (!lb.closes_group || lane != 0 || lb.ticket == ws.skip_publish || !look_back_done(lb)) return;
-#ifdef ZCCL_TRACE
-    atomicAdd(&g_trace[19], 1ull);
-#endif
     st_state(ws.group_state + lb.gslot0 + lb.g, pack_state(epoch, 1u, lb.sum_a + lb.sum_b + lb.total));
 }
 
@@ -508,18 +487,9 @@ __device__ __noinline__ uint32_t flush_tile(const JobBatch* jb, Workspace ws, in
 {
     const Job& jp = jb->job[job];
     uint32_t st = 0;
-#ifdef ZCCL_TRACE
-    const long long c0 = clock64();
-#endif
     const bool placed = look_back_finish(ws, lb, epoch, lane, st);
-#ifdef ZCCL_TRACE
-    const long long c1 = clock64();
-#endif
     emit_tile(jp, lb.ticket - jp.tile_begin, blob, dir ? blob_words - 1u : 0u, dir ? -1 : 1, lb.total, look_back_result(lb), placed, eb_abs,
               s, lane, st);
-#ifdef ZCCL_TRACE
-    if (lane == 0) { atomicAdd(&g_trace[21], (unsigned long long)(c1 - c0)); atomicAdd(&g_trace[22], (unsigned long long)(clock64() - c1)); atomicAdd(&g_trace[23], 1ull); }
-#endif
     return st;
 }
 
@@ -701,14 +671,7 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
         pend.valid = false;
     };
 
-    TR_DECL;
-#ifdef ZCCL_TRACE
-    unsigned long long tr_tile_end[3] = {0, 0, 0}; unsigned tr_ntiles = 0;
-#endif
     uint32_t ticket = take_ticket(ws, lane);
-#ifdef ZCCL_TRACE
-    const unsigned tr_first_ticket = ticket;
-#endif
     TileInfo cur = locate(ticket);
     uint32_t p = 0;   // stage that holds (or will hold) the round about to be encoded
     request(p, cur, 0);
@@ -719,7 +682,6 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
         const uint32_t nb = (len + kBlock - 1) / kBlock;
         const uint32_t padw = (nb + 3) >> 2;
         const uint32_t rounds = (nb + 31) >> 5;
-        const float* __restrict__ xt = cur.xt;
         const uint32_t dir = pend.dir ^ 1u;   // the end of the blob area the waiting tile does not use
         const uint32_t org = dir ? (uint32_t)kEncBlobWords - 1u : 0u;
         const int sgn = dir ? -1 : 1;
@@ -736,7 +698,6 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
         float carry_x = 0.0f;
         int32_t q_first = 0;
         bool general = false;
-        TR_MARK(0);   // tile set-up
         // a tile without elements runs the loop once, for the hand-over to the next tile only
         for (uint32_t rd = 0; rd < (rounds ? rounds : 1u); ++rd) {
             __syncwarp();   // every lane is done with the other stage (it held the round before this one)
@@ -753,9 +714,7 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
             const bool looking = pend.valid && !look_back_done(pend.lb);
             LookBackTrip<1> trip;
             if (looking) look_back_issue(ws, pend.lb, epoch, lane, trip);
-            TR_MARK(1);   // request of the next round
             arrive(p);   // the round has landed
-            TR_MARK(2);   // wait for this round's data
             const float* st = sh.stage[p];
             const char* row = reinterpret_cast<const char*>(st) + 128 * lane;
             const uint32_t sw = ((uint32_t)lane & 7u) << 4;
@@ -776,9 +735,7 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
                 if (rc != 2 || !pend.valid) break;
                 flush_pending();   // no room next to the waiting tile: place that one now, then try again
             }
-            TR_MARK(3);   // encode
             if (looking && pend.valid) (void)look_back_eval(ws, pend.lb, epoch, lane, trip);
-            TR_MARK(4);   // look-back evaluation
             p ^= 1u;
             if (rc != 0) {
                 general = true;
@@ -816,29 +773,15 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
             }
             __syncwarp();   // the blob's words, written by all lanes, are visible to all
             if (lane == 0) publish_size_finish(ws, lb_cur, acc_old, epoch);   // before any wait: others may need the group's size
-            TR_MARK(5);   // publish
-#ifdef ZCCL_TRACE
-            if (tr_ntiles < 3) tr_tile_end[tr_ntiles] = gtime();
-            ++tr_ntiles;
-#endif
             if (pend.valid) flush_pending();
             pend.valid = true; pend.job = cur.job; pend.dir = dir;
             pend.lb = lb_cur;
             if (look_back_done(pend.lb)) look_back_publish(ws, pend.lb, epoch, lane);   // the job's first tile
-#ifdef ZCCL_EXP_NODEFER
-            flush_pending();
-#endif
-            TR_MARK(6);   // flush of the waiting tile
         }
         cur = nxt;
         ticket = next;
     }
     if (pend.valid) flush_pending();
-    TR_MARK(7);   // last flush
-    TR_FLUSH;
-#ifdef ZCCL_TRACE
-    if (lane == 0) { unsigned long long* rec = g_rec + 8 * (blockIdx.x * kCodecWarps + warp); rec[0] = tr_g0; rec[1] = tr_tile_end[0]; rec[2] = tr_tile_end[1]; rec[3] = tr_tile_end[2]; rec[4] = gtime(); rec[5] = tr_ntiles; rec[6] = tr_first_ticket; }
-#endif
     if (status) atomicOr(ws.status, status);
     finish_launch(ws, epoch, tid, ws.ticket, (jb.total_tiles >> 5) + (uint32_t)jb.count + 1u);
 }
@@ -1049,13 +992,8 @@ __global__ void __launch_bounds__(kCodecThreads, 4) encode_rounds_kernel(const _
             cy.pay_used = 0;
             const uint32_t bi = 32u * cur.rd + (uint32_t)lane;
             // laid out like a tile's blob whose word 0 sits in front of the buffer: code-length bytes at words 1.., payload at word 9
-#ifdef ZCCL_EXP_NOCOMPUTE
-            const int rc = 0;
-            cy.pay_used = (uint32_t)(xprev + *reinterpret_cast<const float*>(row + sw)) & 15u;
-#else
             const int rc = encode_round(row, sw, xprev, r, bi < nb, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, cy, lane,
                                         status);
-#endif
             if (rc == 0) {
                 __syncwarp();   // the buffer's words, written by all lanes, are visible to lane 0's store
                 if (lane == 0) {
@@ -1116,9 +1054,6 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         }
         j = lo;
     }
-#ifdef ZCCL_TRACE
-    if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 0] = gtime();
-#endif
     const Job& job = jb.job[j];
     if (from_stream) {   // a hop: bound and step are the incoming stream's, and the job counts only if its streams agree with it
         const StreamInfo h1 = read_header(job.in_c, job.in_cap);
@@ -1130,9 +1065,6 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         prm.eb_abs = h1.eb_abs; prm.s = h1.s; prm.valid = ok ? 1 : 0;
     }
     pdl_enter();
-#ifdef ZCCL_TRACE
-    if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 1] = gtime();
-#endif
     const uint32_t epoch = *reinterpret_cast<volatile uint32_t*>(ws.epoch);
     const uint32_t g = blockIdx.x - gt.begin[j];
     const uint32_t tiles = (j + 1 < jb.count ? jb.job[j + 1].tile_begin : jb.total_tiles) - job.tile_begin;
@@ -1185,9 +1117,6 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         __syncthreads();
         // the group's place: the groups of the job in front of it are full ones (33 fixed words per tile) with the
         // payload that step 1 added up per group; the tile's place inside the group: the tiles in front of it
-#ifdef ZCCL_TRACE
-        if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 3] = gtime();
-#endif
         const uint32_t wl = s_words[lane];
         const uint32_t incl = warp_incl_scan(wl, lane);
         const uint32_t my_off = __shfl_sync(kFull, incl - wl, warp);
@@ -1227,10 +1156,6 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
             if (tile == 0) write_header(out, lane, n, prm.eb_abs, prm.s, nT);
         }
     }
-#ifdef ZCCL_TRACE
-    __syncthreads();
-    if (tid == 0 && blockIdx.x < 512 && ZCCL_TRACE_PLACE) g_rec[8 * blockIdx.x + 4] = gtime();
-#endif
     if (status) atomicOr(ws.status, status);
     // the last CTA to get here re-arms the workspace: group sums back to zero, launch counter on
     __shared__ uint32_t s_last;
@@ -1665,13 +1590,7 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
 {
     // split_shift 0: a warp's unit of work is a tile; 1: two rounds; 2: a round (small launches: more warps at work, and
     // none of them walks four rounds in a row)
-#ifdef ZCCL_TRACE
-    unsigned long long tr0 = gtime(), tr_cnt = 0, tr_blob = 0, tr_dec = 0, tr_enc = 0;
-#endif
     pdl_enter();
-#ifdef ZCCL_TRACE
-    const unsigned long long tr1 = gtime();
-#endif
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     HopWarpShared& sh = reinterpret_cast<HopWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
@@ -1801,9 +1720,6 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
             ++bfill;
         }
 
-#ifdef ZCCL_TRACE
-        if (tr_cnt == 0) tr_blob = gtime();
-#endif
         // what the two blobs say
         const uint32_t* blob1 = nullptr;
         const uint32_t* blob2 = nullptr;
@@ -1880,9 +1796,6 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
                     else { if (pl) lbulk0 = false; else lbulk1 = false; }
                 }
                 __syncwarp();   // the stage's rows, written by all lanes, are visible
-#ifdef ZCCL_TRACE
-                if (tr_cnt == 0) tr_dec = gtime();
-#endif
                 const float* ys = loc;
                 const char* row = reinterpret_cast<const char*>(ys) + 128 * lane;
                 const uint32_t sw = ((uint32_t)lane & 7u) << 4;
@@ -1911,10 +1824,6 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
                 } else {
                     status |= encode_round_general_staged(ys, xprev, bi < nb, rd, r, slot, ws.round_words + u, ws.outliers + t, ws.group_acc + gslot, lane);
                 }
-#ifdef ZCCL_TRACE
-                if (tr_cnt == 0) tr_enc = gtime();
-                ++tr_cnt;
-#endif
                 if (job.y) {
                     const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
                     if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
@@ -1933,9 +1842,6 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
         un = unn;
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-#ifdef ZCCL_TRACE
-    if (lane == 0) { unsigned long long* rec = g_rec + 8 * (blockIdx.x * kCodecWarps + warp); if (blockIdx.x * kCodecWarps + warp < 4096) { rec[0] = tr0; rec[1] = tr1; rec[2] = tr_blob; rec[3] = tr_dec; rec[4] = tr_enc; rec[5] = gtime(); rec[6] = tr_cnt; } }
-#endif
     if (status) atomicOr(ws.status, status);
 }
 
@@ -2071,16 +1977,6 @@ cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_
     return launch_k(decode_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kDecSmemBytes, st, jb, maps, ws);
 }
 
-#ifdef ZCCL_TRACE
-extern "C" int zccl_debug_rec(unsigned long long* out, int n) { return cudaMemcpyFromSymbol(out, g_rec, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -1; }
-extern "C" int zccl_debug_trace(unsigned long long* out16)
-{
-    unsigned long long z[32] = {};
-    z[9] = z[11] = ~0ull;
-    if (cudaMemcpyFromSymbol(out16, g_trace, sizeof(z)) != cudaSuccess) return -1;
-    return cudaMemcpyToSymbol(g_trace, z, sizeof(z)) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool device_params, Params host_params, int sm_count,
                                 cudaStream_t st)
@@ -2106,9 +2002,6 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
     }
     const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     unsigned long long cap = (unsigned long long)sm_count * d->enc_ctas;
-#ifdef ZCCL_TRACE
-    if (const char* ev = getenv("ZCCL_EXP_CTAS")) cap = (unsigned long long)sm_count * atoi(ev);
-#endif
     const unsigned grid = (unsigned)(want < cap ? want : cap);
     return launch_k(enc_kernel, dim3(grid), dim3(kCodecThreads), kEncSmemBytes, st, jb, maps, ws, host_params, device_params ? 1 : 0);
 }
