@@ -229,6 +229,7 @@ __device__ __forceinline__ int encode_round(const char* row, uint32_t sw, float 
     if (__any_sync(kFull, beyond)) return 1;
     if (cy.pay_used + round_total > pay_cap) return 2;
     if (guard >= kGuardSmall && block_tmax(row, sw, r) > 32768.5f) status |= kStPrecision;
+    __syncwarp();   // every lane has read its row for the last time: the blob may lie over the stage
     if (L) {
         uint32_t* dst = blob + ((int)org + sgn * (int)(pay_base + cy.pay_used + (incl - nw)));
         dst[0] = sign;
@@ -1567,12 +1568,12 @@ __device__ __noinline__ void skip_round(const uint32_t* blob, uint32_t padw, uin
 __device__ __forceinline__ uint32_t cj_begin_of(const JobBatch& jb, int j) { return jb.job[j].tile_begin; }
 
 struct alignas(1024) HopWarpShared {
-    float loc[2][kRound];                  // the operand's rounds, replaced in place by the combined values; 1024-byte boundaries
+    float loc[2][kRound];                  // the operand's rounds, replaced in place by the combined values and then by
+                                           // the encoded round; 1024-byte boundaries
     alignas(16) uint32_t blob[kDecBlobWords];
-    alignas(16) uint32_t out[kRoundBufWords];
     alignas(8) unsigned long long bar_loc[2], bar_blob;
 };
-static_assert(sizeof(HopWarpShared) == 15 * 1024, "a warp's share of the shared memory");
+static_assert(sizeof(HopWarpShared) == 13 * 1024, "a warp's share of the shared memory");
 
 // The owner's copy as the dequantised value float(q(y)) * s: `count` elements of the stage, coalesced.
 __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, const float* stage, uint32_t count, float r, float s, int lane)
@@ -1585,7 +1586,7 @@ __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, cons
     }
 }
 
-__global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps loc_maps,
+__global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps loc_maps,
                                                                      const __grid_constant__ TileMaps raw_maps, Workspace ws, uint32_t split_shift)
 {
     // split_shift 0: a warp's unit of work is a tile; 1: two rounds; 2: a round (small launches: more warps at work, and
@@ -1804,7 +1805,18 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
                 carry_y = read_last_of_row(ys, 31);
                 const uint32_t e0 = rd * (uint32_t)kRound;
                 uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
-                uint32_t* buf = sh.out;
+                if (job.y) {   // an uncompressed copy of the result leaves the stage before the encoder writes over it
+                    const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
+                    if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
+                    else if ((((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
+                        if (lane == 0) {
+                            tensor_store_round(&raw_maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), ys);
+                            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        }
+                    } else store_round_ragged(job.y + start + e0, ys, count, lane);
+                    __syncwarp();
+                }
+                uint32_t* buf = reinterpret_cast<uint32_t*>(loc);   // in place: a round's code never outgrows its 4 KiB
                 cy.pay_used = 0;
                 const uint32_t bi = 32u * rd + (uint32_t)lane;
                 const int rc = encode_round_call(row, sw, xprev, r, bi < nb, buf, &cy, lane, &status);
@@ -1823,13 +1835,6 @@ __global__ void __launch_bounds__(kCodecThreads, 3) hop_tiles_kernel(const __gri
                     }
                 } else {
                     status |= encode_round_general_staged(ys, xprev, bi < nb, rd, r, slot, ws.round_words + u, ws.outliers + t, ws.group_acc + gslot, lane);
-                }
-                if (job.y) {
-                    const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
-                    if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
-                    else if ((((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
-                        if (lane == 0) tensor_store_round(&raw_maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), ys);
-                    } else store_round_ragged(job.y + start + e0, ys, count, lane);
                 }
             }
             pl ^= 1u;
