@@ -198,10 +198,12 @@ struct EncodeCarry {
 // sets the lane's code-length byte.  `active`: the block exists (ragged tiles have fewer than 128).  Returns 0 when
 // done; otherwise nothing was stored: 1 when the round is beyond what this path covers (a code length above 16, or
 // codes for which fp32 is not exact) and the whole tile has to take the general route, 2 when the blob would
-// outgrow `pay_cap` payload words.
+// outgrow `pay_cap` payload words.  `mid` is called once, by all lanes, when the rows have been read and the sizes are
+// known, before anything is stored.
+template <class Mid>
 __device__ __forceinline__ int encode_round(const char* row, uint32_t sw, float xprev, float r, bool active, uint32_t block_in_tile,
                                             uint32_t lbytes, uint32_t* __restrict__ blob, uint32_t org, int sgn, uint32_t pay_base,
-                                            uint32_t pay_cap, EncodeCarry& cy, int lane, uint32_t& status)
+                                            uint32_t pay_cap, EncodeCarry& cy, int lane, uint32_t& status, Mid&& mid)
 {
     BlockPack<8> a;
     BlockPack<16> h;
@@ -226,6 +228,7 @@ __device__ __forceinline__ int encode_round(const char* row, uint32_t sw, float 
     const uint32_t nw = L ? L + 1u : 0u;
     const uint32_t incl = warp_incl_scan(nw, lane);
     const uint32_t round_total = __shfl_sync(kFull, incl, 31);
+    mid();   // the caller's business between the two halves (all lanes, once per call)
     if (__any_sync(kFull, beyond)) return 1;
     if (cy.pay_used + round_total > pay_cap) return 2;
     if (guard >= kGuardSmall && block_tmax(row, sw, r) > 32768.5f) status |= kStPrecision;
@@ -732,7 +735,7 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
             for (;;) {
                 const uint32_t held = pend.valid ? pend.lb.total : 0u;
                 rc = encode_round(row, sw, xprev, r, bi < nb, bi, 4u * padw, sh.blob, org, sgn, 1u + padw, room > held ? room - held : 0u, cy,
-                                  lane, status);
+                                  lane, status, [] {});
                 if (rc != 2 || !pend.valid) break;
                 flush_pending();   // no room next to the waiting tile: place that one now, then try again
             }
@@ -797,24 +800,13 @@ __global__ void __launch_bounds__(kCodecThreads, 12 / kCodecWarps) enc_kernel(co
 // Step 2 (place_kernel) turns the slots into the stream.
 
 constexpr int kRoundBufWords = 8 + 32 * 17;   // code-length bytes + payload at code length 16 (longer codes go the general route)
+constexpr int kRoundStages = 3;
 struct alignas(1024) RoundWarpShared {
-    float stage[2][kRound];                   // each on a 1024-byte boundary
-    alignas(16) uint32_t out[2][kRoundBufWords];
-    alignas(8) unsigned long long bar[2];
+    float stage[kRoundStages][kRound];        // each on a 1024-byte boundary; a round is encoded in place and leaves from here
+    alignas(16) float front[kRoundStages][4]; // the four elements in front of each stage's round
+    alignas(8) unsigned long long bar[kRoundStages];
 };
 static_assert(sizeof(RoundWarpShared) == 13 * 1024, "a warp's share of the shared memory");
-
-// A round of the launch as a warp sees it.
-struct RoundInfo {
-    int job;            // -1: beyond the launch's last round
-    uint32_t tile;      // launch number of the round's tile
-    uint32_t jtile;     // the tile's number within its job
-    uint32_t rd;        // the round within the tile
-    uint32_t len;       // elements of the tile (0: nothing to encode)
-    uint32_t gslot;     // slot of the accumulator of the tile's group
-    const float* xt;    // the tile's first element
-    bool mapped;
-};
 
 // General route for one round: any code length, straight from global memory into the round's slot.
 __device__ __noinline__ uint32_t encode_round_general(const float* __restrict__ xt, uint32_t len, uint32_t rd, float r, uint32_t* __restrict__ slot,
@@ -889,6 +881,42 @@ __device__ __noinline__ uint32_t encode_round_general_staged(const float* stage,
     return status;
 }
 
+// What a warp has to know of a tile when it gets to encode its round.
+struct RoundAt {
+    uint32_t t;          // launch number of the tile (beyond the launch: done)
+    uint32_t len;        // elements of the tile (0: nothing to encode)
+    uint32_t gslot;      // slot of the accumulator of the tile's group
+    const float* xt;     // the tile's first element
+};
+
+// A warp's walk over the tiles of a launch, G tiles at a time: where the tile is and how long.
+struct TileCursor {
+    uint32_t t;          // launch number of the tile (beyond the launch: done)
+    int job;
+    uint32_t begin, count;   // the job's first tile and its number of tiles
+    uint32_t len;        // elements of the tile (0: nothing to encode)
+    const float* xt;     // the tile's first element
+    bool aligned;        // the job's array starts on a 16-byte boundary
+};
+
+__device__ __forceinline__ void cursor_settle(TileCursor& c, const JobBatch& jb, bool valid)
+{
+    c.len = 0;
+    if (c.t >= jb.total_tiles) return;
+    if (c.t - c.begin >= c.count) {
+        c.job = find_job(jb, c.t);
+        c.begin = jb.job[c.job].tile_begin;
+        c.count = (c.job + 1 < jb.count ? jb.job[c.job + 1].tile_begin : jb.total_tiles) - c.begin;
+        c.aligned = (((uintptr_t)jb.job[c.job].x) & 15u) == 0;
+    }
+    const Job& q = jb.job[c.job];
+    const unsigned long long start = (unsigned long long)(c.t - c.begin) * kTile;
+    if (q.n && valid) {
+        c.len = (uint32_t)((q.n - start < (unsigned long long)kTile) ? (q.n - start) : kTile);
+        c.xt = q.x + start;
+    }
+}
+
 __global__ void __launch_bounds__(kCodecThreads, 4) encode_rounds_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
                                                                          Workspace ws, Params hp, int use_dev_params)
 {
@@ -900,127 +928,118 @@ __global__ void __launch_bounds__(kCodecThreads, 4) encode_rounds_kernel(const _
     Params prm = hp;
     if (use_dev_params) prm = *ws.params;
     const float r = prm.r;
-    const uint32_t total_rounds = jb.total_tiles * (uint32_t)kRoundsPerTile;
 
     if (lane == 0) {
-        mbar_init(&sh.bar[0], 1);
-        mbar_init(&sh.bar[1], 1);
+#pragma unroll
+        for (int k = 0; k < kRoundStages; ++k) mbar_init(&sh.bar[k], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    uint32_t fills0 = 0, fills1 = 0;      // tensor copies completed per stage (phase parity of its mbarrier)
-    bool bulk0 = false, bulk1 = false;    // the round on its way into each stage comes by a tensor copy
 
-    // the job of the round looked up last: consecutive look-ups mostly stay inside it
-    int cj = -1;
-    uint32_t cj_begin = 0, cj_count = 0;
-    const float* cj_x = nullptr;
-    unsigned long long cj_n = 0;
-    auto locate = [&](uint32_t u) {
-        RoundInfo ri;
-        ri.job = -1; ri.tile = 0; ri.jtile = 0; ri.rd = 0; ri.len = 0; ri.gslot = 0; ri.xt = nullptr; ri.mapped = false;
-        if (u >= total_rounds) return ri;
-        const uint32_t t = u >> 2;
-        if (t - cj_begin >= cj_count) {
-            cj = find_job(jb, t);
-            const Job& q = jb.job[cj];
-            cj_begin = q.tile_begin;
-            cj_count = (cj + 1 < jb.count ? jb.job[cj + 1].tile_begin : jb.total_tiles) - cj_begin;
-            cj_x = q.x;
-            cj_n = q.n;
+    // The CTA's four warps take the four rounds of the same tile, and the CTAs of the launch take the tiles in turn
+    // (no counter: same-address atomics would bound the kernel at about 1.5 ns per round).
+    const uint32_t G = gridDim.x;
+    const uint32_t rd = (uint32_t)warp, e0 = rd * (uint32_t)kRound;
+    const uint32_t sw = ((uint32_t)lane & 7u) << 4;
+
+    // Asks for the warp's round of the tile under cursor `c` into stage `st`.  Every request completes one phase of the
+    // stage's mbarrier, whatever its kind: a tensor copy (with a 16-byte copy of the words in front, whose last one
+    // is the element in front of the round), plain loads, or nothing at all.
+    auto request = [&](const TileCursor& c, uint32_t st) {
+        float* stage = sh.stage[st];
+        if (c.t < jb.total_tiles && e0 < c.len) {
+            if (c.aligned && e0 + (uint32_t)kRound <= c.len) {
+                if (lane == 0) {
+                    mbar_expect_tx(&sh.bar[st], kRound * 4 + (rd ? 16u : 0u));
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                                 ::"r"(smem_u32(stage)), "l"(&maps.m[c.job]), "r"(0), "r"((int)((c.t - c.begin) * (uint32_t)kBlocksPerTile + (e0 >> 5))),
+                                   "r"(smem_u32(&sh.bar[st])) : "memory");
+                    if (rd)
+                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], 16, [%2];"
+                                     ::"r"(smem_u32(sh.front[st])), "l"(c.xt + e0 - 4), "r"(smem_u32(&sh.bar[st])) : "memory");
+                }
+                return;
+            }
+            load_round_ragged(stage, c.xt, e0, c.len, lane);
+            if (lane == 0 && rd) sh.front[st][3] = __ldg(c.xt + e0 - 1u);
+            __syncwarp();
         }
-        ri.job = cj; ri.tile = t; ri.jtile = t - cj_begin; ri.rd = u & 3u;
-        ri.gslot = (cj_begin >> 5) + (uint32_t)cj + (ri.jtile >> 5);
-        const unsigned long long start = (unsigned long long)ri.jtile * kTile;
-        if (cj_n && prm.valid) {
-            ri.len = (uint32_t)((cj_n - start < (unsigned long long)kTile) ? (cj_n - start) : kTile);
-            ri.xt = cj_x + start;
-            ri.mapped = (((uintptr_t)cj_x) & 15u) == 0;
-        }
-        return ri;
-    };
-    // asks for a round into stage `buf`; lane 0 also fetches the element in front of the round
-    auto request = [&](uint32_t buf, const RoundInfo& ri, float& front) {
-        bool bulk = false;
-        const uint32_t e0 = ri.rd * (uint32_t)kRound;
-        if (e0 < ri.len) {
-            if (ri.mapped && e0 + (uint32_t)kRound <= ri.len) {
-                if (lane == 0) tensor_load_round(sh.stage[buf], &sh.bar[buf], &maps.m[ri.job], ri.jtile * (uint32_t)kBlocksPerTile + (e0 >> 5));
-                bulk = true;
-            } else load_round_ragged(sh.stage[buf], ri.xt, e0, ri.len, lane);
-            if (lane == 0) front = __ldg(ri.xt + (e0 ? e0 - 1u : 0u));   // a tile's first element is its own predecessor
-        }
-        if (buf) bulk1 = bulk; else bulk0 = bulk;
-    };
-    auto arrive = [&](uint32_t buf) {
-        if (buf ? bulk1 : bulk0) {
-            if (!mbar_wait(&sh.bar[buf], (buf ? fills1 : fills0) & 1u)) status |= kStTimeout;
-            if (buf) ++fills1; else ++fills0;
-        }
-        if (buf) bulk1 = false; else bulk0 = false;
-        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.bar[st]);
     };
 
-    // Rounds are dealt round-robin over the warps of the launch (no counter: same-address atomics would bound the kernel
-    // at about 1.5 ns per round), and the next round's input is asked for before this round is encoded.
-    const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
-    const uint32_t u0 = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
-    uint32_t u1 = u0 + stride;
-    if (u1 < u0) u1 = 0xFFFFFFFFu;
-    RoundInfo cur = locate(u0), nxt = locate(u1);
-    uint32_t p = 0;
-    float front = 0.0f, front1 = 0.0f;
-    request(0, cur, front);
+    TileCursor ahead;   // the tile two steps on, whose round is asked for while the current one is encoded
+    ahead.t = blockIdx.x; ahead.job = 0; ahead.begin = 0; ahead.count = 0; ahead.len = 0; ahead.xt = nullptr; ahead.aligned = false;
+    auto at = [&](const TileCursor& c) {
+        RoundAt a;
+        a.t = c.t; a.len = c.len; a.xt = c.xt;
+        a.gslot = (c.begin >> 5) + (uint32_t)c.job + ((c.t - c.begin) >> 5);
+        return a;
+    };
+    auto step = [&]() {
+        ahead.t = ahead.t + G < ahead.t ? 0xFFFFFFFFu : ahead.t + G;
+        cursor_settle(ahead, jb, prm.valid != 0);
+    };
+    cursor_settle(ahead, jb, prm.valid != 0);
+    RoundAt cur = at(ahead);
+    request(ahead, 0);
+    step();
+    RoundAt nxt = at(ahead);
+    request(ahead, 1);
+    step();
+
+    uint32_t st = 0, st2 = 2, phase = 0;   // stage of the current round, stage of the request, parity of the current stage's phase
     EncodeCarry cy;
     cy.pay_used = 0; cy.wide = false;
 
-    while (cur.job >= 0) {
-        __syncwarp();   // every lane is done with the other stage
-        request(p ^ 1u, nxt, front1);
-        const uint32_t u = 4u * cur.tile + cur.rd;
+    while (cur.t < jb.total_tiles) {
+        const uint32_t u = 4u * cur.t + rd;
         const uint32_t nb = (cur.len + kBlock - 1) / kBlock;
-        if (32u * cur.rd < nb) {
-            arrive(p);
-            uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
-            const float* st = sh.stage[p];
-            const char* row = reinterpret_cast<const char*>(st) + 128 * lane;
-            const uint32_t sw = ((uint32_t)lane & 7u) << 4;
-            const float xprev = lane ? read_last_of_row(st, (uint32_t)lane - 1u) : front;
-            // the buffer this round is encoded into was sent off two rounds ago: that store has to be through with it
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+        if (!mbar_wait(&sh.bar[st], phase)) status |= kStTimeout;
+        // the stage two steps on was encoded in place and sent off in the step before: the copy engine has to be through
+        // with it before the next request lands there; by the time the rows are read and sized it mostly is
+        auto mid = [&]() {
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             __syncwarp();
-            uint32_t* buf = sh.out[p];
+            request(ahead, st2);
+        };
+        if (32u * rd < nb) {
+            uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
+            float* stage = sh.stage[st];
+            const char* row = reinterpret_cast<const char*>(stage) + 128 * lane;
+            const float first = stage[0];
+            const float xprev = lane ? read_last_of_row(stage, (uint32_t)lane - 1u) : (rd ? sh.front[st][3] : first);
+            const uint32_t gslot = cur.gslot;
             cy.pay_used = 0;
-            const uint32_t bi = 32u * cur.rd + (uint32_t)lane;
-            // laid out like a tile's blob whose word 0 sits in front of the buffer: code-length bytes at words 1.., payload at word 9
-            const int rc = encode_round(row, sw, xprev, r, bi < nb, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, cy, lane,
-                                        status);
+            // in place: the stage becomes the round's slot image (code-length bytes at words 0.., payload at word 8), laid
+            // out like a tile's blob whose word 0 sits in front of it
+            const int rc = encode_round(row, sw, xprev, r, 32u * rd + (uint32_t)lane < nb, (uint32_t)lane, 32u, reinterpret_cast<uint32_t*>(stage) - 1,
+                                        0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, cy, lane, status, mid);
             if (rc == 0) {
-                __syncwarp();   // the buffer's words, written by all lanes, are visible to lane 0's store
+                __syncwarp();   // the words written by all lanes are visible to lane 0's store
                 if (lane == 0) {
                     const uint32_t bytes = (32u + 4u * cy.pay_used + 15u) & ~15u;
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(slot), "r"(smem_u32(buf)), "r"(bytes) : "memory");
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(slot), "r"(smem_u32(stage)), "r"(bytes) : "memory");
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     ws.round_words[u] = cy.pay_used;
-                    atomicAdd(ws.group_acc + cur.gslot, (unsigned long long)cy.pay_used);
-                    if (cur.rd == 0) {
-                        // exact while |x r| < 2^22; larger codes take the general route
-                        ws.outliers[cur.tile] = (int32_t)(__float_as_uint(__fadd_rn(__fmul_rn(front, r), kRoundMagic)) - kRoundMagicBits);
-                    }
+                    atomicAdd(ws.group_acc + gslot, (unsigned long long)cy.pay_used);
+                    // exact while |x r| < 2^22; larger codes take the general route
+                    if (rd == 0) ws.outliers[cur.t] = (int32_t)(__float_as_uint(__fadd_rn(__fmul_rn(first, r), kRoundMagic)) - kRoundMagicBits);
                 }
             } else {
-                status |= encode_round_general(cur.xt, cur.len, cur.rd, r, slot, ws.round_words + u, ws.outliers + cur.tile, ws.group_acc + cur.gslot,
-                                               lane);
+                status |= encode_round_general(cur.xt, cur.len, rd, r, slot, ws.round_words + u, ws.outliers + cur.t, ws.group_acc + gslot, lane);
             }
         } else {
+            mid();
             if (lane == 0) ws.round_words[u] = 0;   // a round beyond the tile's last block, or a tile without elements
         }
-        u1 = u1 + stride < u1 ? 0xFFFFFFFFu : u1 + stride;
         cur = nxt;
-        nxt = locate(u1);
-        front = front1;
-        p ^= 1u;
+        nxt = at(ahead);
+        step();
+        st2 = st;
+        st = st == (uint32_t)kRoundStages - 1u ? 0u : st + 1u;
+        if (st == 0) phase ^= 1u;
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the stores have read shared memory and are complete
     if (status) atomicOr(ws.status, status);
@@ -1543,7 +1562,7 @@ __device__ __noinline__ int encode_round_call(const char* row, uint32_t sw, floa
                                               uint32_t* status)
 {
     // laid out like a tile's blob whose word 0 sits in front of the buffer: code-length bytes at words 1.., payload at word 9
-    return encode_round(row, sw, xprev, r, active, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, *cy, lane, *status);
+    return encode_round(row, sw, xprev, r, active, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, *cy, lane, *status, [] {});
 }
 
 // Advances (pay_off, code) over round e of a tile without expanding it: the blocks' sizes from their code lengths,
