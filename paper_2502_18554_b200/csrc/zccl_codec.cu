@@ -1788,20 +1788,23 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
             carry_y = combine(op, xa, xb);
         }
         for (uint32_t rd = rd_first; rd < rd_stop; ++rd) {
-            // the copy engine is through with what it was handed in the round before: the other operand stage (an
-            // uncompressed copy of the result left from there) and the output buffer
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            __syncwarp();
+            // The other operand stage holds the round before, encoded in place and handed to the copy engine: the next
+            // operand round is asked into it once the engine is through with it, which by the end of this round's decoding it
+            // mostly is.
+            auto release_other = [&]() {
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                __syncwarp();
+            };
             float* loc = sh.loc[pl];
             const uint32_t u = 4u * t + rd;
             if (!good) {
+                release_other();
                 if (rd + 1 < rd_stop) request_loc(jcur, tile, rd + 1, pl ^ 1u);
                 else if (next_has_operand) request_loc(njob, ntile, nrd, pl ^ 1u);
                 else { if (pl) lbulk0 = false; else lbulk1 = false; }
                 arrive_loc(pl);
                 if (lane == 0) ws.round_words[u] = 0;
             } else {
-                if (rd + 1 < rd_stop) request_loc(jcur, tile, rd + 1, pl ^ 1u);
                 arrive_loc(pl);
                 if (blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
                     if (mode2 == 1) decode_round_call<0>(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr);
@@ -1810,7 +1813,9 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
                 }
                 if (mode1 == 1 && summing) decode_round_call<1>(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc);
                 else decode_round_general(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc, op);
-                if (rd + 1 == rd_stop) {   // the blob is decoded: the next unit's may come, and its first operand round
+                release_other();
+                if (rd + 1 < rd_stop) request_loc(jcur, tile, rd + 1, pl ^ 1u);
+                else {   // the blob is decoded: the next unit's may come, and its first operand round
                     look_ahead();
                     if (next_has_operand) request_loc(njob, ntile, nrd, pl ^ 1u);
                     else { if (pl) lbulk0 = false; else lbulk1 = false; }
@@ -1858,7 +1863,11 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
             }
             pl ^= 1u;
         }
-        if (rd_first >= rd_stop && next_has_operand) request_loc(njob, ntile, nrd, pl);
+        if (rd_first >= rd_stop && next_has_operand) {
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the stage may still be on its way out
+            __syncwarp();
+            request_loc(njob, ntile, nrd, pl);
+        }
         // rounds the tile does not have
         if ((uint32_t)lane >= rd_first && (uint32_t)lane < rd_end && (uint32_t)lane >= rounds) ws.round_words[4u * t + (uint32_t)lane] = 0;
         (void)next_known;
