@@ -64,8 +64,9 @@ enum { ZCCL_TILE = 4096, ZCCL_BLOCK = 32, ZCCL_HEADER_BYTES = 32, ZCCL_MAX_RANKS
        ZCCL_NOALLOC_MAX_ELEMS = 1 << 26 };  /* element limit of zccl_compress_noalloc (256 MiB of fp32) */
 
 /*
- * Context: look-back scan workspace for streams of up to `max_elems` elements, the device status word, the
- * resolved-bound block and, when max_ranks >= 2, an arena of compressed-chunk slots for zccl_sim_* sized for
+ * Context: placement workspace for streams of up to `max_elems` elements (a slot of 4128 bytes per 1024 elements, in
+ * which an encoded round waits for its place in the stream: about 1.01 times the size of the largest input, plus a
+ * few words per tile), the device status word, the resolved-bound block and, when max_ranks >= 2, an arena of compressed-chunk slots for zccl_sim_* sized for
  * max_ranks ranks exchanging max_elems elements in total per rank buffer (about (max_ranks + 2) *
  * zccl_compress_bound(max_elems) bytes).  Allocates on the current device; the only allocating call.
  * Returns ZCCL_E_ARG for max_elems == 0 or max_ranks outside [0, ZCCL_MAX_RANKS], ZCCL_E_CUDA if allocation fails.
@@ -89,10 +90,13 @@ int zccl_status(zccl_ctx* ctx, void* stream);
 unsigned long long zccl_launch_count(void);
 
 /*
- * Test hook for the bounded waits of the placement scan (failure detection; no paper counterpart).  While set,
- * the encoders do not publish the size of tile number `tile` of a launch, so the tiles after it find nothing to
- * wait for: their look-back gives up after its poll limit (a fraction of a second), writes nothing for those tiles
- * and records ZCCL_E_TIMEOUT; the context stays usable.  tile < 0 switches the hook off (the default).
+ * Test hook for the bounded waits of the single-pass encoder (failure detection; no paper counterpart).  That
+ * encoder, which zccl_compress_noalloc always uses, places tiles by a decoupled look-back: a warp waits, with a
+ * poll limit, for the sizes of the tiles in front of its own.  While the hook is set, zccl_compress takes the same
+ * encoder instead of its two wait-free launches and does not publish the size of tile number `tile` of a launch,
+ * so the tiles after it find nothing to wait for: their look-back gives up after its poll limit (a fraction of a
+ * second), writes nothing for those tiles and records ZCCL_E_TIMEOUT; the context stays usable.  tile < 0 switches
+ * the hook off (the default).
  */
 int zccl_debug_skip_publish(zccl_ctx* ctx, long long tile);
 
@@ -111,7 +115,9 @@ const char* zccl_strerror(int code);
  * fZ-light compression (Section 3.3; stream with the chunk-size index of Section 3.5.2).
  * Per 4096-element tile: q_i = rint(x_i * r), r = 1/s, s = 2 * (eb_abs * (1 - 2^-6)); 1-D Lorenzo deltas with the
  * tile's first code kept as a 4-byte outlier; per 32-element block the code length L = bit length of the largest
- * |delta| and, if L > 0, sign bits and L bit planes; tiles placed by a device-wide prefix scan of their sizes.
+ * |delta| and, if L > 0, sign bits and L bit planes.  Two launches, neither of which has a block waiting for
+ * another: rounds of 1024 elements are encoded into fixed slots of the context's workspace, then placed in the
+ * stream from the prefix sums of their sizes.
  *   x [device]          n floats (finite values); may be NULL only if n == 0
  *   out [device]        receives the stream; 4-byte aligned; out_capacity bytes writable
  *   out_bytes [device]  one size_t, receives the stream length in bytes (readable after the stream has run)
@@ -136,7 +142,10 @@ int zccl_decompress(zccl_ctx* ctx, const void* in, size_t in_bytes_max,
 
 /*
  * One reduce-scatter hop of the collective computation framework (Section 3.1.2; error chain of Eq. 2):
- * out_c = compress( decompress(in_c) + local ), in one kernel, with no uncompressed intermediate in memory.
+ * out_c = compress( decompress(in_c) + local ): decoding, reduction and encoding happen in one kernel, round by
+ * round in shared memory, with no uncompressed intermediate in global memory; a second, small launch places the
+ * encoded rounds in the stream, as for zccl_compress.  No block of either launch waits for another block, so
+ * hops of several contexts may run side by side on one device whatever share of it each gets.
  * y_i = fl32( fl32(float(q_i) * s) + local_i ), the decoded operand on the left; bound and step are in_c's.
  * With ZCCL_OP_MAX / ZCCL_OP_MIN in flags the addition becomes the larger / the smaller of the two operands.
  *   in_c [device]      received compressed chunk (at most in_bytes_max bytes are read)
@@ -158,17 +167,20 @@ int zccl_decompress_reduce_compress(zccl_ctx* ctx, const void* in_c, size_t in_b
  * of this library).  Work captured into a CUDA graph or running where an allocation would synchronise or is not
  * allowed, plug-ins living inside a host application's fixed memory budget, and out-of-memory or teardown
  * handlers cannot call zccl_ctx_create, because it calls cudaMalloc.  This entry point needs no context: its
- * placement-scan workspace is a fixed array inside the library (about 129 KiB of device memory on every GPU that
+ * placement-scan workspace is a fixed array inside the library (about 140 KiB of device memory on every GPU that
  * loads the library, until the process exits), and it calls no cudaMalloc, cudaFree or other allocating routine.
+ * Having no room for per-round slots, it compresses in a single pass (a warp per tile, positions by a decoupled
+ * look-back with bounded waits) instead of the two launches of zccl_compress.
  *   x, out, out_capacity, out_bytes [device], stream: as in zccl_compress;  eb_abs: absolute error bound
  *   n: at most ZCCL_NOALLOC_MAX_ELEMS, else ZCCL_E_TOO_LARGE is returned and nothing is enqueued
  * Produces the same bytes as zccl_compress(ctx, x, n, ZCCL_EB_ABS, eb_abs, ...).  There is no status word to read:
  * if the device detects an error (capacity overrun, value out of range) *out_bytes is set to 0 and the contents of
  * `out` are unspecified; the precision warning is not reported.
- * The first call on a device looks up the array's device address and initialises it with one small asynchronous
- * copy on `stream`; make that first call outside any stream capture.  All calls on a device share the array, which
- * keeps the previous call's contents (each call re-arms what it needs): calls whose kernels could overlap on the
- * GPU, for example on two streams, race and must be ordered by the caller.
+ * The first call on a device looks up the array's device address (a host-side look-up: nothing is enqueued, the
+ * array's counters carry their starting values in the module image), so the first call may come from any thread,
+ * on any stream, inside a capture or not.  All calls on a device share the array, which keeps the previous call's
+ * contents (each call re-arms what it needs): calls whose kernels could overlap on the GPU, for example on two
+ * streams, race and must be ordered by the caller.
  */
 int zccl_compress_noalloc(const float* x, size_t n, float eb_abs, void* out, size_t out_capacity,
                           size_t* out_bytes, void* stream);

@@ -1974,9 +1974,7 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     cudaError_t e = device_setup(&d);
     if (e != cudaSuccess) return e;
     if (!ws.slots) return cudaErrorInvalidValue;
-    static TileMaps loc_maps, raw_maps;   // too large for the stack of some callers; guarded by the lock below
-    static std::mutex mu;
-    std::lock_guard<std::mutex> lock(mu);
+    thread_local TileMaps loc_maps, raw_maps;   // 16 KiB: kept off the stack, one pair per calling thread
     memset(&loc_maps, 0, sizeof(loc_maps));
     memset(&raw_maps, 0, sizeof(raw_maps));
     for (int j = 0; j < jb.count; ++j) {

@@ -308,6 +308,7 @@ cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t
     const uint32_t nT = (uint32_t)((n + T - 1) / T);
     const unsigned grid = nT < (unsigned)sm_count * 4u ? (nT ? nT : 1u) : (unsigned)sm_count * 4u;
     const int dp = device_params ? 1 : 0;
+    count_launches(3);
     generic_encode_kernel<<<grid, 256, 0, st>>>(x, n, T, nT, hp, dp, sizes, out, go, 0, ws);
     generic_scan_kernel<<<1, 1024, 0, st>>>(sizes, n, T, nT, hp, dp, out, out_cap, out_bytes, go, ws);
     generic_encode_kernel<<<grid, 256, 0, st>>>(x, n, T, nT, hp, dp, sizes, out, go, 1, ws);
@@ -320,6 +321,7 @@ cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_byt
     const unsigned long long nT = (y_cap + T - 1) / T;
     const unsigned cap = (unsigned)sm_count * 4u;
     const unsigned grid = nT < cap ? (unsigned)(nT ? nT : 1) : cap;
+    count_launches(1);
     generic_decode_kernel<<<grid, 256, 0, st>>>(in, cap_bytes, T, y, y_cap, ws);
     return cudaGetLastError();
 }

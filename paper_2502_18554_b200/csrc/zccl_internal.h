@@ -167,5 +167,6 @@ cudaError_t launch_quality(const float* x, const float* y, unsigned long long n,
                            uint32_t* counter, int sm_count, cudaStream_t st);
 cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
 unsigned long long launch_count();
+void count_launches(unsigned k);   // adds to the process-wide count of kernels this library has launched
 
 }  // namespace zccl

@@ -362,6 +362,7 @@ std::atomic<unsigned long long> g_launches{0};   // kernels launched by this lib
 // ------------------------------------------------------------------------------------------------ launchers
 
 unsigned long long launch_count() { return g_launches; }
+void count_launches(unsigned k) { g_launches += k; }
 
 cudaError_t launch_range(const RangeBatch& rb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
@@ -417,12 +418,10 @@ cudaError_t launch_quality(const float* x, const float* y, unsigned long long n,
                            uint32_t* counter, int sm_count, cudaStream_t st)
 {
     unsigned long long want = (n / 4 + 255) / 256;
-    static int per_sm = 0;     // one wave of resident CTAs, each striding over the arrays
-    if (per_sm == 0) {
-        int a = 0;
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, quality_kernel, 256, 0);
-        per_sm = a > 0 ? a : 1;
-    }
+    // one wave of resident CTAs, each striding over the arrays; asked of the current device on every call (a host-side
+    // computation, no state shared between threads or devices)
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, quality_kernel, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
     unsigned long long cap = (unsigned long long)sm_count * per_sm;
     if (cap > (unsigned long long)kQualityCtas) cap = kQualityCtas;
     const unsigned grid = (unsigned)(want < cap ? (want ? want : 1) : cap);

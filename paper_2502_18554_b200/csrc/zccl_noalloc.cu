@@ -21,20 +21,24 @@ namespace {
 constexpr size_t kMaxElems = (size_t)ZCCL_NOALLOC_MAX_ELEMS;
 constexpr size_t kMaxTiles = kMaxElems / kTile + 1;
 constexpr size_t kStateBytes = ((kMaxTiles + 2 * (size_t)group_slots(kMaxTiles)) * 8 + 255) / 256 * 256;
-constexpr size_t kScratchBytes = kStateBytes + 256;   // scan states, then counters / status / parameter block
+constexpr size_t kScratchBytes = kStateBytes;
 
-// Scratch shared by every call on a device (about 129 KiB, held by each GPU that loads the library until exit).
+// Scratch shared by every call on a device (about 140 KiB of scan states plus a block of counters, held by each GPU
+// that loads the library until exit).  The counter block carries its starting values in the module image (the scan
+// states are validated against a launch counter that starts at 1), so no call ever has to initialise anything and
+// calls from any thread on any stream find the scratch ready.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
+static __device__ __align__(256) uint32_t g_noalloc_ctrl[64] = {0u /* ticket */, 0u /* done */, 1u /* launch counter */};
 
 struct DeviceSetup {
     bool ready = false;
     unsigned char* base = nullptr;   // device address of g_noalloc_scratch on that device
+    uint32_t* ctrl = nullptr;        // and of g_noalloc_ctrl
     int sm_count = 0;
 };
 constexpr int kMaxDevices = 64;
 DeviceSetup g_setup[kMaxDevices];
 std::mutex g_setup_mu;
-const uint32_t kEpochOne = 1u;
 
 // Runs after the encoder on the same stream: a device-side error turns the reported length into 0, and the shared
 // status word is cleared so that the next call starts clean.
@@ -45,13 +49,12 @@ __global__ void noalloc_finalize_kernel(uint32_t* status, size_t* out_bytes)
     *status = 0;
 }
 
-Workspace workspace_at(unsigned char* base)
+Workspace workspace_at(unsigned char* base, uint32_t* sm)
 {
     Workspace ws{};
     ws.tile_state = reinterpret_cast<unsigned long long*>(base);
     ws.group_state = ws.tile_state + kMaxTiles;
     ws.group_acc = ws.group_state + group_slots(kMaxTiles);
-    uint32_t* sm = reinterpret_cast<uint32_t*>(base + kStateBytes);
     ws.ticket = sm + 0;
     ws.done = sm + 1;
     ws.epoch = sm + 2;
@@ -64,8 +67,9 @@ Workspace workspace_at(unsigned char* base)
     return ws;
 }
 
-// First call on a device, with that device current: resolve the array's device address and arm the scan epoch.
-int setup_current_device(DeviceSetup** out, cudaStream_t st)
+// First call on a device, with that device current: resolve the arrays' device addresses (host-side look-ups: nothing
+// is enqueued, so there is nothing for a concurrent caller on another stream to wait for).
+int setup_current_device(DeviceSetup** out)
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return ZCCL_E_CUDA;
@@ -74,14 +78,14 @@ int setup_current_device(DeviceSetup** out, cudaStream_t st)
     DeviceSetup& s = g_setup[dev];
     if (!s.ready) {
         void* ptr = nullptr;
+        void* ctrl = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return ZCCL_E_CUDA;
+        if (cudaGetSymbolAddress(&ctrl, g_noalloc_ctrl) != cudaSuccess || ctrl == nullptr) return ZCCL_E_CUDA;
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return ZCCL_E_CUDA;
         s.base = static_cast<unsigned char*>(ptr);
+        s.ctrl = static_cast<uint32_t*>(ctrl);
         s.sm_count = sms;
-        // the array starts zeroed; scan states are validated against a launch counter that must start at 1
-        Workspace ws = workspace_at(s.base);
-        if (cudaMemcpyAsync(ws.epoch, &kEpochOne, sizeof(uint32_t), cudaMemcpyHostToDevice, st) != cudaSuccess) return ZCCL_E_CUDA;
         s.ready = true;
     }
     *out = &s;
@@ -110,9 +114,9 @@ extern "C" int zccl_compress_noalloc(const float* x, size_t n, float eb_abs, voi
 
     cudaStream_t st = (cudaStream_t)stream;
     DeviceSetup* dev = nullptr;
-    const int rc = setup_current_device(&dev, st);
+    const int rc = setup_current_device(&dev);
     if (rc != ZCCL_OK) return rc;
-    const Workspace ws = workspace_at(dev->base);
+    const Workspace ws = workspace_at(dev->base, dev->ctrl);
 
     JobBatch jb{};
     jb.count = 1;
@@ -120,6 +124,7 @@ extern "C" int zccl_compress_noalloc(const float* x, size_t n, float eb_abs, voi
     j.x = x; j.out = (uint32_t*)out; j.out_bytes = out_bytes; j.n = n; j.out_cap = out_capacity; j.tile_begin = 0;
     jb.total_tiles = (uint32_t)(nT ? nT : 1);
     if (launch_encode(jb, kEncodeRaw, ws, false, hp, dev->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
+    count_launches(1);
     noalloc_finalize_kernel<<<1, 1, 0, st>>>(ws.status, out_bytes);
     return cudaGetLastError() == cudaSuccess ? ZCCL_OK : ZCCL_E_CUDA;
 }
