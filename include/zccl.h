@@ -40,7 +40,8 @@ typedef struct zccl_ctx zccl_ctx;
 
 /* How `eb` is read.  The paper's tables quote value-range-relative bounds ("REL", Tables 1-4). */
 enum { ZCCL_EB_ABS = 0,    /* eb is the absolute bound eb_abs */
-       ZCCL_EB_REL = 1 };  /* eb_abs = eb * (max - min) of the input (of all ranks' inputs in zccl_sim_*) */
+       ZCCL_EB_REL = 1,    /* eb_abs = eb * (max - min) of the input (of all ranks' inputs in zccl_sim_*) */
+       ZCCL_EB_RESOLVED = 2 };  /* the bound zccl_resolve_range left in the context, on the device; eb is ignored */
 
 enum { ZCCL_OK = 0,
        ZCCL_E_ARG = -1,         /* NULL pointer, size beyond the context's limits, eb not positive and finite */
@@ -81,7 +82,8 @@ size_t zccl_compress_bound(size_t n);
 
 /*
  * Synchronises `stream`, returns the most severe condition recorded on the device since the last call
- * (errors before the warning, ZCCL_OK if none) and clears the record.
+ * (TIMEOUT, DEGENERATE, BAD_STREAM, RANGE, CAPACITY in that order, then the warning, ZCCL_OK if none) and clears
+ * the record.
  */
 int zccl_status(zccl_ctx* ctx, void* stream);
 
@@ -295,17 +297,26 @@ int zccl_decompress_tiled(zccl_ctx* ctx, const void* in, size_t in_bytes_max, un
 int zccl_stream_stats(zccl_ctx* ctx, const void* in, size_t in_bytes_max, unsigned long long* hist, void* stream);
 
 /*
- * The two per-rank steps of a real ring that are not a codec call (Section 3.2: the error bound is resolved once
+ * The per-rank steps of a real ring that are not a codec call (Section 3.2: the error bound is resolved once
  * per collective, over the data of all ranks; Corollary 2: Average = Sum / N).
  *   zccl_range: minmax [device, 2 floats] <- (min, max) of x [device, n floats]; (+inf, -inf) when n == 0.  A
  *               rank combines these with its peers' (min of minima, max of maxima), forms
  *               eb_abs = fl32(eb * fl32(max - min)) and passes it to the codec calls as ZCCL_EB_ABS; that is the
  *               bound a ZCCL_EB_REL call over the concatenated data would resolve.
+ *   zccl_resolve_range: the same resolution without the host: minmax [device, 2 floats] is the combined pair
+ *               (for example after a Min/Max all-reduce of the ranks' pairs); the bound
+ *               eb_abs = fl32(eb_rel * fl32(max - min)), its step and reciprocal go into the context's resolved-bound
+ *               block, where zccl_compress and the zccl_*_host forms find them when called with ZCCL_EB_RESOLVED;
+ *               eb_abs_out [device, 1 float, or NULL] also receives eb_abs (0 when the range is degenerate).  The
+ *               block keeps its contents until the next zccl_resolve_range or ZCCL_EB_REL call on the context.
+ *               Device-side: DEGENERATE when max - min is zero, negative, infinite or not a number; codec calls
+ *               that use the block then write a header-less, empty stream (length 0).
  *   zccl_scale: y [device, n floats] <- y / divisor, one IEEE fp32 division per element.
- * Both enqueue on `stream` and return at once.  ZCCL_E_ARG for null or misaligned pointers, n beyond the
- * context's max_elems (range), a divisor that is not a positive finite number (scale).
+ * All enqueue on `stream` and return at once.  ZCCL_E_ARG for null or misaligned pointers, n beyond the
+ * context's max_elems (range), a bound or divisor that is not a positive finite number (resolve_range, scale).
  */
 int zccl_range(zccl_ctx* ctx, const float* x, size_t n, float* minmax, void* stream);
+int zccl_resolve_range(zccl_ctx* ctx, const float* minmax, float eb_rel, float* eb_abs_out, void* stream);
 int zccl_scale(zccl_ctx* ctx, float* y, size_t n, float divisor, void* stream);
 
 /*

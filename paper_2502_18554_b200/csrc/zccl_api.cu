@@ -66,6 +66,7 @@ int resolve_abs_host(float eb, Params& p)
 
 inline bool eb_ok(int mode, float eb)
 {
+    if (mode == ZCCL_EB_RESOLVED) return true;   // the bound is the context's resolved block; eb is not looked at
     return (mode == ZCCL_EB_ABS || mode == ZCCL_EB_REL) && eb > 0.0f && std::isfinite(eb);
 }
 
@@ -96,6 +97,11 @@ int resolve_bound(zccl_ctx* c, const RangeList& rl, int mode, float eb, Params& 
 {
     on_device = false;
     if (mode == ZCCL_EB_ABS) return resolve_abs_host(eb, hp);
+    if (mode == ZCCL_EB_RESOLVED) {     // zccl_resolve_range (or an earlier ZCCL_EB_REL call) left the bound on the device
+        hp = Params{0.f, 1.f, 1.f, 1};
+        on_device = true;
+        return ZCCL_OK;
+    }
     size_t total = 0;
     for (size_t v : rl.n) total += v;
     if (total == 0) return ZCCL_E_DEGENERATE;
@@ -291,8 +297,8 @@ int zccl_status(zccl_ctx* c, void* stream)
     if (cudaMemsetAsync(c->ws.status, 0, 4, st) != cudaSuccess) return ZCCL_E_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return ZCCL_E_CUDA;
     if (bits & kStTimeout) return ZCCL_E_TIMEOUT;
+    if (bits & kStDegenerate) return ZCCL_E_DEGENERATE;   // the cause of the empty streams that later calls then reject
     if (bits & kStBadStream) return ZCCL_E_BAD_STREAM;
-    if (bits & kStDegenerate) return ZCCL_E_DEGENERATE;
     if (bits & kStRange) return ZCCL_E_RANGE;
     if (bits & kStCapacity) return ZCCL_E_CAPACITY;
     if (bits & kStPrecision) return ZCCL_W_PRECISION;
@@ -753,6 +759,13 @@ int zccl_range(zccl_ctx* c, const float* x, size_t n, float* minmax, void* strea
     rb.finish = kRangeExport;
     rb.out = minmax;
     return cuda_rc(launch_range(rb, c->ws, c->sm_count, st));
+}
+
+int zccl_resolve_range(zccl_ctx* c, const float* minmax, float eb_rel, float* eb_abs_out, void* stream)
+{
+    if (!c || !minmax || !(eb_rel > 0.0f) || !std::isfinite(eb_rel)) return ZCCL_E_ARG;
+    if (((uintptr_t)minmax & 3u) || ((uintptr_t)eb_abs_out & 3u)) return ZCCL_E_ARG;
+    return cuda_rc(launch_resolve_range(minmax, eb_rel, c->ws, eb_abs_out, (cudaStream_t)stream));
 }
 
 int zccl_scale(zccl_ctx* c, float* y, size_t n, float divisor, void* stream)

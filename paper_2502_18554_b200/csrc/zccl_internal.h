@@ -152,6 +152,7 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
 cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st);
+cudaError_t launch_resolve_range(const float* minmax, float eb, const Workspace& ws, float* eb_abs_out, cudaStream_t st);
 cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* sizes,
                                   uint32_t* go, uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws,
                                   int sm_count, cudaStream_t st);

@@ -14,18 +14,12 @@ namespace {
 
 // eb -> (eb_abs, s, r), the reading used throughout: eb_abs = eb * (max - min); step shrunk by 1 - 2^-6;
 // r by one IEEE division.  Consumes and re-arms the min/max keys.  One thread.
-__device__ void resolve_params(float eb, const Workspace& ws)
+__device__ void resolve_from_range(float eb, float range, const Workspace& ws, float* eb_abs_out)
 {
     Params p;
     p.valid = 1;
-    const uint32_t kmin = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 0);
-    const uint32_t kmax = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 1);
-    float range = 0.0f;
-    if (kmin <= kmax) range = __fsub_rn(key2f(kmax), key2f(kmin));
     if (!(range > 0.0f) || !isfinite(range)) p.valid = 0;
     const float ea = __fmul_rn(eb, range);
-    ws.minmax[0] = 0xFFFFFFFFu;
-    ws.minmax[1] = 0u;
     const float ebq = __fmul_rn(ea, 0.984375f);
     const float s = __fmul_rn(ebq, 2.0f);
     if (!(s > 0.0f) || !isfinite(s)) p.valid = 0;
@@ -33,7 +27,28 @@ __device__ void resolve_params(float eb, const Workspace& ws)
     if (!isfinite(r)) p.valid = 0;
     p.eb_abs = ea; p.s = s; p.r = r;
     *ws.params = p;
+    if (eb_abs_out) *eb_abs_out = p.valid ? ea : 0.0f;
     if (!p.valid) atomicOr(ws.status, kStDegenerate);
+}
+__device__ void resolve_params(float eb, const Workspace& ws)
+{
+    const uint32_t kmin = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 0);
+    const uint32_t kmax = *reinterpret_cast<volatile uint32_t*>(ws.minmax + 1);
+    float range = 0.0f;
+    if (kmin <= kmax) range = __fsub_rn(key2f(kmax), key2f(kmin));
+    ws.minmax[0] = 0xFFFFFFFFu;
+    ws.minmax[1] = 0u;
+    resolve_from_range(eb, range, ws, nullptr);
+}
+
+// The same from a (min, max) pair the caller has on the device: a rank's own pair combined with its peers'.
+__global__ void resolve_range_kernel(const float* __restrict__ minmax, float eb, Workspace ws, float* eb_abs_out)
+{
+    pdl_enter();
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        const float lo = minmax[0], hi = minmax[1];
+        resolve_from_range(eb, lo <= hi ? __fsub_rn(hi, lo) : 0.0f, ws, eb_abs_out);
+    }
 }
 
 // Hands the minimum and maximum to the caller (out[0] = min, out[1] = max; +inf, -inf when nothing was scanned)
@@ -402,6 +417,12 @@ cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, 
     unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
     ++g_launches;
     return launch_k(copy_kernel, dim3(gx ? gx : 1, cb.count), dim3(256), 0, st, cb, ws);
+}
+
+cudaError_t launch_resolve_range(const float* minmax, float eb, const Workspace& ws, float* eb_abs_out, cudaStream_t st)
+{
+    ++g_launches;
+    return launch_k(resolve_range_kernel, dim3(1), dim3(32), 0, st, minmax, eb, ws, eb_abs_out);
 }
 
 cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st)

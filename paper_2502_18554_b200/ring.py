@@ -52,6 +52,9 @@ class DegenerateRange(ValueError):
     """A relative bound over data whose range is zero, infinite or not a number."""
 
 
+RESOLVED = object()   # stands for "the bound the codec resolved on the device" where an absolute bound is expected
+
+
 class DeviceCodec:
     """The per-rank codec steps on the rank's GPU; each method enqueues one call of the C boundary."""
 
@@ -68,8 +71,17 @@ class DeviceCodec:
         self.ctx.range(x, out)
         return out
 
-    def compress(self, x, eb_abs: float, out, out_bytes):
-        self.ctx.compress(x, z.EB_ABS, eb_abs, out, out_bytes)
+    def resolve(self, minmax: torch.Tensor, eb_rel: float):
+        """The relative bound over a (min, max) pair that is on the device, resolved on the device: no value comes
+        back to the host.  Returns the token that compress takes in place of an absolute bound."""
+        self.ctx.resolve_range(minmax, eb_rel)
+        return RESOLVED
+
+    def compress(self, x, eb_abs, out, out_bytes):
+        if eb_abs is RESOLVED:
+            self.ctx.compress(x, z.EB_RESOLVED, 0.0, out, out_bytes)
+        else:
+            self.ctx.compress(x, z.EB_ABS, eb_abs, out, out_bytes)
 
     def drc(self, in_c, n: int, local, out, out_bytes, raw_out, flags: int):
         if n == 0:
@@ -84,7 +96,12 @@ class DeviceCodec:
 
     def finish(self) -> int:
         """Waits for the enqueued work and raises on a device-side error; returns the warning code, if any."""
-        return self.ctx.check()
+        try:
+            return self.ctx.check()
+        except z.ZcclError as exc:
+            if exc.code == z.E_DEGENERATE:
+                raise DegenerateRange("relative bound over data without a finite, non-zero range") from exc
+            raise
 
 
 class _Msg:
@@ -199,9 +216,11 @@ class Ring:
 
     # ------------------------------------------------------------------------------------------------ the bound
 
-    def resolve(self, x: torch.Tensor, eb_mode: int, eb: float, collective: bool = True) -> float:
+    def resolve(self, x: torch.Tensor, eb_mode: int, eb: float, collective: bool = True):
         """eb -> absolute bound.  A relative bound refers to the range of the data of all ranks (of x alone when
-        `collective` is false): eb_abs = fl32(eb * fl32(max - min))."""
+        `collective` is false): eb_abs = fl32(eb * fl32(max - min)).  A codec that can resolve on the device gets
+        the combined (min, max) there and the host never waits for it (a range without extent then shows up as
+        DegenerateRange when the collective finishes, on every rank alike); otherwise the host forms the bound."""
         if not (eb > 0) or not np.isfinite(eb):
             raise ValueError("the error bound must be a positive finite number")
         if eb_mode == z.EB_ABS:
@@ -212,6 +231,9 @@ class Ring:
         t = torch.stack([-mm[0], mm[1]])
         if collective and self.N > 1:
             t = self.link.all_max(t)
+        if hasattr(self.codec, "resolve"):
+            pair = torch.stack([-t[0], t[1]]).to(mm.device)   # back on the codec's device when the messages go through the host
+            return self.codec.resolve(pair, float(np.float32(eb)))
         lo, hi = np.float32(-t[0].item()), np.float32(t[1].item())
         with np.errstate(all="ignore"):
             rng = np.float32(hi - lo)

@@ -15,7 +15,7 @@ LIB_PATH = _PKG / "libzccl.so"
 OK, E_ARG, E_CUDA, E_CAPACITY, E_RANGE, E_BAD_STREAM, E_TIMEOUT, E_DEGENERATE, W_PRECISION = 0, -1, -2, -3, -4, -5, -6, -7, 1
 E_TOO_LARGE = -8
 NOALLOC_MAX_ELEMS = 1 << 26
-EB_ABS, EB_REL = 0, 1
+EB_ABS, EB_REL, EB_RESOLVED = 0, 1, 2
 CONSISTENT_OWNER = 1
 OP_SUM, OP_MAX, OP_MIN, OP_AVG = 0, 2, 4, 6   # reduce operation, or-ed into flags
 TILE, BLOCK, HEADER_BYTES = 4096, 32, 32
@@ -24,7 +24,7 @@ EXPORTS = [
     "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_reduce_scatter", "zccl_sim_scatter",
-    "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_scale", "zccl_stream_stats",
+    "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_resolve_range", "zccl_scale", "zccl_stream_stats",
     "zccl_compress_bound_tiled", "zccl_compress_tiled", "zccl_decompress_tiled",
     "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
     "zccl_debug_set_launch_counter",
@@ -68,6 +68,7 @@ def lib():
         L.zccl_sim_scatter.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
         L.zccl_quality.argtypes = [vp, vp, vp, sz, vp, vp]
         L.zccl_range.argtypes = [vp, vp, sz, vp, vp]
+        L.zccl_resolve_range.argtypes = [vp, vp, C.c_float, vp, vp]
         L.zccl_stream_stats.argtypes = [vp, vp, sz, vp, vp]
         L.zccl_compress_bound_tiled.argtypes = [sz, C.c_uint]
         L.zccl_compress_bound_tiled.restype = sz
@@ -257,6 +258,13 @@ class Context:
         """zccl_range: minmax (float32[2], device) <- (min x, max x)."""
         _check(lib().zccl_range(self._h, _dev_ptr(x, torch.float32) if x.numel() else None, x.numel(),
                                 _dev_ptr(minmax, torch.float32), _stream_ptr(stream)), "zccl_range")
+
+    def resolve_range(self, minmax: torch.Tensor, eb_rel: float, eb_abs_out: torch.Tensor | None = None, stream=None):
+        """zccl_resolve_range: the bound eb_rel * (max - min) from a device (min, max) pair into the context's
+        resolved-bound block, for calls with EB_RESOLVED; eb_abs_out (float32[1], device) also receives it."""
+        _check(lib().zccl_resolve_range(self._h, _dev_ptr(minmax, torch.float32), eb_rel,
+                                        _dev_ptr(eb_abs_out, torch.float32) if eb_abs_out is not None else None,
+                                        _stream_ptr(stream)), "zccl_resolve_range")
 
     def scale(self, y: torch.Tensor, divisor: float, stream=None):
         """zccl_scale: y <- y / divisor in place."""

@@ -832,3 +832,115 @@ def test_allreduce_whose_hops_fit_the_device_at_once(z):
     for r in range(N):
         assert_same_bits(recv[r].cpu().numpy(), want[r])
     c.close()
+
+
+def test_resolve_range_on_the_device(z, ctx):
+    """zccl_resolve_range + ZCCL_EB_RESOLVED give the stream a relative bound over the combined range gives: the pair
+    is put together from two arrays' pairs on the device, as two ranks of a ring would, and the oracle resolves the
+    same bound from the concatenated data."""
+    a = fields.smooth_1d(50_000, seed=3)
+    b = (fields.smooth_1d(50_000, seed=4) * np.float32(1.7)).astype(np.float32)
+    xa, xb = dev(a), dev(b)
+    ma = torch.zeros(2, dtype=torch.float32, device="cuda")
+    mb = torch.zeros(2, dtype=torch.float32, device="cuda")
+    ctx.range(xa, ma)
+    ctx.range(xb, mb)
+    mm = torch.stack([torch.minimum(ma[0], mb[0]), torch.maximum(ma[1], mb[1])])
+    ea_dev = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ctx.resolve_range(mm, 1e-3, ea_dev)
+    ea, s, r = oracle.resolve(oracle.EB_REL, 1e-3, np.concatenate([a, b]))
+    for arr, x in ((a, xa), (b, xb)):     # the block keeps its contents from call to call
+        cap = z.compress_bound(arr.size)
+        out = torch.empty(cap, dtype=torch.uint8, device="cuda")
+        nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+        ctx.compress(x, z.EB_RESOLVED, 0.0, out, nb)
+        assert ctx.check() in (z.OK, z.W_PRECISION)
+        want, _ = oracle.compress_core(arr, ea, s, r)
+        assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+    assert np.float32(ea_dev.item()) == np.float32(ea)
+    # a pair without extent: the device reports it, nothing is written
+    ctx.resolve_range(torch.tensor([2.0, 2.0], device="cuda"), 1e-3, ea_dev)
+    out = torch.empty(z.compress_bound(a.size), dtype=torch.uint8, device="cuda")
+    nb = torch.ones(1, dtype=torch.int64, device="cuda")
+    ctx.compress(xa, z.EB_RESOLVED, 0.0, out, nb)
+    assert ctx.status() == z.E_DEGENERATE
+    assert int(nb.item()) == 0 and float(ea_dev.item()) == 0.0
+    with pytest.raises(z.ZcclError):
+        ctx.resolve_range(mm, 0.0)
+
+
+def test_two_contexts_on_two_streams_run_hops_side_by_side(z):
+    """Fused hops of two contexts enqueued on two streams without any ordering between them: whichever share of the
+    device each launch gets, and in whichever order their blocks run, both results are the oracle's.  (No block of
+    the hop's launches waits for another block, so there is nothing for co-scheduling to break.)"""
+    n = 3_000_000
+    ctxs = [z.Context(n, 0), z.Context(n, 0)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    cases = []
+    for k in range(2):
+        a = fields.smooth_1d(n, seed=10 + k)
+        b = fields.smooth_1d(n, seed=20 + k)
+        ea, s, r = oracle.resolve(oracle.EB_REL, 1e-3, np.concatenate([a, b]))
+        sa, _ = oracle.compress_core(a, ea, s, r)
+        want, _, wraw = oracle.drc(sa, local=b, want_raw=True)
+        cap = z.compress_bound(n)
+        cases.append(dict(sa=torch.from_numpy(sa.copy()).cuda(), b=dev(b), want=want, wraw=wraw,
+                          out=[torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(6)],
+                          nb=[torch.zeros(1, dtype=torch.int64, device="cuda") for _ in range(6)],
+                          raw=[torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(6)]))
+    torch.cuda.synchronize()
+    for rep in range(6):                      # interleaved enqueues: the launches of the two streams overlap on the device
+        for k in range(2):
+            c = cases[k]
+            with torch.cuda.stream(streams[k]):
+                ctxs[k].decompress_reduce_compress(c["sa"], n, c["out"][rep], c["nb"][rep], local=c["b"], raw_out=c["raw"][rep],
+                                                   stream=streams[k])
+    torch.cuda.synchronize()
+    for k in range(2):
+        assert ctxs[k].check() in (z.OK, z.W_PRECISION)
+        c = cases[k]
+        for rep in range(6):
+            got = c["out"][rep][: int(c["nb"][rep].item())].cpu().numpy()
+            assert np.array_equal(got, c["want"])
+            assert_same_bits(c["raw"][rep].cpu().numpy(), c["wraw"])
+
+
+def test_launches_from_several_threads(z):
+    """Four host threads, each with a context and a stream of its own, compress and decompress at the same time: the
+    launchers share no mutable state, so every thread gets the oracle's stream."""
+    import threading
+    n = 400_000
+    arrs = [fields.smooth_1d(n, seed=30 + k) for k in range(4)]
+    wants = [oracle.compress(a, oracle.EB_ABS, 1e-3)[0] for a in arrs]
+    errors = []
+
+    def work(k):
+        try:
+            torch.cuda.set_device(0)
+            st = torch.cuda.Stream()
+            ctx = z.Context(n, 0)
+            x = torch.from_numpy(arrs[k]).cuda()
+            cap = z.compress_bound(n)
+            for _ in range(8):
+                out = torch.empty(cap, dtype=torch.uint8, device="cuda")
+                nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+                y = torch.empty(n, dtype=torch.float32, device="cuda")
+                with torch.cuda.stream(st):
+                    ctx.compress(x, z.EB_ABS, 1e-3, out, nb, stream=st)
+                    ctx.decompress(out, y, stream=st)
+                st.synchronize()
+                if ctx.check(stream=st) not in (z.OK, z.W_PRECISION):
+                    errors.append((k, "status"))
+                if not np.array_equal(out[: int(nb.item())].cpu().numpy(), wants[k]):
+                    errors.append((k, "stream"))
+                if not np.array_equal(y.cpu().numpy(), oracle.decompress(wants[k])):
+                    errors.append((k, "values"))
+        except Exception as exc:   # a thread's exception must fail the test
+            errors.append((k, repr(exc)))
+
+    threads = [threading.Thread(target=work, args=(k,)) for k in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors

@@ -1,5 +1,5 @@
 """The allocation-free compressor (zccl_compress_noalloc), through the C-ABI, against the context-based entry
-point it mirrors.  Some callers of this library cannot allocate device memory (work captured into a CUDA graph,
+point it mirrors and against the CPU oracle.  Some callers of this library cannot allocate device memory (work captured into a CUDA graph,
 plug-ins with a fixed memory budget, out-of-memory handlers), so they cannot create a context; this entry point
 keeps its scan workspace in a fixed array inside the library instead.  The array is shared by all calls and keeps
 the previous call's contents, hence the check on two calls in a row with different inputs.
@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2502_18554_b200 import fields
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +45,7 @@ def test_noalloc_matches_context_entry_point_on_two_calls_in_a_row(z):
         got = out[: int(nbytes.item())].cpu().numpy()
         assert got.size == want.size
         assert np.array_equal(got, want)                              # same bytes as zccl_compress
+        assert np.array_equal(got, oracle.compress(x, oracle.EB_ABS, eb)[0])   # and as the CPU oracle
         assert bool((out[z.compress_bound(x.size):] == 0xEE).all())   # nothing written past the capacity
     ctx.close()
 
