@@ -33,10 +33,11 @@ REL = 1e-3
 RANKS = 8
 AG_PER_RANK = 1 << 18               # allgather: 1 MiB per rank
 ROT = 4                             # rotating buffer sets, each larger than L2
-# dram__bytes_read.sum + dram__bytes_write.sum of one 64 MiB launch of the fused kernel, from the ncu capture
-# summarised in profiles/encode_decode_fused_kernels_cfg1_64MiB.md (78.2 MB read + 3.8 MB written; the 12 MB output
-# stream is mostly still in L2 when the kernel ends)
-DRAM_TRAFFIC_FUSED_64MIB = 82.0e6
+MIN_TIMED_MS = 500.0                # the timed region lasts at least this long (steps are replayed to get there)
+# dram__bytes_read.sum + dram__bytes_write.sum of one 64 MiB call of the fused hop (its two launches together), from an
+# ncu capture of this workload: 78.6 MB read + 4.2 MB written by the hop kernel, 0.3 MB by the placement (the encoded
+# rounds wait in L2 between the two, and most of the 12 MB output stream is still there when the call ends)
+DRAM_TRAFFIC_FUSED_64MIB = 83.1e6
 METRIC = "compress / decompress / fused decomp-reduce-comp GB/s (uncompressed bytes through the codec per step)"
 WORKLOAD = ("cfg1: 256^3 fp32 Fourier-mode field (64 MiB), REL 1e-3; step = compress + decompress + fused hop + "
             "8-rank ring allreduce (8 MiB/rank) + 8-rank allgather (1 MiB/rank)")
@@ -203,6 +204,42 @@ def _timed(fn, sets: int, warmup: int = 10, iters: int = 10):
         b.synchronize()
         ts.append(a.elapsed_time(b) * 1e3 / sets)
     return statistics.mean(ts), min(ts)
+
+
+def _timed_long(fn, sets: int, device_index: int, min_launches: int = 200, min_ms: float = 400.0, warmup: int = 3):
+    """Device time (us) of one call fn(set index) over a long run: a CUDA graph of `sets` calls is replayed until
+    at least `min_launches` calls and `min_ms` milliseconds have gone by, inside ONE pair of events, with the SM clock
+    sampled meanwhile.  Returns (us per call, calls, median SM MHz or None)."""
+    import torch
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for i in range(sets):
+            fn(i)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(sets):
+            fn(i)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(warmup):
+        g.replay()
+    b.record()
+    b.synchronize()
+    est_ms = max(a.elapsed_time(b) / warmup, 1e-3)
+    replays = max(-(-min_launches // sets), int(min_ms / est_ms) + 1)
+    sampler = ClockSampler(device_index)
+    sampler.start()
+    time.sleep(0.25)            # the sampler's first line takes this long to come
+    a.record()
+    for _ in range(replays):
+        g.replay()
+    b.record()
+    b.synchronize()
+    clocks = sampler.stop()
+    return a.elapsed_time(b) * 1e3 / (replays * sets), replays * sets, clocks.get("sm_mhz")
 
 
 def _codec_row(z, ctx, name, x_h, mode, eb, with_oracle: bool, loc_h=None):
@@ -383,6 +420,51 @@ def config_table(args):
 
 # --------------------------------------------------------------------------------------------- CUDA arm
 
+def other_configs(z, peak: float, x1, loc1) -> dict:
+    """The configurations the step itself does not cover, timed like the rows of --table (10 warm-up + 10 timed graph
+    replays per call): cfg1 at the looser and the tighter bound (all three calls), cfg3 (1 GiB gradient-like array,
+    compress and decompress) and cfg2 at full size (emulated 8-rank ring Allreduce of 64 MiB per rank).  `frac` =
+    algorithmic bytes (input + output of the call) / time / the measured copy bandwidth."""
+    import torch
+    from paper_2502_18554_b200 import fields
+    out = {}
+
+    def fracs(row):
+        nbytes, cbytes = row["bytes"], row["bytes"] / row["ratio"]
+        r = {"ratio": row["ratio"], "status": row["status"],
+             "compress_us": row["compress_us_mean"], "compress_frac": round((nbytes + cbytes) / row["compress_us_mean"] / 1e3 / peak, 3),
+             "decompress_us": row["decompress_us_mean"], "decompress_frac": round((nbytes + cbytes) / row["decompress_us_mean"] / 1e3 / peak, 3),
+             "compress_gbs": row["compress_gbs"], "decompress_gbs": row["decompress_gbs"]}
+        if "fused_us_mean" in row:
+            fbytes = nbytes / row["fused_out_ratio"]
+            r.update({"fused_us": row["fused_us_mean"], "fused_gbs": row["fused_gbs"],
+                      "fused_frac": round((cbytes + nbytes + fbytes) / row["fused_us_mean"] / 1e3 / peak, 3)})
+        return r
+
+    big = z.Context(1 << 28, 1)
+    for eb in (1e-2, 1e-4):
+        out[f"cfg1 REL {eb:g}"] = fracs(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, False, loc1))
+    out["cfg3 ABS 1e-05 (1 GiB)"] = fracs(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, False))
+    big.close()
+    torch.cuda.empty_cache()
+
+    N = RANKS
+    ctx = z.Context(1 << 27, N)
+    send = [torch.from_numpy(a).cuda() for a in fields.rank_fields(N, 1 << 24, base_seed=100)]
+    recv = [torch.empty(1 << 24, dtype=torch.float32, device="cuda") for _ in range(N)]
+    ar_mean, ar_best = _timed(lambda i: ctx.sim_allreduce(send, recv, z.EB_REL, REL), 1)
+    rc = ctx.check()
+    chunk_bytes = 4 * (1 << 21)
+    units = N * chunk_bytes + 2 * (N - 1) * N * chunk_bytes
+    out["cfg2 allreduce 8 x 64 MiB REL 0.001"] = {
+        "status": rc, "allreduce_us": round(ar_mean, 1), "allreduce_us_best": round(ar_best, 1),
+        "codec_gbs": round(units / ar_mean / 1e3, 1), "algbw_gbs": round(4 * (1 << 24) / ar_mean / 1e3, 1)}
+    ctx.close()
+    del send, recv
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -390,6 +472,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="leave the `configs` object (cfg1 at other bounds, cfg2, cfg3) out")
     ap.add_argument("--no-graph", action="store_true", help="time eagerly launched steps instead of CUDA graph replays")
     ap.add_argument("--table", action="store_true",
                     help="time configurations 0-4 one by one (one JSON line per row) instead of the benchmark step")
@@ -511,25 +594,40 @@ def main():
             print(f"bench: CUDA graph capture failed ({exc!r}); timing the eager step", file=sys.stderr)
             graphs = None
 
+    # Every step is run `replays` times in a row, so that the timed region lasts half a second or more whatever
+    # --steps says (the clock sampler then sees it, and the figure does not depend on the run's length); ms_per_step
+    # stays the time of ONE pass.  All ranks use the same count.
+    replays = 1
+    if graphs is not None:
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        for k in range(ROT):
+            graphs[k].replay()
+        p1.record(stream)
+        p1.synchronize()
+        est_ms = max_over_ranks(p0.elapsed_time(p1), dev) / ROT
+        replays = max(1, int(-(-MIN_TIMED_MS // (est_ms * args.steps))))
     sampler = ClockSampler(local_rank)
     fence()
     sampler.start()
+    time.sleep(0.25)            # the sampler's first line takes this long to come
     launches0 = z.launch_count()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record(stream)
     for i in range(args.steps):
         if graphs is not None:
-            graphs[(args.warmup + i) % ROT].replay()
+            for _ in range(replays):
+                graphs[(args.warmup + i) % ROT].replay()
         else:
             step(args.warmup + i)
     t_end.record(stream)
     fence()
-    launches = (launches_per_step * args.steps) if graphs is not None else (z.launch_count() - launches0)
+    launches = (launches_per_step * args.steps * replays) if graphs is not None else (z.launch_count() - launches0)
     clocks = sampler.stop()
     ctx.check()
     ms_total = max_over_ranks(t_begin.elapsed_time(t_end), dev)
-    ms_step = ms_total / args.steps
+    ms_step = ms_total / (args.steps * replays)
     units = step_units_bytes()
     total_bytes = sum(units.values())
     value = whole_job_gbs(total_bytes, world, ms_step)
@@ -549,9 +647,10 @@ def main():
     op_ms = {nm: statistics.mean(evs[i][j].elapsed_time(evs[i][j + 1]) for i in range(args.steps))
              for j, nm in enumerate(names)}
 
-    # ---- roofline of the dominant kernel.  decompress and the fused hop are exactly one kernel launch per call,
-    # so their event brackets time that kernel alone; compress under a relative bound also holds the range pass,
-    # so the encoder kernel is additionally timed alone with the pre-resolved absolute bound.
+    # ---- roofline of the codec's three calls, each timed by itself: back-to-back calls replayed from a CUDA graph over
+    # the rotating buffer sets, at least 200 of them and at least 0.4 s, inside one pair of events, with the SM clock
+    # sampled meanwhile.  compress is timed with the pre-resolved absolute bound (a relative bound adds the range pass):
+    # two launches (rounds into slots, then placement); decompress is one launch; the fused hop two (hop, placement).
     peaks = {}
     pk = ROOT / "MEASURED_PEAKS.json"
     peak_src = "fallback"
@@ -563,28 +662,30 @@ def main():
         except Exception:
             pass
     eb_abs = float(np.float32(REL) * (np.float32(x_h.max()) - np.float32(x_h.min())))
-    enc_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for i in range(args.steps):
-        k = i % ROT
-        enc_ev[i][0].record(stream)
-        ctx.compress(xs[k], z.EB_ABS, eb_abs, cs[k], nb1)
-        enc_ev[i][1].record(stream)
+    for k in range(ROT):                       # the streams the decoder and the hop read
+        ctx.compress(xs[k], z.EB_REL, REL, cs[k], nb1)
     torch.cuda.synchronize()
-    enc_ms = statistics.mean(a.elapsed_time(b) for a, b in enc_ev)
+    enc_us, enc_calls, enc_mhz = _timed_long(lambda k: ctx.compress(xs[k], z.EB_ABS, eb_abs, c2s[k], nb2), ROT, local_rank)
+    dec_us, dec_calls, dec_mhz = _timed_long(lambda k: ctx.decompress(cs[k], ys[k]), ROT, local_rank)
+    hop_us, hop_calls, hop_mhz = _timed_long(
+        lambda k: ctx.decompress_reduce_compress(cs[k], N_ELEMS, c2s[k], nb2, local=locs[k]), ROT, local_rank)
+    ctx.check()
     in_b = 4 * N_ELEMS
     c1_b = in_b / ratio1
     c2_b = in_b / ratio2
     kern = {
-        "encode(compress, ABS bound)": {"ms": enc_ms, "bytes": in_b + c1_b},
-        "decode(decompress)": {"ms": op_ms["decompress"], "bytes": c1_b + in_b},
-        "encode_fused(decompress-add-recompress)": {"ms": op_ms["fused"], "bytes": c1_b + in_b + c2_b},
+        "encode(compress, ABS bound): encode_rounds + place": {"ms": enc_us * 1e-3, "bytes": in_b + c1_b, "calls": enc_calls, "sm_mhz": enc_mhz},
+        "decode(decompress): decode_tiles": {"ms": dec_us * 1e-3, "bytes": c1_b + in_b, "calls": dec_calls, "sm_mhz": dec_mhz},
+        "encode_fused(decompress-add-recompress): hop_tiles + place": {"ms": hop_us * 1e-3, "bytes": c1_b + in_b + c2_b, "calls": hop_calls,
+                                                                     "sm_mhz": hop_mhz},
     }
     for v in kern.values():
         v["achieved_gbs"] = v["bytes"] / (v["ms"] * 1e-3) / 1e9
         v["frac"] = v["achieved_gbs"] / peak
         v["uncompressed_gbs"] = in_b / (v["ms"] * 1e-3) / 1e9
+        v["us_x_mhz"] = v["ms"] * 1e3 * v["sm_mhz"] if v["sm_mhz"] else None   # clock-independent cost: cycles per call
     # the fused kernel also runs the 56 chunk hops of the allreduce: it carries the largest share of the step
-    dom = "encode_fused(decompress-add-recompress)"
+    dom = "encode_fused(decompress-add-recompress): hop_tiles + place"
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["achieved_gbs"], "peak": peak, "unit": "GB/s",
                 "frac": kern[dom]["frac"], "traffic": None, "peak_source": f"of {peak_src}",
                 "algorithmic_bytes_per_launch": kern[dom]["bytes"]}
@@ -596,14 +697,9 @@ def main():
     for k in range(ROT):
         ctx.compress(xs[k], z.EB_REL, REL, cs[k], nb1)
         ctx.decompress(cs[k], ys[k])
-    q_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for i in range(args.steps):
-        k = (i + 1) % ROT if i + 1 < args.steps else 0   # the last launch looks at the batch the ratios are quoted on
-        q_ev[i][0].record(stream)
-        ctx.quality(xs[k], ys[k], qout)
-        q_ev[i][1].record(stream)
+    q_us, q_calls, q_mhz = _timed_long(lambda k: ctx.quality(xs[k], ys[k], qout), ROT, local_rank)
+    ctx.quality(xs[0], ys[0], qout)   # the batch the ratios are quoted on
     torch.cuda.synchronize()
-    q_ms = statistics.mean(a.elapsed_time(b) for a, b in q_ev)
     qv = qout.cpu().numpy()
     hist = torch.zeros(33, dtype=torch.int64, device=dev)
     ctx.stream_stats(cs[0], hist)     # the stream of the batch the ratios are quoted on (length from its header)
@@ -612,7 +708,8 @@ def main():
     quality = {"max_abs_err": float(qv[0]), "nrmse": float(qv[2]), "psnr_db": float(qv[3]), "bit_rate": 32.0 / ratio1,
                "eb_abs": eb_abs, "constant_block_pct": 100.0 * hh[0] / max(hh[32], 1.0),
                "mean_code_length": float((hh[:32] * np.arange(32)).sum() / max(hh[32], 1.0))}
-    kern["quality(metrics)"] = {"ms": q_ms, "bytes": 2.0 * in_b}
+    kern["quality(metrics)"] = {"ms": q_us * 1e-3, "bytes": 2.0 * in_b, "calls": q_calls, "sm_mhz": q_mhz,
+                                "us_x_mhz": q_us * q_mhz if q_mhz else None}
     kq = kern["quality(metrics)"]
     kq["achieved_gbs"] = kq["bytes"] / (kq["ms"] * 1e-3) / 1e9
     kq["frac"] = kq["achieved_gbs"] / peak
@@ -640,6 +737,15 @@ def main():
            "what": "zccl_compress_host + zccl_decompress_host of the 64 MiB batch (uncompressed bytes per op / time)",
            "ms_per_step": e2e_ms, "h2d_bytes_per_step": in_b + nb, "d2h_bytes_per_step": nb + 8 + in_b}
 
+    # ---- the other configurations of the workload list, a few graph replays each (single-GPU runs only)
+    configs = None
+    if rank == 0 and world == 1 and not args.no_configs:
+        ctx.close()
+        ctx = None
+        del xs, locs, cs, c2s, ys, ars, ags
+        torch.cuda.empty_cache()
+        configs = other_configs(z, peak, x_h, loc_h)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
@@ -659,14 +765,17 @@ def main():
             "config": {"workload": WORKLOAD, "l2": f"inputs and outputs rotate over {ROT} buffer sets, each above L2",
                        "rel_bound": REL, "ratio_compress": ratio1, "ratio_fused_out": ratio2,
                        "parallelism": f"{world} independent replicas" if world > 1 else "single GPU",
-                       "launch": "CUDA graph replay, one graph per buffer set" if graphs is not None else "eager"},
+                       "launch": "CUDA graph replay, one graph per buffer set" if graphs is not None else "eager",
+                       "timed_region_ms": ms_total},
+            "replays_per_step": replays,
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu,
             "ms_per_step_eager": ms_step_eager, "ops_ms": op_ms, "ops_uncompressed_gbs": {nm: units[nm] / (op_ms[nm] * 1e-3) / 1e9 for nm in names},
-            "kernels": kern, "quality": quality,
+            "kernels": kern, "quality": quality, "configs": configs,
         }
         print(json.dumps(line))
-    ctx.close()
+    if ctx is not None:
+        ctx.close()
     if world > 1:
         dist.destroy_process_group()
 
