@@ -69,20 +69,28 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane)
 // number N * h + i sits in bits [N h, N h + N).  Afterwards word k holds plane k: bit N * h + i = bit k of that value.
 // Each stage exchanges, between words i and i + d, the bits whose in-value position has bit d set against those that
 // have it clear: two shifts and two bit-selects per pair.  The transpose is its own inverse.
+// (The stages are separate instantiations rather than a loop over d: left to the unroller, the 16-word form kept its
+// words in local memory, indexed at run time.)
+template <int N, int D>
+__device__ __forceinline__ void bit_transpose_stage(uint32_t (&w)[N])
+{
+    constexpr uint32_t m = D == 16 ? 0x0000FFFFu : D == 8 ? 0x00FF00FFu : D == 4 ? 0x0F0F0F0Fu : D == 2 ? 0x33333333u : 0x55555555u;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        if (i & D) continue;
+        const uint32_t a = w[i], b = w[i + D];
+        w[i] = (a & m) | ((b << D) & ~m);
+        w[i + D] = ((a >> D) & m) | (b & ~m);
+    }
+}
 template <int N>
 __device__ __forceinline__ void bit_transpose(uint32_t (&w)[N])
 {
-#pragma unroll
-    for (int d = N / 2; d >= 1; d >>= 1) {
-        const uint32_t m = d == 16 ? 0x0000FFFFu : d == 8 ? 0x00FF00FFu : d == 4 ? 0x0F0F0F0Fu : d == 2 ? 0x33333333u : 0x55555555u;
-#pragma unroll
-        for (int i = 0; i < N; ++i) {
-            if (i & d) continue;
-            const uint32_t a = w[i], b = w[i + d];
-            w[i] = (a & m) | ((b << d) & ~m);
-            w[i + d] = ((a >> d) & m) | (b & ~m);
-        }
-    }
+    if constexpr (N >= 32) bit_transpose_stage<N, 16>(w);
+    if constexpr (N >= 16) bit_transpose_stage<N, 8>(w);
+    bit_transpose_stage<N, 4>(w);
+    bit_transpose_stage<N, 2>(w);
+    bit_transpose_stage<N, 1>(w);
 }
 
 // ------------------------------------------------------------------------------------------------ stages
@@ -200,53 +208,33 @@ struct EncodeCarry {
 // codes for which fp32 is not exact) and the whole tile has to take the general route, 2 when the blob would
 // outgrow `pay_cap` payload words.  `mid` is called once, by all lanes, when the rows have been read and the sizes are
 // known, before anything is stored.
-template <class Mid>
-__device__ __forceinline__ int encode_round(const char* row, uint32_t sw, float xprev, float r, bool active, uint32_t block_in_tile,
-                                            uint32_t lbytes, uint32_t* __restrict__ blob, uint32_t org, int sgn, uint32_t pay_base,
-                                            uint32_t pay_cap, EncodeCarry& cy, int lane, uint32_t& status, Mid&& mid)
+// This is one width class (N = 8 or 16 bits per packed magnitude); it returns 3, with nothing stored and `mid` not
+// called, when a lane's code is longer than N.
+template <int N, class Mid>
+__device__ __forceinline__ int encode_round_n(const char* row, uint32_t sw, float xprev, float r, bool active, uint32_t block_in_tile,
+                                              uint32_t lbytes, uint32_t* __restrict__ blob, uint32_t org, int sgn, uint32_t pay_base,
+                                              uint32_t pay_cap, EncodeCarry& cy, int lane, uint32_t& status, Mid&& mid)
 {
-    BlockPack<8> a;
-    BlockPack<16> h;
-    uint32_t L = 0, sign = 0;
-    float guard = 0.0f;
-    bool need16 = cy.wide;   // uniform over the warp
-    if (!need16) {
-        block_pass<8>(row, sw, xprev, r, a);
-        L = code_length(a.orb);
-        sign = a.sign;
-        guard = a.guard;
-        need16 = L > 8u;     // only these lanes run the second pass
-    }
-    if (need16) {
-        block_pass<16>(row, sw, xprev, r, h);
-        L = code_length(h.orb);
-        sign = h.sign;
-        guard = h.guard;
-    }
-    if (!active) L = 0;
-    const bool beyond = !(guard < kGuardExact) || L > 16u;
+    BlockPack<N> a;
+    block_pass<N>(row, sw, xprev, r, a);
+    uint32_t L = active ? code_length(a.orb) : 0u;
+    if (N == 8 && __any_sync(kFull, L > 8u)) return 3;
+    const bool beyond = !(a.guard < kGuardExact) || L > 16u;
     const uint32_t nw = L ? L + 1u : 0u;
     const uint32_t incl = warp_incl_scan(nw, lane);
     const uint32_t round_total = __shfl_sync(kFull, incl, 31);
-    mid();   // the caller's business between the two halves (all lanes, once per call)
+    mid();   // the caller's business between the two halves (all lanes, once per round)
     if (__any_sync(kFull, beyond)) return 1;
     if (cy.pay_used + round_total > pay_cap) return 2;
-    if (guard >= kGuardSmall && block_tmax(row, sw, r) > 32768.5f) status |= kStPrecision;
+    if (a.guard >= kGuardSmall && block_tmax(row, sw, r) > 32768.5f) status |= kStPrecision;
     __syncwarp();   // every lane has read its row for the last time: the blob may lie over the stage
     if (L) {
         uint32_t* dst = blob + ((int)org + sgn * (int)(pay_base + cy.pay_used + (incl - nw)));
-        dst[0] = sign;
-        if (!cy.wide && L <= 8u) {
-            bit_transpose<8>(a.w);
+        dst[0] = a.sign;
+        bit_transpose<N>(a.w);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-                if ((uint32_t)k < L) dst[sgn * (1 + k)] = a.w[k];
-        } else {
-            bit_transpose<16>(h.w);
-#pragma unroll
-            for (int k = 0; k < 16; ++k)
-                if ((uint32_t)k < L) dst[sgn * (1 + k)] = h.w[k];
-        }
+        for (int k = 0; k < N; ++k)
+            if ((uint32_t)k < L) dst[sgn * (1 + k)] = a.w[k];
     }
     if (block_in_tile < lbytes) {
         const uint32_t wi = 1u + (block_in_tile >> 2);
@@ -255,6 +243,21 @@ __device__ __forceinline__ int encode_round(const char* row, uint32_t sw, float 
     cy.pay_used += round_total;
     cy.wide = __any_sync(kFull, L > 8u);
     return 0;
+}
+
+// One width class for the whole warp: a pass at 8 bits first unless the round before was wide; if any lane then has a
+// longer code, every lane repeats the pass at 16 bits (the warp would execute those instructions anyway, and with
+// one class at a time only one set of packed words is alive).
+template <class Mid>
+__device__ __forceinline__ int encode_round(const char* row, uint32_t sw, float xprev, float r, bool active, uint32_t block_in_tile,
+                                            uint32_t lbytes, uint32_t* __restrict__ blob, uint32_t org, int sgn, uint32_t pay_base,
+                                            uint32_t pay_cap, EncodeCarry& cy, int lane, uint32_t& status, Mid&& mid)
+{
+    if (!cy.wide) {
+        const int rc = encode_round_n<8>(row, sw, xprev, r, active, block_in_tile, lbytes, blob, org, sgn, pay_base, pay_cap, cy, lane, status, mid);
+        if (rc != 3) return rc;
+    }
+    return encode_round_n<16>(row, sw, xprev, r, active, block_in_tile, lbytes, blob, org, sgn, pay_base, pay_cap, cy, lane, status, mid);
 }
 
 // ---- general route: any code length, any alignment, codes up to 2^30, blobs of any size; straight from and to
@@ -1374,6 +1377,45 @@ __device__ __noinline__ void store_round_ragged(float* __restrict__ y, const flo
 // One round of a tile whose codes are exact in fp32: blocks 32 rd + lane.  Arguments as for decode_round_general;
 // MODE as for expand_block.  The lanes of a warp mostly share one width class; a round with a code length above 16
 // takes the general route.
+template <int N, int MODE>
+__device__ __forceinline__ void decode_round_n(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t& pay_off, int32_t& code, float s,
+                                               float* stage, int lane, const float* loc_stage)
+{
+    const uint32_t bi = 32u * rd + (uint32_t)lane;
+    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
+    const uint32_t nw = L ? L + 1u : 0u;
+    const uint32_t incl = warp_incl_scan(nw, lane);
+    const uint32_t* pay = blob + 1 + padw + pay_off + (incl - nw);
+    pay_off += __shfl_sync(kFull, incl, 31);
+    char* row = reinterpret_cast<char*>(stage) + 128 * lane;
+    const char* loc = reinterpret_cast<const char*>(loc_stage) + 128 * lane;
+    const uint32_t sw = ((uint32_t)lane & 7u) << 4;
+    // The block's sum of deltas first, so that the scan over the lanes gives the code in front of every block before
+    // any element is expanded.
+    uint32_t sign;
+    uint32_t w[N];
+    const int32_t total = load_planes<N>(pay, L, sign, w);
+    int32_t inc = total;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int32_t v = __shfl_up_sync(kFull, inc, d);
+        if (lane >= d) inc += v;
+    }
+    bit_transpose<N>(w);
+    expand_block<N, MODE>(w, sign, code + inc - total, s, row, sw, loc);
+    code += __shfl_sync(kFull, inc, 31);
+}
+// The width class of round rd of a tile, the same for all lanes: 8, 16, or 0 when a code length above 16 sends the
+// round down the general route.
+__device__ __forceinline__ int round_class(const uint32_t* blob, uint32_t nb, uint32_t rd, int lane)
+{
+    const uint32_t bi = 32u * rd + (uint32_t)lane;
+    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
+    if (__any_sync(kFull, L > 16u)) return 0;
+    return __any_sync(kFull, L > 8u) ? 16 : 8;
+}
+// The decoder's own form: one function with both classes (measured faster there than the two instantiations above
+// behind a dispatch, which the hop uses out of line to keep its register count down).
 template <int MODE>
 __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t& pay_off, int32_t& code, float s,
                                              float* stage, int lane, const float* loc_stage = nullptr)
@@ -1391,8 +1433,6 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
     char* row = reinterpret_cast<char*>(stage) + 128 * lane;
     const char* loc = reinterpret_cast<const char*>(loc_stage) + 128 * lane;
     const uint32_t sw = ((uint32_t)lane & 7u) << 4;
-    // The block's sum of deltas first, so that the scan over the lanes gives the code in front of every block before
-    // any element is expanded.
     uint32_t sign;
     int32_t total;
     if (!__any_sync(kFull, L > 8u)) {
@@ -1552,17 +1592,28 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
 
 // Out-of-line copies for the hop, whose kernel holds a decoder and an encoder: inlined, the compiler multiplied their
 // code along the kernel's branches until instruction fetch bounded it (four times the size, 15 % slower).
-template <int MODE>
+template <int N, int MODE>
 __device__ __noinline__ void decode_round_call(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t* pay_off, int32_t* code, float s,
                                                float* stage, int lane, const float* loc_stage)
 {
-    decode_round<MODE>(blob, padw, nb, rd, *pay_off, *code, s, stage, lane, loc_stage);
+    decode_round_n<N, MODE>(blob, padw, nb, rd, *pay_off, *code, s, stage, lane, loc_stage);
 }
+// the round by its width class (MODE as for expand_block); op: the reduce operation, for the general route
+template <int MODE>
+__device__ __forceinline__ void decode_round_classes(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t* pay_off, int32_t* code,
+                                                     float s, float* stage, int lane, const float* loc_stage, uint32_t op)
+{
+    const int cls = round_class(blob, nb, rd, lane);
+    if (cls == 8) decode_round_call<8, MODE>(blob, padw, nb, rd, pay_off, code, s, stage, lane, loc_stage);
+    else if (cls == 16) decode_round_call<16, MODE>(blob, padw, nb, rd, pay_off, code, s, stage, lane, loc_stage);
+    else decode_round_general(blob, padw, nb, rd, pay_off, code, s, stage, lane, loc_stage, op);
+}
+template <int N>
 __device__ __noinline__ int encode_round_call(const char* row, uint32_t sw, float xprev, float r, bool active, uint32_t* buf, EncodeCarry* cy, int lane,
                                               uint32_t* status)
 {
     // laid out like a tile's blob whose word 0 sits in front of the buffer: code-length bytes at words 1.., payload at word 9
-    return encode_round(row, sw, xprev, r, active, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, *cy, lane, *status, [] {});
+    return encode_round_n<N>(row, sw, xprev, r, active, (uint32_t)lane, 32u, buf - 1, 0u, 1, 9u, (uint32_t)kRoundBufWords - 8u, *cy, lane, *status, [] {});
 }
 
 // Advances (pay_off, code) over round e of a tile without expanding it: the blocks' sizes from their code lengths,
@@ -1807,11 +1858,11 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
             } else {
                 arrive_loc(pl);
                 if (blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
-                    if (mode2 == 1) decode_round_call<0>(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr);
+                    if (mode2 == 1) decode_round_classes<0>(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr, 0u);
                     else decode_round_general(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr, 0u);
                     __syncwarp();
                 }
-                if (mode1 == 1 && summing) decode_round_call<1>(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc);
+                if (mode1 == 1 && summing) decode_round_classes<1>(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc, op);
                 else decode_round_general(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc, op);
                 release_other();
                 if (rd + 1 < rd_stop) request_loc(jcur, tile, rd + 1, pl ^ 1u);
@@ -1843,7 +1894,9 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
                 uint32_t* buf = reinterpret_cast<uint32_t*>(loc);   // in place: a round's code never outgrows its 4 KiB
                 cy.pay_used = 0;
                 const uint32_t bi = 32u * rd + (uint32_t)lane;
-                const int rc = encode_round_call(row, sw, xprev, r, bi < nb, buf, &cy, lane, &status);
+                int rc = 3;
+                if (!cy.wide) rc = encode_round_call<8>(row, sw, xprev, r, bi < nb, buf, &cy, lane, &status);
+                if (rc == 3) rc = encode_round_call<16>(row, sw, xprev, r, bi < nb, buf, &cy, lane, &status);
                 const uint32_t gslot = (cj_begin_of(jb, jcur) >> 5) + (uint32_t)jcur + (tile >> 5);
                 if (rc == 0) {
                     __syncwarp();   // the buffer's words, written by all lanes, are visible to lane 0's store
