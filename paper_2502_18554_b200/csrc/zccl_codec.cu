@@ -1309,11 +1309,9 @@ struct BlobRef {
 // operation.  blob: the tile's words (shared or global memory); pay_off: payload words of the rounds before; code:
 // the code in front of the round; loc_stage: the stage with the operand's round, or nullptr.  Leaves the values in
 // `stage`.  Compact rather than fast: the rounds that come here are rare.
-__device__ __noinline__ void decode_round_general(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t* pay_off_io, int32_t* code_io,
+__device__ __noinline__ void decode_round_general(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t* pay_off_io, int32_t* code_io,
                                                   float s, float* stage, int lane, const float* loc_stage, uint32_t op)
 {
-    const uint32_t bi = 32u * rd + (uint32_t)lane;
-    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
     const uint32_t nw = L ? L + 1u : 0u;
     const uint32_t incl = warp_incl_scan(nw, lane);
     const uint32_t* pay = blob + 1 + padw + *pay_off_io + (incl - nw);
@@ -1348,7 +1346,55 @@ __device__ __noinline__ void decode_round_general(const uint32_t* blob, uint32_t
     }
 }
 
-constexpr int kDecBlobWords = 1024 + 8;   // staged blobs: up to 4 KiB plus the slack of the 16-byte-aligned cover
+constexpr int kDecBlobWords = 1024 + 8;   // blob buffers: a window of 4 KiB plus the slack of the 16-byte-aligned cover
+
+// The code lengths of a lane's four blocks of a tile (blocks lane, 32 + lane, 64 + lane, 96 + lane), one per byte, from
+// the head of the tile's blob: kept in a register, because the window over a large blob moves away from its head.
+__device__ __forceinline__ uint32_t lane_code_lengths(const uint32_t* blob, uint32_t nb, int lane)
+{
+    const unsigned char* lb = reinterpret_cast<const unsigned char*>(blob + 1);
+    uint32_t lp = 0;
+#pragma unroll
+    for (uint32_t e = 0; e < (uint32_t)kRoundsPerTile; ++e) {
+        const uint32_t bi = 32u * e + (uint32_t)lane;
+        if (bi < nb) lp |= (uint32_t)lb[bi] << (8u * e);
+    }
+    return lp;
+}
+
+// The window a warp has over its current tile's blob: words [0, end) of the blob can be read at base[word].  A blob
+// that a bulk copy can bring (BlobRef::staged) is staged a window at a time: first its front, and when a round reaches
+// past the window's end, the window moves to that round's first word.  Other blobs are read where they are.
+struct BlobWindow {
+    const uint32_t* base;
+    uint32_t end;
+};
+// How much of a blob the copy that brings words [first, ...) covers: bytes to copy from the 16-byte boundary at or
+// below that word (at most a buffer's worth, at most to the 16-byte boundary at or above the blob's end).
+__device__ __forceinline__ uint32_t window_bytes(const BlobRef& br, uint32_t first)
+{
+    const uintptr_t g = (uintptr_t)(br.ptr + first), e = (uintptr_t)(br.ptr + br.words);
+    const uintptr_t a_beg = g & ~(uintptr_t)15, a_end = (e + 15) & ~(uintptr_t)15;
+    const uintptr_t bytes = a_end - a_beg;
+    return (uint32_t)(bytes < (uintptr_t)(kDecBlobWords * 4) ? bytes : (uintptr_t)(kDecBlobWords * 4));
+}
+// The window after that copy has landed in `buf`.
+__device__ __forceinline__ BlobWindow window_at(const BlobRef& br, uint32_t first, const uint32_t* buf)
+{
+    const uint32_t lead = (uint32_t)(((uintptr_t)(br.ptr + first)) & 15u) >> 2;   // words between the boundary and the first word
+    BlobWindow w;
+    w.base = buf + lead - first;
+    const uint32_t got = first + (window_bytes(br, first) >> 2) - lead;
+    w.end = got < br.words ? got : br.words;
+    return w;
+}
+// Issues the copy (one lane).
+__device__ __forceinline__ void window_request(const BlobRef& br, uint32_t first, uint32_t* buf, unsigned long long* bar)
+{
+    const uint32_t bytes = window_bytes(br, first);
+    mbar_expect_tx(bar, bytes);
+    bulk_load(buf, (const void*)(((uintptr_t)(br.ptr + first)) & ~(uintptr_t)15), bytes, bar);
+}
 struct alignas(1024) DecWarpShared {
     float out[2][kRound];                  // each on a 1024-byte boundary
     alignas(16) uint32_t blob[2][kDecBlobWords];
@@ -1378,11 +1424,9 @@ __device__ __noinline__ void store_round_ragged(float* __restrict__ y, const flo
 // MODE as for expand_block.  The lanes of a warp mostly share one width class; a round with a code length above 16
 // takes the general route.
 template <int N, int MODE>
-__device__ __forceinline__ void decode_round_n(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t& pay_off, int32_t& code, float s,
+__device__ __forceinline__ void decode_round_n(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t& pay_off, int32_t& code, float s,
                                                float* stage, int lane, const float* loc_stage)
 {
-    const uint32_t bi = 32u * rd + (uint32_t)lane;
-    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
     const uint32_t nw = L ? L + 1u : 0u;
     const uint32_t incl = warp_incl_scan(nw, lane);
     const uint32_t* pay = blob + 1 + padw + pay_off + (incl - nw);
@@ -1407,23 +1451,19 @@ __device__ __forceinline__ void decode_round_n(const uint32_t* blob, uint32_t pa
 }
 // The width class of round rd of a tile, the same for all lanes: 8, 16, or 0 when a code length above 16 sends the
 // round down the general route.
-__device__ __forceinline__ int round_class(const uint32_t* blob, uint32_t nb, uint32_t rd, int lane)
+__device__ __forceinline__ int round_class(uint32_t L)
 {
-    const uint32_t bi = 32u * rd + (uint32_t)lane;
-    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
     if (__any_sync(kFull, L > 16u)) return 0;
     return __any_sync(kFull, L > 8u) ? 16 : 8;
 }
 // The decoder's own form: one function with both classes (measured faster there than the two instantiations above
 // behind a dispatch, which the hop uses out of line to keep its register count down).
 template <int MODE>
-__device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t& pay_off, int32_t& code, float s,
+__device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t& pay_off, int32_t& code, float s,
                                              float* stage, int lane, const float* loc_stage = nullptr)
 {
-    const uint32_t bi = 32u * rd + (uint32_t)lane;
-    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
     if (__any_sync(kFull, L > 16u)) {
-        decode_round_general(blob, padw, nb, rd, &pay_off, &code, s, stage, lane, loc_stage, 0u);
+        decode_round_general(blob, padw, L, &pay_off, &code, s, stage, lane, loc_stage, 0u);
         return;
     }
     const uint32_t nw = L ? L + 1u : 0u;
@@ -1508,13 +1548,9 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
         if (w_end <= w_beg || (blob0 + w_end) * 4ull > q.in_cap) { br.words = 0xFFFFFFFFu; return br; }   // marks a damaged index
         br.ptr = q.in_c + blob0 + w_beg;
         br.words = w_end - w_beg;
-        const uintptr_t b = (uintptr_t)br.ptr, e = (uintptr_t)(br.ptr + br.words);
-        const uintptr_t a_beg = b & ~(uintptr_t)15, a_end = (e + 15) & ~(uintptr_t)15;
-        if (a_end - a_beg <= (uintptr_t)(kDecBlobWords * 4) && a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {
-            if (lane == 0) {
-                mbar_expect_tx(&sh.bar[buf], (uint32_t)(a_end - a_beg));
-                bulk_load(sh.blob[buf], (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar[buf]);
-            }
+        const uintptr_t a_end = ((uintptr_t)(br.ptr + br.words) + 15) & ~(uintptr_t)15;
+        if (a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {   // the copies may read up to the boundary behind the blob
+            if (lane == 0) window_request(br, 0, sh.blob[buf], &sh.bar[buf]);
             br.staged = true;
         }
         return br;
@@ -1547,22 +1583,35 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
             const unsigned long long start = (unsigned long long)tile * kTile;
             const uint32_t len = (uint32_t)((hc.n - start < (unsigned long long)kTile) ? (hc.n - start) : kTile);
             const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2;
-            const uint32_t* blob = cur.staged ? sh.blob[p] + ((((uintptr_t)cur.ptr) & 15u) >> 2) : cur.ptr;
-            const int mode = describe_blob(blob, cur.words, nb, lane);
+            BlobWindow win;
+            win.base = cur.ptr; win.end = cur.words;
+            if (cur.staged) win = window_at(cur, 0, sh.blob[p]);
+            const int mode = describe_blob(win.base, cur.words, nb, lane);   // the head (at most 33 words) is in every first window
             if (mode == 0) status |= kStBadStream;
             else {
                 float* __restrict__ y = job.y + start;
                 const bool mapped = (((uintptr_t)job.y) & 15u) == 0;
                 uint32_t pay_off = 0;
-                int32_t code = (int32_t)blob[0];
+                int32_t code = (int32_t)win.base[0];
+                const uint32_t lp = lane_code_lengths(win.base, nb, lane);
                 const uint32_t rounds = (nb + 31) >> 5;
                 for (uint32_t rd = 0; rd < rounds; ++rd) {
+                    const uint32_t L = (lp >> (8u * rd)) & 0xFFu;
+                    const uint32_t first = 1u + padw + pay_off, beyond = first + __reduce_add_sync(kFull, L ? L + 1u : 0u);
+                    if (beyond > win.end) {   // the round reaches past the window (describe_blob has checked it against the blob)
+                        __syncwarp();         // every lane is done with the window as it is
+                        if (lane == 0) window_request(cur, first, sh.blob[p], &sh.bar[p]);
+                        if (!mbar_wait(&sh.bar[p], (p ? fills1 : fills0) & 1u)) status |= kStTimeout;
+                        if (p) ++fills1; else ++fills0;
+                        win = window_at(cur, first, sh.blob[p]);
+                    }
+                    const uint32_t* blob = win.base;
                     // the stage about to be written was handed to a tensor store two rounds ago
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                     float* stage = sh.out[so];
-                    if (mode == 1) decode_round<0>(blob, padw, nb, rd, pay_off, code, hc.s, stage, lane);
-                    else decode_round_general(blob, padw, nb, rd, &pay_off, &code, hc.s, stage, lane, nullptr, 0u);
+                    if (mode == 1) decode_round<0>(blob, padw, L, pay_off, code, hc.s, stage, lane);
+                    else decode_round_general(blob, padw, L, &pay_off, &code, hc.s, stage, lane, nullptr, 0u);
                     __syncwarp();   // the stage's rows, written by all lanes, are visible
                     const uint32_t e0 = rd * (uint32_t)kRound;
                     if (mapped && e0 + (uint32_t)kRound <= len) {
@@ -1593,20 +1642,20 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
 // Out-of-line copies for the hop, whose kernel holds a decoder and an encoder: inlined, the compiler multiplied their
 // code along the kernel's branches until instruction fetch bounded it (four times the size, 15 % slower).
 template <int N, int MODE>
-__device__ __noinline__ void decode_round_call(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t* pay_off, int32_t* code, float s,
+__device__ __noinline__ void decode_round_call(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t* pay_off, int32_t* code, float s,
                                                float* stage, int lane, const float* loc_stage)
 {
-    decode_round_n<N, MODE>(blob, padw, nb, rd, *pay_off, *code, s, stage, lane, loc_stage);
+    decode_round_n<N, MODE>(blob, padw, L, *pay_off, *code, s, stage, lane, loc_stage);
 }
 // the round by its width class (MODE as for expand_block); op: the reduce operation, for the general route
 template <int MODE>
-__device__ __forceinline__ void decode_round_classes(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t rd, uint32_t* pay_off, int32_t* code,
+__device__ __forceinline__ void decode_round_classes(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t* pay_off, int32_t* code,
                                                      float s, float* stage, int lane, const float* loc_stage, uint32_t op)
 {
-    const int cls = round_class(blob, nb, rd, lane);
-    if (cls == 8) decode_round_call<8, MODE>(blob, padw, nb, rd, pay_off, code, s, stage, lane, loc_stage);
-    else if (cls == 16) decode_round_call<16, MODE>(blob, padw, nb, rd, pay_off, code, s, stage, lane, loc_stage);
-    else decode_round_general(blob, padw, nb, rd, pay_off, code, s, stage, lane, loc_stage, op);
+    const int cls = round_class(L);
+    if (cls == 8) decode_round_call<8, MODE>(blob, padw, L, pay_off, code, s, stage, lane, loc_stage);
+    else if (cls == 16) decode_round_call<16, MODE>(blob, padw, L, pay_off, code, s, stage, lane, loc_stage);
+    else decode_round_general(blob, padw, L, pay_off, code, s, stage, lane, loc_stage, op);
 }
 template <int N>
 __device__ __noinline__ int encode_round_call(const char* row, uint32_t sw, float xprev, float r, bool active, uint32_t* buf, EncodeCarry* cy, int lane,
@@ -1618,10 +1667,8 @@ __device__ __noinline__ int encode_round_call(const char* row, uint32_t sw, floa
 
 // Advances (pay_off, code) over round e of a tile without expanding it: the blocks' sizes from their code lengths,
 // their sums of deltas from population counts of their planes.  Lets a warp start in the middle of a tile.
-__device__ __noinline__ void skip_round(const uint32_t* blob, uint32_t padw, uint32_t nb, uint32_t e, uint32_t* pay_off, int32_t* code, int lane)
+__device__ __noinline__ void skip_round(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t* pay_off, int32_t* code, int lane)
 {
-    const uint32_t bi = 32u * e + (uint32_t)lane;
-    const uint32_t L = bi < nb ? reinterpret_cast<const unsigned char*>(blob + 1)[bi] : 0u;
     const uint32_t nw = L ? L + 1u : 0u;
     const uint32_t incl = warp_incl_scan(nw, lane);
     const uint32_t* pay = blob + 1 + padw + *pay_off + (incl - nw);
@@ -1718,13 +1765,9 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
         if (!job_ok || q.n == 0 || tile >= h1.nT) return br;
         br = blob_of(q.in_c, q.in_cap, h1.nT, tile);
         if (!br.ptr) return br;
-        const uintptr_t b = (uintptr_t)br.ptr, e = (uintptr_t)(br.ptr + br.words);
-        const uintptr_t a_beg = b & ~(uintptr_t)15, a_end = (e + 15) & ~(uintptr_t)15;
-        if (a_end - a_beg <= (uintptr_t)(kDecBlobWords * 4) && a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {
-            if (lane == 0) {
-                mbar_expect_tx(&sh.bar_blob, (uint32_t)(a_end - a_beg));
-                bulk_load(sh.blob, (const void*)a_beg, (uint32_t)(a_end - a_beg), &sh.bar_blob);
-            }
+        const uintptr_t a_end = ((uintptr_t)(br.ptr + br.words) + 15) & ~(uintptr_t)15;
+        if (a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {   // the copies may read up to the boundary behind the blob
+            if (lane == 0) window_request(br, 0, sh.blob, &sh.bar_blob);
             br.staged = true;
         }
         return br;
@@ -1794,11 +1837,15 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
         // what the two blobs say
         const uint32_t* blob1 = nullptr;
         const uint32_t* blob2 = nullptr;
+        BlobWindow win;   // over the incoming blob
+        win.base = nullptr; win.end = 0;
         int mode1 = 0, mode2 = 1;
         if (len) {
             if (cur.ptr) {
-                blob1 = cur.staged ? sh.blob + ((((uintptr_t)cur.ptr) & 15u) >> 2) : cur.ptr;
-                mode1 = describe_blob(blob1, cur.words, nb, lane);
+                win.base = cur.ptr; win.end = cur.words;
+                if (cur.staged) win = window_at(cur, 0, sh.blob);
+                blob1 = win.base;
+                mode1 = describe_blob(blob1, cur.words, nb, lane);   // the head (at most 33 words) is in every first window
             }
             if (job.in_c2) {
                 const BlobRef b2 = blob_of(job.in_c2, job.in2_cap, hc2.nT, tile);
@@ -1811,6 +1858,21 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
 
         uint32_t pay1 = 0, pay2 = 0;
         int32_t code1 = good ? (int32_t)blob1[0] : 0, code2 = (good && blob2) ? (int32_t)blob2[0] : 0;
+        const uint32_t lp1 = good ? lane_code_lengths(blob1, nb, lane) : 0u, lp2 = (good && blob2) ? lane_code_lengths(blob2, nb, lane) : 0u;
+        // moves the window over the incoming blob to round e's first word when the round reaches past its end
+        auto reach = [&](uint32_t e) {
+            const uint32_t L = (lp1 >> (8u * e)) & 0xFFu;
+            const uint32_t first = 1u + padw + pay1, beyond = first + __reduce_add_sync(kFull, L ? L + 1u : 0u);
+            if (beyond > win.end) {
+                __syncwarp();   // every lane is done with the window as it is
+                if (lane == 0) window_request(cur, first, sh.blob, &sh.bar_blob);
+                if (!mbar_wait(&sh.bar_blob, bfill & 1u)) status |= kStTimeout;
+                ++bfill;
+                win = window_at(cur, first, sh.blob);
+                blob1 = win.base;
+            }
+            return L;
+        };
         float carry_y = 0.0f;
         // The next tile's blob goes into the one blob buffer as soon as this tile's last round is decoded; that look-up
         // moves the job on, so the next tile's facts are kept from there.
@@ -1831,8 +1893,9 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
         if (good && rd_first != 0 && rd_first < rd_stop) {
             // a unit that starts inside its tile: sizes and codes of the rounds in front, and the value in front of it
             for (uint32_t e = 0; e < rd_first; ++e) {
-                skip_round(blob1, padw, nb, e, &pay1, &code1, lane);
-                if (blob2) skip_round(blob2, padw, nb, e, &pay2, &code2, lane);
+                const uint32_t Le = reach(e);
+                skip_round(blob1, padw, Le, &pay1, &code1, lane);
+                if (blob2) skip_round(blob2, padw, (lp2 >> (8u * e)) & 0xFFu, &pay2, &code2, lane);
             }
             const float xa = __fmul_rn(__int2float_rn(code1), s);
             const float xb = blob2 ? __fmul_rn(__int2float_rn(code2), s) : __ldg(job.x + start + rd_first * (uint32_t)kRound - 1u);
@@ -1858,12 +1921,14 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
             } else {
                 arrive_loc(pl);
                 if (blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
-                    if (mode2 == 1) decode_round_classes<0>(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr, 0u);
-                    else decode_round_general(blob2, padw, nb, rd, &pay2, &code2, s, loc, lane, nullptr, 0u);
+                    const uint32_t L2 = (lp2 >> (8u * rd)) & 0xFFu;
+                    if (mode2 == 1) decode_round_classes<0>(blob2, padw, L2, &pay2, &code2, s, loc, lane, nullptr, 0u);
+                    else decode_round_general(blob2, padw, L2, &pay2, &code2, s, loc, lane, nullptr, 0u);
                     __syncwarp();
                 }
-                if (mode1 == 1 && summing) decode_round_classes<1>(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc, op);
-                else decode_round_general(blob1, padw, nb, rd, &pay1, &code1, s, loc, lane, loc, op);
+                const uint32_t L1 = reach(rd);
+                if (mode1 == 1 && summing) decode_round_classes<1>(blob1, padw, L1, &pay1, &code1, s, loc, lane, loc, op);
+                else decode_round_general(blob1, padw, L1, &pay1, &code1, s, loc, lane, loc, op);
                 release_other();
                 if (rd + 1 < rd_stop) request_loc(jcur, tile, rd + 1, pl ^ 1u);
                 else {   // the blob is decoded: the next unit's may come, and its first operand round
