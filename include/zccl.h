@@ -317,6 +317,16 @@ int zccl_stream_stats(zccl_ctx* ctx, const void* in, size_t in_bytes_max, unsign
  */
 int zccl_range(zccl_ctx* ctx, const float* x, size_t n, float* minmax, void* stream);
 int zccl_resolve_range(zccl_ctx* ctx, const float* minmax, float eb_rel, float* eb_abs_out, void* stream);
+
+/*
+ * The same resolution as a pure host function (no context, no device): from the combined minimum and maximum of the
+ * data and the relative bound, eb_abs = fl32(eb_rel * fl32(mx - mn)), the quantisation step s = 2 * fl32(eb_abs *
+ * (1 - 2^-6)) and its reciprocal r = fl32(1 / s), each by one IEEE fp32 operation, as the device computes them
+ * (Section 3.2: one bound per collective).  Any of the three outputs [host] may be NULL.  Returns ZCCL_E_ARG for a
+ * bound that is not a positive finite number, ZCCL_E_DEGENERATE when mx - mn is zero, negative, infinite or not a
+ * number, or when step or reciprocal leave the finite range.
+ */
+int zccl_resolve_range_host(float mn, float mx, float eb_rel, float* eb_abs, float* step, float* reciprocal);
 int zccl_scale(zccl_ctx* ctx, float* y, size_t n, float divisor, void* stream);
 
 /*

@@ -761,6 +761,21 @@ int zccl_range(zccl_ctx* c, const float* x, size_t n, float* minmax, void* strea
     return cuda_rc(launch_range(rb, c->ws, c->sm_count, st));
 }
 
+int zccl_resolve_range_host(float mn, float mx, float eb_rel, float* eb_abs, float* step, float* reciprocal)
+{
+    if (!(eb_rel > 0.0f) || !std::isfinite(eb_rel)) return ZCCL_E_ARG;
+    volatile float range = mx - mn;            // volatile: one IEEE fp32 operation each, as on the device
+    if (!(mn <= mx) || !((float)range > 0.0f) || !std::isfinite((float)range)) return ZCCL_E_DEGENERATE;
+    volatile float ea = eb_rel * range;
+    Params p;
+    const int rc = resolve_abs_host(ea, p);
+    if (rc != ZCCL_OK) return rc;
+    if (eb_abs) *eb_abs = ea;
+    if (step) *step = p.s;
+    if (reciprocal) *reciprocal = p.r;
+    return ZCCL_OK;
+}
+
 int zccl_resolve_range(zccl_ctx* c, const float* minmax, float eb_rel, float* eb_abs_out, void* stream)
 {
     if (!c || !minmax || !(eb_rel > 0.0f) || !std::isfinite(eb_rel)) return ZCCL_E_ARG;

@@ -234,13 +234,10 @@ class Ring:
         if hasattr(self.codec, "resolve"):
             pair = torch.stack([-t[0], t[1]]).to(mm.device)   # back on the codec's device when the messages go through the host
             return self.codec.resolve(pair, float(np.float32(eb)))
-        lo, hi = np.float32(-t[0].item()), np.float32(t[1].item())
-        with np.errstate(all="ignore"):
-            rng = np.float32(hi - lo)
-            ea = np.float32(np.float32(eb) * rng)
-        if not (rng > 0) or not np.isfinite(rng) or not np.isfinite(ea) or not (ea > 0):
+        rc, ea, _, _ = z.resolve_range_host(float(-t[0].item()), float(t[1].item()), float(np.float32(eb)))
+        if rc != z.OK:
             raise DegenerateRange("relative bound over data without a finite, non-zero range")
-        return float(ea)
+        return ea
 
     # ------------------------------------------------------------------------------------------------ one message
 

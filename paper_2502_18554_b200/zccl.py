@@ -24,7 +24,7 @@ EXPORTS = [
     "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_reduce_scatter", "zccl_sim_scatter",
-    "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_resolve_range", "zccl_scale", "zccl_stream_stats",
+    "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_resolve_range", "zccl_resolve_range_host", "zccl_scale", "zccl_stream_stats",
     "zccl_compress_bound_tiled", "zccl_compress_tiled", "zccl_decompress_tiled",
     "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
     "zccl_debug_set_launch_counter",
@@ -69,6 +69,7 @@ def lib():
         L.zccl_quality.argtypes = [vp, vp, vp, sz, vp, vp]
         L.zccl_range.argtypes = [vp, vp, sz, vp, vp]
         L.zccl_resolve_range.argtypes = [vp, vp, C.c_float, vp, vp]
+        L.zccl_resolve_range_host.argtypes = [C.c_float, C.c_float, C.c_float, vp, vp, vp]
         L.zccl_stream_stats.argtypes = [vp, vp, sz, vp, vp]
         L.zccl_compress_bound_tiled.argtypes = [sz, C.c_uint]
         L.zccl_compress_bound_tiled.restype = sz
@@ -88,6 +89,14 @@ def lib():
 
 def compress_bound(n: int) -> int:
     return int(lib().zccl_compress_bound(n))
+
+
+def resolve_range_host(mn: float, mx: float, eb_rel: float) -> tuple[int, float, float, float]:
+    """zccl_resolve_range_host: (status, eb_abs, step, reciprocal) of a relative bound over [mn, mx]; a pure host
+    function (no GPU needed)."""
+    ea, s, r = C.c_float(0.0), C.c_float(0.0), C.c_float(0.0)
+    rc = int(lib().zccl_resolve_range_host(mn, mx, eb_rel, C.byref(ea), C.byref(s), C.byref(r)))
+    return rc, float(ea.value), float(s.value), float(r.value)
 
 
 def compress_bound_tiled(n: int, tile: int) -> int:

@@ -77,3 +77,30 @@ def test_compress_bound_for_other_tile_sizes_is_the_oracles():
             assert zccl.compress_bound_tiled(n, T) == oracle.compress_bound(n, T)
     assert zccl.compress_bound_tiled(1000, 5000) == 0 and zccl.compress_bound_tiled(1000, 512) == 0
     assert zccl.compress_bound_tiled(12345, 4096) == zccl.compress_bound(12345)
+
+
+def test_resolve_range_host_is_the_oracles_arithmetic(lib):
+    """The host-side resolution of a relative bound (what a ring rank without a device-side resolver calls) against
+    the oracle's, bit for bit, over ranges of many magnitudes, and its refusals."""
+    import numpy as np
+    from paper_2502_18554_b200 import zccl
+    rng = np.random.default_rng(7)
+    cases = [(-1.0, 1.0, 1e-3), (0.0, 3.0, 1e-2), (-7.25, -7.0, 1e-4), (1e-30, 2e-30, 1e-3), (-3e38, 3e38, 1e-3)]
+    for _ in range(200):
+        a, b = np.sort(rng.standard_normal(2).astype(np.float32) * np.float32(10.0 ** rng.integers(-20, 20)))
+        cases.append((float(a), float(b), float(10.0 ** rng.uniform(-6, -1))))
+    for mn, mx, eb in cases:
+        rc, ea, s, r = zccl.resolve_range_host(mn, mx, eb)
+        try:
+            want = oracle.resolve(oracle.EB_REL, eb, mn=mn, mx=mx)
+        except oracle.OracleError as exc:
+            assert rc == exc.code, (mn, mx, eb)
+            continue
+        assert rc == zccl.OK, (mn, mx, eb)
+        assert np.float32(ea).tobytes() + np.float32(s).tobytes() + np.float32(r).tobytes() == \
+            np.float32(want[0]).tobytes() + np.float32(want[1]).tobytes() + np.float32(want[2]).tobytes(), (mn, mx, eb)
+    assert zccl.resolve_range_host(2.0, 2.0, 1e-3)[0] == zccl.E_DEGENERATE
+    assert zccl.resolve_range_host(3.0, 2.0, 1e-3)[0] == zccl.E_DEGENERATE
+    assert zccl.resolve_range_host(0.0, float("inf"), 1e-3)[0] == zccl.E_DEGENERATE
+    assert zccl.resolve_range_host(0.0, 1.0, 0.0)[0] == zccl.E_ARG
+    assert zccl.resolve_range_host(0.0, 1.0, float("nan"))[0] == zccl.E_ARG
