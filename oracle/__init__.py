@@ -1,6 +1,6 @@
 """CPU oracle for the ZCCL hot path -- TEST INFRASTRUCTURE, not the product.
 
-Thin ctypes access to ``zccl_oracle.c`` (plain C, single thread).  Only tests, the smoke check and the
+Thin ctypes access to ``zccl_oracle.c`` and ``zccl_oracle_f64.c`` (plain C, single thread).  Only tests, the smoke check and the
 benchmark's CPU-baseline legs may import this package; the CUDA path never does and shares no code with it.
 """
 from __future__ import annotations
@@ -14,6 +14,7 @@ import numpy as np
 
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "zccl_oracle.c"
+_SRC_F64 = _HERE / "zccl_oracle_f64.c"
 _LIB = _HERE / "libzccl_oracle.so"
 
 OK, E_ARG, E_CAPACITY, E_RANGE, E_BAD_STREAM, E_DEGENERATE, W_PRECISION = 0, -1, -3, -4, -5, -7, 1
@@ -26,10 +27,10 @@ HEADER_BYTES = 32
 
 def build(force: bool = False) -> Path:
     """Compile the oracle with gcc (IEEE arithmetic, no contraction)."""
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < max(_SRC.stat().st_mtime, _SRC_F64.stat().st_mtime):
         tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
         subprocess.check_call(["gcc", "-O2", "-ffp-contract=off", "-fno-fast-math", "-std=c99", "-fPIC", "-shared",
-                               "-o", str(tmp), str(_SRC), "-lm"])
+                               "-o", str(tmp), str(_SRC), str(_SRC_F64), "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -65,6 +66,11 @@ def lib():
         L.zo_stream_stats.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
         L.zo_sim_scatter.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_size_t, C.c_int, C.c_float, C.c_uint32,
                                      C.c_void_p, C.c_void_p]
+        dp = C.POINTER(C.c_double)
+        L.zo_resolve_f64.argtypes = [C.c_int, C.c_double, C.c_double, C.c_double, dp, dp, dp]
+        L.zo_quantise_f64.argtypes = [C.c_void_p, C.c_size_t, C.c_double, C.c_void_p]
+        L.zo_compress_f64.argtypes = [C.c_void_p, C.c_size_t, C.c_int, C.c_double, C.c_uint32, C.c_void_p, C.c_size_t, szp]
+        L.zo_decompress_f64.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_size_t, szp]
         _lib = L
     return _lib
 
@@ -262,3 +268,54 @@ def stream_stats(stream):
     if rc != OK:
         raise OracleError(rc, "stream_stats")
     return hist
+
+
+# ------------------------------------------------------------------------------------------------ binary64 input
+
+def _f64(x) -> np.ndarray:
+    return np.ascontiguousarray(x, dtype=np.float64)
+
+
+def resolve_f64(eb_mode: int, eb: float, mn: float = 0.0, mx: float = 0.0):
+    ea, s, r = C.c_double(0.0), C.c_double(0.0), C.c_double(0.0)
+    rc = lib().zo_resolve_f64(eb_mode, eb, mn, mx, C.byref(ea), C.byref(s), C.byref(r))
+    if rc != OK:
+        raise OracleError(rc, "resolve_f64")
+    return ea.value, s.value, r.value
+
+
+def quantise_f64(x, r: float) -> np.ndarray:
+    x = _f64(x)
+    q = np.empty(x.size, np.int32)
+    rc = lib().zo_quantise_f64(_ptr(x), x.size, r, _ptr(q))
+    if rc < 0:
+        raise OracleError(rc, "quantise_f64")
+    return q
+
+
+def compress_f64(x, eb_mode: int, eb: float, T: int = DEFAULT_TILE, cap: int | None = None) -> np.ndarray:
+    """Stream bytes (uint8 array) of a binary64 array."""
+    x = _f64(x)
+    cap = compress_bound(x.size, T) if cap is None else cap
+    out = np.zeros(max(cap, 1), np.uint8)
+    nb = C.c_size_t(0)
+    rc = lib().zo_compress_f64(_ptr(x), x.size, eb_mode, eb, T, _ptr(out), cap, C.byref(nb))
+    if rc < 0:
+        raise OracleError(rc, "compress_f64")
+    return out[: nb.value].copy()
+
+
+def decompress_f64(stream, want_codes: bool = False):
+    st = np.ascontiguousarray(stream, dtype=np.uint8)
+    if st.size < HEADER_BYTES:
+        raise OracleError(E_BAD_STREAM, "decompress_f64")
+    n = stream_n(st)
+    if n > (1 << 40):
+        raise OracleError(E_BAD_STREAM, "decompress_f64")
+    y = np.empty(n, np.float64)
+    q = np.empty(n, np.int32) if want_codes else None
+    no = C.c_size_t(0)
+    rc = lib().zo_decompress_f64(_ptr(st), st.size, _ptr(y), _ptr(q) if want_codes else None, n, C.byref(no))
+    if rc != OK:
+        raise OracleError(rc, "decompress_f64")
+    return (y, q) if want_codes else y
