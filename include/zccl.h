@@ -330,6 +330,24 @@ int zccl_resolve_range_host(float mn, float mx, float eb_rel, float* eb_abs, flo
 int zccl_scale(zccl_ctx* ctx, float* y, size_t n, float divisor, void* stream);
 
 /*
+ * fZ-light for binary64 input (Section 3.3 read for double precision; the paper's data sets are single precision and
+ * it states no width).  Everything behind the quantisation is the codec above: 32-bit codes, 1-D Lorenzo deltas per
+ * 4096-element tile, code length per 32-element block, sign word and bit planes, the index at the front.
+ *   bound     eb_abs = eb (ZCCL_EB_ABS) or fl64(eb * fl64(max - min)) over the array (ZCCL_EB_REL)
+ *   step      s = 2 * fl64(eb_abs * (1 - 2^-20)), r = fl64(1 / s)
+ *   codes     q_i = nearest integer, ties to even, of fl64(x_i * r); RANGE unless every |x_i * r| < 2^30
+ *   values    x'_i = fl64((double)q_i * s); |x_i - x'_i| <= eb_abs for every code in range (no precision warning)
+ * The stream's version word carries data type 1 and header bytes 16..23 hold the step as one binary64; binary32
+ * entry points reject such a stream and the other way round (BAD_STREAM).  Plain kernels (three launches to compress,
+ * one to decompress), 8 bytes per element read or written.
+ *   x [device] n doubles, 8-byte aligned; y [device] receives n doubles; the rest as for zccl_compress / zccl_decompress.
+ * Errors as for those two; ZCCL_E_DEGENERATE at once for a relative bound with n == 0.
+ */
+int zccl_compress_f64(zccl_ctx* ctx, const double* x, size_t n, int eb_mode, double eb,
+                      void* out, size_t out_capacity, size_t* out_bytes, void* stream);
+int zccl_decompress_f64(zccl_ctx* ctx, const void* in, size_t in_bytes_max, double* y, size_t y_capacity_elems, void* stream);
+
+/*
  * Host-buffer convenience forms: copy the input from host memory into a staging area of the context, run the
  * device path, copy the result back, all enqueued on `stream` (pinned host memory makes the copies asynchronous).
  * They exist so that end-to-end cost including PCIe transfers can be measured through this boundary.

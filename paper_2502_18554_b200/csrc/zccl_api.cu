@@ -236,6 +236,8 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
         c->ws.status = sm + 3;
         c->ws.params = (Params*)(sm + 4);
         c->ws.minmax = sm + 8;
+        c->ws.params64 = (ParamsF64*)(b + off_small + 64);
+        c->ws.minmax64 = (unsigned long long*)(b + off_small + 96);
         c->ws.max_tiles = (uint32_t)max_tiles;
         c->ws.skip_publish = 0xFFFFFFFFu;
         c->sim_sizes = (size_t*)(b + off_sizes);
@@ -243,8 +245,10 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
         c->quality_partials = (double*)(b + off_quality);
         c->quality_counter = (uint32_t*)(b + off_quality + sizeof(double) * 4 * (size_t)kQualityCtas);
         const uint32_t init[3] = {1u, 0xFFFFFFFFu, 0u};   // epoch, min key, max key
+        const unsigned long long init64[2] = {0xFFFFFFFFFFFFFFFFull, 0ull};
         ok = cudaMemcpy(c->ws.epoch, &init[0], 4, cudaMemcpyHostToDevice) == cudaSuccess &&
-             cudaMemcpy(c->ws.minmax, &init[1], 8, cudaMemcpyHostToDevice) == cudaSuccess;
+             cudaMemcpy(c->ws.minmax, &init[1], 8, cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMemcpy(c->ws.minmax64, init64, 16, cudaMemcpyHostToDevice) == cudaSuccess;
     }
     if (ok) {
         const size_t off_rw = align_up(max_tiles * 4 * (size_t)kRoundSlotWords * 4, 256);
@@ -728,6 +732,42 @@ int zccl_compress_tiled(zccl_ctx* c, const float* x, size_t n, int eb_mode, floa
     if (rc != ZCCL_OK) return rc;
     return cuda_rc(launch_generic_encode(x, n, tile, hp, dev, c->gen_sizes, c->gen_sizes + c->gen_tiles, (uint32_t*)out,
                                          out_capacity, out_bytes, c->ws, c->sm_count, st));
+}
+
+int zccl_compress_f64(zccl_ctx* c, const double* x, size_t n, int eb_mode, double eb, void* out, size_t out_capacity,
+                      size_t* out_bytes, void* stream)
+{
+    if (!c || (!x && n) || !out || !out_bytes || n > c->max_elems) return ZCCL_E_ARG;
+    if ((eb_mode != ZCCL_EB_ABS && eb_mode != ZCCL_EB_REL) || !(eb > 0.0) || !std::isfinite(eb)) return ZCCL_E_ARG;
+    if (((uintptr_t)x & 7u) || ((uintptr_t)out & 3u)) return ZCCL_E_ARG;
+    const size_t nT = tiles_of(n);
+    if (nT > c->gen_tiles) return ZCCL_E_ARG;
+    if (out_capacity < kHeaderBytes + 4 * nT) return ZCCL_E_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    ParamsF64 hp{0.0, 1.0, 1.0, 1};
+    bool dev = false;
+    if (eb_mode == ZCCL_EB_REL) {
+        if (n == 0) return ZCCL_E_DEGENERATE;
+        if (launch_range_f64(x, n, eb, c->ws, c->sm_count, st) != cudaSuccess) return ZCCL_E_CUDA;
+        dev = true;
+    } else {
+        volatile double ebq = eb * (1.0 - 9.5367431640625e-07);   // 1 - 2^-20: one IEEE operation each, as on the device
+        volatile double s = ebq * 2.0;
+        if (!(s > 0.0) || !std::isfinite((double)s)) return ZCCL_E_DEGENERATE;
+        volatile double r = 1.0 / s;
+        if (!std::isfinite((double)r)) return ZCCL_E_DEGENERATE;
+        hp.eb_abs = eb; hp.s = s; hp.r = r;
+    }
+    return cuda_rc(launch_encode_f64(x, n, hp, dev, c->gen_sizes, c->gen_sizes + c->gen_tiles, (uint32_t*)out, out_capacity, out_bytes,
+                                     c->ws, c->sm_count, st));
+}
+
+int zccl_decompress_f64(zccl_ctx* c, const void* in, size_t in_bytes_max, double* y, size_t y_capacity_elems, void* stream)
+{
+    if (!c || !in || (!y && y_capacity_elems)) return ZCCL_E_ARG;
+    if (((uintptr_t)in & 3u) || ((uintptr_t)y & 7u)) return ZCCL_E_ARG;
+    if (in_bytes_max < (size_t)kHeaderBytes) return ZCCL_E_CAPACITY;
+    return cuda_rc(launch_decode_f64((const uint32_t*)in, in_bytes_max, y, y_capacity_elems, c->ws, c->sm_count, (cudaStream_t)stream));
 }
 
 int zccl_decompress_tiled(zccl_ctx* c, const void* in, size_t in_bytes_max, unsigned tile, float* y, size_t y_capacity_elems,

@@ -15,33 +15,59 @@ constexpr int kGenMaxBlocks = kGenericMaxTile / kBlock;   // 256
 
 __device__ __forceinline__ uint32_t bitlen(uint32_t v) { return 32u - (uint32_t)__clz((int)v); }
 
+// The two value types.  Everything behind the quantisation works on 32-bit codes and is the same for both; what
+// differs is one multiplication and one conversion on the way in (q = rint(x * r)), one conversion and one
+// multiplication on the way out (x' = q * s), the data-type field of the version word, and header words 4..5
+// (binary32: bound and step; binary64: the step as one binary64; the bound itself is not stored).
+__device__ __forceinline__ float vmul(float a, float b) { return __fmul_rn(a, b); }
+__device__ __forceinline__ double vmul(double a, double b) { return __dmul_rn(a, b); }
+__device__ __forceinline__ int32_t vrint(float t) { return __float2int_rn(t); }
+__device__ __forceinline__ int32_t vrint(double t) { return __double2int_rn(t); }
+__device__ __forceinline__ float vabs(float t) { return fabsf(t); }
+__device__ __forceinline__ double vabs(double t) { return fabs(t); }
+__device__ __forceinline__ void from_code(int32_t q, float s, float* y) { *y = __fmul_rn(__int2float_rn(q), s); }
+__device__ __forceinline__ void from_code(int32_t q, double s, double* y) { *y = __dmul_rn(__int2double_rn(q), s); }
+template <class V> struct Bound;
+template <> struct Bound<float> { using type = Params; static constexpr uint32_t version = kVersion; };
+template <> struct Bound<double> { using type = ParamsF64; static constexpr uint32_t version = kVersionF64; };
+__device__ __forceinline__ void header_step_words(const Params& p, uint32_t& w4, uint32_t& w5) { w4 = __float_as_uint(p.eb_abs); w5 = __float_as_uint(p.s); }
+__device__ __forceinline__ void header_step_words(const ParamsF64& p, uint32_t& w4, uint32_t& w5)
+{
+    const unsigned long long b = (unsigned long long)__double_as_longlong(p.s);
+    w4 = (uint32_t)b; w5 = (uint32_t)(b >> 32);
+}
+__device__ __forceinline__ float step_from_header(uint32_t w4, uint32_t w5, float) { (void)w4; return __uint_as_float(w5); }
+__device__ __forceinline__ double step_from_header(uint32_t w4, uint32_t w5, double) { return __longlong_as_double((long long)(((unsigned long long)w5 << 32) | w4)); }
+
 // Delta of element e of a tile (its code minus its predecessor's; 0 for the first element and for the padding
 // lanes of a ragged last block, which repeat the last element).  `t_abs` receives |x * r| for the range checks.
-__device__ __forceinline__ int32_t delta_at(const float* __restrict__ xt, uint32_t e, uint32_t last, float r, float& t_abs,
-                                            int32_t& q_out)
+template <class V>
+__device__ __forceinline__ int32_t delta_at(const V* __restrict__ xt, uint32_t e, uint32_t last, V r, V& t_abs, int32_t& q_out)
 {
     const uint32_t ec = e < last ? e : last;
     const uint32_t em = e ? e - 1 : 0;
     const uint32_t ep = em < last ? em : last;
-    const float t = __fmul_rn(__ldg(xt + ec), r), tp = __fmul_rn(__ldg(xt + ep), r);
-    t_abs = fabsf(t);
-    const int32_t q = __float2int_rn(t), qp = __float2int_rn(tp);
+    const V t = vmul(__ldg(xt + ec), r), tp = vmul(__ldg(xt + ep), r);
+    t_abs = vabs(t);
+    const int32_t q = vrint(t), qp = vrint(tp);
     q_out = q;
     return q - qp;
 }
 
 // Pass 1 (emit == 0): words of every tile's blob into sizes[].  Pass 3 (emit == 1): the blobs themselves, at the
 // places the index (written by the scan in between) gives them.
-__global__ void __launch_bounds__(256) generic_encode_kernel(const float* __restrict__ x, unsigned long long n, uint32_t T, uint32_t nT,
-                                                             Params hp, int use_dev_params, uint32_t* __restrict__ sizes,
-                                                             uint32_t* __restrict__ out, const uint32_t* __restrict__ go, int emit,
-                                                             Workspace ws)
+template <class V>
+__global__ void __launch_bounds__(256) generic_encode_kernel(const V* __restrict__ x, unsigned long long n, uint32_t T, uint32_t nT,
+                                                             typename Bound<V>::type hp, const typename Bound<V>::type* dev_params,
+                                                             uint32_t* __restrict__ sizes, uint32_t* __restrict__ out,
+                                                             const uint32_t* __restrict__ go, int emit, Workspace ws)
 {
+    using P = typename Bound<V>::type;
     __shared__ uint32_t Ls[kGenMaxBlocks];
     __shared__ uint32_t offs[kGenMaxBlocks + 1];
     __shared__ uint32_t wsum[8];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const Params p = use_dev_params ? *ws.params : hp;
+    const P p = dev_params ? *dev_params : hp;
     if (!p.valid) return;
     if (emit && *go == 0) return;
     uint32_t status = 0;
@@ -49,11 +75,11 @@ __global__ void __launch_bounds__(256) generic_encode_kernel(const float* __rest
         const unsigned long long start = (unsigned long long)t * T;
         const uint32_t len = (uint32_t)((n - start < (unsigned long long)T) ? (n - start) : (unsigned long long)T);
         const uint32_t nb = (len + kBlock - 1) / kBlock;
-        const float* xt = x + start;
-        float tmax = 0.0f;
+        const V* xt = x + start;
+        V tmax = 0;
         uint32_t words = 0;
         for (uint32_t b = warp; b < nb; b += 8) {
-            float ta; int32_t q;
+            V ta; int32_t q;
             const int32_t d = delta_at(xt, 32u * b + lane, len - 1, p.r, ta, q);
             tmax = fmaxf(tmax, ta);
             const uint32_t L = bitlen(__reduce_or_sync(kFull, (uint32_t)(d < 0 ? -d : d)));
@@ -61,9 +87,9 @@ __global__ void __launch_bounds__(256) generic_encode_kernel(const float* __rest
             words += L ? L + 1 : 0;
         }
 #pragma unroll
-        for (int s = 16; s; s >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(kFull, tmax, s));
-        if (!(tmax < 1073741824.0f)) status |= kStRange;
-        else if (tmax > 32768.5f) status |= kStPrecision;
+        for (int s = 16; s; s >>= 1) { const V o = __shfl_xor_sync(kFull, tmax, s); tmax = o > tmax ? o : tmax; }
+        if (!(tmax < (V)1073741824.0)) status |= kStRange;
+        else if (sizeof(V) == 4 && tmax > (V)32768.5) status |= kStPrecision;   // binary64 keeps its bound over the whole code range
         if (lane == 0) wsum[warp] = words;
         __syncthreads();
         if (!emit) {
@@ -92,7 +118,7 @@ __global__ void __launch_bounds__(256) generic_encode_kernel(const float* __rest
             __syncthreads();
             uint32_t* blob = out + kHeaderWords + nT + (t ? __ldg(out + kHeaderWords + t - 1) : 0u);
             if (tid == 0) {
-                float ta; int32_t q0;
+                V ta; int32_t q0;
                 (void)delta_at(xt, 0, len - 1, p.r, ta, q0);
                 blob[0] = (uint32_t)q0;                     // the tile's outlier: the code of its first element
             }
@@ -103,7 +129,7 @@ __global__ void __launch_bounds__(256) generic_encode_kernel(const float* __rest
             }
             for (uint32_t b = warp; b < nb; b += 8) {
                 const uint32_t L = Ls[b];
-                float ta; int32_t q;
+                V ta; int32_t q;
                 const int32_t d = delta_at(xt, 32u * b + lane, len - 1, p.r, ta, q);   // warp-uniform trip count below
                 if (L) {
                     const uint32_t a = (uint32_t)(d < 0 ? -d : d);
@@ -123,15 +149,16 @@ __global__ void __launch_bounds__(256) generic_encode_kernel(const float* __rest
 }
 
 // Pass 2: inclusive prefix of the tile sizes = the index; header; stream length; capacity check.  One CTA.
+template <class V>
 __global__ void __launch_bounds__(1024) generic_scan_kernel(const uint32_t* __restrict__ sizes, unsigned long long n, uint32_t T, uint32_t nT,
-                                                            Params hp, int use_dev_params, uint32_t* __restrict__ out,
+                                                            typename Bound<V>::type hp, const typename Bound<V>::type* dev_params, uint32_t* __restrict__ out,
                                                             unsigned long long out_cap, size_t* __restrict__ out_bytes,
                                                             uint32_t* __restrict__ go, Workspace ws)
 {
     __shared__ unsigned long long wtot[32];
     __shared__ unsigned long long carry_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const Params p = use_dev_params ? *ws.params : hp;
+    const typename Bound<V>::type p = dev_params ? *dev_params : hp;
     if (!p.valid) {
         if (tid == 0) { *out_bytes = 0; *go = 0; }
         return;
@@ -156,9 +183,11 @@ __global__ void __launch_bounds__(1024) generic_scan_kernel(const uint32_t* __re
     }
     if (!fits) return;
     if (tid == 0) {
-        out[0] = kMagic; out[1] = kVersion;
+        out[0] = kMagic; out[1] = Bound<V>::version;
         out[2] = (uint32_t)n; out[3] = (uint32_t)(n >> 32);
-        out[4] = __float_as_uint(p.eb_abs); out[5] = __float_as_uint(p.s);
+        uint32_t w4, w5;
+        header_step_words(p, w4, w5);
+        out[4] = w4; out[5] = w5;
         out[6] = T; out[7] = nT;
     }
     __syncthreads();
@@ -184,8 +213,9 @@ __global__ void __launch_bounds__(1024) generic_scan_kernel(const uint32_t* __re
 
 // Decompression: one CTA per tile.  Code-length bytes -> slot offsets; every warp rebuilds the deltas of its blocks
 // and their running sums inside the block; block totals are then chained through shared memory.
+template <class V>
 __global__ void __launch_bounds__(256) generic_decode_kernel(const uint32_t* __restrict__ in, unsigned long long cap_bytes, uint32_t T,
-                                                             float* __restrict__ y, unsigned long long y_cap, Workspace ws)
+                                                             V* __restrict__ y, unsigned long long y_cap, Workspace ws)
 {
     __shared__ uint32_t Ls[kGenMaxBlocks];
     __shared__ uint32_t offs[kGenMaxBlocks + 1];
@@ -197,13 +227,13 @@ __global__ void __launch_bounds__(256) generic_decode_kernel(const uint32_t* __r
     bool ok = cap_bytes >= (unsigned long long)kHeaderBytes;
     unsigned long long n = 0;
     uint32_t nT = 0, total_w = 0;
-    float s = 1.0f;
+    V s = 1;
     if (ok) {
         n = (unsigned long long)__ldg(in + 2) | ((unsigned long long)__ldg(in + 3) << 32);
-        s = __uint_as_float(__ldg(in + 5));
+        s = step_from_header(__ldg(in + 4), __ldg(in + 5), V());
         nT = __ldg(in + 7);
-        ok = __ldg(in + 0) == kMagic && __ldg(in + 1) == kVersion && __ldg(in + 6) == T && (n + T - 1) / T == nT &&
-             cap_bytes >= (unsigned long long)kHeaderBytes + 4ull * nT && s > 0.0f && isfinite(s);
+        ok = __ldg(in + 0) == kMagic && __ldg(in + 1) == Bound<V>::version && __ldg(in + 6) == T && (n + T - 1) / T == nT &&
+             cap_bytes >= (unsigned long long)kHeaderBytes + 4ull * nT && s > (V)0 && isfinite(s);
     }
     if (ok && nT) {
         total_w = __ldg(in + kHeaderWords + nT - 1);
@@ -289,7 +319,7 @@ __global__ void __launch_bounds__(256) generic_decode_kernel(const uint32_t* __r
         __syncthreads();
         if (!bad) {
             for (uint32_t e = tid; e < len; e += 256)
-                y[start + e] = __fmul_rn(__int2float_rn(btot[e >> 5] + pre[e]), s);
+                from_code(btot[e >> 5] + pre[e], s, y + start + e);
         } else if (tid == 0) {
             atomicOr(ws.status, kStBadStream);
         }
@@ -299,30 +329,125 @@ __global__ void __launch_bounds__(256) generic_decode_kernel(const uint32_t* __r
     }
 }
 
+// Minimum and maximum of a binary64 array into two ordered 64-bit keys; the last CTA to get there turns them and the
+// relative bound into the resolved block for binary64 (the reading of the binary32 path with the shrink 1 - 2^-20,
+// which keeps |x - x'| <= eb_abs over the whole code range) and re-arms the keys.
+__device__ __forceinline__ unsigned long long d2key(double v)
+{
+    const unsigned long long b = (unsigned long long)__double_as_longlong(v);
+    return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
+__device__ __forceinline__ double key2d(unsigned long long k)
+{
+    return __longlong_as_double((long long)((k >> 63) ? (k & 0x7FFFFFFFFFFFFFFFull) : ~k));
+}
+__device__ void resolve_f64(double ea, bool range_ok, const Workspace& ws)
+{
+    ParamsF64 p;
+    p.valid = range_ok ? 1 : 0;
+    const double ebq = __dmul_rn(ea, 1.0 - 9.5367431640625e-07);   // 1 - 2^-20
+    const double s = __dmul_rn(ebq, 2.0);
+    if (!(s > 0.0) || !isfinite(s)) p.valid = 0;
+    const double r = __ddiv_rn(1.0, s);
+    if (!isfinite(r)) p.valid = 0;
+    p.eb_abs = ea; p.s = s; p.r = r;
+    *ws.params64 = p;
+    if (!p.valid) atomicOr(ws.status, kStDegenerate);
+}
+__global__ void __launch_bounds__(256) range_f64_kernel(const double* __restrict__ x, unsigned long long n, double eb, Workspace ws)
+{
+    double lo = __longlong_as_double(0x7FF0000000000000ll), hi = __longlong_as_double((long long)0xFFF0000000000000ull);
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (unsigned long long)gridDim.x * blockDim.x) {
+        const double v = __ldg(x + i);
+        lo = v < lo ? v : lo;
+        hi = v > hi ? v : hi;
+    }
+#pragma unroll
+    for (int s = 16; s; s >>= 1) {
+        const double a = __shfl_xor_sync(kFull, lo, s), b = __shfl_xor_sync(kFull, hi, s);
+        lo = a < lo ? a : lo;
+        hi = b > hi ? b : hi;
+    }
+    __shared__ uint32_t last_s;
+    if ((threadIdx.x & 31) == 0 && lo <= hi) { atomicMin(ws.minmax64 + 0, d2key(lo)); atomicMax(ws.minmax64 + 1, d2key(hi)); }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        last_s = atomicAdd(ws.done, 1u) == gridDim.x - 1 ? 1u : 0u;
+    }
+    __syncthreads();
+    if (last_s && threadIdx.x == 0) {
+        __threadfence();
+        *ws.done = 0;
+        const unsigned long long kmin = *reinterpret_cast<volatile unsigned long long*>(ws.minmax64 + 0);
+        const unsigned long long kmax = *reinterpret_cast<volatile unsigned long long*>(ws.minmax64 + 1);
+        double range = 0.0;
+        if (kmin <= kmax) range = __dsub_rn(key2d(kmax), key2d(kmin));
+        ws.minmax64[0] = 0xFFFFFFFFFFFFFFFFull;
+        ws.minmax64[1] = 0ull;
+        resolve_f64(__dmul_rn(eb, range), range > 0.0 && isfinite(range), ws);
+    }
+}
+
 }  // namespace
 
-cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* sizes,
-                                  uint32_t* go, uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws,
-                                  int sm_count, cudaStream_t st)
+template <class V>
+static cudaError_t generic_encode(const V* x, unsigned long long n, uint32_t T, typename Bound<V>::type hp, const typename Bound<V>::type* dev_params,
+                                  uint32_t* sizes, uint32_t* go, uint32_t* out, unsigned long long out_cap, size_t* out_bytes,
+                                  const Workspace& ws, int sm_count, cudaStream_t st)
 {
     const uint32_t nT = (uint32_t)((n + T - 1) / T);
     const unsigned grid = nT < (unsigned)sm_count * 4u ? (nT ? nT : 1u) : (unsigned)sm_count * 4u;
-    const int dp = device_params ? 1 : 0;
     count_launches(3);
-    generic_encode_kernel<<<grid, 256, 0, st>>>(x, n, T, nT, hp, dp, sizes, out, go, 0, ws);
-    generic_scan_kernel<<<1, 1024, 0, st>>>(sizes, n, T, nT, hp, dp, out, out_cap, out_bytes, go, ws);
-    generic_encode_kernel<<<grid, 256, 0, st>>>(x, n, T, nT, hp, dp, sizes, out, go, 1, ws);
+    generic_encode_kernel<V><<<grid, 256, 0, st>>>(x, n, T, nT, hp, dev_params, sizes, out, go, 0, ws);
+    generic_scan_kernel<V><<<1, 1024, 0, st>>>(sizes, n, T, nT, hp, dev_params, out, out_cap, out_bytes, go, ws);
+    generic_encode_kernel<V><<<grid, 256, 0, st>>>(x, n, T, nT, hp, dev_params, sizes, out, go, 1, ws);
     return cudaGetLastError();
 }
-
-cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, float* y, unsigned long long y_cap,
-                                  const Workspace& ws, int sm_count, cudaStream_t st)
+template <class V>
+static cudaError_t generic_decode(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, V* y, unsigned long long y_cap, const Workspace& ws,
+                                  int sm_count, cudaStream_t st)
 {
     const unsigned long long nT = (y_cap + T - 1) / T;
     const unsigned cap = (unsigned)sm_count * 4u;
     const unsigned grid = nT < cap ? (unsigned)(nT ? nT : 1) : cap;
     count_launches(1);
-    generic_decode_kernel<<<grid, 256, 0, st>>>(in, cap_bytes, T, y, y_cap, ws);
+    generic_decode_kernel<V><<<grid, 256, 0, st>>>(in, cap_bytes, T, y, y_cap, ws);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* sizes,
+                                  uint32_t* go, uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws,
+                                  int sm_count, cudaStream_t st)
+{
+    return generic_encode<float>(x, n, T, hp, device_params ? ws.params : nullptr, sizes, go, out, out_cap, out_bytes, ws, sm_count, st);
+}
+
+cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, float* y, unsigned long long y_cap,
+                                  const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    return generic_decode<float>(in, cap_bytes, T, y, y_cap, ws, sm_count, st);
+}
+
+cudaError_t launch_encode_f64(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* sizes, uint32_t* go,
+                              uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    return generic_encode<double>(x, n, (uint32_t)kTile, hp, device_params ? ws.params64 : nullptr, sizes, go, out, out_cap, out_bytes, ws,
+                                  sm_count, st);
+}
+
+cudaError_t launch_decode_f64(const uint32_t* in, unsigned long long cap_bytes, double* y, unsigned long long y_cap, const Workspace& ws,
+                              int sm_count, cudaStream_t st)
+{
+    return generic_decode<double>(in, cap_bytes, (uint32_t)kTile, y, y_cap, ws, sm_count, st);
+}
+
+cudaError_t launch_range_f64(const double* x, unsigned long long n, double eb, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    const unsigned long long want = (n + 255) / 256;
+    const unsigned cap = (unsigned)sm_count * 8u;
+    count_launches(1);
+    range_f64_kernel<<<(unsigned)(want < cap ? (want ? want : 1) : cap), 256, 0, st>>>(x, n, eb, ws);
     return cudaGetLastError();
 }
 

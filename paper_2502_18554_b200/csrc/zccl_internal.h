@@ -8,6 +8,7 @@ namespace zccl {
 
 constexpr uint32_t kMagic = 0x314C435Au;    // 'Z','C','L','1'
 constexpr uint32_t kVersion = 0x05000001u;  // version 1, dtype 0 (fp32), log2(block) = 5
+constexpr uint32_t kVersionF64 = 0x05000101u;  // the same with dtype 1 (fp64): header words 4..5 hold the step as one binary64
 constexpr int kHeaderBytes = 32;
 constexpr int kHeaderWords = 8;
 constexpr int kBlock = 32;                  // elements per block = warp width
@@ -38,6 +39,14 @@ struct Params {
     int valid;    // 0: resolution failed (degenerate range); codec kernels then write nothing
 };
 
+// Resolved bound for binary64 input (device resident when the mode is value-range relative).
+struct ParamsF64 {
+    double eb_abs;
+    double s;     // quantisation step: 2 * fl64(eb_abs * (1 - 2^-20))
+    double r;     // fl64(1 / s)
+    int valid;
+};
+
 // Scan / bookkeeping workspace owned by the context.
 struct Workspace {
     unsigned long long* tile_state;  // one 64-bit {epoch:31 | inclusive:1 | words:32} per tile of a launch
@@ -49,6 +58,8 @@ struct Workspace {
     uint32_t* status;                // device status bits
     Params* params;                  // resolved bound for REL mode
     uint32_t* minmax;                // two ordered-int keys: running min and max
+    ParamsF64* params64;             // the same two for binary64 input (null in the allocation-free workspace)
+    unsigned long long* minmax64;
     // Two-step compression (encode rounds into fixed slots, then place): null where there is no room for it (the
     // allocation-free entry point), which then compresses in a single pass.
     uint32_t* slots;                 // per round of a launch (4 per tile): kRoundSlotWords words
@@ -158,6 +169,11 @@ cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t
                                   int sm_count, cudaStream_t st);
 cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, float* y, unsigned long long y_cap,
                                   const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_encode_f64(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* sizes, uint32_t* go,
+                              uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_decode_f64(const uint32_t* in, unsigned long long cap_bytes, double* y, unsigned long long y_cap, const Workspace& ws,
+                              int sm_count, cudaStream_t st);
+cudaError_t launch_range_f64(const double* x, unsigned long long n, double eb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_stream_stats(const uint32_t* in, unsigned long long cap_bytes, unsigned long long* hist, const Workspace& ws,
                                 int sm_count, cudaStream_t st);
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);

@@ -61,6 +61,7 @@ Workspace workspace_at(unsigned char* base, uint32_t* sm)
     ws.status = sm + 3;
     ws.params = reinterpret_cast<Params*>(sm + 4);
     ws.minmax = sm + 8;
+    ws.params64 = nullptr; ws.minmax64 = nullptr;
     ws.slots = nullptr; ws.round_words = nullptr; ws.outliers = nullptr;
     ws.max_tiles = (uint32_t)kMaxTiles;
     ws.skip_publish = 0xFFFFFFFFu;

@@ -24,7 +24,7 @@ EXPORTS = [
     "zccl_ctx_create", "zccl_ctx_destroy", "zccl_compress_bound", "zccl_launch_count", "zccl_status", "zccl_strerror",
     "zccl_compress", "zccl_decompress", "zccl_decompress_reduce_compress",
     "zccl_sim_allreduce", "zccl_sim_allgather", "zccl_sim_bcast", "zccl_sim_reduce_scatter", "zccl_sim_scatter",
-    "zccl_sim_sizes", "zccl_quality", "zccl_range", "zccl_resolve_range", "zccl_resolve_range_host", "zccl_scale", "zccl_stream_stats",
+    "zccl_sim_sizes", "zccl_quality", "zccl_compress_f64", "zccl_decompress_f64", "zccl_range", "zccl_resolve_range", "zccl_resolve_range_host", "zccl_scale", "zccl_stream_stats",
     "zccl_compress_bound_tiled", "zccl_compress_tiled", "zccl_decompress_tiled",
     "zccl_compress_host", "zccl_decompress_host", "zccl_compress_noalloc", "zccl_debug_skip_publish",
     "zccl_debug_set_launch_counter",
@@ -68,6 +68,8 @@ def lib():
         L.zccl_sim_scatter.argtypes = [vp, vp, vp, C.c_int, sz, C.c_int, C.c_float, vp]
         L.zccl_quality.argtypes = [vp, vp, vp, sz, vp, vp]
         L.zccl_range.argtypes = [vp, vp, sz, vp, vp]
+        L.zccl_compress_f64.argtypes = [vp, vp, sz, C.c_int, C.c_double, vp, sz, vp, vp]
+        L.zccl_decompress_f64.argtypes = [vp, vp, sz, vp, sz, vp]
         L.zccl_resolve_range.argtypes = [vp, vp, C.c_float, vp, vp]
         L.zccl_resolve_range_host.argtypes = [C.c_float, C.c_float, C.c_float, vp, vp, vp]
         L.zccl_stream_stats.argtypes = [vp, vp, sz, vp, vp]
@@ -262,6 +264,18 @@ class Context:
         """zccl_stream_stats: hist (int64[33], device) <- blocks per code length 0..31, then the number of blocks."""
         _check(lib().zccl_stream_stats(self._h, _dev_ptr(stream_bytes, torch.uint8), stream_bytes.numel(),
                                        _dev_ptr(hist, torch.int64), _stream_ptr(stream)), "zccl_stream_stats")
+
+    def compress_f64(self, x: torch.Tensor, eb_mode: int, eb: float, out: torch.Tensor, out_bytes: torch.Tensor, stream=None):
+        """zccl_compress_f64: x float64 [n] -> stream bytes in `out` (uint8), length in `out_bytes` (int64[1], device)."""
+        _check(lib().zccl_compress_f64(self._h, _dev_ptr(x, torch.float64) if x.numel() else None, x.numel(), eb_mode, eb,
+                                       _dev_ptr(out, torch.uint8), out.numel(), _dev_ptr(out_bytes, torch.int64),
+                                       _stream_ptr(stream)), "zccl_compress_f64")
+
+    def decompress_f64(self, in_c: torch.Tensor, y: torch.Tensor, stream=None):
+        """zccl_decompress_f64: stream bytes -> y float64 (capacity y.numel())."""
+        _check(lib().zccl_decompress_f64(self._h, _dev_ptr(in_c, torch.uint8), in_c.numel(),
+                                         _dev_ptr(y, torch.float64) if y.numel() else None, y.numel(), _stream_ptr(stream)),
+               "zccl_decompress_f64")
 
     def range(self, x: torch.Tensor, minmax: torch.Tensor, stream=None):
         """zccl_range: minmax (float32[2], device) <- (min x, max x)."""

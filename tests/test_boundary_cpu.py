@@ -21,7 +21,7 @@ def lib():
 def declared_symbols():
     text = (ROOT / "include" / "zccl.h").read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(zccl_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(zccl_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_header_symbols_are_exported(lib):
