@@ -206,7 +206,7 @@ def _timed(fn, sets: int, warmup: int = 10, iters: int = 10):
     return statistics.mean(ts), min(ts)
 
 
-def _timed_long(fn, sets: int, device_index: int, min_launches: int = 200, min_ms: float = 400.0, warmup: int = 3):
+def _timed_long(fn, sets: int, device_index: int, min_ms: float = 400.0, min_launches: int = 200, warmup: int = 3):
     """Device time (us) of one call fn(set index) over a long run: a CUDA graph of `sets` calls is replayed until
     at least `min_launches` calls and `min_ms` milliseconds have gone by, inside ONE pair of events, with the SM clock
     sampled meanwhile.  Returns (us per call, calls, median SM MHz or None)."""
@@ -445,6 +445,25 @@ def other_configs(z, peak: float, x1, loc1) -> dict:
     for eb in (1e-2, 1e-4):
         out[f"cfg1 REL {eb:g}"] = fracs(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, False, loc1))
     out["cfg3 ABS 1e-05 (1 GiB)"] = fracs(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, False))
+    # the cfg1 field as binary64 (128 MiB) through the binary64 entry points: plain kernels, 8 bytes per element
+    n = x1.size
+    sets = 4
+    xd = [torch.from_numpy(x1.astype(np.float64)).cuda() for _ in range(sets)]
+    od = [torch.empty(z.compress_bound(n), dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    yd = [torch.empty(n, dtype=torch.float64, device="cuda") for _ in range(sets)]
+    szd = torch.zeros(1, dtype=torch.int64, device="cuda")
+    c_us, _ = _timed(lambda i: big.compress_f64(xd[i], z.EB_REL, REL, od[i], szd), sets)
+    rc = big.check()
+    cb = int(szd.item())
+    d_us, _ = _timed(lambda i: big.decompress_f64(od[i][:cb], yd[i]), sets)
+    big.check()
+    out["cfg1 as binary64 REL 0.001"] = {
+        "ratio": round(8 * n / cb, 3), "status": rc, "compress_us": round(c_us, 2), "decompress_us": round(d_us, 2),
+        "compress_gbs": round(8 * n / c_us / 1e3, 1), "decompress_gbs": round(8 * n / d_us / 1e3, 1),
+        "compress_frac": round((2 * 8 * n + cb) / c_us / 1e3 / peak, 3),   # the input is read twice (sizes, then blobs) and once more for the range
+        "decompress_frac": round((8 * n + cb) / d_us / 1e3 / peak, 3),
+        "max_abs_err": float((yd[0] - xd[0]).abs().max().item())}
+    del xd, od, yd
     big.close()
     torch.cuda.empty_cache()
 
@@ -472,6 +491,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
+                    help="shortest timed region in ms (steps and per-call loops are replayed to get there); 0 for a profiler's launch list")
     ap.add_argument("--no-configs", action="store_true", help="leave the `configs` object (cfg1 at other bounds, cfg2, cfg3) out")
     ap.add_argument("--no-graph", action="store_true", help="time eagerly launched steps instead of CUDA graph replays")
     ap.add_argument("--table", action="store_true",
@@ -606,7 +627,7 @@ def main():
         p1.record(stream)
         p1.synchronize()
         est_ms = max_over_ranks(p0.elapsed_time(p1), dev) / ROT
-        replays = max(1, int(-(-MIN_TIMED_MS // (est_ms * args.steps))))
+        replays = max(1, int(-(-args.min_ms // (est_ms * args.steps))))
     sampler = ClockSampler(local_rank)
     fence()
     sampler.start()
@@ -665,10 +686,11 @@ def main():
     for k in range(ROT):                       # the streams the decoder and the hop read
         ctx.compress(xs[k], z.EB_REL, REL, cs[k], nb1)
     torch.cuda.synchronize()
-    enc_us, enc_calls, enc_mhz = _timed_long(lambda k: ctx.compress(xs[k], z.EB_ABS, eb_abs, c2s[k], nb2), ROT, local_rank)
-    dec_us, dec_calls, dec_mhz = _timed_long(lambda k: ctx.decompress(cs[k], ys[k]), ROT, local_rank)
+    kmin_ms, kmin_n = (400.0, 200) if args.min_ms > 0 else (0.0, 2 * ROT)
+    enc_us, enc_calls, enc_mhz = _timed_long(lambda k: ctx.compress(xs[k], z.EB_ABS, eb_abs, c2s[k], nb2), ROT, local_rank, kmin_ms, kmin_n)
+    dec_us, dec_calls, dec_mhz = _timed_long(lambda k: ctx.decompress(cs[k], ys[k]), ROT, local_rank, kmin_ms, kmin_n)
     hop_us, hop_calls, hop_mhz = _timed_long(
-        lambda k: ctx.decompress_reduce_compress(cs[k], N_ELEMS, c2s[k], nb2, local=locs[k]), ROT, local_rank)
+        lambda k: ctx.decompress_reduce_compress(cs[k], N_ELEMS, c2s[k], nb2, local=locs[k]), ROT, local_rank, kmin_ms, kmin_n)
     ctx.check()
     in_b = 4 * N_ELEMS
     c1_b = in_b / ratio1
@@ -697,7 +719,7 @@ def main():
     for k in range(ROT):
         ctx.compress(xs[k], z.EB_REL, REL, cs[k], nb1)
         ctx.decompress(cs[k], ys[k])
-    q_us, q_calls, q_mhz = _timed_long(lambda k: ctx.quality(xs[k], ys[k], qout), ROT, local_rank)
+    q_us, q_calls, q_mhz = _timed_long(lambda k: ctx.quality(xs[k], ys[k], qout), ROT, local_rank, kmin_ms, kmin_n)
     ctx.quality(xs[0], ys[0], qout)   # the batch the ratios are quoted on
     torch.cuda.synchronize()
     qv = qout.cpu().numpy()
