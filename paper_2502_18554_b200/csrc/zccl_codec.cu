@@ -1597,8 +1597,9 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
                 const uint32_t rounds = (nb + 31) >> 5;
                 for (uint32_t rd = 0; rd < rounds; ++rd) {
                     const uint32_t L = (lp >> (8u * rd)) & 0xFFu;
-                    const uint32_t first = 1u + padw + pay_off, beyond = first + __reduce_add_sync(kFull, L ? L + 1u : 0u);
-                    if (beyond > win.end) {   // the round reaches past the window (describe_blob has checked it against the blob)
+                    const uint32_t first = 1u + padw + pay_off;
+                    // only a blob larger than its buffer has a window that ends before the blob does
+                    if (win.end < cur.words && first + __reduce_add_sync(kFull, L ? L + 1u : 0u) > win.end) {   // the round reaches past the window
                         __syncwarp();         // every lane is done with the window as it is
                         if (lane == 0) window_request(cur, first, sh.blob[p], &sh.bar[p]);
                         if (!mbar_wait(&sh.bar[p], (p ? fills1 : fills0) & 1u)) status |= kStTimeout;
@@ -1862,8 +1863,8 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
         // moves the window over the incoming blob to round e's first word when the round reaches past its end
         auto reach = [&](uint32_t e) {
             const uint32_t L = (lp1 >> (8u * e)) & 0xFFu;
-            const uint32_t first = 1u + padw + pay1, beyond = first + __reduce_add_sync(kFull, L ? L + 1u : 0u);
-            if (beyond > win.end) {
+            const uint32_t first = 1u + padw + pay1;
+            if (win.end < cur.words && first + __reduce_add_sync(kFull, L ? L + 1u : 0u) > win.end) {
                 __syncwarp();   // every lane is done with the window as it is
                 if (lane == 0) window_request(cur, first, sh.blob, &sh.bar_blob);
                 if (!mbar_wait(&sh.bar_blob, bfill & 1u)) status |= kStTimeout;
