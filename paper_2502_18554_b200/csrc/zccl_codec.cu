@@ -1397,10 +1397,10 @@ __device__ __forceinline__ void window_request(const BlobRef& br, uint32_t first
 }
 struct alignas(1024) DecWarpShared {
     float out[2][kRound];                  // each on a 1024-byte boundary
-    alignas(16) uint32_t blob[2][kDecBlobWords];
-    alignas(8) unsigned long long bar[2];
+    alignas(16) uint32_t blob[kDecBlobWords];
+    alignas(8) unsigned long long bar;
 };
-static_assert(sizeof(DecWarpShared) == 17 * 1024, "a warp's share of the shared memory");
+static_assert(sizeof(DecWarpShared) == 13 * 1024, "a warp's share of the shared memory");
 
 // Tiled tensor store of a stage to rows [row0, row0 + 32) of the array behind `map` (one thread).
 __device__ __forceinline__ void tensor_store_round(const CUtensorMap* map, uint32_t row0, const float* stage)
@@ -1502,7 +1502,7 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
     }
 }
 
-__global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
+__global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
                                                                         Workspace ws)
 {
     pdl_enter();
@@ -1511,12 +1511,11 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
     DecWarpShared& sh = reinterpret_cast<DecWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
     uint32_t status = 0;
     if (lane == 0) {
-        mbar_init(&sh.bar[0], 1);
-        mbar_init(&sh.bar[1], 1);
+        mbar_init(&sh.bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed per blob buffer (phase parity of its mbarrier)
+    uint32_t fills = 0;   // bulk copies completed into the blob buffer (phase parity of its mbarrier)
 
     // the job of the tile looked up last, with its stream's header
     int cj = -1;
@@ -1532,9 +1531,9 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
             h = read_header(q.in_c, q.in_cap);
         }
     };
-    // The blob of tile t of the launch, from the index alone; its 16-byte-aligned cover is requested into blob buffer
-    // `buf` when it fits there and lies inside the readable bytes.  Uniform over the warp.
-    auto request = [&](uint32_t t, uint32_t buf) {
+    // The blob of tile t of the launch, from the index alone; the front of its 16-byte-aligned cover is requested into the
+    // blob buffer when the cover lies inside the readable bytes.  Uniform over the warp.
+    auto request = [&](uint32_t t) {
         BlobRef br;
         br.ptr = nullptr; br.words = 0; br.staged = false;
         if (t >= jb.total_tiles) return br;
@@ -1550,7 +1549,7 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
         br.words = w_end - w_beg;
         const uintptr_t a_end = ((uintptr_t)(br.ptr + br.words) + 15) & ~(uintptr_t)15;
         if (a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {   // the copies may read up to the boundary behind the blob
-            if (lane == 0) window_request(br, 0, sh.blob[buf], &sh.bar[buf]);
+            if (lane == 0) window_request(br, 0, sh.blob, &sh.bar);
             br.staged = true;
         }
         return br;
@@ -1558,9 +1557,8 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
 
     const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
     uint32_t t = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
-    uint32_t p = 0;    // blob buffer of the current tile
     uint32_t so = 0;   // output stage to use next
-    BlobRef cur = request(t, 0);
+    BlobRef cur = request(t);
     while (t < jb.total_tiles) {
         // the current tile's facts, before the look-up of the next tile moves on to another job
         enter_job(t);
@@ -1569,12 +1567,20 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
         const StreamInfo hc = h;
         const int jcur = cj;
         const bool job_bad = !hc.ok, too_small = hc.ok && hc.n > job.n;
-        __syncwarp();   // every lane is done with the other blob buffer
         const uint32_t tn = t + stride < t ? 0xFFFFFFFFu : t + stride;
-        const BlobRef nxt = request(tn, p ^ 1u);
+        // The one blob buffer takes the next tile's blob as soon as this tile's last round is decoded (16 warps per SM
+        // with one buffer beat 12 with two: 4096 tiles leave the busiest of 2368 warps two tiles instead of three).
+        BlobRef nxt;
+        nxt.ptr = nullptr; nxt.words = 0; nxt.staged = false;
+        bool asked = false;
+        auto ask_next = [&]() {
+            __syncwarp();   // every lane is done with the blob buffer
+            nxt = request(tn);
+            asked = true;
+        };
         if (cur.staged) {
-            if (!mbar_wait(&sh.bar[p], (p ? fills1 : fills0) & 1u)) status |= kStTimeout;
-            if (p) ++fills1; else ++fills0;
+            if (!mbar_wait(&sh.bar, fills & 1u)) status |= kStTimeout;
+            ++fills;
         }
         if (job_bad) status |= kStBadStream;
         else if (too_small) status |= kStCapacity;
@@ -1585,7 +1591,7 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
             const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2;
             BlobWindow win;
             win.base = cur.ptr; win.end = cur.words;
-            if (cur.staged) win = window_at(cur, 0, sh.blob[p]);
+            if (cur.staged) win = window_at(cur, 0, sh.blob);
             const int mode = describe_blob(win.base, cur.words, nb, lane);   // the head (at most 33 words) is in every first window
             if (mode == 0) status |= kStBadStream;
             else {
@@ -1601,10 +1607,10 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
                     // only a blob larger than its buffer has a window that ends before the blob does
                     if (win.end < cur.words && first + __reduce_add_sync(kFull, L ? L + 1u : 0u) > win.end) {   // the round reaches past the window
                         __syncwarp();         // every lane is done with the window as it is
-                        if (lane == 0) window_request(cur, first, sh.blob[p], &sh.bar[p]);
-                        if (!mbar_wait(&sh.bar[p], (p ? fills1 : fills0) & 1u)) status |= kStTimeout;
-                        if (p) ++fills1; else ++fills0;
-                        win = window_at(cur, first, sh.blob[p]);
+                        if (lane == 0) window_request(cur, first, sh.blob, &sh.bar);
+                        if (!mbar_wait(&sh.bar, fills & 1u)) status |= kStTimeout;
+                        ++fills;
+                        win = window_at(cur, first, sh.blob);
                     }
                     const uint32_t* blob = win.base;
                     // the stage about to be written was handed to a tensor store two rounds ago
@@ -1613,6 +1619,7 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
                     float* stage = sh.out[so];
                     if (mode == 1) decode_round<0>(blob, padw, L, pay_off, code, hc.s, stage, lane);
                     else decode_round_general(blob, padw, L, &pay_off, &code, hc.s, stage, lane, nullptr, 0u);
+                    if (rd + 1 == rounds) ask_next();
                     __syncwarp();   // the stage's rows, written by all lanes, are visible
                     const uint32_t e0 = rd * (uint32_t)kRound;
                     if (mapped && e0 + (uint32_t)kRound <= len) {
@@ -1624,9 +1631,9 @@ __global__ void __launch_bounds__(kCodecThreads, 3) decode_tiles_kernel(const __
                 }
             }
         }
+        if (!asked) ask_next();
         cur = nxt;
         t = tn;
-        p ^= 1u;
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     if (status) atomicOr(ws.status, status);
