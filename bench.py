@@ -759,6 +759,33 @@ def main():
            "what": "zccl_compress_host + zccl_decompress_host of the 64 MiB batch (uncompressed bytes per op / time)",
            "ms_per_step": e2e_ms, "h2d_bytes_per_step": in_b + nb, "d2h_bytes_per_step": nb + 8 + in_b}
 
+    # The same pairs as two independent pipelines (a context and a stream each, taking turns): one pipeline's upload
+    # runs while the other's download does, which is what a PCIe link's two directions allow; a single call chain can
+    # only use one direction at a time.
+    ctx_b = z.Context(N_ELEMS, 0)
+    pipes = [(ctx, torch.cuda.Stream(), oh, yh),
+             (ctx_b, torch.cuda.Stream(), torch.empty(cap, dtype=torch.uint8).pin_memory(), torch.empty(N_ELEMS, dtype=torch.float32).pin_memory())]
+    for c, s_, o_, y_ in pipes:
+        c.decompress_host(o_, c.compress_host(xh, z.EB_REL, REL, o_, stream=s_), y_, stream=s_)
+    fence()
+    p0 = torch.cuda.Event(enable_timing=True)
+    p0.record(pipes[0][1])
+    for _ in range(e2e_steps):
+        for c, s_, o_, y_ in pipes:
+            c.decompress_host(o_, c.compress_host(xh, z.EB_REL, REL, o_, stream=s_), y_, stream=s_)
+    ends = []
+    for c, s_, o_, y_ in pipes:
+        e_ = torch.cuda.Event(enable_timing=True)
+        e_.record(s_)
+        ends.append(e_)
+    fence()
+    ctx.check()
+    ctx_b.check()
+    two_ms = max_over_ranks(max(p0.elapsed_time(e_) for e_ in ends), dev) / (2 * e2e_steps)
+    e2e["two_pipelines"] = {"value": whole_job_gbs(2 * in_b, world, two_ms), "unit": "GB/s", "ms_per_step": two_ms,
+                            "what": "the same pairs issued in turn on two contexts and two streams"}
+    ctx_b.close()
+
     # ---- the other configurations of the workload list, a few graph replays each (single-GPU runs only)
     configs = None
     if rank == 0 and world == 1 and not args.no_configs:

@@ -351,8 +351,12 @@ int zccl_decompress_f64(zccl_ctx* ctx, const void* in, size_t in_bytes_max, doub
  * Host-buffer convenience forms: copy the input from host memory into a staging area of the context, run the
  * device path, copy the result back, all enqueued on `stream` (pinned host memory makes the copies asynchronous).
  * They exist so that end-to-end cost including PCIe transfers can be measured through this boundary.
- *   zccl_compress_host:   x_host n floats -> out_host (out_capacity bytes), *out_bytes_host after the stream ran
- *   zccl_decompress_host: in_host in_bytes bytes -> y_host (y_capacity_elems floats)
+ *   zccl_compress_host:   x_host n floats -> out_host (out_capacity bytes) and *out_bytes_host; synchronises `stream`
+ *                         (the length has to reach the host before the stream can be copied), so both are valid when
+ *                         the call returns
+ *   zccl_decompress_host: in_host in_bytes bytes -> y_host (y_capacity_elems floats), valid once `stream` has run; the
+ *                         element count is read from in_host's header on the host when the call is made, so in_host
+ *                         must hold the stream by then
  * Need max_elems >= n.  Errors as for the device forms.
  */
 int zccl_compress_host(zccl_ctx* ctx, const float* x_host, size_t n, int eb_mode, float eb,

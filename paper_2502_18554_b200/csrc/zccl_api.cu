@@ -856,6 +856,8 @@ int zccl_compress_host(zccl_ctx* c, const float* x_host, size_t n, int eb_mode, 
     const size_t nbytes = *out_bytes_host;
     if (nbytes > out_capacity) return ZCCL_E_CAPACITY;
     if (nbytes && cudaMemcpyAsync(out_host, c->stage_c, nbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZCCL_E_CUDA;
+    // the stream is in host memory when the call returns: zccl_decompress_host reads its header on the host
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ZCCL_E_CUDA;
     return ZCCL_OK;
 }
 
