@@ -1711,8 +1711,11 @@ __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, cons
     }
 }
 
-__global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps loc_maps,
-                                                                     const __grid_constant__ TileMaps raw_maps, Workspace ws, uint32_t split_shift)
+// maps: tensor map of job j's uncompressed operand at [j] and, in launches of at most kMaxJobs / 2 jobs, of its
+// uncompressed result at [kMaxJobs / 2 + j] (a second array of maps made the parameters 22 KB and the launch 1.6 us
+// slower; launches with more jobs write such results with plain stores).
+__global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
+                                                                     Workspace ws, uint32_t split_shift)
 {
     // split_shift 0: a warp's unit of work is a tile; 1: two rounds; 2: a round (small launches: more warps at work, and
     // none of them walks four rounds in a row)
@@ -1790,7 +1793,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
             const uint32_t e0 = rd * (uint32_t)kRound;
             if (e0 < len) {
                 if ((((uintptr_t)q.x) & 15u) == 0 && e0 + (uint32_t)kRound <= len) {
-                    if (lane == 0) tensor_load_round(sh.loc[buf], &sh.bar_loc[buf], &loc_maps.m[job_index], tile * (uint32_t)kBlocksPerTile + (e0 >> 5));
+                    if (lane == 0) tensor_load_round(sh.loc[buf], &sh.bar_loc[buf], &maps.m[job_index], tile * (uint32_t)kBlocksPerTile + (e0 >> 5));
                     bulk = true;
                 } else load_round_ragged(sh.loc[buf], q.x + start, e0, len, lane);
             }
@@ -1956,9 +1959,9 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
                 if (job.y) {   // an uncompressed copy of the result leaves the stage before the encoder writes over it
                     const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
                     if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
-                    else if ((((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
+                    else if (jb.count <= kMaxJobs / 2 && (((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
                         if (lane == 0) {
-                            tensor_store_round(&raw_maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), ys);
+                            tensor_store_round(&maps.m[kMaxJobs / 2 + jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), ys);
                             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                         }
                     } else store_round_ragged(job.y + start + e0, ys, count, lane);
@@ -2100,12 +2103,12 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     cudaError_t e = device_setup(&d);
     if (e != cudaSuccess) return e;
     if (!ws.slots) return cudaErrorInvalidValue;
-    thread_local TileMaps loc_maps, raw_maps;   // 16 KiB: kept off the stack, one pair per calling thread
-    memset(&loc_maps, 0, sizeof(loc_maps));
-    memset(&raw_maps, 0, sizeof(raw_maps));
+    thread_local TileMaps maps;   // 8 KiB: kept off the stack, one per calling thread
+    memset(&maps, 0, sizeof(maps));
     for (int j = 0; j < jb.count; ++j) {
-        if (jb.job[j].x && (e = make_row_map(&loc_maps.m[j], jb.job[j].x, jb.job[j].n)) != cudaSuccess) return e;
-        if (jb.job[j].y && (e = make_row_map(&raw_maps.m[j], jb.job[j].y, jb.job[j].n)) != cudaSuccess) return e;
+        if (jb.job[j].x && (e = make_row_map(&maps.m[j], jb.job[j].x, jb.job[j].n)) != cudaSuccess) return e;
+        if (jb.count <= kMaxJobs / 2 && jb.job[j].y && (e = make_row_map(&maps.m[kMaxJobs / 2 + j], jb.job[j].y, jb.job[j].n)) != cudaSuccess)
+            return e;
     }
     GroupTable gt;
     const uint32_t groups = group_table(jb, gt);
@@ -2114,7 +2117,7 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     const unsigned long long warps = cap * kCodecWarps;
     const uint32_t split_shift = 4ull * jb.total_tiles <= warps ? 2u : 2ull * jb.total_tiles <= warps ? 1u : 0u;
     const unsigned long long want = ((((unsigned long long)jb.total_tiles) << split_shift) + kCodecWarps - 1) / kCodecWarps;
-    e = launch_k(hop_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kHopSmemBytes, st, jb, loc_maps, raw_maps, ws,
+    e = launch_k(hop_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws,
                  split_shift);
     if (e != cudaSuccess) return e;
     return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
