@@ -19,7 +19,9 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kBlocksPerWarp = kBlocksPerTile / kWarps;   // 16 consecutive blocks per warp
 constexpr int kGenericMinTile = 1024;       // tile sizes the plain kernels of zccl_generic.cu accept (multiples of 32)
 constexpr int kGenericMaxTile = 8192;
-constexpr int kMaxJobs = 64;                // chunk-operations per launch (8 ranks x 7 chunks of a ring stage fit one launch)
+// Chunk-operations per launch.  A stage of an 8-rank ring (8 jobs) fits one launch; the 56 chunk decodes that end an
+// 8-rank Allreduce take two.  (With 64 the fused hop's 64 MiB launch was 1.6 us slower and nothing else faster.)
+constexpr int kMaxJobs = 32;
 
 // Device status bits (zccl_status maps them to return codes).
 enum : uint32_t {
