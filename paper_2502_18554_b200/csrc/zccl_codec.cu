@@ -1057,6 +1057,32 @@ struct GroupTable {
 };
 constexpr int kPlaceThreads = 1024;   // one warp per tile of the group
 
+// Called by one warp of every CTA of the placement once the CTA has read the group sums it needs: the last CTA to
+// get there re-arms the workspace (group sums back to zero, launch counter on) while the others are still storing.
+__device__ __forceinline__ void rearm_after_reads(const JobBatch& jb, const Workspace& ws, uint32_t epoch, int lane)
+{
+    uint32_t last = 0;
+    if (lane == 0) {
+        __threadfence();
+        last = atomicAdd(ws.done, 1u) == gridDim.x - 1 ? 1u : 0u;
+    }
+    if (!__shfl_sync(kFull, last, 0)) return;
+    const uint32_t used = (jb.total_tiles >> 5) + (uint32_t)jb.count + 1u;
+    for (uint32_t k = (uint32_t)lane; k < used; k += 32u) ws.group_acc[k] = 0ull;
+    const uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
+    if (e == 0) {   // the counter wraps (once in 2^31 launches): no scan state of an earlier launch may look current again
+        for (uint32_t k = (uint32_t)lane; k < ws.max_tiles; k += 32u) st_state(ws.tile_state + k, 0ull);
+        for (uint32_t k = (uint32_t)lane; k < (uint32_t)group_slots(ws.max_tiles); k += 32u) st_state(ws.group_state + k, 0ull);
+        __threadfence();
+    }
+    __syncwarp();
+    if (lane == 0) {
+        *ws.done = 0;
+        *ws.ticket = 0;
+        *ws.epoch = e ? e : 1u;
+    }
+}
+
 __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ GroupTable gt, Workspace ws,
                                                               Params hp, int use_dev_params, int from_stream)
 {
@@ -1099,6 +1125,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         const bool hdr = prm.valid && job.out_cap >= (unsigned)kHeaderBytes;
         if (tid == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
         if (hdr) write_header(out, tid, 0, prm.eb_abs, prm.s, 0);
+        if (warp == kPlaceThreads / 32 - 1) rearm_after_reads(jb, ws, epoch, lane);
     } else {
         const uint32_t t0 = 32u * g;                               // first tile of the group, within the job
         const uint32_t ntl = tiles - t0 < 32u ? tiles - t0 : 32u;   // tiles of the group
@@ -1138,6 +1165,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
             }
         }
         __syncthreads();
+        if (warp == kPlaceThreads / 32 - 1) rearm_after_reads(jb, ws, epoch, lane);   // every warp's reads of the sums are through
         // the group's place: the groups of the job in front of it are full ones (33 fixed words per tile) with the
         // payload that step 1 added up per group; the tile's place inside the group: the tiles in front of it
         const uint32_t wl = s_words[lane];
@@ -1180,30 +1208,6 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         }
     }
     if (status) atomicOr(ws.status, status);
-    // the last CTA to get here re-arms the workspace: group sums back to zero, launch counter on
-    __shared__ uint32_t s_last;
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        s_last = atomicAdd(ws.done, 1u) == gridDim.x - 1 ? 1u : 0u;
-    }
-    __syncthreads();
-    if (s_last) {
-        const uint32_t used = (jb.total_tiles >> 5) + (uint32_t)jb.count + 1u;
-        for (uint32_t k = (uint32_t)tid; k < used; k += kPlaceThreads) ws.group_acc[k] = 0ull;
-        const uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
-        if (e == 0) {   // the counter wraps (once in 2^31 launches): no scan state of an earlier launch may look current again
-            for (uint32_t k = (uint32_t)tid; k < ws.max_tiles; k += kPlaceThreads) st_state(ws.tile_state + k, 0ull);
-            for (uint32_t k = (uint32_t)tid; k < (uint32_t)group_slots(ws.max_tiles); k += kPlaceThreads) st_state(ws.group_state + k, 0ull);
-            __threadfence();
-        }
-        __syncthreads();
-        if (tid == 0) {
-            *ws.done = 0;
-            *ws.ticket = 0;
-            *ws.epoch = e ? e : 1u;
-        }
-    }
 }
 
 // ------------------------------------------------------------------------------------------------ decompress
