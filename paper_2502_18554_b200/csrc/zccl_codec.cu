@@ -1056,6 +1056,8 @@ struct GroupTable {
     uint32_t begin[kMaxJobs + 1];   // first group (= CTA) of each job; begin[count] = number of groups
 };
 constexpr int kPlaceThreads = 1024;   // one warp per tile of the group
+constexpr int kPlaceHeadWords = 320;  // payload words of a round that are fetched before its size is known (code lengths up to 9 on average)
+constexpr size_t kPlaceSmemBytes = (size_t)(kPlaceThreads / 32) * kRoundsPerTile * kPlaceHeadWords * 4;
 
 // Called by one warp of every CTA of the placement once the CTA has read the group sums it needs: the last CTA to
 // get there re-arms the workspace (group sums back to zero, launch counter on) while the others are still storing.
@@ -1089,7 +1091,15 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
     // What this kernel reads before it waits for step 1 is older than step 1's launch: job table, the incoming
     // streams' headers, the resolved bound.
     __shared__ uint32_t s_words[32], s_part[kPlaceThreads / 32];
+    __shared__ alignas(8) unsigned long long s_bar[kPlaceThreads / 32];
+    extern __shared__ __align__(16) unsigned char place_smem[];   // per warp: the first 1024 payload bytes of its tile's four rounds
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t* stage = reinterpret_cast<uint32_t*>(place_smem) + (size_t)warp * (kRoundsPerTile * kPlaceHeadWords);
+    if (lane == 0) {
+        mbar_init(&s_bar[warp], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
     uint32_t status = 0;
     Params prm = hp;
     if (use_dev_params) prm = *ws.params;
@@ -1140,12 +1150,11 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         const uint4 nq4 = *reinterpret_cast<const uint4*>(ws.round_words + 4u * T);
         const uint32_t lword = slot[(size_t)(lane >> 3) * kRoundSlotWords + (lane & 7)];   // code-length word `lane` of the tile
         const uint32_t first = (uint32_t)ws.outliers[T];
-        uint32_t v[kRoundsPerTile][8];
+        if (mine && lane == 0) {   // the copy engine brings the heads of the four payloads: four requests instead of 32 loads per lane
+            mbar_expect_tx(&s_bar[warp], kRoundsPerTile * kPlaceHeadWords * 4);
 #pragma unroll
-        for (int q = 0; q < kRoundsPerTile; ++q) {
-            const uint32_t* __restrict__ src = slot + (size_t)q * kRoundSlotWords + 8;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) v[q][k] = src[lane + 32 * k];
+            for (int q = 0; q < kRoundsPerTile; ++q)
+                bulk_load(stage + q * kPlaceHeadWords, slot + (size_t)q * kRoundSlotWords + 8, kPlaceHeadWords * 4, &s_bar[warp]);
         }
         unsigned long long part = 0;
         {
@@ -1187,17 +1196,18 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
                 if (lane == 0) dst[0] = first;
                 if ((uint32_t)lane < tpadw) dst[1 + lane] = lword;
                 uint32_t* __restrict__ d = dst + 1 + tpadw;
+                if (!mbar_wait(&s_bar[warp], 0u)) status |= kStTimeout;
 #pragma unroll
                 for (int q = 0; q < kRoundsPerTile; ++q) {
                     const uint32_t nq = nqs[q];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
+                    for (int k = 0; k < kPlaceHeadWords / 32; ++k) {
                         const uint32_t i = (uint32_t)lane + 32u * k;
-                        if (i < nq) d[i] = v[q][k];
+                        if (i < nq) d[i] = stage[q * kPlaceHeadWords + i];
                     }
-                    if (nq > 256u) {   // code lengths beyond 7 on average: the rest of the round
+                    if (nq > (uint32_t)kPlaceHeadWords) {   // code lengths beyond 7 on average: the rest of the round
                         const uint32_t* __restrict__ src = slot + (size_t)q * kRoundSlotWords + 8;
-                        for (uint32_t i = 256u + (uint32_t)lane; i < nq; i += 32) d[i] = src[i];
+                        for (uint32_t i = (uint32_t)kPlaceHeadWords + (uint32_t)lane; i < nq; i += 32) d[i] = src[i];
                     }
                     d += nq;
                 }
@@ -2060,6 +2070,8 @@ cudaError_t device_setup(const DeviceSetup** out)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_kernel, kCodecThreads, kDecSmemBytes);
         if (e != cudaSuccess) return e;
         d.dec_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPlaceSmemBytes);
+        if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(hop_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
         if (e != cudaSuccess) return e;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, hop_tiles_kernel, kCodecThreads, kHopSmemBytes);
@@ -2124,7 +2136,7 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     e = launch_k(hop_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws,
                  split_shift);
     if (e != cudaSuccess) return e;
-    return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
+    return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
 }
 
 cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
@@ -2162,7 +2174,7 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
         e = launch_k(encode_rounds_kernel, dim3((unsigned)(want_a < cap_a ? want_a : cap_a)), dim3(kCodecThreads), kRoundSmemBytes, st, jb, maps, ws,
                      host_params, device_params ? 1 : 0);
         if (e != cudaSuccess) return e;
-        return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), 0, st, jb, gt, ws, host_params, device_params ? 1 : 0, 0);
+        return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, host_params, device_params ? 1 : 0, 0);
     }
     const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     unsigned long long cap = (unsigned long long)sm_count * d->enc_ctas;
