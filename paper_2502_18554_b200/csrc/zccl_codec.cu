@@ -1056,7 +1056,7 @@ struct GroupTable {
     uint32_t begin[kMaxJobs + 1];   // first group (= CTA) of each job; begin[count] = number of groups
 };
 constexpr int kPlaceThreads = 1024;   // one warp per tile of the group
-constexpr int kPlaceHeadWords = 320;  // payload words of a round that are fetched before its size is known (code lengths up to 9 on average)
+constexpr int kPlaceHeadWords = 288;  // payload words of a round that are fetched before its size is known (code lengths up to 8 on average); measured best of 192 ... 448
 constexpr size_t kPlaceSmemBytes = (size_t)(kPlaceThreads / 32) * kRoundsPerTile * kPlaceHeadWords * 4;
 
 // Called by one warp of every CTA of the placement once the CTA has read the group sums it needs: the last CTA to
