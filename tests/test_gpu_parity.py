@@ -944,3 +944,33 @@ def test_launches_from_several_threads(z):
     for t in threads:
         t.join()
     assert not errors, errors
+
+
+@pytest.mark.parametrize("tiles", [3, 40, 200, 700])
+def test_large_blobs_are_staged_a_window_at_a_time(z, ctx, tiles):
+    """Tiles whose blobs are larger than a 4 KiB staging buffer (code lengths 9 to 24, up to 12 KiB per tile): the
+    decoder and the hop move a window over them; few tiles make the hop start its warps inside tiles (units of one or
+    two rounds, which skip over the rounds in front through the window), many make it take whole tiles.  Both operands
+    compressed as well (the second one is read in place)."""
+    n = tiles * 4096 - 777
+    rng = np.random.default_rng(tiles)
+    scale = np.repeat(10.0 ** rng.uniform(-0.5, 4.0, (n + 1023) // 1024), 1024)[:n]      # the code length changes from round to round
+    a = (rng.standard_normal(n) * scale).astype(np.float32)
+    b = (rng.standard_normal(n) * scale[::-1]).astype(np.float32)
+    ea, s, r = oracle.resolve(oracle.EB_ABS, 2e-3)
+    sa, _ = oracle.compress_core(a, ea, s, r)
+    assert sa.size > 1.5 * 4096 * tiles                                                 # blobs above the buffer on average
+    got_y, rcd = gpu_decompress(z, ctx, sa, n)
+    assert rcd == z.OK
+    assert_same_bits(got_y, oracle.decompress(sa))
+    want, wrc, wraw = oracle.drc(sa, local=b, want_raw=True)
+    got, rc, raw = _drc_gpu(z, ctx, sa, n, local=b, raw=True)
+    assert rc == wrc and np.array_equal(got, want)
+    assert_same_bits(raw, wraw)
+    sb, _ = oracle.compress_core(b, ea, s, r)
+    want2, wrc2 = oracle.drc(sa, local_c=sb)
+    got2, rc2, _ = _drc_gpu(z, ctx, sa, n, local_c=sb)
+    assert rc2 == wrc2 and np.array_equal(got2, want2)
+    # and the compressor on the same data
+    st, rcc = gpu_compress(z, ctx, a, z.EB_ABS, 2e-3)
+    assert np.array_equal(st, sa)
