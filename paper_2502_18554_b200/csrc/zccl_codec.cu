@@ -1188,6 +1188,9 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
             const unsigned long long word0 = (unsigned long long)kHeaderWords + nT + base + my_off;
             const bool fits = (word0 + words) * 4ull <= job.out_cap;
             if (!fits) status |= kStCapacity;
+            // the copies into this warp's shared memory land before anything else happens (also when the tile does not fit:
+            // a CTA must not end with copies into its shared memory still on their way)
+            if (!mbar_wait(&s_bar[warp], 0u)) status |= kStTimeout;
             if (fits && placed) {
                 uint32_t* __restrict__ dst = out + word0;
                 const unsigned long long tleft = n - (unsigned long long)tile * kTile;
@@ -1196,7 +1199,6 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
                 if (lane == 0) dst[0] = first;
                 if ((uint32_t)lane < tpadw) dst[1 + lane] = lword;
                 uint32_t* __restrict__ d = dst + 1 + tpadw;
-                if (!mbar_wait(&s_bar[warp], 0u)) status |= kStTimeout;
 #pragma unroll
                 for (int q = 0; q < kRoundsPerTile; ++q) {
                     const uint32_t nq = nqs[q];
