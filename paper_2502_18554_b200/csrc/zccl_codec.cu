@@ -923,6 +923,17 @@ __device__ __forceinline__ void cursor_settle(TileCursor& c, const JobBatch& jb,
 __global__ void __launch_bounds__(kCodecThreads, 4) encode_rounds_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
                                                                          Workspace ws, Params hp, int use_dev_params)
 {
+    // Before the kernel in front on the stream is waited for: the warp's first two rounds are asked into L2.  (A prefetch
+    // only moves lines into L2, which stays coherent with whatever that kernel still writes.)
+    if ((threadIdx.x & 31) == 0) {
+        const uint32_t rd0 = threadIdx.x >> 5;
+        for (uint32_t t = blockIdx.x, k = 0; k < 2 && t < jb.total_tiles; ++k, t += gridDim.x) {
+            const int j = find_job(jb, t);
+            const Job& q = jb.job[j];
+            const unsigned long long e = (unsigned long long)(t - q.tile_begin) * kTile + (unsigned long long)rd0 * kRound;
+            if (q.x && (((uintptr_t)q.x) & 15u) == 0 && e + kRound <= q.n) bulk_prefetch_l2(q.x + e, 4u * kRound);
+        }
+    }
     pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
