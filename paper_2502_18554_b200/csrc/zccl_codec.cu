@@ -1741,6 +1741,7 @@ __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, cons
 // maps: tensor map of job j's uncompressed operand at [j] and, in launches of at most kMaxJobs / 2 jobs, of its
 // uncompressed result at [kMaxJobs / 2 + j] (a second array of maps made the parameters 22 KB and the launch 1.6 us
 // slower; launches with more jobs write such results with plain stores).
+template <bool C2, bool Y>
 __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
                                                                      Workspace ws, uint32_t split_shift)
 {
@@ -1774,7 +1775,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
             cj_count = (cj + 1 < jb.count ? jb.job[cj + 1].tile_begin : jb.total_tiles) - cj_begin;
             h1 = read_header(q.in_c, q.in_cap);
             job_ok = h1.ok && h1.n == q.n;
-            if (q.in_c2) {
+            if (C2 && q.in_c2) {
                 h2 = read_header(q.in_c2, q.in2_cap);
                 job_ok = job_ok && h2.ok && h2.n == q.n && __float_as_uint(h2.s) == __float_as_uint(h1.s);
             }
@@ -1885,7 +1886,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
                 blob1 = win.base;
                 mode1 = describe_blob(blob1, cur.words, nb, lane);   // the head (at most 33 words) is in every first window
             }
-            if (job.in_c2) {
+            if (C2 && job.in_c2) {
                 const BlobRef b2 = blob_of(job.in_c2, job.in2_cap, hc2.nT, tile);
                 blob2 = b2.ptr;
                 mode2 = b2.ptr ? describe_blob(b2.ptr, b2.words, nb, lane) : 0;
@@ -1895,8 +1896,8 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
         const bool good = len != 0 && mode1 != 0 && mode2 != 0;
 
         uint32_t pay1 = 0, pay2 = 0;
-        int32_t code1 = good ? (int32_t)blob1[0] : 0, code2 = (good && blob2) ? (int32_t)blob2[0] : 0;
-        const uint32_t lp1 = good ? lane_code_lengths(blob1, nb, lane) : 0u, lp2 = (good && blob2) ? lane_code_lengths(blob2, nb, lane) : 0u;
+        int32_t code1 = good ? (int32_t)blob1[0] : 0, code2 = (C2 && good && blob2) ? (int32_t)blob2[0] : 0;
+        const uint32_t lp1 = good ? lane_code_lengths(blob1, nb, lane) : 0u, lp2 = (C2 && good && blob2) ? lane_code_lengths(blob2, nb, lane) : 0u;
         // moves the window over the incoming blob to round e's first word when the round reaches past its end
         auto reach = [&](uint32_t e) {
             const uint32_t L = (lp1 >> (8u * e)) & 0xFFu;
@@ -1933,10 +1934,10 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
             for (uint32_t e = 0; e < rd_first; ++e) {
                 const uint32_t Le = reach(e);
                 skip_round(blob1, padw, Le, &pay1, &code1, lane);
-                if (blob2) skip_round(blob2, padw, (lp2 >> (8u * e)) & 0xFFu, &pay2, &code2, lane);
+                if (C2 && blob2) skip_round(blob2, padw, (lp2 >> (8u * e)) & 0xFFu, &pay2, &code2, lane);
             }
             const float xa = __fmul_rn(__int2float_rn(code1), s);
-            const float xb = blob2 ? __fmul_rn(__int2float_rn(code2), s) : __ldg(job.x + start + rd_first * (uint32_t)kRound - 1u);
+            const float xb = (C2 && blob2) ? __fmul_rn(__int2float_rn(code2), s) : __ldg(job.x + start + rd_first * (uint32_t)kRound - 1u);
             carry_y = combine(op, xa, xb);
         }
         for (uint32_t rd = rd_first; rd < rd_stop; ++rd) {
@@ -1958,7 +1959,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
                 if (lane == 0) ws.round_words[u] = 0;
             } else {
                 arrive_loc(pl);
-                if (blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
+                if (C2 && blob2) {   // the operand is compressed too: its round goes where an uncompressed one would be
                     const uint32_t L2 = (lp2 >> (8u * rd)) & 0xFFu;
                     if (mode2 == 1) decode_round_classes<0>(blob2, padw, L2, &pay2, &code2, s, loc, lane, nullptr, 0u);
                     else decode_round_general(blob2, padw, L2, &pay2, &code2, s, loc, lane, nullptr, 0u);
@@ -1983,7 +1984,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
                 carry_y = read_last_of_row(ys, 31);
                 const uint32_t e0 = rd * (uint32_t)kRound;
                 uint32_t* slot = ws.slots + (size_t)u * kRoundSlotWords;
-                if (job.y) {   // an uncompressed copy of the result leaves the stage before the encoder writes over it
+                if (Y && job.y) {   // an uncompressed copy of the result leaves the stage before the encoder writes over it
                     const uint32_t count = len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound;
                     if (deq) store_round_dequantised(job.y + start + e0, ys, count, r, s, lane);
                     else if (jb.count <= kMaxJobs / 2 && (((uintptr_t)job.y) & 15u) == 0 && count == (uint32_t)kRound) {
@@ -2085,9 +2086,12 @@ cudaError_t device_setup(const DeviceSetup** out)
         d.dec_ctas = a > 0 ? a : 1;
         e = cudaFuncSetAttribute(place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPlaceSmemBytes);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(hop_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
+        e = cudaFuncSetAttribute(hop_tiles_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(hop_tiles_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(hop_tiles_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(hop_tiles_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
         if (e != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, hop_tiles_kernel, kCodecThreads, kHopSmemBytes);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, hop_tiles_kernel<true, true>, kCodecThreads, kHopSmemBytes);
         if (e != cudaSuccess) return e;
         d.hop_ctas = a > 0 ? a : 1;
         d.ready = true;
@@ -2146,8 +2150,15 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     const unsigned long long warps = cap * kCodecWarps;
     const uint32_t split_shift = 4ull * jb.total_tiles <= warps ? 2u : 2ull * jb.total_tiles <= warps ? 1u : 0u;
     const unsigned long long want = ((((unsigned long long)jb.total_tiles) << split_shift) + kCodecWarps - 1) / kCodecWarps;
-    e = launch_k(hop_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws,
-                 split_shift);
+    // the kernel comes in four forms: with or without the code for a compressed second operand and for an uncompressed
+    // copy of the result, which most hops of a ring do not have
+    bool c2 = false, y = false;
+    for (int j = 0; j < jb.count; ++j) { c2 = c2 || jb.job[j].in_c2 != nullptr; y = y || jb.job[j].y != nullptr; }
+    const dim3 grid((unsigned)(want < cap ? want : cap));
+    if (c2 && y) e = launch_k(hop_tiles_kernel<true, true>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
+    else if (c2) e = launch_k(hop_tiles_kernel<true, false>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
+    else if (y) e = launch_k(hop_tiles_kernel<false, true>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
+    else e = launch_k(hop_tiles_kernel<false, false>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
     if (e != cudaSuccess) return e;
     return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
 }
