@@ -1741,10 +1741,11 @@ __device__ __noinline__ void store_round_dequantised(float* __restrict__ y, cons
 // maps: tensor map of job j's uncompressed operand at [j] and, in launches of at most kMaxJobs / 2 jobs, of its
 // uncompressed result at [kMaxJobs / 2 + j] (a second array of maps made the parameters 22 KB and the launch 1.6 us
 // slower; launches with more jobs write such results with plain stores).
-template <bool C2, bool Y>
+template <bool C2, bool Y, bool SPLIT>
 __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
-                                                                     Workspace ws, uint32_t split_shift)
+                                                                     Workspace ws, uint32_t split_shift_arg)
 {
+    const uint32_t split_shift = SPLIT ? split_shift_arg : 0u;   // SPLIT false: whole tiles only, known when the kernel is compiled
     // split_shift 0: a warp's unit of work is a tile; 1: two rounds; 2: a round (small launches: more warps at work, and
     // none of them walks four rounds in a row)
     pdl_enter();
@@ -2051,6 +2052,23 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode_tiled = nullptr;   // the driver's cuTensorMapEncodeTiled, looked up through the runtime
 
+// The eight forms of the hop kernel (see hop_tiles_kernel's template parameters), by index 4 C2 + 2 Y + SPLIT.
+using HopLaunch = cudaError_t (*)(dim3, cudaStream_t, const JobBatch&, const TileMaps&, const Workspace&, uint32_t);
+template <bool C2, bool Y, bool SPLIT>
+cudaError_t hop_launch(dim3 grid, cudaStream_t st, const JobBatch& jb, const TileMaps& maps, const Workspace& ws, uint32_t split_shift)
+{
+    return launch_k(hop_tiles_kernel<C2, Y, SPLIT>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
+}
+inline HopLaunch hop_form(bool c2, bool y, bool split)
+{
+    static const HopLaunch forms[8] = {hop_launch<false, false, false>, hop_launch<false, false, true>, hop_launch<false, true, false>,
+                                       hop_launch<false, true, true>,   hop_launch<true, false, false>, hop_launch<true, false, true>,
+                                       hop_launch<true, true, false>,   hop_launch<true, true, true>};
+    return forms[(c2 ? 4 : 0) + (y ? 2 : 0) + (split ? 1 : 0)];
+}
+template <bool C2, bool Y, bool SPLIT>
+cudaError_t hop_smem_attr() { return cudaFuncSetAttribute(hop_tiles_kernel<C2, Y, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes); }
+
 cudaError_t device_setup(const DeviceSetup** out)
 {
     int dev = 0;
@@ -2086,12 +2104,16 @@ cudaError_t device_setup(const DeviceSetup** out)
         d.dec_ctas = a > 0 ? a : 1;
         e = cudaFuncSetAttribute(place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPlaceSmemBytes);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(hop_tiles_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(hop_tiles_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(hop_tiles_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(hop_tiles_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHopSmemBytes);
+        e = hop_smem_attr<false, false, false>();
+        if (e == cudaSuccess) e = hop_smem_attr<false, false, true>();
+        if (e == cudaSuccess) e = hop_smem_attr<false, true, false>();
+        if (e == cudaSuccess) e = hop_smem_attr<false, true, true>();
+        if (e == cudaSuccess) e = hop_smem_attr<true, false, false>();
+        if (e == cudaSuccess) e = hop_smem_attr<true, false, true>();
+        if (e == cudaSuccess) e = hop_smem_attr<true, true, false>();
+        if (e == cudaSuccess) e = hop_smem_attr<true, true, true>();
         if (e != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, hop_tiles_kernel<true, true>, kCodecThreads, kHopSmemBytes);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, hop_tiles_kernel<true, true, true>, kCodecThreads, kHopSmemBytes);
         if (e != cudaSuccess) return e;
         d.hop_ctas = a > 0 ? a : 1;
         d.ready = true;
@@ -2150,15 +2172,12 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     const unsigned long long warps = cap * kCodecWarps;
     const uint32_t split_shift = 4ull * jb.total_tiles <= warps ? 2u : 2ull * jb.total_tiles <= warps ? 1u : 0u;
     const unsigned long long want = ((((unsigned long long)jb.total_tiles) << split_shift) + kCodecWarps - 1) / kCodecWarps;
-    // the kernel comes in four forms: with or without the code for a compressed second operand and for an uncompressed
-    // copy of the result, which most hops of a ring do not have
+    // the kernel comes in eight forms: with or without the code for a compressed second operand, for an uncompressed copy
+    // of the result, and for units that start inside tiles, none of which the hop of a large chunk has
     bool c2 = false, y = false;
     for (int j = 0; j < jb.count; ++j) { c2 = c2 || jb.job[j].in_c2 != nullptr; y = y || jb.job[j].y != nullptr; }
     const dim3 grid((unsigned)(want < cap ? want : cap));
-    if (c2 && y) e = launch_k(hop_tiles_kernel<true, true>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
-    else if (c2) e = launch_k(hop_tiles_kernel<true, false>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
-    else if (y) e = launch_k(hop_tiles_kernel<false, true>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
-    else e = launch_k(hop_tiles_kernel<false, false>, grid, dim3(kCodecThreads), kHopSmemBytes, st, jb, maps, ws, split_shift);
+    e = hop_form(c2, y, split_shift != 0)(grid, st, jb, maps, ws, split_shift);
     if (e != cudaSuccess) return e;
     return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
 }
