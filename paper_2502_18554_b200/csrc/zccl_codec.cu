@@ -1564,12 +1564,24 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
         BlobRef br;
         br.ptr = nullptr; br.words = 0; br.staged = false;
         if (t >= jb.total_tiles) return br;
+        // the tile's index entries are asked for before the job's header is looked at (they need only the job table), so that
+        // a warp's first tile waits for one round trip, not two
+        uint32_t w_end = 0, w_beg = 0;
+        {
+            const bool same = t - cj_begin < cj_count;
+            const int jn = same ? cj : find_job(jb, t);
+            const Job& qn = jb.job[jn];
+            const uint32_t tl = t - qn.tile_begin;
+            if ((unsigned long long)kHeaderBytes + 4ull * ((unsigned long long)tl + 1ull) <= qn.in_cap) {
+                const uint32_t* idx = qn.in_c + kHeaderWords;
+                w_end = ldg_u32(idx + tl);
+                w_beg = tl ? ldg_u32(idx + tl - 1) : 0u;
+            }
+        }
         enter_job(t);
         const Job& q = jb.job[cj];
         const uint32_t tile = t - cj_begin;
         if (!h.ok || h.n > q.n || tile >= h.nT) return br;
-        const uint32_t* idx = q.in_c + kHeaderWords;
-        const uint32_t w_end = ldg_u32(idx + tile), w_beg = tile ? ldg_u32(idx + tile - 1) : 0u;
         const unsigned long long blob0 = (unsigned long long)kHeaderWords + h.nT;
         if (w_end <= w_beg || (blob0 + w_end) * 4ull > q.in_cap) { br.words = 0xFFFFFFFFu; return br; }   // marks a damaged index
         br.ptr = q.in_c + blob0 + w_beg;
