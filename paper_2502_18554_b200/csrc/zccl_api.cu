@@ -515,9 +515,13 @@ int zccl_sim_allgather(zccl_ctx* c, const float* const* send, float* const* recv
             ChainJob& j = cb.job[r];
             j.src0 = (const uint32_t*)gslot(r, r); j.bytes = own_sz + r; j.first_rank = (r + 1) % N; j.chunk = r;
         }
-        if ((rc = cuda_rc(launch_copy_chain(cb, c->ws, c->sm_count, st))) != ZCCL_OK) return rc;
+        // own contributions stay uncompressed: their copies ride along in the forwarding launch when they fit its grid
+        CopyBatcher own;
+        if (N <= kMaxJobs)
+            for (int r = 0; r < N; ++r) own.add_fixed(send[r], recv[r] + (size_t)r * n, sizeof(float) * n);
+        if ((rc = cuda_rc(launch_copy_chain(cb, c->ws, c->sm_count, st, N <= kMaxJobs ? &own.cb : nullptr))) != ZCCL_OK) return rc;
     }
-    {   // own contributions stay uncompressed: one launch copies them all
+    if (N == 1 || N > kMaxJobs) {   // ... or take a launch of their own
         CopyBatcher cb;
         for (int r = 0; r < N; ++r) {
             cb.add_fixed(send[r], recv[r] + (size_t)r * n, sizeof(float) * n);

@@ -184,7 +184,8 @@ cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, 
 constexpr int kQualityCtas = 1024;
 cudaError_t launch_quality(const float* x, const float* y, unsigned long long n, double* out, double* partials,
                            uint32_t* counter, int sm_count, cudaStream_t st);
-cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st);
+// extra: plain copies that ride along in the same launch (or nullptr)
+cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st, const CopyBatch* extra = nullptr);
 unsigned long long launch_count();
 void count_launches(unsigned k);   // adds to the process-wide count of kernels this library has launched
 

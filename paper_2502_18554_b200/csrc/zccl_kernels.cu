@@ -129,10 +129,8 @@ __global__ void __launch_bounds__(256) range_kernel(RangeBatch rb, Workspace ws)
 // ------------------------------------------------------------------------------------------------ blob copy
 
 // One forwarding hop of compressed bytes whose length lives on the device (grid.y = job).
-__global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
+__device__ __forceinline__ void copy_job(const CopyJob& job, const Workspace& ws)
 {
-    pdl_enter();
-    const CopyJob& job = cb.job[blockIdx.y];
     const unsigned long long bytes = job.bytes ? *job.bytes : job.fixed_bytes;
     if (bytes > job.cap) {
         if (threadIdx.x == 0 && blockIdx.x == 0) { atomicOr(ws.status, kStCapacity); if (job.bytes_out) *job.bytes_out = 0; }
@@ -153,13 +151,24 @@ __global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
     for (unsigned long long i = done_words + tid; i < words; i += nth) job.dst[i] = __ldg(job.src + i);
     if (tid == 0 && job.bytes_out) *job.bytes_out = (size_t)bytes;
 }
+__global__ void __launch_bounds__(256) copy_kernel(CopyBatch cb, Workspace ws)
+{
+    pdl_enter();
+    copy_job(cb.job[blockIdx.y], ws);
+}
 
 // Every forwarding hop of an Allgather stage (grid.y = chain).  A thread carries its 16-byte pieces through all the
 // hops: each hop loads the piece from where the previous hop stored it (the same thread's own store, so no
 // synchronisation is needed) and stores it into the next rank's slot.
-__global__ void __launch_bounds__(256) copy_chain_kernel(ChainBatch cb, Workspace ws)
+// Rows of the grid beyond the chains are plain copies (`extra`): what else a collective has to move at that point goes
+// along in the same launch.
+__global__ void __launch_bounds__(256) copy_chain_kernel(ChainBatch cb, CopyBatch extra, Workspace ws)
 {
     pdl_enter();
+    if ((int)blockIdx.y >= cb.count) {
+        copy_job(extra.job[blockIdx.y - cb.count], ws);
+        return;
+    }
     const ChainJob& job = cb.job[blockIdx.y];
     const unsigned long long bytes = *job.bytes;
     const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -457,12 +466,17 @@ cudaError_t launch_stream_stats(const uint32_t* in, unsigned long long cap_bytes
     return launch_k(stream_stats_kernel, dim3((unsigned)sm_count * 2), dim3(256), 0, st, in, cap_bytes, hist, ws);
 }
 
-cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st)
+cudaError_t launch_copy_chain(const ChainBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st, const CopyBatch* extra)
 {
-    if (cb.count <= 0 || cb.hops == 0) return cudaSuccess;
-    unsigned gx = (unsigned)((sm_count * 4 + cb.count - 1) / cb.count);
+    static const CopyBatch none{};
+    const int more = extra ? extra->count : 0;
+    if ((cb.count <= 0 || cb.hops == 0) && more == 0) return cudaSuccess;
+    ChainBatch chains = cb;
+    if (cb.hops == 0) chains.count = 0;
+    const int rows = chains.count + more;
+    unsigned gx = (unsigned)((sm_count * 4 + rows - 1) / rows);
     ++g_launches;
-    return launch_k(copy_chain_kernel, dim3(gx ? gx : 1, cb.count), dim3(256), 0, st, cb, ws);
+    return launch_k(copy_chain_kernel, dim3(gx ? gx : 1, rows), dim3(256), 0, st, chains, extra ? *extra : none, ws);
 }
 
 }  // namespace zccl
