@@ -1096,8 +1096,11 @@ __device__ __forceinline__ void rearm_after_reads(const JobBatch& jb, const Work
     }
 }
 
+// from_stream: 0 = a compression (bound in hp, or on the device), 1 = a hop (bound and step from the incoming stream's
+// header), 2 = a compression of binary64 input (bound in hp64, or on the device; the header carries the step as one
+// binary64).
 __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ GroupTable gt, Workspace ws,
-                                                              Params hp, int use_dev_params, int from_stream)
+                                                              Params hp, int use_dev_params, int from_stream, ParamsF64 hp64)
 {
     // What this kernel reads before it waits for step 1 is older than step 1's launch: job table, the incoming
     // streams' headers, the resolved bound.
@@ -1113,7 +1116,22 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
     __syncwarp();
     uint32_t status = 0;
     Params prm = hp;
-    if (use_dev_params) prm = *ws.params;
+    double step64 = hp64.s;
+    if (from_stream == 2) {
+        if (use_dev_params) { const ParamsF64 p = *ws.params64; step64 = p.s; prm.valid = p.valid; }
+        else prm.valid = hp64.valid;
+    } else if (use_dev_params) prm = *ws.params;
+    auto put_header = [&](uint32_t* out, int who, unsigned long long n, uint32_t nT) {
+        if (from_stream != 2) { write_header(out, who, n, prm.eb_abs, prm.s, nT); return; }
+        if (who < kHeaderWords) {
+            const uint32_t words[kHeaderWords] = {kMagic, kVersionF64, (uint32_t)n, (uint32_t)(n >> 32), (uint32_t)__double2loint(step64),
+                                                  (uint32_t)__double2hiint(step64), (uint32_t)kTile, nT};
+            uint32_t hv = words[0];
+#pragma unroll
+            for (int k = 1; k < kHeaderWords; ++k) hv = who == k ? words[k] : hv;
+            out[who] = hv;
+        }
+    };
 
     int j = 0;
     {
@@ -1125,7 +1143,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
         j = lo;
     }
     const Job& job = jb.job[j];
-    if (from_stream) {   // a hop: bound and step are the incoming stream's, and the job counts only if its streams agree with it
+    if (from_stream == 1) {   // a hop: bound and step are the incoming stream's, and the job counts only if its streams agree with it
         const StreamInfo h1 = read_header(job.in_c, job.in_cap);
         bool ok = h1.ok && h1.n == job.n;
         if (job.in_c2) {
@@ -1145,7 +1163,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
     if (n == 0 || !prm.valid) {   // a job without elements, or no valid bound: header and length only
         const bool hdr = prm.valid && job.out_cap >= (unsigned)kHeaderBytes;
         if (tid == 0) *job.out_bytes = hdr ? kHeaderBytes : 0;
-        if (hdr) write_header(out, tid, 0, prm.eb_abs, prm.s, 0);
+        if (hdr) put_header(out, tid, 0, 0);
         if (warp == kPlaceThreads / 32 - 1) rearm_after_reads(jb, ws, epoch, lane);
     } else {
         const uint32_t t0 = 32u * g;                               // first tile of the group, within the job
@@ -1227,7 +1245,7 @@ __global__ void __launch_bounds__(kPlaceThreads) place_kernel(const __grid_const
                 if (lane == 0) out[kHeaderWords + tile] = base + my_off + words;
             }
             if (lane == 0 && tile == nT - 1) *job.out_bytes = (size_t)((word0 + words) * 4ull);
-            if (tile == 0) write_header(out, lane, n, prm.eb_abs, prm.s, nT);
+            if (tile == 0) put_header(out, lane, n, nT);
         }
     }
     if (status) atomicOr(ws.status, status);
@@ -2048,15 +2066,19 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
     if (status) atomicOr(ws.status, status);
 }
 
+#include "zccl_codec_f64.cuh"
+
 // Per-device launch set-up (shared-memory attribute, resident CTAs per SM), done once per device under a lock.
 constexpr int kMaxDevices = 64;
 constexpr size_t kEncSmemBytes = sizeof(EncWarpShared) * kCodecWarps + 1024;   // + room to reach a 1024-byte boundary
 constexpr size_t kRoundSmemBytes = sizeof(RoundWarpShared) * kCodecWarps + 1024;
 constexpr size_t kDecSmemBytes = sizeof(DecWarpShared) * kCodecWarps + 1024;
 constexpr size_t kHopSmemBytes = sizeof(HopWarpShared) * kCodecWarps + 1024;
+constexpr size_t kRound64SmemBytes = sizeof(RoundWarpShared64) * kCodecWarps + 1024;
+constexpr size_t kDec64SmemBytes = sizeof(DecWarpShared64) * kCodecWarps + 1024;
 struct DeviceSetup {
     bool ready = false;
-    int enc_ctas = 1, round_ctas = 1, dec_ctas = 1, hop_ctas = 1;
+    int enc_ctas = 1, round_ctas = 1, dec_ctas = 1, hop_ctas = 1, round64_ctas = 1, dec64_ctas = 1;
 };
 DeviceSetup g_dev[kMaxDevices];
 std::mutex g_dev_mu;
@@ -2128,6 +2150,16 @@ cudaError_t device_setup(const DeviceSetup** out)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, hop_tiles_kernel<true, true, true>, kCodecThreads, kHopSmemBytes);
         if (e != cudaSuccess) return e;
         d.hop_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(encode_rounds_f64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRound64SmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_rounds_f64_kernel, kCodecThreads, kRound64SmemBytes);
+        if (e != cudaSuccess) return e;
+        d.round64_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(decode_tiles_f64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDec64SmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_f64_kernel, kCodecThreads, kDec64SmemBytes);
+        if (e != cudaSuccess) return e;
+        d.dec64_ctas = a > 0 ? a : 1;
         d.ready = true;
     }
     *out = &d;
@@ -2144,6 +2176,20 @@ cudaError_t make_row_map(CUtensorMap* map, const float* x, unsigned long long n)
     const cuuint32_t box[2] = {(cuuint32_t)kBlock, 32u};
     const cuuint32_t estr[2] = {1u, 1u};
     const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(x), dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// The array x of n doubles as rows of 16 doubles, copied in tiles of 64 rows with the 128-byte swizzle.
+cudaError_t make_row_map_f64(CUtensorMap* map, const double* x, unsigned long long n)
+{
+    if ((((uintptr_t)x) & 15u) != 0 || n < 16ull) return cudaSuccess;
+    const cuuint64_t dims[2] = {16u, (cuuint64_t)(n / 16ull)};
+    const cuuint64_t strides[1] = {16u * sizeof(double)};
+    const cuuint32_t box[2] = {16u, (cuuint32_t)kRowsPerRound64};
+    const cuuint32_t estr[2] = {1u, 1u};
+    const CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 2, const_cast<double*>(x), dims, strides, box, estr,
                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
@@ -2191,7 +2237,7 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     const dim3 grid((unsigned)(want < cap ? want : cap));
     e = hop_form(c2, y, split_shift != 0)(grid, st, jb, maps, ws, split_shift);
     if (e != cudaSuccess) return e;
-    return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1);
+    return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1, ParamsF64{0.0, 1.0, 1.0, 1});
 }
 
 cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
@@ -2229,12 +2275,60 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
         e = launch_k(encode_rounds_kernel, dim3((unsigned)(want_a < cap_a ? want_a : cap_a)), dim3(kCodecThreads), kRoundSmemBytes, st, jb, maps, ws,
                      host_params, device_params ? 1 : 0);
         if (e != cudaSuccess) return e;
-        return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, host_params, device_params ? 1 : 0, 0);
+        return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, host_params, device_params ? 1 : 0, 0, ParamsF64{0.0, 1.0, 1.0, 1});
     }
     const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     unsigned long long cap = (unsigned long long)sm_count * d->enc_ctas;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
     return launch_k(enc_kernel, dim3(grid), dim3(kCodecThreads), kEncSmemBytes, st, jb, maps, ws, host_params, device_params ? 1 : 0);
+}
+
+// Binary64 input, array on a 16-byte boundary: rounds into their slots, then the placement (two launches).
+cudaError_t launch_encode_f64_lanes(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* out,
+                                    unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    const DeviceSetup* d = nullptr;
+    cudaError_t e = device_setup(&d);
+    if (e != cudaSuccess) return e;
+    if (!ws.slots || (((uintptr_t)x) & 15u) != 0) return cudaErrorInvalidValue;
+    CUtensorMap map;
+    memset(&map, 0, sizeof(map));
+    if ((e = make_row_map_f64(&map, x, n)) != cudaSuccess) return e;
+    const unsigned long long nT = (n + kTile - 1) / kTile;
+    thread_local JobBatch jb;
+    memset(&jb, 0, sizeof(jb));
+    jb.count = 1;
+    jb.total_tiles = (uint32_t)(nT ? nT : 1);
+    jb.job[0].x = reinterpret_cast<const float*>(x);
+    jb.job[0].out = out; jb.job[0].out_bytes = out_bytes; jb.job[0].n = n; jb.job[0].out_cap = out_cap;
+    if (jb.total_tiles > ws.max_tiles) return cudaErrorInvalidValue;
+    GroupTable gt;
+    const uint32_t groups = group_table(jb, gt);
+    const unsigned long long cap = (unsigned long long)sm_count * d->round64_ctas;
+    const unsigned grid = (unsigned)(jb.total_tiles < cap ? jb.total_tiles : cap);
+    e = launch_k(encode_rounds_f64_kernel, dim3(grid), dim3(kCodecThreads), kRound64SmemBytes, st, x, n, jb.total_tiles, map, ws, hp,
+                 device_params ? 1 : 0);
+    if (e != cudaSuccess) return e;
+    return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, device_params ? 1 : 0, 2,
+                    hp);
+}
+
+cudaError_t launch_decode_f64_lanes(const uint32_t* in, unsigned long long cap_bytes, double* y, unsigned long long y_cap, const Workspace& ws,
+                                    int sm_count, cudaStream_t st)
+{
+    const DeviceSetup* d = nullptr;
+    cudaError_t e = device_setup(&d);
+    if (e != cudaSuccess) return e;
+    CUtensorMap map;
+    memset(&map, 0, sizeof(map));
+    const bool mapped = (((uintptr_t)y) & 15u) == 0 && y_cap >= 16ull;
+    if (mapped && (e = make_row_map_f64(&map, y, y_cap)) != cudaSuccess) return e;
+    const unsigned long long tiles = (y_cap + kTile - 1) / kTile;
+    if (tiles >= 0xFFFFFFFFull) return cudaErrorInvalidValue;
+    const unsigned long long want = (tiles + kCodecWarps - 1) / kCodecWarps;
+    const unsigned long long cap = (unsigned long long)sm_count * d->dec64_ctas;
+    return launch_k(decode_tiles_f64_kernel, dim3((unsigned)(want < cap ? (want ? want : 1) : cap)), dim3(kCodecThreads), kDec64SmemBytes, st, in,
+                    cap_bytes, y, y_cap, (uint32_t)tiles, map, mapped ? 1 : 0, ws);
 }
 
 }  // namespace zccl

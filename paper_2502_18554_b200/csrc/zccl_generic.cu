@@ -7,6 +7,8 @@
 // 1024 and 8192 elements.
 #include "zccl_internal.h"
 
+#include <cstdlib>
+
 namespace zccl {
 namespace {
 
@@ -357,11 +359,26 @@ __device__ void resolve_f64(double ea, bool range_ok, const Workspace& ws)
 __global__ void __launch_bounds__(256) range_f64_kernel(const double* __restrict__ x, unsigned long long n, double eb, Workspace ws)
 {
     double lo = __longlong_as_double(0x7FF0000000000000ll), hi = __longlong_as_double((long long)0xFFF0000000000000ull);
-    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (unsigned long long)gridDim.x * blockDim.x) {
-        const double v = __ldg(x + i);
-        lo = v < lo ? v : lo;
-        hi = v > hi ? v : hi;
+    auto take = [&](double v) { lo = v < lo ? v : lo; hi = v > hi ? v : hi; };
+    const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned long long nthreads = (unsigned long long)gridDim.x * blockDim.x;
+    // peel to a 16-byte boundary, then 128-bit loads, four of them in flight per thread
+    unsigned long long head = ((uintptr_t)x & 15u) ? 1u : 0u;
+    if (head > n) head = n;
+    if (tid < head) take(x[tid]);
+    const unsigned long long nvec = (n - head) >> 1;
+    const double2* xv = reinterpret_cast<const double2*>(x + head);
+    unsigned long long i = tid;
+    for (; i + 3 * nthreads < nvec; i += 4 * nthreads) {
+        const double2 a = __ldg(xv + i), b = __ldg(xv + i + nthreads), c = __ldg(xv + i + 2 * nthreads), d = __ldg(xv + i + 3 * nthreads);
+        take(a.x); take(a.y); take(b.x); take(b.y); take(c.x); take(c.y); take(d.x); take(d.y);
     }
+    for (; i < nvec; i += nthreads) {
+        const double2 v = __ldg(xv + i);
+        take(v.x); take(v.y);
+    }
+    const unsigned long long tail0 = head + (nvec << 1);
+    if (tail0 + tid < n) take(x[tail0 + tid]);
 #pragma unroll
     for (int s = 16; s; s >>= 1) {
         const double a = __shfl_xor_sync(kFull, lo, s), b = __shfl_xor_sync(kFull, hi, s);
@@ -429,9 +446,20 @@ cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_byt
     return generic_decode<float>(in, cap_bytes, T, y, y_cap, ws, sm_count, st);
 }
 
+// ZCCL_F64_PLAIN=1 in the environment keeps binary64 on the plain kernels (for comparison).
+static bool plain_f64_forced()
+{
+    static const bool forced = [] { const char* v = getenv("ZCCL_F64_PLAIN"); return v && v[0] == '1'; }();
+    return forced;
+}
+
 cudaError_t launch_encode_f64(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* sizes, uint32_t* go,
                               uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st)
 {
+    if (ws.slots && (((uintptr_t)x) & 15u) == 0 && (n + kTile - 1) / kTile <= ws.max_tiles && !plain_f64_forced()) {
+        count_launches(2);
+        return launch_encode_f64_lanes(x, n, hp, device_params, out, out_cap, out_bytes, ws, sm_count, st);
+    }
     return generic_encode<double>(x, n, (uint32_t)kTile, hp, device_params ? ws.params64 : nullptr, sizes, go, out, out_cap, out_bytes, ws,
                                   sm_count, st);
 }
@@ -439,12 +467,16 @@ cudaError_t launch_encode_f64(const double* x, unsigned long long n, ParamsF64 h
 cudaError_t launch_decode_f64(const uint32_t* in, unsigned long long cap_bytes, double* y, unsigned long long y_cap, const Workspace& ws,
                               int sm_count, cudaStream_t st)
 {
+    if (!plain_f64_forced()) {
+        count_launches(1);
+        return launch_decode_f64_lanes(in, cap_bytes, y, y_cap, ws, sm_count, st);
+    }
     return generic_decode<double>(in, cap_bytes, (uint32_t)kTile, y, y_cap, ws, sm_count, st);
 }
 
 cudaError_t launch_range_f64(const double* x, unsigned long long n, double eb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
-    const unsigned long long want = (n + 255) / 256;
+    const unsigned long long want = (n / 2 + 255) / 256;
     const unsigned cap = (unsigned)sm_count * 8u;
     count_launches(1);
     range_f64_kernel<<<(unsigned)(want < cap ? (want ? want : 1) : cap), 256, 0, st>>>(x, n, eb, ws);

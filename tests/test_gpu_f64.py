@@ -98,3 +98,88 @@ def test_errors(z, ctx):
     with pytest.raises(z.ZcclError):
         ctx.compress_f64(torch.zeros(8, dtype=torch.float64, device="cuda"), z.EB_ABS, 0.0,
                          torch.empty(1024, dtype=torch.uint8, device="cuda"), torch.zeros(1, dtype=torch.int64, device="cuda"))
+
+
+@pytest.mark.parametrize("n", [5000, 3 * 4096 + 1024, 3 * 4096 + 1025, 200_001])
+@pytest.mark.parametrize("shift_x,shift_y", [(1, 0), (0, 1), (1, 1)])
+def test_arrays_off_the_16_byte_boundary(z, ctx, n, shift_x, shift_y):
+    """Input or output that starts 8 bytes past a 16-byte boundary: the plain kernels (input) and the plain stores
+    (output) take over; streams and values stay those of the oracle."""
+    x = as_f64(fields.smooth_1d(n, seed=7), n + 1)
+    want = oracle.compress_f64(x, oracle.EB_ABS, 1e-5)
+    buf = torch.empty(n + 2, dtype=torch.float64, device="cuda")
+    dx = buf[shift_x: shift_x + n]
+    dx.copy_(torch.from_numpy(x))
+    assert dx.data_ptr() % 16 == 8 * shift_x
+    out = torch.empty(z.compress_bound(n), dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx.compress_f64(dx, z.EB_ABS, 1e-5, out, nb)
+    assert ctx.status() == z.OK
+    assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+    ybuf = torch.full((n + 2,), -7.0, dtype=torch.float64, device="cuda")
+    y = ybuf[shift_y: shift_y + n]
+    ctx.decompress_f64(torch.from_numpy(want.copy()).cuda(), y)
+    assert ctx.status() == z.OK
+    assert np.array_equal(y.cpu().numpy().view(np.uint64), oracle.decompress_f64(want).view(np.uint64))
+    edge = ybuf.cpu().numpy()
+    assert all(edge[k] == -7.0 for k in list(range(shift_y)) + list(range(shift_y + n, n + 2)))   # nothing written outside
+
+
+@pytest.mark.parametrize("scale,eb", [(1.0, 1e-3), (1.0, 1e-6), (3e3, 1e-4), (5e4, 1e-3)])
+def test_noise_of_every_width(z, ctx, scale, eb):
+    """Uncorrelated values: code lengths from a few bits up to 31 (the general route), blobs larger than the decoder's
+    window, mixed with smooth tiles and constant ones."""
+    rng = np.random.default_rng(11)
+    n = 40 * 4096 + 777
+    x = rng.standard_normal(n) * scale
+    x[3 * 4096: 5 * 4096] = fields.smooth_1d(2 * 4096, seed=3).astype(np.float64)
+    x[9 * 4096: 10 * 4096] = 0.25
+    x[20 * 4096 + 100: 20 * 4096 + 164] = 1e-9          # a constant block inside a wide tile
+    got, y, rc = gpu_round_trip(z, ctx, x, z.EB_ABS, eb)
+    want = oracle.compress_f64(x, oracle.EB_ABS, eb)
+    assert rc == z.OK
+    assert np.array_equal(got, want)
+    assert np.array_equal(y.view(np.uint64), oracle.decompress_f64(want).view(np.uint64))
+    assert float(np.abs(x - y).max()) <= eb
+
+
+def test_range_error_inside_a_large_array(z, ctx):
+    x = fields.smooth_1d(100_000, seed=5).astype(np.float64)
+    x[77_777] = 1e12
+    _, _, rc = gpu_round_trip(z, ctx, x, z.EB_ABS, 1e-3)
+    assert rc == z.E_RANGE
+    x[77_777] = np.nan
+    _, _, rc = gpu_round_trip(z, ctx, x, z.EB_ABS, 1e-3)
+    assert rc == z.E_RANGE
+
+
+def test_damaged_streams_are_refused(z, ctx):
+    x = as_f64(fields.smooth_1d(30_000, seed=9), 4)
+    good = oracle.compress_f64(x, oracle.EB_ABS, 1e-5)
+    y = torch.empty(x.size, dtype=torch.float64, device="cuda")
+
+    def status_of(stream, cap=None):
+        d = torch.from_numpy(stream.copy()).cuda()
+        ctx.decompress_f64(d if cap is None else d[:cap], y)
+        return ctx.status()
+
+    assert status_of(good) == z.OK
+    words = good.view(np.uint32).copy()
+    bad = words.copy(); bad[8 + 2] = bad[8 + 1]                       # an index entry that does not grow
+    assert status_of(bad.view(np.uint8)) == z.E_BAD_STREAM
+    nT = int(words[7])
+    bad = words.copy(); bad[8 + nT + 1] |= 0x20                       # a code length of 32 or more in tile 0
+    assert status_of(bad.view(np.uint8)) == z.E_BAD_STREAM
+    assert status_of(good, cap=len(good) - 64) == z.E_BAD_STREAM     # the last blob reaches past the readable bytes
+    small = torch.empty(x.size - 1, dtype=torch.float64, device="cuda")
+    ctx.decompress_f64(torch.from_numpy(good.copy()).cuda(), small)
+    assert ctx.status() == z.E_CAPACITY
+
+
+def test_output_capacity_too_small(z, ctx):
+    x = np.random.default_rng(3).standard_normal(50_000)
+    dx = torch.from_numpy(x).cuda()
+    out = torch.empty(40_000, dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx.compress_f64(dx, z.EB_ABS, 1e-6, out, nb)
+    assert ctx.status() == z.E_CAPACITY
