@@ -338,8 +338,10 @@ int zccl_scale(zccl_ctx* ctx, float* y, size_t n, float divisor, void* stream);
  *   codes     q_i = nearest integer, ties to even, of fl64(x_i * r); RANGE unless every |x_i * r| < 2^30
  *   values    x'_i = fl64((double)q_i * s); |x_i - x'_i| <= eb_abs for every code in range (no precision warning)
  * The stream's version word carries data type 1 and header bytes 16..23 hold the step as one binary64; binary32
- * entry points reject such a stream and the other way round (BAD_STREAM).  Plain kernels (three launches to compress,
- * one to decompress), 8 bytes per element read or written.
+ * entry points reject such a stream and the other way round (BAD_STREAM).  Two launches to compress (rounds into the
+ * context's slots, then the placement) and one to decompress, on kernels of the same design as the binary32 ones; an
+ * input that does not start on a 16-byte boundary is compressed by plain kernels instead (three launches, several
+ * times slower), an output off that boundary is written with plain stores.
  *   x [device] n doubles, 8-byte aligned; y [device] receives n doubles; the rest as for zccl_compress / zccl_decompress.
  * Errors as for those two; ZCCL_E_DEGENERATE at once for a relative bound with n == 0.
  */
