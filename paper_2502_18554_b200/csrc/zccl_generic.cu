@@ -356,22 +356,26 @@ __device__ void resolve_f64(double ea, bool range_ok, const Workspace& ws)
     *ws.params64 = p;
     if (!p.valid) atomicOr(ws.status, kStDegenerate);
 }
-__global__ void __launch_bounds__(256) range_f64_kernel(const double* __restrict__ x, unsigned long long n, double eb, Workspace ws)
+__global__ void __launch_bounds__(512, 2) range_f64_kernel(const double* __restrict__ x, unsigned long long n, double eb, Workspace ws)
 {
     double lo = __longlong_as_double(0x7FF0000000000000ll), hi = __longlong_as_double((long long)0xFFF0000000000000ull);
     auto take = [&](double v) { lo = v < lo ? v : lo; hi = v > hi ? v : hi; };
     const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     const unsigned long long nthreads = (unsigned long long)gridDim.x * blockDim.x;
-    // peel to a 16-byte boundary, then 128-bit loads, four of them in flight per thread
+    // peel to a 16-byte boundary, then 128-bit loads, eight of them in flight per thread
     unsigned long long head = ((uintptr_t)x & 15u) ? 1u : 0u;
     if (head > n) head = n;
     if (tid < head) take(x[tid]);
     const unsigned long long nvec = (n - head) >> 1;
     const double2* xv = reinterpret_cast<const double2*>(x + head);
     unsigned long long i = tid;
-    for (; i + 3 * nthreads < nvec; i += 4 * nthreads) {
-        const double2 a = __ldg(xv + i), b = __ldg(xv + i + nthreads), c = __ldg(xv + i + 2 * nthreads), d = __ldg(xv + i + 3 * nthreads);
-        take(a.x); take(a.y); take(b.x); take(b.y); take(c.x); take(c.y); take(d.x); take(d.y);
+    constexpr int kInFlight = 8;
+    for (; i + (kInFlight - 1) * nthreads < nvec; i += kInFlight * nthreads) {
+        double2 v[kInFlight];
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k) v[k] = __ldcs(xv + i + k * nthreads);
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k) { take(v[k].x); take(v[k].y); }
     }
     for (; i < nvec; i += nthreads) {
         const double2 v = __ldg(xv + i);
@@ -385,10 +389,14 @@ __global__ void __launch_bounds__(256) range_f64_kernel(const double* __restrict
         lo = a < lo ? a : lo;
         hi = b > hi ? b : hi;
     }
+    // one pair of keys per CTA (an atomic on one address costs about 1.5 ns, whoever issues it: large CTAs, few of them)
     __shared__ uint32_t last_s;
-    if ((threadIdx.x & 31) == 0 && lo <= hi) { atomicMin(ws.minmax64 + 0, d2key(lo)); atomicMax(ws.minmax64 + 1, d2key(hi)); }
+    __shared__ double s_lo[32], s_hi[32];
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
     __syncthreads();
     if (threadIdx.x == 0) {
+        for (unsigned w = 1; w < (blockDim.x >> 5); ++w) { lo = s_lo[w] < lo ? s_lo[w] : lo; hi = s_hi[w] > hi ? s_hi[w] : hi; }
+        if (lo <= hi) { atomicMin(ws.minmax64 + 0, d2key(lo)); atomicMax(ws.minmax64 + 1, d2key(hi)); }
         __threadfence();
         last_s = atomicAdd(ws.done, 1u) == gridDim.x - 1 ? 1u : 0u;
     }
@@ -476,10 +484,10 @@ cudaError_t launch_decode_f64(const uint32_t* in, unsigned long long cap_bytes, 
 
 cudaError_t launch_range_f64(const double* x, unsigned long long n, double eb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
-    const unsigned long long want = (n / 2 + 255) / 256;
-    const unsigned cap = (unsigned)sm_count * 8u;
+    const unsigned long long want = (n / 2 + 511) / 512;
+    const unsigned cap = (unsigned)sm_count * 2u;
     count_launches(1);
-    range_f64_kernel<<<(unsigned)(want < cap ? (want ? want : 1) : cap), 256, 0, st>>>(x, n, eb, ws);
+    range_f64_kernel<<<(unsigned)(want < cap ? (want ? want : 1) : cap), 512, 0, st>>>(x, n, eb, ws);
     return cudaGetLastError();
 }
 
