@@ -183,3 +183,71 @@ def test_output_capacity_too_small(z, ctx):
     nb = torch.zeros(1, dtype=torch.int64, device="cuda")
     ctx.compress_f64(dx, z.EB_ABS, 1e-6, out, nb)
     assert ctx.status() == z.E_CAPACITY
+
+
+def _draw_f64_case(seed):
+    """Length, values (several kinds, some unkind to the codec), bound and the two arrays' offsets from a 16-byte
+    boundary, from one seed."""
+    rng = np.random.default_rng(seed)
+    pick = rng.random()
+    if pick < 0.15:
+        n = int(rng.integers(1, 70))
+    elif pick < 0.45:
+        n = int(rng.integers(1, 9)) * 4096 + int(rng.integers(-40, 41))
+    else:
+        n = int(rng.integers(100, 300_000))
+    kind = int(rng.integers(0, 6))
+    if kind == 0:
+        x = fields.smooth_1d(n, seed=int(rng.integers(1 << 30))).astype(np.float64) * (1 + 1e-11 * rng.standard_normal(n))
+    elif kind == 1:
+        x = rng.normal(0.0, 10.0 ** rng.uniform(-3, 3), n)
+    elif kind == 2:
+        x = np.repeat(rng.normal(0, 1, n // 50 + 1), 50)[:n]
+    elif kind == 3:
+        x = fields.smooth_1d(n, seed=int(rng.integers(1 << 30))).astype(np.float64)
+        for _ in range(int(rng.integers(1, 6))):
+            a = int(rng.integers(0, max(n - 1, 1)))
+            b = min(n, a + int(rng.integers(1, 3000)))
+            x[a:b] += rng.normal(0, 10.0 ** rng.uniform(-2, 1), b - a)
+    elif kind == 4:
+        x = 10.0 ** rng.uniform(0, 4) + rng.normal(0, 1e-2, n)
+    else:
+        x = rng.normal(0, 1e-300, n)
+        x[rng.random(n) < 0.2] = 0.0
+        x[rng.random(n) < 0.1] = -0.0
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    span = float(x.max() - x.min())
+    if span == 0.0 or rng.random() < 0.5:
+        # an absolute bound that keeps |x / (2 eb)| below 2^30, from coarse to nearly that fine
+        floor = max(float(np.abs(x).max()), 1e-300) / 2.0 ** 29
+        mode, eb = oracle.EB_ABS, float(floor * 10.0 ** rng.uniform(0.1, 7))
+    else:
+        mode, eb = oracle.EB_REL, float(10.0 ** rng.uniform(-8, -1))
+    return x, mode, eb, int(rng.integers(0, 2)), int(rng.integers(0, 2))
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_seeded_random_cases(z, ctx, seed):
+    x, mode, eb, shift_x, shift_y = _draw_f64_case(1000 + seed)
+    n = x.size
+    try:
+        want = oracle.compress_f64(x, mode, eb)
+    except oracle.OracleError as e:
+        want = e
+    buf = torch.empty(n + 2, dtype=torch.float64, device="cuda")
+    dx = buf[shift_x: shift_x + n]
+    dx.copy_(torch.from_numpy(x))
+    out = torch.empty(z.compress_bound(n), dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx.compress_f64(dx, mode, eb, out, nb)
+    rc = ctx.status()
+    if isinstance(want, Exception):
+        assert rc == want.code          # the oracle's status codes are the library's
+        return
+    assert rc == z.OK
+    assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+    ybuf = torch.zeros(n + 2, dtype=torch.float64, device="cuda")
+    y = ybuf[shift_y: shift_y + n]
+    ctx.decompress_f64(out[: int(nb.item())], y)
+    assert ctx.status() == z.OK
+    assert np.array_equal(y.cpu().numpy().view(np.uint64), oracle.decompress_f64(want).view(np.uint64))
