@@ -38,6 +38,9 @@
 // A single-pass encoder (enc_kernel: a warp per tile, positions by a two-level decoupled look-back over per-tile and
 // per-group states, every wait bounded and reported through the status word) remains for contexts without slots:
 // the allocation-free entry point.
+//
+// Binary64 input has kernels of the same design with 8 KiB rounds (zccl_codec_f64.cuh, included below; they share
+// the back ends, the slots and place_kernel).
 #include "zccl_device.cuh"
 
 #include <cuda.h>
