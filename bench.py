@@ -349,7 +349,7 @@ def config_table(args):
         x1, loc1 = fields.fourier_field_3d(SIDE, seed=1), fields.fourier_field_3d(SIDE, seed=2)
         for eb in (1e-2, 1e-3, 1e-4):
             emit(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, orc and eb == 1e-3, loc1))
-        emit(_tiled_row(z, big, "cfg1, tile of 5120 (plain kernels)", x1, z.EB_REL, 1e-3, 5120))
+        emit(_tiled_row(z, big, "cfg1, tile of 5120", x1, z.EB_REL, 1e-3, 5120))
     if "cfg3" in want:
         emit(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, orc))
 

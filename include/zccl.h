@@ -271,8 +271,11 @@ int zccl_quality(zccl_ctx* ctx, const float* x, const float* y, size_t n, double
 /*
  * Other tile sizes.  The tile (elements per Lorenzo restart and per index entry) is a header field of the stream;
  * Section 3.5.2 cuts the data into chunks of 5120 points.  The entry points above are built around 4096; these two
- * take any tile size that is a multiple of 32 between 1024 and 8192, through plain kernels (three launches to
- * compress, one to decompress) that produce and accept exactly the streams the format defines for that tile size.
+ * take any tile size that is a multiple of 32 between 1024 and 8192 and produce and accept exactly the streams the
+ * format defines for that tile size: two launches to compress and one to decompress, on kernels of the same design
+ * as those for 4096 (a tile is ceil(tile / 1024) rounds of 1024 elements; the context's round slots cover every
+ * n <= max_elems when the tile size is a multiple of 1024, and n <= max_elems * 4 * tile / (4096 * ceil(tile / 1024))
+ * otherwise; larger inputs are compressed by plain kernels, three launches and several times slower).
  * Arguments, asynchrony and error reporting are those of zccl_compress and zccl_decompress; a stream whose header
  * names another tile size than `tile` sets ZCCL_E_BAD_STREAM.  ZCCL_E_ARG also for a tile size outside the range.
  * zccl_compress_bound_tiled returns 0 for such a tile size.

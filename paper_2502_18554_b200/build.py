@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libzccl.so"
 SOURCES = [CSRC / "zccl_kernels.cu", CSRC / "zccl_codec.cu", CSRC / "zccl_api.cu", CSRC / "zccl_noalloc.cu", CSRC / "zccl_generic.cu"]
-HEADERS = [CSRC / "zccl_internal.h", CSRC / "zccl_device.cuh", CSRC / "zccl_codec_f64.cuh", PKG.parent / "include" / "zccl.h"]
+HEADERS = [CSRC / "zccl_internal.h", CSRC / "zccl_device.cuh", CSRC / "zccl_codec_f64.cuh", CSRC / "zccl_codec_tiled.cuh", PKG.parent / "include" / "zccl.h"]
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

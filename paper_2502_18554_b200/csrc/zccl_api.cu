@@ -218,7 +218,7 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
     const size_t off_state = 0;
     const size_t off_group = off_state + 8 * max_tiles;
     const size_t off_acc = off_group + 8 * (size_t)group_slots(max_tiles);
-    const size_t off_small = align_up(off_acc + 8 * (size_t)group_slots(max_tiles), 256);
+    const size_t off_small = align_up(off_acc + 8 * (size_t)group_slots(4 * max_tiles), 256);   // groups of 32 tiles of 1024 elements at most
     const size_t off_sizes = off_small + 256;
     const size_t off_quality = align_up(off_sizes + sizeof(size_t) * (size_t)(c->sim_sizes_cap + 1), 256);
     const size_t small_bytes = off_quality + sizeof(double) * 4 * (size_t)kQualityCtas + 256;
@@ -253,7 +253,7 @@ int zccl_ctx_create(zccl_ctx** out, size_t max_elems, int max_ranks)
     if (ok) {
         const size_t off_rw = align_up(max_tiles * 4 * (size_t)kRoundSlotWords * 4, 256);
         const size_t off_ol = align_up(off_rw + max_tiles * 4 * 4, 256);
-        ok = cudaMalloc(&c->slot_block, off_ol + max_tiles * 4) == cudaSuccess;
+        ok = cudaMalloc(&c->slot_block, off_ol + max_tiles * 4 * 4) == cudaSuccess;   // a first code per tile, tiles of 1024 elements at most
         if (ok) {
             uint8_t* b = (uint8_t*)c->slot_block;
             c->ws.slots = (uint32_t*)b;

@@ -1075,7 +1075,8 @@ constexpr size_t kPlaceSmemBytes = (size_t)(kPlaceThreads / 32) * kRoundsPerTile
 
 // Called by one warp of every CTA of the placement once the CTA has read the group sums it needs: the last CTA to
 // get there re-arms the workspace (group sums back to zero, launch counter on) while the others are still storing.
-__device__ __forceinline__ void rearm_after_reads(const JobBatch& jb, const Workspace& ws, uint32_t epoch, int lane)
+// `used`: group sums the launch may have touched.
+__device__ __forceinline__ void rearm_groups(uint32_t used, const Workspace& ws, uint32_t epoch, int lane)
 {
     uint32_t last = 0;
     if (lane == 0) {
@@ -1083,7 +1084,6 @@ __device__ __forceinline__ void rearm_after_reads(const JobBatch& jb, const Work
         last = atomicAdd(ws.done, 1u) == gridDim.x - 1 ? 1u : 0u;
     }
     if (!__shfl_sync(kFull, last, 0)) return;
-    const uint32_t used = (jb.total_tiles >> 5) + (uint32_t)jb.count + 1u;
     for (uint32_t k = (uint32_t)lane; k < used; k += 32u) ws.group_acc[k] = 0ull;
     const uint32_t e = (epoch + 1u) & 0x7FFFFFFFu;
     if (e == 0) {   // the counter wraps (once in 2^31 launches): no scan state of an earlier launch may look current again
@@ -1097,6 +1097,11 @@ __device__ __forceinline__ void rearm_after_reads(const JobBatch& jb, const Work
         *ws.ticket = 0;
         *ws.epoch = e ? e : 1u;
     }
+}
+
+__device__ __forceinline__ void rearm_after_reads(const JobBatch& jb, const Workspace& ws, uint32_t epoch, int lane)
+{
+    rearm_groups((jb.total_tiles >> 5) + (uint32_t)jb.count + 1u, ws, epoch, lane);
 }
 
 // from_stream: 0 = a compression (bound in hp, or on the device), 1 = a hop (bound and step from the incoming stream's
@@ -2070,6 +2075,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) hop_tiles_kernel(const __gri
 }
 
 #include "zccl_codec_f64.cuh"
+#include "zccl_codec_tiled.cuh"
 
 // Per-device launch set-up (shared-memory attribute, resident CTAs per SM), done once per device under a lock.
 constexpr int kMaxDevices = 64;
@@ -2081,7 +2087,7 @@ constexpr size_t kRound64SmemBytes = sizeof(RoundWarpShared64) * kCodecWarps + 1
 constexpr size_t kDec64SmemBytes = sizeof(DecWarpShared64) * kCodecWarps + 1024;
 struct DeviceSetup {
     bool ready = false;
-    int enc_ctas = 1, round_ctas = 1, dec_ctas = 1, hop_ctas = 1, round64_ctas = 1, dec64_ctas = 1;
+    int enc_ctas = 1, round_ctas = 1, dec_ctas = 1, hop_ctas = 1, round64_ctas = 1, dec64_ctas = 1, round_tiled_ctas = 1, dec_tiled_ctas = 1;
 };
 DeviceSetup g_dev[kMaxDevices];
 std::mutex g_dev_mu;
@@ -2163,6 +2169,16 @@ cudaError_t device_setup(const DeviceSetup** out)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_f64_kernel, kCodecThreads, kDec64SmemBytes);
         if (e != cudaSuccess) return e;
         d.dec64_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(encode_rounds_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRoundSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_rounds_tiled_kernel, kCodecThreads, kRoundSmemBytes);
+        if (e != cudaSuccess) return e;
+        d.round_tiled_ctas = a > 0 ? a : 1;
+        e = cudaFuncSetAttribute(decode_tiles_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_tiled_kernel, kCodecThreads, kDecSmemBytes);
+        if (e != cudaSuccess) return e;
+        d.dec_tiled_ctas = a > 0 ? a : 1;
         d.ready = true;
     }
     *out = &d;
@@ -2332,6 +2348,59 @@ cudaError_t launch_decode_f64_lanes(const uint32_t* in, unsigned long long cap_b
     const unsigned long long cap = (unsigned long long)sm_count * d->dec64_ctas;
     return launch_k(decode_tiles_f64_kernel, dim3((unsigned)(want < cap ? (want ? want : 1) : cap)), dim3(kCodecThreads), kDec64SmemBytes, st, in,
                     cap_bytes, y, y_cap, (uint32_t)tiles, map, mapped ? 1 : 0, ws);
+}
+
+// Binary32 at another tile size on the tuned kernels: rounds into their slots, then the placement.  False when the
+// context's slots do not cover the launch (the caller then takes the plain kernels).
+bool tiled_lanes_fit(unsigned long long n, uint32_t T, const Workspace& ws)
+{
+    const unsigned long long tiles = (n + T - 1) / T, R = (T + kRound - 1) / kRound;
+    return ws.slots && tiles * R <= 4ull * ws.max_tiles;   // one slot per round; first codes and group sums are laid out for tiles of 1024
+}
+
+cudaError_t launch_encode_tiled_lanes(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* out,
+                                      unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    const DeviceSetup* d = nullptr;
+    cudaError_t e = device_setup(&d);
+    if (e != cudaSuccess) return e;
+    if (!tiled_lanes_fit(n, T, ws)) return cudaErrorInvalidValue;
+    CUtensorMap map;
+    memset(&map, 0, sizeof(map));
+    const bool mapped = (((uintptr_t)x) & 15u) == 0 && n >= (unsigned long long)kBlock;
+    if (mapped && (e = make_row_map(&map, x, n)) != cudaSuccess) return e;
+    TiledShape sp;
+    sp.T = T; sp.R = (T + kRound - 1) / kRound; sp.lw_full = (T / kBlock + 3) / 4;
+    const unsigned long long nT = (n + T - 1) / T;
+    const uint32_t tiles = (uint32_t)(nT ? nT : 1);
+    const unsigned long long rounds = (unsigned long long)tiles * sp.R;
+    const unsigned long long want = (rounds + kCodecWarps - 1) / kCodecWarps;
+    const unsigned long long cap = (unsigned long long)sm_count * d->round_tiled_ctas;
+    e = launch_k(encode_rounds_tiled_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kRoundSmemBytes, st, x, n, sp, tiles, map,
+                 mapped ? 1 : 0, ws, hp, device_params ? 1 : 0);
+    if (e != cudaSuccess) return e;
+    return launch_k(place_tiled_kernel, dim3((tiles + 31u) / 32u), dim3(kPlaceThreads), 0, st, out, out_cap, out_bytes, n, sp, tiles, ws, hp,
+                    device_params ? 1 : 0);
+}
+
+cudaError_t launch_decode_tiled_lanes(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, float* y, unsigned long long y_cap,
+                                      const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    const DeviceSetup* d = nullptr;
+    cudaError_t e = device_setup(&d);
+    if (e != cudaSuccess) return e;
+    CUtensorMap map;
+    memset(&map, 0, sizeof(map));
+    const bool mapped = (((uintptr_t)y) & 15u) == 0 && y_cap >= (unsigned long long)kBlock;
+    if (mapped && (e = make_row_map(&map, y, y_cap)) != cudaSuccess) return e;
+    TiledShape sp;
+    sp.T = T; sp.R = (T + kRound - 1) / kRound; sp.lw_full = (T / kBlock + 3) / 4;
+    const unsigned long long tiles = (y_cap + T - 1) / T;
+    if (tiles >= 0xFFFFFFFFull) return cudaErrorInvalidValue;
+    const unsigned long long want = (tiles + kCodecWarps - 1) / kCodecWarps;
+    const unsigned long long cap = (unsigned long long)sm_count * d->dec_tiled_ctas;
+    return launch_k(decode_tiles_tiled_kernel, dim3((unsigned)(want < cap ? (want ? want : 1) : cap)), dim3(kCodecThreads), kDecSmemBytes, st, in,
+                    cap_bytes, sp, y, y_cap, (uint32_t)tiles, map, mapped ? 1 : 0, ws);
 }
 
 }  // namespace zccl

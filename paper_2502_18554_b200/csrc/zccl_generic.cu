@@ -441,30 +441,38 @@ static cudaError_t generic_decode(const uint32_t* in, unsigned long long cap_byt
     return cudaGetLastError();
 }
 
+// ZCCL_PLAIN=1 in the environment keeps other tile sizes and binary64 on the plain kernels of this file (for comparison).
+static bool plain_forced()
+{
+    static const bool forced = [] { const char* v = getenv("ZCCL_PLAIN"); return v && v[0] == '1'; }();
+    return forced;
+}
+
 cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* sizes,
                                   uint32_t* go, uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws,
                                   int sm_count, cudaStream_t st)
 {
+    if (tiled_lanes_fit(n, T, ws) && !plain_forced()) {
+        count_launches(2);
+        return launch_encode_tiled_lanes(x, n, T, hp, device_params, out, out_cap, out_bytes, ws, sm_count, st);
+    }
     return generic_encode<float>(x, n, T, hp, device_params ? ws.params : nullptr, sizes, go, out, out_cap, out_bytes, ws, sm_count, st);
 }
 
 cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, float* y, unsigned long long y_cap,
                                   const Workspace& ws, int sm_count, cudaStream_t st)
 {
+    if (!plain_forced()) {
+        count_launches(1);
+        return launch_decode_tiled_lanes(in, cap_bytes, T, y, y_cap, ws, sm_count, st);
+    }
     return generic_decode<float>(in, cap_bytes, T, y, y_cap, ws, sm_count, st);
-}
-
-// ZCCL_F64_PLAIN=1 in the environment keeps binary64 on the plain kernels (for comparison).
-static bool plain_f64_forced()
-{
-    static const bool forced = [] { const char* v = getenv("ZCCL_F64_PLAIN"); return v && v[0] == '1'; }();
-    return forced;
 }
 
 cudaError_t launch_encode_f64(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* sizes, uint32_t* go,
                               uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st)
 {
-    if (ws.slots && (((uintptr_t)x) & 15u) == 0 && (n + kTile - 1) / kTile <= ws.max_tiles && !plain_f64_forced()) {
+    if (ws.slots && (((uintptr_t)x) & 15u) == 0 && (n + kTile - 1) / kTile <= ws.max_tiles && !plain_forced()) {
         count_launches(2);
         return launch_encode_f64_lanes(x, n, hp, device_params, out, out_cap, out_bytes, ws, sm_count, st);
     }
@@ -475,7 +483,7 @@ cudaError_t launch_encode_f64(const double* x, unsigned long long n, ParamsF64 h
 cudaError_t launch_decode_f64(const uint32_t* in, unsigned long long cap_bytes, double* y, unsigned long long y_cap, const Workspace& ws,
                               int sm_count, cudaStream_t st)
 {
-    if (!plain_f64_forced()) {
+    if (!plain_forced()) {
         count_launches(1);
         return launch_decode_f64_lanes(in, cap_bytes, y, y_cap, ws, sm_count, st);
     }

@@ -733,7 +733,7 @@ def test_stream_stats_constant_and_damaged(z, ctx):
     assert ctx.status() == z.E_BAD_STREAM
 
 
-# ----------------------------------------------------------------------------- other tile sizes (plain kernels)
+# ----------------------------------------------------------------------------- other tile sizes
 
 def _tiled_case(z, ctx, x, mode, eb, T):
     want, wrc = oracle.compress(x, mode, eb, T)
@@ -762,6 +762,34 @@ def test_other_tile_sizes_match_oracle(z, ctx, T, n):
         x[n // 2: n // 2 + 1500] += np.random.default_rng(n).normal(0, 0.4, 1500).astype(f32)
     _tiled_case(z, ctx, x, z.EB_REL if n > 1 else z.EB_ABS, 1e-3, T)
     _tiled_case(z, ctx, x, z.EB_ABS, 3e-6, T)       # long codes, precision warning on the larger arrays
+
+
+@pytest.mark.parametrize("T", [5120, 1024, 7168, 4128])
+def test_other_tile_sizes_many_groups_and_alignments(z, T):
+    """Hundreds of tiles (several groups of 32 in the placement), wide and narrow code lengths side by side, input and
+    output on and off a 16-byte boundary; at T = 4128 the last array is too large for the context's round slots and
+    goes to the plain kernels."""
+    c = z.Context(1 << 21, 0)
+    try:
+        for n, shift in ((1 << 21, 0), ((1 << 20) + 4321, 1), (900_000, 3)):
+            x = fields.fourier_field_3d(128, seed=T % 7)[:n].copy()
+            x[n // 3: n // 3 + 70_000] += np.random.default_rng(T).normal(0, 0.3, 70_000).astype(f32)
+            want, wrc = oracle.compress(x, oracle.EB_REL, 1e-4, T)
+            buf = torch.empty(n + 4, dtype=torch.float32, device="cuda")
+            dx = buf[shift: shift + n]
+            dx.copy_(torch.from_numpy(x))
+            out = torch.empty(z.compress_bound_tiled(n, T), dtype=torch.uint8, device="cuda")
+            nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+            c.compress_tiled(dx, z.EB_REL, 1e-4, T, out, nb)
+            assert c.status() == wrc
+            assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+            ybuf = torch.full((n + 4,), 7.0, dtype=torch.float32, device="cuda")
+            c.decompress_tiled(out[: int(nb.item())], T, ybuf[shift: shift + n])
+            assert c.status() == z.OK
+            assert_same_bits(ybuf[shift: shift + n].cpu().numpy(), oracle.decompress(want))
+            assert bool((ybuf[:shift] == 7.0).all()) and bool((ybuf[shift + n:] == 7.0).all())
+    finally:
+        c.close()
 
 
 def test_tile_4096_streams_of_both_routes_are_the_same(z, ctx):
