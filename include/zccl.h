@@ -343,8 +343,7 @@ int zccl_scale(zccl_ctx* ctx, float* y, size_t n, float divisor, void* stream);
  * The stream's version word carries data type 1 and header bytes 16..23 hold the step as one binary64; binary32
  * entry points reject such a stream and the other way round (BAD_STREAM).  Two launches to compress (rounds into the
  * context's slots, then the placement) and one to decompress, on kernels of the same design as the binary32 ones; an
- * input that does not start on a 16-byte boundary is compressed by plain kernels instead (three launches, several
- * times slower), an output off that boundary is written with plain stores.
+ * array that does not start on a 16-byte boundary is read or written with plain accesses instead of the copy engine.
  *   x [device] n doubles, 8-byte aligned; y [device] receives n doubles; the rest as for zccl_compress / zccl_decompress.
  * Errors as for those two; ZCCL_E_DEGENERATE at once for a relative bound with n == 0.
  */

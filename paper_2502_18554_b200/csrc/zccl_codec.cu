@@ -2302,17 +2302,18 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
     return launch_k(enc_kernel, dim3(grid), dim3(kCodecThreads), kEncSmemBytes, st, jb, maps, ws, host_params, device_params ? 1 : 0);
 }
 
-// Binary64 input, array on a 16-byte boundary: rounds into their slots, then the placement (two launches).
+// Binary64 input: rounds into their slots, then the placement (two launches).
 cudaError_t launch_encode_f64_lanes(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* out,
                                     unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st)
 {
     const DeviceSetup* d = nullptr;
     cudaError_t e = device_setup(&d);
     if (e != cudaSuccess) return e;
-    if (!ws.slots || (((uintptr_t)x) & 15u) != 0) return cudaErrorInvalidValue;
+    if (!ws.slots) return cudaErrorInvalidValue;
     CUtensorMap map;
     memset(&map, 0, sizeof(map));
-    if ((e = make_row_map_f64(&map, x, n)) != cudaSuccess) return e;
+    const bool mapped = (((uintptr_t)x) & 15u) == 0 && n >= 16ull;
+    if (mapped && (e = make_row_map_f64(&map, x, n)) != cudaSuccess) return e;
     const unsigned long long nT = (n + kTile - 1) / kTile;
     thread_local JobBatch jb;
     memset(&jb, 0, sizeof(jb));
@@ -2325,8 +2326,8 @@ cudaError_t launch_encode_f64_lanes(const double* x, unsigned long long n, Param
     const uint32_t groups = group_table(jb, gt);
     const unsigned long long cap = (unsigned long long)sm_count * d->round64_ctas;
     const unsigned grid = (unsigned)(jb.total_tiles < cap ? jb.total_tiles : cap);
-    e = launch_k(encode_rounds_f64_kernel, dim3(grid), dim3(kCodecThreads), kRound64SmemBytes, st, x, n, jb.total_tiles, map, ws, hp,
-                 device_params ? 1 : 0);
+    e = launch_k(encode_rounds_f64_kernel, dim3(grid), dim3(kCodecThreads), kRound64SmemBytes, st, x, n, jb.total_tiles, map, mapped ? 1 : 0, ws,
+                 hp, device_params ? 1 : 0);
     if (e != cudaSuccess) return e;
     return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, device_params ? 1 : 0, 2,
                     hp);

@@ -10,7 +10,7 @@
 // A round is still 32 blocks = 1024 elements, now 8 KiB: the array is described to the copy engine as rows of 16
 // doubles (128 bytes, the widest row the 128-byte swizzle takes), a round is a box of 64 rows, and lane l owns rows
 // 2 l and 2 l + 1.  Chunk c (16 bytes = two doubles) of row t sits at chunk c ^ (t & 7) of that row.  Kernels here
-// take one array per launch, which must start on a 16-byte boundary (others go to the plain kernels).
+// take one array per launch; one that does not start on a 16-byte boundary is loaded with plain accesses.
 
 constexpr double kMagic52 = 6755399441055744.0;         // 1.5 * 2^52
 constexpr double kIntBias = 4503601774854144.0;         // 2^52 + 2^31
@@ -181,6 +181,17 @@ __device__ __noinline__ uint32_t encode_round_general_f64(const double* __restri
     return status;
 }
 
+// A full round of an array that the copy engine cannot take (not on a 16-byte boundary): plain coalesced loads into the
+// stage's layout.
+__device__ __noinline__ void load_round_plain_f64(double* stage, const double* __restrict__ xr, int lane)
+{
+#pragma unroll 4
+    for (uint32_t k = 0; k < 32u; ++k) {
+        const uint32_t e = 32u * k + (uint32_t)lane;
+        *reinterpret_cast<double*>(reinterpret_cast<char*>(stage) + stage_chunk_byte(e >> 4, (e & 15u) >> 1) + 8u * (e & 1u)) = __ldg(xr + e);
+    }
+}
+
 struct alignas(1024) RoundWarpShared64 {
     double stage[kStages64][kRound];           // 8 KiB each, on 1024-byte boundaries; a round is encoded in place and leaves from here
     alignas(16) double front[kStages64][2];    // the two elements in front of each stage's round
@@ -192,8 +203,8 @@ struct alignas(1024) RoundWarpShared64 {
 // in place and leaves by one bulk store to its slot, exactly as in encode_rounds_kernel; partial rounds (the end of
 // the array) take the general route.
 __global__ void __launch_bounds__(kCodecThreads, kStages64 == 2 ? 3 : 2) encode_rounds_f64_kernel(const double* __restrict__ x, unsigned long long n, uint32_t tiles,
-                                                                             const __grid_constant__ CUtensorMap map, Workspace ws, ParamsF64 hp,
-                                                                             int use_dev_params)
+                                                                             const __grid_constant__ CUtensorMap map, int mapped, Workspace ws,
+                                                                             ParamsF64 hp, int use_dev_params)
 {
     pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -221,19 +232,25 @@ __global__ void __launch_bounds__(kCodecThreads, kStages64 == 2 ? 3 : 2) encode_
     // Asks for the warp's round of tile t into stage st; completes one phase of the stage's mbarrier whether there is
     // anything to copy or not.
     auto request = [&](unsigned long long t, uint32_t st) {
-        if (lane != 0) return;
         if (e0 + (uint32_t)kRound <= tile_len(t)) {
-            mbar_expect_tx(&sh.bar[st], kRound * 8 + (rd ? 16u : 0u));
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                         ::"r"(smem_u32(sh.stage[st])), "l"(&map), "r"(0), "r"((int)((uint32_t)t * 256u + rd * (uint32_t)kRowsPerRound64)),
-                           "r"(smem_u32(&sh.bar[st])) : "memory");
-            if (rd)
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], 16, [%2];"
-                             ::"r"(smem_u32(sh.front[st])), "l"(x + t * kTile + e0 - 2), "r"(smem_u32(&sh.bar[st])) : "memory");
-        } else {
-            mbar_arrive(&sh.bar[st]);
+            if (mapped) {
+                if (lane == 0) {
+                    mbar_expect_tx(&sh.bar[st], kRound * 8 + (rd ? 16u : 0u));
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                                 ::"r"(smem_u32(sh.stage[st])), "l"(&map), "r"(0), "r"((int)((uint32_t)t * 256u + rd * (uint32_t)kRowsPerRound64)),
+                                   "r"(smem_u32(&sh.bar[st])) : "memory");
+                    if (rd)
+                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], 16, [%2];"
+                                     ::"r"(smem_u32(sh.front[st])), "l"(x + t * kTile + e0 - 2), "r"(smem_u32(&sh.bar[st])) : "memory");
+                }
+                return;
+            }
+            load_round_plain_f64(sh.stage[st], x + t * kTile + e0, lane);
+            if (lane == 0 && rd) sh.front[st][1] = __ldg(x + t * kTile + e0 - 1);
+            __syncwarp();
         }
+        if (lane == 0) mbar_arrive(&sh.bar[st]);
     };
 
     unsigned long long t = blockIdx.x;

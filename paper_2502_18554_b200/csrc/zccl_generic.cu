@@ -472,7 +472,7 @@ cudaError_t launch_generic_decode(const uint32_t* in, unsigned long long cap_byt
 cudaError_t launch_encode_f64(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* sizes, uint32_t* go,
                               uint32_t* out, unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st)
 {
-    if (ws.slots && (((uintptr_t)x) & 15u) == 0 && (n + kTile - 1) / kTile <= ws.max_tiles && !plain_forced()) {
+    if (ws.slots && (n + kTile - 1) / kTile <= ws.max_tiles && !plain_forced()) {
         count_launches(2);
         return launch_encode_f64_lanes(x, n, hp, device_params, out, out_cap, out_bytes, ws, sm_count, st);
     }

@@ -181,7 +181,7 @@ cudaError_t launch_encode_tiled_lanes(const float* x, unsigned long long n, uint
                                       unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_decode_tiled_lanes(const uint32_t* in, unsigned long long cap_bytes, uint32_t T, float* y, unsigned long long y_cap,
                                       const Workspace& ws, int sm_count, cudaStream_t st);
-// binary64 on the tuned kernels (array on a 16-byte boundary, a context with round slots)
+// binary64 on the tuned kernels (a context with round slots)
 cudaError_t launch_encode_f64_lanes(const double* x, unsigned long long n, ParamsF64 hp, bool device_params, uint32_t* out,
                                     unsigned long long out_cap, size_t* out_bytes, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_decode_f64_lanes(const uint32_t* in, unsigned long long cap_bytes, double* y, unsigned long long y_cap, const Workspace& ws,

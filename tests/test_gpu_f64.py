@@ -103,8 +103,8 @@ def test_errors(z, ctx):
 @pytest.mark.parametrize("n", [5000, 3 * 4096 + 1024, 3 * 4096 + 1025, 200_001])
 @pytest.mark.parametrize("shift_x,shift_y", [(1, 0), (0, 1), (1, 1)])
 def test_arrays_off_the_16_byte_boundary(z, ctx, n, shift_x, shift_y):
-    """Input or output that starts 8 bytes past a 16-byte boundary: the plain kernels (input) and the plain stores
-    (output) take over; streams and values stay those of the oracle."""
+    """Input or output that starts 8 bytes past a 16-byte boundary: plain loads and stores take the place of the
+    tensor copies; streams and values stay those of the oracle."""
     x = as_f64(fields.smooth_1d(n, seed=7), n + 1)
     want = oracle.compress_f64(x, oracle.EB_ABS, 1e-5)
     buf = torch.empty(n + 2, dtype=torch.float64, device="cuda")
