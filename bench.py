@@ -301,7 +301,7 @@ def _codec_row(z, ctx, name, x_h, mode, eb, with_oracle: bool, loc_h=None):
 
 
 def _tiled_row(z, ctx, name, x_h, mode, eb, tile):
-    """Compress and decompress through the plain kernels for another tile size (same protocol as _codec_row)."""
+    """Compress and decompress at another tile size (same protocol as _codec_row)."""
     import torch
     n = x_h.size
     nbytes = 4 * n
@@ -445,6 +445,8 @@ def other_configs(z, peak: float, x1, loc1) -> dict:
     for eb in (1e-2, 1e-4):
         out[f"cfg1 REL {eb:g}"] = fracs(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, False, loc1))
     out["cfg3 ABS 1e-05 (1 GiB)"] = fracs(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, False))
+    # cfg1 in tiles of 5120 elements, the paper's chunk (encode_rounds_tiled + place_tiled, decode_tiles_tiled)
+    out["cfg1 tile 5120 ABS"] = fracs(_tiled_row(z, big, "cfg1, tile of 5120", x1, z.EB_ABS, REL * float(x1.max() - x1.min()), 5120))
     # the cfg1 field as binary64 (128 MiB) through the binary64 entry points (encode_rounds_f64 + place, decode_tiles_f64)
     n = x1.size
     sets = 4
