@@ -424,15 +424,18 @@ def other_configs(z, peak: float, x1, loc1) -> dict:
     """The configurations the step itself does not cover, timed like the rows of --table (10 warm-up + 10 timed graph
     replays per call): cfg1 at the looser and the tighter bound (all three calls), cfg3 (1 GiB gradient-like array,
     compress and decompress) and cfg2 at full size (emulated 8-rank ring Allreduce of 64 MiB per rank).  `frac` =
-    algorithmic bytes (input + output of the call) / time / the measured copy bandwidth."""
+    algorithmic bytes (input + output of the call, the input twice where a relative bound adds the range pass) / time /
+    the measured copy bandwidth."""
     import torch
     from paper_2502_18554_b200 import fields
     out = {}
 
     def fracs(row):
         nbytes, cbytes = row["bytes"], row["bytes"] / row["ratio"]
+        range_bytes = nbytes if str(row.get("bound", "")).startswith("REL") else 0   # a relative bound reads the input once more
         r = {"ratio": row["ratio"], "status": row["status"],
-             "compress_us": row["compress_us_mean"], "compress_frac": round((nbytes + cbytes) / row["compress_us_mean"] / 1e3 / peak, 3),
+             "compress_us": row["compress_us_mean"],
+             "compress_frac": round((range_bytes + nbytes + cbytes) / row["compress_us_mean"] / 1e3 / peak, 3),
              "decompress_us": row["decompress_us_mean"], "decompress_frac": round((nbytes + cbytes) / row["decompress_us_mean"] / 1e3 / peak, 3),
              "compress_gbs": row["compress_gbs"], "decompress_gbs": row["decompress_gbs"]}
         if "fused_us_mean" in row:
