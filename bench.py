@@ -38,6 +38,9 @@ MIN_TIMED_MS = 500.0                # the timed region lasts at least this long 
 # ncu capture of this workload: 78.5 MB read + 4.4 MB written by the hop kernel, 0.3 MB by the placement (the encoded
 # rounds wait in L2 between the two, and most of the 12 MB output stream is still there when the call ends)
 DRAM_TRAFFIC_FUSED_64MIB = 83.2e6
+# smsp__inst_executed.sum x 32 / 2^24 of the hop kernel with both operands compressed (64 MiB, cfg1), from an ncu capture
+# (31 345 480 warp-instructions per launch)
+HOP_C2_INSTR_PER_ELEMENT = 59.8
 METRIC = "compress / decompress / fused decomp-reduce-comp GB/s (uncompressed bytes through the codec per step)"
 WORKLOAD = ("cfg1: 256^3 fp32 Fourier-mode field (64 MiB), REL 1e-3; step = compress + decompress + fused hop + "
             "8-rank ring allreduce (8 MiB/rank) + 8-rank allgather (1 MiB/rank)")
@@ -420,7 +423,7 @@ def config_table(args):
 
 # --------------------------------------------------------------------------------------------- CUDA arm
 
-def other_configs(z, peak: float, x1, loc1) -> dict:
+def other_configs(z, peak: float, x1, loc1, sm_mhz=None) -> dict:
     """The configurations the step itself does not cover, timed like the rows of --table (10 warm-up + 10 timed graph
     replays per call): cfg1 at the looser and the tighter bound (all three calls), cfg3 (1 GiB gradient-like array,
     compress and decompress) and cfg2 at full size (emulated 8-rank ring Allreduce of 64 MiB per rank).  `frac` =
@@ -448,6 +451,35 @@ def other_configs(z, peak: float, x1, loc1) -> dict:
     for eb in (1e-2, 1e-4):
         out[f"cfg1 REL {eb:g}"] = fracs(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, False, loc1))
     out["cfg3 ABS 1e-05 (1 GiB)"] = fracs(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, False))
+    # the hop with both operands compressed (a variant: the paper's hop adds the rank's own uncompressed chunk).  It moves
+    # about 2 bytes per element, so HBM is not what bounds it: `issue_frac` states it against the issue rate instead
+    # (thread-instructions per element from an ncu capture of this launch x elements / time / (SMs x 4 schedulers x 32
+    # lanes x SM clock)).
+    n = x1.size
+    sets = 6
+    ebx = REL * float(x1.max() - x1.min())
+    cap = z.compress_bound(n)
+    sz = torch.zeros(1, dtype=torch.int64, device="cuda")
+    xa, xb = torch.from_numpy(x1).cuda(), torch.from_numpy(loc1).cuda()
+    sa = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    sb = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    so = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(sets)]
+    for i in range(sets):
+        big.compress(xa, z.EB_ABS, ebx, sa[i], sz)
+        ca = int(sz.item())
+        big.compress(xb, z.EB_ABS, ebx, sb[i], sz)
+        cb = int(sz.item())
+    h_us, _ = _timed(lambda i: big.decompress_reduce_compress(sa[i][:ca], n, so[i], sz, local_c=sb[i][:cb]), sets)
+    rc = big.check()
+    co = int(sz.item())
+    props = torch.cuda.get_device_properties(0)
+    issue_peak = props.multi_processor_count * 4 * 32 * sm_mhz * 1e6 if sm_mhz else None
+    out["cfg1 hop, both operands compressed (ABS)"] = {
+        "status": rc, "fused_us": round(h_us, 2), "ratio_in": round(4 * n / ca, 3), "ratio_out": round(4 * n / co, 3),
+        "algorithmic_bytes": ca + cb + co, "hbm_frac": round((ca + cb + co) / h_us / 1e3 / peak, 3), "bound": "alu",
+        "thread_instructions_per_element": HOP_C2_INSTR_PER_ELEMENT,
+        "issue_frac": round(HOP_C2_INSTR_PER_ELEMENT * n / (h_us * 1e-6) / issue_peak, 3) if issue_peak else None}
+    del xa, xb, sa, sb, so
     # cfg1 in tiles of 5120 elements, the paper's chunk (encode_rounds_tiled + place_tiled, decode_tiles_tiled)
     out["cfg1 tile 5120 ABS"] = fracs(_tiled_row(z, big, "cfg1, tile of 5120", x1, z.EB_ABS, REL * float(x1.max() - x1.min()), 5120))
     # the cfg1 field as binary64 (128 MiB) through the binary64 entry points (encode_rounds_f64 + place, decode_tiles_f64)
@@ -806,7 +838,7 @@ def main():
         ctx = None
         del xs, locs, cs, c2s, ys, ars, ags
         torch.cuda.empty_cache()
-        configs = other_configs(z, peak, x_h, loc_h)
+        configs = other_configs(z, peak, x_h, loc_h, clocks.get("sm_mhz") if clocks else None)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
