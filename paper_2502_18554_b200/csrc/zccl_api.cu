@@ -73,11 +73,12 @@ inline bool eb_ok(int mode, float eb)
 inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? ZCCL_OK : ZCCL_E_CUDA; }
 
 // Collects jobs and launches them in batches of at most kMaxJobs.
-struct Batcher {
-    JobBatch jb{};
+template <int CAP>
+struct BatcherT {
+    JobBatchT<CAP> jb{};
     void reset() { jb.count = 0; jb.total_tiles = 0; }
-    Batcher() { reset(); }
-    bool full() const { return jb.count == kMaxJobs; }
+    BatcherT() { reset(); }
+    bool full() const { return jb.count == CAP; }
     void add(const Job& j, size_t tiles)
     {
         Job& d = jb.job[jb.count++];
@@ -86,6 +87,9 @@ struct Batcher {
         jb.total_tiles += (uint32_t)(tiles ? tiles : 1);
     }
 };
+
+using Batcher = BatcherT<kMaxJobs>;
+using DecodeBatcher = BatcherT<kMaxDecodeJobs>;
 
 struct RangeList {
     std::vector<const float*> x;
@@ -138,6 +142,13 @@ int flush_decode(zccl_ctx* c, Batcher& b, cudaStream_t st)
 {
     if (b.jb.count == 0) return ZCCL_OK;
     cudaError_t e = launch_decode(b.jb, c->ws, c->sm_count, st);
+    b.reset();
+    return cuda_rc(e);
+}
+int flush_decode(zccl_ctx* c, DecodeBatcher& b, cudaStream_t st)
+{
+    if (b.jb.count == 0) return ZCCL_OK;
+    cudaError_t e = launch_decode_wide(b.jb, c->ws, c->sm_count, st);
     b.reset();
     return cuda_rc(e);
 }
@@ -451,17 +462,18 @@ int zccl_sim_allreduce(zccl_ctx* c, const float* const* send, float* const* recv
         if ((rc = cuda_rc(launch_copy_chain(cb, c->ws, c->sm_count, st))) != ZCCL_OK) return rc;
     }
     // every rank decompresses the chunks it does not own
+    DecodeBatcher db;
     for (int r = 0; r < N; ++r) {
         for (int ch = 0; ch < N; ++ch) {
             if (ch == (r + 1) % N) continue;
             size_t off, len; chunk_span(n, N, ch, off, len);
             Job j{};
             j.in_c = (const uint32_t*)gslot(r, ch); j.in_cap = slot; j.y = recv[r] + off; j.n = len;
-            b.add(j, tiles_of(len));
-            if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+            db.add(j, tiles_of(len));
+            if (db.full() && (rc = flush_decode(c, db, st)) != ZCCL_OK) return rc;
         }
     }
-    if ((rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+    if ((rc = flush_decode(c, db, st)) != ZCCL_OK) return rc;
     if ((flags & ZCCL_OP_MASK) == ZCCL_OP_AVG) {   // Average = Sum / N: one division per element of every rank's result
         ScaleBatch sb{};
         sb.n = n; sb.divisor = (float)N; sb.count = 0;
@@ -529,16 +541,17 @@ int zccl_sim_allgather(zccl_ctx* c, const float* const* send, float* const* recv
         }
         if ((rc = flush_copy(c, cb, st)) != ZCCL_OK) return rc;
     }
+    DecodeBatcher db;
     for (int r = 0; r < N; ++r) {
         for (int src = 0; src < N; ++src) {
             if (src == r) continue;
             Job j{};
             j.in_c = (const uint32_t*)gslot(r, src); j.in_cap = slot; j.y = recv[r] + (size_t)src * n; j.n = n;
-            b.add(j, tiles_of(n));
-            if (b.full() && (rc = flush_decode(c, b, st)) != ZCCL_OK) return rc;
+            db.add(j, tiles_of(n));
+            if (db.full() && (rc = flush_decode(c, db, st)) != ZCCL_OK) return rc;
         }
     }
-    return flush_decode(c, b, st);
+    return flush_decode(c, db, st);
 }
 
 int zccl_sim_bcast(zccl_ctx* c, const float* root, float* const* recv, int nsinks, size_t n,

@@ -588,9 +588,11 @@ struct alignas(1024) EncWarpShared {
 static_assert(sizeof(EncWarpShared) == 18 * 1024, "a warp's share of the shared memory");
 
 // One tensor map per job of a launch: the job's input seen as rows of 32 floats.
-struct alignas(64) TileMaps {
-    CUtensorMap m[kMaxJobs];
+template <int CAP>
+struct alignas(64) TileMapsT {
+    CUtensorMap m[CAP];
 };
+using TileMaps = TileMapsT<kMaxJobs>;
 
 // A tile of the launch as a warp sees it.
 struct TileInfo {
@@ -1555,8 +1557,9 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
     }
 }
 
-__global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __grid_constant__ JobBatch jb, const __grid_constant__ TileMaps maps,
-                                                                        Workspace ws)
+template <int CAP>
+__global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __grid_constant__ JobBatchT<CAP> jb,
+                                                                        const __grid_constant__ TileMapsT<CAP> maps, Workspace ws)
 {
     pdl_enter();
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -2140,9 +2143,11 @@ cudaError_t device_setup(const DeviceSetup** out)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, encode_rounds_kernel, kCodecThreads, kRoundSmemBytes);
         if (e != cudaSuccess) return e;
         d.round_ctas = a > 0 ? a : 1;
-        e = cudaFuncSetAttribute(decode_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecSmemBytes);
+        e = cudaFuncSetAttribute(decode_tiles_kernel<kMaxJobs>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecSmemBytes);
         if (e != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_kernel, kCodecThreads, kDecSmemBytes);
+        e = cudaFuncSetAttribute(decode_tiles_kernel<kMaxDecodeJobs>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDecSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, decode_tiles_kernel<kMaxJobs>, kCodecThreads, kDecSmemBytes);
         if (e != cudaSuccess) return e;
         d.dec_ctas = a > 0 ? a : 1;
         e = cudaFuncSetAttribute(place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPlaceSmemBytes);
@@ -2259,18 +2264,27 @@ cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_cou
     return launch_k(place_kernel, dim3(groups), dim3(kPlaceThreads), kPlaceSmemBytes, st, jb, gt, ws, Params{0.f, 1.f, 1.f, 1}, 0, 1, ParamsF64{0.0, 1.0, 1.0, 1});
 }
 
-cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
+template <int CAP>
+static cudaError_t launch_decode_lanes_t(const JobBatchT<CAP>& jb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
     const DeviceSetup* d = nullptr;
     cudaError_t e = device_setup(&d);
     if (e != cudaSuccess) return e;
-    TileMaps maps;
+    thread_local TileMapsT<CAP> maps;   // kept off the stack, one per calling thread
     memset(&maps, 0, sizeof(maps));
     for (int j = 0; j < jb.count; ++j)
         if ((e = make_row_map(&maps.m[j], jb.job[j].y, jb.job[j].n)) != cudaSuccess) return e;
     const unsigned long long want = ((unsigned long long)jb.total_tiles + kCodecWarps - 1) / kCodecWarps;
     const unsigned long long cap = (unsigned long long)sm_count * d->dec_ctas;
-    return launch_k(decode_tiles_kernel, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kDecSmemBytes, st, jb, maps, ws);
+    return launch_k(decode_tiles_kernel<CAP>, dim3((unsigned)(want < cap ? want : cap)), dim3(kCodecThreads), kDecSmemBytes, st, jb, maps, ws);
+}
+cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    return launch_decode_lanes_t<kMaxJobs>(jb, ws, sm_count, st);
+}
+cudaError_t launch_decode_lanes_wide(const DecodeBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    return launch_decode_lanes_t<kMaxDecodeJobs>(jb, ws, sm_count, st);
 }
 
 

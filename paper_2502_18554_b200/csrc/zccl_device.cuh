@@ -94,7 +94,8 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 }
 
 // The job that owns tile number `ticket` of the launch: the last one whose first tile is not beyond it.
-__device__ __forceinline__ int find_job(const JobBatch& jb, uint32_t ticket)
+template <class JB>
+__device__ __forceinline__ int find_job(const JB& jb, uint32_t ticket)
 {
     int lo = 0, hi = jb.count;
 #pragma unroll 1

@@ -93,11 +93,16 @@ struct Job {
     uint32_t flags;
 };
 
-struct JobBatch {
-    Job job[kMaxJobs];
+template <int CAP>
+struct JobBatchT {
+    Job job[CAP];
     int count;
     uint32_t total_tiles;
 };
+using JobBatch = JobBatchT<kMaxJobs>;
+// Decoding launches take twice as many: the 56 chunk decodes that end an 8-rank Allreduce or Allgather are one launch.
+constexpr int kMaxDecodeJobs = 64;
+using DecodeBatch = JobBatchT<kMaxDecodeJobs>;
 
 struct CopyJob {
     const uint32_t* src;
@@ -164,6 +169,8 @@ cudaError_t launch_encode_lanes(const JobBatch& jb, const Workspace& ws, bool de
 cudaError_t launch_hop_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_decode_lanes(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_decode_wide(const DecodeBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
+cudaError_t launch_decode_lanes_wide(const DecodeBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st);
 cudaError_t launch_scale(const ScaleBatch& sb, int sm_count, cudaStream_t st);
 cudaError_t launch_resolve_range(const float* minmax, float eb, const Workspace& ws, float* eb_abs_out, cudaStream_t st);
 cudaError_t launch_generic_encode(const float* x, unsigned long long n, uint32_t T, Params hp, bool device_params, uint32_t* sizes,

@@ -420,6 +420,13 @@ cudaError_t launch_decode(const JobBatch& jb, const Workspace& ws, int sm_count,
     return launch_decode_lanes(jb, ws, sm_count, st);
 }
 
+cudaError_t launch_decode_wide(const DecodeBatch& jb, const Workspace& ws, int sm_count, cudaStream_t st)
+{
+    if (jb.total_tiles == 0) return cudaSuccess;
+    ++g_launches;
+    return launch_decode_lanes_wide(jb, ws, sm_count, st);
+}
+
 cudaError_t launch_copy(const CopyBatch& cb, const Workspace& ws, int sm_count, cudaStream_t st)
 {
     if (cb.count <= 0) return cudaSuccess;
