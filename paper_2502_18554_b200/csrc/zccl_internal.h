@@ -19,8 +19,8 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kBlocksPerWarp = kBlocksPerTile / kWarps;   // 16 consecutive blocks per warp
 constexpr int kGenericMinTile = 1024;       // tile sizes the plain kernels of zccl_generic.cu accept (multiples of 32)
 constexpr int kGenericMaxTile = 8192;
-// Chunk-operations per launch.  A stage of an 8-rank ring (8 jobs) fits one launch; the 56 chunk decodes that end an
-// 8-rank Allreduce take two.  (With 64 the fused hop's 64 MiB launch was 1.6 us slower and nothing else faster.)
+// Chunk-operations per launch.  A stage of an 8-rank ring (8 jobs) fits one launch.  (With 64 the fused hop's 64 MiB
+// launch was 1.6 us slower; decoding launches alone take 64, see kMaxDecodeJobs.)
 constexpr int kMaxJobs = 32;
 
 // Device status bits (zccl_status maps them to return codes).
