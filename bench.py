@@ -450,6 +450,13 @@ def other_configs(z, peak: float, x1, loc1, sm_mhz=None) -> dict:
     big = z.Context(1 << 28, 1)
     for eb in (1e-2, 1e-4):
         out[f"cfg1 REL {eb:g}"] = fracs(_codec_row(z, big, "cfg1", x1, z.EB_REL, eb, False, loc1))
+    # the cfg1 field four and sixteen times over (256 MiB, 1 GiB), absolute bound: what the calls reach when their fixed costs
+    # (launch ramps, the first round trip, the placement's tail) weigh less
+    ebx1 = REL * float(x1.max() - x1.min())
+    for reps in (4, 16):
+        xr, lr = np.tile(x1, reps), np.tile(loc1, reps)
+        out[f"cfg1 x{reps} ({reps * 64} MiB) ABS"] = fracs(_codec_row(z, big, f"cfg1 x{reps}", xr, z.EB_ABS, ebx1, False, lr))
+        del xr, lr
     out["cfg3 ABS 1e-05 (1 GiB)"] = fracs(_codec_row(z, big, "cfg3", fields.gradient_like(1 << 28, seed=3), z.EB_ABS, 1e-5, False))
     # the hop with both operands compressed (a variant: the paper's hop adds the rank's own uncompressed chunk).  It moves
     # about 2 bytes per element, so HBM is not what bounds it: `issue_frac` states it against the issue rate instead
