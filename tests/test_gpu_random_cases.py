@@ -160,3 +160,34 @@ def test_random_collectives(z, ctx, seed):
     assert ctx.status() == wrc
     for r in range(N):
         assert same_bits(recv[r].cpu().numpy(), want[r]), f"reduce-scatter rank {r}"
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_tile_sizes(z, ctx, seed):
+    """Any multiple of 32 between 1024 and 8192 as the tile size, random lengths, kinds of data, bounds and offsets of
+    both arrays from a 16-byte boundary: stream and values are the oracle's for that tile size."""
+    rng = np.random.default_rng(7000 + seed)
+    T = int(rng.integers(32, 257)) * 32
+    n = draw_length(rng)
+    x = draw_field(rng, n)
+    mode, eb = draw_bound(rng, x)
+    sx, sy = int(rng.integers(0, 4)), int(rng.integers(0, 4))
+    try:
+        want, wrc = oracle.compress(x, mode, eb, T)
+    except oracle.OracleError as e:
+        want, wrc = None, e.code
+    buf = torch.empty(n + 4, dtype=torch.float32, device="cuda")
+    dx = buf[sx: sx + n]
+    dx.copy_(torch.from_numpy(x))
+    out = torch.empty(z.compress_bound_tiled(n, T), dtype=torch.uint8, device="cuda")
+    nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx.compress_tiled(dx, mode, eb, T, out, nb)
+    assert ctx.status() == wrc
+    if want is None:
+        return
+    assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+    ybuf = torch.full((n + 4,), -3.0, dtype=torch.float32, device="cuda")
+    ctx.decompress_tiled(out[: int(nb.item())], T, ybuf[sy: sy + n])
+    assert ctx.status() == z.OK
+    assert same_bits(ybuf[sy: sy + n].cpu().numpy(), oracle.decompress(want))
+    assert bool((ybuf[:sy] == -3.0).all()) and bool((ybuf[sy + n:] == -3.0).all())
