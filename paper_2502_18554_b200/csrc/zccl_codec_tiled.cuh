@@ -224,12 +224,20 @@ __global__ void __launch_bounds__(kPlaceThreads) place_tiled_kernel(uint32_t* __
             for (uint32_t rd = 0; rd < sp.R; ++rd) {
                 const uint32_t cnt = __shfl_sync(kFull, nq, (int)rd);
                 const uint32_t* __restrict__ src = slot0 + (size_t)rd * kRoundSlotWords + 8;
-                uint32_t i = (uint32_t)lane;
-                for (; i + 96u < cnt; i += 128u) {   // four loads in flight
-                    const uint32_t a = src[i], b = src[i + 32u], c = src[i + 64u], e = src[i + 96u];
-                    d[i] = a; d[i + 32u] = b; d[i + 64u] = c; d[i + 96u] = e;
+                // eight loads in flight per lane: a round of mean code length 4 is one trip
+                for (uint32_t i0 = 0; i0 < cnt; i0 += 256u) {
+                    uint32_t v[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t i = i0 + 32u * k + (uint32_t)lane;
+                        v[k] = i < cnt ? src[i] : 0u;
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t i = i0 + 32u * k + (uint32_t)lane;
+                        if (i < cnt) d[i] = v[k];
+                    }
                 }
-                for (; i < cnt; i += 32u) d[i] = src[i];
                 d += cnt;
             }
             if (lane == 0) out[kHeaderWords + tile] = base + my_off + words;
