@@ -767,8 +767,8 @@ def test_other_tile_sizes_match_oracle(z, ctx, T, n):
 @pytest.mark.parametrize("T", [5120, 1024, 7168, 4128])
 def test_other_tile_sizes_many_groups_and_alignments(z, T):
     """Hundreds of tiles (several groups of 32 in the placement), wide and narrow code lengths side by side, input and
-    output on and off a 16-byte boundary; at T = 4128 the last array is too large for the context's round slots and
-    goes to the plain kernels."""
+    output on and off a 16-byte boundary; at T = 4128 the first array (5 rounds per tile of 4128 elements) is too large
+    for the context's round slots and goes to the plain kernels."""
     c = z.Context(1 << 21, 0)
     try:
         for n, shift in ((1 << 21, 0), ((1 << 20) + 4321, 1), (900_000, 3)):
@@ -790,6 +790,46 @@ def test_other_tile_sizes_many_groups_and_alignments(z, T):
             assert bool((ybuf[:shift] == 7.0).all()) and bool((ybuf[shift + n:] == 7.0).all())
     finally:
         c.close()
+
+
+def test_plain_kernels_forced_by_the_environment():
+    """ZCCL_PLAIN=1 keeps other tile sizes and binary64 on the plain kernels (the fallback when a context's round slots
+    do not cover an input): the same streams and values, checked in a process of its own because the switch is read
+    once."""
+    import os
+    import subprocess
+    import sys
+    code = r"""
+import numpy as np, torch
+import oracle
+from paper_2502_18554_b200 import fields, zccl as z
+c = z.Context(1 << 20, 0)
+nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+for T, n in ((5120, 300_001), (1024, 70_000), (8192, 5)):
+    x = fields.smooth_1d(n, seed=T % 11)
+    want, wrc = oracle.compress(x, oracle.EB_REL if n > 1 else oracle.EB_ABS, 1e-3, T)
+    out = torch.empty(z.compress_bound_tiled(n, T), dtype=torch.uint8, device="cuda")
+    c.compress_tiled(torch.from_numpy(x).cuda(), z.EB_REL, 1e-3, T, out, nb)
+    assert c.status() == wrc and np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+    y = torch.empty(n, dtype=torch.float32, device="cuda")
+    c.decompress_tiled(out[: int(nb.item())], T, y)
+    assert c.status() == z.OK and np.array_equal(y.cpu().numpy().view(np.uint32), oracle.decompress(want).view(np.uint32))
+x = fields.smooth_1d(200_003, seed=3).astype(np.float64) * (1 + 1e-12)
+want = oracle.compress_f64(x, oracle.EB_ABS, 1e-7)
+out = torch.empty(z.compress_bound(x.size), dtype=torch.uint8, device="cuda")
+c.compress_f64(torch.from_numpy(x).cuda(), z.EB_ABS, 1e-7, out, nb)
+assert c.status() == z.OK and np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+y = torch.empty(x.size, dtype=torch.float64, device="cuda")
+c.decompress_f64(out[: int(nb.item())], y)
+assert c.status() == z.OK and np.array_equal(y.cpu().numpy().view(np.uint64), oracle.decompress_f64(want).view(np.uint64))
+print("launches", z.launch_count())
+"""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, ZCCL_PLAIN="1", PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=600, cwd=root)
+    assert r.returncode == 0, r.stdout + r.stderr
+    # three launches per compression and one per decompression on the plain kernels, plus a range pass per relative bound
+    assert "launches 19" in r.stdout, r.stdout
 
 
 def test_tile_4096_streams_of_both_routes_are_the_same(z, ctx):
