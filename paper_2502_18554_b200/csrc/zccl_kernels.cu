@@ -299,6 +299,30 @@ __global__ void __launch_bounds__(256, 4) quality_kernel(const float* __restrict
             dsum += dd * dd;
         }
     };
+    // The same arithmetic on two elements at a time (sm_100's packed fp32: each half rounds as the scalar operation
+    // does), for the pairs of sums 2 k and 2 k + 1; a pair in which a difference is not an fp32 number goes element by
+    // element.
+    auto neg2 = [](float2 v) { return make_float2(-v.x, -v.y); };
+    auto take2 = [&](float2 a, float2 b, int k) {
+        const float2 d = __fadd2_rn(a, neg2(b));
+        const float2 bb = __fadd2_rn(d, neg2(a));
+        const float2 err = __fadd2_rn(__fadd2_rn(a, neg2(__fadd2_rn(d, neg2(bb)))), neg2(__fadd2_rn(b, bb)));
+        if (err.x == 0.0f && err.y == 0.0f) {
+            lo = fminf(lo, fminf(a.x, a.y));
+            hi = fmaxf(hi, fmaxf(a.x, a.y));
+            emax = fmaxf(emax, fmaxf(fabsf(d.x), fabsf(d.y)));
+            const float2 shp = make_float2(sh8[2 * k], sh8[2 * k + 1]), slp = make_float2(sl8[2 * k], sl8[2 * k + 1]);
+            const float2 p = __fmul2_rn(d, d), e = __ffma2_rn(d, d, neg2(p));
+            const float2 t = __fadd2_rn(shp, p), z = __fadd2_rn(t, neg2(shp));
+            const float2 r2 = __fadd2_rn(shp, neg2(__fadd2_rn(t, neg2(z)))), r3 = __fadd2_rn(p, neg2(z));
+            const float2 sln = __fadd2_rn(slp, __fadd2_rn(__fadd2_rn(r2, r3), e));
+            sh8[2 * k] = t.x; sh8[2 * k + 1] = t.y;
+            sl8[2 * k] = sln.x; sl8[2 * k + 1] = sln.y;
+        } else {
+            take(a.x, b.x, 2 * k);
+            take(a.y, b.y, 2 * k + 1);
+        }
+    };
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + tid;
     const unsigned long long nth = (unsigned long long)gridDim.x * blockDim.x;
     unsigned long long done = 0;
@@ -309,8 +333,8 @@ __global__ void __launch_bounds__(256, 4) quality_kernel(const float* __restrict
         unsigned long long i = gtid;
         for (; i + nth < nv; i += 2 * nth) {   // two independent pairs of loads in flight
             const float4 a0 = __ldg(x4 + i), b0 = __ldg(y4 + i), a1 = __ldg(x4 + i + nth), b1 = __ldg(y4 + i + nth);
-            take(a0.x, b0.x, 0); take(a0.y, b0.y, 1); take(a0.z, b0.z, 2); take(a0.w, b0.w, 3);
-            take(a1.x, b1.x, 4); take(a1.y, b1.y, 5); take(a1.z, b1.z, 6); take(a1.w, b1.w, 7);
+            take2(make_float2(a0.x, a0.y), make_float2(b0.x, b0.y), 0); take2(make_float2(a0.z, a0.w), make_float2(b0.z, b0.w), 1);
+            take2(make_float2(a1.x, a1.y), make_float2(b1.x, b1.y), 2); take2(make_float2(a1.z, a1.w), make_float2(b1.z, b1.w), 3);
         }
         for (; i < nv; i += nth) {
             const float4 a = __ldg(x4 + i), b = __ldg(y4 + i);
