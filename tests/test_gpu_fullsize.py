@@ -178,3 +178,36 @@ def test_config4_allgather_and_bcast(z, n):
     for k in range(N):
         assert _same_bits(b_recv[k].cpu().numpy(), wantb[k])
     ctx.close()
+
+
+def test_two_gib_of_binary64_and_one_gib_in_tiles_of_5120(z):
+    """2^28 elements and a ragged end through the binary64 kernels (2 GiB in) and through the kernels for other tile
+    sizes (1 GiB in, tiles of 5120): tile, round and row numbers of the copy engine's maps at the top of the range."""
+    n = (1 << 28) + 12345
+    x = np.tile(fields.fourier_field_3d(256, seed=1).astype(np.float64), 17)[:n] * (1 + 1e-9)
+    ctx = z.Context(n, 0)
+    try:
+        nb = torch.zeros(1, dtype=torch.int64, device="cuda")
+        out = torch.empty(z.compress_bound(n), dtype=torch.uint8, device="cuda")
+        ctx.compress_f64(torch.from_numpy(x).cuda(), z.EB_REL, 1e-4, out, nb)
+        assert ctx.status() == z.OK
+        want = oracle.compress_f64(x, oracle.EB_REL, 1e-4)
+        assert np.array_equal(out[: int(nb.item())].cpu().numpy(), want)
+        y = torch.empty(n, dtype=torch.float64, device="cuda")
+        ctx.decompress_f64(out[: int(nb.item())], y)
+        assert ctx.status() == z.OK
+        assert np.array_equal(y.cpu().numpy().view(np.uint64), oracle.decompress_f64(want).view(np.uint64))
+        del out, y, x, want
+        n2 = (1 << 28) + 777
+        x2 = np.tile(fields.fourier_field_3d(256, seed=2), 17)[:n2]
+        out2 = torch.empty(z.compress_bound_tiled(n2, 5120), dtype=torch.uint8, device="cuda")
+        ctx.compress_tiled(torch.from_numpy(x2).cuda(), z.EB_REL, 1e-3, 5120, out2, nb)
+        want2, wrc2 = oracle.compress(x2, oracle.EB_REL, 1e-3, 5120)
+        assert ctx.status() == wrc2
+        assert np.array_equal(out2[: int(nb.item())].cpu().numpy(), want2)
+        y2 = torch.empty(n2, dtype=torch.float32, device="cuda")
+        ctx.decompress_tiled(out2[: int(nb.item())], 5120, y2)
+        assert ctx.status() == z.OK
+        assert _same_bits(y2.cpu().numpy(), oracle.decompress(want2))
+    finally:
+        ctx.close()
