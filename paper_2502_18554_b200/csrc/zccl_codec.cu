@@ -1479,12 +1479,6 @@ __device__ __forceinline__ void window_request(const BlobRef& br, uint32_t first
     mbar_expect_tx(bar, bytes);
     bulk_load(buf, (const void*)(((uintptr_t)(br.ptr + first)) & ~(uintptr_t)15), bytes, bar);
 }
-struct alignas(1024) DecWarpShared {
-    float out[2][kRound];                  // each on a 1024-byte boundary
-    alignas(16) uint32_t blob[kDecBlobWords];
-    alignas(8) unsigned long long bar;
-};
-static_assert(sizeof(DecWarpShared) == 13 * 1024, "a warp's share of the shared memory");
 
 // Tiled tensor store of a stage to rows [row0, row0 + 32) of the array behind `map` (one thread).
 __device__ __forceinline__ void tensor_store_round(const CUtensorMap* map, uint32_t row0, const float* stage)
@@ -1542,11 +1536,14 @@ __device__ __forceinline__ int round_class(uint32_t L)
 }
 // The decoder's own form: one function with both classes (measured faster there than the two instantiations above
 // behind a dispatch, which the hop uses out of line to keep its register count down).
-template <int MODE>
+// `ready` is called once by all lanes, after the planes are read and transposed and before the first value is stored:
+// the place to make sure the stage is free.
+template <int MODE, class Ready>
 __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t& pay_off, int32_t& code, float s,
-                                             float* stage, int lane, const float* loc_stage = nullptr)
+                                             float* stage, int lane, const float* loc_stage, Ready&& ready)
 {
     if (__any_sync(kFull, L > 16u)) {
+        ready();
         decode_round_general(blob, padw, L, &pay_off, &code, s, stage, lane, loc_stage, 0u);
         return;
     }
@@ -1569,6 +1566,7 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
             if (lane >= d) inc += v;
         }
         bit_transpose<8>(w);
+        ready();
         expand_block<8, MODE>(w, sign, code + inc - total, s, row, sw, loc);
         code += __shfl_sync(kFull, inc, 31);
     } else {
@@ -1581,11 +1579,24 @@ __device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw
             if (lane >= d) inc += v;
         }
         bit_transpose<16>(w);
+        ready();
         expand_block<16, MODE>(w, sign, code + inc - total, s, row, sw, loc);
         code += __shfl_sync(kFull, inc, 31);
     }
 }
+template <int MODE>
+__device__ __forceinline__ void decode_round(const uint32_t* blob, uint32_t padw, uint32_t L, uint32_t& pay_off, int32_t& code, float s,
+                                             float* stage, int lane, const float* loc_stage = nullptr)
+{
+    decode_round<MODE>(blob, padw, L, pay_off, code, s, stage, lane, loc_stage, [] {});
+}
 
+struct alignas(1024) DecWarpShared {
+    float out[kRound];                     // one output stage
+    alignas(16) uint32_t blob[2][kDecBlobWords];   // this tile's blob (or a window over it) and the next tile's
+    alignas(8) unsigned long long bar[2];
+};
+static_assert(sizeof(DecWarpShared) == 13 * 1024, "a warp's share of the shared memory");
 template <int CAP>
 __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __grid_constant__ JobBatchT<CAP> jb,
                                                                         const __grid_constant__ TileMapsT<CAP> maps, Workspace ws)
@@ -1596,11 +1607,12 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
     DecWarpShared& sh = reinterpret_cast<DecWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
     uint32_t status = 0;
     if (lane == 0) {
-        mbar_init(&sh.bar, 1);
+        mbar_init(&sh.bar[0], 1); mbar_init(&sh.bar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
-    uint32_t fills = 0;   // bulk copies completed into the blob buffer (phase parity of its mbarrier)
+    uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed into each blob buffer (phase parities of their mbarriers)
+    uint32_t cb = 0;                   // the buffer with the current tile's blob
 
     // the job of the tile looked up last, with its stream's header
     int cj = -1;
@@ -1618,7 +1630,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
     };
     // The blob of tile t of the launch, from the index alone; the front of its 16-byte-aligned cover is requested into the
     // blob buffer when the cover lies inside the readable bytes.  Uniform over the warp.
-    auto request = [&](uint32_t t) {
+    auto request = [&](uint32_t t, uint32_t buf) {
         BlobRef br;
         br.ptr = nullptr; br.words = 0; br.staged = false;
         if (t >= jb.total_tiles) return br;
@@ -1646,7 +1658,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
         br.words = w_end - w_beg;
         const uintptr_t a_end = ((uintptr_t)(br.ptr + br.words) + 15) & ~(uintptr_t)15;
         if (a_end - (uintptr_t)q.in_c <= (uintptr_t)q.in_cap) {   // the copies may read up to the boundary behind the blob
-            if (lane == 0) window_request(br, 0, sh.blob, &sh.bar);
+            if (lane == 0) window_request(br, 0, sh.blob[buf], &sh.bar[buf]);
             br.staged = true;
         }
         return br;
@@ -1655,7 +1667,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
     const uint32_t stride = gridDim.x * (uint32_t)kCodecWarps;
     uint32_t t = blockIdx.x * (uint32_t)kCodecWarps + (uint32_t)warp;
     uint32_t so = 0;   // output stage to use next
-    BlobRef cur = request(t);
+    BlobRef cur = request(t, 0);
     while (t < jb.total_tiles) {
         // the current tile's facts, before the look-up of the next tile moves on to another job
         enter_job(t);
@@ -1665,20 +1677,21 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
         const int jcur = cj;
         const bool job_bad = !hc.ok, too_small = hc.ok && hc.n > job.n;
         const uint32_t tn = t + stride < t ? 0xFFFFFFFFu : t + stride;
-        // The one blob buffer takes the next tile's blob as soon as this tile's last round is decoded (16 warps per SM
-        // with one buffer beat 12 with two: 4096 tiles leave the busiest of 2368 warps two tiles instead of three).
+        // Two blob buffers and ONE output stage in the 13 KiB that keep 16 warps on an SM: the next tile's blob is asked for
+        // when this tile's has arrived, a whole tile ahead (with one buffer it was asked for after this tile's last round
+        // and every tile began with a wait for it: 19.0 us per 64 MiB against 18.0), and the wait for the tensor store that
+        // drains the stage sits behind the reading and transposing of the next round's planes, where it costs nothing.
         BlobRef nxt;
         nxt.ptr = nullptr; nxt.words = 0; nxt.staged = false;
-        bool asked = false;
         auto ask_next = [&]() {
-            __syncwarp();   // every lane is done with the blob buffer
-            nxt = request(tn);
-            asked = true;
+            __syncwarp();   // every lane is done with the other blob buffer (the tile before)
+            nxt = request(tn, cb ^ 1u);
         };
         if (cur.staged) {
-            if (!mbar_wait(&sh.bar, fills & 1u)) status |= kStTimeout;
-            ++fills;
+            if (!mbar_wait(&sh.bar[cb], (cb ? fills1 : fills0) & 1u)) status |= kStTimeout;
+            if (cb) ++fills1; else ++fills0;
         }
+        ask_next();   // the other blob buffer takes the next tile's blob while this tile is decoded
         if (job_bad) status |= kStBadStream;
         else if (too_small) status |= kStCapacity;
         else if (cur.words == 0xFFFFFFFFu) status |= kStBadStream;
@@ -1688,7 +1701,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
             const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2;
             BlobWindow win;
             win.base = cur.ptr; win.end = cur.words;
-            if (cur.staged) win = window_at(cur, 0, sh.blob);
+            if (cur.staged) win = window_at(cur, 0, sh.blob[cb]);
             const int mode = describe_blob(win.base, cur.words, nb, lane);   // the head (at most 33 words) is in every first window
             if (mode == 0) status |= kStBadStream;
             else {
@@ -1704,32 +1717,35 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_kernel(const __
                     // only a blob larger than its buffer has a window that ends before the blob does
                     if (win.end < cur.words && first + __reduce_add_sync(kFull, L ? L + 1u : 0u) > win.end) {   // the round reaches past the window
                         __syncwarp();         // every lane is done with the window as it is
-                        if (lane == 0) window_request(cur, first, sh.blob, &sh.bar);
-                        if (!mbar_wait(&sh.bar, fills & 1u)) status |= kStTimeout;
-                        ++fills;
-                        win = window_at(cur, first, sh.blob);
+                        if (lane == 0) window_request(cur, first, sh.blob[cb], &sh.bar[cb]);
+                        if (!mbar_wait(&sh.bar[cb], (cb ? fills1 : fills0) & 1u)) status |= kStTimeout;
+                        if (cb) ++fills1; else ++fills0;
+                        win = window_at(cur, first, sh.blob[cb]);
                     }
                     const uint32_t* blob = win.base;
                     // the stage about to be written was handed to a tensor store two rounds ago
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    __syncwarp();
-                    float* stage = sh.out[so];
-                    if (mode == 1) decode_round<0>(blob, padw, L, pay_off, code, hc.s, stage, lane);
-                    else decode_round_general(blob, padw, L, &pay_off, &code, hc.s, stage, lane, nullptr, 0u);
-                    if (rd + 1 == rounds) ask_next();
+                    // the one output stage was handed to a tensor store a round ago: by the time this round's planes are read and
+                    // transposed the store has drained it
+                    auto ready = [&]() {
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+                    };
+                    float* stage = sh.out;
+                    if (mode == 1) decode_round<0>(blob, padw, L, pay_off, code, hc.s, stage, lane, nullptr, ready);
+                    else { ready(); decode_round_general(blob, padw, L, &pay_off, &code, hc.s, stage, lane, nullptr, 0u); }
                     __syncwarp();   // the stage's rows, written by all lanes, are visible
                     const uint32_t e0 = rd * (uint32_t)kRound;
                     if (mapped && e0 + (uint32_t)kRound <= len) {
                         if (lane == 0) tensor_store_round(&maps.m[jcur], tile * (uint32_t)kBlocksPerTile + (e0 >> 5), stage);
-                        so ^= 1u;
+                        
                     } else {
                         store_round_ragged(y + e0, stage, len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound, lane);
                     }
                 }
             }
         }
-        if (!asked) ask_next();
         cur = nxt;
+        cb ^= 1u;
         t = tn;
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");

@@ -281,8 +281,8 @@ __device__ __forceinline__ int describe_blob_wide(const uint32_t* blob, uint32_t
     return (ao < (1u << 23) && spread < (1u << 23)) ? 1 : 2;
 }
 
-// A warp decodes a tile of its own, round after round, as decode_tiles_kernel does (blob staged by bulk copies, a
-// window at a time when it is larger than the buffer; one tensor store per full round of an output on a 16-byte
+// A warp decodes a tile of its own, round after round, as decode_tiles_kernel does (blob staged by bulk copies, the
+// next tile's into the other of two buffers, a window at a time when it is larger than a buffer; one tensor store per full round of an output on a 16-byte
 // boundary, plain coalesced stores otherwise).
 __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(const uint32_t* __restrict__ in, unsigned long long in_cap, TiledShape sp,
                                                                               float* __restrict__ y, unsigned long long y_cap, uint32_t tiles,
@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(co
     DecWarpShared& sh = reinterpret_cast<DecWarpShared*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u))[warp];
     uint32_t status = 0;
     if (lane == 0) {
-        mbar_init(&sh.bar, 1);
+        mbar_init(&sh.bar[0], 1); mbar_init(&sh.bar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
@@ -314,10 +314,11 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(co
         if (tid == 0 && blockIdx.x == 0) atomicOr(ws.status, ok ? kStCapacity : kStBadStream);
         return;
     }
-    uint32_t fills = 0;
+    uint32_t fills0 = 0, fills1 = 0;   // bulk copies completed into each blob buffer (phase parities of their mbarriers)
+    uint32_t cb = 0;                   // the buffer with the current tile's blob
     const unsigned long long blob0 = (unsigned long long)kHeaderWords + nT;
     const uint32_t last_tile = nT < tiles ? nT : tiles;
-    auto request = [&](unsigned long long t) {
+    auto request = [&](unsigned long long t, uint32_t buf) {
         BlobRef br;
         br.ptr = nullptr; br.words = 0; br.staged = false;
         if (t >= last_tile) return br;
@@ -329,7 +330,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(co
         br.words = w_end - w_beg;
         const uintptr_t a_end = ((uintptr_t)(br.ptr + br.words) + 15) & ~(uintptr_t)15;
         if (a_end - (uintptr_t)in <= (uintptr_t)in_cap) {
-            if (lane == 0) window_request(br, 0, sh.blob, &sh.bar);
+            if (lane == 0) window_request(br, 0, sh.blob[buf], &sh.bar[buf]);
             br.staged = true;
         }
         return br;
@@ -337,22 +338,17 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(co
 
     const unsigned long long stride = (unsigned long long)gridDim.x * kCodecWarps;
     unsigned long long t = (unsigned long long)blockIdx.x * kCodecWarps + (unsigned long long)warp;
-    uint32_t so = 0;
-    BlobRef cur = request(t);
+    BlobRef cur = request(t, 0);
     while (t < last_tile) {
         const unsigned long long tn = t + stride;
         BlobRef nxt;
         nxt.ptr = nullptr; nxt.words = 0; nxt.staged = false;
-        bool asked = false;
-        auto ask_next = [&]() {
-            __syncwarp();
-            nxt = request(tn);
-            asked = true;
-        };
         if (cur.staged) {
-            if (!mbar_wait(&sh.bar, fills & 1u)) status |= kStTimeout;
-            ++fills;
+            if (!mbar_wait(&sh.bar[cb], (cb ? fills1 : fills0) & 1u)) status |= kStTimeout;
+            if (cb) ++fills1; else ++fills0;
         }
+        __syncwarp();
+        nxt = request(tn, cb ^ 1u);   // the other blob buffer takes the next tile's blob while this tile is decoded
         if (cur.words == 0xFFFFFFFFu) status |= kStBadStream;
         else if (cur.ptr) {
             const unsigned long long start = t * sp.T;
@@ -360,7 +356,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(co
             const uint32_t nb = (len + kBlock - 1) / kBlock, padw = (nb + 3) >> 2;
             BlobWindow win;
             win.base = cur.ptr; win.end = cur.words;
-            if (cur.staged) win = window_at(cur, 0, sh.blob);
+            if (cur.staged) win = window_at(cur, 0, sh.blob[cb]);
             const int mode = describe_blob_wide(win.base, cur.words, nb, lane);   // the head (at most 65 words) is in every first window
             if (mode == 0) status |= kStBadStream;
             else {
@@ -382,17 +378,18 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(co
                     const uint32_t first = 1u + padw + pay_off;
                     if (win.end < cur.words && first + __reduce_add_sync(kFull, L ? L + 1u : 0u) > win.end) {   // the round reaches past the window
                         __syncwarp();
-                        if (lane == 0) window_request(cur, first, sh.blob, &sh.bar);
-                        if (!mbar_wait(&sh.bar, fills & 1u)) status |= kStTimeout;
-                        ++fills;
-                        win = window_at(cur, first, sh.blob);
+                        if (lane == 0) window_request(cur, first, sh.blob[cb], &sh.bar[cb]);
+                        if (!mbar_wait(&sh.bar[cb], (cb ? fills1 : fills0) & 1u)) status |= kStTimeout;
+                        if (cb) ++fills1; else ++fills0;
+                        win = window_at(cur, first, sh.blob[cb]);
                     }
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the stage was handed to a tensor store two rounds ago
-                    __syncwarp();
-                    float* stage = sh.out[so];
-                    if (mode == 1) decode_round<0>(win.base, padw, L, pay_off, code, s, stage, lane);
-                    else decode_round_general(win.base, padw, L, &pay_off, &code, s, stage, lane, nullptr, 0u);
-                    if (rd + 1 == rounds) ask_next();
+                    auto ready = [&]() {   // the one output stage was handed to a tensor store a round ago
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                        __syncwarp();
+                    };
+                    float* stage = sh.out;
+                    if (mode == 1) decode_round<0>(win.base, padw, L, pay_off, code, s, stage, lane, nullptr, ready);
+                    else { ready(); decode_round_general(win.base, padw, L, &pay_off, &code, s, stage, lane, nullptr, 0u); }
                     __syncwarp();
                     const uint32_t e0 = rd * (uint32_t)kRound;
                     if (mapped && e0 + (uint32_t)kRound <= len) {
@@ -402,15 +399,14 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_tiles_tiled_kernel(co
                                          ::"l"(&map), "r"(0), "r"((int)((start + e0) >> 5)), "r"(smem_u32(stage)) : "memory");
                             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         }
-                        so ^= 1u;
                     } else {
                         store_round_ragged(y + start + e0, stage, len - e0 < (uint32_t)kRound ? len - e0 : (uint32_t)kRound, lane);
                     }
                 }
             }
         }
-        if (!asked) ask_next();
         cur = nxt;
+        cb ^= 1u;
         t = tn;
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
